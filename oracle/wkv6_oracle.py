@@ -1,0 +1,136 @@
+"""ctypes front end of the fp64 CPU oracle (``wkv6_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the test-suite, the smoke check and the CPU-baseline leg
+of the benchmark may import this module; the CUDA library and its Python binding
+never do, and this module imports nothing from them.
+
+All functions take numpy arrays or torch CPU tensors.  r, k, v, x may be float32 or
+bfloat16 (torch); they are widened exactly to float32 for transport and to float64
+inside the C code, so the oracle sees precisely the values the GPU sees.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "wkv6_oracle.c")
+_LIB = os.path.join(_HERE, "libwkv6_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle next to its source (gcc, OpenMP) and return the path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.wkv6_oracle_threads.restype = ctypes.c_int
+        _lib.wkv6_oracle_prefill.restype = None
+        _lib.wkv6_oracle_prefill_varlen.restype = None
+    return _lib
+
+
+def threads() -> int:
+    """Number of host threads the oracle's OpenMP loops use."""
+    return int(_load().wkv6_oracle_threads())
+
+
+def _f32(a):
+    """Exact float32 numpy copy of a numpy array / torch tensor (bf16 widens exactly)."""
+    if a is None:
+        return None
+    if hasattr(a, "detach"):  # torch tensor
+        a = a.detach().cpu().float().numpy()
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.float64:
+        b = a.astype(np.float32)
+        if not np.array_equal(b.astype(np.float64), a, equal_nan=True):
+            raise ValueError("float64 input is not exactly representable in float32")
+        a = b
+    if a.dtype != np.float32:
+        raise TypeError(f"unsupported dtype {a.dtype}")
+    return a
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def prefill(r, k, v, x, u, state_in=None, w=None):
+    """Dense WKV-6 prefill.  r,k,v,x: [B,T,H,N]; u: [H,N]; state_in: [B,H,N,N] or None.
+
+    ``w`` (float64 [B,T,H,N]), if given, is used as the decay directly and ``x`` is
+    ignored (x may then be None): this states the w == 1 / w == 0 invariants exactly.
+    Returns (y float64 [B,T,H,N], state_out float64 [B,H,N,N]).
+    """
+    lib = _load()
+    r, k, v, u = _f32(r), _f32(k), _f32(v), _f32(u)
+    x = _f32(x)
+    state_in = _f32(state_in)
+    B, T, H, N = r.shape
+    assert k.shape == r.shape and v.shape == r.shape and u.shape == (H, N)
+    if w is not None:
+        w = np.ascontiguousarray(np.asarray(w, dtype=np.float64))
+        assert w.shape == r.shape
+    else:
+        assert x is not None and x.shape == r.shape
+    if state_in is not None:
+        assert state_in.shape == (B, H, N, N)
+    y = np.zeros((B, T, H, N), dtype=np.float64)
+    s_out = np.zeros((B, H, N, N), dtype=np.float64)
+    f, d = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_prefill(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(w, d), _p(u, f),
+                            _p(state_in, f), _p(s_out, d), _p(y, d),
+                            ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(H), ctypes.c_long(N))
+    return y, s_out
+
+
+def prefill_varlen(r, k, v, x, u, cu_seqlens, state_in=None):
+    """Packed variable-length prefill.  r,k,v,x: [total_T,H,N]; cu_seqlens: int32 [S+1];
+    state_in: [S,H,N,N] or None.  Returns (y [total_T,H,N], state_out [S,H,N,N]) in float64."""
+    lib = _load()
+    r, k, v, x, u = _f32(r), _f32(k), _f32(v), _f32(x), _f32(u)
+    state_in = _f32(state_in)
+    if hasattr(cu_seqlens, "detach"):
+        cu_seqlens = cu_seqlens.detach().cpu().numpy()
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    total_T, H, N = r.shape
+    S = cu.shape[0] - 1
+    assert cu[0] == 0 and cu[-1] == total_T and np.all(np.diff(cu) >= 0)
+    if state_in is not None:
+        assert state_in.shape == (S, H, N, N)
+    y = np.zeros((total_T, H, N), dtype=np.float64)
+    s_out = np.zeros((S, H, N, N), dtype=np.float64)
+    f, d = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_prefill_varlen(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(u, f),
+                                   _p(state_in, f), _p(s_out, d), _p(y, d),
+                                   cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                   ctypes.c_long(S), ctypes.c_long(H), ctypes.c_long(N))
+    return y, s_out
+
+
+def step(r, k, v, x, u, state_in):
+    """Single-token decode step: r,k,v,x [B,H,N]; state_in [B,H,N,N].  Defined as a
+    prefill of length one (new-token generation runs the same recurrence)."""
+    r, k, v, x = (_f32(a)[:, None] for a in (r, k, v, x))
+    y, s = prefill(r, k, v, x, u, state_in)
+    return y[:, 0], s
+
+
+def rel_l2(a, b) -> float:
+    """||a - b||_2 / ||b||_2 in float64 (b is the reference)."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    den = float(np.linalg.norm(b))
+    num = float(np.linalg.norm(a - b))
+    return num / den if den > 0 else num
