@@ -1,0 +1,289 @@
+#!/usr/bin/env python
+"""Benchmark of the WKV-6 prefill hot path on the 1.5B-class shape.
+
+One step = one pass of the hot path over one batch: 16 sequential gf_wkv6_prefill calls
+(B=4, T=16384, H=32, N=64, bf16 r/k/v/x/y, fp32 u/state, independent seeds), modelling the
+Finch-C2 two thirds of a 24-layer stack.  Metric: tokens*heads per second (B*T*H*16 / step time).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched by torch.distributed.run, one rank per GPU; the (batch, head) units are
+independent, so every rank runs its own 16 calls (weak scaling) and there is no data-path
+collective: only the timing barrier and a max-reduce of the elapsed time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "WKV-6 prefill tokens*heads/s at 1.5B-class shape"
+UNIT = "token*heads/s"
+WORKLOAD = dict(B=4, T=16384, H=32, N=64, calls=16)
+BYTES_PER_TOKEN_HEAD = 640            # bf16 r,k,v,x in (4*64*2) + bf16 y out (64*2)
+STATE_BYTES_PER_UNIT = 64 * 64 * 4    # fp32 final state written once per (b,h) (state_in is NULL)
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--calls", type=int, default=WORKLOAD["calls"], help=argparse.SUPPRESS)
+    ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help=argparse.SUPPRESS)
+    ap.add_argument("--no-e2e", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--no-cpu-baseline", action="store_true", help=argparse.SUPPRESS)
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        # the first samples may predate the load: the median over the region is what is reported
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_oracle_rate(calls_equiv: float, B, T, H, N, seed):
+    """Times the fp64 oracle, as it stands, on `calls_equiv` calls' worth of the workload
+    (whole (b,h) units of full length T).  Returns (token*heads/s, threads, description)."""
+    from oracle import wkv6_oracle as orc
+    from paper_2407_12077_b200 import synth
+    n_units = max(1, int(round(calls_equiv * B * H)))
+    Hs = min(H, n_units)
+    Bs = max(1, n_units // Hs)
+    inp = synth.make_dense(Bs, T, Hs, N, "bf16", seed=seed)
+    r, k, v, x = (t.float().numpy() for t in (inp.r, inp.k, inp.v, inp.x))
+    u = inp.u.numpy()
+    t0 = time.perf_counter()
+    orc.prefill(r, k, v, x, u, None)
+    dt = time.perf_counter() - t0
+    return Bs * T * Hs / dt, orc.threads(), f"{Bs * Hs} whole (b,h) units of T={T} ({Bs * Hs / (B * H):.3g} of one call)", dt
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on host cores, a bounded sample of the workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    B, T, H, N = WORKLOAD["B"], args.seq_len, WORKLOAD["H"], WORKLOAD["N"]
+    rates, th, desc = [], 1, ""
+    for i in range(args.warmup + args.steps):
+        rate, th, desc, dt = cpu_oracle_rate(0.5, B, T, H, N, seed=2000 + i)
+        if i >= args.warmup:
+            rates.append((rate, dt))
+    value = sum(r for r, _ in rates) / len(rates)
+    units_per_step = B * T * H * args.calls
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": units_per_step / value * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"cfg2: {args.calls} x gf_wkv6_prefill B={B} T={T} H={H} N={N} bf16 inputs",
+                   "note": "CPU oracle on a bounded sample per step; ms_per_step extrapolated to the full step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": th, "kind": "oracle", "sample": desc + " per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2407_12077_b200 as gf
+    from paper_2407_12077_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    gf.load_library()
+
+    B, T, H, N, calls = WORKLOAD["B"], args.seq_len, WORKLOAD["H"], WORKLOAD["N"], args.calls
+    # ---- seeded synthetic inputs, resident in HBM, distinct buffers per call (1.34 GB each >> L2)
+    batches = []
+    for c in range(calls):
+        inp = synth.make_dense(B, T, H, N, "bf16", seed=2000 + 100 * rank + c, device=dev)
+        y = torch.empty_like(inp.r)
+        s_out = torch.empty((B, H, N, N), device=dev, dtype=torch.float32)
+        batches.append((inp, y, s_out))
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        for c, (inp, y, s_out) in enumerate(batches):
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, None, state_out=s_out, y=y, stream=stream)
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    gf.last_device_status()
+
+    # ---- timed region: exactly K steps between barriers, device time, max over ranks
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = gf.launch_count()
+    kernel_events = []
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        step(kernel_events)
+    t_end.record(stream)
+    barrier()
+    elapsed_ms = t_begin.elapsed_time(t_end)
+    launches = gf.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    gf.last_device_status()
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    units_per_step = B * T * H * calls * world
+    value = units_per_step / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel (one prefill launch) from the live per-launch events
+    launch_ms = statistics.mean(a.elapsed_time(b) for a, b in kernel_events)
+    alg_bytes = B * T * H * BYTES_PER_TOKEN_HEAD + B * H * STATE_BYTES_PER_UNIT
+    peak, peak_kind = measured_peaks()
+    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
+                "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms, "algorithmic_bytes": alg_bytes}
+
+    # ---- end to end through the host-buffer entry point: pinned host inputs -> y on the host
+    e2e = None
+    if not args.no_e2e:
+        inp0 = batches[0][0]
+        host = [t.cpu().pin_memory() for t in (inp0.r, inp0.k, inp0.v, inp0.x, inp0.u)]
+        y_h = torch.empty(inp0.r.shape, dtype=torch.bfloat16).pin_memory()
+        s_h = torch.empty((B, H, N, N), dtype=torch.float32).pin_memory()
+        ws = torch.empty(gf.host_workspace_bytes(B, T, H, N), dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            for _ in range(calls):
+                gf.prefill_host(host[0], host[1], host[2], host[3], host[4], None, s_h, y_h, ws, stream=stream)
+
+        e2e_steps = max(1, min(args.steps, 2))
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        tok = B * T * H * N * 2
+        e2e = {"value": units_per_step / (e_ms / e2e_steps * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": calls * (4 * tok + H * N * 4),
+               "d2h_bytes_per_step": calls * (tok + B * H * N * N * 4), "steps": e2e_steps}
+        del ws
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rate, th, desc, dt = cpu_oracle_rate(2.0, B, T, H, N, seed=2000)
+        cpu_baseline = {"value": rate, "unit": UNIT, "cores": th, "kind": "oracle",
+                        "sample": f"{desc}, {dt:.1f} s of CPU time"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 state and accumulation",
+            "data": "synthetic",
+            "config": {"workload": f"cfg2: {calls} x gf_wkv6_prefill B={B} T={T} H={H} N={N}, bf16 r/k/v/x/y, "
+                                   f"fp32 u/state, independent seeds per call",
+                       "l2": "inputs larger than L2 (1.34 GB per call, distinct buffers per call)",
+                       "parallelism": f"(b,h) units replicated per GPU x{world}, no collective"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,144 @@
+/*
+ * gf_wkv6 -- WKV-6 (Finch / RWKV-6) time-mix recurrence for GoldFinch-style linear
+ * pre-fill on NVIDIA B200 (sm_100a).  Plain C ABI: pointers and sizes only.
+ *
+ * What is computed (per sequence b and head h independently; the Finch-C2 time-mixing
+ * formulae are stated per head).  With N the head size, S an N x N fp32 state whose
+ * row index i is the key channel and column index j the value channel:
+ *
+ *     w_t       = exp(-exp(x_t))                                (Finch-C2 decay equation)
+ *     y_t[j]    = sum_i r_t[i] * ( S_{t-1}[i][j] + u[i] * k_t[i] * v_t[j] )
+ *     S_t[i][j] = w_t[i] * S_{t-1}[i][j] + k_t[i] * v_t[j]
+ *
+ * S_{t-1} is the paper's wkv_t = sum_{i<t} diag(prod_{j=i+1..t-1} w_j) k_i^T v_i and
+ * r_t . wkv_t its per-head output before LayerNorm (Finch-C2 wkv_t / o_t equations);
+ * the diag(u) term is classic Finch's "bonus" (pass u = 0 for the Finch-C2 form).
+ * x is the decay *logit* d_t, not w and not log w.  k arrives final (any k*(1-w)
+ * factor is the caller's).  The output uses the state before the update.
+ *
+ * Conventions common to every compute call
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, unless the
+ *     function name ends in _host.  The library never allocates, frees or keeps
+ *     user memory; compute calls only enqueue work on `stream` and return without
+ *     synchronising the host.
+ *   - Layout: r,k,v,x,y are [B][T][H][N] contiguous with N fastest (packed calls:
+ *     [total_T][H][N]); u is [H][N] fp32; states are [B][H][N][N] fp32 row-major
+ *     ([i][j], i = key channel).  Base pointers must be 16-byte aligned.
+ *   - dtype of r,k,v,x,y: bf16 for the un-suffixed names, fp32 for the _f32 twins.
+ *     u and the states are always fp32.  All accumulation is fp32.
+ *   - state_in == NULL means a zero initial state.  state_out == NULL skips the
+ *     final-state write.  state_out may alias state_in (in-place update).  y must
+ *     not overlap any input.
+ *   - N must be 64 (GF_ERR_UNSUPPORTED otherwise).  B, T, S or a sequence length of
+ *     zero is legal: no y rows are written for it and its state passes through.
+ *   - x may be any finite value or -inf (w = 1); +inf gives w = 0.  NaN inputs give
+ *     NaN outputs.
+ *   - Errors: argument errors are detected on the host before anything is enqueued
+ *     and returned at once; a failed launch returns GF_ERR_CUDA.  No exception
+ *     crosses this boundary.  Results are run-to-run deterministic.
+ */
+#ifndef GF_WKV6_H
+#define GF_WKV6_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define GF_API __attribute__((visibility("default")))
+#else
+#define GF_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GF_OK = 0,
+    GF_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, negative size, bad cu_seqlens bound */
+    GF_ERR_UNSUPPORTED = 2, /* head size other than 64, unknown kernel selector */
+    GF_ERR_CUDA = 3,        /* a CUDA runtime / driver call failed */
+    GF_ERR_WORKSPACE = 4,   /* caller-supplied workspace too small */
+    GF_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (see gf_wkv6_last_device_status) */
+} gf_status_t;
+
+/* A CUDA stream handle (cudaStream_t); NULL is the legacy default stream. */
+typedef struct CUstream_st *gf_stream_t;
+
+/* Kernel selector for the bf16 prefill entry points. */
+typedef enum {
+    GF_KERNEL_AUTO = 0,    /* chunked tensor-core kernel, exact kernel where it does not apply */
+    GF_KERNEL_EXACT = 1,   /* token-by-token fp32 recurrence on the ALUs */
+    GF_KERNEL_CHUNKED = 2  /* chunked tensor-core formulation */
+} gf_kernel_t;
+
+/* Dense prefill, bf16 r,k,v,x,y.  Runs the recurrence above over t = 1..T for every
+ * (b,h) (the linear-time pre-fill of the Finch-C2 layers: wkv_t / o_t equations) and
+ * writes y [B][T][H][N] and, if state_out != NULL, S_T [B][H][N][N]. */
+GF_API gf_status_t gf_wkv6_prefill(const void *r, const void *k, const void *v, const void *x,
+                            const float *u, const float *state_in, float *state_out, void *y,
+                            int B, int T, int H, int N, gf_stream_t stream);
+
+/* Same with fp32 r,k,v,x,y (token-by-token fp32 recurrence). */
+GF_API gf_status_t gf_wkv6_prefill_f32(const float *r, const float *k, const float *v, const float *x,
+                                const float *u, const float *state_in, float *state_out, float *y,
+                                int B, int T, int H, int N, gf_stream_t stream);
+
+/* Packed variable-length prefill (batched serving).  Sequence s occupies rows
+ * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
+ * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a
+ * DEVICE int32 array of S+1 non-decreasing entries with cu_seqlens[0] = 0 and
+ * cu_seqlens[S] = total_T (the caller guarantees this; it is not read on the host).
+ * max_seqlen is an upper bound on any sequence length.  States are [S][H][N][N]. */
+GF_API gf_status_t gf_wkv6_prefill_varlen(const void *r, const void *k, const void *v, const void *x,
+                                   const float *u, const float *state_in, float *state_out,
+                                   void *y, const int32_t *cu_seqlens, int S, int total_T,
+                                   int max_seqlen, int H, int N, gf_stream_t stream);
+
+GF_API gf_status_t gf_wkv6_prefill_varlen_f32(const float *r, const float *k, const float *v,
+                                       const float *x, const float *u, const float *state_in,
+                                       float *state_out, float *y, const int32_t *cu_seqlens,
+                                       int S, int total_T, int max_seqlen, int H, int N,
+                                       gf_stream_t stream);
+
+/* Single-token decode step (new-token generation with the state pre-fill left behind):
+ * identical to a prefill with T = 1.  r,k,v,x,y are [B][H][N]; states [B][H][N][N]. */
+GF_API gf_status_t gf_wkv6_step(const void *r, const void *k, const void *v, const void *x,
+                         const float *u, const float *state_in, float *state_out, void *y,
+                         int B, int H, int N, gf_stream_t stream);
+
+GF_API gf_status_t gf_wkv6_step_f32(const float *r, const float *k, const float *v, const float *x,
+                             const float *u, const float *state_in, float *state_out, float *y,
+                             int B, int H, int N, gf_stream_t stream);
+
+/* End-to-end dense prefill from HOST buffers (bf16 r,k,v,x,y; fp32 u and states, all in
+ * host memory, pinned for full copy speed).  Copies the inputs to `dev_ws`, runs
+ * gf_wkv6_prefill there and copies y and state_out back, all on `stream`; returns
+ * without synchronising, so the caller synchronises `stream` before reading y.
+ * dev_ws is a caller-owned DEVICE buffer of at least gf_wkv6_host_workspace_bytes()
+ * bytes, 256-byte aligned (GF_ERR_WORKSPACE if dev_ws_bytes is too small). */
+GF_API gf_status_t gf_wkv6_prefill_host(const void *r, const void *k, const void *v, const void *x,
+                                 const float *u, const float *state_in, float *state_out, void *y,
+                                 int B, int T, int H, int N, void *dev_ws, size_t dev_ws_bytes,
+                                 gf_stream_t stream);
+GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
+
+/* Forces the kernel used by the bf16 prefill calls of this process (default
+ * GF_KERNEL_AUTO).  Process-wide, not thread-safe against concurrent compute calls. */
+GF_API gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel);
+
+/* Synchronises `stream`, then returns GF_ERR_TIMEOUT if any kernel launched by this
+ * library since the last query gave up on a bounded wait (its outputs are then
+ * undefined), GF_ERR_CUDA if the stream reports an error, else GF_OK.  Clears the flag. */
+GF_API gf_status_t gf_wkv6_last_device_status(gf_stream_t stream);
+
+/* Number of kernels this library has launched in this process (for benchmarks). */
+GF_API uint64_t gf_wkv6_launch_count(void);
+
+GF_API const char *gf_status_string(gf_status_t status);
+GF_API int gf_wkv6_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GF_WKV6_H */

@@ -1,0 +1,217 @@
+"""Python binding of the gf_wkv6 C-ABI CUDA library (argument marshalling only).
+
+Every function mirrors the entry point of the same name in ``include/gf_wkv6.h``:
+torch tensors supply device memory and the current CUDA stream, all arithmetic runs
+in the library's kernels.  There is no CPU or PyTorch fallback: if the shared library
+is missing or a tensor is not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import _build
+
+__all__ = [
+    "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
+    "prefill_host", "host_workspace_bytes", "set_kernel", "last_device_status",
+    "launch_count", "status_string", "version",
+    "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
+]
+
+KERNEL_AUTO, KERNEL_EXACT, KERNEL_CHUNKED = 0, 1, 2
+GF_OK = 0
+
+_lib = None
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+
+# name -> (restype, argtypes); the single place the ABI is mirrored in Python
+_SIGNATURES = {
+    "gf_wkv6_prefill": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
+    "gf_wkv6_prefill_f32": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
+    "gf_wkv6_prefill_varlen": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
+    "gf_wkv6_prefill_varlen_f32": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
+    "gf_wkv6_step": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
+    "gf_wkv6_step_f32": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
+    "gf_wkv6_prefill_host": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_host_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_set_kernel": (_i, [_i]),
+    "gf_wkv6_last_device_status": (_i, [_vp]),
+    "gf_wkv6_launch_count": (ctypes.c_uint64, []),
+    "gf_status_string": (ctypes.c_char_p, [_i]),
+    "gf_wkv6_version": (_i, []),
+}
+
+
+class GfError(RuntimeError):
+    """A gf_wkv6 call returned a status other than GF_OK."""
+
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {status_string(status)} (gf_status_t {int(status)})")
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def load_library(build_if_missing: bool = True):
+    """dlopen libgfwkv6.so (building it with nvcc first if it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if build_if_missing and _build.is_stale():
+        _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2407_12077_b200._build`; "
+                           "there is no fallback path")
+    lib = ctypes.CDLL(path)
+    for name, (res, args) in _SIGNATURES.items():
+        fn = getattr(lib, name)            # AttributeError here = header / library mismatch
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().gf_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(load_library().gf_wkv6_version())
+
+
+def launch_count() -> int:
+    return int(load_library().gf_wkv6_launch_count())
+
+
+def set_kernel(kernel: int) -> None:
+    _check(load_library().gf_wkv6_set_kernel(int(kernel)), "gf_wkv6_set_kernel")
+
+
+def _check(status: int, where: str) -> None:
+    if status != GF_OK:
+        raise GfError(status, where)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev(t: torch.Tensor | None, name: str, dtype=None, shape=None):
+    """Device pointer of a contiguous CUDA tensor (None -> NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (no CPU fallback exists)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    return t.data_ptr()
+
+
+def _suffix(dtype) -> str:
+    if dtype == torch.bfloat16:
+        return ""
+    if dtype == torch.float32:
+        return "_f32"
+    raise TypeError(f"r,k,v,x must be bfloat16 or float32, got {dtype}")
+
+
+def last_device_status(stream=None) -> None:
+    """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
+    _check(load_library().gf_wkv6_last_device_status(_stream(stream)), "gf_wkv6_last_device_status")
+
+
+def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, want_state=True):
+    """gf_wkv6_prefill / gf_wkv6_prefill_f32.  r,k,v,x: [B,T,H,N] CUDA tensors (bf16 or fp32);
+    u: [H,N] fp32; state_in: [B,H,N,N] fp32 or None (zero).  Returns (y, state_out);
+    both are allocated here unless passed in (state_out may be state_in)."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    sfx = _suffix(r.dtype)
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None and want_state:
+        state_out = torch.empty((B, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r", shape=(B, T, H, N)), _dev(k, "k", r.dtype, r.shape), _dev(v, "v", r.dtype, r.shape),
+            _dev(x, "x", r.dtype, r.shape), _dev(u, "u", torch.float32, (H, N)),
+            _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", r.dtype, r.shape)]
+    with torch.cuda.device(r.device):
+        _check(getattr(lib, "gf_wkv6_prefill" + sfx)(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill" + sfx)
+    return y, state_out
+
+
+def prefill_varlen(r, k, v, x, u, cu_seqlens, max_seqlen, state_in=None, state_out=None, y=None,
+                   stream=None, want_state=True):
+    """gf_wkv6_prefill_varlen(_f32).  r,k,v,x: [total_T,H,N]; cu_seqlens: int32 CUDA [S+1];
+    states [S,H,N,N].  Returns (y, state_out)."""
+    lib = load_library()
+    total_T, H, N = r.shape
+    S = cu_seqlens.numel() - 1
+    sfx = _suffix(r.dtype)
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None and want_state:
+        state_out = torch.empty((S, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r"), _dev(k, "k", r.dtype, r.shape), _dev(v, "v", r.dtype, r.shape),
+            _dev(x, "x", r.dtype, r.shape), _dev(u, "u", torch.float32, (H, N)),
+            _dev(state_in, "state_in", torch.float32, (S, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (S, H, N, N)), _dev(y, "y", r.dtype, r.shape),
+            _dev(cu_seqlens, "cu_seqlens", torch.int32)]
+    with torch.cuda.device(r.device):
+        _check(getattr(lib, "gf_wkv6_prefill_varlen" + sfx)(*args, S, total_T, int(max_seqlen), H, N, _stream(stream)),
+               "gf_wkv6_prefill_varlen" + sfx)
+    return y, state_out
+
+
+def step(r, k, v, x, u, state_in, state_out=None, y=None, stream=None):
+    """gf_wkv6_step(_f32): one decode token per sequence.  r,k,v,x: [B,H,N]; state [B,H,N,N].
+    state_out defaults to state_in (in-place update).  Returns (y, state_out)."""
+    lib = load_library()
+    B, H, N = r.shape
+    sfx = _suffix(r.dtype)
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None:
+        state_out = state_in if state_in is not None else torch.empty((B, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r"), _dev(k, "k", r.dtype, r.shape), _dev(v, "v", r.dtype, r.shape),
+            _dev(x, "x", r.dtype, r.shape), _dev(u, "u", torch.float32, (H, N)),
+            _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", r.dtype, r.shape)]
+    with torch.cuda.device(r.device):
+        _check(getattr(lib, "gf_wkv6_step" + sfx)(*args, B, H, N, _stream(stream)), "gf_wkv6_step" + sfx)
+    return y, state_out
+
+
+def host_workspace_bytes(B, T, H, N) -> int:
+    return int(load_library().gf_wkv6_host_workspace_bytes(B, T, H, N))
+
+
+def _host(t: torch.Tensor | None, name: str):
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    return t.data_ptr()
+
+
+def prefill_host(r, k, v, x, u, state_in, state_out, y, dev_ws, stream=None):
+    """gf_wkv6_prefill_host: bf16 host tensors in (pinned for speed), y / state_out host tensors
+    out, staged through the caller's CUDA byte buffer ``dev_ws``.  Asynchronous on the stream."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    args = [_host(r, "r"), _host(k, "k"), _host(v, "v"), _host(x, "x"), _host(u, "u"),
+            _host(state_in, "state_in"), _host(state_out, "state_out"), _host(y, "y")]
+    with torch.cuda.device(dev_ws.device):
+        _check(lib.gf_wkv6_prefill_host(*args, B, T, H, N, _dev(dev_ws, "dev_ws"), dev_ws.numel() * dev_ws.element_size(),
+                                        _stream(stream)), "gf_wkv6_prefill_host")

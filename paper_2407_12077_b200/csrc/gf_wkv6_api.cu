@@ -1,0 +1,254 @@
+// C ABI of the gf_wkv6 library: argument validation, kernel selection and launches.
+// Every entry point is declared and documented in include/gf_wkv6.h.
+#include "gf_wkv6.h"
+
+#include <atomic>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "wkv6_chunked.cuh"
+#include "wkv6_exact.cuh"
+#include "wkv6_step.cuh"
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_kernel{GF_KERNEL_AUTO};
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Pointer checks shared by all compute calls; `need_state_in` is false where NULL means zero.
+gf_status_t check_ptrs(const void* r, const void* k, const void* v, const void* x, const float* u,
+                       const float* state_in, const float* state_out, const void* y)
+{
+    if (!r || !k || !v || !x || !u || !y) return GF_ERR_INVALID_ARG;
+    if (misaligned(r) || misaligned(k) || misaligned(v) || misaligned(x) || misaligned(u) ||
+        misaligned(y) || misaligned(state_in) || misaligned(state_out))
+        return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x) return GF_ERR_INVALID_ARG;
+    return GF_OK;
+}
+
+inline gf_status_t launch_result()
+{
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+// state_out <- state_in (or zero) for calls that have no tokens to process.
+gf_status_t pass_state(const float* state_in, float* state_out, size_t n_units, cudaStream_t st)
+{
+    if (!state_out || n_units == 0) return GF_OK;
+    const size_t bytes = n_units * 64 * 64 * sizeof(float);
+    cudaError_t e = cudaSuccess;
+    if (!state_in) e = cudaMemsetAsync(state_out, 0, bytes, st);
+    else if (state_in != state_out) e = cudaMemcpyAsync(state_out, state_in, bytes, cudaMemcpyDeviceToDevice, st);
+    return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+template <typename IO>
+gf_status_t run_exact(const IO* r, const IO* k, const IO* v, const IO* x, const float* u,
+                      const float* state_in, float* state_out, IO* y, const int32_t* cu,
+                      int n_seq, int T, int H, cudaStream_t st)
+{
+    const long long units = (long long)n_seq * H;
+    if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    gf::wkv6_exact_kernel<IO><<<(unsigned)units, gf::EX_THREADS, 0, st>>>(r, k, v, x, u, state_in, state_out, y, cu, T, H);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
+template <typename IO>
+gf_status_t prefill_dense(const IO* r, const IO* k, const IO* v, const IO* x, const float* u,
+                          const float* state_in, float* state_out, IO* y, int B, int T, int H, int N,
+                          cudaStream_t st, bool allow_chunked)
+{
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if ((long long)B * T >= (1LL << 31)) return GF_ERR_INVALID_ARG;
+    if (B == 0 || H == 0) return GF_OK;
+    if (T == 0) return pass_state(state_in, state_out, (size_t)B * H, st);
+    gf_status_t s = check_ptrs(r, k, v, x, u, state_in, state_out, y);
+    if (s != GF_OK) return s;
+    const int sel = g_kernel.load(std::memory_order_relaxed);
+    if (allow_chunked && sel != GF_KERNEL_EXACT) {
+        s = gf::chunked_prefill(reinterpret_cast<const __nv_bfloat16*>(r), reinterpret_cast<const __nv_bfloat16*>(k),
+                                reinterpret_cast<const __nv_bfloat16*>(v), reinterpret_cast<const __nv_bfloat16*>(x),
+                                u, state_in, state_out, reinterpret_cast<__nv_bfloat16*>(y), nullptr,
+                                B, T, (long long)B * T, H, st, &g_launches);
+        if (s != GF_ERR_UNSUPPORTED || sel == GF_KERNEL_CHUNKED) return s;
+    }
+    return run_exact<IO>(r, k, v, x, u, state_in, state_out, y, nullptr, B, T, H, st);
+}
+
+template <typename IO>
+gf_status_t prefill_varlen(const IO* r, const IO* k, const IO* v, const IO* x, const float* u,
+                           const float* state_in, float* state_out, IO* y, const int32_t* cu, int S,
+                           int total_T, int max_seqlen, int H, int N, cudaStream_t st, bool allow_chunked)
+{
+    if (S < 0 || total_T < 0 || max_seqlen < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (max_seqlen > total_T) max_seqlen = total_T;
+    if (S == 0 || H == 0) return GF_OK;
+    if (!cu || (reinterpret_cast<uintptr_t>(cu) & 3u)) return GF_ERR_INVALID_ARG;
+    if (total_T == 0) return pass_state(state_in, state_out, (size_t)S * H, st);
+    gf_status_t s = check_ptrs(r, k, v, x, u, state_in, state_out, y);
+    if (s != GF_OK) return s;
+    const int sel = g_kernel.load(std::memory_order_relaxed);
+    if (allow_chunked && sel != GF_KERNEL_EXACT) {
+        s = gf::chunked_prefill(reinterpret_cast<const __nv_bfloat16*>(r), reinterpret_cast<const __nv_bfloat16*>(k),
+                                reinterpret_cast<const __nv_bfloat16*>(v), reinterpret_cast<const __nv_bfloat16*>(x),
+                                u, state_in, state_out, reinterpret_cast<__nv_bfloat16*>(y), cu,
+                                S, max_seqlen, (long long)total_T, H, st, &g_launches);
+        if (s != GF_ERR_UNSUPPORTED || sel == GF_KERNEL_CHUNKED) return s;
+    }
+    return run_exact<IO>(r, k, v, x, u, state_in, state_out, y, cu, S, max_seqlen, H, st);
+}
+
+template <typename IO>
+gf_status_t step_impl(const IO* r, const IO* k, const IO* v, const IO* x, const float* u,
+                      const float* state_in, float* state_out, IO* y, int B, int H, int N, cudaStream_t st)
+{
+    if (B < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    gf_status_t s = check_ptrs(r, k, v, x, u, state_in, state_out, y);
+    if (s != GF_OK) return s;
+    const long long units = (long long)B * H;
+    if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    gf::wkv6_step_kernel<IO><<<(unsigned)units, gf::ST_THREADS, 0, st>>>(r, k, v, x, u, state_in, state_out, y, H);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
+}  // namespace
+
+extern "C" {
+
+gf_status_t gf_wkv6_prefill(const void* r, const void* k, const void* v, const void* x, const float* u,
+                            const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                            gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    return prefill_dense<bf>((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
+                             (bf*)y, B, T, H, N, (cudaStream_t)stream, true);
+}
+
+gf_status_t gf_wkv6_prefill_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
+                                const float* state_in, float* state_out, float* y, int B, int T, int H, int N,
+                                gf_stream_t stream)
+{
+    return prefill_dense<float>(r, k, v, x, u, state_in, state_out, y, B, T, H, N, (cudaStream_t)stream, false);
+}
+
+gf_status_t gf_wkv6_prefill_varlen(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                   const float* state_in, float* state_out, void* y, const int32_t* cu_seqlens,
+                                   int S, int total_T, int max_seqlen, int H, int N, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    return prefill_varlen<bf>((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
+                              (bf*)y, cu_seqlens, S, total_T, max_seqlen, H, N, (cudaStream_t)stream, true);
+}
+
+gf_status_t gf_wkv6_prefill_varlen_f32(const float* r, const float* k, const float* v, const float* x,
+                                       const float* u, const float* state_in, float* state_out, float* y,
+                                       const int32_t* cu_seqlens, int S, int total_T, int max_seqlen, int H,
+                                       int N, gf_stream_t stream)
+{
+    return prefill_varlen<float>(r, k, v, x, u, state_in, state_out, y, cu_seqlens, S, total_T, max_seqlen, H, N,
+                                 (cudaStream_t)stream, false);
+}
+
+gf_status_t gf_wkv6_step(const void* r, const void* k, const void* v, const void* x, const float* u,
+                         const float* state_in, float* state_out, void* y, int B, int H, int N, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    return step_impl<bf>((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out, (bf*)y,
+                         B, H, N, (cudaStream_t)stream);
+}
+
+gf_status_t gf_wkv6_step_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
+                             const float* state_in, float* state_out, float* y, int B, int H, int N,
+                             gf_stream_t stream)
+{
+    return step_impl<float>(r, k, v, x, u, state_in, state_out, y, B, H, N, (cudaStream_t)stream);
+}
+
+size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N)
+{
+    if (B < 0 || T < 0 || H < 0 || N < 0) return 0;
+    const size_t tok = (size_t)B * T * H * N * 2;                 // one bf16 tensor
+    const size_t pad = 256;
+    auto up = [&](size_t b) { return (b + pad - 1) / pad * pad; };
+    return 5 * up(tok) + up((size_t)H * N * 4) + 2 * up((size_t)B * H * N * N * 4);
+}
+
+gf_status_t gf_wkv6_prefill_host(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                 const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                                 void* dev_ws, size_t dev_ws_bytes, gf_stream_t stream)
+{
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (!r || !k || !v || !x || !u || !y) return GF_ERR_INVALID_ARG;
+    if (!dev_ws || (reinterpret_cast<uintptr_t>(dev_ws) & 255u)) return GF_ERR_INVALID_ARG;
+    if (dev_ws_bytes < gf_wkv6_host_workspace_bytes(B, T, H, N)) return GF_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t tok = (size_t)B * T * H * N * 2, ub = (size_t)H * N * 4, sb = (size_t)B * H * N * N * 4;
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    char* p = static_cast<char*>(dev_ws);
+    char* d_r = p; p += up(tok);
+    char* d_k = p; p += up(tok);
+    char* d_v = p; p += up(tok);
+    char* d_x = p; p += up(tok);
+    char* d_y = p; p += up(tok);
+    float* d_u = reinterpret_cast<float*>(p); p += up(ub);
+    float* d_si = reinterpret_cast<float*>(p); p += up(sb);
+    float* d_so = reinterpret_cast<float*>(p);
+    bool ok = true;
+    auto h2d = [&](void* d, const void* h, size_t n) {
+        if (n) ok = ok && cudaMemcpyAsync(d, h, n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    h2d(d_r, r, tok); h2d(d_k, k, tok); h2d(d_v, v, tok); h2d(d_x, x, tok); h2d(d_u, u, ub);
+    if (state_in) h2d(d_si, state_in, sb);
+    if (!ok) return GF_ERR_CUDA;
+    gf_status_t s = gf_wkv6_prefill(d_r, d_k, d_v, d_x, d_u, state_in ? d_si : nullptr,
+                                    state_out ? d_so : nullptr, d_y, B, T, H, N, stream);
+    if (s != GF_OK) return s;
+    if (tok) ok = ok && cudaMemcpyAsync(y, d_y, tok, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (state_out && sb) ok = ok && cudaMemcpyAsync(state_out, d_so, sb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    return ok ? GF_OK : GF_ERR_CUDA;
+}
+
+gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel)
+{
+    if (kernel != GF_KERNEL_AUTO && kernel != GF_KERNEL_EXACT && kernel != GF_KERNEL_CHUNKED)
+        return GF_ERR_UNSUPPORTED;
+    g_kernel.store((int)kernel, std::memory_order_relaxed);
+    return GF_OK;
+}
+
+gf_status_t gf_wkv6_last_device_status(gf_stream_t stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return GF_ERR_CUDA;
+    int flag = 0;
+    if (gf::read_and_clear_device_status(&flag) != cudaSuccess) return GF_ERR_CUDA;
+    return flag ? GF_ERR_TIMEOUT : GF_OK;
+}
+
+uint64_t gf_wkv6_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* gf_status_string(gf_status_t s)
+{
+    switch (s) {
+    case GF_OK: return "ok";
+    case GF_ERR_INVALID_ARG: return "invalid argument";
+    case GF_ERR_UNSUPPORTED: return "unsupported configuration";
+    case GF_ERR_CUDA: return "CUDA error";
+    case GF_ERR_WORKSPACE: return "workspace too small";
+    case GF_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int gf_wkv6_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,101 @@
+"""Host-side checks of the C-ABI boundary that need no GPU: the library builds, loads,
+exports every symbol the header declares, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2407_12077_b200 as gf
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "gf_wkv6.h")
+
+
+def declared_symbols():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"GF_API[^;(]*?\b(gf_\w+)\s*\(", src)))
+
+
+def test_header_declares_the_three_named_entry_points():
+    names = declared_symbols()
+    for must in ("gf_wkv6_prefill", "gf_wkv6_prefill_varlen", "gf_wkv6_step"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    gf.load_library()
+    raw = ctypes.CDLL(gf.library_path())
+    names = declared_symbols()
+    assert len(names) >= 13
+    for name in names:
+        assert hasattr(raw, name), f"{name} declared in gf_wkv6.h but not exported"
+    # and the binding mirrors exactly the declared set
+    assert sorted(gf._SIGNATURES) == names
+
+
+def test_version_and_status_strings():
+    assert gf.version() >= 100
+    assert gf.status_string(0) == "ok"
+    seen = {gf.status_string(i) for i in range(6)}
+    assert len(seen) == 6
+
+
+def _call(name, *args):
+    return getattr(gf.load_library(), name)(*args)
+
+
+A = 0x1000  # a fake, 16-byte aligned, never dereferenced "device pointer"
+
+
+def test_rejects_bad_arguments_before_any_launch():
+    ptrs = [A] * 8
+    # head size other than 64
+    assert _call("gf_wkv6_prefill", *ptrs, 1, 8, 1, 32, None) == 2
+    assert _call("gf_wkv6_step", *ptrs, 1, 1, 128, None) == 2
+    assert _call("gf_wkv6_prefill_varlen", *ptrs, A, 1, 8, 8, 1, 48, None) == 2
+    # negative sizes
+    assert _call("gf_wkv6_prefill", *ptrs, -1, 8, 1, 64, None) == 1
+    assert _call("gf_wkv6_prefill_f32", *ptrs, 1, -8, 1, 64, None) == 1
+    assert _call("gf_wkv6_step_f32", *ptrs, 1, -1, 64, None) == 1
+    # NULL required pointer, misaligned pointer, y aliasing an input
+    for bad in (0, 3, 7):
+        p = list(ptrs)
+        p[bad] = None
+        assert _call("gf_wkv6_prefill", *p, 1, 8, 1, 64, None) == 1
+    p = list(ptrs)
+    p[1] = A + 2
+    assert _call("gf_wkv6_prefill", *p, 1, 8, 1, 64, None) == 1
+    p = [A + 0x100 * i for i in range(8)]
+    p[7] = p[2]
+    assert _call("gf_wkv6_prefill", *p, 1, 8, 1, 64, None) == 1
+    # varlen without cu_seqlens
+    assert _call("gf_wkv6_prefill_varlen", *ptrs, None, 2, 8, 8, 1, 64, None) == 1
+    # empty problems are legal no-ops that never reach CUDA
+    assert _call("gf_wkv6_prefill", *ptrs, 0, 8, 1, 64, None) == 0
+    assert _call("gf_wkv6_step", *ptrs, 0, 4, 64, None) == 0
+    assert _call("gf_wkv6_prefill_varlen", *ptrs, A, 0, 0, 0, 4, 64, None) == 0
+
+
+def test_host_entry_point_checks_workspace():
+    need = gf.host_workspace_bytes(2, 128, 4, 64)
+    tok = 2 * 128 * 4 * 64 * 2
+    assert need >= 5 * tok + 4 * 64 * 4 + 2 * 2 * 4 * 64 * 64 * 4
+    ptrs = [A] * 8
+    assert _call("gf_wkv6_prefill_host", *ptrs, 2, 128, 4, 64, 0x10000, need - 1, None) == 4
+    assert _call("gf_wkv6_prefill_host", *ptrs, 2, 128, 4, 64, None, need, None) == 1
+    assert _call("gf_wkv6_prefill_host", *ptrs, 2, 128, 4, 32, 0x10000, need, None) == 2
+
+
+def test_kernel_selector_validation():
+    assert _call("gf_wkv6_set_kernel", 7) == 2
+    assert _call("gf_wkv6_set_kernel", gf.KERNEL_AUTO) == 0
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    t = torch.zeros((1, 4, 1, 64), dtype=torch.bfloat16)
+    u = torch.zeros((1, 64))
+    with pytest.raises(ValueError):
+        gf.prefill(t, t, t, t, u, y=t.clone(), state_out=torch.zeros(1, 1, 64, 64))
