@@ -12,14 +12,16 @@
 // >= 0.69); a chunk that violates it is processed token by token in fp32 instead, so any finite
 // or infinite decay logit gives the exact-recurrence result.
 //
-// Warp roles (544 threads), pipelined across chunks through mbarriers:
-//   warp 0      TMA producer: r,k,x tiles (3-stage ring) and v tiles (5-stage ring), 128B swizzle
-//   warps 1-8   elementwise: decay, cumulative sum, scaled bf16 operands R^ = r 2^{a_{t-1}},
-//               K^ = k 2^{-a_t}, chunk decay 2^{a_L}, bonus coefficients, safety vote
-//   warps 9-12  scores: P = tril(R^ K^T, -1) + diag(bonus) -> bf16 tile
-//   warps 13-16 state/output: hold S^T in mma accumulators for the whole sequence;
-//               Y^T = S^T R^^T + V^T P^T, S^T <- (S^T + V^T K^) diag(2^{a_L}); y staged through
-//               shared memory and written with TMA
+// Warp roles (672 threads), pipelined across chunks through mbarriers:
+//   warp 0       TMA producer: x tiles (4-stage ring) and {r,k,v} tiles (5-stage ring), 128B swizzle
+//   warps 1-8    elementwise: decay, cumulative sum (phase A, one chunk ahead), then in place
+//                R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t} (phase B); chunk decay 2^{a_L}, bonus
+//                coefficients, safety vote
+//   warps 9-12   state chain: S <- diag(2^{a_L}) (S + K^^T V) in mma accumulators for the whole
+//                sequence; publishes a bf16 copy of every chunk-start state
+//   warps 13-20  output, two groups alternating chunks: Y = R^ S_0 + (tril(R^ K^^T,-1) + diag(bonus)) V
+//                with the score block kept in registers between its two contractions; every warp
+//                stores its own 16 rows of y with TMA
 // Every wait is bounded: on expiry the kernel raises a status flag and all roles leave.
 #pragma once
 #include <atomic>
@@ -49,45 +51,48 @@ namespace ck {
 
 constexpr int L = 64;                  // tokens per chunk
 constexpr int TILE = 64 * 64 * 2;      // one bf16 [64 x 64] tile
-constexpr int NSTAGE_A = 3;            // r,k,x ring depth
-constexpr int NSTAGE_V = 5;            // v ring depth
-constexpr int NBUF_RK = 2;             // scaled-operand buffers
-constexpr int NBUF_P = 2;
-constexpr int NBUF_Y = 2;
+constexpr int NX = 4;                  // x ring depth
+constexpr int NS = 5;                  // {r,k,v} ring depth
+constexpr int NSB = 3;                 // bf16 chunk-start state buffers
+constexpr int NTOT = 4;                // per-warp decay-total buffers (phase A runs one chunk ahead)
 constexpr int N_EW = 8;                // elementwise warps
-constexpr int THREADS = 32 * (1 + N_EW + 4 + 4);
+constexpr int N_SW = 4;                // state warps
+constexpr int N_YW = 8;                // output warps (two groups of four)
+constexpr int WARP_S0 = 1 + N_EW;      // first state warp
+constexpr int WARP_Y0 = WARP_S0 + N_SW;
+constexpr int THREADS = 32 * (1 + N_EW + N_SW + N_YW);
 constexpr float A2_MAX = 96.f;         // largest in-chunk |cumulative log2 decay| on the tensor-core path
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LOG2_LOG2E = 0.5287663729448977f;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr int OFF_A = 0;                                   // [NSTAGE_A][3][TILE]  r,k,x
-constexpr int OFF_V = OFF_A + NSTAGE_A * 3 * TILE;         // [NSTAGE_V][TILE]
-constexpr int OFF_RK = OFF_V + NSTAGE_V * TILE;            // [NBUF_RK][2][TILE]   R^, K^
-constexpr int OFF_P = OFF_RK + NBUF_RK * 2 * TILE;         // [NBUF_P][TILE]
-constexpr int OFF_Y = OFF_P + NBUF_P * TILE;               // [NBUF_Y][TILE]
-constexpr int OFF_DL = OFF_Y + NBUF_Y * TILE;              // [NBUF_RK][64] float  2^{a_L}
-constexpr int OFF_DU = OFF_DL + NBUF_RK * 64 * 4;          // [NBUF_RK][64] float  bonus coefficient per token
-constexpr int OFF_TOT = OFF_DU + NBUF_RK * 64 * 4;         // [2][N_EW][64] float  per-warp decay totals
-constexpr int OFF_SAFE = OFF_TOT + 2 * N_EW * 64 * 4;      // [NBUF_RK] int
-constexpr int OFF_ABORT = OFF_SAFE + 16;                   // int
+constexpr int OFF_X = 0;                                   // [NX][TILE]           x
+constexpr int OFF_RKV = OFF_X + NX * TILE;                 // [NS][3][TILE]        r -> R^, k -> K^, v
+constexpr int OFF_SB = OFF_RKV + NS * 3 * TILE;            // [NSB][TILE]          bf16 chunk-start state [c][j]
+constexpr int OFF_Y = OFF_SB + NSB * TILE;                 // [N_YW][16 rows x 128 B] y staging, one slab per warp
+constexpr int OFF_SCR = OFF_Y + N_YW * 2048;               // [64][64] float       state scratch (token-by-token path)
+constexpr int OFF_TOT = OFF_SCR + 64 * 64 * 4;             // [NTOT][N_EW][64] float
+constexpr int OFF_DL = OFF_TOT + NTOT * N_EW * 64 * 4;     // [NS][64] float       2^{a_L}
+constexpr int OFF_DU = OFF_DL + NS * 64 * 4;               // [NS][64] float       bonus coefficient per token
+constexpr int OFF_SAFE = OFF_DU + NS * 64 * 4;             // [NS] int (padded)
+constexpr int OFF_ABORT = OFF_SAFE + 32;                   // int
 constexpr int OFF_BAR = OFF_ABORT + 16;                    // mbarriers (8 bytes each)
 enum {
-    BAR_FULL_A = 0,
-    BAR_EMPTY_A = BAR_FULL_A + NSTAGE_A,
-    BAR_FULL_V = BAR_EMPTY_A + NSTAGE_A,
-    BAR_EMPTY_V = BAR_FULL_V + NSTAGE_V,
-    BAR_RK_READY = BAR_EMPTY_V + NSTAGE_V,
-    BAR_RK_FREE = BAR_RK_READY + NBUF_RK,
-    BAR_P_READY = BAR_RK_FREE + NBUF_RK,
-    BAR_P_FREE = BAR_P_READY + NBUF_P,
-    BAR_ESYNC = BAR_P_FREE + NBUF_P,
-    BAR_YSYNC = BAR_ESYNC + 1,          // two of them
-    BAR_COUNT = BAR_YSYNC + 2
+    BAR_FULL_X = 0,
+    BAR_EMPTY_X = BAR_FULL_X + NX,
+    BAR_FULL_RKV = BAR_EMPTY_X + NX,
+    BAR_EMPTY_RKV = BAR_FULL_RKV + NS,
+    BAR_RK_READY = BAR_EMPTY_RKV + NS,
+    BAR_S_READY = BAR_RK_READY + NS,
+    BAR_S_FREE = BAR_S_READY + NSB,
+    BAR_ESYNC = BAR_S_FREE + NSB,       // two, alternating by chunk parity
+    BAR_SSYNC = BAR_ESYNC + 2,          // state-warp rendezvous (token-by-token path only)
+    BAR_COUNT = BAR_SSYNC + 1
 };
 constexpr int SMEM_BYTES = OFF_BAR + BAR_COUNT * 8;
 constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;              // slack for manual 1024-byte alignment
+static_assert(SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -203,9 +208,18 @@ __device__ __forceinline__ void stsm_x4_t(uint32_t a, uint32_t r0, uint32_t r1, 
 // D(16x8, fp32) += A(16x16, bf16 row) * B(16x8, bf16 col)
 __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    // not volatile: a pure function of its register operands, so the compiler may schedule the
+    // (ordered, volatile) shared-memory loads of later steps ahead of it
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+
+__device__ __forceinline__ void stsm_x4(uint32_t a, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+{
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};"
+                 ::"r"(a), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
 }
 
 struct Params {
@@ -219,11 +233,24 @@ struct Params {
     int H;
 };
 
+// Writes a warp's 16 x 64 fp32 accumulator block (acc[n][0..1] = row g, cols 8n+2q,+1;
+// acc[n][2..3] = row g+8) as bf16 into rows row0 .. row0+15 of a 128B-swizzled [rows][64] tile.
+__device__ __forceinline__ void store_acc_bf16(uint32_t tile, int row0, const float (&acc)[8][4], int lane)
+{
+    const int mi = lane >> 3, rr = lane & 7;
+    const int row = row0 + rr + 8 * (mi & 1);
+#pragma unroll
+    for (int m = 0; m < 4; ++m)
+        stsm_x4(tile + swz(row, (2 * m + (mi >> 1)) << 4),
+                pack_bf16(acc[2 * m][0], acc[2 * m][1]), pack_bf16(acc[2 * m][2], acc[2 * m][3]),
+                pack_bf16(acc[2 * m + 1][0], acc[2 * m + 1][1]), pack_bf16(acc[2 * m + 1][2], acc[2 * m + 1][3]));
+}
+
 // ---------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
-                    const __grid_constant__ CUtensorMap tm_y, const Params p)
+                    const __grid_constant__ CUtensorMap tm_y16, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -249,13 +276,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     const size_t C = (size_t)p.H * 64;
 
     if (tid == 0) {
-        for (int i = 0; i < NSTAGE_A; ++i) { mbar_init(bar(BAR_FULL_A + i), 1); mbar_init(bar(BAR_EMPTY_A + i), N_EW); }
-        for (int i = 0; i < NSTAGE_V; ++i) { mbar_init(bar(BAR_FULL_V + i), 1); mbar_init(bar(BAR_EMPTY_V + i), 4); }
-        for (int i = 0; i < NBUF_RK; ++i) { mbar_init(bar(BAR_RK_READY + i), N_EW); mbar_init(bar(BAR_RK_FREE + i), 8); }
-        for (int i = 0; i < NBUF_P; ++i) { mbar_init(bar(BAR_P_READY + i), 4); mbar_init(bar(BAR_P_FREE + i), 4); }
+        for (int i = 0; i < NX; ++i) { mbar_init(bar(BAR_FULL_X + i), 1); mbar_init(bar(BAR_EMPTY_X + i), N_EW); }
+        for (int i = 0; i < NS; ++i) {
+            mbar_init(bar(BAR_FULL_RKV + i), 1);
+            mbar_init(bar(BAR_EMPTY_RKV + i), N_SW + N_YW / 2);
+            mbar_init(bar(BAR_RK_READY + i), N_EW);
+        }
+        for (int i = 0; i < NSB; ++i) { mbar_init(bar(BAR_S_READY + i), N_SW); mbar_init(bar(BAR_S_FREE + i), N_YW / 2); }
         mbar_init(bar(BAR_ESYNC), N_EW);
-        mbar_init(bar(BAR_YSYNC), 4);
-        mbar_init(bar(BAR_YSYNC + 1), 4);
+        mbar_init(bar(BAR_ESYNC + 1), N_EW);
+        mbar_init(bar(BAR_SSYNC), N_SW);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
@@ -265,81 +295,108 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     if (warp == 0) {
         // ============================== TMA producer ==============================
         if (lane == 0) {
-            int issued = 0;
-            for (int c = 0; c < nchunks; ++c) {
-                const int sa = c % NSTAGE_A, sv = c % NSTAGE_V;
+            int issued_x = 0, issued_s = 0;
+            auto load_x = [&](int c) -> bool {
+                const int sx = c % NX;
+                if (c >= NX && !mbar_wait(bar(BAR_EMPTY_X + sx), ((c / NX) & 1) ^ 1, abort_flag)) return false;
+                mbar_expect_tx(bar(BAR_FULL_X + sx), TILE);
+                tma_load_2d(sbase + OFF_X + sx * TILE, &tm_x, col0, (int)(row0 + (long long)c * L), bar(BAR_FULL_X + sx));
+                issued_x = c + 1;
+                return true;
+            };
+            bool ok = true;
+            for (int c = 0; c < min(NX - 1, nchunks) && ok; ++c) ok = load_x(c);
+            for (int c = 0; c < nchunks && ok; ++c) {
+                if (c + NX - 1 < nchunks && !load_x(c + NX - 1)) break;
+                const int s = c % NS;
+                if (c >= NS && !mbar_wait(bar(BAR_EMPTY_RKV + s), ((c / NS) & 1) ^ 1, abort_flag)) break;
                 const int row = (int)(row0 + (long long)c * L);
-                if (c >= NSTAGE_A && !mbar_wait(bar(BAR_EMPTY_A + sa), ((c / NSTAGE_A) & 1) ^ 1, abort_flag)) break;
-                if (c >= NSTAGE_V && !mbar_wait(bar(BAR_EMPTY_V + sv), ((c / NSTAGE_V) & 1) ^ 1, abort_flag)) break;
-                const uint32_t dstA = sbase + OFF_A + sa * 3 * TILE;
-                mbar_expect_tx(bar(BAR_FULL_A + sa), 3 * TILE);
-                tma_load_2d(dstA, &tm_x, col0, row, bar(BAR_FULL_A + sa));
-                tma_load_2d(dstA + TILE, &tm_r, col0, row, bar(BAR_FULL_A + sa));
-                tma_load_2d(dstA + 2 * TILE, &tm_k, col0, row, bar(BAR_FULL_A + sa));
-                mbar_expect_tx(bar(BAR_FULL_V + sv), TILE);
-                tma_load_2d(sbase + OFF_V + sv * TILE, &tm_v, col0, row, bar(BAR_FULL_V + sv));
-                issued = c + 1;
+                const uint32_t dst = sbase + OFF_RKV + s * 3 * TILE;
+                mbar_expect_tx(bar(BAR_FULL_RKV + s), 3 * TILE);
+                tma_load_2d(dst, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
+                tma_load_2d(dst + TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
+                tma_load_2d(dst + 2 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
+                issued_s = c + 1;
             }
             // do not leave while copies into this CTA's shared memory may still be in flight
-            for (int c = max(0, issued - NSTAGE_A); c < issued; ++c)
-                mbar_wait(bar(BAR_FULL_A + c % NSTAGE_A), (c / NSTAGE_A) & 1, abort_flag, false);
-            for (int c = max(0, issued - NSTAGE_V); c < issued; ++c)
-                mbar_wait(bar(BAR_FULL_V + c % NSTAGE_V), (c / NSTAGE_V) & 1, abort_flag, false);
+            for (int c = max(0, issued_x - NX); c < issued_x; ++c)
+                mbar_wait(bar(BAR_FULL_X + c % NX), (c / NX) & 1, abort_flag, false);
+            for (int c = max(0, issued_s - NS); c < issued_s; ++c)
+                mbar_wait(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
         }
-    } else if (warp <= N_EW) {
+    } else if (warp < WARP_S0) {
         // ============================== elementwise warps ==============================
         const int tq = warp - 1;                 // tokens 8*tq .. 8*tq+7 of the chunk
         const int cb = lane * 4;                 // byte column of this lane's channel pair (2*lane, 2*lane+1)
+        const int etid = tid - 32;               // 0..255
         const float2 u2 = *reinterpret_cast<const float2*>(p.u + h * 64 + 2 * lane);
         float* tot = reinterpret_cast<float*>(smem + OFF_TOT);
-        for (int c = 0; c < nchunks; ++c) {
-            const int sa = c % NSTAGE_A, b = c % NBUF_RK;
+        // phase A of chunk c: log2-decay magnitudes and this warp's local cumulative sums
+        auto phase_a = [&](int c, float (&l0)[8], float (&l1)[8]) -> bool {
+            const int sx = c % NX;
             const int valid = min(L, len - c * L);
-            const uint32_t tx = sbase + OFF_A + sa * 3 * TILE, tr = tx + TILE, tk = tx + 2 * TILE;
-            if (!mbar_wait(bar(BAR_FULL_A + sa), (c / NSTAGE_A) & 1, abort_flag)) break;
-            // ---- phase A: log2-decay magnitudes and the warp-local cumulative sums
-            float l0[8], l1[8];
-            {
-                float a0 = 0.f, a1 = 0.f;
+            const uint32_t tx = sbase + OFF_X + sx * TILE;
+            if (!mbar_wait(bar(BAR_FULL_X + sx), (c / NX) & 1, abort_flag)) return false;
+            float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-                for (int tt = 0; tt < 8; ++tt) {
-                    const int t = 8 * tq + tt;
-                    const uint32_t xw = lds32(tx + swz(t, cb));
-                    float e0 = ex2(fmaf(bf_lo(xw), LOG2E, LOG2_LOG2E));
-                    float e1 = ex2(fmaf(bf_hi(xw), LOG2E, LOG2_LOG2E));
-                    if (t >= valid) { e0 = 0.f; e1 = 0.f; }
-                    a0 -= e0; a1 -= e1;
-                    l0[tt] = a0; l1[tt] = a1;
-                }
+            for (int tt = 0; tt < 8; ++tt) {
+                const int t = 8 * tq + tt;
+                const uint32_t xw = lds32(tx + swz(t, cb));
+                float e0 = ex2(fmaf(bf_lo(xw), LOG2E, LOG2_LOG2E));
+                float e1 = ex2(fmaf(bf_hi(xw), LOG2E, LOG2_LOG2E));
+                if (t >= valid) { e0 = 0.f; e1 = 0.f; }
+                a0 -= e0; a1 -= e1;
+                l0[tt] = a0; l1[tt] = a1;
             }
-            float* totc = tot + (c & 1) * (N_EW * 64);
-            *reinterpret_cast<float2*>(totc + tq * 64 + 2 * lane) = make_float2(l0[7], l1[7]);
+            *reinterpret_cast<float2*>(tot + ((c % NTOT) * N_EW + tq) * 64 + 2 * lane) = make_float2(a0, a1);
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_ESYNC));
-            if (!mbar_wait(bar(BAR_ESYNC), c & 1, abort_flag)) break;
+            if (lane == 0) {
+                mbar_arrive(bar(BAR_EMPTY_X + sx));
+                mbar_arrive(bar(BAR_ESYNC + (c & 1)));
+            }
+            return true;
+        };
+        float l0[8], l1[8];
+        bool live = nchunks > 0 && phase_a(0, l0, l1);
+        for (int c = 0; c < nchunks && live; ++c) {
+            float n0[8], n1[8];
+            if (c + 1 < nchunks && !phase_a(c + 1, n0, n1)) break;
+            const int s = c % NS;
+            const int valid = min(L, len - c * L);
+            if (!mbar_wait(bar(BAR_ESYNC + (c & 1)), (c >> 1) & 1, abort_flag)) break;
             float off0 = 0.f, off1 = 0.f;
+            const float* totc = tot + (c % NTOT) * N_EW * 64;
             for (int q = 0; q < tq; ++q) {
                 const float2 t2 = *reinterpret_cast<const float2*>(totc + q * 64 + 2 * lane);
                 off0 += t2.x; off1 += t2.y;
             }
-            if (c >= NBUF_RK && !mbar_wait(bar(BAR_RK_FREE + b), ((c / NBUF_RK) & 1) ^ 1, abort_flag)) break;
-            // ---- phase B: scaled operands R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t}; bonus partials
-            const uint32_t trh = sbase + OFF_RK + b * 2 * TILE, tkh = trh + TILE;
+            if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) break;
+            // ---- phase B, in place: r -> R^ = r 2^{a_{t-1}}, k -> K^ = k 2^{-a_t}; bonus partials
+            const uint32_t tr = sbase + OFF_RKV + s * 3 * TILE, tk = tr + TILE, tv = tr + 2 * TILE;
             float du[8];
+            uint32_t rw[8], kw[8];
+#pragma unroll
+            for (int tt = 0; tt < 8; ++tt) {                 // all loads first: they are ordered with the stores below
+                rw[tt] = lds32(tr + swz(8 * tq + tt, cb));
+                kw[tt] = lds32(tk + swz(8 * tq + tt, cb));
+            }
 #pragma unroll
             for (int tt = 0; tt < 8; ++tt) {
                 const int t = 8 * tq + tt;
                 const float ap0 = off0 + (tt ? l0[tt - 1] : 0.f), ap1 = off1 + (tt ? l1[tt - 1] : 0.f);
                 const float ac0 = off0 + l0[tt], ac1 = off1 + l1[tt];
-                const uint32_t rw = lds32(tr + swz(t, cb)), kw = lds32(tk + swz(t, cb));
-                const float r0 = bf_lo(rw), r1 = bf_hi(rw), k0 = bf_lo(kw), k1 = bf_hi(kw);
+                const float r0 = bf_lo(rw[tt]), r1 = bf_hi(rw[tt]), k0 = bf_lo(kw[tt]), k1 = bf_hi(kw[tt]);
                 uint32_t rh = pack_bf16(r0 * ex2(ap0), r1 * ex2(ap1));
                 uint32_t kh = pack_bf16(k0 * ex2(-ac0), k1 * ex2(-ac1));
                 float d = fmaf(r0 * k0, u2.x, r1 * k1 * u2.y);
                 if (t >= valid) { rh = 0u; kh = 0u; d = 0.f; }
-                sts32(trh + swz(t, cb), rh);
-                sts32(tkh + swz(t, cb), kh);
+                rw[tt] = rh; kw[tt] = kh;
                 du[tt] = d;
+            }
+#pragma unroll
+            for (int tt = 0; tt < 8; ++tt) {
+                sts32(tr + swz(8 * tq + tt, cb), rw[tt]);
+                sts32(tk + swz(8 * tq + tt, cb), kw[tt]);
             }
             // reduce the 8 bonus partials over the 32 lanes (transposing butterfly): lane 4m ends with token m
             {
@@ -362,276 +419,270 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 2);
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
                 if ((lane & 3) == 0)
-                    reinterpret_cast<float*>(smem + OFF_DU)[b * 64 + 8 * tq + (lane >> 2)] = w1;
+                    reinterpret_cast<float*>(smem + OFF_DU)[s * 64 + 8 * tq + (lane >> 2)] = w1;
             }
             if (tq == N_EW - 1) {
                 const float aL0 = off0 + l0[7], aL1 = off1 + l1[7];
-                *reinterpret_cast<float2*>(reinterpret_cast<float*>(smem + OFF_DL) + b * 64 + 2 * lane) =
+                *reinterpret_cast<float2*>(reinterpret_cast<float*>(smem + OFF_DL) + s * 64 + 2 * lane) =
                     make_float2(ex2(aL0), ex2(aL1));
                 const bool ok = (aL0 >= -A2_MAX) && (aL1 >= -A2_MAX);       // false for NaN as well
                 const bool all_ok = __all_sync(0xffffffffu, ok);
-                if (lane == 0) safe_flag[b] = all_ok ? 1 : 0;
+                if (lane == 0) safe_flag[s] = all_ok ? 1 : 0;
+            }
+            if (valid < L) {
+                // v rows past the end of the sequence hold another sequence's tokens (or fill): zero them
+                for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
+                    sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(BAR_EMPTY_A + sa));
-                mbar_arrive(bar(BAR_RK_READY + b));
-            }
+            if (lane == 0) mbar_arrive(bar(BAR_RK_READY + s));
+#pragma unroll
+            for (int tt = 0; tt < 8; ++tt) { l0[tt] = n0[tt]; l1[tt] = n1[tt]; }
         }
-    } else if (warp <= N_EW + 4) {
-        // ============================== score warps ==============================
-        const int pw = warp - (N_EW + 1);        // rows t = 16*pw .. 16*pw+15
+    } else if (warp < WARP_Y0) {
+        // ============================== state warps ==============================
+        const int sw = warp - WARP_S0;           // key channels c = 16*sw .. 16*sw+15 (state rows)
         const int g = lane >> 2, q = lane & 3;
-        for (int c = 0; c < nchunks; ++c) {
-            const int b = c % NBUF_RK, pb = c % NBUF_P;
-            if (!mbar_wait(bar(BAR_RK_READY + b), (c / NBUF_RK) & 1, abort_flag)) break;
-            if (c >= NBUF_P && !mbar_wait(bar(BAR_P_FREE + pb), ((c / NBUF_P) & 1) ^ 1, abort_flag)) break;
-            if (safe_flag[b]) {
-                const uint32_t trh = sbase + OFF_RK + b * 2 * TILE, tkh = trh + TILE, tp = sbase + OFF_P + pb * TILE;
-                const float* du = reinterpret_cast<const float*>(smem + OFF_DU) + b * 64;
-                uint32_t a[4][4];
-                {
-                    const int row = 16 * pw + (lane & 7) + 8 * ((lane >> 3) & 1);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        ldsm_x4(trh + swz(row, 32 * kk + 16 * (lane >> 4)), a[kk][0], a[kk][1], a[kk][2], a[kk][3]);
-                }
-                for (int ib = 0; ib <= pw; ++ib) {
-                    float acc[2][4] = {};
-                    const int irow = 16 * ib + (lane & 7) + 8 * (lane >> 4);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        uint32_t b0, b1, b2, b3;
-                        ldsm_x4(tkh + swz(irow, 32 * kk + 16 * ((lane >> 3) & 1)), b0, b1, b2, b3);
-                        mma16816(acc[0], a[kk], b0, b1);
-                        mma16816(acc[1], a[kk], b2, b3);
-                    }
-                    if (ib == pw) {
-                        // diagonal 16x16 block: strictly-lower entries stay, the diagonal takes the bonus
-                        // coefficient, the upper triangle is zero
-                        const float d_lo = du[16 * pw + g], d_hi = du[16 * pw + g + 8];
-#pragma unroll
-                        for (int nb = 0; nb < 2; ++nb) {
-#pragma unroll
-                            for (int e = 0; e < 2; ++e) {
-                                const int il = 8 * nb + 2 * q + e;
-                                acc[nb][e] = il < g ? acc[nb][e] : (il == g ? d_lo : 0.f);
-                                acc[nb][2 + e] = il < g + 8 ? acc[nb][2 + e] : (il == g + 8 ? d_hi : 0.f);
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int nb = 0; nb < 2; ++nb) {
-                        const int colb = (16 * ib + 8 * nb + 2 * q) * 2;
-                        sts32(tp + swz(16 * pw + g, colb), pack_bf16(acc[nb][0], acc[nb][1]));
-                        sts32(tp + swz(16 * pw + g + 8, colb), pack_bf16(acc[nb][2], acc[nb][3]));
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(BAR_P_READY + pb));
-                mbar_arrive(bar(BAR_RK_FREE + b));
-            }
-        }
-    } else {
-        // ============================== state / output warps ==============================
-        const int yw = warp - (N_EW + 5);        // value channels j = 16*yw .. 16*yw+15
-        const int ytid = tid - 32 * (N_EW + 5);  // 0..127
-        const int g = lane >> 2, q = lane & 3;
-        const int j0 = 16 * yw + g;
+        const int c_lo = 16 * sw + g;
         const size_t sb = (size_t)unit * 4096;
-        // S^T[j][c] in accumulator layout: st[n][0..1] = (j0, c = 8n+2q, +1), st[n][2..3] = (j0+8, same c)
+        // S[c][j] in accumulator layout: st[n][0..1] = (c_lo, j = 8n+2q, +1), st[n][2..3] = (c_lo+8, same j)
         float st[8][4];
 #pragma unroll
         for (int n = 0; n < 8; ++n) {
-            const int c0 = 8 * n + 2 * q;
             if (p.state_in) {
-                st[n][0] = p.state_in[sb + (size_t)c0 * 64 + j0];
-                st[n][1] = p.state_in[sb + (size_t)(c0 + 1) * 64 + j0];
-                st[n][2] = p.state_in[sb + (size_t)c0 * 64 + j0 + 8];
-                st[n][3] = p.state_in[sb + (size_t)(c0 + 1) * 64 + j0 + 8];
+                const float2 lo = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)c_lo * 64 + 8 * n + 2 * q);
+                const float2 hi = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
+                st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
             } else {
                 st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
             }
         }
-        int ysync_uses[2] = {0, 0};
-        int ybuf_uses = 0;
-        bool live = true;
-        auto ysync = [&](int which) -> bool {
+        int ssync_uses = 0;
+        auto ssync = [&]() -> bool {
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_YSYNC + which));
-            const bool ok = mbar_wait(bar(BAR_YSYNC + which), ysync_uses[which] & 1, abort_flag);
-            ++ysync_uses[which];
+            if (lane == 0) mbar_arrive(bar(BAR_SSYNC));
+            const bool ok = mbar_wait(bar(BAR_SSYNC), ssync_uses & 1, abort_flag);
+            ++ssync_uses;
             return ok;
         };
-        for (int c = 0; c < nchunks && live; ++c) {
-            const int sv = c % NSTAGE_V, b = c % NBUF_RK, pb = c % NBUF_P;
+        if (nchunks > 0) {
+            store_acc_bf16(sbase + OFF_SB, 16 * sw, st, lane);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_S_READY));
+        }
+        for (int c = 0; c < nchunks; ++c) {
+            const int s = c % NS;
             const int valid = min(L, len - c * L);
-            const uint32_t tv = sbase + OFF_V + sv * TILE;
-            const uint32_t trh = sbase + OFF_RK + b * 2 * TILE, tkh = trh + TILE, tp = sbase + OFF_P + pb * TILE;
-            if (!mbar_wait(bar(BAR_FULL_V + sv), (c / NSTAGE_V) & 1, abort_flag)) break;
-            if (!mbar_wait(bar(BAR_RK_READY + b), (c / NBUF_RK) & 1, abort_flag)) break;
-            if (!mbar_wait(bar(BAR_P_READY + pb), (c / NBUF_P) & 1, abort_flag)) break;
-            if (safe_flag[b]) {
-                if (valid < L) {
-                    // rows past the end of the sequence hold another sequence's tokens (or fill): zero them
-                    for (int i = ytid; i < (L - valid) * 8; i += 128)
-                        sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
-                    if (!ysync(0)) break;
-                }
-                float ya[8][4];
-#pragma unroll
-                for (int n = 0; n < 8; ++n) ya[n][0] = ya[n][1] = ya[n][2] = ya[n][3] = 0.f;
-                // ---- Y^T += S^T R^^T   (M = j, N = t, K = c); A straight from the fp32 accumulators
-                {
-                    const int trow = (lane & 7) + 8 * (lane >> 4);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        uint32_t sa[4];
-                        sa[0] = pack_bf16(st[2 * kk][0], st[2 * kk][1]);
-                        sa[1] = pack_bf16(st[2 * kk][2], st[2 * kk][3]);
-                        sa[2] = pack_bf16(st[2 * kk + 1][0], st[2 * kk + 1][1]);
-                        sa[3] = pack_bf16(st[2 * kk + 1][2], st[2 * kk + 1][3]);
-#pragma unroll
-                        for (int np = 0; np < 4; ++np) {
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4(trh + swz(16 * np + trow, 32 * kk + 16 * ((lane >> 3) & 1)), b0, b1, b2, b3);
-                            mma16816(ya[2 * np], sa, b0, b1);
-                            mma16816(ya[2 * np + 1], sa, b2, b3);
-                        }
-                    }
-                }
-                // ---- V^T fragments (M = j, K = i) from the raw v tile [i][j]
-                uint32_t va[4][4];
+            const uint32_t tk = sbase + OFF_RKV + s * 3 * TILE + TILE, tv = tk + TILE;
+            if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_RK_READY + s), (c / NS) & 1, abort_flag)) break;
+            if (safe_flag[s]) {
+                // ---- S += K^^T V   (M = c, N = j, K = i), then scale row c by 2^{a_L[c]}
+                uint32_t ka[4][4];
                 {
                     const int irow = (lane & 7) + 8 * (lane >> 4);
-                    const int jb = (16 * yw + 8 * ((lane >> 3) & 1)) * 2;
+                    const int cbyte = (16 * sw + 8 * ((lane >> 3) & 1)) * 2;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        ldsm_x4_t(tv + swz(16 * kk + irow, jb), va[kk][0], va[kk][1], va[kk][2], va[kk][3]);
+                        ldsm_x4_t(tk + swz(16 * kk + irow, cbyte), ka[kk][0], ka[kk][1], ka[kk][2], ka[kk][3]);
                 }
-                // ---- Y^T += V^T P^T   (M = j, N = t, K = i), causal: token block np needs i-steps kk <= np
-                {
-                    const int trow = (lane & 7) + 8 * (lane >> 4);
+                const int krow = (lane & 7) + 8 * ((lane >> 3) & 1);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
+                for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-                        for (int np = kk; np < 4; ++np) {
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4(tp + swz(16 * np + trow, 32 * kk + 16 * ((lane >> 3) & 1)), b0, b1, b2, b3);
-                            mma16816(ya[2 * np], va[kk], b0, b1);
-                            mma16816(ya[2 * np + 1], va[kk], b2, b3);
-                        }
+                    for (int jp = 0; jp < 4; ++jp) {
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4_t(tv + swz(16 * kk + krow, 32 * jp + 16 * (lane >> 4)), b0, b1, b2, b3);
+                        mma16816(st[2 * jp], ka[kk], b0, b1);
+                        mma16816(st[2 * jp + 1], ka[kk], b2, b3);
                     }
                 }
-                // ---- S^T += V^T K^   (M = j, N = c, K = i), then scale column c by 2^{a_L[c]}
-                {
-                    const int irow = (lane & 7) + 8 * ((lane >> 3) & 1);
+                const float* dl = reinterpret_cast<const float*>(smem + OFF_DL) + s * 64;
+                const float d_lo = dl[c_lo], d_hi = dl[c_lo + 8];
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-                        for (int cp2 = 0; cp2 < 4; ++cp2) {
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4_t(tkh + swz(16 * kk + irow, 32 * cp2 + 16 * (lane >> 4)), b0, b1, b2, b3);
-                            mma16816(st[2 * cp2], va[kk], b0, b1);
-                            mma16816(st[2 * cp2 + 1], va[kk], b2, b3);
-                        }
-                    }
-                    const float* dl = reinterpret_cast<const float*>(smem + OFF_DL) + b * 64;
-#pragma unroll
-                    for (int n = 0; n < 8; ++n) {
-                        const float2 d2 = *reinterpret_cast<const float2*>(dl + 8 * n + 2 * q);
-                        st[n][0] *= d2.x; st[n][1] *= d2.y; st[n][2] *= d2.x; st[n][3] *= d2.y;
-                    }
-                }
+                for (int n = 0; n < 8; ++n) { st[n][0] *= d_lo; st[n][1] *= d_lo; st[n][2] *= d_hi; st[n][3] *= d_hi; }
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(BAR_EMPTY_V + sv));
-                    mbar_arrive(bar(BAR_RK_FREE + b));
-                    mbar_arrive(bar(BAR_P_FREE + pb));
-                }
-                // ---- epilogue: Y^T accumulators -> bf16 [t][j] tile -> global
-                const uint32_t ty = sbase + OFF_Y + (ybuf_uses % NBUF_Y) * TILE;
-                ++ybuf_uses;
-                if (ytid == 0) bulk_wait_read<NBUF_Y - 1>();     // the store that last used this buffer has read it
-                if (!ysync(0)) break;
-#pragma unroll
-                for (int np = 0; np < 4; ++np) {
-                    const int mi = lane >> 3, rr = lane & 7;
-                    const int t = 8 * (2 * np + (mi >> 1)) + rr;
-                    stsm_x4_t(ty + swz(t, (2 * yw + (mi & 1)) << 4),
-                              pack_bf16(ya[2 * np][0], ya[2 * np][1]), pack_bf16(ya[2 * np][2], ya[2 * np][3]),
-                              pack_bf16(ya[2 * np + 1][0], ya[2 * np + 1][1]), pack_bf16(ya[2 * np + 1][2], ya[2 * np + 1][3]));
-                }
-                fence_proxy_async();
-                if (!ysync(1)) break;
-                if (valid == L) {
-                    if (ytid == 0) {
-                        tma_store_2d(&tm_y, col0, (int)(row0 + (long long)c * L), ty);
-                        bulk_commit();
-                    }
-                } else {
-                    // ragged tail: the rows after `valid` belong to someone else, so copy row by row
-                    for (int i = ytid; i < valid * 8; i += 128) {
-                        const int t = i >> 3, ch = i & 7;
-                        uint4 val;
-                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                     : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(ty + swz(t, ch << 4)));
-                        *reinterpret_cast<uint4*>(p.y + (size_t)(row0 + (long long)c * L + t) * C + col0 + ch * 8) = val;
-                    }
-                    if (ytid == 0) bulk_commit();
-                }
+                if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));
             } else {
-                // ---- decay too strong for one in-chunk reference point: exact fp32 recurrence, token by token
+                // ---- decay too strong for one in-chunk reference point: exact fp32 recurrence, token by
+                // token, on a copy of the state in shared memory where a warp owns 16 value channels for
+                // all 64 key channels.
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(bar(BAR_EMPTY_V + sv));
-                    mbar_arrive(bar(BAR_RK_FREE + b));
-                    mbar_arrive(bar(BAR_P_FREE + pb));
-                }
-                const float* ug = p.u + h * 64;
-                for (int t = 0; t < valid; ++t) {
-                    const size_t ro = (size_t)(row0 + (long long)c * L + t) * C + col0;
-                    // bonus coefficient over all 64 channels
-                    float cf = __bfloat162float(p.r[ro + lane]) * ug[lane] * __bfloat162float(p.k[ro + lane]) +
-                               __bfloat162float(p.r[ro + lane + 32]) * ug[lane + 32] * __bfloat162float(p.k[ro + lane + 32]);
+                if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));
+                float* scr = reinterpret_cast<float*>(smem + OFF_SCR);
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) cf += __shfl_xor_sync(0xffffffffu, cf, o);
-                    const float v_lo = __bfloat162float(p.v[ro + j0]), v_hi = __bfloat162float(p.v[ro + j0 + 8]);
-                    float y_lo = 0.f, y_hi = 0.f;
-#pragma unroll
-                    for (int n = 0; n < 8; ++n) {
-                        const int c0 = 8 * n + 2 * q;
-                        const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + c0);
-                        const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + c0);
-                        const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + c0);
-                        const float w0 = expf(-expf(bf_lo(xw))), w1 = expf(-expf(bf_hi(xw)));
-                        y_lo = fmaf(bf_lo(rw), st[n][0], y_lo); y_lo = fmaf(bf_hi(rw), st[n][1], y_lo);
-                        y_hi = fmaf(bf_lo(rw), st[n][2], y_hi); y_hi = fmaf(bf_hi(rw), st[n][3], y_hi);
-                        st[n][0] = fmaf(w0, st[n][0], bf_lo(kw) * v_lo); st[n][1] = fmaf(w1, st[n][1], bf_hi(kw) * v_lo);
-                        st[n][2] = fmaf(w0, st[n][2], bf_lo(kw) * v_hi); st[n][3] = fmaf(w1, st[n][3], bf_hi(kw) * v_hi);
-                    }
-                    y_lo += __shfl_xor_sync(0xffffffffu, y_lo, 1); y_lo += __shfl_xor_sync(0xffffffffu, y_lo, 2);
-                    y_hi += __shfl_xor_sync(0xffffffffu, y_hi, 1); y_hi += __shfl_xor_sync(0xffffffffu, y_hi, 2);
-                    if (q == 0) {
-                        p.y[ro + j0] = __float2bfloat16_rn(fmaf(cf, v_lo, y_lo));
-                        p.y[ro + j0 + 8] = __float2bfloat16_rn(fmaf(cf, v_hi, y_hi));
+                for (int n = 0; n < 8; ++n) {
+                    *reinterpret_cast<float2*>(scr + c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
+                    *reinterpret_cast<float2*>(scr + (c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
+                }
+                if (!ssync()) break;
+                {
+                    // lane = 16*half + jl works on S[32*half .. +31][16*sw + jl], kept in the fp32 scratch
+                    const int half = lane >> 4, j = 16 * sw + (lane & 15);
+                    float* scol = scr + (32 * half) * 64 + j;
+                    const float* ug = p.u + h * 64 + 32 * half;
+                    for (int t = 0; t < valid; ++t) {
+                        const size_t ro = (size_t)(row0 + (long long)c * L + t) * C + col0;
+                        const float vj = __bfloat162float(p.v[ro + j]);
+                        float yj = 0.f, cf = 0.f;
+#pragma unroll 4
+                        for (int i = 0; i < 32; i += 2) {
+                            const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
+                            const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + 32 * half + i);
+                            const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + 32 * half + i);
+                            const float s0 = scol[i * 64], s1 = scol[(i + 1) * 64];
+                            cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
+                            cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
+                            yj = fmaf(bf_lo(rw), s0, yj);
+                            yj = fmaf(bf_hi(rw), s1, yj);
+                            scol[i * 64] = fmaf(expf(-expf(bf_lo(xw))), s0, bf_lo(kw) * vj);
+                            scol[(i + 1) * 64] = fmaf(expf(-expf(bf_hi(xw))), s1, bf_hi(kw) * vj);
+                        }
+                        yj += __shfl_xor_sync(0xffffffffu, yj, 16);
+                        cf += __shfl_xor_sync(0xffffffffu, cf, 16);
+                        if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
                     }
                 }
+                if (!ssync()) break;
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                    const float2 lo = *reinterpret_cast<const float2*>(scr + c_lo * 64 + 8 * n + 2 * q);
+                    const float2 hi = *reinterpret_cast<const float2*>(scr + (c_lo + 8) * 64 + 8 * n + 2 * q);
+                    st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
+                }
+                if (!ssync()) break;          // everyone has re-read the scratch before it can be rewritten
+            }
+            if (c + 1 < nchunks) {
+                const int nb = (c + 1) % NSB;
+                if (c + 1 >= NSB && !mbar_wait(bar(BAR_S_FREE + nb), (((c + 1) / NSB) & 1) ^ 1, abort_flag)) break;
+                store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sw, st, lane);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_S_READY + nb));
             }
         }
-        if (ytid == 0) bulk_wait<0>();
         if (p.state_out && !*abort_flag) {
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
-                const int c0 = 8 * n + 2 * q;
-                p.state_out[sb + (size_t)c0 * 64 + j0] = st[n][0];
-                p.state_out[sb + (size_t)(c0 + 1) * 64 + j0] = st[n][1];
-                p.state_out[sb + (size_t)c0 * 64 + j0 + 8] = st[n][2];
-                p.state_out[sb + (size_t)(c0 + 1) * 64 + j0 + 8] = st[n][3];
+                *reinterpret_cast<float2*>(p.state_out + sb + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
+                *reinterpret_cast<float2*>(p.state_out + sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
             }
         }
+    } else {
+        // ============================== output warps ==============================
+        const int yw = warp - WARP_Y0;           // 0..7
+        const int grp = yw >> 2, w4 = yw & 3;    // group grp takes chunks grp, grp+2, ...
+        const int g = lane >> 2, q = lane & 3;
+        const uint32_t slab = sbase + OFF_Y + yw * 2048;
+        const int krow = (lane & 7) + 8 * ((lane >> 3) & 1);      // [k][n] tiles read with .trans
+        for (int c = grp; c < nchunks; c += 2) {
+            const int s = c % NS, sbi = c % NSB;
+            const int valid = min(L, len - c * L);
+            // alternate the row block between rounds so the causal triangle's work evens out
+            const int rb = ((c >> 1) & 1) ? 3 - w4 : w4;          // rows t = 16*rb .. 16*rb+15
+            const uint32_t tr = sbase + OFF_RKV + s * 3 * TILE, tk = tr + TILE, tv = tr + 2 * TILE;
+            const uint32_t tsb = sbase + OFF_SB + sbi * TILE;
+            if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_RK_READY + s), (c / NS) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_S_READY + sbi), (c / NSB) & 1, abort_flag)) break;
+            if (!safe_flag[s]) {
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(bar(BAR_S_FREE + sbi)); mbar_arrive(bar(BAR_EMPTY_RKV + s)); }
+                continue;
+            }
+            // R^ rows of this block are re-read from shared memory at every use (A fragments, 4 registers
+            // at a time) instead of being held for the whole chunk: registers are the scarcer resource
+            const uint32_t ta = tr + (16 * rb + (lane & 7) + 8 * ((lane >> 3) & 1)) * 128;
+            const int ta_x = (lane & 7) << 4, ta_c = 16 * (lane >> 4);
+            float ya[8][4];
+#pragma unroll
+            for (int n = 0; n < 8; ++n) ya[n][0] = ya[n][1] = ya[n][2] = ya[n][3] = 0.f;
+            // ---- Y = R^ S_0   (M = t, N = j, K = c)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                uint32_t a[4];
+                ldsm_x4(ta + ((32 * kk + ta_c) ^ ta_x), a[0], a[1], a[2], a[3]);
+#pragma unroll
+                for (int jp = 0; jp < 4; ++jp) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(tsb + swz(16 * kk + krow, 32 * jp + 16 * (lane >> 4)), b0, b1, b2, b3);
+                    mma16816(ya[2 * jp], a, b0, b1);
+                    mma16816(ya[2 * jp + 1], a, b2, b3);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_S_FREE + sbi));
+            // ---- Y += (tril(R^ K^^T, -1) + diag(bonus)) V, one 16-token block of past tokens at a time
+            const float* du = reinterpret_cast<const float*>(smem + OFF_DU) + s * 64;
+            for (int ib = 0; ib <= rb; ++ib) {
+                float acc[2][4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[0][e] = acc[1][e] = 0.f;
+                const int irow = 16 * ib + (lane & 7) + 8 * (lane >> 4);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    uint32_t a[4], b0, b1, b2, b3;
+                    ldsm_x4(ta + ((32 * kk + ta_c) ^ ta_x), a[0], a[1], a[2], a[3]);
+                    ldsm_x4(tk + swz(irow, 32 * kk + 16 * ((lane >> 3) & 1)), b0, b1, b2, b3);
+                    mma16816(acc[0], a, b0, b1);
+                    mma16816(acc[1], a, b2, b3);
+                }
+                if (ib == rb) {
+                    // diagonal block: strictly-lower entries stay, the diagonal takes the bonus
+                    // coefficient, the upper triangle is zero
+                    const float d_lo = du[16 * rb + g], d_hi = du[16 * rb + g + 8];
+#pragma unroll
+                    for (int nb = 0; nb < 2; ++nb) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int il = 8 * nb + 2 * q + e;
+                            acc[nb][e] = il < g ? acc[nb][e] : (il == g ? d_lo : 0.f);
+                            acc[nb][2 + e] = il < g + 8 ? acc[nb][2 + e] : (il == g + 8 ? d_hi : 0.f);
+                        }
+                    }
+                }
+                uint32_t pa[4];
+                pa[0] = pack_bf16(acc[0][0], acc[0][1]);
+                pa[1] = pack_bf16(acc[0][2], acc[0][3]);
+                pa[2] = pack_bf16(acc[1][0], acc[1][1]);
+                pa[3] = pack_bf16(acc[1][2], acc[1][3]);
+#pragma unroll
+                for (int jp = 0; jp < 4; ++jp) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(tv + swz(16 * ib + krow, 32 * jp + 16 * (lane >> 4)), b0, b1, b2, b3);
+                    mma16816(ya[2 * jp], pa, b0, b1);
+                    mma16816(ya[2 * jp + 1], pa, b2, b3);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar(BAR_EMPTY_RKV + s));
+                bulk_wait_read<0>();              // this warp's previous store has finished reading the slab
+            }
+            __syncwarp();
+            // ---- epilogue: this warp's 16 rows of y -> bf16 slab -> global
+            store_acc_bf16(slab, 0, ya, lane);
+            fence_proxy_async();
+            __syncwarp();
+            const int rows = valid - 16 * rb;
+            const long long grow = row0 + (long long)c * L + 16 * rb;
+            if (rows >= 16) {
+                if (lane == 0) {
+                    tma_store_2d(&tm_y16, col0, (int)grow, slab);
+                    bulk_commit();
+                }
+            } else {
+                // ragged tail: the rows after `valid` belong to someone else, so copy row by row
+                for (int i = lane; i < rows * 8; i += 32) {
+                    const int t = i >> 3, ch = i & 7;
+                    uint4 val;
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(slab + swz(t, ch << 4)));
+                    *reinterpret_cast<uint4*>(p.y + (size_t)(grow + t) * C + col0 + ch * 8) = val;
+                }
+                __syncwarp();
+            }
+        }
+        if (lane == 0) bulk_wait<0>();
     }
 }
 
@@ -653,14 +704,14 @@ inline EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [rows][C] bf16 tensor, box = 64 rows x 64 channels (128 bytes), 128-byte swizzle
-inline bool make_map(CUtensorMap* tm, const void* base, long long rows, long long C)
+// [rows][C] bf16 tensor, box = box_rows rows x 64 channels (128 bytes), 128-byte swizzle
+inline bool make_map(CUtensorMap* tm, const void* base, long long rows, long long C, int box_rows)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)C * 2};
-    cuuint32_t box[2] = {64, 64};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -690,9 +741,9 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     }
     CUtensorMap tr, tk, tv, tx, ty;
     const long long C = (long long)H * 64;
-    if (!ck::make_map(&tr, r, total_rows, C) || !ck::make_map(&tk, k, total_rows, C) ||
-        !ck::make_map(&tv, v, total_rows, C) || !ck::make_map(&tx, x, total_rows, C) ||
-        !ck::make_map(&ty, y, total_rows, C))
+    if (!ck::make_map(&tr, r, total_rows, C, 64) || !ck::make_map(&tk, k, total_rows, C, 64) ||
+        !ck::make_map(&tv, v, total_rows, C, 64) || !ck::make_map(&tx, x, total_rows, C, 64) ||
+        !ck::make_map(&ty, y, total_rows, C, 16))
         return GF_ERR_CUDA;
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H};
     ck::wkv6_chunked_kernel<<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
