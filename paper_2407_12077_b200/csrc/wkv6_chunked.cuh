@@ -16,17 +16,18 @@
 // violates it is processed token by token in fp32 instead, so any finite or infinite decay
 // logit gives the exact-recurrence result.
 //
-// Warp roles (704 threads), pipelined across chunks through mbarriers:
-//   warp 0        TMA producer: x tiles (4-stage ring) and {r,k,v} tiles (5-stage ring)
+// Warp roles (960 threads), pipelined across chunks through mbarriers:
+//   warp 0        TMA producer: {x,r,k,v} tiles of a chunk into one stage of a 5-stage ring
 //   warp 1        tensor-memory allocation; one lane issues every tcgen05.mma:
-//                   P = R^ K^^T, dS = K^^T V (one chunk ahead), then Y = R^ S_0 + P' V
+//                   P = R^ K^^T, dS = K^^T V (one chunk ahead) interleaved with Y0 = R^ S_0, PV = P' V
 //   warps 2-5     state: S <- diag(2^{a_L}) (S + dS) in fp32 registers for the whole sequence;
 //                 publishes a bf16 copy of every chunk-start state as an MMA operand
 //   warps 6-9     scores: P from tensor memory -> P' = tril(P,-1) + diag(bonus) -> bf16 operand tile
-//   warps 10-13   output: Y from tensor memory -> bf16 -> TMA store (each warp its own 16 rows)
-//   warps 14-21   elementwise: decay, cumulative sum (phase A, one chunk ahead), then in place
-//                 R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t} (phase B); chunk decay 2^{a_L}, bonus
-//                 coefficients, safety vote
+//   warps 10-13   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows)
+//   warps 14-29   elementwise, two sets of eight warps taking alternate chunks: decay and
+//                 cumulative sum (phase A), then in place R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t}
+//                 (phase B); chunk decay 2^{a_L}, bonus coefficients, safety vote.  A lane owns
+//                 4 tokens x 4 channels (64-bit shared-memory accesses, packed fp32x2 arithmetic)
 // A warp reads the tensor-memory lanes of its own sub-partition (warp index mod 4), which hold
 // accumulator rows 16*(warp mod 4) .. +15 of a 64-row tile.
 // Every wait is bounded: on expiry the kernel raises a status flag and all roles leave.
@@ -58,36 +59,36 @@ namespace ck {
 
 constexpr int L = 64;                  // tokens per chunk
 constexpr int TILE = 64 * 64 * 2;      // one bf16 [64 x 64] tile
-constexpr int NX = 4;                  // x ring depth
-constexpr int NS = 5;                  // {r,k,v} ring depth
+constexpr int NS = 5;                  // {x,r,k,v} ring depth
 constexpr int NSB = 2;                 // bf16 chunk-start state operand tiles
 constexpr int NPP = 2;                 // bf16 masked-score operand tiles
-constexpr int NTOT = 4;                // per-warp decay-total buffers (phase A runs one chunk ahead)
-constexpr int N_EW = 8;                // elementwise warps
+constexpr int NTOT = 4;                // per-warp decay-total buffers (two per elementwise set)
+constexpr int N_EW = 8;                // elementwise warps per set
+constexpr int N_ESET = 2;              // elementwise sets (alternate chunks)
 constexpr int N_GW = 4;                // warps per tensor-memory reader group (one per sub-partition)
 constexpr int WARP_MMA = 1;
 constexpr int WARP_S0 = 2;             // state warps
 constexpr int WARP_P0 = WARP_S0 + N_GW;   // score warps
 constexpr int WARP_Y0 = WARP_P0 + N_GW;   // output warps
 constexpr int WARP_E0 = WARP_Y0 + N_GW;   // elementwise warps
-constexpr int THREADS = 32 * (WARP_E0 + N_EW);
+constexpr int THREADS = 32 * (WARP_E0 + N_ESET * N_EW);
 constexpr float A2_MAX = 96.f;         // largest in-chunk |cumulative log2 decay| on the tensor-core path
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LOG2_LOG2E = 0.5287663729448977f;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+constexpr uint32_t TRY_WAIT_HINT_NS = 20000;                  // a waiting thread may be suspended this long per try
 
 // tensor memory: 64 fp32 columns per 64x64 accumulator, two buffers each
 constexpr int TM_COLS = 512;
-constexpr int TM_P = 0, TM_DS = 128, TM_Y = 256;
+constexpr int TM_P = 0, TM_DS = 128, TM_Y0 = 256, TM_PV = 384;
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr int OFF_X = 0;                                   // [NX][TILE]           x
-constexpr int OFF_RKV = OFF_X + NX * TILE;                 // [NS][3][TILE]        r -> R^, k -> K^, v
-constexpr int OFF_SB = OFF_RKV + NS * 3 * TILE;            // [NSB][TILE]          bf16 chunk-start state [c][j]
+constexpr int STAGE = 4 * TILE;                            // one ring stage: x, r -> R^, k -> K^, v
+constexpr int OFF_RING = 0;                                // [NS][STAGE]
+constexpr int OFF_SB = OFF_RING + NS * STAGE;              // [NSB][TILE]          bf16 chunk-start state [c][j]
 constexpr int OFF_PP = OFF_SB + NSB * TILE;                // [NPP][TILE]          bf16 masked scores [t][i]
 constexpr int OFF_Y = OFF_PP + NPP * TILE;                 // [N_GW][16 rows x 128 B] y staging, one slab per warp
-constexpr int OFF_SCR = OFF_Y + N_GW * 2048;               // [64][64] float       state scratch (token-by-token path)
-constexpr int OFF_TOT = OFF_SCR + 64 * 64 * 4;             // [NTOT][N_EW][64] float
+constexpr int OFF_TOT = OFF_Y + N_GW * 2048;               // [NTOT][N_EW][64] float
 constexpr int OFF_DL = OFF_TOT + NTOT * N_EW * 64 * 4;     // [NS][64] float       2^{a_L}
 constexpr int OFF_DU = OFF_DL + NS * 64 * 4;               // [NS][64] float       bonus coefficient per token
 constexpr int OFF_SAFE = OFF_DU + NS * 64 * 4;             // [NS] int (padded)
@@ -95,9 +96,7 @@ constexpr int OFF_ABORT = OFF_SAFE + 32;                   // int
 constexpr int OFF_TMEM = OFF_ABORT + 8;                    // uint32: tensor-memory base address
 constexpr int OFF_BAR = OFF_ABORT + 16;                    // mbarriers (8 bytes each)
 enum {
-    BAR_FULL_X = 0,
-    BAR_EMPTY_X = BAR_FULL_X + NX,
-    BAR_FULL_RKV = BAR_EMPTY_X + NX,
+    BAR_FULL_RKV = 0,
     BAR_EMPTY_RKV = BAR_FULL_RKV + NS,
     BAR_RK_READY = BAR_EMPTY_RKV + NS,
     BAR_S_READY = BAR_RK_READY + NS,
@@ -110,7 +109,7 @@ enum {
     BAR_DS_EMPTY = BAR_DS_FULL + 2,
     BAR_Y_FULL = BAR_DS_EMPTY + 2,
     BAR_Y_EMPTY = BAR_Y_FULL + 2,
-    BAR_ESYNC = BAR_Y_EMPTY + 2,         // two, alternating by chunk parity
+    BAR_ESYNC = BAR_Y_EMPTY + 2,         // one per elementwise set
     BAR_SSYNC = BAR_ESYNC + 2,           // state-warp rendezvous (token-by-token path only)
     BAR_COUNT = BAR_SSYNC + 1
 };
@@ -138,9 +137,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(TRY_WAIT_HINT_NS) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ unsigned long long globaltimer()
@@ -169,6 +168,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, poll_abort);
+}
+
+// Warp-uniform form: every lane of a converged warp waits and all get the same answer, so the
+// caller's control flow stays uniform (the compiler can then keep addresses in uniform registers).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool poll_abort = true)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, poll_abort));
+}
+// True on exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar)
@@ -232,20 +249,17 @@ constexpr uint32_t IDESC_K_K = IDESC;
 constexpr uint32_t IDESC_K_MN = IDESC | (1u << 16);
 constexpr uint32_t IDESC_MN_MN = IDESC | (1u << 15) | (1u << 16);
 
-// Reads this warp's 16 rows x 64 fp32 columns of an accumulator (lanes of its own sub-partition)
-// and waits for the data: v[n][0..1] = (row g, cols 8n+2q, +1), v[n][2..3] = (row g+8, same cols)
-// with g = lane / 4, q = lane % 4.
-__device__ __forceinline__ void tmem_ld_16x64(uint32_t taddr, float (&v)[8][4])
+// Reads 16 rows x 32 fp32 columns of an accumulator from this warp's sub-partition and waits for
+// the data: v[n][0..1] = (row g, cols 8n+2q, +1), v[n][2..3] = (row g+8, same cols) relative to the
+// address, with g = lane / 4, q = lane % 4.
+__device__ __forceinline__ void tmem_ld_16x32(uint32_t taddr, float (&v)[4][4])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
         "tcgen05.wait::ld.sync.aligned;"
         : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3]),
-          "=f"(v[2][0]), "=f"(v[2][1]), "=f"(v[2][2]), "=f"(v[2][3]), "=f"(v[3][0]), "=f"(v[3][1]), "=f"(v[3][2]), "=f"(v[3][3]),
-          "=f"(v[4][0]), "=f"(v[4][1]), "=f"(v[4][2]), "=f"(v[4][3]), "=f"(v[5][0]), "=f"(v[5][1]), "=f"(v[5][2]), "=f"(v[5][3]),
-          "=f"(v[6][0]), "=f"(v[6][1]), "=f"(v[6][2]), "=f"(v[6][3]), "=f"(v[7][0]), "=f"(v[7][1]), "=f"(v[7][2]), "=f"(v[7][3])
+          "=f"(v[2][0]), "=f"(v[2][1]), "=f"(v[2][2]), "=f"(v[2][3]), "=f"(v[3][0]), "=f"(v[3][1]), "=f"(v[3][2]), "=f"(v[3][3])
         : "r"(taddr) : "memory");
 }
 
@@ -255,19 +269,61 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ uint32_t lds32(uint32_t a)
+// packed fp32x2 arithmetic (one instruction for two lanes of a float2)
+__device__ __forceinline__ unsigned long long pk(float2 a)
 {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a.x), "f"(a.y));
+    return r;
+}
+__device__ __forceinline__ float2 upk(unsigned long long r)
+{
+    float2 a;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a.x), "=f"(a.y) : "l"(r));
+    return a;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
+{
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(pk(a)), "l"(pk(b)), "l"(pk(c)));
+    return upk(d);
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b)
+{
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pk(a)), "l"(pk(b)));
+    return upk(d);
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b)
+{
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pk(a)), "l"(pk(b)));
+    return upk(d);
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b)
+{
+    unsigned long long d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pk(a)), "l"(pk(b)));
+    return upk(d);
+}
+__device__ __forceinline__ float2 ex2_2(float2 a) { return make_float2(ex2(a.x), ex2(a.y)); }
+__device__ __forceinline__ uint2 lds64(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
     return v;
 }
-__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void sts64(uint32_t a, uint2 v)
+{
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
+}
 __device__ __forceinline__ void sts128z(uint32_t a)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ float2 bf_pair(uint32_t w) { return make_float2(bf_lo(w), bf_hi(w)); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
@@ -305,23 +361,47 @@ __device__ __forceinline__ void store_acc_bf16(uint32_t tile, int row0, const fl
                 pack_bf16(acc[2 * m][0], acc[2 * m][1]), pack_bf16(acc[2 * m][2], acc[2 * m][3]),
                 pack_bf16(acc[2 * m + 1][0], acc[2 * m + 1][1]), pack_bf16(acc[2 * m + 1][2], acc[2 * m + 1][3]));
 }
+// The same for one half of the columns: acc holds columns 32*HALF .. 32*HALF+31.
+template <int HALF>
+__device__ __forceinline__ void store_half_bf16(uint32_t tile, int row0, const float (&acc)[4][4], int lane)
+{
+    const int mi = lane >> 3, rr = lane & 7;
+    const int row = row0 + rr + 8 * (mi & 1);
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+        stsm_x4(tile + swz(row, (2 * (2 * HALF + m) + (mi >> 1)) << 4),
+                pack_bf16(acc[2 * m][0], acc[2 * m][1]), pack_bf16(acc[2 * m][2], acc[2 * m][3]),
+                pack_bf16(acc[2 * m + 1][0], acc[2 * m + 1][1]), pack_bf16(acc[2 * m + 1][2], acc[2 * m + 1][3]));
+}
 
-// P' = tril(P, -1) + diag(bonus) on one warp's 16 rows (rows 16*SP + g and + 8) of the score block.
-template <int SP>
-__device__ __forceinline__ void mask_scores(float (&acc)[8][4], int g, int q, float d_lo, float d_hi)
+// P' = tril(P, -1) + diag(bonus) on columns 32*HALF .. +31 of one warp's 16 rows (rows 16*SP + g
+// and + 8) of the score block.
+template <int SP, int HALF>
+__device__ __forceinline__ void mask_scores(float (&acc)[4][4], int g, int q, float d_lo, float d_hi)
 {
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
+    for (int nn = 0; nn < 4; ++nn) {
+        const int n = 4 * HALF + nn;
         if (n > 2 * SP + 1) {
-            acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;            // above the diagonal block
+            acc[nn][0] = acc[nn][1] = acc[nn][2] = acc[nn][3] = 0.f;         // above the diagonal block
         } else if (n >= 2 * SP) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int il = 8 * (n - 2 * SP) + 2 * q + e;                 // column inside the 16 x 16 diagonal block
-                acc[n][e] = il < g ? acc[n][e] : (il == g ? d_lo : 0.f);
-                acc[n][2 + e] = il < g + 8 ? acc[n][2 + e] : (il == g + 8 ? d_hi : 0.f);
+                acc[nn][e] = il < g ? acc[nn][e] : (il == g ? d_lo : 0.f);
+                acc[nn][2 + e] = il < g + 8 ? acc[nn][2 + e] : (il == g + 8 ? d_hi : 0.f);
             }
         }
+    }
+}
+template <int HALF>
+__device__ __forceinline__ void mask_scores_sp(int sp, float (&acc)[4][4], int g, int q, float d_lo, float d_hi)
+{
+    switch (sp) {
+    case 0: mask_scores<0, HALF>(acc, g, q, d_lo, d_hi); break;
+    case 1: mask_scores<1, HALF>(acc, g, q, d_lo, d_hi); break;
+    case 2: mask_scores<2, HALF>(acc, g, q, d_lo, d_hi); break;
+    default: mask_scores<3, HALF>(acc, g, q, d_lo, d_hi); break;
     }
 }
 
@@ -355,7 +435,6 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     const size_t C = (size_t)p.H * 64;
 
     if (tid == 0) {
-        for (int i = 0; i < NX; ++i) { mbar_init(bar(BAR_FULL_X + i), 1); mbar_init(bar(BAR_EMPTY_X + i), N_EW); }
         for (int i = 0; i < NS; ++i) {
             mbar_init(bar(BAR_FULL_RKV + i), 1);
             mbar_init(bar(BAR_EMPTY_RKV + i), 1 + 3 * N_GW);       // MMA commit + state, score and output warps
@@ -367,8 +446,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             mbar_init(bar(BAR_P_FULL + i), 1);  mbar_init(bar(BAR_P_EMPTY + i), N_GW);
             mbar_init(bar(BAR_DS_FULL + i), 1); mbar_init(bar(BAR_DS_EMPTY + i), N_GW);
             mbar_init(bar(BAR_Y_FULL + i), 1);  mbar_init(bar(BAR_Y_EMPTY + i), N_GW);
-            mbar_init(bar(BAR_ESYNC + i), N_EW);
         }
+        for (int i = 0; i < N_ESET; ++i) mbar_init(bar(BAR_ESYNC + i), N_EW);
         mbar_init(bar(BAR_SSYNC), N_GW);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -382,99 +461,104 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
 
     if (warp == 0) {
         // ============================== TMA producer ==============================
-        if (lane == 0) {
-            int issued_x = 0, issued_s = 0;
-            auto load_x = [&](int c) -> bool {
-                const int sx = c % NX;
-                if (c >= NX && !mbar_wait(bar(BAR_EMPTY_X + sx), ((c / NX) & 1) ^ 1, abort_flag)) return false;
-                mbar_expect_tx(bar(BAR_FULL_X + sx), TILE);
-                tma_load_2d(sbase + OFF_X + sx * TILE, &tm_x, col0, (int)(row0 + (long long)c * L), bar(BAR_FULL_X + sx));
-                issued_x = c + 1;
-                return true;
-            };
-            bool ok = true;
-            for (int c = 0; c < min(NX - 1, nchunks) && ok; ++c) ok = load_x(c);
-            for (int c = 0; c < nchunks && ok; ++c) {
-                if (c + NX - 1 < nchunks && !load_x(c + NX - 1)) break;
-                const int s = c % NS;
-                if (c >= NS && !mbar_wait(bar(BAR_EMPTY_RKV + s), ((c / NS) & 1) ^ 1, abort_flag)) break;
-                const int row = (int)(row0 + (long long)c * L);
-                const uint32_t dst = sbase + OFF_RKV + s * 3 * TILE;
-                mbar_expect_tx(bar(BAR_FULL_RKV + s), 3 * TILE);
-                tma_load_2d(dst, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
-                tma_load_2d(dst + TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
-                tma_load_2d(dst + 2 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
-                issued_s = c + 1;
+        int issued = 0;
+        for (int c = 0; c < nchunks; ++c) {
+            const int s = c % NS;
+            if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ((c / NS) & 1) ^ 1, abort_flag)) break;
+            const int row = (int)(row0 + (long long)c * L);
+            const uint32_t dst = sbase + OFF_RING + s * STAGE;
+            if (elect_one()) {
+                mbar_expect_tx(bar(BAR_FULL_RKV + s), STAGE);
+                tma_load_2d(dst, &tm_x, col0, row, bar(BAR_FULL_RKV + s));
+                tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
+                tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
+                tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
             }
-            // do not leave while copies into this CTA's shared memory may still be in flight
-            for (int c = max(0, issued_x - NX); c < issued_x; ++c)
-                mbar_wait(bar(BAR_FULL_X + c % NX), (c / NX) & 1, abort_flag, false);
-            for (int c = max(0, issued_s - NS); c < issued_s; ++c)
-                mbar_wait(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
+            __syncwarp();
+            issued = c + 1;
         }
+        // do not leave while copies into this CTA's shared memory may still be in flight
+        for (int c = max(0, issued - NS); c < issued; ++c)
+            mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
     } else if (warp == WARP_MMA) {
         // ============================== MMA issuer ==============================
-        if (lane == 0) {
-            // P_c = R^ K^^T and dS_c = K^^T V: depend on the inputs of chunk c only
-            auto front = [&](int c) -> bool {
+        {
+            // One step issues, interleaved so that four independent accumulation chains are in flight,
+            //   P_{c+1} = R^ K^^T, dS_{c+1} = K^^T V      (inputs of chunk c+1 only)
+            //   Y0_c = R^ S_0,  PV_c = P' V               (need the chunk-start state and the masked scores)
+            // Consecutive tcgen05.mma on one accumulator wait for each other; different ones pipeline.
+            auto wait_front = [&](int c) -> bool {
                 const int s = c % NS, tb = c & 1;
-                const uint32_t tr = sbase + OFF_RKV + s * 3 * TILE, tk = tr + TILE, tv = tr + 2 * TILE;
-                if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) return false;
-                if (!mbar_wait(bar(BAR_RK_READY + s), (c / NS) & 1, abort_flag)) return false;
-                const bool safe = safe_flag[s] != 0;
+                if (!mbar_wait_warp(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) return false;
+                if (!mbar_wait_warp(bar(BAR_RK_READY + s), (c / NS) & 1, abort_flag)) return false;
                 if (c >= 2) {
-                    if (!mbar_wait(bar(BAR_P_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                    if (!mbar_wait(bar(BAR_DS_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                }
-                tc_fence_after();
-                if (safe) {
-                    const uint64_t dr = smem_desc(tr), dk = smem_desc(tk), dv = smem_desc(tv);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)           // M = t, N = i, K = c: both operands K-major
-                        tc_mma(tmem + TM_P + 64 * tb, dr + (uint64_t)(2 * kk), dk + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
-                    tc_commit(bar(BAR_P_FULL + tb));
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)           // M = c, N = j, K = i: both operands MN-major
-                        tc_mma(tmem + TM_DS + 64 * tb, dk + (uint64_t)(128 * kk), dv + (uint64_t)(128 * kk), IDESC_MN_MN, kk > 0);
-                    tc_commit(bar(BAR_DS_FULL + tb));
-                } else {
-                    tc_commit(bar(BAR_P_FULL + tb));
-                    tc_commit(bar(BAR_DS_FULL + tb));
+                    if (!mbar_wait_warp(bar(BAR_P_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
+                    if (!mbar_wait_warp(bar(BAR_DS_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
                 }
                 return true;
             };
-            // Y_c = R^ S_0 + P' V: needs the chunk-start state and the masked scores
-            auto back = [&](int c) -> bool {
-                const int s = c % NS, tb = c & 1, sbi = c % NSB, ppi = c % NPP;
-                const uint32_t tr = sbase + OFF_RKV + s * 3 * TILE, tv = tr + 2 * TILE;
-                const bool safe = safe_flag[s] != 0;
-                if (c >= 2 && !mbar_wait(bar(BAR_Y_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                if (!mbar_wait(bar(BAR_S_READY + sbi), (c / NSB) & 1, abort_flag)) return false;
-                tc_fence_after();
-                if (safe) {
-                    const uint64_t dr = smem_desc(tr), ds = smem_desc(sbase + OFF_SB + sbi * TILE);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)           // M = t, N = j, K = c: A K-major, B MN-major
-                        tc_mma(tmem + TM_Y + 64 * tb, dr + (uint64_t)(2 * kk), ds + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
-                }
-                tc_commit(bar(BAR_S_FREE + sbi));
-                if (!mbar_wait(bar(BAR_PP_READY + ppi), (c / NPP) & 1, abort_flag)) return false;
-                tc_fence_after();
-                if (safe) {
-                    const uint64_t dp = smem_desc(sbase + OFF_PP + ppi * TILE), dv = smem_desc(tv);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)           // M = t, N = j, K = i: A K-major, B MN-major
-                        tc_mma(tmem + TM_Y + 64 * tb, dp + (uint64_t)(2 * kk), dv + (uint64_t)(128 * kk), IDESC_K_MN, 1);
-                }
-                tc_commit(bar(BAR_PP_FREE + ppi));
-                tc_commit(bar(BAR_EMPTY_RKV + s));
-                tc_commit(bar(BAR_Y_FULL + tb));
+            auto wait_back = [&](int c) -> bool {
+                const int tb = c & 1, sbi = c % NSB, ppi = c % NPP;
+                if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
+                if (!mbar_wait_warp(bar(BAR_S_READY + sbi), (c / NSB) & 1, abort_flag)) return false;
+                if (!mbar_wait_warp(bar(BAR_PP_READY + ppi), (c / NPP) & 1, abort_flag)) return false;
                 return true;
             };
-            bool ok = nchunks > 0 && front(0);
-            for (int c = 0; c < nchunks && ok; ++c) {
-                if (c + 1 < nchunks && !front(c + 1)) break;
-                ok = back(c);
+            // c_front = chunk whose P / dS are issued (-1: none), c_back = chunk whose Y0 / PV are issued (-1: none)
+            auto step = [&](int c_front, int c_back) {
+                uint64_t dr_f = 0, dk_f = 0, dv_f = 0, dr_b = 0, ds_b = 0, dp_b = 0, dv_b = 0;
+                bool do_f = false, do_b = false;
+                if (c_front >= 0) {
+                    const int s = c_front % NS;
+                    const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
+                    do_f = safe_flag[s] != 0;
+                    dr_f = smem_desc(tr); dk_f = smem_desc(tr + TILE); dv_f = smem_desc(tr + 2 * TILE);
+                }
+                if (c_back >= 0) {
+                    const int s = c_back % NS;
+                    const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
+                    do_b = safe_flag[s] != 0;
+                    dr_b = smem_desc(tr); dv_b = smem_desc(tr + 2 * TILE);
+                    ds_b = smem_desc(sbase + OFF_SB + (c_back % NSB) * TILE);
+                    dp_b = smem_desc(sbase + OFF_PP + (c_back % NPP) * TILE);
+                }
+                const uint32_t tf = 64 * (c_front & 1), tbk = 64 * (c_back & 1);
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (do_f) {
+                        // M = t, N = i, K = c: both operands K-major;  M = c, N = j, K = i: both MN-major
+                        tc_mma(tmem + TM_P + tf, dr_f + (uint64_t)(2 * kk), dk_f + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
+                        tc_mma(tmem + TM_DS + tf, dk_f + (uint64_t)(128 * kk), dv_f + (uint64_t)(128 * kk), IDESC_MN_MN, kk > 0);
+                    }
+                    if (do_b) {
+                        // M = t, N = j, K = c and M = t, N = j, K = i: A K-major, B MN-major
+                        tc_mma(tmem + TM_Y0 + tbk, dr_b + (uint64_t)(2 * kk), ds_b + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+                        tc_mma(tmem + TM_PV + tbk, dp_b + (uint64_t)(2 * kk), dv_b + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+                    }
+                }
+                if (c_front >= 0) {
+                    tc_commit(bar(BAR_P_FULL + (c_front & 1)));
+                    tc_commit(bar(BAR_DS_FULL + (c_front & 1)));
+                }
+                if (c_back >= 0) {
+                    tc_commit(bar(BAR_S_FREE + c_back % NSB));
+                    tc_commit(bar(BAR_PP_FREE + c_back % NPP));
+                    tc_commit(bar(BAR_EMPTY_RKV + c_back % NS));
+                    tc_commit(bar(BAR_Y_FULL + (c_back & 1)));
+                }
+                }
+                __syncwarp();
+            };
+            if (nchunks > 0 && wait_front(0)) {
+                step(0, -1);
+                for (int c = 0; c < nchunks; ++c) {
+                    const bool has_next = c + 1 < nchunks;
+                    if (has_next && !wait_front(c + 1)) break;
+                    if (!wait_back(c)) break;
+                    step(has_next ? c + 1 : -1, c);
+                }
             }
         }
     } else if (warp < WARP_P0) {
@@ -516,17 +600,24 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             tc_fence_after();
             if (safe_flag[s]) {
                 // ---- S <- diag(2^{a_L}) (S + K^^T V)
-                float d[8][4];
-                tmem_ld_16x64(tmem + ((uint32_t)(32 * sp) << 16) + TM_DS + 64 * tb, d);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_DS_EMPTY + tb));
                 const float* dl = reinterpret_cast<const float*>(smem + OFF_DL) + s * 64;
                 const float d_lo = dl[c_lo], d_hi = dl[c_lo + 8];
+                const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_DS + 64 * tb;
 #pragma unroll
-                for (int n = 0; n < 8; ++n) {
-                    st[n][0] = (st[n][0] + d[n][0]) * d_lo; st[n][1] = (st[n][1] + d[n][1]) * d_lo;
-                    st[n][2] = (st[n][2] + d[n][2]) * d_hi; st[n][3] = (st[n][3] + d[n][3]) * d_hi;
+                for (int hf = 0; hf < 2; ++hf) {
+                    float d[4][4];
+                    tmem_ld_16x32(ta + 32 * hf, d);
+                    if (hf == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar(BAR_DS_EMPTY + tb));
+                    }
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) {
+                        float (&sn)[4] = st[4 * hf + n];
+                        sn[0] = (sn[0] + d[n][0]) * d_lo; sn[1] = (sn[1] + d[n][1]) * d_lo;
+                        sn[2] = (sn[2] + d[n][2]) * d_hi; sn[3] = (sn[3] + d[n][3]) * d_hi;
+                    }
                 }
             } else {
                 // ---- decay too strong for one in-chunk reference point: exact fp32 recurrence, token by
@@ -534,7 +625,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // all 64 key channels.
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_DS_EMPTY + tb));
-                float* scr = reinterpret_cast<float*>(smem + OFF_SCR);
+                // The scratch is the x and r tiles of this chunk's ring stage: nothing reads them any more
+                // (the inputs are re-read from global memory here) and the stage is not refilled before
+                // these warps release it.
+                float* scr = reinterpret_cast<float*>(smem + OFF_RING + s * STAGE);
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     *reinterpret_cast<float2*>(scr + c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
@@ -604,29 +698,31 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (!mbar_wait(bar(BAR_P_FULL + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const bool safe = safe_flag[s] != 0;
-            float acc[8][4];
-            if (safe) {
-                tmem_ld_16x64(tmem + ((uint32_t)(32 * sp) << 16) + TM_P + 64 * tb, acc);
-                tc_fence_before();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_P_EMPTY + tb));
+            float d_lo = 0.f, d_hi = 0.f;
             if (safe) {
                 const float* du = reinterpret_cast<const float*>(smem + OFF_DU) + s * 64;
-                const float d_lo = du[16 * sp + g], d_hi = du[16 * sp + g + 8];
-                switch (sp) {
-                case 0: mask_scores<0>(acc, g, q, d_lo, d_hi); break;
-                case 1: mask_scores<1>(acc, g, q, d_lo, d_hi); break;
-                case 2: mask_scores<2>(acc, g, q, d_lo, d_hi); break;
-                default: mask_scores<3>(acc, g, q, d_lo, d_hi); break;
-                }
+                d_lo = du[16 * sp + g]; d_hi = du[16 * sp + g + 8];
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));           // done with this slot's bonus vector and flag
             if (c >= NPP && !mbar_wait(bar(BAR_PP_FREE + ppi), ((c / NPP) & 1) ^ 1, abort_flag)) break;
             if (safe) {
-                store_acc_bf16(sbase + OFF_PP + ppi * TILE, 16 * sp, acc, lane);
+                const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_P + 64 * tb;
+                const uint32_t tp = sbase + OFF_PP + ppi * TILE;
+                float acc[4][4];
+                tmem_ld_16x32(ta, acc);
+                mask_scores_sp<0>(sp, acc, g, q, d_lo, d_hi);
+                store_half_bf16<0>(tp, 16 * sp, acc, lane);
+                tmem_ld_16x32(ta + 32, acc);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_P_EMPTY + tb));
+                mask_scores_sp<1>(sp, acc, g, q, d_lo, d_hi);
+                store_half_bf16<1>(tp, 16 * sp, acc, lane);
                 fence_proxy_async();
+            } else {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_P_EMPTY + tb));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_PP_READY + ppi));
@@ -641,21 +737,39 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (!mbar_wait(bar(BAR_Y_FULL + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const bool safe = safe_flag[s] != 0;
-            float ya[8][4];
-            if (safe) {
-                tmem_ld_16x64(tmem + ((uint32_t)(32 * sp) << 16) + TM_Y + 64 * tb, ya);
-                tc_fence_before();
-            }
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(bar(BAR_Y_EMPTY + tb));
                 mbar_arrive(bar(BAR_EMPTY_RKV + s));                      // done with this slot's flag
                 bulk_wait_read<0>();              // this warp's previous store has finished reading the slab
             }
             __syncwarp();
-            if (!safe) continue;                  // the state warps wrote this chunk's y themselves
+            if (!safe) {                          // the state warps wrote this chunk's y themselves
+                if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
+                continue;
+            }
             // ---- this warp's 16 rows of y -> bf16 slab -> global
-            store_acc_bf16(slab, 0, ya, lane);
+            {
+                const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_Y0 + 64 * tb;
+                const uint32_t tc = tmem + ((uint32_t)(32 * sp) << 16) + TM_PV + 64 * tb;
+                float ya[4][4], yb[4][4];
+                tmem_ld_16x32(ta, ya);
+                tmem_ld_16x32(tc, yb);
+#pragma unroll
+                for (int n = 0; n < 4; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) ya[n][e] += yb[n][e];
+                store_half_bf16<0>(slab, 0, ya, lane);
+                tmem_ld_16x32(ta + 32, ya);
+                tmem_ld_16x32(tc + 32, yb);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
+#pragma unroll
+                for (int n = 0; n < 4; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) ya[n][e] += yb[n][e];
+                store_half_bf16<1>(slab, 0, ya, lane);
+            }
             fence_proxy_async();
             __syncwarp();
             const int rows = valid - 16 * sp;
@@ -680,110 +794,116 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         if (lane == 0) bulk_wait<0>();
     } else {
         // ============================== elementwise warps ==============================
-        const int tq = warp - WARP_E0;           // tokens 8*tq .. 8*tq+7 of the chunk
-        const int cb = lane * 4;                 // byte column of this lane's channel pair (2*lane, 2*lane+1)
-        const int etid = tid - 32 * WARP_E0;     // 0..255
-        const float2 u2 = *reinterpret_cast<const float2*>(p.u + h * 64 + 2 * lane);
+        const int eset = (warp - WARP_E0) / N_EW;        // this set takes chunks eset, eset + 2, ...
+        const int tq = (warp - WARP_E0) % N_EW;          // tokens 8*tq .. 8*tq+7 of the chunk
+        const int cq = lane & 15, th = lane >> 4;        // channels 4*cq .. 4*cq+3, tokens 8*tq + 4*th + (0..3)
+        const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
+        const float4 u4 = *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
+        const float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
         float* tot = reinterpret_cast<float*>(smem + OFF_TOT);
-        // phase A of chunk c: log2-decay magnitudes and this warp's local cumulative sums
-        auto phase_a = [&](int c, float (&l0)[8], float (&l1)[8]) -> bool {
-            const int sx = c % NX;
-            const int valid = min(L, len - c * L);
-            const uint32_t tx = sbase + OFF_X + sx * TILE;
-            if (!mbar_wait(bar(BAR_FULL_X + sx), (c / NX) & 1, abort_flag)) return false;
-            float a0 = 0.f, a1 = 0.f;
+        uint32_t roff[4];                                // swizzled byte offsets of this lane's 8 bytes in its 4 rows
 #pragma unroll
-            for (int tt = 0; tt < 8; ++tt) {
-                const int t = 8 * tq + tt;
-                const uint32_t xw = lds32(tx + swz(t, cb));
-                float e0 = ex2(fmaf(bf_lo(xw), LOG2E, LOG2_LOG2E));
-                float e1 = ex2(fmaf(bf_hi(xw), LOG2E, LOG2_LOG2E));
-                if (t >= valid) { e0 = 0.f; e1 = 0.f; }
-                a0 -= e0; a1 -= e1;
-                l0[tt] = a0; l1[tt] = a1;
-            }
-            *reinterpret_cast<float2*>(tot + ((c % NTOT) * N_EW + tq) * 64 + 2 * lane) = make_float2(a0, a1);
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(BAR_EMPTY_X + sx));
-                mbar_arrive(bar(BAR_ESYNC + (c & 1)));
-            }
-            return true;
-        };
-        float l0[8], l1[8];
-        bool live = nchunks > 0 && phase_a(0, l0, l1);
-        for (int c = 0; c < nchunks && live; ++c) {
-            float n0[8], n1[8];
-            if (c + 1 < nchunks && !phase_a(c + 1, n0, n1)) break;
+        for (int tt = 0; tt < 4; ++tt) roff[tt] = swz(8 * tq + 4 * th + tt, 8 * cq);
+        const float2 kLog2e = make_float2(LOG2E, LOG2E), kLogLog = make_float2(LOG2_LOG2E, LOG2_LOG2E);
+        for (int c = eset; c < nchunks; c += N_ESET) {
             const int s = c % NS;
             const int valid = min(L, len - c * L);
-            if (!mbar_wait(bar(BAR_ESYNC + (c & 1)), (c >> 1) & 1, abort_flag)) break;
-            float off0 = 0.f, off1 = 0.f;
-            const float* totc = tot + (c % NTOT) * N_EW * 64;
-            for (int qq = 0; qq < tq; ++qq) {
-                const float2 t2 = *reinterpret_cast<const float2*>(totc + qq * 64 + 2 * lane);
-                off0 += t2.x; off1 += t2.y;
-            }
+            const bool tail = valid < L;
+            const uint32_t tx = sbase + OFF_RING + s * STAGE, tr = tx + TILE, tk = tr + TILE, tv = tk + TILE;
             if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) break;
-            // ---- phase B, in place: r -> R^ = r 2^{a_{t-1}}, k -> K^ = k 2^{-a_t}; bonus partials
-            const uint32_t tr = sbase + OFF_RKV + s * 3 * TILE, tk = tr + TILE, tv = tr + 2 * TILE;
-            float du[8];
-            uint32_t rw[8], kw[8];
-#pragma unroll
-            for (int tt = 0; tt < 8; ++tt) {                 // all loads first: they are ordered with the stores below
-                rw[tt] = lds32(tr + swz(8 * tq + tt, cb));
-                kw[tt] = lds32(tk + swz(8 * tq + tt, cb));
-            }
-#pragma unroll
-            for (int tt = 0; tt < 8; ++tt) {
-                const int t = 8 * tq + tt;
-                const float ap0 = off0 + (tt ? l0[tt - 1] : 0.f), ap1 = off1 + (tt ? l1[tt - 1] : 0.f);
-                const float ac0 = off0 + l0[tt], ac1 = off1 + l1[tt];
-                const float r0 = bf_lo(rw[tt]), r1 = bf_hi(rw[tt]), k0 = bf_lo(kw[tt]), k1 = bf_hi(kw[tt]);
-                uint32_t rh = pack_bf16(r0 * ex2(ap0), r1 * ex2(ap1));
-                uint32_t kh = pack_bf16(k0 * ex2(-ac0), k1 * ex2(-ac1));
-                float d = fmaf(r0 * k0, u2.x, r1 * k1 * u2.y);
-                if (t >= valid) { rh = 0u; kh = 0u; d = 0.f; }
-                rw[tt] = rh; kw[tt] = kh;
-                du[tt] = d;
-            }
-#pragma unroll
-            for (int tt = 0; tt < 8; ++tt) {
-                sts32(tr + swz(8 * tq + tt, cb), rw[tt]);
-                sts32(tk + swz(8 * tq + tt, cb), kw[tt]);
-            }
-            // reduce the 8 bonus partials over the 32 lanes (transposing butterfly): lane 4m ends with token m
+            // ---- phase A: log2-decay magnitudes e = exp(x) log2(e), inclusive cumulative sums over this lane's tokens
+            float2 aa[4], ab[4];                         // -(cumulative e): channel pairs (0,1) and (2,3)
             {
-                const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
-                float w4[4], w2[2], w1;
+                uint2 xw[4];
 #pragma unroll
-                for (int m = 0; m < 4; ++m) {
-                    const float send = h16 ? du[m] : du[m + 4], keep = h16 ? du[m + 4] : du[m];
-                    w4[m] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                for (int tt = 0; tt < 4; ++tt) xw[tt] = lds64(tx + roff[tt]);
+                float2 ra = make_float2(0.f, 0.f), rb = ra;
+#pragma unroll
+                for (int tt = 0; tt < 4; ++tt) {
+                    float2 ea = ex2_2(fma2(bf_pair(xw[tt].x), kLog2e, kLogLog));
+                    float2 eb = ex2_2(fma2(bf_pair(xw[tt].y), kLog2e, kLogLog));
+                    if (tail && 8 * tq + 4 * th + tt >= valid) { ea = make_float2(0.f, 0.f); eb = ea; }
+                    ra = sub2(ra, ea); rb = sub2(rb, eb);
+                    aa[tt] = ra; ab[tt] = rb;
                 }
+            }
+            // the other half-warp's total: lanes th = 1 start after it, lanes th = 0 add it to form the warp's total
+            float2 oa, ob;
+            oa.x = __shfl_xor_sync(0xffffffffu, aa[3].x, 16); oa.y = __shfl_xor_sync(0xffffffffu, aa[3].y, 16);
+            ob.x = __shfl_xor_sync(0xffffffffu, ab[3].x, 16); ob.y = __shfl_xor_sync(0xffffffffu, ab[3].y, 16);
+            float* totc = tot + (c % NTOT) * N_EW * 64;
+            if (th == 0) {
+                const float2 wa = add2(aa[3], oa), wb = add2(ab[3], ob);
+                *reinterpret_cast<float4*>(totc + tq * 64 + 4 * cq) = make_float4(wa.x, wa.y, wb.x, wb.y);
+                oa = make_float2(0.f, 0.f); ob = oa;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_ESYNC + eset));
+            if (!mbar_wait(bar(BAR_ESYNC + eset), (c >> 1) & 1, abort_flag)) break;
+            for (int qq = 0; qq < tq; ++qq) {            // cumulative sum at the end of the warps before this one
+                const float4 t4 = *reinterpret_cast<const float4*>(totc + qq * 64 + 4 * cq);
+                oa = add2(oa, make_float2(t4.x, t4.y)); ob = add2(ob, make_float2(t4.z, t4.w));
+            }
+            // ---- phase B, in place: r -> R^ = r 2^{a_{t-1}}, k -> K^ = k 2^{-a_t}; bonus partials
+            uint2 rw[4], kw[4];
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {             // all loads first: they are ordered with the stores below
+                rw[tt] = lds64(tr + roff[tt]);
+                kw[tt] = lds64(tk + roff[tt]);
+            }
+            float du[4];
+            float2 pa = oa, pb = ob;                     // a_{t-1}
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                const float2 ca = add2(oa, aa[tt]), cb = add2(ob, ab[tt]);     // a_t
+                const float2 sra = ex2_2(pa), srb = ex2_2(pb);
+                const float2 ska = ex2_2(make_float2(-ca.x, -ca.y)), skb = ex2_2(make_float2(-cb.x, -cb.y));
+                const float2 r0 = bf_pair(rw[tt].x), r1 = bf_pair(rw[tt].y), k0 = bf_pair(kw[tt].x), k1 = bf_pair(kw[tt].y);
+                const float2 rh0 = mul2(r0, sra), rh1 = mul2(r1, srb), kh0 = mul2(k0, ska), kh1 = mul2(k1, skb);
+                const float2 acc = fma2(mul2(r1, k1), ub, mul2(mul2(r0, k0), ua));
+                rw[tt] = make_uint2(pack_bf16(rh0.x, rh0.y), pack_bf16(rh1.x, rh1.y));
+                kw[tt] = make_uint2(pack_bf16(kh0.x, kh0.y), pack_bf16(kh1.x, kh1.y));
+                du[tt] = acc.x + acc.y;
+                if (tail && 8 * tq + 4 * th + tt >= valid) { rw[tt] = make_uint2(0u, 0u); kw[tt] = rw[tt]; du[tt] = 0.f; }
+                pa = ca; pb = cb;
+            }
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                sts64(tr + roff[tt], rw[tt]);
+                sts64(tk + roff[tt], kw[tt]);
+            }
+            // reduce the 4 bonus partials over the 16 lanes of a half-warp (transposing butterfly):
+            // lanes with bits (3,2) = (b8, b4) end with token 2*b8 + b4
+            {
+                const bool b8 = lane & 8, b4 = lane & 4;
+                float w2[2], w1;
 #pragma unroll
                 for (int m = 0; m < 2; ++m) {
-                    const float send = h8 ? w4[m] : w4[m + 2], keep = h8 ? w4[m + 2] : w4[m];
+                    const float send = b8 ? du[m] : du[m + 2], keep = b8 ? du[m + 2] : du[m];
                     w2[m] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
                 }
                 {
-                    const float send = h4 ? w2[0] : w2[1], keep = h4 ? w2[1] : w2[0];
+                    const float send = b4 ? w2[0] : w2[1], keep = b4 ? w2[1] : w2[0];
                     w1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
                 }
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 2);
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
                 if ((lane & 3) == 0)
-                    reinterpret_cast<float*>(smem + OFF_DU)[s * 64 + 8 * tq + (lane >> 2)] = w1;
+                    reinterpret_cast<float*>(smem + OFF_DU)[s * 64 + 8 * tq + 4 * th + 2 * (b8 ? 1 : 0) + (b4 ? 1 : 0)] = w1;
             }
             if (tq == N_EW - 1) {
-                const float aL0 = off0 + l0[7], aL1 = off1 + l1[7];
-                *reinterpret_cast<float2*>(reinterpret_cast<float*>(smem + OFF_DL) + s * 64 + 2 * lane) =
-                    make_float2(ex2(aL0), ex2(aL1));
-                const bool ok = (aL0 >= -A2_MAX) && (aL1 >= -A2_MAX);       // false for NaN as well
+                // pa, pb now hold a_L on the lanes that own the chunk's last tokens (th = 1)
+                bool ok = true;
+                if (th == 1) {
+                    const float2 da = ex2_2(pa), db = ex2_2(pb);
+                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(smem + OFF_DL) + s * 64 + 4 * cq) =
+                        make_float4(da.x, da.y, db.x, db.y);
+                    ok = (pa.x >= -A2_MAX) && (pa.y >= -A2_MAX) && (pb.x >= -A2_MAX) && (pb.y >= -A2_MAX);   // false for NaN as well
+                }
                 const bool all_ok = __all_sync(0xffffffffu, ok);
                 if (lane == 0) safe_flag[s] = all_ok ? 1 : 0;
             }
-            if (valid < L) {
+            if (tail) {
                 // v rows past the end of the sequence hold another sequence's tokens (or fill): zero them
                 for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
                     sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
@@ -791,8 +911,6 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             fence_proxy_async();                  // the scaled tiles are read by the tensor core (async proxy)
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_RK_READY + s));
-#pragma unroll
-            for (int tt = 0; tt < 8; ++tt) { l0[tt] = n0[tt]; l1[tt] = n1[tt]; }
         }
     }
 
