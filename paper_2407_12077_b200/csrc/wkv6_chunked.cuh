@@ -16,15 +16,15 @@
 // violates it is processed token by token in fp32 instead, so any finite or infinite decay
 // logit gives the exact-recurrence result.
 //
-// Warp roles (960 threads), pipelined across chunks through mbarriers:
+// Warp roles (992 threads), pipelined across chunks through mbarriers:
 //   warp 0        TMA producer: {x,r,k,v} tiles of a chunk into one stage of a 5-stage ring
-//   warp 1        tensor-memory allocation; one lane issues every tcgen05.mma:
-//                   P = R^ K^^T, dS = K^^T V (one chunk ahead) interleaved with Y0 = R^ S_0, PV = P' V
-//   warps 2-5     state: S <- diag(2^{a_L}) (S + dS) in fp32 registers for the whole sequence;
+//   warp 1        tensor-memory allocation; an elected lane issues P = R^ K^^T and dS = K^^T V
+//   warp 2        an elected lane issues Y0 = R^ S_0 and PV = P' V
+//   warps 3-6     state: S <- diag(2^{a_L}) (S + dS) in fp32 registers for the whole sequence;
 //                 publishes a bf16 copy of every chunk-start state as an MMA operand
-//   warps 6-9     scores: P from tensor memory -> P' = tril(P,-1) + diag(bonus) -> bf16 operand tile
-//   warps 10-13   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows)
-//   warps 14-29   elementwise, two sets of eight warps taking alternate chunks: decay and
+//   warps 7-10    scores: P from tensor memory -> P' = tril(P,-1) + diag(bonus) -> bf16 operand tile
+//   warps 11-14   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows)
+//   warps 15-30   elementwise, two sets of eight warps taking alternate chunks: decay and
 //                 cumulative sum (phase A), then in place R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t}
 //                 (phase B); chunk decay 2^{a_L}, bonus coefficients, safety vote.  A lane owns
 //                 4 tokens x 4 channels (64-bit shared-memory accesses, packed fp32x2 arithmetic)
@@ -60,14 +60,15 @@ namespace ck {
 constexpr int L = 64;                  // tokens per chunk
 constexpr int TILE = 64 * 64 * 2;      // one bf16 [64 x 64] tile
 constexpr int NS = 5;                  // {x,r,k,v} ring depth
-constexpr int NSB = 2;                 // bf16 chunk-start state operand tiles
-constexpr int NPP = 2;                 // bf16 masked-score operand tiles
+constexpr int NSB = 2;                 // bf16 chunk-start state operand tiles (by chunk parity)
+constexpr int NPP = 2;                 // bf16 masked-score operand tiles (by chunk parity)
 constexpr int NTOT = 4;                // per-warp decay-total buffers (two per elementwise set)
 constexpr int N_EW = 8;                // elementwise warps per set
 constexpr int N_ESET = 2;              // elementwise sets (alternate chunks)
 constexpr int N_GW = 4;                // warps per tensor-memory reader group (one per sub-partition)
-constexpr int WARP_MMA = 1;
-constexpr int WARP_S0 = 2;             // state warps
+constexpr int WARP_MMA_F = 1;          // issues P = R^ K^^T and dS = K^^T V; owns the tensor-memory allocation
+constexpr int WARP_MMA_B = 2;          // issues Y0 = R^ S_0 and PV = P' V
+constexpr int WARP_S0 = 3;             // state warps
 constexpr int WARP_P0 = WARP_S0 + N_GW;   // score warps
 constexpr int WARP_Y0 = WARP_P0 + N_GW;   // output warps
 constexpr int WARP_E0 = WARP_Y0 + N_GW;   // elementwise warps
@@ -99,16 +100,12 @@ enum {
     BAR_FULL_RKV = 0,
     BAR_EMPTY_RKV = BAR_FULL_RKV + NS,
     BAR_RK_READY = BAR_EMPTY_RKV + NS,
-    BAR_S_READY = BAR_RK_READY + NS,
-    BAR_S_FREE = BAR_S_READY + NSB,
-    BAR_PP_READY = BAR_S_FREE + NSB,
-    BAR_PP_FREE = BAR_PP_READY + NPP,
-    BAR_P_FULL = BAR_PP_FREE + NPP,      // tensor-memory buffers: two each
-    BAR_P_EMPTY = BAR_P_FULL + 2,
-    BAR_DS_FULL = BAR_P_EMPTY + 2,
-    BAR_DS_EMPTY = BAR_DS_FULL + 2,
-    BAR_Y_FULL = BAR_DS_EMPTY + 2,
-    BAR_Y_EMPTY = BAR_Y_FULL + 2,
+    BAR_S_READY = BAR_RK_READY + NS,     // bf16 state operand tile written            (by chunk parity)
+    BAR_PP_READY = BAR_S_READY + 2,      // masked-score operand tile written
+    BAR_F_FULL = BAR_PP_READY + 2,       // P and dS accumulators complete
+    BAR_F_EMPTY = BAR_F_FULL + 2,        // ... and read back by the state and score warps
+    BAR_B_DONE = BAR_F_EMPTY + 2,        // Y0 and PV accumulators complete; state / score operand tiles free again
+    BAR_Y_EMPTY = BAR_B_DONE + 2,        // ... and read back by the output warps
     BAR_ESYNC = BAR_Y_EMPTY + 2,         // one per elementwise set
     BAR_SSYNC = BAR_ESYNC + 2,           // state-warp rendezvous (token-by-token path only)
     BAR_COUNT = BAR_SSYNC + 1
@@ -440,12 +437,13 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             mbar_init(bar(BAR_EMPTY_RKV + i), 1 + 3 * N_GW);       // MMA commit + state, score and output warps
             mbar_init(bar(BAR_RK_READY + i), N_EW);
         }
-        for (int i = 0; i < NSB; ++i) { mbar_init(bar(BAR_S_READY + i), N_GW); mbar_init(bar(BAR_S_FREE + i), 1); }
-        for (int i = 0; i < NPP; ++i) { mbar_init(bar(BAR_PP_READY + i), N_GW); mbar_init(bar(BAR_PP_FREE + i), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(BAR_P_FULL + i), 1);  mbar_init(bar(BAR_P_EMPTY + i), N_GW);
-            mbar_init(bar(BAR_DS_FULL + i), 1); mbar_init(bar(BAR_DS_EMPTY + i), N_GW);
-            mbar_init(bar(BAR_Y_FULL + i), 1);  mbar_init(bar(BAR_Y_EMPTY + i), N_GW);
+            mbar_init(bar(BAR_S_READY + i), N_GW);
+            mbar_init(bar(BAR_PP_READY + i), N_GW);
+            mbar_init(bar(BAR_F_FULL + i), 1);
+            mbar_init(bar(BAR_F_EMPTY + i), 2 * N_GW);
+            mbar_init(bar(BAR_B_DONE + i), 1);
+            mbar_init(bar(BAR_Y_EMPTY + i), N_GW);
         }
         for (int i = 0; i < N_ESET; ++i) mbar_init(bar(BAR_ESYNC + i), N_EW);
         mbar_init(bar(BAR_SSYNC), N_GW);
@@ -453,7 +451,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (warp == WARP_MMA) tmem_alloc(sbase + OFF_TMEM, TM_COLS);
+    if (warp == WARP_MMA_F) tmem_alloc(sbase + OFF_TMEM, TM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -480,86 +478,62 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // do not leave while copies into this CTA's shared memory may still be in flight
         for (int c = max(0, issued - NS); c < issued; ++c)
             mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
-    } else if (warp == WARP_MMA) {
-        // ============================== MMA issuer ==============================
-        {
-            // One step issues, interleaved so that four independent accumulation chains are in flight,
-            //   P_{c+1} = R^ K^^T, dS_{c+1} = K^^T V      (inputs of chunk c+1 only)
-            //   Y0_c = R^ S_0,  PV_c = P' V               (need the chunk-start state and the masked scores)
-            // Consecutive tcgen05.mma on one accumulator wait for each other; different ones pipeline.
-            auto wait_front = [&](int c) -> bool {
-                const int s = c % NS, tb = c & 1;
-                if (!mbar_wait_warp(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) return false;
-                if (!mbar_wait_warp(bar(BAR_RK_READY + s), (c / NS) & 1, abort_flag)) return false;
-                if (c >= 2) {
-                    if (!mbar_wait_warp(bar(BAR_P_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                    if (!mbar_wait_warp(bar(BAR_DS_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                }
-                return true;
-            };
-            auto wait_back = [&](int c) -> bool {
-                const int tb = c & 1, sbi = c % NSB, ppi = c % NPP;
-                if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), ((c >> 1) & 1) ^ 1, abort_flag)) return false;
-                if (!mbar_wait_warp(bar(BAR_S_READY + sbi), (c / NSB) & 1, abort_flag)) return false;
-                if (!mbar_wait_warp(bar(BAR_PP_READY + ppi), (c / NPP) & 1, abort_flag)) return false;
-                return true;
-            };
-            // c_front = chunk whose P / dS are issued (-1: none), c_back = chunk whose Y0 / PV are issued (-1: none)
-            auto step = [&](int c_front, int c_back) {
-                uint64_t dr_f = 0, dk_f = 0, dv_f = 0, dr_b = 0, ds_b = 0, dp_b = 0, dv_b = 0;
-                bool do_f = false, do_b = false;
-                if (c_front >= 0) {
-                    const int s = c_front % NS;
-                    const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
-                    do_f = safe_flag[s] != 0;
-                    dr_f = smem_desc(tr); dk_f = smem_desc(tr + TILE); dv_f = smem_desc(tr + 2 * TILE);
-                }
-                if (c_back >= 0) {
-                    const int s = c_back % NS;
-                    const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
-                    do_b = safe_flag[s] != 0;
-                    dr_b = smem_desc(tr); dv_b = smem_desc(tr + 2 * TILE);
-                    ds_b = smem_desc(sbase + OFF_SB + (c_back % NSB) * TILE);
-                    dp_b = smem_desc(sbase + OFF_PP + (c_back % NPP) * TILE);
-                }
-                const uint32_t tf = 64 * (c_front & 1), tbk = 64 * (c_back & 1);
-                tc_fence_after();
-                if (elect_one()) {
+    } else if (warp == WARP_MMA_F) {
+        // ============================== MMA issuer, input-only products ==============================
+        // P_c = R^ K^^T (M = t, N = i, K = c: both operands K-major) and dS_c = K^^T V (M = c, N = j,
+        // K = i: both MN-major), interleaved: consecutive tcgen05.mma on one accumulator wait for each
+        // other, different accumulators pipeline.
+        int s = 0, ph = 0;                       // ring stage and its phase bit
+        for (int c = 0; c < nchunks; ++c) {
+            const int tb = c & 1, pt = (c >> 1) & 1;
+            if (!mbar_wait_warp(bar(BAR_RK_READY + s), ph, abort_flag)) break;
+            if (c >= 2 && !mbar_wait_warp(bar(BAR_F_EMPTY + tb), pt ^ 1, abort_flag)) break;
+            const bool safe = safe_flag[s] != 0;
+            const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
+            tc_fence_after();
+            if (elect_one()) {
+                if (safe) {
+                    const uint64_t dr = smem_desc(tr), dk = smem_desc(tr + TILE), dv = smem_desc(tr + 2 * TILE);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    if (do_f) {
-                        // M = t, N = i, K = c: both operands K-major;  M = c, N = j, K = i: both MN-major
-                        tc_mma(tmem + TM_P + tf, dr_f + (uint64_t)(2 * kk), dk_f + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
-                        tc_mma(tmem + TM_DS + tf, dk_f + (uint64_t)(128 * kk), dv_f + (uint64_t)(128 * kk), IDESC_MN_MN, kk > 0);
-                    }
-                    if (do_b) {
-                        // M = t, N = j, K = c and M = t, N = j, K = i: A K-major, B MN-major
-                        tc_mma(tmem + TM_Y0 + tbk, dr_b + (uint64_t)(2 * kk), ds_b + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
-                        tc_mma(tmem + TM_PV + tbk, dp_b + (uint64_t)(2 * kk), dv_b + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        tc_mma(tmem + TM_P + 64 * tb, dr + (uint64_t)(2 * kk), dk + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
+                        tc_mma(tmem + TM_DS + 64 * tb, dk + (uint64_t)(128 * kk), dv + (uint64_t)(128 * kk), IDESC_MN_MN, kk > 0);
                     }
                 }
-                if (c_front >= 0) {
-                    tc_commit(bar(BAR_P_FULL + (c_front & 1)));
-                    tc_commit(bar(BAR_DS_FULL + (c_front & 1)));
-                }
-                if (c_back >= 0) {
-                    tc_commit(bar(BAR_S_FREE + c_back % NSB));
-                    tc_commit(bar(BAR_PP_FREE + c_back % NPP));
-                    tc_commit(bar(BAR_EMPTY_RKV + c_back % NS));
-                    tc_commit(bar(BAR_Y_FULL + (c_back & 1)));
-                }
-                }
-                __syncwarp();
-            };
-            if (nchunks > 0 && wait_front(0)) {
-                step(0, -1);
-                for (int c = 0; c < nchunks; ++c) {
-                    const bool has_next = c + 1 < nchunks;
-                    if (has_next && !wait_front(c + 1)) break;
-                    if (!wait_back(c)) break;
-                    step(has_next ? c + 1 : -1, c);
-                }
+                tc_commit(bar(BAR_F_FULL + tb));
             }
+            __syncwarp();
+            if (++s == NS) { s = 0; ph ^= 1; }
+        }
+    } else if (warp == WARP_MMA_B) {
+        // ============================== MMA issuer, state-dependent products ==============================
+        // Y0_c = R^ S_0 (M = t, N = j, K = c) and PV_c = P' V (M = t, N = j, K = i): A K-major, B MN-major.
+        // The masked scores of chunk c exist only after P_c completed, so every product that reads
+        // ring stage s is complete when these complete: the last commit releases the stage.
+        int s = 0;
+        for (int c = 0; c < nchunks; ++c) {
+            const int tb = c & 1, pt = (c >> 1) & 1;
+            if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), pt ^ 1, abort_flag)) break;
+            if (!mbar_wait_warp(bar(BAR_S_READY + tb), pt, abort_flag)) break;
+            if (!mbar_wait_warp(bar(BAR_PP_READY + tb), pt, abort_flag)) break;
+            const bool safe = safe_flag[s] != 0;
+            const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
+            tc_fence_after();
+            if (elect_one()) {
+                if (safe) {
+                    const uint64_t dr = smem_desc(tr), dv = smem_desc(tr + 2 * TILE);
+                    const uint64_t ds = smem_desc(sbase + OFF_SB + tb * TILE), dp = smem_desc(sbase + OFF_PP + tb * TILE);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        tc_mma(tmem + TM_Y0 + 64 * tb, dr + (uint64_t)(2 * kk), ds + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+                        tc_mma(tmem + TM_PV + 64 * tb, dp + (uint64_t)(2 * kk), dv + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+                    }
+                }
+                tc_commit(bar(BAR_B_DONE + tb));
+                tc_commit(bar(BAR_EMPTY_RKV + s));
+            }
+            __syncwarp();
+            if (++s == NS) s = 0;
         }
     } else if (warp < WARP_P0) {
         // ============================== state warps ==============================
@@ -596,7 +570,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         for (int c = 0; c < nchunks; ++c) {
             const int s = c % NS, tb = c & 1;
             const int valid = min(L, len - c * L);
-            if (!mbar_wait(bar(BAR_DS_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_F_FULL + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             if (safe_flag[s]) {
                 // ---- S <- diag(2^{a_L}) (S + K^^T V)
@@ -610,7 +584,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     if (hf == 1) {
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(BAR_DS_EMPTY + tb));
+                        if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
                     }
 #pragma unroll
                     for (int n = 0; n < 4; ++n) {
@@ -624,7 +598,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // token, on a copy of the state in shared memory where a warp owns 16 value channels for
                 // all 64 key channels.
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_DS_EMPTY + tb));
+                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
                 // The scratch is the x and r tiles of this chunk's ring stage: nothing reads them any more
                 // (the inputs are re-read from global memory here) and the stage is not refilled before
                 // these warps release it.
@@ -675,7 +649,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));           // done with this slot's decay vector and flag
             if (c + 1 < nchunks) {
                 const int nb = (c + 1) % NSB;
-                if (c + 1 >= NSB && !mbar_wait(bar(BAR_S_FREE + nb), (((c + 1) / NSB) & 1) ^ 1, abort_flag)) break;
+                if (c + 1 >= NSB && !mbar_wait(bar(BAR_B_DONE + nb), (((c + 1) / NSB) & 1) ^ 1, abort_flag)) break;
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
                 fence_proxy_async();
                 __syncwarp();
@@ -695,7 +669,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int g = lane >> 2, q = lane & 3;
         for (int c = 0; c < nchunks; ++c) {
             const int s = c % NS, tb = c & 1, ppi = c % NPP;
-            if (!mbar_wait(bar(BAR_P_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_F_FULL + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const bool safe = safe_flag[s] != 0;
             float d_lo = 0.f, d_hi = 0.f;
@@ -705,7 +679,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));           // done with this slot's bonus vector and flag
-            if (c >= NPP && !mbar_wait(bar(BAR_PP_FREE + ppi), ((c / NPP) & 1) ^ 1, abort_flag)) break;
+            if (c >= NPP && !mbar_wait(bar(BAR_B_DONE + ppi), ((c / NPP) & 1) ^ 1, abort_flag)) break;
             if (safe) {
                 const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_P + 64 * tb;
                 const uint32_t tp = sbase + OFF_PP + ppi * TILE;
@@ -716,13 +690,13 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 tmem_ld_16x32(ta + 32, acc);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_P_EMPTY + tb));
+                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
                 mask_scores_sp<1>(sp, acc, g, q, d_lo, d_hi);
                 store_half_bf16<1>(tp, 16 * sp, acc, lane);
                 fence_proxy_async();
             } else {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_P_EMPTY + tb));
+                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_PP_READY + ppi));
@@ -734,7 +708,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         for (int c = 0; c < nchunks; ++c) {
             const int s = c % NS, tb = c & 1;
             const int valid = min(L, len - c * L);
-            if (!mbar_wait(bar(BAR_Y_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_B_DONE + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
             const bool safe = safe_flag[s] != 0;
             __syncwarp();
@@ -917,7 +891,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     // every role is done with tensor memory (or the CTA is aborting): release it
     tc_fence_before();
     __syncthreads();
-    if (warp == WARP_MMA) {
+    if (warp == WARP_MMA_F) {
         tc_fence_after();
         tmem_dealloc(tmem, TM_COLS);
     }
