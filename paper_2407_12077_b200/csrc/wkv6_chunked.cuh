@@ -21,9 +21,11 @@
 //   warp 1        tensor-memory allocation; an elected lane issues P = R^ K^^T and dS = K^^T V
 //   warp 2        an elected lane issues Y0 = R^ S_0 and PV = P' V
 //   warps 3-6     state: S <- diag(2^{a_L}) (S + dS) in fp32 registers for the whole sequence;
-//                 publishes a bf16 copy of every chunk-start state as an MMA operand
+//                 publishes a bf16 copy of every chunk-start state as an MMA operand; for a chunk on
+//                 the token-by-token path it parks the fp32 state in shared memory instead
 //   warps 7-10    scores: P from tensor memory -> P' = tril(P,-1) + diag(bonus) -> bf16 operand tile
-//   warps 11-14   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows)
+//   warps 11-14   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows);
+//                 runs the token-by-token path (16 value channels per warp) when a chunk needs it
 //   warps 15-30   elementwise, two sets of eight warps taking alternate chunks: decay and
 //                 cumulative sum (phase A), then in place R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t}
 //                 (phase B); chunk decay 2^{a_L}, bonus coefficients, safety vote.  A lane owns
@@ -62,6 +64,8 @@ constexpr int TILE = 64 * 64 * 2;      // one bf16 [64 x 64] tile
 constexpr int NS = 5;                  // {x,r,k,v} ring depth
 constexpr int NSB = 2;                 // bf16 chunk-start state operand tiles (by chunk parity)
 constexpr int NPP = 2;                 // bf16 masked-score operand tiles (by chunk parity)
+constexpr int NSIDE = 8;               // ring of per-chunk side vectors (chunk decay, bonus, safety flag): deeper than
+                                       // every consumer's lag behind the elementwise warps, so it needs no release
 constexpr int NTOT = 4;                // per-warp decay-total buffers (two per elementwise set)
 constexpr int N_EW = 8;                // elementwise warps per set
 constexpr int N_ESET = 2;              // elementwise sets (alternate chunks)
@@ -90,10 +94,10 @@ constexpr int OFF_SB = OFF_RING + NS * STAGE;              // [NSB][TILE]       
 constexpr int OFF_PP = OFF_SB + NSB * TILE;                // [NPP][TILE]          bf16 masked scores [t][i]
 constexpr int OFF_Y = OFF_PP + NPP * TILE;                 // [N_GW][16 rows x 128 B] y staging, one slab per warp
 constexpr int OFF_TOT = OFF_Y + N_GW * 2048;               // [NTOT][N_EW][64] float
-constexpr int OFF_DL = OFF_TOT + NTOT * N_EW * 64 * 4;     // [NS][64] float       2^{a_L}
-constexpr int OFF_DU = OFF_DL + NS * 64 * 4;               // [NS][64] float       bonus coefficient per token
-constexpr int OFF_SAFE = OFF_DU + NS * 64 * 4;             // [NS] int (padded)
-constexpr int OFF_ABORT = OFF_SAFE + 32;                   // int
+constexpr int OFF_DL = OFF_TOT + NTOT * N_EW * 64 * 4;     // [NSIDE][64] float    2^{a_L}
+constexpr int OFF_DU = OFF_DL + NSIDE * 64 * 4;            // [NSIDE][64] float    bonus coefficient per token
+constexpr int OFF_SAFE = OFF_DU + NSIDE * 64 * 4;          // [NSIDE] int
+constexpr int OFF_ABORT = OFF_SAFE + NSIDE * 4;            // int
 constexpr int OFF_TMEM = OFF_ABORT + 8;                    // uint32: tensor-memory base address
 constexpr int OFF_BAR = OFF_ABORT + 16;                    // mbarriers (8 bytes each)
 enum {
@@ -107,8 +111,10 @@ enum {
     BAR_B_DONE = BAR_F_EMPTY + 2,        // Y0 and PV accumulators complete; state / score operand tiles free again
     BAR_Y_EMPTY = BAR_B_DONE + 2,        // ... and read back by the output warps
     BAR_ESYNC = BAR_Y_EMPTY + 2,         // one per elementwise set
-    BAR_SSYNC = BAR_ESYNC + 2,           // state-warp rendezvous (token-by-token path only)
-    BAR_COUNT = BAR_SSYNC + 1
+    BAR_SSYNC = BAR_ESYNC + 2,           // token-by-token path only: state-warp rendezvous,
+    BAR_FB_READY = BAR_SSYNC + 1,        //   fp32 state copy in place for the output warps,
+    BAR_FB_DONE = BAR_FB_READY + 1,      //   and advanced by them over the chunk
+    BAR_COUNT = BAR_FB_DONE + 1
 };
 constexpr int SMEM_BYTES = OFF_BAR + BAR_COUNT * 8;
 constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;              // slack for manual 1024-byte alignment
@@ -129,6 +135,30 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ uint32_t lds32(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ float ldsf(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void stsf(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+__device__ __forceinline__ float4 ldsf4(uint32_t a)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void stsf4(uint32_t a, float4 v)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -147,21 +177,22 @@ __device__ __forceinline__ unsigned long long globaltimer()
 }
 // Bounded wait.  Returns false if the CTA is aborting or the wait ran out of time (the
 // status flag is then raised and the CTA-wide abort flag set so every role leaves).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool poll_abort)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag, bool poll_abort)
 {
     const unsigned long long t0 = globaltimer();
     for (;;) {
         for (int it = 0; it < 64; ++it)
             if (mbar_try_wait(bar, parity)) return true;
-        if (poll_abort && *abort_flag) return false;
+        if (poll_abort && lds32(abort_flag)) return false;
         if (globaltimer() - t0 > WAIT_LIMIT_NS) break;
         __nanosleep(64);
     }
-    *abort_flag = 1;
+    sts32(abort_flag, 1u);
     atomicExch(&g_dev_status, 1);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool poll_abort = true)
+// abort_flag: shared-memory address of the CTA-wide abort word
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag, bool poll_abort = true)
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, poll_abort);
@@ -169,7 +200,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // Warp-uniform form: every lane of a converged warp waits and all get the same answer, so the
 // caller's control flow stays uniform (the compiler can then keep addresses in uniform registers).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool poll_abort = true)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, uint32_t abort_flag, bool poll_abort = true)
 {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, poll_abort));
 }
@@ -260,13 +291,24 @@ __device__ __forceinline__ void tmem_ld_16x32(uint32_t taddr, float (&v)[4][4])
         : "r"(taddr) : "memory");
 }
 
+// The same for 16 columns (two 8-column blocks).
+__device__ __forceinline__ void tmem_ld_16x16(uint32_t taddr, float (&v)[2][4])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3])
+        : "r"(taddr) : "memory");
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// packed fp32x2 arithmetic (one instruction for two lanes of a float2)
+// two-lane fp32 arithmetic on float2 values
+#ifndef GF_SCALAR_F32
 __device__ __forceinline__ unsigned long long pk(float2 a)
 {
     unsigned long long r;
@@ -303,6 +345,12 @@ __device__ __forceinline__ float2 sub2(float2 a, float2 b)
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pk(a)), "l"(pk(b)));
     return upk(d);
 }
+#else
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y)); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return make_float2(a.x * b.x, a.y * b.y); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+#endif
 __device__ __forceinline__ float2 ex2_2(float2 a) { return make_float2(ex2(a.x), ex2(a.y)); }
 __device__ __forceinline__ uint2 lds64(uint32_t a)
 {
@@ -371,6 +419,16 @@ __device__ __forceinline__ void store_half_bf16(uint32_t tile, int row0, const f
                 pack_bf16(acc[2 * m + 1][0], acc[2 * m + 1][1]), pack_bf16(acc[2 * m + 1][2], acc[2 * m + 1][3]));
 }
 
+__device__ __forceinline__ void add_acc(float (&a)[4][4], const float (&b)[4][4])
+{
+#pragma unroll
+    for (int n = 0; n < 4; ++n) {
+        const float2 lo = add2(make_float2(a[n][0], a[n][1]), make_float2(b[n][0], b[n][1]));
+        const float2 hi = add2(make_float2(a[n][2], a[n][3]), make_float2(b[n][2], b[n][3]));
+        a[n][0] = lo.x; a[n][1] = lo.y; a[n][2] = hi.x; a[n][3] = hi.y;
+    }
+}
+
 // P' = tril(P, -1) + diag(bonus) on columns 32*HALF .. +31 of one warp's 16 rows (rows 16*SP + g
 // and + 8) of the score block.
 template <int SP, int HALF>
@@ -402,6 +460,41 @@ __device__ __forceinline__ void mask_scores_sp(int sp, float (&acc)[4][4], int g
     }
 }
 
+// Token-by-token fp32 recurrence over `valid` tokens of one chunk for one state warp: the warp owns value
+// channels 16*sp .. 16*sp+15 for all 64 key channels of the fp32 state copy `scr` ([64][64], row = key
+// channel); lane = 16*half + jl works on S[32*half .. +31][16*sp + jl].  Inputs are re-read from global
+// memory and y is written there.  The loops are kept rolled: this is the exceptional path, and unrolling
+// them costs the fast path registers.
+__device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, int sp, int lane, long long first_row,
+                                         int valid, size_t C, int col0)
+{
+    const int half = lane >> 4, j = 16 * sp + (lane & 15);
+    float* scol = scr + (32 * half) * 64 + j;
+    const float* ug = p.u + h * 64 + 32 * half;
+#pragma unroll 1
+    for (int t = 0; t < valid; ++t) {
+        const size_t ro = (size_t)(first_row + t) * C + col0;
+        const float vj = __bfloat162float(p.v[ro + j]);
+        float yj = 0.f, cf = 0.f;
+#pragma unroll 1
+        for (int i = 0; i < 32; i += 2) {
+            const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
+            const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + 32 * half + i);
+            const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + 32 * half + i);
+            const float s0 = scol[i * 64], s1 = scol[(i + 1) * 64];
+            cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
+            cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
+            yj = fmaf(bf_lo(rw), s0, yj);
+            yj = fmaf(bf_hi(rw), s1, yj);
+            scol[i * 64] = fmaf(expf(-expf(bf_lo(xw))), s0, bf_lo(kw) * vj);
+            scol[(i + 1) * 64] = fmaf(expf(-expf(bf_hi(xw))), s1, bf_hi(kw) * vj);
+        }
+        yj += __shfl_xor_sync(0xffffffffu, yj, 16);
+        cf += __shfl_xor_sync(0xffffffffu, cf, 16);
+        if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
+    }
+}
+
 // ---------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
@@ -411,8 +504,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_ABORT);
-    volatile int* safe_flag = reinterpret_cast<volatile int*>(smem + OFF_SAFE);
+    const uint32_t abort_flag = sbase + OFF_ABORT;           // shared addresses of the abort word and the safety flags
+    auto safe_at = [&](int sd) { return lds32(sbase + OFF_SAFE + 4 * sd) != 0; };
     auto bar = [&](int i) { return sbase + OFF_BAR + 8 * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -434,7 +527,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     if (tid == 0) {
         for (int i = 0; i < NS; ++i) {
             mbar_init(bar(BAR_FULL_RKV + i), 1);
-            mbar_init(bar(BAR_EMPTY_RKV + i), 1 + 3 * N_GW);       // MMA commit + state, score and output warps
+            mbar_init(bar(BAR_EMPTY_RKV + i), 1);                  // the commit after the last product that reads the stage
             mbar_init(bar(BAR_RK_READY + i), N_EW);
         }
         for (int i = 0; i < 2; ++i) {
@@ -447,7 +540,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         for (int i = 0; i < N_ESET; ++i) mbar_init(bar(BAR_ESYNC + i), N_EW);
         mbar_init(bar(BAR_SSYNC), N_GW);
-        *abort_flag = 0;
+        mbar_init(bar(BAR_FB_READY), N_GW);
+        mbar_init(bar(BAR_FB_DONE), N_GW);
+        sts32(abort_flag, 0u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -455,15 +550,15 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_TMEM);
+    const uint32_t tmem = lds32(sbase + OFF_TMEM);
 
     if (warp == 0) {
         // ============================== TMA producer ==============================
         int issued = 0;
-        for (int c = 0; c < nchunks; ++c) {
-            const int s = c % NS;
-            if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ((c / NS) & 1) ^ 1, abort_flag)) break;
-            const int row = (int)(row0 + (long long)c * L);
+        int s = 0, ph = 1;                       // ring stage and the parity of its previous release
+        int row = (int)row0;
+        for (int c = 0; c < nchunks; ++c, row += L) {
+            if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) break;
             const uint32_t dst = sbase + OFF_RING + s * STAGE;
             if (elect_one()) {
                 mbar_expect_tx(bar(BAR_FULL_RKV + s), STAGE);
@@ -474,6 +569,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             __syncwarp();
             issued = c + 1;
+            if (++s == NS) { s = 0; ph ^= 1; }
         }
         // do not leave while copies into this CTA's shared memory may still be in flight
         for (int c = max(0, issued - NS); c < issued; ++c)
@@ -488,7 +584,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             const int tb = c & 1, pt = (c >> 1) & 1;
             if (!mbar_wait_warp(bar(BAR_RK_READY + s), ph, abort_flag)) break;
             if (c >= 2 && !mbar_wait_warp(bar(BAR_F_EMPTY + tb), pt ^ 1, abort_flag)) break;
-            const bool safe = safe_flag[s] != 0;
+            const bool safe = safe_at(c & (NSIDE - 1));
             const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
             tc_fence_after();
             if (elect_one()) {
@@ -516,7 +612,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), pt ^ 1, abort_flag)) break;
             if (!mbar_wait_warp(bar(BAR_S_READY + tb), pt, abort_flag)) break;
             if (!mbar_wait_warp(bar(BAR_PP_READY + tb), pt, abort_flag)) break;
-            const bool safe = safe_flag[s] != 0;
+            const bool safe = safe_at(c & (NSIDE - 1));
             const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
             tc_fence_after();
             if (elect_one()) {
@@ -553,14 +649,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
             }
         }
-        int ssync_uses = 0;
-        auto ssync = [&]() -> bool {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_SSYNC));
-            const bool ok = mbar_wait(bar(BAR_SSYNC), ssync_uses & 1, abort_flag);
-            ++ssync_uses;
-            return ok;
-        };
+        int fb_uses = 0;                         // chunks that took the token-by-token path so far
         if (nchunks > 0) {
             store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
             fence_proxy_async();
@@ -568,95 +657,73 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (lane == 0) mbar_arrive(bar(BAR_S_READY));
         }
         for (int c = 0; c < nchunks; ++c) {
-            const int s = c % NS, tb = c & 1;
-            const int valid = min(L, len - c * L);
-            if (!mbar_wait(bar(BAR_F_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+            const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
+            if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
-            if (safe_flag[s]) {
+            bool next_tile_free = c == 0;        // the products of chunk c-1 have finished reading operand tile tb^1
+            if (safe_at(sd)) {
                 // ---- S <- diag(2^{a_L}) (S + K^^T V)
-                const float* dl = reinterpret_cast<const float*>(smem + OFF_DL) + s * 64;
-                const float d_lo = dl[c_lo], d_hi = dl[c_lo + 8];
+                const uint32_t dl = sbase + OFF_DL + 4 * (sd * 64 + c_lo);
+                const float d_lo = ldsf(dl), d_hi = ldsf(dl + 32);
+                const float2 dlo2 = make_float2(d_lo, d_lo), dhi2 = make_float2(d_hi, d_hi);
                 const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_DS + 64 * tb;
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    float d[4][4];
-                    tmem_ld_16x32(ta + 32 * hf, d);
-                    if (hf == 1) {
+                for (int qt = 0; qt < 4; ++qt) {
+                    float d[2][4];
+                    tmem_ld_16x16(ta + 16 * qt, d);
+                    if (qt == 3) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
                     }
 #pragma unroll
-                    for (int n = 0; n < 4; ++n) {
-                        float (&sn)[4] = st[4 * hf + n];
-                        sn[0] = (sn[0] + d[n][0]) * d_lo; sn[1] = (sn[1] + d[n][1]) * d_lo;
-                        sn[2] = (sn[2] + d[n][2]) * d_hi; sn[3] = (sn[3] + d[n][3]) * d_hi;
+                    for (int n = 0; n < 2; ++n) {
+                        float (&sn)[4] = st[2 * qt + n];
+                        const float2 a = mul2(add2(make_float2(sn[0], sn[1]), make_float2(d[n][0], d[n][1])), dlo2);
+                        const float2 b = mul2(add2(make_float2(sn[2], sn[3]), make_float2(d[n][2], d[n][3])), dhi2);
+                        sn[0] = a.x; sn[1] = a.y; sn[2] = b.x; sn[3] = b.y;
                     }
                 }
             } else {
-                // ---- decay too strong for one in-chunk reference point: exact fp32 recurrence, token by
-                // token, on a copy of the state in shared memory where a warp owns 16 value channels for
-                // all 64 key channels.
+                // ---- decay too strong for one in-chunk reference point: the output warps run the exact fp32
+                // recurrence over this chunk, token by token, on a copy of the state in shared memory.
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
-                // The scratch is the x and r tiles of this chunk's ring stage: nothing reads them any more
-                // (the inputs are re-read from global memory here) and the stage is not refilled before
-                // these warps release it.
-                float* scr = reinterpret_cast<float*>(smem + OFF_RING + s * STAGE);
+                // The copy lives in the pair of bf16 state operand tiles: this chunk's tile has no reader (its
+                // products are skipped) and the other one is free once the products of chunk c-1 are done.
+                if (c >= 1 && !mbar_wait(bar(BAR_B_DONE + (tb ^ 1)), ((c - 1) >> 1) & 1, abort_flag)) break;
+                next_tile_free = true;
+                float* scr = reinterpret_cast<float*>(smem + OFF_SB);
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     *reinterpret_cast<float2*>(scr + c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
                     *reinterpret_cast<float2*>(scr + (c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
                 }
-                if (!ssync()) break;
-                {
-                    // lane = 16*half + jl works on S[32*half .. +31][16*sp + jl], kept in the fp32 scratch
-                    const int half = lane >> 4, j = 16 * sp + (lane & 15);
-                    float* scol = scr + (32 * half) * 64 + j;
-                    const float* ug = p.u + h * 64 + 32 * half;
-                    for (int t = 0; t < valid; ++t) {
-                        const size_t ro = (size_t)(row0 + (long long)c * L + t) * C + col0;
-                        const float vj = __bfloat162float(p.v[ro + j]);
-                        float yj = 0.f, cf = 0.f;
-#pragma unroll 4
-                        for (int i = 0; i < 32; i += 2) {
-                            const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
-                            const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + 32 * half + i);
-                            const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + 32 * half + i);
-                            const float s0 = scol[i * 64], s1 = scol[(i + 1) * 64];
-                            cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
-                            cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
-                            yj = fmaf(bf_lo(rw), s0, yj);
-                            yj = fmaf(bf_hi(rw), s1, yj);
-                            scol[i * 64] = fmaf(expf(-expf(bf_lo(xw))), s0, bf_lo(kw) * vj);
-                            scol[(i + 1) * 64] = fmaf(expf(-expf(bf_hi(xw))), s1, bf_hi(kw) * vj);
-                        }
-                        yj += __shfl_xor_sync(0xffffffffu, yj, 16);
-                        cf += __shfl_xor_sync(0xffffffffu, cf, 16);
-                        if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
-                    }
-                }
-                if (!ssync()) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_FB_READY));
+                if (!mbar_wait(bar(BAR_FB_DONE), fb_uses & 1, abort_flag)) break;
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     const float2 lo = *reinterpret_cast<const float2*>(scr + c_lo * 64 + 8 * n + 2 * q);
                     const float2 hi = *reinterpret_cast<const float2*>(scr + (c_lo + 8) * 64 + 8 * n + 2 * q);
                     st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
                 }
-                if (!ssync()) break;          // everyone has re-read the scratch before it can be rewritten
+                // every state warp has re-read the copy before the operand tiles are rewritten
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_SSYNC));
+                if (!mbar_wait(bar(BAR_SSYNC), fb_uses & 1, abort_flag)) break;
+                ++fb_uses;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));           // done with this slot's decay vector and flag
             if (c + 1 < nchunks) {
-                const int nb = (c + 1) % NSB;
-                if (c + 1 >= NSB && !mbar_wait(bar(BAR_B_DONE + nb), (((c + 1) / NSB) & 1) ^ 1, abort_flag)) break;
+                const int nb = tb ^ 1;
+                if (!next_tile_free && !mbar_wait(bar(BAR_B_DONE + nb), ((c - 1) >> 1) & 1, abort_flag)) break;
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_S_READY + nb));
             }
         }
-        if (p.state_out && !*abort_flag) {
+        if (p.state_out && !lds32(abort_flag)) {
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
                 *reinterpret_cast<float2*>(p.state_out + sb + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
@@ -668,18 +735,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int sp = warp & 3;                 // rows t = 16*sp .. 16*sp+15 of the score block
         const int g = lane >> 2, q = lane & 3;
         for (int c = 0; c < nchunks; ++c) {
-            const int s = c % NS, tb = c & 1, ppi = c % NPP;
-            if (!mbar_wait(bar(BAR_F_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+            const int tb = c & 1, pt = (c >> 1) & 1, ppi = tb, sd = c & (NSIDE - 1);
+            if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
-            const bool safe = safe_flag[s] != 0;
+            const bool safe = safe_at(sd);
             float d_lo = 0.f, d_hi = 0.f;
             if (safe) {
-                const float* du = reinterpret_cast<const float*>(smem + OFF_DU) + s * 64;
-                d_lo = du[16 * sp + g]; d_hi = du[16 * sp + g + 8];
+                const uint32_t du = sbase + OFF_DU + 4 * (sd * 64 + 16 * sp + g);
+                d_lo = ldsf(du); d_hi = ldsf(du + 32);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_EMPTY_RKV + s));           // done with this slot's bonus vector and flag
-            if (c >= NPP && !mbar_wait(bar(BAR_B_DONE + ppi), ((c / NPP) & 1) ^ 1, abort_flag)) break;
+            if (c >= NPP && !mbar_wait(bar(BAR_B_DONE + ppi), pt ^ 1, abort_flag)) break;
             if (safe) {
                 const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_P + 64 * tb;
                 const uint32_t tp = sbase + OFF_PP + ppi * TILE;
@@ -705,20 +770,24 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // ============================== output warps ==============================
         const int sp = warp & 3;                 // rows t = 16*sp .. 16*sp+15 of the chunk
         const uint32_t slab = sbase + OFF_Y + sp * 2048;
+        int fb_uses = 0;                         // chunks that took the token-by-token path so far
         for (int c = 0; c < nchunks; ++c) {
-            const int s = c % NS, tb = c & 1;
-            const int valid = min(L, len - c * L);
+            const int tb = c & 1;
             if (!mbar_wait(bar(BAR_B_DONE + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
-            const bool safe = safe_flag[s] != 0;
+            const bool safe = safe_at(c & (NSIDE - 1));
+            if (lane == 0) bulk_wait_read<0>();   // this warp's previous store has finished reading the slab
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar(BAR_EMPTY_RKV + s));                      // done with this slot's flag
-                bulk_wait_read<0>();              // this warp's previous store has finished reading the slab
-            }
-            __syncwarp();
-            if (!safe) {                          // the state warps wrote this chunk's y themselves
+            if (!safe) {
+                // decay too strong for the tensor-core formulation: exact recurrence on the fp32 state copy
+                // the state warps put in shared memory; writes this chunk's y rows itself
                 if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
+                if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
+                exact_chunk(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
+                            min(L, len - c * L), C, col0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_FB_DONE));
+                ++fb_uses;
                 continue;
             }
             // ---- this warp's 16 rows of y -> bf16 slab -> global
@@ -728,25 +797,19 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 float ya[4][4], yb[4][4];
                 tmem_ld_16x32(ta, ya);
                 tmem_ld_16x32(tc, yb);
-#pragma unroll
-                for (int n = 0; n < 4; ++n)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) ya[n][e] += yb[n][e];
+                add_acc(ya, yb);
                 store_half_bf16<0>(slab, 0, ya, lane);
                 tmem_ld_16x32(ta + 32, ya);
                 tmem_ld_16x32(tc + 32, yb);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
-#pragma unroll
-                for (int n = 0; n < 4; ++n)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) ya[n][e] += yb[n][e];
+                add_acc(ya, yb);
                 store_half_bf16<1>(slab, 0, ya, lane);
             }
             fence_proxy_async();
             __syncwarp();
-            const int rows = valid - 16 * sp;
+            const int rows = min(L, len - c * L) - 16 * sp;
             const long long grow = row0 + (long long)c * L + 16 * sp;
             if (rows >= 16) {
                 if (lane == 0) {
@@ -774,17 +837,30 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
         const float4 u4 = *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
         const float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
-        float* tot = reinterpret_cast<float*>(smem + OFF_TOT);
         uint32_t roff[4];                                // swizzled byte offsets of this lane's 8 bytes in its 4 rows
 #pragma unroll
         for (int tt = 0; tt < 4; ++tt) roff[tt] = swz(8 * tq + 4 * th + tt, 8 * cq);
         const float2 kLog2e = make_float2(LOG2E, LOG2E), kLogLog = make_float2(LOG2_LOG2E, LOG2_LOG2E);
+        int s = eset, ph = 0;                            // ring stage of this set's current chunk and its phase bit
         for (int c = eset; c < nchunks; c += N_ESET) {
-            const int s = c % NS;
-            const int valid = min(L, len - c * L);
-            const bool tail = valid < L;
+            const int sd = c & (NSIDE - 1);
             const uint32_t tx = sbase + OFF_RING + s * STAGE, tr = tx + TILE, tk = tr + TILE, tv = tk + TILE;
-            if (!mbar_wait(bar(BAR_FULL_RKV + s), (c / NS) & 1, abort_flag)) break;
+            if (!mbar_wait(bar(BAR_FULL_RKV + s), ph, abort_flag)) break;
+            if (len - c * L < L) {
+                // Ragged last chunk: rows past the end of the sequence hold another sequence's tokens (or the
+                // out-of-range fill).  Each lane rewrites its own part of those rows before it reads them
+                // back: x = -inf (no decay), r = k = 0; the v rows are zeroed for the tensor core.
+                const int valid = len - c * L;
+#pragma unroll
+                for (int tt = 0; tt < 4; ++tt)
+                    if (8 * tq + 4 * th + tt >= valid) {
+                        sts64(tx + roff[tt], make_uint2(0xff80ff80u, 0xff80ff80u));
+                        sts64(tr + roff[tt], make_uint2(0u, 0u));
+                        sts64(tk + roff[tt], make_uint2(0u, 0u));
+                    }
+                for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
+                    sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
+            }
             // ---- phase A: log2-decay magnitudes e = exp(x) log2(e), inclusive cumulative sums over this lane's tokens
             float2 aa[4], ab[4];                         // -(cumulative e): channel pairs (0,1) and (2,3)
             {
@@ -794,9 +870,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 float2 ra = make_float2(0.f, 0.f), rb = ra;
 #pragma unroll
                 for (int tt = 0; tt < 4; ++tt) {
-                    float2 ea = ex2_2(fma2(bf_pair(xw[tt].x), kLog2e, kLogLog));
-                    float2 eb = ex2_2(fma2(bf_pair(xw[tt].y), kLog2e, kLogLog));
-                    if (tail && 8 * tq + 4 * th + tt >= valid) { ea = make_float2(0.f, 0.f); eb = ea; }
+                    const float2 ea = ex2_2(fma2(bf_pair(xw[tt].x), kLog2e, kLogLog));
+                    const float2 eb = ex2_2(fma2(bf_pair(xw[tt].y), kLog2e, kLogLog));
                     ra = sub2(ra, ea); rb = sub2(rb, eb);
                     aa[tt] = ra; ab[tt] = rb;
                 }
@@ -805,17 +880,17 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             float2 oa, ob;
             oa.x = __shfl_xor_sync(0xffffffffu, aa[3].x, 16); oa.y = __shfl_xor_sync(0xffffffffu, aa[3].y, 16);
             ob.x = __shfl_xor_sync(0xffffffffu, ab[3].x, 16); ob.y = __shfl_xor_sync(0xffffffffu, ab[3].y, 16);
-            float* totc = tot + (c % NTOT) * N_EW * 64;
+            const uint32_t totc = sbase + OFF_TOT + 4 * ((c % NTOT) * N_EW * 64 + 4 * cq);
             if (th == 0) {
                 const float2 wa = add2(aa[3], oa), wb = add2(ab[3], ob);
-                *reinterpret_cast<float4*>(totc + tq * 64 + 4 * cq) = make_float4(wa.x, wa.y, wb.x, wb.y);
+                stsf4(totc + 256 * tq, make_float4(wa.x, wa.y, wb.x, wb.y));
                 oa = make_float2(0.f, 0.f); ob = oa;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_ESYNC + eset));
             if (!mbar_wait(bar(BAR_ESYNC + eset), (c >> 1) & 1, abort_flag)) break;
             for (int qq = 0; qq < tq; ++qq) {            // cumulative sum at the end of the warps before this one
-                const float4 t4 = *reinterpret_cast<const float4*>(totc + qq * 64 + 4 * cq);
+                const float4 t4 = ldsf4(totc + 256 * qq);
                 oa = add2(oa, make_float2(t4.x, t4.y)); ob = add2(ob, make_float2(t4.z, t4.w));
             }
             // ---- phase B, in place: r -> R^ = r 2^{a_{t-1}}, k -> K^ = k 2^{-a_t}; bonus partials
@@ -838,7 +913,6 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 rw[tt] = make_uint2(pack_bf16(rh0.x, rh0.y), pack_bf16(rh1.x, rh1.y));
                 kw[tt] = make_uint2(pack_bf16(kh0.x, kh0.y), pack_bf16(kh1.x, kh1.y));
                 du[tt] = acc.x + acc.y;
-                if (tail && 8 * tq + 4 * th + tt >= valid) { rw[tt] = make_uint2(0u, 0u); kw[tt] = rw[tt]; du[tt] = 0.f; }
                 pa = ca; pb = cb;
             }
 #pragma unroll
@@ -863,28 +937,24 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 2);
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
                 if ((lane & 3) == 0)
-                    reinterpret_cast<float*>(smem + OFF_DU)[s * 64 + 8 * tq + 4 * th + 2 * (b8 ? 1 : 0) + (b4 ? 1 : 0)] = w1;
+                    stsf(sbase + OFF_DU + 4 * (sd * 64 + 8 * tq + 4 * th + 2 * (b8 ? 1 : 0) + (b4 ? 1 : 0)), w1);
             }
             if (tq == N_EW - 1) {
                 // pa, pb now hold a_L on the lanes that own the chunk's last tokens (th = 1)
                 bool ok = true;
                 if (th == 1) {
                     const float2 da = ex2_2(pa), db = ex2_2(pb);
-                    *reinterpret_cast<float4*>(reinterpret_cast<float*>(smem + OFF_DL) + s * 64 + 4 * cq) =
-                        make_float4(da.x, da.y, db.x, db.y);
+                    stsf4(sbase + OFF_DL + 4 * (sd * 64 + 4 * cq), make_float4(da.x, da.y, db.x, db.y));
                     ok = (pa.x >= -A2_MAX) && (pa.y >= -A2_MAX) && (pb.x >= -A2_MAX) && (pb.y >= -A2_MAX);   // false for NaN as well
                 }
                 const bool all_ok = __all_sync(0xffffffffu, ok);
-                if (lane == 0) safe_flag[s] = all_ok ? 1 : 0;
-            }
-            if (tail) {
-                // v rows past the end of the sequence hold another sequence's tokens (or fill): zero them
-                for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
-                    sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
+                if (lane == 0) sts32(sbase + OFF_SAFE + 4 * sd, all_ok ? 1u : 0u);
             }
             fence_proxy_async();                  // the scaled tiles are read by the tensor core (async proxy)
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_RK_READY + s));
+            s += N_ESET;
+            if (s >= NS) { s -= NS; ph ^= 1; }
         }
     }
 
