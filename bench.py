@@ -32,8 +32,8 @@ BYTES_PER_TOKEN_HEAD = 640            # bf16 r,k,v,x in (4*64*2) + bf16 y out (6
 STATE_BYTES_PER_UNIT = 64 * 64 * 4    # fp32 final state written once per (b,h) (state_in is NULL)
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture exists)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# capture summarised under profiles/ (null once the kernel has changed since the counters were taken)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 1272915968  # 4 x (268.50 + 49.73 MB) measured at T=4096, scaled by tokens
 
 
 def parse():
