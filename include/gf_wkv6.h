@@ -123,6 +123,21 @@ GF_API gf_status_t gf_wkv6_prefill_host(const void *r, const void *k, const void
                                  gf_stream_t stream);
 GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
 
+/* Optional scratch for dense bf16 prefill calls with few (sequence, head) units.  One CTA walks one
+ * unit's sequence, so a call with fewer units than half the GPU's SMs (long-context prefill of one
+ * sequence) would leave most SMs idle.  With a workspace registered such a call cuts every sequence
+ * into up to 8 segments: a first launch carries the state over each segment from a zero start and
+ * leaves per segment its decay product and state increment (the pair (D, dS) of the recurrence
+ * S <- diag(D) S + dS, which composes associatively across segments of the wkv_t sum) in the workspace,
+ * the second launch folds them into each segment's start state and computes y.  Results agree with the
+ * unsplit call to rounding.  gf_wkv6_workspace_bytes returns what gf_wkv6_prefill(B,T,H,N) would use on
+ * the current device (0: the call does not split).  gf_wkv6_set_workspace registers a caller-owned
+ * DEVICE buffer (256-byte aligned; NULL unregisters) for all later calls of this process; the library
+ * never frees it.  A registered buffer that is too small is ignored (the call runs unsplit).  Calls that
+ * use the workspace and overlap on the GPU (different streams) race on it. */
+GF_API size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N);
+GF_API gf_status_t gf_wkv6_set_workspace(void *dev_ptr, size_t bytes);
+
 /* Forces the kernel used by the bf16 prefill calls of this process (default
  * GF_KERNEL_AUTO).  Process-wide, not thread-safe against concurrent compute calls. */
 GF_API gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel);

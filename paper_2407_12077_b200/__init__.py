@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
-    "prefill_host", "host_workspace_bytes", "set_kernel", "last_device_status",
+    "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -37,6 +37,8 @@ _SIGNATURES = {
     "gf_wkv6_step_f32": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
     "gf_wkv6_prefill_host": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_host_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_set_workspace": (_i, [_vp, _sz]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
     "gf_wkv6_launch_count": (ctypes.c_uint64, []),
@@ -126,15 +128,43 @@ def _suffix(dtype) -> str:
     raise TypeError(f"r,k,v,x must be bfloat16 or float32, got {dtype}")
 
 
+_workspace = None            # the registered scratch tensor is kept alive here
+
+
+def workspace_bytes(B, T, H, N=64) -> int:
+    """Scratch gf_wkv6_prefill(B,T,H,N) would use on the current device (0: the call does not split)."""
+    return int(load_library().gf_wkv6_workspace_bytes(int(B), int(T), int(H), int(N)))
+
+
+def set_workspace(buf: torch.Tensor | None) -> None:
+    """gf_wkv6_set_workspace: register a CUDA byte tensor as the library's scratch (None unregisters)."""
+    global _workspace
+    lib = load_library()
+    if buf is None:
+        _check(lib.gf_wkv6_set_workspace(None, 0), "gf_wkv6_set_workspace")
+    else:
+        _check(lib.gf_wkv6_set_workspace(_dev(buf, "workspace"), buf.numel() * buf.element_size()), "gf_wkv6_set_workspace")
+    _workspace = buf
+
+
+def _ensure_workspace(B, T, H, N, device) -> None:
+    """Device memory is torch's job: grow the registered scratch when a call could use more."""
+    need = workspace_bytes(B, T, H, N)
+    have = 0 if _workspace is None or _workspace.device != device else _workspace.numel()
+    if need > have:
+        set_workspace(torch.empty(need, dtype=torch.uint8, device=device))
+
+
 def last_device_status(stream=None) -> None:
     """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
     _check(load_library().gf_wkv6_last_device_status(_stream(stream)), "gf_wkv6_last_device_status")
 
 
-def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, want_state=True):
+def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, want_state=True, split=True):
     """gf_wkv6_prefill / gf_wkv6_prefill_f32.  r,k,v,x: [B,T,H,N] CUDA tensors (bf16 or fp32);
     u: [H,N] fp32; state_in: [B,H,N,N] fp32 or None (zero).  Returns (y, state_out);
-    both are allocated here unless passed in (state_out may be state_in)."""
+    both are allocated here unless passed in (state_out may be state_in).  split=False unregisters
+    the scratch workspace first, so that a call with few (b,h) units runs as a single launch."""
     lib = load_library()
     B, T, H, N = r.shape
     sfx = _suffix(r.dtype)
@@ -147,6 +177,10 @@ def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, w
             _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
             _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", r.dtype, r.shape)]
     with torch.cuda.device(r.device):
+        if sfx == "" and split:
+            _ensure_workspace(B, T, H, N, r.device)
+        elif not split and _workspace is not None:
+            set_workspace(None)
         _check(getattr(lib, "gf_wkv6_prefill" + sfx)(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill" + sfx)
     return y, state_out
 

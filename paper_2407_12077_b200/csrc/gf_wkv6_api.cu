@@ -14,6 +14,9 @@ namespace {
 
 std::atomic<uint64_t> g_launches{0};
 std::atomic<int> g_kernel{GF_KERNEL_AUTO};
+// caller-owned scratch registered with gf_wkv6_set_workspace (NULL: none)
+std::atomic<float*> g_ws{nullptr};
+std::atomic<size_t> g_ws_bytes{0};
 
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -74,7 +77,8 @@ gf_status_t prefill_dense(const IO* r, const IO* k, const IO* v, const IO* x, co
         s = gf::chunked_prefill(reinterpret_cast<const __nv_bfloat16*>(r), reinterpret_cast<const __nv_bfloat16*>(k),
                                 reinterpret_cast<const __nv_bfloat16*>(v), reinterpret_cast<const __nv_bfloat16*>(x),
                                 u, state_in, state_out, reinterpret_cast<__nv_bfloat16*>(y), nullptr,
-                                B, T, (long long)B * T, H, st, &g_launches);
+                                B, T, (long long)B * T, H, st, &g_launches, g_ws.load(std::memory_order_relaxed),
+                                g_ws_bytes.load(std::memory_order_relaxed));
         if (s != GF_ERR_UNSUPPORTED || sel == GF_KERNEL_CHUNKED) return s;
     }
     return run_exact<IO>(r, k, v, x, u, state_in, state_out, y, nullptr, B, T, H, st);
@@ -216,6 +220,24 @@ gf_status_t gf_wkv6_prefill_host(const void* r, const void* k, const void* v, co
     if (tok) ok = ok && cudaMemcpyAsync(y, d_y, tok, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     if (state_out && sb) ok = ok && cudaMemcpyAsync(state_out, d_so, sb, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     return ok ? GF_OK : GF_ERR_CUDA;
+}
+
+size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N)
+{
+    if (B <= 0 || T <= 0 || H <= 0 || N != 64) return 0;
+    int seg_chunks = 0;
+    size_t need = 0;
+    gf::choose_split((long long)B * H, T, gf::sm_count(), &seg_chunks, &need);
+    return need;
+}
+
+gf_status_t gf_wkv6_set_workspace(void* dev_ptr, size_t bytes)
+{
+    if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return GF_ERR_INVALID_ARG;
+    g_ws_bytes.store(0, std::memory_order_relaxed);
+    g_ws.store(static_cast<float*>(dev_ptr), std::memory_order_relaxed);
+    g_ws_bytes.store(dev_ptr ? bytes : 0, std::memory_order_relaxed);
+    return GF_OK;
 }
 
 gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel)

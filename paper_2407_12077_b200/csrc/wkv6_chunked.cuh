@@ -392,7 +392,17 @@ struct Params {
     const int32_t* cu_seqlens;             // nullptr: dense
     int T;                                 // dense sequence length
     int H;
+    // Sequence split (dense calls with few (sequence, head) units): every sequence is cut into nseg
+    // segments of seg_chunks chunks (the last takes the rest).  A summary launch (grid = units x
+    // (nseg - 1)) leaves, per segment but the last, its decay product D[64] and the state dS[64][64] it
+    // reaches from a zero start in `summaries` ([unit][segment][64 + 4096] fp32); the main launch
+    // (grid = units x nseg) folds the summaries before its segment into its start state:
+    // S <- diag(D) S + dS, the associative scan step across segments.  nseg = 1: no split.
+    float* summaries;
+    int seg_chunks;
+    int nseg;
 };
+constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
 // Writes a warp's 16 x 64 fp32 accumulator block (acc[n][0..1] = row g, cols 8n+2q,+1;
 // acc[n][2..3] = row g+8) as bf16 into rows row0 .. row0+15 of a 128B-swizzled [rows][64] tile.
@@ -465,6 +475,7 @@ __device__ __forceinline__ void mask_scores_sp(int sp, float (&acc)[4][4], int g
 // channel); lane = 16*half + jl works on S[32*half .. +31][16*sp + jl].  Inputs are re-read from global
 // memory and y is written there.  The loops are kept rolled: this is the exceptional path, and unrolling
 // them costs the fast path registers.
+template <bool WITH_OUTPUT>
 __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, int sp, int lane, long long first_row,
                                          int valid, size_t C, int col0)
 {
@@ -478,24 +489,33 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
         float yj = 0.f, cf = 0.f;
 #pragma unroll 1
         for (int i = 0; i < 32; i += 2) {
-            const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
             const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + 32 * half + i);
             const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + 32 * half + i);
             const float s0 = scol[i * 64], s1 = scol[(i + 1) * 64];
-            cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
-            cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
-            yj = fmaf(bf_lo(rw), s0, yj);
-            yj = fmaf(bf_hi(rw), s1, yj);
+            if (WITH_OUTPUT) {
+                const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
+                cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
+                cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
+                yj = fmaf(bf_lo(rw), s0, yj);
+                yj = fmaf(bf_hi(rw), s1, yj);
+            }
             scol[i * 64] = fmaf(expf(-expf(bf_lo(xw))), s0, bf_lo(kw) * vj);
             scol[(i + 1) * 64] = fmaf(expf(-expf(bf_hi(xw))), s1, bf_hi(kw) * vj);
         }
-        yj += __shfl_xor_sync(0xffffffffu, yj, 16);
-        cf += __shfl_xor_sync(0xffffffffu, cf, 16);
-        if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
+        if (WITH_OUTPUT) {
+            yj += __shfl_xor_sync(0xffffffffu, yj, 16);
+            cf += __shfl_xor_sync(0xffffffffu, cf, 16);
+            if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
+        }
     }
 }
 
 // ---------------------------------------------------------------- the kernel
+// SUMMARY = false: the prefill proper.  SUMMARY = true: the first pass of a split call, which only
+// carries the state over a segment from a zero start (no r, no scores, no outputs: the score warps and
+// the second MMA warp idle, the output warps only serve the token-by-token path) and writes the
+// segment's summary.
+template <bool SUMMARY>
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
@@ -509,7 +529,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     auto bar = [&](int i) { return sbase + OFF_BAR + 8 * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int unit = blockIdx.x;
+    const int gsegs = SUMMARY ? p.nseg - 1 : p.nseg;      // segments per unit that this launch covers
+    const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs;
     const int seq = unit / p.H, h = unit % p.H;
     long long row0;
     int len;
@@ -519,6 +540,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     } else {
         row0 = (long long)seq * p.T;
         len = p.T;
+    }
+    if (p.nseg > 1) {                                      // this CTA's segment of the sequence
+        const int first = min(len, seg * p.seg_chunks * L);
+        row0 += first;
+        len = (seg == p.nseg - 1) ? len - first : min(len - first, p.seg_chunks * L);
     }
     const int nchunks = (len + L - 1) / L;
     const int col0 = h * 64;
@@ -534,7 +560,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             mbar_init(bar(BAR_S_READY + i), N_GW);
             mbar_init(bar(BAR_PP_READY + i), N_GW);
             mbar_init(bar(BAR_F_FULL + i), 1);
-            mbar_init(bar(BAR_F_EMPTY + i), 2 * N_GW);
+            mbar_init(bar(BAR_F_EMPTY + i), 2 * N_GW);              // state + score warps (summary pass: state + output warps)
             mbar_init(bar(BAR_B_DONE + i), 1);
             mbar_init(bar(BAR_Y_EMPTY + i), N_GW);
         }
@@ -561,9 +587,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) break;
             const uint32_t dst = sbase + OFF_RING + s * STAGE;
             if (elect_one()) {
-                mbar_expect_tx(bar(BAR_FULL_RKV + s), STAGE);
+                mbar_expect_tx(bar(BAR_FULL_RKV + s), SUMMARY ? 3 * TILE : STAGE);
                 tma_load_2d(dst, &tm_x, col0, row, bar(BAR_FULL_RKV + s));
-                tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
+                if (!SUMMARY) tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
                 tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
                 tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
             }
@@ -592,11 +618,13 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     const uint64_t dr = smem_desc(tr), dk = smem_desc(tr + TILE), dv = smem_desc(tr + 2 * TILE);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        tc_mma(tmem + TM_P + 64 * tb, dr + (uint64_t)(2 * kk), dk + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
+                        if (!SUMMARY)
+                            tc_mma(tmem + TM_P + 64 * tb, dr + (uint64_t)(2 * kk), dk + (uint64_t)(2 * kk), IDESC_K_K, kk > 0);
                         tc_mma(tmem + TM_DS + 64 * tb, dk + (uint64_t)(128 * kk), dv + (uint64_t)(128 * kk), IDESC_MN_MN, kk > 0);
                     }
                 }
                 tc_commit(bar(BAR_F_FULL + tb));
+                if (SUMMARY) tc_commit(bar(BAR_EMPTY_RKV + s));    // no other product reads the stage
             }
             __syncwarp();
             if (++s == NS) { s = 0; ph ^= 1; }
@@ -607,7 +635,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // The masked scores of chunk c exist only after P_c completed, so every product that reads
         // ring stage s is complete when these complete: the last commit releases the stage.
         int s = 0;
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1;
             if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), pt ^ 1, abort_flag)) break;
             if (!mbar_wait_warp(bar(BAR_S_READY + tb), pt, abort_flag)) break;
@@ -641,7 +669,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         float st[8][4];
 #pragma unroll
         for (int n = 0; n < 8; ++n) {
-            if (p.state_in) {
+            if (!SUMMARY && p.state_in) {
                 const float2 lo = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)c_lo * 64 + 8 * n + 2 * q);
                 const float2 hi = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
                 st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
@@ -649,8 +677,23 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
             }
         }
+        if (!SUMMARY) {
+            // start state of a later segment: fold the summaries of the segments before it, in order
+            for (int gg = 0; gg < seg; ++gg) {
+                const float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + gg) * SUMMARY_FLOATS;
+                const float d_lo = sm[c_lo], d_hi = sm[c_lo + 8];
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                    const float2 lo = *reinterpret_cast<const float2*>(sm + 64 + c_lo * 64 + 8 * n + 2 * q);
+                    const float2 hi = *reinterpret_cast<const float2*>(sm + 64 + (c_lo + 8) * 64 + 8 * n + 2 * q);
+                    st[n][0] = fmaf(d_lo, st[n][0], lo.x); st[n][1] = fmaf(d_lo, st[n][1], lo.y);
+                    st[n][2] = fmaf(d_hi, st[n][2], hi.x); st[n][3] = fmaf(d_hi, st[n][3], hi.y);
+                }
+            }
+        }
+        float dprod_lo = 1.f, dprod_hi = 1.f;    // summary pass: decay product of the segment for this lane's two rows
         int fb_uses = 0;                         // chunks that took the token-by-token path so far
-        if (nchunks > 0) {
+        if (!SUMMARY && nchunks > 0) {
             store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
             fence_proxy_async();
             __syncwarp();
@@ -661,10 +704,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             bool next_tile_free = c == 0;        // the products of chunk c-1 have finished reading operand tile tb^1
+            const uint32_t dl = sbase + OFF_DL + 4 * (sd * 64 + c_lo);
+            const float d_lo = ldsf(dl), d_hi = ldsf(dl + 32);        // 2^{a_L} of this lane's two rows
+            if (SUMMARY) { dprod_lo *= d_lo; dprod_hi *= d_hi; }
             if (safe_at(sd)) {
                 // ---- S <- diag(2^{a_L}) (S + K^^T V)
-                const uint32_t dl = sbase + OFF_DL + 4 * (sd * 64 + c_lo);
-                const float d_lo = ldsf(dl), d_hi = ldsf(dl + 32);
                 const float2 dlo2 = make_float2(d_lo, d_lo), dhi2 = make_float2(d_hi, d_hi);
                 const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_DS + 64 * tb;
 #pragma unroll
@@ -691,7 +735,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
                 // The copy lives in the pair of bf16 state operand tiles: this chunk's tile has no reader (its
                 // products are skipped) and the other one is free once the products of chunk c-1 are done.
-                if (c >= 1 && !mbar_wait(bar(BAR_B_DONE + (tb ^ 1)), ((c - 1) >> 1) & 1, abort_flag)) break;
+                // (The summary pass does not use these tiles at all.)
+                if (!SUMMARY && c >= 1 && !mbar_wait(bar(BAR_B_DONE + (tb ^ 1)), ((c - 1) >> 1) & 1, abort_flag)) break;
                 next_tile_free = true;
                 float* scr = reinterpret_cast<float*>(smem + OFF_SB);
 #pragma unroll
@@ -714,7 +759,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (!mbar_wait(bar(BAR_SSYNC), fb_uses & 1, abort_flag)) break;
                 ++fb_uses;
             }
-            if (c + 1 < nchunks) {
+            if (!SUMMARY && c + 1 < nchunks) {
                 const int nb = tb ^ 1;
                 if (!next_tile_free && !mbar_wait(bar(BAR_B_DONE + nb), ((c - 1) >> 1) & 1, abort_flag)) break;
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
@@ -723,7 +768,17 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (lane == 0) mbar_arrive(bar(BAR_S_READY + nb));
             }
         }
-        if (p.state_out && !lds32(abort_flag)) {
+        if (SUMMARY) {
+            if (!lds32(abort_flag)) {
+                float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
+                if (q == 0) { sm[c_lo] = dprod_lo; sm[c_lo + 8] = dprod_hi; }
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                    *reinterpret_cast<float2*>(sm + 64 + c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
+                    *reinterpret_cast<float2*>(sm + 64 + (c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
+                }
+            }
+        } else if (p.state_out && seg == p.nseg - 1 && !lds32(abort_flag)) {
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
                 *reinterpret_cast<float2*>(p.state_out + sb + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
@@ -734,7 +789,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // ============================== score warps ==============================
         const int sp = warp & 3;                 // rows t = 16*sp .. 16*sp+15 of the score block
         const int g = lane >> 2, q = lane & 3;
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, ppi = tb, sd = c & (NSIDE - 1);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
@@ -771,7 +826,24 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int sp = warp & 3;                 // rows t = 16*sp .. 16*sp+15 of the chunk
         const uint32_t slab = sbase + OFF_Y + sp * 2048;
         int fb_uses = 0;                         // chunks that took the token-by-token path so far
-        for (int c = 0; c < nchunks; ++c) {
+        if (SUMMARY) {
+            // nothing to output: follow the chunks only to run the token-by-token path where one needs it
+            for (int c = 0; c < nchunks; ++c) {
+                const int tb = c & 1;
+                if (!mbar_wait(bar(BAR_F_FULL + tb), (c >> 1) & 1, abort_flag)) break;
+                if (!safe_at(c & (NSIDE - 1))) {
+                    if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
+                    exact_chunk<false>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
+                                       min(L, len - c * L), C, col0);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(BAR_FB_DONE));
+                    ++fb_uses;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+            }
+        }
+        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1;
             if (!mbar_wait(bar(BAR_B_DONE + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
@@ -783,8 +855,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // the state warps put in shared memory; writes this chunk's y rows itself
                 if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
                 if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
-                exact_chunk(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
-                            min(L, len - c * L), C, col0);
+                exact_chunk<true>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
+                                  min(L, len - c * L), C, col0);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(BAR_FB_DONE));
                 ++fb_uses;
@@ -855,7 +927,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 for (int tt = 0; tt < 4; ++tt)
                     if (8 * tq + 4 * th + tt >= valid) {
                         sts64(tx + roff[tt], make_uint2(0xff80ff80u, 0xff80ff80u));
-                        sts64(tr + roff[tt], make_uint2(0u, 0u));
+                        if (!SUMMARY) sts64(tr + roff[tt], make_uint2(0u, 0u));
                         sts64(tk + roff[tt], make_uint2(0u, 0u));
                     }
                 for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
@@ -897,7 +969,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             uint2 rw[4], kw[4];
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {             // all loads first: they are ordered with the stores below
-                rw[tt] = lds64(tr + roff[tt]);
+                if (!SUMMARY) rw[tt] = lds64(tr + roff[tt]);
                 kw[tt] = lds64(tk + roff[tt]);
             }
             float du[4];
@@ -905,24 +977,28 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
                 const float2 ca = add2(oa, aa[tt]), cb = add2(ob, ab[tt]);     // a_t
-                const float2 sra = ex2_2(pa), srb = ex2_2(pb);
                 const float2 ska = ex2_2(make_float2(-ca.x, -ca.y)), skb = ex2_2(make_float2(-cb.x, -cb.y));
-                const float2 r0 = bf_pair(rw[tt].x), r1 = bf_pair(rw[tt].y), k0 = bf_pair(kw[tt].x), k1 = bf_pair(kw[tt].y);
-                const float2 rh0 = mul2(r0, sra), rh1 = mul2(r1, srb), kh0 = mul2(k0, ska), kh1 = mul2(k1, skb);
-                const float2 acc = fma2(mul2(r1, k1), ub, mul2(mul2(r0, k0), ua));
-                rw[tt] = make_uint2(pack_bf16(rh0.x, rh0.y), pack_bf16(rh1.x, rh1.y));
+                const float2 k0 = bf_pair(kw[tt].x), k1 = bf_pair(kw[tt].y);
+                const float2 kh0 = mul2(k0, ska), kh1 = mul2(k1, skb);
                 kw[tt] = make_uint2(pack_bf16(kh0.x, kh0.y), pack_bf16(kh1.x, kh1.y));
-                du[tt] = acc.x + acc.y;
+                if (!SUMMARY) {
+                    const float2 sra = ex2_2(pa), srb = ex2_2(pb);
+                    const float2 r0 = bf_pair(rw[tt].x), r1 = bf_pair(rw[tt].y);
+                    const float2 rh0 = mul2(r0, sra), rh1 = mul2(r1, srb);
+                    const float2 acc = fma2(mul2(r1, k1), ub, mul2(mul2(r0, k0), ua));
+                    rw[tt] = make_uint2(pack_bf16(rh0.x, rh0.y), pack_bf16(rh1.x, rh1.y));
+                    du[tt] = acc.x + acc.y;
+                }
                 pa = ca; pb = cb;
             }
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
-                sts64(tr + roff[tt], rw[tt]);
+                if (!SUMMARY) sts64(tr + roff[tt], rw[tt]);
                 sts64(tk + roff[tt], kw[tt]);
             }
             // reduce the 4 bonus partials over the 16 lanes of a half-warp (transposing butterfly):
             // lanes with bits (3,2) = (b8, b4) end with token 2*b8 + b4
-            {
+            if (!SUMMARY) {
                 const bool b8 = lane & 8, b4 = lane & 4;
                 float w2[2], w1;
 #pragma unroll
@@ -1001,12 +1077,51 @@ inline bool make_map(CUtensorMap* tm, const void* base, long long rows, long lon
 
 }  // namespace ck
 
+// Number of SMs of the current device (cached per device index; 0 on failure).
+inline int sm_count()
+{
+    static int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached = n;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
+// Chooses the sequence split of a dense call: with fewer (sequence, head) units than half the SMs, each
+// sequence is cut into up to 8 segments of at least 8 chunks so that the grid fills the GPU.  Returns the
+// number of segments (1: no split) and sets seg_chunks; summary_bytes is the scratch the split needs.
+inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_t* summary_bytes)
+{
+    *seg_chunks = 0;
+    *summary_bytes = 0;
+    const int nchunks = (T + ck::L - 1) / ck::L;
+    if (units <= 0 || n_sm <= 0 || units * 2 > n_sm) return 1;
+    int g = (int)(n_sm / units);
+    if (g > 8) g = 8;
+    if (g > nchunks / 8) g = nchunks / 8;
+    if (g < 2) return 1;
+    const int sc = (nchunks + g - 1) / g;
+    g = (nchunks + sc - 1) / sc;
+    if (g < 2) return 1;
+    *seg_chunks = sc;
+    *summary_bytes = (size_t)units * (g - 1) * ck::SUMMARY_FLOATS * sizeof(float);
+    return g;
+}
+
 // Launches the chunked kernel.  Dense: cu == nullptr, n_seq = B, T = sequence length.
 // Packed: cu = device cu_seqlens, n_seq = S, T unused.  total_rows = rows of the [rows][H*64] tensors.
+// scratch / scratch_bytes: optional device memory for the sequence split (see choose_split); without
+// enough of it the call runs unsplit.
 inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                    const __nv_bfloat16* x, const float* u, const float* state_in, float* state_out,
                                    __nv_bfloat16* y, const int32_t* cu, int n_seq, int T, long long total_rows, int H,
-                                   cudaStream_t st, std::atomic<uint64_t>* launches)
+                                   cudaStream_t st, std::atomic<uint64_t>* launches, float* scratch = nullptr,
+                                   size_t scratch_bytes = 0)
 {
     const long long units = (long long)n_seq * H;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
@@ -1015,7 +1130,8 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GF_ERR_CUDA;
     if (!attr_set || attr_dev != dev) {
-        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set = true;
         attr_dev = dev;
@@ -1026,8 +1142,19 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         !ck::make_map(&tv, v, total_rows, C, 64) || !ck::make_map(&tx, x, total_rows, C, 64) ||
         !ck::make_map(&ty, y, total_rows, C, 16))
         return GF_ERR_CUDA;
-    ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H};
-    ck::wkv6_chunked_kernel<<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
+    int seg_chunks = 0, nseg = 1;
+    if (!cu && scratch) {
+        size_t need = 0;
+        nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);
+        if (nseg > 1 && (need > scratch_bytes || units * nseg > 0x7fffffffLL)) nseg = 1;
+    }
+    ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg};
+    if (nseg > 1) {
+        ck::wkv6_chunked_kernel<true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    }
+    ck::wkv6_chunked_kernel<false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

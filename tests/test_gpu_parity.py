@@ -132,6 +132,34 @@ def test_cfg3_long_context_segments_with_state_carry():
     check(y_s, s_s, y_ref, s_ref, 5e-3, "cfg3 sampled")
 
 
+@pytest.mark.parametrize("B,T,H,state_std,x_hi", [
+    (1, 64 * 16 + 37, 2, 0.1, -1.0),     # 2 segments, ragged tail in the last
+    (1, 5000, 4, 0.0, -1.0),             # 8 segments of 10 chunks, the last shorter
+    (2, 3000, 3, 0.1, -1.0),             # 6 units
+    (1, 1100, 2, 0.1, 3.0),              # strong decay: token-by-token chunks inside both passes
+])
+def test_sequence_split_matches_oracle_and_unsplit_call(B, T, H, state_std, x_hi):
+    """Few (b,h) units: the call cuts every sequence into segments (summary launch + main launch over a
+    scratch workspace).  Same result as the oracle, and as the single-launch path to rounding."""
+    assert gf.workspace_bytes(B, T, H, 64) > 0, "this shape is expected to split"
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=1234 + T, state_std=state_std, x_lo=-6.0 if x_hi < 0 else -1.0, x_hi=x_hi)
+    d = inp.to(DEV)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    before = gf.launch_count()
+    y, s = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in)
+    assert gf.launch_count() - before == 2
+    y1, s1 = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in, split=False)
+    assert gf.launch_count() - before == 3
+    y2, s2 = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in)
+    gf.last_device_status()
+    assert torch.equal(y, y2) and torch.equal(s, s2)                 # deterministic, workspace reuse is clean
+    y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+    check(y, s, y_ref, s_ref, 5e-3, "split")
+    check(y1, s1, y_ref, s_ref, 5e-3, "unsplit")
+    assert orc.rel_l2(y.float().cpu().numpy(), y1.float().cpu().numpy()) < 2e-3
+    assert orc.rel_l2(s.cpu().numpy(), s1.cpu().numpy()) < 1e-3
+
+
 def varlen_oracle_units(inp, cu, units):
     ys, ss = {}, {}
     for (s, h) in units:
