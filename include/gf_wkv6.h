@@ -138,6 +138,30 @@ GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
 GF_API size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N);
 GF_API gf_status_t gf_wkv6_set_workspace(void *dev_ptr, size_t bytes);
 
+/* Dense bf16 prefill for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of gf_wkv6_prefill.)  Some hosts of this library own no allocator at the
+ * point of the call: a plug-in inside an inference server whose device memory is planned and handed out
+ * up front, or a latency-critical loop that must never reach cudaMalloc and the device-wide
+ * synchronisation it implies.  Such a caller could not supply the workspace that the sequence split of
+ * gf_wkv6_prefill wants for calls with few (sequence, head) units, and would run those calls at a
+ * fraction of the GPU.  This entry point takes the split with scratch that is built into the library: a
+ * fixed array of GF_WKV6_STATIC_SCRATCH_BYTES in the library's device image (every GPU that loads the
+ * library holds it until the process exits).  It allocates and frees nothing and ignores the registered
+ * workspace; inputs, outputs, layouts and results are those of gf_wkv6_prefill.
+ *   - Limit: a call whose split needs more than the built-in scratch (gf_wkv6_workspace_bytes(B,T,H,N) >
+ *     GF_WKV6_STATIC_SCRATCH_BYTES) returns GF_ERR_WORKSPACE and enqueues nothing.  The size covers
+ *     B*H <= 32 units at any T (the long-context shape: one sequence, 32 heads); calls that do not split
+ *     need no scratch and always pass.
+ *   - The first call on each device looks up the array's device address (with that device current), so
+ *     make that first call before any stream capture begins on that device.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to be
+ *     cleared: the first launch of a call writes every entry its second launch reads.  Calls that overlap
+ *     on the GPU (different streams, or different host threads) race on it: serialise them. */
+#define GF_WKV6_STATIC_SCRATCH_BYTES 1597440u      /* 96 segment summaries of (64 + 64*64) floats */
+GF_API gf_status_t gf_wkv6_prefill_static(const void *r, const void *k, const void *v, const void *x,
+                                   const float *u, const float *state_in, float *state_out, void *y,
+                                   int B, int T, int H, int N, gf_stream_t stream);
+
 /* Forces the kernel used by the bf16 prefill calls of this process (default
  * GF_KERNEL_AUTO).  Process-wide, not thread-safe against concurrent compute calls. */
 GF_API gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel);

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
-    "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -31,6 +31,7 @@ _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
 _SIGNATURES = {
     "gf_wkv6_prefill": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_f32": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
+    "gf_wkv6_prefill_static": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_varlen": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_prefill_varlen_f32": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -183,6 +184,24 @@ def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, w
             set_workspace(None)
         _check(getattr(lib, "gf_wkv6_prefill" + sfx)(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill" + sfx)
     return y, state_out
+
+
+STATIC_SCRATCH_BYTES = 1597440       # GF_WKV6_STATIC_SCRATCH_BYTES
+
+
+def prefill_static(r, k, v, x, u, state_in, state_out, y, stream=None) -> None:
+    """gf_wkv6_prefill_static: the dense bf16 prefill for callers that cannot allocate.  Nothing is
+    allocated here either: y [B,T,H,N] bf16 and state_out [B,H,N,N] fp32 (or None) are the caller's,
+    and the sequence split uses the scratch built into the library.  Raises GfError(GF_ERR_WORKSPACE)
+    when the call would need more than STATIC_SCRATCH_BYTES of it."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    bf = torch.bfloat16
+    args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape),
+            _dev(u, "u", torch.float32, (H, N)), _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", bf, r.shape)]
+    with torch.cuda.device(r.device):
+        _check(lib.gf_wkv6_prefill_static(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill_static")
 
 
 def prefill_varlen(r, k, v, x, u, cu_seqlens, max_seqlen, state_in=None, state_out=None, y=None,

@@ -3,6 +3,7 @@
 #include "gf_wkv6.h"
 
 #include <atomic>
+#include <mutex>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -17,6 +18,27 @@ std::atomic<int> g_kernel{GF_KERNEL_AUTO};
 // caller-owned scratch registered with gf_wkv6_set_workspace (NULL: none)
 std::atomic<float*> g_ws{nullptr};
 std::atomic<size_t> g_ws_bytes{0};
+
+// Scratch of gf_wkv6_prefill_static: lives in the library image on every GPU that loads it.  Its name is
+// only a host-side handle here; the device address comes from cudaGetSymbolAddress (static_scratch()).
+static __device__ __align__(256) float g_static_scratch[GF_WKV6_STATIC_SCRATCH_BYTES / sizeof(float)];
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+float* static_scratch()
+{
+    constexpr int MAX_DEV = 64;
+    static std::mutex mu;
+    static float* addr[MAX_DEV] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        float* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch) != cudaSuccess) return nullptr;
+        addr[dev] = ptr;
+    }
+    return addr[dev];
+}
 
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -135,6 +157,30 @@ gf_status_t gf_wkv6_prefill(const void* r, const void* k, const void* v, const v
     using bf = __nv_bfloat16;
     return prefill_dense<bf>((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
                              (bf*)y, B, T, H, N, (cudaStream_t)stream, true);
+}
+
+gf_status_t gf_wkv6_prefill_static(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                   const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                                   gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if ((long long)B * T >= (1LL << 31)) return GF_ERR_INVALID_ARG;
+    if (B == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (T == 0) return pass_state(state_in, state_out, (size_t)B * H, st);
+    gf_status_t s = check_ptrs(r, k, v, x, u, state_in, state_out, y);
+    if (s != GF_OK) return s;
+    int seg_chunks = 0;
+    size_t need = 0;
+    gf::choose_split((long long)B * H, T, gf::sm_count(), &seg_chunks, &need);
+    if (need > GF_WKV6_STATIC_SCRATCH_BYTES) return GF_ERR_WORKSPACE;     // beyond the built-in scratch
+    float* scratch = static_scratch();
+    if (!scratch) return GF_ERR_CUDA;
+    return gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out, (bf*)y,
+                               nullptr, B, T, (long long)B * T, H, st, &g_launches, scratch,
+                               GF_WKV6_STATIC_SCRATCH_BYTES);
 }
 
 gf_status_t gf_wkv6_prefill_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
