@@ -134,6 +134,27 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm), "source": "nvidia-smi"}
 
 
+def rank_seed(rank: int, call: int) -> int:
+    """Seed of one call's inputs on one rank: every rank draws its own (b,h) units (weak scaling)."""
+    return 2000 + 100 * rank + call
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The job's time for a timed region is the slowest rank's device time."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: the units all ranks processed in a step over the (max-over-ranks) step time."""
+    return units_per_rank_step * world / (ms_per_step * 1e-3)
+
+
 def cpu_oracle_rate(calls_equiv: float, B, T, H, N, seed):
     """Times the fp64 oracle, as it stands, on `calls_equiv` calls' worth of the workload
     (whole (b,h) units of full length T).  Returns (token*heads/s, threads, description)."""
@@ -204,7 +225,7 @@ def main():
     # ---- seeded synthetic inputs, resident in HBM, distinct buffers per call (1.34 GB each >> L2)
     batches = []
     for c in range(calls):
-        inp = synth.make_dense(B, T, H, N, "bf16", seed=2000 + 100 * rank + c, device=dev)
+        inp = synth.make_dense(B, T, H, N, "bf16", seed=rank_seed(rank, c), device=dev)
         y = torch.empty_like(inp.r)
         s_out = torch.empty((B, H, N, N), device=dev, dtype=torch.float32)
         batches.append((inp, y, s_out))
@@ -245,13 +266,10 @@ def main():
     launches = gf.launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     gf.last_device_status()
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, world, dev)
     ms_per_step = elapsed_ms / args.steps
     units_per_step = B * T * H * calls * world
-    value = units_per_step / (ms_per_step * 1e-3)
+    value = whole_job_value(B * T * H * calls, world, ms_per_step)
 
     # ---- roofline of the dominant kernel (one prefill launch) from the live per-launch events
     launch_ms = statistics.mean(a.elapsed_time(b) for a, b in kernel_events)
@@ -285,10 +303,7 @@ def main():
         b.record(stream)
         barrier()
         e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(e_ms, world, dev)
         tok = B * T * H * N * 2
         e2e = {"value": units_per_step / (e_ms / e2e_steps * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": calls * (4 * tok + H * N * 4),
