@@ -131,6 +131,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrival by the lanes whose predicate holds, as one predicated instruction (no divergent branch).
+__device__ __forceinline__ void mbar_arrive_if(uint32_t bar, bool pred)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+        ::"r"(bar), "r"((uint32_t)pred) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -149,6 +158,10 @@ __device__ __forceinline__ float ldsf(uint32_t a)
     return v;
 }
 __device__ __forceinline__ void stsf(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+__device__ __forceinline__ void stsf_if(uint32_t a, float v, bool pred)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.f32 [%0], %1;\n\t}" ::"r"(a), "f"(v), "r"((uint32_t)pred) : "memory");
+}
 __device__ __forceinline__ float4 ldsf4(uint32_t a)
 {
     float4 v;
@@ -158,6 +171,11 @@ __device__ __forceinline__ float4 ldsf4(uint32_t a)
 __device__ __forceinline__ void stsf4(uint32_t a, float4 v)
 {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void stsf4_if(uint32_t a, float4 v, bool pred)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t@p st.shared.v4.f32 [%0], {%1, %2, %3, %4};\n\t}"
+                 ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"((uint32_t)pred) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
@@ -697,7 +715,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
             fence_proxy_async();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_S_READY));
+            mbar_arrive_if(bar(BAR_S_READY), lane == 0);
         }
         for (int c = 0; c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
@@ -718,7 +736,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     if (qt == 3) {
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+                        mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
                     }
 #pragma unroll
                     for (int n = 0; n < 2; ++n) {
@@ -732,7 +750,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // ---- decay too strong for one in-chunk reference point: the output warps run the exact fp32
                 // recurrence over this chunk, token by token, on a copy of the state in shared memory.
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
                 // The copy lives in the pair of bf16 state operand tiles: this chunk's tile has no reader (its
                 // products are skipped) and the other one is free once the products of chunk c-1 are done.
                 // (The summary pass does not use these tiles at all.)
@@ -745,7 +763,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     *reinterpret_cast<float2*>(scr + (c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_FB_READY));
+                mbar_arrive_if(bar(BAR_FB_READY), lane == 0);
                 if (!mbar_wait(bar(BAR_FB_DONE), fb_uses & 1, abort_flag)) break;
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
@@ -755,7 +773,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 }
                 // every state warp has re-read the copy before the operand tiles are rewritten
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_SSYNC));
+                mbar_arrive_if(bar(BAR_SSYNC), lane == 0);
                 if (!mbar_wait(bar(BAR_SSYNC), fb_uses & 1, abort_flag)) break;
                 ++fb_uses;
             }
@@ -765,7 +783,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_S_READY + nb));
+                mbar_arrive_if(bar(BAR_S_READY + nb), lane == 0);
             }
         }
         if (SUMMARY) {
@@ -810,16 +828,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 tmem_ld_16x32(ta + 32, acc);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
                 mask_scores_sp<1>(sp, acc, g, q, d_lo, d_hi);
                 store_half_bf16<1>(tp, 16 * sp, acc, lane);
                 fence_proxy_async();
             } else {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_PP_READY + ppi));
+            mbar_arrive_if(bar(BAR_PP_READY + ppi), lane == 0);
         }
     } else if (warp < WARP_E0) {
         // ============================== output warps ==============================
@@ -836,11 +854,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     exact_chunk<false>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
                                        min(L, len - c * L), C, col0);
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar(BAR_FB_DONE));
+                    mbar_arrive_if(bar(BAR_FB_DONE), lane == 0);
                     ++fb_uses;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_F_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
             }
         }
         for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
@@ -853,12 +871,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (!safe) {
                 // decay too strong for the tensor-core formulation: exact recurrence on the fp32 state copy
                 // the state warps put in shared memory; writes this chunk's y rows itself
-                if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
                 if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
                 exact_chunk<true>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
                                   min(L, len - c * L), C, col0);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_FB_DONE));
+                mbar_arrive_if(bar(BAR_FB_DONE), lane == 0);
                 ++fb_uses;
                 continue;
             }
@@ -875,7 +893,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 tmem_ld_16x32(tc + 32, yb);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_Y_EMPTY + tb));
+                mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
                 add_acc(ya, yb);
                 store_half_bf16<1>(slab, 0, ya, lane);
             }
@@ -953,13 +971,13 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             oa.x = __shfl_xor_sync(0xffffffffu, aa[3].x, 16); oa.y = __shfl_xor_sync(0xffffffffu, aa[3].y, 16);
             ob.x = __shfl_xor_sync(0xffffffffu, ab[3].x, 16); ob.y = __shfl_xor_sync(0xffffffffu, ab[3].y, 16);
             const uint32_t totc = sbase + OFF_TOT + 4 * ((c % NTOT) * N_EW * 64 + 4 * cq);
-            if (th == 0) {
+            {
                 const float2 wa = add2(aa[3], oa), wb = add2(ab[3], ob);
-                stsf4(totc + 256 * tq, make_float4(wa.x, wa.y, wb.x, wb.y));
-                oa = make_float2(0.f, 0.f); ob = oa;
+                stsf4_if(totc + 256 * tq, make_float4(wa.x, wa.y, wb.x, wb.y), th == 0);
+                if (th == 0) { oa = make_float2(0.f, 0.f); ob = oa; }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_ESYNC + eset));
+            mbar_arrive_if(bar(BAR_ESYNC + eset), lane == 0);
             if (!mbar_wait(bar(BAR_ESYNC + eset), (c >> 1) & 1, abort_flag)) break;
             for (int qq = 0; qq < tq; ++qq) {            // cumulative sum at the end of the warps before this one
                 const float4 t4 = ldsf4(totc + 256 * qq);
@@ -1012,8 +1030,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 }
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 2);
                 w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
-                if ((lane & 3) == 0)
-                    stsf(sbase + OFF_DU + 4 * (sd * 64 + 8 * tq + 4 * th + 2 * (b8 ? 1 : 0) + (b4 ? 1 : 0)), w1);
+                stsf_if(sbase + OFF_DU + 4 * (sd * 64 + 8 * tq + (lane >> 2)), w1, (lane & 3) == 0);
             }
             if (tq == N_EW - 1) {
                 // pa, pb now hold a_L on the lanes that own the chunk's last tokens (th = 1)
@@ -1028,7 +1045,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             fence_proxy_async();                  // the scaled tiles are read by the tensor core (async proxy)
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_RK_READY + s));
+            mbar_arrive_if(bar(BAR_RK_READY + s), lane == 0);
             s += N_ESET;
             if (s >= NS) { s -= NS; ph ^= 1; }
         }
