@@ -25,7 +25,10 @@
  * Pins (tests/test_oracle_pins.py): brute-force expansion of the wkv_t sum at
  * T <= 8, w == 1 cumulative-sum closed form, w == 0 special case, constant
  * w = 1/2 geometric closed form, split-and-carry, linearity / k-v rescaling,
- * head independence, orientation probes, a hand-computed worked example.
+ * head independence, orientation probes, a hand-computed worked example.  The Finch-C2
+ * form at the end of this file (k (1 - w) keys, second-value vector, no bonus) is pinned in
+ * tests/test_oracle_pins_c2.py: brute-force expansion, reduction to the bonus-free recurrence on
+ * premultiplied keys, w == 1 / w == 0 special cases, constant w = 1/2 closed form, split-and-carry.
  *
  * Inputs arrive as float (an exact carrier for both fp32 and bf16 data) and are
  * widened to double before any arithmetic; every sum runs in double in plain
@@ -118,5 +121,59 @@ void wkv6_oracle_prefill_varlen(const float *r, const float *k, const float *v, 
             unit_recurrence(r + off, k + off, v + off, x + off, NULL, u + h * N,
                             state_in ? state_in + soff : NULL,
                             state_out ? state_out + soff : NULL, y + off, len, N, C);
+        }
+}
+
+/*
+ * The Finch-C2 form of the same recurrence, as the paper's Finch-C2 block writes it: the key that
+ * enters the state is the projected key times one minus the decay of its own token,
+ *     k'_t = k_t * (1 - w_t)                       (Finch-C2 block, k_t equation)
+ * there is no bonus term, and the per-head output is r_t . wkv_t + u'_t with wkv_t = S_{t-1} and
+ * u'_t the "second value" vector of the token (o_t equation, before LayerNorm / W^O):
+ *     y_t[j]    = sum_i r_t[i] S_{t-1}[i][j] + u2_t[j]
+ *     S_t[i][j] = w_t[i] S_{t-1}[i][j] + k'_t[i] v_t[j]
+ * u2 may be NULL (no added vector).  w_direct as in unit_recurrence.  Same layouts.
+ */
+static void unit_recurrence_c2(const float *r, const float *k, const float *v, const float *x,
+                               const double *w_direct, const float *u2, const float *s_in,
+                               double *s_out, double *y, long T, long N, long row_stride)
+{
+    double *S = (double *)malloc((size_t)N * N * sizeof(double));
+    double *w = (double *)malloc((size_t)N * sizeof(double));
+    for (long i = 0; i < N * N; ++i) S[i] = s_in ? (double)s_in[i] : 0.0;
+    for (long t = 0; t < T; ++t) {
+        const float *rt = r + t * row_stride, *kt = k + t * row_stride, *vt = v + t * row_stride;
+        double *yt = y + t * row_stride;
+        for (long c = 0; c < N; ++c)
+            w[c] = w_direct ? w_direct[t * row_stride + c] : exp(-exp((double)x[t * row_stride + c]));
+        for (long j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (long i = 0; i < N; ++i) acc += (double)rt[i] * S[i * N + j];
+            yt[j] = acc + (u2 ? (double)u2[t * row_stride + j] : 0.0);
+        }
+        for (long i = 0; i < N; ++i) {
+            const double kp = (double)kt[i] * (1.0 - w[i]);
+            for (long j = 0; j < N; ++j) S[i * N + j] = w[i] * S[i * N + j] + kp * (double)vt[j];
+        }
+    }
+    if (s_out) memcpy(s_out, S, (size_t)N * N * sizeof(double));
+    free(S);
+    free(w);
+}
+
+void wkv6_oracle_prefill_c2(const float *r, const float *k, const float *v, const float *x,
+                            const double *w_direct, const float *u2, const float *state_in,
+                            double *state_out, double *y, long B, long T, long H, long N)
+{
+    const long C = H * N;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (long b = 0; b < B; ++b)
+        for (long h = 0; h < H; ++h) {
+            const size_t off = (size_t)b * T * C + (size_t)h * N;
+            const size_t soff = ((size_t)b * H + h) * N * N;
+            unit_recurrence_c2(r + off, k + off, v + off, x ? x + off : NULL,
+                               w_direct ? w_direct + off : NULL, u2 ? u2 + off : NULL,
+                               state_in ? state_in + soff : NULL,
+                               state_out ? state_out + soff : NULL, y + off, T, N, C);
         }
 }

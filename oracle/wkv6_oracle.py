@@ -37,6 +37,7 @@ def _load():
         _lib.wkv6_oracle_threads.restype = ctypes.c_int
         _lib.wkv6_oracle_prefill.restype = None
         _lib.wkv6_oracle_prefill_varlen.restype = None
+        _lib.wkv6_oracle_prefill_c2.restype = None
     return _lib
 
 
@@ -92,6 +93,28 @@ def prefill(r, k, v, x, u, state_in=None, w=None):
     lib.wkv6_oracle_prefill(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(w, d), _p(u, f),
                             _p(state_in, f), _p(s_out, d), _p(y, d),
                             ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(H), ctypes.c_long(N))
+    return y, s_out
+
+
+def prefill_c2(r, k, v, x, u2=None, state_in=None, w=None):
+    """Finch-C2 form (the paper's Finch-C2 block): the key entering the state is k (1 - w), no bonus,
+    y_t = r_t . wkv_t + u2_t.  r,k,v,x,u2: [B,T,H,N] (u2 may be None); ``w`` as in prefill().
+    Returns (y float64 [B,T,H,N], state_out float64 [B,H,N,N])."""
+    lib = _load()
+    r, k, v, x, u2, state_in = _f32(r), _f32(k), _f32(v), _f32(x), _f32(u2), _f32(state_in)
+    B, T, H, N = r.shape
+    assert k.shape == r.shape and v.shape == r.shape and (u2 is None or u2.shape == r.shape)
+    if w is not None:
+        w = np.ascontiguousarray(np.asarray(w, dtype=np.float64))
+        assert w.shape == r.shape
+    else:
+        assert x is not None and x.shape == r.shape
+    y = np.zeros((B, T, H, N), dtype=np.float64)
+    s_out = np.zeros((B, H, N, N), dtype=np.float64)
+    f, d = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_prefill_c2(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(w, d), _p(u2, f),
+                               _p(state_in, f), _p(s_out, d), _p(y, d),
+                               ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(H), ctypes.c_long(N))
     return y, s_out
 
 
