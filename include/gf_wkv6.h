@@ -79,6 +79,20 @@ GF_API gf_status_t gf_wkv6_prefill(const void *r, const void *k, const void *v, 
                             const float *u, const float *state_in, float *state_out, void *y,
                             int B, int T, int H, int N, gf_stream_t stream);
 
+/* Dense prefill in the Finch-C2 form, bf16 r,k,v,x,u2,y: the paper's Finch-C2 block as written.  k is the
+ * projected key BEFORE the block's "(1 - w_t)" factor; the call applies it (k'_t = k_t (1 - w_t), the k_t
+ * equation), uses no bonus, and adds the token's second-value vector to the per-head output (the o_t
+ * equation before LayerNorm and W^O):
+ *     y_t = r_t . wkv_t + u2_t,     wkv_t = S_{t-1},     S_t = diag(w_t) S_{t-1} + k'_t^T v_t.
+ * u2 is [B][T][H][N] bf16 (the block's u'_t), or NULL for no added vector.  Everything else (layouts,
+ * states, sequence split with the registered workspace, error behaviour) is as for gf_wkv6_prefill.  The
+ * factor is formed from the key scales the kernel already has (2^{-a_t} - 2^{-a_{t-1}}), which costs no
+ * extra exponential; its relative error is about 2^-22 / (1 - w_t), i.e. below bf16 rounding for
+ * w_t <= 0.9999. */
+GF_API gf_status_t gf_wkv6_prefill_c2(const void *r, const void *k, const void *v, const void *x,
+                               const void *u2, const float *state_in, float *state_out, void *y,
+                               int B, int T, int H, int N, gf_stream_t stream);
+
 /* Same with fp32 r,k,v,x,y (token-by-token fp32 recurrence). */
 GF_API gf_status_t gf_wkv6_prefill_f32(const float *r, const float *k, const float *v, const float *x,
                                 const float *u, const float *state_in, float *state_out, float *y,

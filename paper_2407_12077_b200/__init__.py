@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
-    "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "prefill_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -32,6 +32,7 @@ _SIGNATURES = {
     "gf_wkv6_prefill": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_f32": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_static": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
+    "gf_wkv6_prefill_c2": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_varlen": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_prefill_varlen_f32": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -183,6 +184,28 @@ def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, w
         elif not split and _workspace is not None:
             set_workspace(None)
         _check(getattr(lib, "gf_wkv6_prefill" + sfx)(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill" + sfx)
+    return y, state_out
+
+
+def prefill_c2(r, k, v, x, u2=None, state_in=None, state_out=None, y=None, stream=None, want_state=True, split=True):
+    """gf_wkv6_prefill_c2: the Finch-C2 form.  r,k,v,x (and u2, the per-token second-value vector, or
+    None): [B,T,H,N] bf16 CUDA tensors; k is the key before the (1 - w) factor.  Returns (y, state_out)."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    bf = torch.bfloat16
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None and want_state:
+        state_out = torch.empty((B, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape),
+            _dev(u2, "u2", bf, r.shape), _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", bf, r.shape)]
+    with torch.cuda.device(r.device):
+        if split:
+            _ensure_workspace(B, T, H, N, r.device)
+        elif _workspace is not None:
+            set_workspace(None)
+        _check(lib.gf_wkv6_prefill_c2(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill_c2")
     return y, state_out
 
 

@@ -183,6 +183,28 @@ gf_status_t gf_wkv6_prefill_static(const void* r, const void* k, const void* v, 
                                GF_WKV6_STATIC_SCRATCH_BYTES);
 }
 
+gf_status_t gf_wkv6_prefill_c2(const void* r, const void* k, const void* v, const void* x, const void* u2,
+                               const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                               gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if ((long long)B * T >= (1LL << 31)) return GF_ERR_INVALID_ARG;
+    if (B == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (T == 0) return pass_state(state_in, state_out, (size_t)B * H, st);
+    if (!r || !k || !v || !x || !y) return GF_ERR_INVALID_ARG;
+    if (misaligned(r) || misaligned(k) || misaligned(v) || misaligned(x) || misaligned(u2) || misaligned(y) ||
+        misaligned(state_in) || misaligned(state_out))
+        return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x || y == u2) return GF_ERR_INVALID_ARG;
+    return gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, nullptr, state_in, state_out,
+                               (bf*)y, nullptr, B, T, (long long)B * T, H, st, &g_launches,
+                               g_ws.load(std::memory_order_relaxed), g_ws_bytes.load(std::memory_order_relaxed),
+                               (const bf*)u2, 1);
+}
+
 gf_status_t gf_wkv6_prefill_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
                                 const float* state_in, float* state_out, float* y, int B, int T, int H, int N,
                                 gf_stream_t stream)

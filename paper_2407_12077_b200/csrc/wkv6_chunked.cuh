@@ -93,7 +93,8 @@ constexpr int OFF_RING = 0;                                // [NS][STAGE]
 constexpr int OFF_SB = OFF_RING + NS * STAGE;              // [NSB][TILE]          bf16 chunk-start state [c][j]
 constexpr int OFF_PP = OFF_SB + NSB * TILE;                // [NPP][TILE]          bf16 masked scores [t][i]
 constexpr int OFF_Y = OFF_PP + NPP * TILE;                 // [N_GW][16 rows x 128 B] y staging, one slab per warp
-constexpr int OFF_TOT = OFF_Y + N_GW * 2048;               // [NTOT][N_EW][64] float
+constexpr int OFF_U2 = OFF_Y + N_GW * 2048;                // [N_GW][16 rows x 128 B] second-value slabs (Finch-C2 form)
+constexpr int OFF_TOT = OFF_U2 + N_GW * 2048;              // [NTOT][N_EW][64] float
 constexpr int OFF_DL = OFF_TOT + NTOT * N_EW * 64 * 4;     // [NSIDE][64] float    2^{a_L}
 constexpr int OFF_DU = OFF_DL + NSIDE * 64 * 4;            // [NSIDE][64] float    bonus coefficient per token
 constexpr int OFF_SAFE = OFF_DU + NSIDE * 64 * 4;          // [NSIDE] int
@@ -114,7 +115,8 @@ enum {
     BAR_SSYNC = BAR_ESYNC + 2,           // token-by-token path only: state-warp rendezvous,
     BAR_FB_READY = BAR_SSYNC + 1,        //   fp32 state copy in place for the output warps,
     BAR_FB_DONE = BAR_FB_READY + 1,      //   and advanced by them over the chunk
-    BAR_COUNT = BAR_FB_DONE + 1
+    BAR_U2 = BAR_FB_DONE + 1,            // Finch-C2 form: one per output warp, its second-value slab has landed
+    BAR_COUNT = BAR_U2 + N_GW
 };
 constexpr int SMEM_BYTES = OFF_BAR + BAR_COUNT * 8;
 constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;              // slack for manual 1024-byte alignment
@@ -401,6 +403,12 @@ __device__ __forceinline__ void stsm_x4(uint32_t a, uint32_t r0, uint32_t r1, ui
                  ::"r"(a), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
 }
 
+__device__ __forceinline__ void ldsm_x4(uint32_t a, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(a) : "memory");
+}
+
 struct Params {
     const __nv_bfloat16 *r, *k, *v, *x;   // raw pointers, used only by the token-by-token path
     __nv_bfloat16* y;
@@ -419,6 +427,11 @@ struct Params {
     float* summaries;
     int seg_chunks;
     int nseg;
+    // Finch-C2 form (the paper's Finch-C2 block): c2 != 0 multiplies every key by one minus the decay of
+    // its own token and drops the bonus (u is not read); u2, if not NULL, is the per-token second-value
+    // vector [rows][H*64] bf16 added to the output.
+    const __nv_bfloat16* u2;
+    int c2;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -445,6 +458,21 @@ __device__ __forceinline__ void store_half_bf16(uint32_t tile, int row0, const f
         stsm_x4(tile + swz(row, (2 * (2 * HALF + m) + (mi >> 1)) << 4),
                 pack_bf16(acc[2 * m][0], acc[2 * m][1]), pack_bf16(acc[2 * m][2], acc[2 * m][3]),
                 pack_bf16(acc[2 * m + 1][0], acc[2 * m + 1][1]), pack_bf16(acc[2 * m + 1][2], acc[2 * m + 1][3]));
+}
+
+// acc += the bf16 values of columns 32*HALF .. +31 of a 128B-swizzled [16 rows][64] slab (accumulator layout).
+template <int HALF>
+__device__ __forceinline__ void add_slab_bf16(float (&acc)[4][4], uint32_t slab, int lane)
+{
+    const int mi = lane >> 3, rr = lane & 7;
+    const int row = rr + 8 * (mi & 1);
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+        uint32_t w0, w1, w2, w3;     // (rows 0-7, block 2m), (rows 8-15, block 2m), (rows 0-7, block 2m+1), (rows 8-15, block 2m+1)
+        ldsm_x4(slab + swz(row, (2 * (2 * HALF + m) + (mi >> 1)) << 4), w0, w1, w2, w3);
+        acc[2 * m][0] += bf_lo(w0); acc[2 * m][1] += bf_hi(w0); acc[2 * m][2] += bf_lo(w1); acc[2 * m][3] += bf_hi(w1);
+        acc[2 * m + 1][0] += bf_lo(w2); acc[2 * m + 1][1] += bf_hi(w2); acc[2 * m + 1][2] += bf_lo(w3); acc[2 * m + 1][3] += bf_hi(w3);
+    }
 }
 
 __device__ __forceinline__ void add_acc(float (&a)[4][4], const float (&b)[4][4])
@@ -500,6 +528,7 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
     const int half = lane >> 4, j = 16 * sp + (lane & 15);
     float* scol = scr + (32 * half) * 64 + j;
     const float* ug = p.u + h * 64 + 32 * half;
+    const bool c2 = p.c2 != 0;
 #pragma unroll 1
     for (int t = 0; t < valid; ++t) {
         const size_t ro = (size_t)(first_row + t) * C + col0;
@@ -510,20 +539,29 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
             const uint32_t kw = *reinterpret_cast<const uint32_t*>(p.k + ro + 32 * half + i);
             const uint32_t xw = *reinterpret_cast<const uint32_t*>(p.x + ro + 32 * half + i);
             const float s0 = scol[i * 64], s1 = scol[(i + 1) * 64];
+            const float w0 = expf(-expf(bf_lo(xw))), w1 = expf(-expf(bf_hi(xw)));
+            float k0 = bf_lo(kw), k1 = bf_hi(kw);
+            if (c2) { k0 *= 1.f - w0; k1 *= 1.f - w1; }
             if (WITH_OUTPUT) {
                 const uint32_t rw = *reinterpret_cast<const uint32_t*>(p.r + ro + 32 * half + i);
-                cf = fmaf(bf_lo(rw) * ug[i], bf_lo(kw), cf);
-                cf = fmaf(bf_hi(rw) * ug[i + 1], bf_hi(kw), cf);
+                if (!c2) {
+                    cf = fmaf(bf_lo(rw) * ug[i], k0, cf);
+                    cf = fmaf(bf_hi(rw) * ug[i + 1], k1, cf);
+                }
                 yj = fmaf(bf_lo(rw), s0, yj);
                 yj = fmaf(bf_hi(rw), s1, yj);
             }
-            scol[i * 64] = fmaf(expf(-expf(bf_lo(xw))), s0, bf_lo(kw) * vj);
-            scol[(i + 1) * 64] = fmaf(expf(-expf(bf_hi(xw))), s1, bf_hi(kw) * vj);
+            scol[i * 64] = fmaf(w0, s0, k0 * vj);
+            scol[(i + 1) * 64] = fmaf(w1, s1, k1 * vj);
         }
         if (WITH_OUTPUT) {
             yj += __shfl_xor_sync(0xffffffffu, yj, 16);
             cf += __shfl_xor_sync(0xffffffffu, cf, 16);
-            if (half == 0) p.y[ro + j] = __float2bfloat16_rn(fmaf(cf, vj, yj));
+            if (half == 0) {
+                float out = fmaf(cf, vj, yj);
+                if (p.u2) out += __bfloat162float(p.u2[ro + j]);
+                p.y[ro + j] = __float2bfloat16_rn(out);
+            }
         }
     }
 }
@@ -533,11 +571,13 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
 // carries the state over a segment from a zero start (no r, no scores, no outputs: the score warps and
 // the second MMA warp idle, the output warps only serve the token-by-token path) and writes the
 // segment's summary.
-template <bool SUMMARY>
+// C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus, optional second-value vector).
+template <bool SUMMARY, bool C2>
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
-                    const __grid_constant__ CUtensorMap tm_y16, const Params p)
+                    const __grid_constant__ CUtensorMap tm_y16, const __grid_constant__ CUtensorMap tm_u2_16,
+                    const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -586,6 +626,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         mbar_init(bar(BAR_SSYNC), N_GW);
         mbar_init(bar(BAR_FB_READY), N_GW);
         mbar_init(bar(BAR_FB_DONE), N_GW);
+        for (int i = 0; i < N_GW; ++i) mbar_init(bar(BAR_U2 + i), 1);
         sts32(abort_flag, 0u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
@@ -861,6 +902,20 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 mbar_arrive_if(bar(BAR_F_EMPTY + tb), lane == 0);
             }
         }
+        // Finch-C2 form: this warp's 16 rows of the second-value tensor come by TMA into a slab of its own,
+        // one chunk ahead (requested as soon as the previous chunk's rows have been read out of it)
+        const bool has_u2 = !SUMMARY && C2 && p.u2 != nullptr;
+        const uint32_t u2slab = sbase + OFF_U2 + sp * 2048;
+        bool u2_pending = false;
+        auto load_u2 = [&](int c) {
+            if (elect_one()) {
+                mbar_expect_tx(bar(BAR_U2 + sp), 2048);
+                tma_load_2d(u2slab, &tm_u2_16, col0, (int)(row0 + (long long)c * L + 16 * sp), bar(BAR_U2 + sp));
+            }
+            __syncwarp();
+            u2_pending = true;
+        };
+        if (has_u2 && nchunks > 0) load_u2(0);
         for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1;
             if (!mbar_wait(bar(BAR_B_DONE + tb), (c >> 1) & 1, abort_flag)) break;
@@ -872,6 +927,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // decay too strong for the tensor-core formulation: exact recurrence on the fp32 state copy
                 // the state warps put in shared memory; writes this chunk's y rows itself
                 mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
+                if (has_u2) {                     // keep the slab's phase in step: consume, then request the next
+                    if (!mbar_wait(bar(BAR_U2 + sp), c & 1, abort_flag)) break;
+                    u2_pending = false;
+                    if (c + 1 < nchunks) load_u2(c + 1);
+                }
                 if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
                 exact_chunk<true>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
                                   min(L, len - c * L), C, col0);
@@ -888,6 +948,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 tmem_ld_16x32(ta, ya);
                 tmem_ld_16x32(tc, yb);
                 add_acc(ya, yb);
+                if (has_u2) {
+                    if (!mbar_wait(bar(BAR_U2 + sp), c & 1, abort_flag)) break;
+                    u2_pending = false;
+                    add_slab_bf16<0>(ya, u2slab, lane);
+                }
                 store_half_bf16<0>(slab, 0, ya, lane);
                 tmem_ld_16x32(ta + 32, ya);
                 tmem_ld_16x32(tc + 32, yb);
@@ -895,6 +960,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
                 add_acc(ya, yb);
+                if (has_u2) {
+                    add_slab_bf16<1>(ya, u2slab, lane);
+                    __syncwarp();
+                    if (c + 1 < nchunks) load_u2(c + 1);
+                }
                 store_half_bf16<1>(slab, 0, ya, lane);
             }
             fence_proxy_async();
@@ -919,13 +989,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
         }
         if (lane == 0) bulk_wait<0>();
+        // leaving early (abort) with a slab copy still in flight: wait for it, it targets this CTA's memory
+        if (u2_pending) mbar_wait(bar(BAR_U2 + sp), 0, abort_flag, false) || mbar_wait(bar(BAR_U2 + sp), 1, abort_flag, false);
     } else {
         // ============================== elementwise warps ==============================
         const int eset = (warp - WARP_E0) / N_EW;        // this set takes chunks eset, eset + 2, ...
         const int tq = (warp - WARP_E0) % N_EW;          // tokens 8*tq .. 8*tq+7 of the chunk
         const int cq = lane & 15, th = lane >> 4;        // channels 4*cq .. 4*cq+3, tokens 8*tq + 4*th + (0..3)
         const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
-        const float4 u4 = *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
+        constexpr bool c2 = C2;                          // Finch-C2 form: keys times (1 - w), no bonus
+        const float4 u4 = c2 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
         const float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
         uint32_t roff[4];                                // swizzled byte offsets of this lane's 8 bytes in its 4 rows
 #pragma unroll
@@ -992,12 +1065,17 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             float du[4];
             float2 pa = oa, pb = ob;                     // a_{t-1}
+            // Finch-C2: k (1 - w_t) 2^{-a_t} = k (2^{-a_t} - 2^{-a_{t-1}}) since w_t 2^{-a_t} = 2^{-a_{t-1}}:
+            // the previous token's key scale is subtracted (no further exponential but the run's first)
+            float2 qa = make_float2(0.f, 0.f), qb = qa;
+            if (c2) { qa = ex2_2(make_float2(-oa.x, -oa.y)); qb = ex2_2(make_float2(-ob.x, -ob.y)); }
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
                 const float2 ca = add2(oa, aa[tt]), cb = add2(ob, ab[tt]);     // a_t
                 const float2 ska = ex2_2(make_float2(-ca.x, -ca.y)), skb = ex2_2(make_float2(-cb.x, -cb.y));
                 const float2 k0 = bf_pair(kw[tt].x), k1 = bf_pair(kw[tt].y);
-                const float2 kh0 = mul2(k0, ska), kh1 = mul2(k1, skb);
+                const float2 kh0 = mul2(k0, c2 ? sub2(ska, qa) : ska), kh1 = mul2(k1, c2 ? sub2(skb, qb) : skb);
+                qa = ska; qb = skb;
                 kw[tt] = make_uint2(pack_bf16(kh0.x, kh0.y), pack_bf16(kh1.x, kh1.y));
                 if (!SUMMARY) {
                     const float2 sra = ex2_2(pa), srb = ex2_2(pb);
@@ -1138,7 +1216,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
                                    const __nv_bfloat16* x, const float* u, const float* state_in, float* state_out,
                                    __nv_bfloat16* y, const int32_t* cu, int n_seq, int T, long long total_rows, int H,
                                    cudaStream_t st, std::atomic<uint64_t>* launches, float* scratch = nullptr,
-                                   size_t scratch_bytes = 0)
+                                   size_t scratch_bytes = 0, const __nv_bfloat16* u2 = nullptr, int c2 = 0)
 {
     const long long units = (long long)n_seq * H;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
@@ -1147,17 +1225,19 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GF_ERR_CUDA;
     if (!attr_set || attr_dev != dev) {
-        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set = true;
         attr_dev = dev;
     }
-    CUtensorMap tr, tk, tv, tx, ty;
+    CUtensorMap tr, tk, tv, tx, ty, tu2;
     const long long C = (long long)H * 64;
     if (!ck::make_map(&tr, r, total_rows, C, 64) || !ck::make_map(&tk, k, total_rows, C, 64) ||
         !ck::make_map(&tv, v, total_rows, C, 64) || !ck::make_map(&tx, x, total_rows, C, 64) ||
-        !ck::make_map(&ty, y, total_rows, C, 16))
+        !ck::make_map(&ty, y, total_rows, C, 16) || !ck::make_map(&tu2, u2 ? (const void*)u2 : (const void*)y, total_rows, C, 16))
         return GF_ERR_CUDA;
     int seg_chunks = 0, nseg = 1;
     if (!cu && scratch) {
@@ -1165,13 +1245,15 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);
         if (nseg > 1 && (need > scratch_bytes || units * nseg > 0x7fffffffLL)) nseg = 1;
     }
-    ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg};
+    ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
     if (nseg > 1) {
-        ck::wkv6_chunked_kernel<true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
+        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
-    ck::wkv6_chunked_kernel<false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, p);
+    if (c2) ck::wkv6_chunked_kernel<false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+    else ck::wkv6_chunked_kernel<false, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

@@ -1,0 +1,96 @@
+"""GPU parity of the Finch-C2 form (gf_wkv6_prefill_c2) against the fp64 oracle's Finch-C2 recurrence:
+keys times one minus their decay, no bonus, second-value vector added to the output.  Same tolerance as
+the other bf16 parity tests (relative L2 <= 5e-3 on y and on the final state)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2407_12077_b200 as gf
+from oracle import wkv6_oracle as orc
+from paper_2407_12077_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL = 5e-3
+
+
+def make(B, T, H, seed, state_std=0.1, with_u2=True, **kw):
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=seed, state_std=state_std, **kw)
+    g = torch.Generator().manual_seed(seed + 7)
+    u2 = torch.randn(inp.r.shape, generator=g).bfloat16() if with_u2 else None
+    return inp, u2
+
+
+def run(inp, u2, **kw):
+    d = inp.to(DEV)
+    y, s = gf.prefill_c2(d.r, d.k, d.v, d.x, None if u2 is None else u2.to(DEV), d.state_in, **kw)
+    gf.last_device_status()
+    return y, s
+
+
+def check(y, s, inp, u2, what):
+    y_ref, s_ref = orc.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in)
+    ey, es = orc.rel_l2(y.float().cpu().numpy(), y_ref), orc.rel_l2(s.cpu().numpy(), s_ref)
+    assert np.isfinite(ey) and ey <= TOL, f"{what}: y rel-L2 {ey:.3e}"
+    assert np.isfinite(es) and es <= TOL, f"{what}: state rel-L2 {es:.3e}"
+    return ey, es
+
+
+@pytest.mark.parametrize("T", [1, 2, 17, 63, 64, 65, 128, 200, 321, 1000])
+@pytest.mark.parametrize("with_u2", [True, False])
+def test_c2_ragged_lengths(T, with_u2):
+    inp, u2 = make(2, T, 3, 300 + T, with_u2=with_u2)
+    y, s = run(inp, u2)
+    check(y, s, inp, u2, f"T={T} u2={with_u2}")
+
+
+def test_c2_small_model_shape_full():
+    c = synth.CONFIGS["cfg1"]
+    inp, u2 = make(c["B"], c["T"], c["H"], 1100)
+    y, s = run(inp, u2)
+    check(y, s, inp, u2, "cfg1 shape")
+
+
+@pytest.mark.parametrize("case", ["w_one", "fast_decay", "mixed_extreme", "slow_decay"])
+def test_c2_extreme_decay_logits(case):
+    inp, u2 = make(1, 200, 2, 810)
+    g = torch.Generator().manual_seed(811)
+    if case == "w_one":
+        inp.x = torch.full_like(inp.x, float("-inf"))                              # keys vanish, state frozen
+    elif case == "fast_decay":
+        inp.x = (torch.rand(inp.x.shape, generator=g) * 4 - 1).bfloat16()          # token-by-token chunks
+    elif case == "slow_decay":
+        inp.x = (torch.rand(inp.x.shape, generator=g) * 3 - 9).bfloat16()          # 1 - w down to ~1e-4
+    else:
+        inp.x = (torch.rand(inp.x.shape, generator=g) * 16 - 8).bfloat16()
+        inp.x[:, ::7, :, ::5] = float("-inf")
+    y, s = run(inp, u2)
+    assert torch.isfinite(y.float()).all() and torch.isfinite(s).all()
+    check(y, s, inp, u2, case)
+
+
+def test_c2_sequence_split_and_determinism():
+    inp, u2 = make(1, 5000, 4, 820)
+    assert gf.workspace_bytes(1, 5000, 4, 64) > 0
+    y, s = run(inp, u2)
+    y1, s1 = run(inp, u2, split=False)
+    y2, s2 = run(inp, u2)
+    assert torch.equal(y, y2) and torch.equal(s, s2)
+    check(y, s, inp, u2, "split")
+    check(y1, s1, inp, u2, "unsplit")
+
+
+def test_c2_full_size_sampled_units():
+    """1.5B-class shape in the launch configuration the benchmark uses; the oracle recomputes whole (b,h) units."""
+    c = synth.CONFIGS["cfg2"]
+    inp = synth.make_dense(c["B"], c["T"], c["H"], 64, "bf16", seed=2100, device=DEV)
+    u2 = torch.randn(inp.r.shape, device=DEV, generator=torch.Generator(device=DEV).manual_seed(5)).bfloat16()
+    y, s = gf.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, None)
+    gf.last_device_status()
+    assert torch.isfinite(y.float()).all() and torch.isfinite(s).all()
+    for b, h in [(0, 0), (3, 31), (1, 17)]:
+        pick = lambda t: t[b, :, h].cpu()[None, :, None, :].contiguous()
+        y_ref, s_ref = orc.prefill_c2(pick(inp.r), pick(inp.k), pick(inp.v), pick(inp.x), pick(u2), None)
+        ey = orc.rel_l2(y[b, :, h].float().cpu().numpy(), y_ref[0, :, 0])
+        es = orc.rel_l2(s[b, h].cpu().numpy(), s_ref[0, 0])
+        assert ey <= TOL and es <= TOL, (b, h, ey, es)
