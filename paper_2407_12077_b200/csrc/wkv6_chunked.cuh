@@ -382,6 +382,17 @@ __device__ __forceinline__ void sts64(uint32_t a, uint2 v)
 {
     asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
 }
+// the same at a compile-time byte offset from the address (folded into the instruction)
+template <int OFF> __device__ __forceinline__ uint2 lds64_at(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(a), "n"(OFF));
+    return v;
+}
+template <int OFF> __device__ __forceinline__ void sts64_at(uint32_t a, uint2 v)
+{
+    asm volatile("st.shared.v2.u32 [%0+%3], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y), "n"(OFF) : "memory");
+}
 __device__ __forceinline__ void sts128z(uint32_t a)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
@@ -1007,7 +1018,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         int s = eset, ph = 0;                            // ring stage of this set's current chunk and its phase bit
         for (int c = eset; c < nchunks; c += N_ESET) {
             const int sd = c & (NSIDE - 1);
-            const uint32_t tx = sbase + OFF_RING + s * STAGE, tr = tx + TILE, tk = tr + TILE, tv = tk + TILE;
+            const uint32_t tx = sbase + OFF_RING + s * STAGE, tv = tx + 3 * TILE;
+            uint32_t ax[4];                              // this lane's 8 bytes in its 4 rows of the x tile; r at +TILE, k at +2 TILE
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) ax[tt] = tx + roff[tt];
             if (!mbar_wait(bar(BAR_FULL_RKV + s), ph, abort_flag)) break;
             if (len - c * L < L) {
                 // Ragged last chunk: rows past the end of the sequence hold another sequence's tokens (or the
@@ -1017,9 +1031,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
 #pragma unroll
                 for (int tt = 0; tt < 4; ++tt)
                     if (8 * tq + 4 * th + tt >= valid) {
-                        sts64(tx + roff[tt], make_uint2(0xff80ff80u, 0xff80ff80u));
-                        if (!SUMMARY) sts64(tr + roff[tt], make_uint2(0u, 0u));
-                        sts64(tk + roff[tt], make_uint2(0u, 0u));
+                        sts64(ax[tt], make_uint2(0xff80ff80u, 0xff80ff80u));
+                        if (!SUMMARY) sts64_at<TILE>(ax[tt], make_uint2(0u, 0u));
+                        sts64_at<2 * TILE>(ax[tt], make_uint2(0u, 0u));
                     }
                 for (int i = etid; i < (L - valid) * 8; i += 32 * N_EW)
                     sts128z(tv + (valid + (i >> 3)) * 128 + ((i & 7) << 4));
@@ -1029,7 +1043,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             {
                 uint2 xw[4];
 #pragma unroll
-                for (int tt = 0; tt < 4; ++tt) xw[tt] = lds64(tx + roff[tt]);
+                for (int tt = 0; tt < 4; ++tt) xw[tt] = lds64(ax[tt]);
                 float2 ra = make_float2(0.f, 0.f), rb = ra;
 #pragma unroll
                 for (int tt = 0; tt < 4; ++tt) {
@@ -1060,8 +1074,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             uint2 rw[4], kw[4];
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {             // all loads first: they are ordered with the stores below
-                if (!SUMMARY) rw[tt] = lds64(tr + roff[tt]);
-                kw[tt] = lds64(tk + roff[tt]);
+                if (!SUMMARY) rw[tt] = lds64_at<TILE>(ax[tt]);
+                kw[tt] = lds64_at<2 * TILE>(ax[tt]);
             }
             float du[4];
             float2 pa = oa, pb = ob;                     // a_{t-1}
@@ -1089,8 +1103,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) {
-                if (!SUMMARY) sts64(tr + roff[tt], rw[tt]);
-                sts64(tk + roff[tt], kw[tt]);
+                if (!SUMMARY) sts64_at<TILE>(ax[tt], rw[tt]);
+                sts64_at<2 * TILE>(ax[tt], kw[tt]);
             }
             // reduce the 4 bonus partials over the 16 lanes of a half-warp (transposing butterfly):
             // lanes with bits (3,2) = (b8, b4) end with token 2*b8 + b4
