@@ -242,6 +242,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// Asks the TMA unit to bring a tile into L2 (no shared-memory destination, no completion to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(c0), "r"(c1) : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int c0, int c1, uint32_t src)
 {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
@@ -922,6 +927,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (elect_one()) {
                 mbar_expect_tx(bar(BAR_U2 + sp), 2048);
                 tma_load_2d(u2slab, &tm_u2_16, col0, (int)(row0 + (long long)c * L + 16 * sp), bar(BAR_U2 + sp));
+                // the slab is single: pull the rows of the chunks after this one into L2 meanwhile, so that
+                // their loads, which can only be issued once the slab is free, are short
+                if (c + 2 < nchunks) tma_prefetch_2d(&tm_u2_16, col0, (int)(row0 + (long long)(c + 2) * L + 16 * sp));
+                if (c + 3 < nchunks) tma_prefetch_2d(&tm_u2_16, col0, (int)(row0 + (long long)(c + 3) * L + 16 * sp));
             }
             __syncwarp();
             u2_pending = true;
