@@ -7,7 +7,7 @@
 //   P[t,i] = sum_c (r_t[c] 2^{a_{t-1}[c]}) (k_i[c] 2^{-a_i[c]})
 //   S_L  = diag(2^{a_L}) ( S_0 + sum_i (k_i * 2^{-a_i})^T v_i )
 // so a chunk is four 64x64x64 bf16 contractions (fp32 accumulate) around an fp32 elementwise
-// phase.  The contractions are tcgen05.mma instructions issued by one thread, with operands in
+// phase.  The contractions are tcgen05.mma instructions issued by elected lanes of two warps, with operands in
 // 128-byte-swizzled shared memory tiles (the layout TMA delivers) and accumulators in tensor
 // memory; score, state-increment and output accumulators are double buffered there so the
 // tensor pipe runs one chunk ahead of the warps that read them back.
@@ -33,6 +33,11 @@
 // A warp reads the tensor-memory lanes of its own sub-partition (warp index mod 4), which hold
 // accumulator rows 16*(warp mod 4) .. +15 of a 64-row tile.
 // Every wait is bounded: on expiry the kernel raises a status flag and all roles leave.
+//
+// Two template parameters select variants of the same pipeline: SUMMARY (the first pass of a call
+// that splits its sequences into segments: state only, no r / scores / outputs; see Params) and C2
+// (the Finch-C2 form: keys times one minus their decay, no bonus, optional per-token vector added to
+// the output).
 #pragma once
 #include <atomic>
 #include <cuda.h>
