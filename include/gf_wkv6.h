@@ -93,6 +93,17 @@ GF_API gf_status_t gf_wkv6_prefill_c2(const void *r, const void *k, const void *
                                const void *u2, const float *state_in, float *state_out, void *y,
                                int B, int T, int H, int N, gf_stream_t stream);
 
+/* The Finch-C2 form of the packed variable-length prefill and of the decode step (bf16): arguments as for
+ * gf_wkv6_prefill_varlen / gf_wkv6_step with u2 (packed [total_T][H][N], resp. [B][H][N], bf16, or NULL) in
+ * place of u; semantics as for gf_wkv6_prefill_c2 (the k_t and o_t equations of the Finch-C2 block). */
+GF_API gf_status_t gf_wkv6_prefill_varlen_c2(const void *r, const void *k, const void *v, const void *x,
+                                      const void *u2, const float *state_in, float *state_out, void *y,
+                                      const int32_t *cu_seqlens, int S, int total_T, int max_seqlen,
+                                      int H, int N, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_step_c2(const void *r, const void *k, const void *v, const void *x, const void *u2,
+                            const float *state_in, float *state_out, void *y, int B, int H, int N,
+                            gf_stream_t stream);
+
 /* Same with fp32 r,k,v,x,y (token-by-token fp32 recurrence). */
 GF_API gf_status_t gf_wkv6_prefill_f32(const float *r, const float *k, const float *v, const float *x,
                                 const float *u, const float *state_in, float *state_out, float *y,

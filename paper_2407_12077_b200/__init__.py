@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
-    "prefill_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -33,6 +33,8 @@ _SIGNATURES = {
     "gf_wkv6_prefill_f32": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_static": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_c2": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
+    "gf_wkv6_prefill_varlen_c2": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
+    "gf_wkv6_step_c2": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
     "gf_wkv6_prefill_varlen": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_prefill_varlen_f32": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -206,6 +208,45 @@ def prefill_c2(r, k, v, x, u2=None, state_in=None, state_out=None, y=None, strea
         elif _workspace is not None:
             set_workspace(None)
         _check(lib.gf_wkv6_prefill_c2(*args, B, T, H, N, _stream(stream)), "gf_wkv6_prefill_c2")
+    return y, state_out
+
+
+def prefill_varlen_c2(r, k, v, x, u2, cu_seqlens, max_seqlen, state_in=None, state_out=None, y=None,
+                      stream=None, want_state=True):
+    """gf_wkv6_prefill_varlen_c2: packed Finch-C2 prefill.  r,k,v,x,u2 (u2 may be None): [total_T,H,N] bf16."""
+    lib = load_library()
+    total_T, H, N = r.shape
+    S = cu_seqlens.numel() - 1
+    bf = torch.bfloat16
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None and want_state:
+        state_out = torch.empty((S, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape),
+            _dev(u2, "u2", bf, r.shape), _dev(state_in, "state_in", torch.float32, (S, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (S, H, N, N)), _dev(y, "y", bf, r.shape),
+            _dev(cu_seqlens, "cu_seqlens", torch.int32)]
+    with torch.cuda.device(r.device):
+        _check(lib.gf_wkv6_prefill_varlen_c2(*args, S, total_T, int(max_seqlen), H, N, _stream(stream)),
+               "gf_wkv6_prefill_varlen_c2")
+    return y, state_out
+
+
+def step_c2(r, k, v, x, u2, state_in, state_out=None, y=None, stream=None):
+    """gf_wkv6_step_c2: one Finch-C2 decode token per sequence.  r,k,v,x,u2 (u2 may be None): [B,H,N] bf16;
+    state_out defaults to state_in (in-place update)."""
+    lib = load_library()
+    B, H, N = r.shape
+    bf = torch.bfloat16
+    if y is None:
+        y = torch.empty_like(r)
+    if state_out is None:
+        state_out = state_in if state_in is not None else torch.empty((B, H, N, N), device=r.device, dtype=torch.float32)
+    args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape),
+            _dev(u2, "u2", bf, r.shape), _dev(state_in, "state_in", torch.float32, (B, H, N, N)),
+            _dev(state_out, "state_out", torch.float32, (B, H, N, N)), _dev(y, "y", bf, r.shape)]
+    with torch.cuda.device(r.device):
+        _check(lib.gf_wkv6_step_c2(*args, B, H, N, _stream(stream)), "gf_wkv6_step_c2")
     return y, state_out
 
 

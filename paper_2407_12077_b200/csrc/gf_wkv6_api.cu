@@ -205,6 +205,48 @@ gf_status_t gf_wkv6_prefill_c2(const void* r, const void* k, const void* v, cons
                                (const bf*)u2, 1);
 }
 
+gf_status_t gf_wkv6_prefill_varlen_c2(const void* r, const void* k, const void* v, const void* x, const void* u2,
+                                      const float* state_in, float* state_out, void* y, const int32_t* cu_seqlens,
+                                      int S, int total_T, int max_seqlen, int H, int N, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (S < 0 || total_T < 0 || max_seqlen < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (max_seqlen > total_T) max_seqlen = total_T;
+    if (S == 0 || H == 0) return GF_OK;
+    if (!cu_seqlens || (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u)) return GF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (total_T == 0) return pass_state(state_in, state_out, (size_t)S * H, st);
+    if (!r || !k || !v || !x || !y) return GF_ERR_INVALID_ARG;
+    if (misaligned(r) || misaligned(k) || misaligned(v) || misaligned(x) || misaligned(u2) || misaligned(y) ||
+        misaligned(state_in) || misaligned(state_out))
+        return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x || y == u2) return GF_ERR_INVALID_ARG;
+    return gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, nullptr, state_in, state_out,
+                               (bf*)y, cu_seqlens, S, max_seqlen, (long long)total_T, H, st, &g_launches, nullptr, 0,
+                               (const bf*)u2, 1);
+}
+
+gf_status_t gf_wkv6_step_c2(const void* r, const void* k, const void* v, const void* x, const void* u2,
+                            const float* state_in, float* state_out, void* y, int B, int H, int N, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    if (!r || !k || !v || !x || !y) return GF_ERR_INVALID_ARG;
+    if (misaligned(r) || misaligned(k) || misaligned(v) || misaligned(x) || misaligned(u2) || misaligned(y) ||
+        misaligned(state_in) || misaligned(state_out))
+        return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x || y == u2) return GF_ERR_INVALID_ARG;
+    const long long units = (long long)B * H;
+    if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    gf::wkv6_step_kernel<bf, true><<<(unsigned)units, gf::ST_THREADS, 0, (cudaStream_t)stream>>>(
+        (const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, nullptr, state_in, state_out, (bf*)y, H, (const bf*)u2);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
 gf_status_t gf_wkv6_prefill_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
                                 const float* state_in, float* state_out, float* y, int B, int T, int H, int N,
                                 gf_stream_t stream)

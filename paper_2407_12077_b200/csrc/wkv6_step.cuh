@@ -6,7 +6,8 @@
 // columns 4*jq .. 4*jq+3 with 128-bit loads/stores (a warp covers two full 256-byte rows).
 // Column sums over the 16 row groups go through shared memory in a fixed order
 // (deterministic).  state_out may alias state_in: every element is read and written by
-// the same thread.
+// the same thread.  C2 = true is the Finch-C2 form: the key is multiplied by one minus its decay,
+// there is no bonus, and u2 (the token's second-value vector, may be NULL) is added to the output.
 #pragma once
 #include "wkv6_exact.cuh"
 
@@ -14,11 +15,12 @@ namespace gf {
 
 constexpr int ST_THREADS = 256;
 
-template <typename IO>
+template <typename IO, bool C2 = false>
 __global__ void __launch_bounds__(ST_THREADS)
 wkv6_step_kernel(const IO* __restrict__ r, const IO* __restrict__ k, const IO* __restrict__ v,
                  const IO* __restrict__ x, const float* __restrict__ u,
-                 const float* state_in, float* state_out, IO* __restrict__ y, int H)
+                 const float* state_in, float* state_out, IO* __restrict__ y, int H,
+                 const IO* __restrict__ u2 = nullptr)
 {
     __shared__ __align__(16) float rs[64], ks[64], vs[64], ws[64];
     __shared__ float ruk[2];
@@ -38,10 +40,12 @@ wkv6_step_kernel(const IO* __restrict__ r, const IO* __restrict__ k, const IO* _
                         : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (tid < 64) {
-        const float rr = to_f32(r[voff + tid]), kk = to_f32(k[voff + tid]);
+        const float rr = to_f32(r[voff + tid]);
+        const float ww = expf(-expf(to_f32(x[voff + tid])));
+        const float kk = C2 ? to_f32(k[voff + tid]) * (1.f - ww) : to_f32(k[voff + tid]);
         rs[tid] = rr; ks[tid] = kk; vs[tid] = to_f32(v[voff + tid]);
-        ws[tid] = expf(-expf(to_f32(x[voff + tid])));
-        float c = rr * u[h * 64 + tid] * kk;
+        ws[tid] = ww;
+        float c = C2 ? 0.f : rr * u[h * 64 + tid] * kk;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
         if ((tid & 31) == 0) ruk[tid >> 5] = c;
@@ -66,6 +70,7 @@ wkv6_step_kernel(const IO* __restrict__ r, const IO* __restrict__ k, const IO* _
         float s = (ruk[0] + ruk[1]) * vs[tid];
 #pragma unroll
         for (int q = 0; q < 16; ++q) s += part[q][tid];
+        if (C2 && u2) s += to_f32(u2[voff + tid]);
         y[voff + tid] = from_f32<IO>(s);
     }
 }

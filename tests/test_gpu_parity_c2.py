@@ -94,3 +94,41 @@ def test_c2_full_size_sampled_units():
         ey = orc.rel_l2(y[b, :, h].float().cpu().numpy(), y_ref[0, :, 0])
         es = orc.rel_l2(s[b, h].cpu().numpy(), s_ref[0, 0])
         assert ey <= TOL and es <= TOL, (b, h, ey, es)
+
+
+def test_c2_varlen_matches_per_sequence_oracle_including_empty_sequence():
+    lens = [5, 0, 64, 1, 130, 77, 63, 200]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    H = 3
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=830, state_std=0.1)
+    u2 = torch.randn(inp.r.shape, generator=torch.Generator().manual_seed(831)).bfloat16()
+    d = inp.to(DEV)
+    y = torch.full_like(d.r, 12345.0)
+    y, s = gf.prefill_varlen_c2(d.r, d.k, d.v, d.x, u2.to(DEV), d.cu_seqlens, max(lens), d.state_in, y=y)
+    gf.last_device_status()
+    for i, n in enumerate(lens):
+        a, b = int(cu[i]), int(cu[i + 1])
+        if n == 0:
+            assert torch.equal(s[i].cpu(), inp.state_in[i])
+            continue
+        sl = lambda t: t[a:b][None].contiguous()
+        y_ref, s_ref = orc.prefill_c2(sl(inp.r), sl(inp.k), sl(inp.v), sl(inp.x), sl(u2), inp.state_in[i][None].contiguous())
+        ey = orc.rel_l2(y[a:b].float().cpu().numpy(), y_ref[0])
+        es = orc.rel_l2(s[i].cpu().numpy(), s_ref[0])
+        assert ey <= TOL and es <= TOL, (i, n, ey, es)
+
+
+@pytest.mark.parametrize("with_u2", [True, False])
+def test_c2_step_matches_oracle_and_chains_to_a_prefill(with_u2):
+    B, H, T = 3, 5, 6
+    inp, u2 = make(B, T, H, 840, with_u2=with_u2)
+    d = inp.to(DEV)
+    u2d = None if u2 is None else u2.to(DEV)
+    st = d.state_in.clone()
+    ys = []
+    for t in range(T):
+        yt, st = gf.step_c2(d.r[:, t].contiguous(), d.k[:, t].contiguous(), d.v[:, t].contiguous(), d.x[:, t].contiguous(),
+                            None if u2d is None else u2d[:, t].contiguous(), st)
+        ys.append(yt)
+    gf.last_device_status()
+    check(torch.stack(ys, 1), st, inp, u2, f"chain of step_c2 u2={with_u2}")
