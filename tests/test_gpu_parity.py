@@ -160,6 +160,36 @@ def test_sequence_split_matches_oracle_and_unsplit_call(B, T, H, state_std, x_hi
     assert orc.rel_l2(s.cpu().numpy(), s1.cpu().numpy()) < 1e-3
 
 
+def test_random_shapes_and_decay_patterns_against_oracle():
+    """Seeded sweep over lengths (all residues of the ring and buffer depths), unit counts, initial states and
+    decay patterns, including sequences where only some chunks decay too fast for the tensor-core path."""
+    import random
+    rng = random.Random(20240712)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    for it in range(36):
+        B, H = rng.choice([1, 1, 2, 3]), rng.choice([1, 2, 3, 5])
+        T = rng.choice([rng.randint(1, 700), 64 * rng.randint(1, 14), 64 * rng.randint(1, 12) + 1, rng.randint(700, 1500)])
+        mode = rng.choice(["plain", "plain", "fast", "mixed", "patchy"])
+        inp = synth.make_dense(B, T, H, 64, "bf16", seed=5000 + it, state_std=rng.choice([0.0, 0.1]))
+        g = torch.Generator().manual_seed(6000 + it)
+        if mode == "fast":
+            inp.x = (torch.rand(inp.x.shape, generator=g) * 4 - 1).bfloat16()
+        elif mode == "mixed":
+            inp.x = (torch.rand(inp.x.shape, generator=g) * 16 - 8).bfloat16()
+        elif mode == "patchy":
+            xf = inp.x.float()
+            for c in range(0, T, 64):
+                if rng.random() < 0.3:
+                    xf[:, c:c + 64] = torch.rand(xf[:, c:c + 64].shape, generator=g) * 3 + 0.5
+            inp.x = xf.bfloat16()
+        d = inp.to(DEV)
+        y, s = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in, split=rng.choice([True, False]))
+        gf.last_device_status()
+        y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+        assert torch.isfinite(y.float()).all() and torch.isfinite(s).all()
+        check(y, s, y_ref, s_ref, 5e-3, f"case {it}: B{B} T{T} H{H} {mode}")
+
+
 def varlen_oracle_units(inp, cu, units):
     ys, ss = {}, {}
     for (s, h) in units:
