@@ -875,7 +875,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             tc_fence_after();
             const bool safe = safe_at(sd);
             float d_lo = 0.f, d_hi = 0.f;
-            if (safe) {
+            if (safe && !C2) {
                 const uint32_t du = sbase + OFF_DU + 4 * (sd * 64 + 16 * sp + g);
                 d_lo = ldsf(du); d_hi = ldsf(du + 32);
             }
@@ -1109,9 +1109,11 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     const float2 sra = ex2_2(pa), srb = ex2_2(pb);
                     const float2 r0 = bf_pair(rw[tt].x), r1 = bf_pair(rw[tt].y);
                     const float2 rh0 = mul2(r0, sra), rh1 = mul2(r1, srb);
-                    const float2 acc = fma2(mul2(r1, k1), ub, mul2(mul2(r0, k0), ua));
                     rw[tt] = make_uint2(pack_bf16(rh0.x, rh0.y), pack_bf16(rh1.x, rh1.y));
-                    du[tt] = acc.x + acc.y;
+                    if (!C2) {
+                        const float2 acc = fma2(mul2(r1, k1), ub, mul2(mul2(r0, k0), ua));
+                        du[tt] = acc.x + acc.y;
+                    }
                 }
                 pa = ca; pb = cb;
             }
@@ -1122,7 +1124,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             // reduce the 4 bonus partials over the 16 lanes of a half-warp (transposing butterfly):
             // lanes with bits (3,2) = (b8, b4) end with token 2*b8 + b4
-            if (!SUMMARY) {
+            if (!SUMMARY && !C2) {                       // (the Finch-C2 form has no bonus: the diagonal of P' is zero)
                 const bool b8 = lane & 8, b4 = lane & 4;
                 float w2[2], w1;
 #pragma unroll
