@@ -187,6 +187,23 @@ GF_API gf_status_t gf_wkv6_prefill_static(const void *r, const void *k, const vo
                                    const float *u, const float *state_in, float *state_out, void *y,
                                    int B, int T, int H, int N, gf_stream_t stream);
 
+/* Building blocks for splitting ONE sequence over several calls or several GPUs (sequence parallelism).
+ * Over a run of tokens the recurrence acts on the state as the affine map S -> diag(D) S + dS, D the
+ * product of the run's decays per key channel and dS the state the run reaches from zero (the wkv_t sum
+ * restricted to the run); these maps compose in sequence order.
+ * gf_wkv6_sequence_summary writes that pair for every (b,h) of a dense bf16 [B][T][H][N] run:
+ * summary is a DEVICE fp32 array [B][H][64 + 64*64], D first, then dS row-major ([i][j], i = key channel).
+ * It reads k, v, x only (c2 != 0: keys are multiplied by one minus their decay, as in gf_wkv6_prefill_c2).
+ * gf_wkv6_fold_summaries applies n_fold such summaries, laid out [n_fold][B][H][64 + 64*64] in sequence
+ * order, to state_in (NULL: zero) and writes the resulting [B][H][N][N] state to state_out (may alias
+ * state_in).  A rank that holds the p-th piece of a sequence gathers every rank's summary, folds the
+ * first p of them over the sequence's initial state and runs gf_wkv6_prefill on its piece with that start
+ * state; the last rank's state_out is the sequence's final state. */
+GF_API gf_status_t gf_wkv6_sequence_summary(const void *k, const void *v, const void *x, float *summary,
+                                     int B, int T, int H, int N, int c2, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_fold_summaries(const float *state_in, const float *summaries, int n_fold,
+                                   int B, int H, int N, float *state_out, gf_stream_t stream);
+
 /* Forces the kernel used by the bf16 prefill calls of this process (default
  * GF_KERNEL_AUTO).  Process-wide, not thread-safe against concurrent compute calls. */
 GF_API gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel);

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
-    "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -43,6 +43,8 @@ _SIGNATURES = {
     "gf_wkv6_host_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_set_workspace": (_i, [_vp, _sz]),
+    "gf_wkv6_sequence_summary": (_i, [_vp] * 4 + [_i] * 5 + [_vp]),
+    "gf_wkv6_fold_summaries": (_i, [_vp, _vp] + [_i] * 4 + [_vp, _vp]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
     "gf_wkv6_launch_count": (ctypes.c_uint64, []),
@@ -248,6 +250,38 @@ def step_c2(r, k, v, x, u2, state_in, state_out=None, y=None, stream=None):
     with torch.cuda.device(r.device):
         _check(lib.gf_wkv6_step_c2(*args, B, H, N, _stream(stream)), "gf_wkv6_step_c2")
     return y, state_out
+
+
+SUMMARY_FLOATS = 64 + 64 * 64         # per (b,h): decay product D[64], then dS[64][64]
+
+
+def sequence_summary(k, v, x, c2=False, out=None, stream=None):
+    """gf_wkv6_sequence_summary: (D, dS) of every (b,h) of a bf16 [B,T,H,N] run -> fp32 [B,H,64+4096]."""
+    lib = load_library()
+    B, T, H, N = k.shape
+    bf = torch.bfloat16
+    if out is None:
+        out = torch.empty((B, H, SUMMARY_FLOATS), device=k.device, dtype=torch.float32)
+    with torch.cuda.device(k.device):
+        _check(lib.gf_wkv6_sequence_summary(_dev(k, "k", bf), _dev(v, "v", bf, k.shape), _dev(x, "x", bf, k.shape),
+                                            _dev(out, "summary", torch.float32, (B, H, SUMMARY_FLOATS)), B, T, H, N,
+                                            1 if c2 else 0, _stream(stream)), "gf_wkv6_sequence_summary")
+    return out
+
+
+def fold_summaries(state_in, summaries, n_fold, state_out=None, stream=None):
+    """gf_wkv6_fold_summaries: apply the first n_fold of summaries [P,B,H,64+4096] to state_in ([B,H,N,N] or None)."""
+    lib = load_library()
+    P, B, H, F = summaries.shape
+    assert F == SUMMARY_FLOATS and 0 <= n_fold <= P
+    if state_out is None:
+        state_out = torch.empty((B, H, 64, 64), device=summaries.device, dtype=torch.float32)
+    with torch.cuda.device(summaries.device):
+        _check(lib.gf_wkv6_fold_summaries(_dev(state_in, "state_in", torch.float32, (B, H, 64, 64)),
+                                          _dev(summaries, "summaries", torch.float32), int(n_fold), B, H, 64,
+                                          _dev(state_out, "state_out", torch.float32, (B, H, 64, 64)), _stream(stream)),
+               "gf_wkv6_fold_summaries")
+    return state_out
 
 
 STATIC_SCRATCH_BYTES = 1597440       # GF_WKV6_STATIC_SCRATCH_BYTES

@@ -247,6 +247,35 @@ gf_status_t gf_wkv6_step_c2(const void* r, const void* k, const void* v, const v
     return launch_result();
 }
 
+gf_status_t gf_wkv6_sequence_summary(const void* k, const void* v, const void* x, float* summary, int B, int T, int H,
+                                     int N, int c2, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    if (T == 0 || (long long)B * T >= (1LL << 31)) return GF_ERR_INVALID_ARG;
+    if (!k || !v || !x || !summary || misaligned(k) || misaligned(v) || misaligned(x) || misaligned(summary))
+        return GF_ERR_INVALID_ARG;
+    return gf::chunked_summary((const bf*)k, (const bf*)v, (const bf*)x, summary, B, T, H, c2 != 0, (cudaStream_t)stream,
+                               &g_launches);
+}
+
+gf_status_t gf_wkv6_fold_summaries(const float* state_in, const float* summaries, int n_fold, int B, int H, int N,
+                                   float* state_out, gf_stream_t stream)
+{
+    if (B < 0 || H < 0 || N < 0 || n_fold < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    if (!state_out || (n_fold > 0 && !summaries) || misaligned(state_in) || misaligned(state_out) || misaligned(summaries))
+        return GF_ERR_INVALID_ARG;
+    const long long units = (long long)B * H;
+    if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    gf::wkv6_fold_kernel<<<(unsigned)units, 256, 0, (cudaStream_t)stream>>>(state_in, summaries, n_fold, units, state_out);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
 gf_status_t gf_wkv6_prefill_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
                                 const float* state_in, float* state_out, float* y, int B, int T, int H, int N,
                                 gf_stream_t stream)

@@ -1023,7 +1023,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int cq = lane & 15, th = lane >> 4;        // channels 4*cq .. 4*cq+3, tokens 8*tq + 4*th + (0..3)
         const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
         constexpr bool c2 = C2;                          // Finch-C2 form: keys times (1 - w), no bonus
-        const float4 u4 = c2 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
+        // (the bonus vector is only read where the bonus is computed: not in the Finch-C2 form, not in a summary pass)
+        const float4 u4 = (c2 || SUMMARY) ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
         const float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
         uint32_t roff[4];                                // swizzled byte offsets of this lane's 8 bytes in its 4 rows
 #pragma unroll
@@ -1286,6 +1287,52 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     else ck::wkv6_chunked_kernel<false, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+// Summary of whole sequences (the pair of the affine map S -> diag(D) S + dS that a sequence applies to
+// the state): one summary launch with a single segment per unit.  summary: [n_seq*H][64 + 64*64] fp32.
+inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x, float* summary,
+                                   int n_seq, int T, int H, int c2, cudaStream_t st, std::atomic<uint64_t>* launches)
+{
+    const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
+    if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
+    if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+        cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+        return GF_ERR_CUDA;
+    CUtensorMap tk, tv, tx, tdummy;
+    const long long C = (long long)H * 64;
+    if (!ck::make_map(&tk, k, total_rows, C, 64) || !ck::make_map(&tv, v, total_rows, C, 64) ||
+        !ck::make_map(&tx, x, total_rows, C, 64) || !ck::make_map(&tdummy, k, total_rows, C, 16))
+        return GF_ERR_CUDA;
+    // two nominal segments of which the first covers the whole sequence: the summary launch handles
+    // every segment but the last
+    ck::Params p{nullptr, k, v, x, nullptr, nullptr, nullptr, nullptr, nullptr, T, H, summary, (T + ck::L - 1) / ck::L, 2, nullptr, c2};
+    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+// out[unit] = fold of n_fold summaries over state_in[unit] (or zero): S <- diag(D_p) S + dS_p for p = 0 .. n_fold-1,
+// summaries laid out [p][unit][64 + 4096].  One CTA of 256 threads per unit; thread t owns columns of 16 rows.
+__global__ void __launch_bounds__(256)
+wkv6_fold_kernel(const float* __restrict__ state_in, const float* __restrict__ summaries, int n_fold, long long units,
+                 float* __restrict__ out)
+{
+    const long long unit = blockIdx.x;
+    const int j = threadIdx.x & 63, ig = threadIdx.x >> 6;             // rows 16*ig .. 16*ig+15, column j
+    float S[16];
+#pragma unroll
+    for (int ii = 0; ii < 16; ++ii)
+        S[ii] = state_in ? state_in[unit * 4096 + (size_t)(16 * ig + ii) * 64 + j] : 0.f;
+    for (int pi = 0; pi < n_fold; ++pi) {
+        const float* sm = summaries + ((size_t)pi * units + unit) * ck::SUMMARY_FLOATS;
+#pragma unroll
+        for (int ii = 0; ii < 16; ++ii)
+            S[ii] = fmaf(sm[16 * ig + ii], S[ii], sm[64 + (size_t)(16 * ig + ii) * 64 + j]);
+    }
+#pragma unroll
+    for (int ii = 0; ii < 16; ++ii) out[unit * 4096 + (size_t)(16 * ig + ii) * 64 + j] = S[ii];
 }
 
 }  // namespace gf
