@@ -338,10 +338,11 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in/out, fp32 state and accumulation",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": f"cfg2: {calls} x gf_wkv6_prefill B={B} T={T} H={H} N={N}, bf16 r/k/v/x/y, "
                                    f"fp32 u/state, independent seeds per call",
+                       "precision": "bf16 r/k/v/x/y and tensor-core operands, fp32 accumulation, decay sums and state",
                        "l2": "inputs larger than L2 (1.34 GB per call, distinct buffers per call)",
                        "parallelism": f"(b,h) units replicated per GPU x{world}, no collective"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
