@@ -1,0 +1,150 @@
+"""Runs one of the benchmark configurations of the WKV-6 library a few times on the current CUDA device and
+prints one JSON line per case with CUDA-event timings (inputs resident in HBM, seeded synthetic data).
+
+    python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
+
+cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg4-prefill cfg4-decode
+--scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
+
+`bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
+traffic over the time, relative to ``--peak-gbs`` (default: the measured copy bandwidth recorded in
+MEASURED_PEAKS.json at the repository root when present, else 6650 GB/s).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+import paper_2407_12077_b200 as gf
+from paper_2407_12077_b200 import synth
+
+DEV = "cuda:0"
+
+
+def _peak(default=6650.0):
+    p = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"])
+    except Exception:
+        return default
+
+
+def _time(fn, reps):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    gf.last_device_status()
+    return e0.elapsed_time(e1) / reps
+
+
+def _dense(name, B, T, H, dtype, state_std, reps, c2=False):
+    inp = synth.make_dense(B, T, H, 64, dtype, seed=7, device=DEV, state_std=state_std)
+    y = torch.empty_like(inp.r)
+    s = torch.empty((B, H, 64, 64), device=DEV)
+    esz = 2 if dtype == "bf16" else 4
+    nbytes = B * T * H * 64 * esz * 5 + B * H * 16384 * (2 if state_std > 0 else 1)
+    if c2:
+        u2 = torch.randn(inp.r.shape, device=DEV).bfloat16()
+        nbytes += B * T * H * 128
+        fn = lambda: gf.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in, state_out=s, y=y)
+    else:
+        fn = lambda: gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in, state_out=s, y=y)
+    return dict(case=name, shape=f"B={B} T={T} H={H} {dtype}", units=B * T * H, bytes=nbytes, ms=_time(fn, reps))
+
+
+def run(case, reps, scale):
+    c = synth.CONFIGS
+    sc = lambda t: max(64, int(t * scale) // 64 * 64)
+    if case == "cfg0":
+        k = c["cfg0"]
+        return _dense(case, k["B"], k["T"], k["H"], "f32", 0.0, reps)
+    if case == "cfg1":
+        k = c["cfg1"]
+        return _dense(case, k["B"], sc(k["T"]), k["H"], "bf16", 0.1, reps)
+    if case in ("cfg2", "cfg2-c2"):
+        k = c["cfg2"]
+        return _dense(case, k["B"], sc(k["T"]), k["H"], "bf16", 0.0, reps, c2=case.endswith("c2"))
+    if case == "cfg3":                      # one call over the whole context (splits into segments internally)
+        k = c["cfg3"]
+        return _dense(case, 1, sc(k["T"]), k["H"], "bf16", 0.0, reps)
+    if case == "cfg3-segments":             # 8 calls with the state carried from one to the next
+        k = c["cfg3"]
+        T, H, nseg = sc(k["T"]), k["H"], k["segments"]
+        inp = synth.make_dense(1, T, H, 64, "bf16", seed=7, device=DEV)
+        seg = T // nseg
+        parts = [tuple(t[:, i * seg:(i + 1) * seg].contiguous() for t in (inp.r, inp.k, inp.v, inp.x)) for i in range(nseg)]
+        ys = [torch.empty_like(p[0]) for p in parts]
+        st = torch.zeros((1, H, 64, 64), device=DEV)
+
+        def fn():
+            state = None
+            for (r, kk, v, x), y in zip(parts, ys):
+                _, state = gf.prefill(r, kk, v, x, inp.u, state, state_out=st, y=y)
+
+        return dict(case=case, shape=f"B=1 T={nseg}x{seg} H={H} bf16", units=T * H, bytes=T * H * 640 + nseg * 2 * H * 16384,
+                    ms=_time(fn, reps))
+    if case in ("cfg4-prefill", "cfg4-decode"):
+        k = c["cfg4"]
+        S, H = k["S"], k["H"]
+        cu = synth.make_lengths(S, max(1, int(k["len_min"] * scale)), max(2, int(k["len_max"] * scale)), seed=4000)
+        if case == "cfg4-prefill":
+            inp = synth.make_varlen(cu, H, 64, "bf16", seed=4001, device=DEV, state_std=k["state_std"])
+            total, mx = int(cu[-1]), int((cu[1:] - cu[:-1]).max())
+            y = torch.empty_like(inp.r)
+            s = torch.empty((S, H, 64, 64), device=DEV)
+            fn = lambda: gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, mx, inp.state_in, state_out=s, y=y)
+            return dict(case=case, shape=f"S={S} total_T={total} H={H} bf16", units=total * H,
+                        bytes=total * H * 640 + 2 * S * H * 16384, ms=_time(fn, reps))
+        d = synth.make_step(S, H, 64, "bf16", seed=4002, device=DEV)
+        y = torch.empty_like(d.r)
+        steps = 64
+        g = torch.cuda.CUDAGraph()                       # a decode loop replays a captured step sequence
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            gf.step(d.r, d.k, d.v, d.x, d.u, d.state_in, y=y, stream=st)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=st):
+                for _ in range(steps):
+                    gf.step(d.r, d.k, d.v, d.x, d.u, d.state_in, y=y, stream=st)
+        ms = _time(g.replay, reps) / steps
+        return dict(case=case, shape=f"S={S} H={H} bf16, {steps} steps per graph replay, state updated in place",
+                    units=S * H, bytes=S * H * (2 * 16384 + 5 * 128), ms=ms)
+    raise SystemExit(f"unknown case {case}")
+
+
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg4-prefill", "cfg4-decode"]
+
+
+def main():
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("cases", nargs="+")
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--peak-gbs", type=float, default=None)
+    a = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device: the library has no CPU path")
+    gf.load_library()
+    peak = a.peak_gbs or _peak()
+    for case in (ALL if a.cases == ["all"] else a.cases):
+        r = run(case, a.reps, a.scale)
+        r["units_per_s"] = r["units"] / (r["ms"] * 1e-3)
+        r["gbs"] = r["bytes"] / (r["ms"] * 1e-3) / 1e9
+        r["frac"] = r["gbs"] / peak
+        r["peak_gbs"] = peak
+        print(json.dumps(r), flush=True)
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    sys.exit(main())
