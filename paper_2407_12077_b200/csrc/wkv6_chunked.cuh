@@ -927,7 +927,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // one chunk ahead (requested as soon as the previous chunk's rows have been read out of it)
         const bool has_u2 = !SUMMARY && C2 && p.u2 != nullptr;
         const uint32_t u2slab = sbase + OFF_U2 + sp * 2048;
-        bool u2_pending = false;
+        bool u2_pending = false;                 // a slab copy is in flight; it completes the phase of parity u2_parity
+        int u2_parity = 0;
         auto load_u2 = [&](int c) {
             if (elect_one()) {
                 mbar_expect_tx(bar(BAR_U2 + sp), 2048);
@@ -939,6 +940,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             __syncwarp();
             u2_pending = true;
+            u2_parity = c & 1;
         };
         if (has_u2 && nchunks > 0) load_u2(0);
         for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
@@ -1015,7 +1017,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         if (lane == 0) bulk_wait<0>();
         // leaving early (abort) with a slab copy still in flight: wait for it, it targets this CTA's memory
-        if (u2_pending) mbar_wait(bar(BAR_U2 + sp), 0, abort_flag, false) || mbar_wait(bar(BAR_U2 + sp), 1, abort_flag, false);
+        if (u2_pending) mbar_wait(bar(BAR_U2 + sp), u2_parity, abort_flag, false);
     } else {
         // ============================== elementwise warps ==============================
         const int eset = (warp - WARP_E0) / N_EW;        // this set takes chunks eset, eset + 2, ...
