@@ -15,7 +15,7 @@ import torch
 from . import _build
 
 __all__ = [
-    "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step",
+    "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
     "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
@@ -342,6 +342,34 @@ def step(r, k, v, x, u, state_in, state_out=None, y=None, stream=None):
     with torch.cuda.device(r.device):
         _check(getattr(lib, "gf_wkv6_step" + sfx)(*args, B, H, N, _stream(stream)), "gf_wkv6_step" + sfx)
     return y, state_out
+
+
+def bind_step(r, k, v, x, u, state, y=None, stream=None):
+    """Pre-marshalled decode step for loops that reuse the same buffers (the caller refreshes r,k,v,x in
+    place every token, the state is updated in place): checks and pointer extraction happen once here, the
+    returned zero-argument callable is one C call.  Returns (callable, y)."""
+    lib = load_library()
+    B, H, N = r.shape
+    sfx = _suffix(r.dtype)
+    if y is None:
+        y = torch.empty_like(r)
+    args = [_dev(r, "r"), _dev(k, "k", r.dtype, r.shape), _dev(v, "v", r.dtype, r.shape),
+            _dev(x, "x", r.dtype, r.shape), _dev(u, "u", torch.float32, (H, N)),
+            _dev(state, "state", torch.float32, (B, H, N, N)), _dev(state, "state", torch.float32, (B, H, N, N)),
+            _dev(y, "y", r.dtype, r.shape), B, H, N, _stream(stream)]
+    fn = getattr(lib, "gf_wkv6_step" + sfx)
+    keep = (r, k, v, x, u, state, y)                 # the bound buffers must outlive the callable
+    index = r.device.index
+
+    def call():
+        if torch.cuda.current_device() != index:
+            raise RuntimeError("bind_step: the bound tensors' device is not the current device")
+        status = fn(*args)
+        if status != GF_OK:
+            raise GfError(status, "gf_wkv6_step" + sfx)
+
+    call.buffers = keep
+    return call, y
 
 
 def host_workspace_bytes(B, T, H, N) -> int:

@@ -276,6 +276,24 @@ def test_step_matches_oracle_and_prefill_of_length_one(dtype):
     check(y1[:, 0], s1, y_ref, s_ref, TOL[inp.r.dtype], "prefill T=1")
 
 
+def test_bound_step_loop_matches_oracle():
+    """The pre-marshalled decode step over reused buffers (refreshed in place every token)."""
+    B, H, T = 3, 4, 12
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=650, state_std=0.1)
+    d = inp.to(DEV)
+    r, k, v, x = (torch.empty((B, H, 64), device=DEV, dtype=torch.bfloat16) for _ in range(4))
+    state = d.state_in.clone()
+    call, y = gf.bind_step(r, k, v, x, d.u, state)
+    ys = []
+    for t in range(T):
+        r.copy_(d.r[:, t]); k.copy_(d.k[:, t]); v.copy_(d.v[:, t]); x.copy_(d.x[:, t])
+        call()
+        ys.append(y.clone())
+    gf.last_device_status()
+    y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+    check(torch.stack(ys, 1), state, y_ref, s_ref, 5e-3, "bound step loop")
+
+
 def test_prefill_equals_chain_of_steps():
     B, T, H = 2, 40, 2
     inp = synth.make_dense(B, T, H, 64, "f32", seed=600, state_std=0.1)
