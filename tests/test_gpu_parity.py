@@ -190,6 +190,22 @@ def test_random_shapes_and_decay_patterns_against_oracle():
         check(y, s, y_ref, s_ref, 5e-3, f"case {it}: B{B} T{T} H{H} {mode}")
 
 
+def test_quarter_million_tokens_one_head():
+    """One (b,h) unit of 262144 tokens: 4096 chunks cut into 8 segments (every barrier phase and ring slot
+    wraps hundreds of times); the fp32 state must stay on the oracle's over the whole length."""
+    T = 262144
+    inp = synth.make_dense(1, T, 1, 64, "bf16", seed=7000, device=DEV)
+    assert gf.workspace_bytes(1, T, 1, 64) == 7 * (64 + 4096) * 4
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    y, s = gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, None)
+    gf.last_device_status()
+    cpu = inp.to("cpu")
+    y_ref, s_ref = orc.prefill(cpu.r, cpu.k, cpu.v, cpu.x, cpu.u, None)
+    check(y, s, y_ref, s_ref, 5e-3, "T=262144")
+    # and the tail of the sequence on its own, where an error in a carried state would show
+    check(y[:, -4096:], None, y_ref[:, -4096:], None, 5e-3, "last 4096 tokens")
+
+
 def varlen_oracle_units(inp, cu, units):
     ys, ss = {}, {}
     for (s, h) in units:
