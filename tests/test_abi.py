@@ -99,3 +99,32 @@ def test_binding_refuses_cpu_tensors():
     u = torch.zeros((1, 64))
     with pytest.raises(ValueError):
         gf.prefill(t, t, t, t, u, y=t.clone(), state_out=torch.zeros(1, 1, 64, 64))
+
+
+def test_later_entry_points_reject_bad_arguments_before_any_launch():
+    ptrs = [A + 0x100 * i for i in range(8)]
+    for name in ("gf_wkv6_prefill_c2", "gf_wkv6_prefill_static"):
+        assert _call(name, *ptrs, 1, 8, 1, 32, None) == 2                     # head size
+        assert _call(name, *ptrs, -1, 8, 1, 64, None) == 1                    # negative size
+        assert _call(name, *ptrs, 0, 8, 1, 64, None) == 0                     # empty: legal no-op
+        p = list(ptrs); p[0] = None
+        assert _call(name, *p, 1, 8, 1, 64, None) == 1                        # NULL r
+        p = list(ptrs); p[7] = p[1]
+        assert _call(name, *p, 1, 8, 1, 64, None) == 1                        # y aliases k
+    p = list(ptrs); p[4] = A + 2
+    assert _call("gf_wkv6_prefill_c2", *p, 1, 8, 1, 64, None) == 1            # misaligned u2
+    assert _call("gf_wkv6_prefill_varlen_c2", *ptrs, None, 2, 8, 8, 1, 64, None) == 1
+    assert _call("gf_wkv6_prefill_varlen_c2", *ptrs, A, 0, 0, 0, 4, 64, None) == 0
+    assert _call("gf_wkv6_step_c2", *ptrs, 1, 1, 128, None) == 2
+    assert _call("gf_wkv6_step_c2", *ptrs, 0, 4, 64, None) == 0
+    # summaries
+    assert _call("gf_wkv6_sequence_summary", A, A, A, A, 1, 8, 1, 32, 0, None) == 2
+    assert _call("gf_wkv6_sequence_summary", A, A, A, None, 1, 8, 1, 64, 0, None) == 1
+    assert _call("gf_wkv6_sequence_summary", A, A, A, A, 1, 0, 1, 64, 0, None) == 1      # a summary of nothing is not defined here
+    assert _call("gf_wkv6_fold_summaries", None, None, 2, 1, 1, 64, A, None) == 1
+    assert _call("gf_wkv6_fold_summaries", None, A, -1, 1, 1, 64, A, None) == 1
+    assert _call("gf_wkv6_fold_summaries", None, A, 1, 0, 1, 64, A, None) == 0
+    # workspace registration
+    assert _call("gf_wkv6_set_workspace", A + 8, 1 << 20) == 1                # not 256-byte aligned
+    assert _call("gf_wkv6_set_workspace", None, 0) == 0
+    assert gf.workspace_bytes(1, 100000, 32, 48) == 0
