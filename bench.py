@@ -274,13 +274,15 @@ def main():
     value = whole_job_value(B * T * H * calls, world, ms_per_step)
 
     # ---- roofline of the dominant kernel (one prefill launch) from the live per-launch events
-    launch_ms = statistics.mean(a.elapsed_time(b) for a, b in kernel_events)
+    per_launch = [a.elapsed_time(b) for a, b in kernel_events]
+    launch_ms = statistics.mean(per_launch)
     alg_bytes = B * T * H * BYTES_PER_TOKEN_HEAD + B * H * STATE_BYTES_PER_UNIT
     peak, peak_kind = measured_peaks()
     achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
-                "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms, "algorithmic_bytes": alg_bytes}
+                "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms, "launch_ms_median": statistics.median(per_launch),
+                "launch_ms_min": min(per_launch), "launch_ms_max": max(per_launch), "algorithmic_bytes": alg_bytes}
 
     # ---- end to end through the host-buffer entry point: pinned host inputs -> y on the host
     e2e = None
