@@ -114,7 +114,10 @@ GF_API gf_status_t gf_wkv6_prefill_f32(const float *r, const float *k, const flo
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a
  * DEVICE int32 array of S+1 non-decreasing entries with cu_seqlens[0] = 0 and
  * cu_seqlens[S] = total_T (the caller guarantees this; it is not read on the host).
- * max_seqlen is an upper bound on any sequence length.  States are [S][H][N][N]. */
+ * max_seqlen is an upper bound on any sequence length.  States are [S][H][N][N].
+ * A bf16 call with few (sequence, head) units takes the sequence split described at
+ * gf_wkv6_set_workspace, cut by max_seqlen: gf_wkv6_workspace_bytes(S, max_seqlen, H, N) is the
+ * scratch it uses, and segments that lie past a sequence's end do no work. */
 GF_API gf_status_t gf_wkv6_prefill_varlen(const void *r, const void *k, const void *v, const void *x,
                                    const float *u, const float *state_in, float *state_out,
                                    void *y, const int32_t *cu_seqlens, int S, int total_T,
@@ -148,15 +151,15 @@ GF_API gf_status_t gf_wkv6_prefill_host(const void *r, const void *k, const void
                                  gf_stream_t stream);
 GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
 
-/* Optional scratch for dense bf16 prefill calls with few (sequence, head) units.  One CTA walks one
+/* Optional scratch for bf16 prefill calls (dense or packed) with few (sequence, head) units.  One CTA walks one
  * unit's sequence, so a call with fewer units than half the GPU's SMs (long-context prefill of one
  * sequence) would leave most SMs idle.  With a workspace registered such a call cuts every sequence
  * into up to 8 segments: a first launch carries the state over each segment from a zero start and
  * leaves per segment its decay product and state increment (the pair (D, dS) of the recurrence
  * S <- diag(D) S + dS, which composes associatively across segments of the wkv_t sum) in the workspace,
  * the second launch folds them into each segment's start state and computes y.  Results agree with the
- * unsplit call to rounding.  gf_wkv6_workspace_bytes returns what gf_wkv6_prefill(B,T,H,N) would use on
- * the current device (0: the call does not split).  gf_wkv6_set_workspace registers a caller-owned
+ * unsplit call to rounding.  gf_wkv6_workspace_bytes returns what gf_wkv6_prefill(B,T,H,N) (packed:
+ * B = S, T = max_seqlen) would use on the current device (0: the call does not split).  gf_wkv6_set_workspace registers a caller-owned
  * DEVICE buffer (256-byte aligned; NULL unregisters) for all later calls of this process; the library
  * never frees it.  A registered buffer that is too small is ignored (the call runs unsplit).  Calls that
  * use the workspace and overlap on the GPU (different streams) race on it. */

@@ -214,7 +214,7 @@ def prefill_c2(r, k, v, x, u2=None, state_in=None, state_out=None, y=None, strea
 
 
 def prefill_varlen_c2(r, k, v, x, u2, cu_seqlens, max_seqlen, state_in=None, state_out=None, y=None,
-                      stream=None, want_state=True):
+                      stream=None, want_state=True, split=True):
     """gf_wkv6_prefill_varlen_c2: packed Finch-C2 prefill.  r,k,v,x,u2 (u2 may be None): [total_T,H,N] bf16."""
     lib = load_library()
     total_T, H, N = r.shape
@@ -229,6 +229,10 @@ def prefill_varlen_c2(r, k, v, x, u2, cu_seqlens, max_seqlen, state_in=None, sta
             _dev(state_out, "state_out", torch.float32, (S, H, N, N)), _dev(y, "y", bf, r.shape),
             _dev(cu_seqlens, "cu_seqlens", torch.int32)]
     with torch.cuda.device(r.device):
+        if split:
+            _ensure_workspace(S, int(max_seqlen), H, N, r.device)
+        elif _workspace is not None:
+            set_workspace(None)
         _check(lib.gf_wkv6_prefill_varlen_c2(*args, S, total_T, int(max_seqlen), H, N, _stream(stream)),
                "gf_wkv6_prefill_varlen_c2")
     return y, state_out
@@ -303,9 +307,9 @@ def prefill_static(r, k, v, x, u, state_in, state_out, y, stream=None) -> None:
 
 
 def prefill_varlen(r, k, v, x, u, cu_seqlens, max_seqlen, state_in=None, state_out=None, y=None,
-                   stream=None, want_state=True):
+                   stream=None, want_state=True, split=True):
     """gf_wkv6_prefill_varlen(_f32).  r,k,v,x: [total_T,H,N]; cu_seqlens: int32 CUDA [S+1];
-    states [S,H,N,N].  Returns (y, state_out)."""
+    states [S,H,N,N].  Returns (y, state_out).  split as for prefill (cut by max_seqlen)."""
     lib = load_library()
     total_T, H, N = r.shape
     S = cu_seqlens.numel() - 1
@@ -320,6 +324,10 @@ def prefill_varlen(r, k, v, x, u, cu_seqlens, max_seqlen, state_in=None, state_o
             _dev(state_out, "state_out", torch.float32, (S, H, N, N)), _dev(y, "y", r.dtype, r.shape),
             _dev(cu_seqlens, "cu_seqlens", torch.int32)]
     with torch.cuda.device(r.device):
+        if sfx == "" and split:
+            _ensure_workspace(S, int(max_seqlen), H, N, r.device)
+        elif not split and _workspace is not None:
+            set_workspace(None)
         _check(getattr(lib, "gf_wkv6_prefill_varlen" + sfx)(*args, S, total_T, int(max_seqlen), H, N, _stream(stream)),
                "gf_wkv6_prefill_varlen" + sfx)
     return y, state_out

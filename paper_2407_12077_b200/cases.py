@@ -3,7 +3,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
 
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
-cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg4-prefill cfg4-decode
+cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -93,6 +93,16 @@ def run(case, reps, scale):
 
         return dict(case=case, shape=f"B=1 T={nseg}x{seg} H={H} bf16", units=T * H, bytes=T * H * 640 + nseg * 2 * H * 16384,
                     ms=_time(fn, reps))
+    if case == "cfg3-packed":               # two long contexts of different lengths in one packed call (split by max_seqlen)
+        k = c["cfg3"]
+        H, lens = k["H"], [sc(k["T"]), sc(k["T"] * 3 // 8) + 37]
+        cu = torch.tensor([0, lens[0], lens[0] + lens[1]], dtype=torch.int32)
+        inp = synth.make_varlen(cu, H, 64, "bf16", seed=3001, device=DEV, state_std=0.0)
+        y = torch.empty_like(inp.r)
+        s = torch.empty((2, H, 64, 64), device=DEV)
+        fn = lambda: gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, max(lens), None, state_out=s, y=y)
+        return dict(case=case, shape=f"S=2 lens={lens} H={H} bf16", units=sum(lens) * H,
+                    bytes=sum(lens) * H * 640 + 2 * H * 16384, ms=_time(fn, reps))
     if case in ("cfg4-prefill", "cfg4-decode"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -125,7 +135,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg4-prefill", "cfg4-decode"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode"]
 
 
 def main():

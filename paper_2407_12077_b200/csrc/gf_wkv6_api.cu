@@ -124,7 +124,8 @@ gf_status_t prefill_varlen(const IO* r, const IO* k, const IO* v, const IO* x, c
         s = gf::chunked_prefill(reinterpret_cast<const __nv_bfloat16*>(r), reinterpret_cast<const __nv_bfloat16*>(k),
                                 reinterpret_cast<const __nv_bfloat16*>(v), reinterpret_cast<const __nv_bfloat16*>(x),
                                 u, state_in, state_out, reinterpret_cast<__nv_bfloat16*>(y), cu,
-                                S, max_seqlen, (long long)total_T, H, st, &g_launches);
+                                S, max_seqlen, (long long)total_T, H, st, &g_launches,
+                                g_ws.load(std::memory_order_relaxed), g_ws_bytes.load(std::memory_order_relaxed));
         if (s != GF_ERR_UNSUPPORTED || sel == GF_KERNEL_CHUNKED) return s;
     }
     return run_exact<IO>(r, k, v, x, u, state_in, state_out, y, cu, S, max_seqlen, H, st);
@@ -223,7 +224,8 @@ gf_status_t gf_wkv6_prefill_varlen_c2(const void* r, const void* k, const void* 
         return GF_ERR_INVALID_ARG;
     if (y == r || y == k || y == v || y == x || y == u2) return GF_ERR_INVALID_ARG;
     return gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, nullptr, state_in, state_out,
-                               (bf*)y, cu_seqlens, S, max_seqlen, (long long)total_T, H, st, &g_launches, nullptr, 0,
+                               (bf*)y, cu_seqlens, S, max_seqlen, (long long)total_T, H, st, &g_launches,
+                               g_ws.load(std::memory_order_relaxed), g_ws_bytes.load(std::memory_order_relaxed),
                                (const bf*)u2, 1);
 }
 

@@ -1220,8 +1220,9 @@ inline int sm_count()
     return cached;
 }
 
-// Chooses the sequence split of a dense call: with fewer (sequence, head) units than half the SMs, each
-// sequence is cut into up to 8 segments of at least 8 chunks so that the grid fills the GPU.  Returns the
+// Chooses the sequence split of a call: with fewer (sequence, head) units than half the SMs, each
+// sequence is cut into up to 8 segments of at least 8 chunks so that the grid fills the GPU (T: the
+// sequence length, for a packed call the longest one).  Returns the
 // number of segments (1: no split) and sets seg_chunks; summary_bytes is the scratch the split needs.
 inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_t* summary_bytes)
 {
@@ -1242,7 +1243,7 @@ inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_
 }
 
 // Launches the chunked kernel.  Dense: cu == nullptr, n_seq = B, T = sequence length.
-// Packed: cu = device cu_seqlens, n_seq = S, T unused.  total_rows = rows of the [rows][H*64] tensors.
+// Packed: cu = device cu_seqlens, n_seq = S, T = max_seqlen.  total_rows = rows of the [rows][H*64] tensors.
 // scratch / scratch_bytes: optional device memory for the sequence split (see choose_split); without
 // enough of it the call runs unsplit.
 inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
@@ -1273,7 +1274,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         !ck::make_map(&ty, y, total_rows, C, 16) || !ck::make_map(&tu2, u2 ? (const void*)u2 : (const void*)y, total_rows, C, 16))
         return GF_ERR_CUDA;
     int seg_chunks = 0, nseg = 1;
-    if (!cu && scratch) {
+    if (scratch) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
         size_t need = 0;
         nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);
         if (nseg > 1 && (need > scratch_bytes || units * nseg > 0x7fffffffLL)) nseg = 1;

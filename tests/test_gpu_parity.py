@@ -242,6 +242,34 @@ def test_varlen_small_full_including_empty_sequence(kernel, dtype):
     assert torch.equal(s[1].cpu(), inp.state_in[1])                 # empty sequence: state passes through
 
 
+@pytest.mark.parametrize("lens,H,x_hi", [([3000, 1100], 4, -1.0), ([517, 0, 2600, 64], 3, -1.0), ([1500, 2304], 2, 2.5),
+                                         ([4096], 8, -1.0)])
+def test_varlen_sequence_split_matches_oracle_and_unsplit_call(lens, H, x_hi):
+    """Packed call with few (sequence, head) units: sequences are cut by max_seqlen, so the shorter ones
+    own empty segments (identity summaries) and the last segment of each still writes the final state."""
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    assert gf.workspace_bytes(len(lens), max(lens), H, 64) > 0, "this shape is expected to split"
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=4400 + H, state_std=0.1, x_lo=-6.0 if x_hi < 0 else -1.0, x_hi=x_hi)
+    d = inp.to(DEV)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    before = gf.launch_count()
+    y, s = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in)
+    assert gf.launch_count() - before == 2
+    y1, s1 = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in, split=False)
+    assert gf.launch_count() - before == 3
+    gf.last_device_status()
+    y_ref, s_ref = orc.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, cu, inp.state_in)
+    check(y, s, y_ref, s_ref, 5e-3, "packed split")
+    check(y1, s1, y_ref, s_ref, 5e-3, "packed unsplit")
+    for i in range(len(lens)):
+        a, b = int(cu[i]), int(cu[i + 1])
+        if b > a:
+            check(y[a:b], s[i], y_ref[a:b], s_ref[i], 5e-3, f"packed split seq {i}")
+        else:
+            assert torch.equal(s[i].cpu(), inp.state_in[i])
+    assert orc.rel_l2(s.cpu().numpy(), s1.cpu().numpy()) < 1e-3
+
+
 def test_cfg4_varlen_serving_then_decode_steps_sampled():
     c = synth.CONFIGS["cfg4"]
     S, H = c["S"], c["H"]

@@ -118,6 +118,31 @@ def test_c2_varlen_matches_per_sequence_oracle_including_empty_sequence():
         assert ey <= TOL and es <= TOL, (i, n, ey, es)
 
 
+def test_c2_varlen_sequence_split_matches_per_sequence_oracle():
+    """Packed Finch-C2 call with few units: cut by max_seqlen into segments, two launches."""
+    lens = [2100, 0, 700, 3011]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    H = 2
+    assert gf.workspace_bytes(len(lens), max(lens), H, 64) > 0
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=832, state_std=0.1)
+    u2 = torch.randn(inp.r.shape, generator=torch.Generator().manual_seed(833)).bfloat16()
+    d = inp.to(DEV)
+    before = gf.launch_count()
+    y, s = gf.prefill_varlen_c2(d.r, d.k, d.v, d.x, u2.to(DEV), d.cu_seqlens, max(lens), d.state_in)
+    assert gf.launch_count() - before == 2
+    gf.last_device_status()
+    for i, n in enumerate(lens):
+        a, b = int(cu[i]), int(cu[i + 1])
+        if n == 0:
+            assert torch.equal(s[i].cpu(), inp.state_in[i])
+            continue
+        sl = lambda t: t[a:b][None].contiguous()
+        y_ref, s_ref = orc.prefill_c2(sl(inp.r), sl(inp.k), sl(inp.v), sl(inp.x), sl(u2), inp.state_in[i][None].contiguous())
+        ey = orc.rel_l2(y[a:b].float().cpu().numpy(), y_ref[0])
+        es = orc.rel_l2(s[i].cpu().numpy(), s_ref[0])
+        assert ey <= TOL and es <= TOL, (i, n, ey, es)
+
+
 @pytest.mark.parametrize("with_u2", [True, False])
 def test_c2_step_matches_oracle_and_chains_to_a_prefill(with_u2):
     B, H, T = 3, 5, 6
