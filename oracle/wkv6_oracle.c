@@ -177,3 +177,35 @@ void wkv6_oracle_prefill_c2(const float *r, const float *k, const float *v, cons
                                state_out ? state_out + soff : NULL, y + off, T, N, C);
         }
 }
+
+/* ---------------------------------------------------------------------------------------------------
+ * LayerNorm across all heads: the normalisation in the o_t equation of the Finch-C2 block,
+ *     o_t = LayerNorm(concat_h(r_t . wkv_t + u'_t)) W^O,
+ * i.e. one LayerNorm over the D = H*N concatenated channels of a token (the paper replaces Finch's
+ * per-head GroupNorm by it), before the output projection.  The paper gives no formula for the
+ * operator; this is its standard definition (Ba, Kiros, Hinton 2016) with the customary per-channel
+ * affine pair and the eps inside the square root:
+ *     mu = (1/D) sum_c y[c],   var = (1/D) sum_c (y[c] - mu)^2          (biased variance)
+ *     out[c] = (y[c] - mu) / sqrt(var + eps) * gamma[c] + beta[c]
+ * gamma / beta may be NULL (1 / 0).  y, out: [rows][D] double, every sum in index order.
+ * Pins (tests/test_oracle_pins_ln.py): closed form on an arithmetic progression, the two-element row,
+ * a constant row, the library LayerNorm in float64, mean / variance of the output, shift and scale laws,
+ * the difference to a per-head norm, channel indexing of gamma and beta.
+ */
+void c2_oracle_layernorm(const double *y, const double *gamma, const double *beta, double eps,
+                         double *out, long rows, long D)
+{
+#pragma omp parallel for schedule(static)
+    for (long row = 0; row < rows; ++row) {
+        const double *yr = y + (size_t)row * D;
+        double *o = out + (size_t)row * D;
+        double mu = 0.0, var = 0.0;
+        for (long c = 0; c < D; ++c) mu += yr[c];
+        mu /= (double)D;
+        for (long c = 0; c < D; ++c) var += (yr[c] - mu) * (yr[c] - mu);
+        var /= (double)D;
+        const double rstd = 1.0 / sqrt(var + eps);
+        for (long c = 0; c < D; ++c)
+            o[c] = (yr[c] - mu) * rstd * (gamma ? gamma[c] : 1.0) + (beta ? beta[c] : 0.0);
+    }
+}

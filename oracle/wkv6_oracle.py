@@ -38,6 +38,7 @@ def _load():
         _lib.wkv6_oracle_prefill.restype = None
         _lib.wkv6_oracle_prefill_varlen.restype = None
         _lib.wkv6_oracle_prefill_c2.restype = None
+        _lib.c2_oracle_layernorm.restype = None
     return _lib
 
 
@@ -148,6 +149,26 @@ def step(r, k, v, x, u, state_in):
     r, k, v, x = (_f32(a)[:, None] for a in (r, k, v, x))
     y, s = prefill(r, k, v, x, u, state_in)
     return y[:, 0], s
+
+
+def layernorm_heads(y, gamma=None, beta=None, eps=1e-5):
+    """LayerNorm over all D = H*N channels of each token (the o_t equation of the Finch-C2 block, before
+    W^O).  y: [..., H, N] or [rows, D] (numpy / torch, any float type; widened exactly to float64 and
+    flattened to rows of D); gamma, beta: [D] or None.  Returns float64 of y's shape."""
+    lib = _load()
+    if hasattr(y, "detach"):
+        y = y.detach().cpu().double().numpy()
+    y = np.ascontiguousarray(np.asarray(y, dtype=np.float64))
+    D = y.shape[-1] * (y.shape[-2] if y.ndim >= 3 else 1)
+    rows = y.size // D if D else 0
+    cv = lambda a: None if a is None else np.ascontiguousarray(
+        (a.detach().cpu().double().numpy() if hasattr(a, "detach") else np.asarray(a, dtype=np.float64)).reshape(D))
+    gamma, beta = cv(gamma), cv(beta)
+    out = np.zeros_like(y)
+    d = ctypes.c_double
+    lib.c2_oracle_layernorm(_p(y, d), _p(gamma, d), _p(beta, d), d(float(eps)), _p(out, d),
+                            ctypes.c_long(rows), ctypes.c_long(D))
+    return out
 
 
 def rel_l2(a, b) -> float:
