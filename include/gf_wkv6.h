@@ -220,6 +220,23 @@ GF_API gf_status_t gf_wkv6_last_device_status(gf_stream_t stream);
 GF_API uint64_t gf_wkv6_launch_count(void);
 
 GF_API const char *gf_status_string(gf_status_t status);
+/* LayerNorm across all heads: the normalisation that follows the WKV output in the o_t equation of the
+ * Finch-C2 block, o_t = LayerNorm(concat_h(r_t . wkv_t + u'_t)) W^O (the paper replaces Finch's per-head
+ * GroupNorm by one LayerNorm over the D = H*N concatenated channels of a token).  For every row (token):
+ *     mu = mean_c y[c],  var = mean_c (y[c] - mu)^2,  out[c] = (y[c] - mu) / sqrt(var + eps) * gamma[c] + beta[c].
+ * The paper does not spell the operator out; eps inside the root and the per-channel affine pair are the
+ * customary definition.  The output projection W^O is a plain GEMM and not part of this library.
+ *   y, out    DEVICE [rows][H][N] (bf16, resp. fp32 for _f32), 16-byte aligned; out may be y (in place).
+ *             Typically y is the output of a gf_wkv6_prefill* / gf_wkv6_step* call with rows = B*T tokens.
+ *   gamma,beta DEVICE fp32 [H*N], or NULL for 1 resp. 0.     eps >= 0 (HOST value).
+ * Arithmetic in fp32 (two passes: mean, then squared deviations), one rounding to the output type.
+ * H*N must be a multiple of 8 and at most 8192 (GF_ERR_UNSUPPORTED otherwise); rows = 0 is a no-op.
+ * Enqueues one kernel on `stream`, allocates nothing, does not synchronise. */
+GF_API gf_status_t gf_c2_layernorm(const void *y, const float *gamma, const float *beta, float eps, void *out,
+                            long long rows, int H, int N, gf_stream_t stream);
+GF_API gf_status_t gf_c2_layernorm_f32(const float *y, const float *gamma, const float *beta, float eps,
+                                float *out, long long rows, int H, int N, gf_stream_t stream);
+
 GF_API int gf_wkv6_version(void);
 
 #ifdef __cplusplus

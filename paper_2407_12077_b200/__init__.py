@@ -45,6 +45,8 @@ _SIGNATURES = {
     "gf_wkv6_set_workspace": (_i, [_vp, _sz]),
     "gf_wkv6_sequence_summary": (_i, [_vp] * 4 + [_i] * 5 + [_vp]),
     "gf_wkv6_fold_summaries": (_i, [_vp, _vp] + [_i] * 4 + [_vp, _vp]),
+    "gf_c2_layernorm": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
+    "gf_c2_layernorm_f32": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
     "gf_wkv6_launch_count": (ctypes.c_uint64, []),
@@ -286,6 +288,24 @@ def fold_summaries(state_in, summaries, n_fold, state_out=None, stream=None):
                                           _dev(state_out, "state_out", torch.float32, (B, H, 64, 64)), _stream(stream)),
                "gf_wkv6_fold_summaries")
     return state_out
+
+
+def layernorm_heads(y, gamma=None, beta=None, eps=1e-5, out=None, stream=None):
+    """gf_c2_layernorm(_f32): LayerNorm over all H*N channels of every token.  y: [..., H, N] CUDA tensor
+    (bf16 or fp32, contiguous); gamma, beta: fp32 [H*N] (or [H, N]) or None.  out defaults to a new tensor
+    (pass out=y for in place).  Returns out."""
+    lib = load_library()
+    H, N = y.shape[-2], y.shape[-1]
+    rows = y.numel() // (H * N) if H * N else 0
+    sfx = _suffix(y.dtype)
+    if out is None:
+        out = torch.empty_like(y)
+    with torch.cuda.device(y.device):
+        _check(getattr(lib, "gf_c2_layernorm" + sfx)(
+            _dev(y, "y"), _dev(None if gamma is None else gamma.reshape(H * N), "gamma", torch.float32),
+            _dev(None if beta is None else beta.reshape(H * N), "beta", torch.float32), float(eps),
+            _dev(out, "out", y.dtype, y.shape), rows, H, N, _stream(stream)), "gf_c2_layernorm" + sfx)
+    return out
 
 
 STATIC_SCRATCH_BYTES = 1597440       # GF_WKV6_STATIC_SCRATCH_BYTES

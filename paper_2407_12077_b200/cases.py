@@ -3,7 +3,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
 
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
-cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode
+cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode ln-cfg1 ln-cfg2 ln-wide
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -103,6 +103,16 @@ def run(case, reps, scale):
         fn = lambda: gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, max(lens), None, state_out=s, y=y)
         return dict(case=case, shape=f"S=2 lens={lens} H={H} bf16", units=sum(lens) * H,
                     bytes=sum(lens) * H * 640 + 2 * H * 16384, ms=_time(fn, reps))
+    if case in ("ln-cfg1", "ln-cfg2", "ln-wide"):  # LayerNorm across all heads over the tokens of a prefill's output
+        k = c["cfg1" if case == "ln-cfg1" else "cfg2"]
+        rows, H = k["B"] * sc(k["T"]), (128 if case == "ln-wide" else k["H"])
+        g = torch.Generator(device=DEV).manual_seed(9)
+        y = torch.randn((rows, H, 64), device=DEV, generator=g).bfloat16()
+        gamma, beta = torch.rand(H * 64, device=DEV, generator=g) + 0.5, torch.randn(H * 64, device=DEV, generator=g)
+        out = torch.empty_like(y)
+        fn = lambda: gf.layernorm_heads(y, gamma, beta, 1e-5, out=out)
+        return dict(case=case, shape=f"rows={rows} D={H * 64} bf16", units=rows * H, bytes=rows * H * 64 * 4 + 8 * H * 64,
+                    ms=_time(fn, reps))
     if case in ("cfg4-prefill", "cfg4-decode"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -135,7 +145,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "ln-cfg1", "ln-cfg2", "ln-wide"]
 
 
 def main():

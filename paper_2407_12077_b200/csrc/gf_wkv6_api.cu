@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "ln_heads.cuh"
 #include "wkv6_chunked.cuh"
 #include "wkv6_exact.cuh"
 #include "wkv6_step.cuh"
@@ -147,6 +148,21 @@ gf_status_t step_impl(const IO* r, const IO* k, const IO* v, const IO* x, const 
     return launch_result();
 }
 
+}  // namespace
+
+namespace {
+template <typename IO>
+gf_status_t layernorm_call(const IO* y, const float* gamma, const float* beta, float eps, IO* out, long long rows,
+                           int H, int N, gf_stream_t stream)
+{
+    if (rows < 0 || H < 0 || N < 0 || !(eps >= 0.f) || eps > 3.0e38f) return GF_ERR_INVALID_ARG;
+    const long long D = (long long)H * N;
+    if (rows == 0 || D == 0) return GF_OK;
+    if ((D & 7) || D > gf::ln::MAX_D) return GF_ERR_UNSUPPORTED;
+    if (rows > (1LL << 62) / D) return GF_ERR_INVALID_ARG;
+    if (!y || !out || misaligned(y) || misaligned(out) || misaligned(gamma) || misaligned(beta)) return GF_ERR_INVALID_ARG;
+    return gf::layernorm_heads<IO>(y, gamma, beta, eps, out, rows, (int)D, gf::sm_count(), (cudaStream_t)stream, &g_launches);
+}
 }  // namespace
 
 extern "C" {
@@ -398,6 +414,18 @@ gf_status_t gf_wkv6_last_device_status(gf_stream_t stream)
 }
 
 uint64_t gf_wkv6_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+gf_status_t gf_c2_layernorm(const void* y, const float* gamma, const float* beta, float eps, void* out,
+                            long long rows, int H, int N, gf_stream_t stream)
+{
+    return layernorm_call(static_cast<const __nv_bfloat16*>(y), gamma, beta, eps, static_cast<__nv_bfloat16*>(out), rows, H, N, stream);
+}
+
+gf_status_t gf_c2_layernorm_f32(const float* y, const float* gamma, const float* beta, float eps, float* out,
+                                long long rows, int H, int N, gf_stream_t stream)
+{
+    return layernorm_call(y, gamma, beta, eps, out, rows, H, N, stream);
+}
 
 const char* gf_status_string(gf_status_t s)
 {

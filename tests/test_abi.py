@@ -128,3 +128,19 @@ def test_later_entry_points_reject_bad_arguments_before_any_launch():
     assert _call("gf_wkv6_set_workspace", A + 8, 1 << 20) == 1                # not 256-byte aligned
     assert _call("gf_wkv6_set_workspace", None, 0) == 0
     assert gf.workspace_bytes(1, 100000, 32, 48) == 0
+
+
+def test_layernorm_entry_points_validate_before_any_launch():
+    f = ctypes.c_float
+    for name in ("gf_c2_layernorm", "gf_c2_layernorm_f32"):
+        assert _call(name, A, A, A, f(1e-5), A, 0, 32, 64, None) == 0          # no rows: no-op
+        assert _call(name, A, A, A, f(1e-5), A, 4, 0, 64, None) == 0           # no channels: no-op
+        assert _call(name, A, A, A, f(1e-5), A, -1, 32, 64, None) == 1
+        assert _call(name, A, A, A, f(-1.0), A, 4, 32, 64, None) == 1          # negative eps
+        assert _call(name, A, A, A, f(float("nan")), A, 4, 32, 64, None) == 1
+        assert _call(name, None, A, A, f(1e-5), A, 4, 32, 64, None) == 1
+        assert _call(name, A, A, A, f(1e-5), None, 4, 32, 64, None) == 1
+        assert _call(name, A + 2, A, A, f(1e-5), A, 4, 32, 64, None) == 1      # misaligned
+        assert _call(name, A, A + 4, A, f(1e-5), A, 4, 32, 64, None) == 1
+        assert _call(name, A, A, A, f(1e-5), A, 4, 3, 5, None) == 2            # H*N not a multiple of 8
+        assert _call(name, A, A, A, f(1e-5), A, 4, 129, 64, None) == 2         # wider than 8192 channels
