@@ -4,16 +4,22 @@
 // channels of a token, with per-channel gamma / beta and eps inside the square root).
 //
 // The operator is bound by HBM (D elements in, D out per token), so the kernel is built around two
-// budgets: bytes in flight and instructions per element.  A team of W warps (W = 1 up to 2048 channels)
-// owns whole rows: lane l of the team holds the 8-channel slices l + 32*W*j, j < VPL, of a row in
-// registers, so mean and variance are a register pass plus one shuffle reduction each (two true passes:
-// the mean first, then the squared deviations) and cost ten shuffles per row instead of per slice.
-// Narrow rows are taken R = 8 / VPL at a time.  The next group's slices are prefetched in their raw
-// form (no instruction touches them until the group is consumed) while the current group is reduced,
-// normalised and stored.  gamma and beta sit in shared memory, laid out so that every 16-byte read is
-// contiguous across the lanes.  Teams of more than one warp exchange their per-warp (mean, squared
-// deviations) pairs through shared memory with one named barrier per row and merge them by the pairwise
-// update formula (Chan, Golub, LeVeque).  Arithmetic on packed fp32 pairs.
+// budgets: bytes in flight and instructions per element.
+//  - A team of W warps (W = 1 up to 2048 channels, 2 up to 4096, 4 up to 8192) owns whole rows: lane l
+//    of the team holds the 8-channel slices l + 32*W*j, j < VPL, of a row in registers.  Mean and
+//    variance are a register pass plus one shuffle reduction each (two true passes: the mean first, then
+//    the squared deviations), ten shuffles per row rather than per slice.
+//  - Rows narrower than eight slices per lane are taken several at a time, so that every lane keeps at
+//    least 128 bytes in flight (with the prefetch: two groups); one CTA of eight warps per SM walks the
+//    rows.  Measured: more CTAs per SM, or twice the group size, gain nothing or lose.
+//  - The next group's slices are prefetched in their raw form (no instruction touches them until the
+//    group is consumed) while the current group is reduced, normalised and stored.
+//  - gamma and beta sit in shared memory, laid out so that every 16-byte read is contiguous across lanes.
+//  - Teams of several warps exchange per-warp (mean, squared deviations) pairs through shared memory with
+//    one named barrier per row group and merge them by the pairwise update formula (Chan, Golub,
+//    LeVeque), which keeps the accuracy of the two-pass variance.
+//  - Arithmetic on packed fp32 pairs; (y - mean) is formed before the scaling, so a constant row gives
+//    exactly beta.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -98,20 +104,21 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// rows a team takes at a time: at least 128 bytes per lane in flight (8 bf16 slices, 4 fp32 slices)
+constexpr int rows_per_group(int VPL, int esize) { return (16 / esize + VPL - 1) / VPL; }
 constexpr int smem_bytes(int VPL, int W) { return 2 * VPL * 2 * 32 * W * 16; }      // gamma and beta as float4 [VPL][2][32 W]
 
 // y, out: [rows][D] (out may be y); gamma, beta: [D] fp32 or nullptr.  32 * W * VPL * 8 >= D; blockDim.x = 256.
 template <typename IO, int VPL, int W>
-__global__ void __launch_bounds__(MAX_THREADS, sizeof(IO) == 2 ? 2 : 1)
+__global__ void __launch_bounds__(MAX_THREADS, 1)
 layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma, const float* __restrict__ beta,
                        float eps, IO* __restrict__ out, long long rows, int D)
 {
-    constexpr int R = 8 / VPL;                      // rows a team takes at a time
+    constexpr int R = rows_per_group(VPL, sizeof(IO));
     constexpr int TEAMS = MAX_WARPS / W;            // teams per CTA
     constexpr int TL = 32 * W;                      // lanes of a team
-    static_assert(W == 1 || R == 1, "teams of several warps take one row at a time");
     extern __shared__ float4 gb[];                  // gamma [VPL][2][TL], then beta in the same layout
-    __shared__ float2 part[TEAMS][2][W];            // per-warp (mean, squared deviations) by row parity
+    __shared__ float2 part[TEAMS][2][R][W];         // per-warp (mean, squared deviations) by group parity
     __shared__ float cnt[MAX_WARPS];                // channels that each warp holds
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int team = warp / W, wt = warp % W, tl = wt * 32 + lane;
@@ -165,6 +172,7 @@ layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma
         if (r0 + stride < rows) load_group(next, r0 + stride);    // in flight during this group's arithmetic
 
         float2 scale[R], shift[R];                  // out = (x + shift) * scale * gamma + beta, shift = -mean (exact zero on a constant row)
+        float mu[R], m2[R];
 #pragma unroll
         for (int i = 0; i < R; ++i) {
             // ---- mean of this warp's channels, then their squared deviations from it
@@ -173,8 +181,8 @@ layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma
             for (int j = 0; j < VPL; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s2 = add2(s2, x[i][j][e]);
-            const float m_w = warp_sum(s2.x + s2.y) * inv_nw;
-            const float2 neg_m = make_float2(-m_w, -m_w);
+            mu[i] = warp_sum(s2.x + s2.y) * inv_nw;
+            const float2 neg_m = make_float2(-mu[i], -mu[i]);
             float2 q2 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int j = 0; j < VPL; ++j)
@@ -185,27 +193,38 @@ layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma
                         q2 = fma2(dv, dv, q2);
                     }
                 }
-            float mu = m_w, m2 = warp_sum(q2.x + q2.y);
-            if (W > 1) {
-                // ---- merge the team's per-warp pairs
-                if (lane == 0) part[team][par][wt] = make_float2(mu, m2);
-                asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(TL) : "memory");
-                mu = 0.f;
+            m2[i] = warp_sum(q2.x + q2.y);
+        }
+        if (W > 1) {
+            // ---- merge the team's per-warp pairs
+            if (lane == 0) {
 #pragma unroll
-                for (int w = 0; w < W; ++w) mu = fmaf(cnt[team * W + w], part[team][par][w].x, mu);
-                mu *= inv_d;
-                m2 = 0.f;
+                for (int i = 0; i < R; ++i) part[team][par][i][wt] = make_float2(mu[i], m2[i]);
+            }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(TL) : "memory");
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                float m = 0.f;
+#pragma unroll
+                for (int w = 0; w < W; ++w) m = fmaf(cnt[team * W + w], part[team][par][i][w].x, m);
+                m *= inv_d;
+                float q = 0.f;
 #pragma unroll
                 for (int w = 0; w < W; ++w) {
-                    const float2 pw = part[team][par][w];
-                    const float dm = pw.x - mu;
-                    m2 += fmaf(cnt[team * W + w] * dm, dm, pw.y);
+                    const float2 pw = part[team][par][i][w];
+                    const float dm = pw.x - m;
+                    q += fmaf(cnt[team * W + w] * dm, dm, pw.y);
                 }
-                // part[team][par] is next written two rows on, after the barrier of the row between
+                mu[i] = m;
+                m2[i] = q;
             }
-            const float rstd = rsqrtf(fmaf(m2, inv_d, eps));
+            // part[team][par] is next written two groups on, after the barrier of the group between
+        }
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const float rstd = rsqrtf(fmaf(m2[i], inv_d, eps));
             scale[i] = make_float2(rstd, rstd);
-            shift[i] = make_float2(-mu, -mu);
+            shift[i] = make_float2(-mu[i], -mu[i]);
         }
         // ---- normalise and store
 #pragma unroll
@@ -231,8 +250,8 @@ template <typename IO, int VPL, int W>
 inline cudaError_t launch(const IO* y, const float* gamma, const float* beta, float eps, IO* out, long long rows, int D,
                           int n_sm, cudaStream_t st)
 {
-    constexpr int R = 8 / VPL, TEAMS = MAX_WARPS / W, SMEM = smem_bytes(VPL, W);
-    if (SMEM > 48 * 1024) {
+    constexpr int R = rows_per_group(VPL, sizeof(IO)), TEAMS = MAX_WARPS / W, SMEM = smem_bytes(VPL, W);
+    if (SMEM + 1024 > 48 * 1024) {                  // dynamic plus the few static bytes would pass the default limit
         static int attr_dev = -1;                   // opt in to the larger shared-memory size once per device
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -244,8 +263,7 @@ inline cudaError_t launch(const IO* y, const float* gamma, const float* beta, fl
         }
     }
     const long long groups = (rows + (long long)R * TEAMS - 1) / ((long long)R * TEAMS);
-    const long long cap = (long long)n_sm * (sizeof(IO) == 2 ? 2 : 1);
-    const unsigned grid = (unsigned)(groups < cap ? groups : cap);
+    const unsigned grid = (unsigned)(groups < n_sm ? groups : n_sm);      // one resident CTA per SM walks the rows
     layernorm_heads_kernel<IO, VPL, W><<<grid, MAX_THREADS, SMEM, st>>>(y, gamma, beta, eps, out, rows, D);
     return cudaGetLastError();
 }
@@ -259,13 +277,20 @@ inline gf_status_t layernorm_heads(const IO* y, const float* gamma, const float*
 {
     if (D <= 0 || (D & 7) || D > ln::MAX_D || rows <= 0 || n_sm <= 0) return GF_ERR_INVALID_ARG;
     const int nvec = D / 8;
-    cudaError_t e;
-    if (nvec <= 32) e = ln::launch<IO, 1, 1>(y, gamma, beta, eps, out, rows, D, n_sm, st);
-    else if (nvec <= 64) e = ln::launch<IO, 2, 1>(y, gamma, beta, eps, out, rows, D, n_sm, st);
-    else if (nvec <= 128) e = ln::launch<IO, 4, 1>(y, gamma, beta, eps, out, rows, D, n_sm, st);
-    else if (nvec <= 256) e = ln::launch<IO, 8, 1>(y, gamma, beta, eps, out, rows, D, n_sm, st);
-    else if (nvec <= 512) e = ln::launch<IO, 8, 2>(y, gamma, beta, eps, out, rows, D, n_sm, st);
-    else e = ln::launch<IO, 8, 4>(y, gamma, beta, eps, out, rows, D, n_sm, st);
+    const int w = nvec <= 256 ? 1 : (nvec <= 512 ? 2 : 4);
+    const int vpl = (nvec + 32 * w - 1) / (32 * w);                       // 1..8; 5..8 for teams of several warps
+    cudaError_t e = cudaErrorInvalidValue;
+#define GF_LN_CASE(V, W_) \
+    case V: e = ln::launch<IO, V, W_>(y, gamma, beta, eps, out, rows, D, n_sm, st); break;
+    if (w == 1) {
+        switch (vpl) { GF_LN_CASE(1, 1) GF_LN_CASE(2, 1) GF_LN_CASE(3, 1) GF_LN_CASE(4, 1)
+                       GF_LN_CASE(5, 1) GF_LN_CASE(6, 1) GF_LN_CASE(7, 1) GF_LN_CASE(8, 1) }
+    } else if (w == 2) {
+        switch (vpl) { GF_LN_CASE(5, 2) GF_LN_CASE(6, 2) GF_LN_CASE(7, 2) GF_LN_CASE(8, 2) }
+    } else {
+        switch (vpl) { GF_LN_CASE(5, 4) GF_LN_CASE(6, 4) GF_LN_CASE(7, 4) GF_LN_CASE(8, 4) }
+    }
+#undef GF_LN_CASE
     launches->fetch_add(1, std::memory_order_relaxed);
     return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

@@ -46,8 +46,13 @@ def run(y, gamma, beta, eps=1e-5, in_place=False):
     return out
 
 
-@pytest.mark.parametrize("rows", [1, 3, 4, 5, 8, 1001])
-@pytest.mark.parametrize("H,N", [(1, 8), (1, 64), (12, 64), (32, 64), (33, 64), (64, 64), (65, 64), (128, 64), (7, 24)])
+# widths that reach every (slices per lane, warps per row) variant of the kernel, full and ragged
+WIDTHS = [(1, 8), (1, 64), (4, 64), (8, 64), (12, 64), (16, 64), (20, 64), (24, 64), (28, 64), (32, 64), (33, 64),
+          (40, 64), (48, 64), (56, 64), (64, 64), (65, 64), (80, 64), (96, 64), (112, 64), (128, 64), (7, 24), (45, 8)]
+
+
+@pytest.mark.parametrize("rows", [1, 3, 8, 1001])
+@pytest.mark.parametrize("H,N", WIDTHS)
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 def test_layernorm_matches_oracle_over_widths_and_ragged_row_counts(rows, H, N, dtype):
     y, gamma, beta = draw(rows, H, N, dtype, seed=rows * 1000 + H * N)
