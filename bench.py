@@ -284,6 +284,26 @@ def main():
                 "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms, "launch_ms_median": statistics.median(per_launch),
                 "launch_ms_min": min(per_launch), "launch_ms_max": max(per_launch), "algorithmic_bytes": alg_bytes}
 
+    # ---- the step that follows the WKV output in the o_t equation (LayerNorm across all heads), timed on its own
+    # over the y of every call, outside the step and its numbers: reported beside them, not in them
+    g_ln = torch.Generator(device=dev).manual_seed(77)
+    gamma = torch.rand(H * N, device=dev, generator=g_ln) + 0.5
+    beta = torch.randn(H * N, device=dev, generator=g_ln)
+    o_ln = torch.empty_like(batches[0][1])
+    for _, y, _ in batches[:3]:
+        gf.layernorm_heads(y, gamma, beta, 1e-5, out=o_ln, stream=stream)
+    ln_a, ln_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ln_a.record(stream)
+    for _, y, _ in batches:
+        gf.layernorm_heads(y, gamma, beta, 1e-5, out=o_ln, stream=stream)
+    ln_b.record(stream)
+    torch.cuda.synchronize()
+    ln_ms = ln_a.elapsed_time(ln_b) / len(batches)
+    ln_bytes = 2 * B * T * H * N * 2
+    layernorm = {"kernel": "gf_c2_layernorm (one launch over the y of one call)", "launch_ms": ln_ms, "bound": "hbm",
+                 "achieved": ln_bytes / (ln_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                 "frac": ln_bytes / (ln_ms * 1e-3) / 1e9 / peak, "algorithmic_bytes": ln_bytes}
+
     # ---- end to end through the host-buffer entry point: pinned host inputs -> y on the host
     e2e = None
     if not args.no_e2e:
@@ -349,7 +369,8 @@ def main():
                        "precision": "bf16 r/k/v/x/y and tensor-core operands, fp32 accumulation, decay sums and state",
                        "l2": "inputs larger than L2 (1.34 GB per call, distinct buffers per call)",
                        "parallelism": f"(b,h) units replicated per GPU x{world}, no collective"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "layernorm_heads": layernorm, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": launches,
             "clocks": clocks,
         }
         print(json.dumps(line), flush=True)

@@ -27,11 +27,10 @@ static __device__ __align__(256) float g_static_scratch[GF_WKV6_STATIC_SCRATCH_B
 // Device address of g_static_scratch on the current device, looked up once per device.
 float* static_scratch()
 {
-    constexpr int MAX_DEV = 64;
     static std::mutex mu;
-    static float* addr[MAX_DEV] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV) return nullptr;
+    static float* addr[gf::MAX_DEVICES] = {};
+    const int dev = gf::current_device();
+    if (dev < 0) return nullptr;
     std::lock_guard<std::mutex> lock(mu);
     if (!addr[dev]) {
         float* ptr = nullptr;

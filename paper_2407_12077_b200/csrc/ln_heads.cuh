@@ -27,6 +27,7 @@
 
 #include <atomic>
 
+#include "device_info.cuh"
 #include "gf_wkv6.h"
 
 namespace gf {
@@ -252,14 +253,13 @@ inline cudaError_t launch(const IO* y, const float* gamma, const float* beta, fl
 {
     constexpr int R = rows_per_group(VPL, sizeof(IO)), TEAMS = MAX_WARPS / W, SMEM = smem_bytes(VPL, W);
     if (SMEM + 1024 > 48 * 1024) {                  // dynamic plus the few static bytes would pass the default limit
-        static int attr_dev = -1;                   // opt in to the larger shared-memory size once per device
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (attr_dev != dev) {
-            e = cudaFuncSetAttribute(layernorm_heads_kernel<IO, VPL, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+        static PerDeviceFlag attr_set;              // opt in to the larger shared-memory size once per device
+        const int dev = current_device();
+        if (dev < 0) return cudaErrorInvalidDevice;
+        if (!attr_set.is_set(dev)) {
+            const cudaError_t e = cudaFuncSetAttribute(layernorm_heads_kernel<IO, VPL, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
             if (e != cudaSuccess) return e;
-            attr_dev = dev;
+            attr_set.set(dev);
         }
     }
     const long long groups = (rows + (long long)R * TEAMS - 1) / ((long long)R * TEAMS);

@@ -45,6 +45,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "device_info.cuh"
 #include "gf_wkv6.h"
 
 namespace gf {
@@ -1205,21 +1206,6 @@ inline bool make_map(CUtensorMap* tm, const void* base, long long rows, long lon
 
 }  // namespace ck
 
-// Number of SMs of the current device (cached per device index; 0 on failure).
-inline int sm_count()
-{
-    static int cached_dev = -1, cached = 0;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (dev != cached_dev) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached = n;
-        cached_dev = dev;
-    }
-    return cached;
-}
-
 // Chooses the sequence split of a call: with fewer (sequence, head) units than half the SMs, each
 // sequence is cut into up to 8 segments of at least 8 chunks so that the grid fills the GPU (T: the
 // sequence length, for a packed call the longest one).  Returns the
@@ -1242,6 +1228,23 @@ inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_
     return g;
 }
 
+// Opts the four instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
+inline bool chunked_kernel_attributes()
+{
+    static PerDeviceFlag attr_set;                   // zero-initialised
+    const int dev = current_device();
+    if (dev < 0) return false;
+    if (!attr_set.is_set(dev)) {
+        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+            return false;
+        attr_set.set(dev);
+    }
+    return true;
+}
+
 // Launches the chunked kernel.  Dense: cu == nullptr, n_seq = B, T = sequence length.
 // Packed: cu = device cu_seqlens, n_seq = S, T = max_seqlen.  total_rows = rows of the [rows][H*64] tensors.
 // scratch / scratch_bytes: optional device memory for the sequence split (see choose_split); without
@@ -1254,19 +1257,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
 {
     const long long units = (long long)n_seq * H;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
-    static bool attr_set = false;
-    static int attr_dev = -1;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return GF_ERR_CUDA;
-    if (!attr_set || attr_dev != dev) {
-        if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
-            return GF_ERR_CUDA;
-        attr_set = true;
-        attr_dev = dev;
-    }
+    if (!chunked_kernel_attributes()) return GF_ERR_CUDA;
     CUtensorMap tr, tk, tv, tx, ty, tu2;
     const long long C = (long long)H * 64;
     if (!ck::make_map(&tr, r, total_rows, C, 64) || !ck::make_map(&tk, k, total_rows, C, 64) ||
@@ -1299,9 +1290,7 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
 {
     const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
-    if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-        cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
-        return GF_ERR_CUDA;
+    if (!chunked_kernel_attributes()) return GF_ERR_CUDA;
     CUtensorMap tk, tv, tx, tdummy;
     const long long C = (long long)H * 64;
     if (!ck::make_map(&tk, k, total_rows, C, 64) || !ck::make_map(&tv, v, total_rows, C, 64) ||
