@@ -416,3 +416,36 @@ def test_host_buffer_entry_point():
     gf.last_device_status()
     y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
     check(y, s_out, y_ref, s_ref, 5e-3, "host entry point")
+
+
+def test_calls_from_two_host_threads_on_their_own_streams():
+    """The library keeps no per-call host state: two threads, each with its own stream and buffers, call the
+    prefill and the decode step at the same time (shapes that do not split, so no shared workspace)."""
+    import threading
+    cases = [synth.make_dense(5, 200 + 70 * i, 16, 64, "bf16", seed=9100 + i, state_std=0.1) for i in range(2)]
+    assert gf.workspace_bytes(5, 270, 16, 64) == 0
+    results, errors = [None, None], []
+
+    def work(i):
+        try:
+            torch.cuda.set_device(0)
+            st = torch.cuda.Stream()
+            d = cases[i].to(DEV)
+            with torch.cuda.stream(st):
+                for _ in range(20):
+                    y, s = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in, stream=st)
+                st.synchronize()
+            results[i] = (y, s)
+        except Exception as e:                      # surfaced below, in the main thread
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    gf.last_device_status()
+    for i, inp in enumerate(cases):
+        y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+        check(results[i][0], results[i][1], y_ref, s_ref, 5e-3, f"thread {i}")
