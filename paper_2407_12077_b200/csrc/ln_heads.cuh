@@ -9,9 +9,10 @@
 //    of the team holds the 8-channel slices l + 32*W*j, j < VPL, of a row in registers.  Mean and
 //    variance are a register pass plus one shuffle reduction each (two true passes: the mean first, then
 //    the squared deviations), ten shuffles per row rather than per slice.
-//  - Rows narrower than eight slices per lane are taken several at a time, so that every lane keeps at
-//    least 128 bytes in flight (with the prefetch: two groups); one CTA of eight warps per SM walks the
-//    rows.  Measured: more CTAs per SM, or twice the group size, gain nothing or lose.
+//  - Rows narrower than eight slices per lane are taken several at a time (up to 160 bytes per lane and
+//    group, and the prefetch keeps a second group in flight); one CTA of twelve warps per SM walks the
+//    rows (eight for fp32).  Measured: two CTAs per SM, sixteen warps (both spill) or twice the group
+//    size lose; twelve warps beat eight by 2-7 %.
 //  - The next group's slices are prefetched in their raw form (no instruction touches them until the
 //    group is consumed) while the current group is reduced, normalised and stored.
 //  - gamma and beta sit in shared memory, laid out so that every 16-byte read is contiguous across lanes.
@@ -33,9 +34,11 @@
 namespace gf {
 namespace ln {
 
-constexpr int MAX_THREADS = 256;
-constexpr int MAX_WARPS = MAX_THREADS / 32;
-constexpr int MAX_D = 8 * MAX_THREADS * 4;          // VPT <= 4 slices of 8 channels per thread
+// Threads per CTA: the most warps that keep the widest variant free of register spills (12 for bf16, 8 for
+// fp32, whose raw prefetch set is twice as large); divisible by the team widths 1, 2 and 4.
+template <typename IO> constexpr int cta_threads() { return sizeof(IO) == 2 ? 384 : 256; }
+constexpr int MAX_WARPS = 12;
+constexpr int MAX_D = 8 * 32 * 4 * 8;               // lanes x team width x slices per lane, 8 channels each
 
 // Eight consecutive elements as they come from memory; unpacked to fp32 only where they are consumed, so
 // that a prefetched slice costs no instruction that would wait for its load.
@@ -105,18 +108,24 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// rows a team takes at a time: at least 128 bytes per lane in flight (8 bf16 slices, 4 fp32 slices)
-constexpr int rows_per_group(int VPL, int esize) { return (16 / esize + VPL - 1) / VPL; }
+// rows a team takes at a time: as many as keep at most 160 bytes per lane in one group (10 bf16 slices, 5 fp32
+// slices: what the registers hold without spilling), between one and four
+constexpr int rows_per_group(int VPL, int esize)
+{
+    const int r = (20 / esize) / VPL;
+    return r < 1 ? 1 : (r > 4 ? 4 : r);
+}
 constexpr int smem_bytes(int VPL, int W) { return 2 * VPL * 2 * 32 * W * 16; }      // gamma and beta as float4 [VPL][2][32 W]
 
-// y, out: [rows][D] (out may be y); gamma, beta: [D] fp32 or nullptr.  32 * W * VPL * 8 >= D; blockDim.x = 256.
+// y, out: [rows][D] (out may be y); gamma, beta: [D] fp32 or nullptr.  32 * W * VPL * 8 >= D; blockDim.x = cta_threads<IO>().
 template <typename IO, int VPL, int W>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+__global__ void __launch_bounds__(cta_threads<IO>(), 1)
 layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma, const float* __restrict__ beta,
                        float eps, IO* __restrict__ out, long long rows, int D)
 {
     constexpr int R = rows_per_group(VPL, sizeof(IO));
-    constexpr int TEAMS = MAX_WARPS / W;            // teams per CTA
+    constexpr int THREADS = cta_threads<IO>();
+    constexpr int TEAMS = THREADS / 32 / W;         // teams per CTA
     constexpr int TL = 32 * W;                      // lanes of a team
     extern __shared__ float4 gb[];                  // gamma [VPL][2][TL], then beta in the same layout
     __shared__ float2 part[TEAMS][2][R][W];         // per-warp (mean, squared deviations) by group parity
@@ -124,7 +133,7 @@ layernorm_heads_kernel(const IO* __restrict__ y, const float* __restrict__ gamma
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int team = warp / W, wt = warp % W, tl = wt * 32 + lane;
 
-    for (int idx = tid; idx < VPL * 2 * TL; idx += MAX_THREADS) {
+    for (int idx = tid; idx < VPL * 2 * TL; idx += THREADS) {
         const int j = idx / (2 * TL), half = (idx / TL) & 1, l = idx % TL;
         const int c = 8 * (l + TL * j) + 4 * half;
         float4 gv = make_float4(0.f, 0.f, 0.f, 0.f), bv = gv;
@@ -251,7 +260,7 @@ template <typename IO, int VPL, int W>
 inline cudaError_t launch(const IO* y, const float* gamma, const float* beta, float eps, IO* out, long long rows, int D,
                           int n_sm, cudaStream_t st)
 {
-    constexpr int R = rows_per_group(VPL, sizeof(IO)), TEAMS = MAX_WARPS / W, SMEM = smem_bytes(VPL, W);
+    constexpr int R = rows_per_group(VPL, sizeof(IO)), TEAMS = cta_threads<IO>() / 32 / W, SMEM = smem_bytes(VPL, W);
     if (SMEM + 1024 > 48 * 1024) {                  // dynamic plus the few static bytes would pass the default limit
         static PerDeviceFlag attr_set;              // opt in to the larger shared-memory size once per device
         const int dev = current_device();
@@ -264,7 +273,7 @@ inline cudaError_t launch(const IO* y, const float* gamma, const float* beta, fl
     }
     const long long groups = (rows + (long long)R * TEAMS - 1) / ((long long)R * TEAMS);
     const unsigned grid = (unsigned)(groups < n_sm ? groups : n_sm);      // one resident CTA per SM walks the rows
-    layernorm_heads_kernel<IO, VPL, W><<<grid, MAX_THREADS, SMEM, st>>>(y, gamma, beta, eps, out, rows, D);
+    layernorm_heads_kernel<IO, VPL, W><<<grid, cta_threads<IO>(), SMEM, st>>>(y, gamma, beta, eps, out, rows, D);
     return cudaGetLastError();
 }
 
