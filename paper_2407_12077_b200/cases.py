@@ -3,7 +3,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
 
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
-cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode ln-cfg1 ln-cfg2 ln-wide
+cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -113,7 +113,7 @@ def run(case, reps, scale):
         fn = lambda: gf.layernorm_heads(y, gamma, beta, 1e-5, out=out)
         return dict(case=case, shape=f"rows={rows} D={H * 64} bf16", units=rows * H, bytes=rows * H * 64 * 4 + 8 * H * 64,
                     ms=_time(fn, reps))
-    if case in ("cfg4-prefill", "cfg4-decode"):
+    if case in ("cfg4-prefill", "cfg4-decode", "cfg4-decode-layers"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
         cu = synth.make_lengths(S, max(1, int(k["len_min"] * scale)), max(2, int(k["len_max"] * scale)), seed=4000)
@@ -125,6 +125,24 @@ def run(case, reps, scale):
             fn = lambda: gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, mx, inp.state_in, state_out=s, y=y)
             return dict(case=case, shape=f"S={S} total_T={total} H={H} bf16", units=total * H,
                         bytes=total * H * 640 + 2 * S * H * 16384, ms=_time(fn, reps))
+        if case == "cfg4-decode-layers":
+            # a decode loop over a stack of layers: every layer has its own state, so the states of one token step
+            # (12 layers x 33.5 MB) do not fit L2 and every step streams its state from and to HBM
+            layers = 12
+            ds = [synth.make_step(S, H, 64, "bf16", seed=4100 + i, device=DEV) for i in range(layers)]
+            ys = [torch.empty_like(d.r) for d in ds]
+            g = torch.cuda.CUDAGraph()
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for d, y in zip(ds, ys):
+                    gf.step(d.r, d.k, d.v, d.x, d.u, d.state_in, y=y, stream=st)
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=st):
+                    for d, y in zip(ds, ys):
+                        gf.step(d.r, d.k, d.v, d.x, d.u, d.state_in, y=y, stream=st)
+            ms = _time(g.replay, reps) / layers
+            return dict(case=case, shape=f"S={S} H={H} bf16, {layers} layers with their own states per graph replay, in place",
+                        units=S * H, bytes=S * H * (2 * 16384 + 5 * 128), ms=ms)
         d = synth.make_step(S, H, 64, "bf16", seed=4002, device=DEV)
         y = torch.empty_like(d.r)
         steps = 64
@@ -145,7 +163,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "ln-cfg1", "ln-cfg2", "ln-wide"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide"]
 
 
 def main():
