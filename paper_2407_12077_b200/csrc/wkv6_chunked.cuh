@@ -118,13 +118,18 @@ enum {
     BAR_B_DONE = BAR_F_EMPTY + 2,        // Y0 and PV accumulators complete; state / score operand tiles free again
     BAR_Y_EMPTY = BAR_B_DONE + 2,        // ... and read back by the output warps
     BAR_ESYNC = BAR_Y_EMPTY + 2,         // one per elementwise set
-    BAR_SSYNC = BAR_ESYNC + 2,           // token-by-token path only: state-warp rendezvous,
-    BAR_FB_READY = BAR_SSYNC + 1,        //   fp32 state copy in place for the output warps,
+    BAR_SSYNC = BAR_ESYNC + 2,           // token-by-token path only: state-warp rendezvous after the fp32 copy is re-read,
+    BAR_SPRE = BAR_SSYNC + 1,            //   and before it is written,
+    BAR_FB_READY = BAR_SPRE + 1,         //   fp32 state copy in place for the output warps,
     BAR_FB_DONE = BAR_FB_READY + 1,      //   and advanced by them over the chunk
     BAR_U2 = BAR_FB_DONE + 1,            // Finch-C2 form: one per output warp, its second-value slab has landed
     BAR_COUNT = BAR_U2 + N_GW
 };
-constexpr int SMEM_BYTES = OFF_BAR + BAR_COUNT * 8;
+// persistent launches: one descriptor per chunk of the CTA's chunk stream
+// {first row, valid tokens | flags | head << 16, unit, chunks left in the unit}
+constexpr int OFF_DESC = (OFF_BAR + BAR_COUNT * 8 + 15) & ~15;   // [NSIDE] int4
+constexpr int DESC_FIRST = 0x100, DESC_END = 0x200;              // flags beside the valid-token count (low byte)
+constexpr int SMEM_BYTES = OFF_DESC + NSIDE * 16;
 constexpr int SMEM_ALLOC = SMEM_BYTES + 1024;              // slack for manual 1024-byte alignment
 static_assert(SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
 
@@ -454,6 +459,12 @@ struct Params {
     // vector [rows][H*64] bf16 added to the output.
     const __nv_bfloat16* u2;
     int c2;
+    // Persistent launches (more units than SMs): the grid is one CTA per SM and every CTA walks a stream
+    // of units without draining its pipeline in between.  n_units = sequences x heads; `ticket`, if not
+    // NULL, is a zeroed device counter from which the CTAs draw units (packed calls, whose units differ
+    // in length); NULL: unit = blockIdx.x + k gridDim.x (equal lengths).
+    int n_units;
+    unsigned int* ticket;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -594,7 +605,9 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
 // the second MMA warp idle, the output warps only serve the token-by-token path) and writes the
 // segment's summary.
 // C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus, optional second-value vector).
-template <bool SUMMARY, bool C2>
+// PERSIST = true: the CTA walks a stream of units (see Params::n_units); the producer warp leaves a descriptor per
+// chunk and two end markers, which every role passes down its own signalling path before it leaves.
+template <bool SUMMARY, bool C2, bool PERSIST = false>
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
@@ -626,9 +639,33 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         row0 += first;
         len = (seg == p.nseg - 1) ? len - first : min(len - first, p.seg_chunks * L);
     }
-    const int nchunks = (len + L - 1) / L;
+    const int nchunks = PERSIST ? 0 : (len + L - 1) / L;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
+    static_assert(!(PERSIST && SUMMARY), "the summary pass is a single-unit launch");
+
+    // One chunk of this CTA's work.  Single-unit launches derive it from the chunk index; persistent launches
+    // read the descriptor the producer warp left for the chunk, which is visible to any warp that has waited
+    // on a barrier downstream of the chunk's "full" barrier.
+    struct Chunk { int row; int valid; int unit; int h; int rem; bool first; bool end; };
+    auto chunk_at = [&](int c) -> Chunk {
+        Chunk ck;
+        if constexpr (PERSIST) {
+            int4 d;
+            asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(d.x), "=r"(d.y), "=r"(d.z), "=r"(d.w) : "r"(sbase + OFF_DESC + 16 * (c & (NSIDE - 1))) : "memory");
+            ck.row = d.x; ck.valid = d.y & 0xff; ck.unit = d.z; ck.h = d.y >> 16; ck.rem = d.w;
+            ck.first = (d.y & DESC_FIRST) != 0; ck.end = (d.y & DESC_END) != 0;
+        } else {
+            ck.row = (int)(row0 + (long long)c * L); ck.valid = min(L, len - c * L); ck.unit = unit; ck.h = h;
+            ck.rem = nchunks - 1 - c; ck.first = c == 0; ck.end = false;
+        }
+        return ck;
+    };
+    auto chunk_is_end = [&](int c) -> bool {
+        if constexpr (PERSIST) return (lds32(sbase + OFF_DESC + 16 * (c & (NSIDE - 1)) + 4) & DESC_END) != 0;
+        return false;
+    };
 
     if (tid == 0) {
         for (int i = 0; i < NS; ++i) {
@@ -646,6 +683,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         for (int i = 0; i < N_ESET; ++i) mbar_init(bar(BAR_ESYNC + i), N_EW);
         mbar_init(bar(BAR_SSYNC), N_GW);
+        mbar_init(bar(BAR_SPRE), N_GW);
         mbar_init(bar(BAR_FB_READY), N_GW);
         mbar_init(bar(BAR_FB_DONE), N_GW);
         for (int i = 0; i < N_GW; ++i) mbar_init(bar(BAR_U2 + i), 1);
@@ -661,6 +699,83 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
 
     if (warp == 0) {
         // ============================== TMA producer ==============================
+        if constexpr (PERSIST) {
+            int gc = 0, real_end = -1;               // chunks of the stream issued so far; index of the first end marker
+            int s = 0, ph = 1;                       // ring stage and the parity of its previous release
+            bool alive = true;
+            for (int k = 0; alive; ++k) {
+                int u = 0;
+                if (p.ticket) {
+                    if (lane == 0) u = (int)atomicAdd(p.ticket, 1u);
+                    u = __shfl_sync(0xffffffffu, u, 0);
+                } else {
+                    u = blockIdx.x + k * gridDim.x;
+                }
+                if (u >= p.n_units) break;
+                const int useq = u / p.H, uh = u % p.H;
+                long long urow0;
+                int ulen;
+                if (p.cu_seqlens) {
+                    urow0 = p.cu_seqlens[useq];
+                    ulen = p.cu_seqlens[useq + 1] - p.cu_seqlens[useq];
+                } else {
+                    urow0 = (long long)useq * p.T;
+                    ulen = p.T;
+                }
+                const int unch = (ulen + L - 1) / L;
+                if (unch == 0) {
+                    // empty sequence: its state passes through; no chunk enters the stream
+                    if (p.state_out && p.state_out != p.state_in)
+                        for (int i = lane; i < 4096; i += 32)
+                            p.state_out[(size_t)u * 4096 + i] = p.state_in ? p.state_in[(size_t)u * 4096 + i] : 0.f;
+                    continue;
+                }
+                if (p.state_in) {
+                    // the state warps read this unit's start state a few chunks from now: have it in L2 by then
+                    const char* sp0 = reinterpret_cast<const char*>(p.state_in + (size_t)u * 4096);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(sp0 + 128 * (lane + 32 * i)));
+                }
+                for (int c = 0; c < unch; ++c, ++gc) {
+                    if (gc >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) { alive = false; break; }
+                    const int row = (int)(urow0 + (long long)c * L);
+                    const uint32_t dst = sbase + OFF_RING + s * STAGE;
+                    if (elect_one()) {
+                        const int meta = min(L, ulen - c * L) | (c == 0 ? DESC_FIRST : 0) | (uh << 16);
+                        asm volatile("st.shared.v4.s32 [%0], {%1, %2, %3, %4};" ::"r"(sbase + OFF_DESC + 16 * (gc & (NSIDE - 1))),
+                                     "r"(row), "r"(meta), "r"(u), "r"(unch - 1 - c) : "memory");
+                        mbar_expect_tx(bar(BAR_FULL_RKV + s), STAGE);      // (release: the descriptor is visible to the waiters)
+                        tma_load_2d(dst, &tm_x, uh * 64, row, bar(BAR_FULL_RKV + s));
+                        tma_load_2d(dst + TILE, &tm_r, uh * 64, row, bar(BAR_FULL_RKV + s));
+                        tma_load_2d(dst + 2 * TILE, &tm_k, uh * 64, row, bar(BAR_FULL_RKV + s));
+                        tma_load_2d(dst + 3 * TILE, &tm_v, uh * 64, row, bar(BAR_FULL_RKV + s));
+                    }
+                    __syncwarp();
+                    if (++s == NS) { s = 0; ph ^= 1; }
+                }
+            }
+            if (alive) {
+                // two end markers, one for each elementwise set; each role hands them on and leaves
+                real_end = gc;
+                for (int e = 0; e < 2 && alive; ++e, ++gc) {
+                    if (gc >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) { alive = false; break; }
+                    if (elect_one()) {
+                        asm volatile("st.shared.v4.s32 [%0], {%1, %2, %3, %4};" ::"r"(sbase + OFF_DESC + 16 * (gc & (NSIDE - 1))),
+                                     "r"(0), "r"(DESC_END), "r"(0), "r"(0) : "memory");
+                        mbar_arrive(bar(BAR_FULL_RKV + s));                 // no copy: the arrival alone completes the phase
+                    }
+                    __syncwarp();
+                    if (++s == NS) { s = 0; ph ^= 1; }
+                }
+            }
+            // Do not leave while copies into this CTA's shared memory may still be in flight.  A stage that an end
+            // marker re-used was released by its consumers first, so only the chunks after those need the wait.
+            const int issued = real_end >= 0 ? real_end : gc;
+            const int from = (real_end >= 0 && alive) ? max(0, issued - NS + 2) : max(0, issued - NS);
+            for (int c = from; c < issued; ++c)
+                mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
+        } else {
         int issued = 0;
         int s = 0, ph = 1;                       // ring stage and the parity of its previous release
         int row = (int)row0;
@@ -681,16 +796,22 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // do not leave while copies into this CTA's shared memory may still be in flight
         for (int c = max(0, issued - NS); c < issued; ++c)
             mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
+        }
     } else if (warp == WARP_MMA_F) {
         // ============================== MMA issuer, input-only products ==============================
         // P_c = R^ K^^T (M = t, N = i, K = c: both operands K-major) and dS_c = K^^T V (M = c, N = j,
         // K = i: both MN-major), interleaved: consecutive tcgen05.mma on one accumulator wait for each
         // other, different accumulators pipeline.
         int s = 0, ph = 0;                       // ring stage and its phase bit
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1;
             if (!mbar_wait_warp(bar(BAR_RK_READY + s), ph, abort_flag)) break;
             if (c >= 2 && !mbar_wait_warp(bar(BAR_F_EMPTY + tb), pt ^ 1, abort_flag)) break;
+            if (PERSIST && chunk_is_end(c)) {        // hand the end marker to the state and score warps
+                if (elect_one()) mbar_arrive(bar(BAR_F_FULL + tb));
+                __syncwarp();
+                break;
+            }
             const bool safe = safe_at(c & (NSIDE - 1));
             const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
             tc_fence_after();
@@ -716,11 +837,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // The masked scores of chunk c exist only after P_c completed, so every product that reads
         // ring stage s is complete when these complete: the last commit releases the stage.
         int s = 0;
-        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
+        for (int c = 0; PERSIST || c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1;
             if (c >= 2 && !mbar_wait_warp(bar(BAR_Y_EMPTY + tb), pt ^ 1, abort_flag)) break;
             if (!mbar_wait_warp(bar(BAR_S_READY + tb), pt, abort_flag)) break;
             if (!mbar_wait_warp(bar(BAR_PP_READY + tb), pt, abort_flag)) break;
+            if (PERSIST && chunk_is_end(c)) {        // hand the end marker to the output warps
+                if (elect_one()) mbar_arrive(bar(BAR_B_DONE + tb));
+                __syncwarp();
+                break;
+            }
             const bool safe = safe_at(c & (NSIDE - 1));
             const uint32_t tr = sbase + OFF_RING + s * STAGE + TILE;
             tc_fence_after();
@@ -748,16 +874,26 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const size_t sb = (size_t)unit * 4096;
         // S[c][j] in accumulator layout: st[n][0..1] = (c_lo, j = 8n+2q, +1), st[n][2..3] = (c_lo+8, same j)
         float st[8][4];
+        auto load_state = [&](size_t base) {         // this lane's part of state_in[unit] (zero without one)
 #pragma unroll
-        for (int n = 0; n < 8; ++n) {
-            if (!SUMMARY && p.state_in) {
-                const float2 lo = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)c_lo * 64 + 8 * n + 2 * q);
-                const float2 hi = *reinterpret_cast<const float2*>(p.state_in + sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
-                st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
-            } else {
-                st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
+            for (int n = 0; n < 8; ++n) {
+                if (!SUMMARY && p.state_in) {
+                    const float2 lo = *reinterpret_cast<const float2*>(p.state_in + base + (size_t)c_lo * 64 + 8 * n + 2 * q);
+                    const float2 hi = *reinterpret_cast<const float2*>(p.state_in + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
+                    st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
+                } else {
+                    st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
+                }
             }
-        }
+        };
+        auto store_state = [&](size_t base) {
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                *reinterpret_cast<float2*>(p.state_out + base + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
+                *reinterpret_cast<float2*>(p.state_out + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
+            }
+        };
+        if (!PERSIST) load_state(sb);
         if (!SUMMARY) {
             // start state of a later segment: fold the summaries of the segments before it, in order
             for (int gg = 0; gg < seg; ++gg) {
@@ -774,16 +910,36 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         float dprod_lo = 1.f, dprod_hi = 1.f;    // summary pass: decay product of the segment for this lane's two rows
         int fb_uses = 0;                         // chunks that took the token-by-token path so far
-        if (!SUMMARY && nchunks > 0) {
+        if (!PERSIST && !SUMMARY && nchunks > 0) {
             store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
             fence_proxy_async();
             __syncwarp();
             mbar_arrive_if(bar(BAR_S_READY), lane == 0);
         }
-        for (int c = 0; c < nchunks; ++c) {
+        for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
+            const Chunk ck = chunk_at(c);
+            if (PERSIST && ck.end) {
+                // Hand the end marker to the issuer of the state-dependent products, under the same condition as a
+                // real operand tile (the products of chunk c-2 are done): the issuer has then consumed this barrier's
+                // previous phase, so the marker's arrival cannot run two phases ahead of its wait.
+                if (c >= 2 && !mbar_wait(bar(BAR_B_DONE + tb), ((c - 2) >> 1) & 1, abort_flag)) break;
+                __syncwarp();
+                mbar_arrive_if(bar(BAR_S_READY + tb), lane == 0);
+                break;
+            }
+            if (PERSIST && ck.first) {
+                // a new unit starts with this chunk: its state replaces the registers, and the operand tile of
+                // this chunk (last read by the products of chunk c-2) takes its bf16 copy
+                load_state((size_t)ck.unit * 4096);
+                if (c >= 2 && !mbar_wait(bar(BAR_B_DONE + tb), ((c - 2) >> 1) & 1, abort_flag)) break;
+                store_acc_bf16(sbase + OFF_SB + tb * TILE, 16 * sp, st, lane);
+                fence_proxy_async();
+                __syncwarp();
+                mbar_arrive_if(bar(BAR_S_READY + tb), lane == 0);
+            }
             bool next_tile_free = c == 0;        // the products of chunk c-1 have finished reading operand tile tb^1
             const uint32_t dl = sbase + OFF_DL + 4 * (sd * 64 + c_lo);
             const float d_lo = ldsf(dl), d_hi = ldsf(dl + 32);        // 2^{a_L} of this lane's two rows
@@ -819,6 +975,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // (The summary pass does not use these tiles at all.)
                 if (!SUMMARY && c >= 1 && !mbar_wait(bar(BAR_B_DONE + (tb ^ 1)), ((c - 1) >> 1) & 1, abort_flag)) break;
                 next_tile_free = true;
+                // the fp32 copy overlays the bf16 rows of the other state warps: all of them have stored theirs first
+                __syncwarp();
+                mbar_arrive_if(bar(BAR_SPRE), lane == 0);
+                if (!mbar_wait(bar(BAR_SPRE), fb_uses & 1, abort_flag)) break;
                 float* scr = reinterpret_cast<float*>(smem + OFF_SB);
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
@@ -840,7 +1000,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (!mbar_wait(bar(BAR_SSYNC), fb_uses & 1, abort_flag)) break;
                 ++fb_uses;
             }
-            if (!SUMMARY && c + 1 < nchunks) {
+            if (!SUMMARY && ck.rem > 0) {
                 const int nb = tb ^ 1;
                 if (!next_tile_free && !mbar_wait(bar(BAR_B_DONE + nb), ((c - 1) >> 1) & 1, abort_flag)) break;
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
@@ -848,6 +1008,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_S_READY + nb), lane == 0);
             }
+            if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
         if (SUMMARY) {
             if (!lds32(abort_flag)) {
@@ -859,21 +1020,23 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     *reinterpret_cast<float2*>(sm + 64 + (c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
                 }
             }
-        } else if (p.state_out && seg == p.nseg - 1 && !lds32(abort_flag)) {
-#pragma unroll
-            for (int n = 0; n < 8; ++n) {
-                *reinterpret_cast<float2*>(p.state_out + sb + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
-                *reinterpret_cast<float2*>(p.state_out + sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
-            }
+        } else if (!PERSIST && p.state_out && seg == p.nseg - 1 && !lds32(abort_flag)) {
+            store_state(sb);
         }
     } else if (warp < WARP_Y0) {
         // ============================== score warps ==============================
         const int sp = warp & 3;                 // rows t = 16*sp .. 16*sp+15 of the score block
         const int g = lane >> 2, q = lane & 3;
-        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
+        for (int c = 0; PERSIST || c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, ppi = tb, sd = c & (NSIDE - 1);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
+            if (PERSIST && chunk_is_end(c)) {    // hand the end marker on, as above (after the products of chunk c-2)
+                if (c >= NPP && !mbar_wait(bar(BAR_B_DONE + ppi), pt ^ 1, abort_flag)) break;
+                __syncwarp();
+                mbar_arrive_if(bar(BAR_PP_READY + ppi), lane == 0);
+                break;
+            }
             const bool safe = safe_at(sd);
             float d_lo = 0.f, d_hi = 0.f;
             if (safe && !C2) {
@@ -929,25 +1092,31 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const bool has_u2 = !SUMMARY && C2 && p.u2 != nullptr;
         const uint32_t u2slab = sbase + OFF_U2 + sp * 2048;
         bool u2_pending = false;                 // a slab copy is in flight; it completes the phase of parity u2_parity
-        int u2_parity = 0;
-        auto load_u2 = [&](int c) {
+        int u2_parity = 0, u2_loads = 0;         // (the slab's barrier completes one phase per load)
+        // row: first row of the chunk whose 16 rows are wanted, in the unit with head column col; rem: chunks after it
+        auto load_u2 = [&](int row, int col, int rem) {
             if (elect_one()) {
                 mbar_expect_tx(bar(BAR_U2 + sp), 2048);
-                tma_load_2d(u2slab, &tm_u2_16, col0, (int)(row0 + (long long)c * L + 16 * sp), bar(BAR_U2 + sp));
+                tma_load_2d(u2slab, &tm_u2_16, col, row + 16 * sp, bar(BAR_U2 + sp));
                 // the slab is single: pull the rows of the chunks after this one into L2 meanwhile, so that
                 // their loads, which can only be issued once the slab is free, are short
-                if (c + 2 < nchunks) tma_prefetch_2d(&tm_u2_16, col0, (int)(row0 + (long long)(c + 2) * L + 16 * sp));
-                if (c + 3 < nchunks) tma_prefetch_2d(&tm_u2_16, col0, (int)(row0 + (long long)(c + 3) * L + 16 * sp));
+                if (rem >= 2) tma_prefetch_2d(&tm_u2_16, col, row + 2 * L + 16 * sp);
+                if (rem >= 3) tma_prefetch_2d(&tm_u2_16, col, row + 3 * L + 16 * sp);
             }
             __syncwarp();
             u2_pending = true;
-            u2_parity = c & 1;
+            u2_parity = u2_loads & 1;
+            ++u2_loads;
         };
-        if (has_u2 && nchunks > 0) load_u2(0);
-        for (int c = 0; c < (SUMMARY ? 0 : nchunks); ++c) {
+        if (!PERSIST && has_u2 && nchunks > 0) load_u2((int)row0, col0, nchunks - 1);
+        for (int c = 0; PERSIST || c < (SUMMARY ? 0 : nchunks); ++c) {
             const int tb = c & 1;
             if (!mbar_wait(bar(BAR_B_DONE + tb), (c >> 1) & 1, abort_flag)) break;
             tc_fence_after();
+            const Chunk ck = chunk_at(c);
+            if (PERSIST && ck.end) break;
+            const int ccol = PERSIST ? ck.h * 64 : col0;                  // this chunk's head column
+            if (PERSIST && has_u2 && ck.first) load_u2(ck.row, ccol, ck.rem);   // (a unit's first slab is not fetched ahead)
             const bool safe = safe_at(c & (NSIDE - 1));
             if (lane == 0) bulk_wait_read<0>();   // this warp's previous store has finished reading the slab
             __syncwarp();
@@ -956,13 +1125,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 // the state warps put in shared memory; writes this chunk's y rows itself
                 mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
                 if (has_u2) {                     // keep the slab's phase in step: consume, then request the next
-                    if (!mbar_wait(bar(BAR_U2 + sp), c & 1, abort_flag)) break;
+                    if (!mbar_wait(bar(BAR_U2 + sp), u2_parity, abort_flag)) break;
                     u2_pending = false;
-                    if (c + 1 < nchunks) load_u2(c + 1);
+                    if (ck.rem > 0) load_u2(ck.row + L, ccol, ck.rem - 1);
                 }
                 if (!mbar_wait(bar(BAR_FB_READY), fb_uses & 1, abort_flag)) break;
-                exact_chunk<true>(reinterpret_cast<float*>(smem + OFF_SB), p, h, sp, lane, row0 + (long long)c * L,
-                                  min(L, len - c * L), C, col0);
+                exact_chunk<true>(reinterpret_cast<float*>(smem + OFF_SB), p, ck.h, sp, lane, ck.row, ck.valid, C, ccol);
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_FB_DONE), lane == 0);
                 ++fb_uses;
@@ -977,7 +1145,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 tmem_ld_16x32(tc, yb);
                 add_acc(ya, yb);
                 if (has_u2) {
-                    if (!mbar_wait(bar(BAR_U2 + sp), c & 1, abort_flag)) break;
+                    if (!mbar_wait(bar(BAR_U2 + sp), u2_parity, abort_flag)) break;
                     u2_pending = false;
                     add_slab_bf16<0>(ya, u2slab, lane);
                 }
@@ -991,17 +1159,17 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (has_u2) {
                     add_slab_bf16<1>(ya, u2slab, lane);
                     __syncwarp();
-                    if (c + 1 < nchunks) load_u2(c + 1);
+                    if (ck.rem > 0) load_u2(ck.row + L, ccol, ck.rem - 1);
                 }
                 store_half_bf16<1>(slab, 0, ya, lane);
             }
             fence_proxy_async();
             __syncwarp();
-            const int rows = min(L, len - c * L) - 16 * sp;
-            const long long grow = row0 + (long long)c * L + 16 * sp;
+            const int rows = ck.valid - 16 * sp;
+            const long long grow = (long long)ck.row + 16 * sp;
             if (rows >= 16) {
                 if (lane == 0) {
-                    tma_store_2d(&tm_y16, col0, (int)grow, slab);
+                    tma_store_2d(&tm_y16, ccol, (int)grow, slab);
                     bulk_commit();
                 }
             } else {
@@ -1011,7 +1179,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     uint4 val;
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(slab + swz(t, ch << 4)));
-                    *reinterpret_cast<uint4*>(p.y + (size_t)(grow + t) * C + col0 + ch * 8) = val;
+                    *reinterpret_cast<uint4*>(p.y + (size_t)(grow + t) * C + ccol + ch * 8) = val;
                 }
                 __syncwarp();
             }
@@ -1027,25 +1195,43 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
         constexpr bool c2 = C2;                          // Finch-C2 form: keys times (1 - w), no bonus
         // (the bonus vector is only read where the bonus is computed: not in the Finch-C2 form, not in a summary pass)
-        const float4 u4 = (c2 || SUMMARY) ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
-        const float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
+        const float4 u4 = (c2 || SUMMARY || PERSIST) ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(p.u + h * 64 + 4 * cq);
+        float2 ua = make_float2(u4.x, u4.y), ub = make_float2(u4.z, u4.w);
+        int u_head = -1;                                 // persistent launches: the head whose bonus vector ua, ub hold
         uint32_t roff[4];                                // swizzled byte offsets of this lane's 8 bytes in its 4 rows
 #pragma unroll
         for (int tt = 0; tt < 4; ++tt) roff[tt] = swz(8 * tq + 4 * th + tt, 8 * cq);
         const float2 kLog2e = make_float2(LOG2E, LOG2E), kLogLog = make_float2(LOG2_LOG2E, LOG2_LOG2E);
         int s = eset, ph = 0;                            // ring stage of this set's current chunk and its phase bit
-        for (int c = eset; c < nchunks; c += N_ESET) {
+        for (int c = eset; PERSIST || c < nchunks; c += N_ESET) {
             const int sd = c & (NSIDE - 1);
             const uint32_t tx = sbase + OFF_RING + s * STAGE, tv = tx + 3 * TILE;
             uint32_t ax[4];                              // this lane's 8 bytes in its 4 rows of the x tile; r at +TILE, k at +2 TILE
 #pragma unroll
             for (int tt = 0; tt < 4; ++tt) ax[tt] = tx + roff[tt];
             if (!mbar_wait(bar(BAR_FULL_RKV + s), ph, abort_flag)) break;
-            if (len - c * L < L) {
+            Chunk ck;                                    // (this role needs the valid-token count, the head and the end flag only)
+            if constexpr (PERSIST) {
+                const int meta = (int)lds32(sbase + OFF_DESC + 16 * (c & (NSIDE - 1)) + 4);
+                ck.valid = meta & 0xff; ck.h = meta >> 16; ck.end = (meta & DESC_END) != 0;
+            } else {
+                ck.valid = min(L, len - c * L); ck.h = h; ck.end = false;
+            }
+            if (PERSIST && ck.end) {                     // hand the end marker to the issuer of the input-only products
+                __syncwarp();
+                mbar_arrive_if(bar(BAR_RK_READY + s), lane == 0);
+                break;
+            }
+            if (PERSIST && !c2 && ck.h != u_head) {      // the stream moved on to another head: its bonus vector
+                const float4 un = *reinterpret_cast<const float4*>(p.u + ck.h * 64 + 4 * cq);
+                ua = make_float2(un.x, un.y); ub = make_float2(un.z, un.w);
+                u_head = ck.h;
+            }
+            if (ck.valid < L) {
                 // Ragged last chunk: rows past the end of the sequence hold another sequence's tokens (or the
                 // out-of-range fill).  Each lane rewrites its own part of those rows before it reads them
                 // back: x = -inf (no decay), r = k = 0; the v rows are zeroed for the tensor core.
-                const int valid = len - c * L;
+                const int valid = ck.valid;
 #pragma unroll
                 for (int tt = 0; tt < 4; ++tt)
                     if (8 * tq + 4 * th + tt >= valid) {
@@ -1228,7 +1414,7 @@ inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_
     return g;
 }
 
-// Opts the four instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
+// Opts the six instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
 inline bool chunked_kernel_attributes()
 {
     static PerDeviceFlag attr_set;                   // zero-initialised
@@ -1238,7 +1424,9 @@ inline bool chunked_kernel_attributes()
         if (cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
             return false;
         attr_set.set(dev);
     }
@@ -1267,10 +1455,30 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     int seg_chunks = 0, nseg = 1;
     if (scratch) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
         size_t need = 0;
-        nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);
+        nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);   // (never splits with more units than half the SMs)
         if (nseg > 1 && (need > scratch_bytes || units * nseg > 0x7fffffffLL)) nseg = 1;
     }
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
+    const int n_sm = sm_count();
+    // More units than SMs: one CTA per SM walks a stream of units, so that a unit's pipeline fill overlaps the
+    // drain of the one before it.  That saves about 4.5 us per unit and costs about 3 % more instructions per
+    // chunk (descriptor reads), so it is taken for short units or many units per SM (measured: 512 units of 64
+    // chunks lose 3 %, 1184 units of 32 chunks gain 2 %, 4096 units of 8 chunks gain 30 %).  Packed calls draw
+    // their units from a counter in the scratch (their lengths differ); dense calls take every gridDim-th unit
+    // (drawing them from the counter too was measured 3 % slower).
+    const int max_chunks = (T + ck::L - 1) / ck::L;
+    if (nseg == 1 && n_sm > 0 && units > n_sm && (units >= 6LL * n_sm || max_chunks <= 48) &&
+        (!cu || (scratch && scratch_bytes >= sizeof(unsigned int)))) {
+        p.n_units = (int)units;
+        if (cu) {
+            p.ticket = reinterpret_cast<unsigned int*>(scratch);
+            if (cudaMemsetAsync(p.ticket, 0, sizeof(unsigned int), st) != cudaSuccess) return GF_ERR_CUDA;
+        }
+        if (c2) ck::wkv6_chunked_kernel<false, true, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        else ck::wkv6_chunked_kernel<false, false, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+    }
     if (nseg > 1) {
         if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
         else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);

@@ -449,3 +449,74 @@ def test_calls_from_two_host_threads_on_their_own_streams():
     for i, inp in enumerate(cases):
         y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
         check(results[i][0], results[i][1], y_ref, s_ref, 5e-3, f"thread {i}")
+
+
+# ---- more units than SMs: one CTA per SM walks a stream of units (persistent launch)
+
+@pytest.mark.parametrize("B,T,H,x_hi", [(40, 200, 5, -1.0), (19, 64, 16, -1.0), (33, 130, 10, 2.5), (400, 1, 1, -1.0),
+                                          (7, 700, 32, -1.0)])
+def test_dense_call_with_more_units_than_sms_matches_oracle(B, T, H, x_hi):
+    """Several units per CTA, unit boundaries at every alignment of the ring and the double buffers (T = 64: one
+    chunk per unit; T = 1: one token), strong decays that take the token-by-token path inside the stream."""
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=7000 + B, state_std=0.1, x_lo=-6.0 if x_hi < 0 else -1.0, x_hi=x_hi)
+    d = inp.to(DEV)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    before = gf.launch_count()
+    y, s = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in)
+    assert gf.launch_count() - before == 1
+    y2, s2 = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in)
+    gf.last_device_status()
+    assert torch.equal(y, y2) and torch.equal(s, s2)
+    y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+    check(y, s, y_ref, s_ref, 5e-3, f"persistent dense B{B} T{T} H{H}")
+    # every unit on its own: a unit that got another unit's state or bonus vector would show here
+    yn, sn = y.float().cpu().numpy(), s.cpu().numpy()
+    for b in range(0, B, max(1, B // 7)):
+        for h in range(H):
+            assert orc.rel_l2(yn[b, :, h], y_ref[b, :, h]) <= 6e-3, (b, h)
+            assert orc.rel_l2(sn[b, h], s_ref[b, h]) <= 6e-3, (b, h)
+
+
+def test_packed_call_with_more_units_than_sms_draws_units_dynamically():
+    """Packed, 60 sequences x 4 heads with lengths from 0 to 300 (empty sequences, single tokens, ragged tails):
+    units are handed out through the counter in the workspace; with the workspace taken away the same call
+    runs one CTA per unit; both match the oracle."""
+    import random
+    rng = random.Random(5)
+    lens = [rng.choice([0, 1, 63, 64, 65, rng.randint(2, 300)]) for _ in range(60)]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    H = 4
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=7100, state_std=0.1)
+    d = inp.to(DEV)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    assert gf.workspace_bytes(len(lens), max(lens), H, 64) > 0
+    y, s = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in)
+    y2, s2 = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in)
+    y1, s1 = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in, split=False)
+    gf.last_device_status()
+    assert torch.equal(y, y2) and torch.equal(s, s2)
+    assert torch.equal(y, y1) and torch.equal(s, s1)      # the same arithmetic per unit, whoever runs it
+    y_ref, s_ref = orc.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, cu, inp.state_in)
+    check(y, s, y_ref, s_ref, 5e-3, "persistent packed")
+    for i, n in enumerate(lens):
+        a, b = int(cu[i]), int(cu[i + 1])
+        if n == 0:
+            assert torch.equal(s[i].cpu(), inp.state_in[i])
+        else:
+            check(y[a:b], s[i], y_ref[a:b], s_ref[i], 6e-3, f"persistent packed seq {i} len {n}")
+
+
+def test_persistent_launch_without_states_and_in_place_state():
+    B, T, H = 30, 150, 8
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=7200, state_std=0.1)
+    d = inp.to(DEV)
+    y0, s0 = gf.prefill(d.r, d.k, d.v, d.x, d.u, None)                       # zero start state
+    st = d.state_in.clone()
+    y1, s1 = gf.prefill(d.r, d.k, d.v, d.x, d.u, st, state_out=st)            # state updated in place
+    y2, _ = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in, want_state=False)  # no final state wanted
+    gf.last_device_status()
+    y_ref0, s_ref0 = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, None)
+    y_ref1, s_ref1 = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+    check(y0, s0, y_ref0, s_ref0, 5e-3, "zero state")
+    check(y1, s1, y_ref1, s_ref1, 5e-3, "in place")
+    assert torch.equal(y1, y2)

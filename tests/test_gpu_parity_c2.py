@@ -157,3 +157,35 @@ def test_c2_step_matches_oracle_and_chains_to_a_prefill(with_u2):
         ys.append(yt)
     gf.last_device_status()
     check(torch.stack(ys, 1), st, inp, u2, f"chain of step_c2 u2={with_u2}")
+
+
+@pytest.mark.parametrize("with_u2", [True, False])
+def test_c2_more_units_than_sms(with_u2):
+    """Persistent launch of the Finch-C2 form: the second-value slab of a unit's first chunk is fetched when the
+    stream reaches the unit."""
+    inp, u2 = make(25, 210, 8, 880, with_u2=with_u2)
+    y, s = run(inp, u2)
+    check(y, s, inp, u2, f"persistent C2 u2={with_u2}")
+
+
+def test_c2_packed_more_units_than_sms():
+    import random
+    rng = random.Random(9)
+    lens = [rng.choice([0, 1, 64, rng.randint(2, 260)]) for _ in range(50)]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    H = 4
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=890, state_std=0.1)
+    u2 = torch.randn(inp.r.shape, generator=torch.Generator().manual_seed(891)).bfloat16()
+    d = inp.to(DEV)
+    y, s = gf.prefill_varlen_c2(d.r, d.k, d.v, d.x, u2.to(DEV), d.cu_seqlens, max(lens), d.state_in)
+    gf.last_device_status()
+    for i, n in enumerate(lens):
+        a, b = int(cu[i]), int(cu[i + 1])
+        if n == 0:
+            assert torch.equal(s[i].cpu(), inp.state_in[i])
+            continue
+        sl = lambda t: t[a:b][None].contiguous()
+        y_ref, s_ref = orc.prefill_c2(sl(inp.r), sl(inp.k), sl(inp.v), sl(inp.x), sl(u2), inp.state_in[i][None].contiguous())
+        ey = orc.rel_l2(y[a:b].float().cpu().numpy(), y_ref[0])
+        es = orc.rel_l2(s[i].cpu().numpy(), s_ref[0])
+        assert ey <= TOL and es <= TOL, (i, n, ey, es)
