@@ -159,11 +159,12 @@ GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
  * S <- diag(D) S + dS, which composes associatively across segments of the wkv_t sum) in the workspace,
  * the second launch folds them into each segment's start state and computes y.  Results agree with the
  * unsplit call to rounding.  Calls with MORE units than SMs run one CTA per SM that walks a stream of units
- * (a unit's pipeline fill overlaps the drain of the one before); a packed call of that kind draws its units
- * from a 4-byte counter at the start of the workspace (zeroed on `stream` by the call itself) and falls back
- * to one CTA per unit without a workspace; a dense one needs none.  gf_wkv6_workspace_bytes returns what
- * gf_wkv6_prefill(B,T,H,N) (packed: B = S, T = max_seqlen) would use on the current device: the summaries of
- * a split, 256 for more units than SMs, else 0.  gf_wkv6_set_workspace registers a caller-owned
+ * (a unit's pipeline fill overlaps the drain of the one before); a packed call of that kind draws its units,
+ * longest sequences first, from a counter in the workspace (a small kernel of the call itself, on `stream`,
+ * zeroes the counter and ranks the sequences there) and falls back to one CTA per unit without a workspace; a
+ * dense one needs none.  gf_wkv6_workspace_bytes returns what gf_wkv6_prefill(B,T,H,N) (packed: B = S,
+ * T = max_seqlen) would use on the current device: the summaries of a split, 64 + 4*S bytes (rounded up to
+ * 256) for more units than SMs, else 0.  gf_wkv6_set_workspace registers a caller-owned
  * DEVICE buffer (256-byte aligned; NULL unregisters) for all later calls of this process; the library
  * never frees it.  A registered buffer that is too small is ignored (the call runs unsplit).  Calls that
  * use the workspace and overlap on the GPU (different streams) race on it. */

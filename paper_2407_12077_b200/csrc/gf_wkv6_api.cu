@@ -384,8 +384,8 @@ size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N)
     int seg_chunks = 0;
     size_t need = 0;
     gf::choose_split((long long)B * H, T, gf::sm_count(), &seg_chunks, &need);
-    // a packed call with more units than SMs draws its units from a counter in the workspace
-    if (need == 0 && (long long)B * H > gf::sm_count()) need = 256;
+    // a packed call with more units than SMs draws its units, longest sequences first, from a counter in the workspace
+    if (need == 0 && (long long)B * H > gf::sm_count()) need = (gf::persistent_scratch_bytes(B) + 255) / 256 * 256;
     return need;
 }
 

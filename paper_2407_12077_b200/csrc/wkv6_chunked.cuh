@@ -465,6 +465,9 @@ struct Params {
     // in length); NULL: unit = blockIdx.x + k gridDim.x (equal lengths).
     int n_units;
     unsigned int* ticket;
+    // With a ticket: sequences in the order in which their units are handed out (longest first, so that the
+    // launch does not end on a long unit while the other SMs idle); NULL: in index order.
+    const int32_t* order;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -712,7 +715,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     u = blockIdx.x + k * gridDim.x;
                 }
                 if (u >= p.n_units) break;
-                const int useq = u / p.H, uh = u % p.H;
+                int useq = u / p.H;
+                const int uh = u % p.H;
+                if (p.ticket && p.order) {               // the ticket counts through the sequences longest first
+                    useq = p.order[useq];
+                    u = useq * p.H + uh;
+                }
                 long long urow0;
                 int ulen;
                 if (p.cu_seqlens) {
@@ -1433,6 +1441,32 @@ inline bool chunked_kernel_attributes()
     return true;
 }
 
+// Prepares the scratch of a packed persistent launch: zeroes the unit counter and, for up to ORDER_MAX_SEQ
+// sequences, writes the sequence indices by decreasing length (rank by counting; ties by index).
+constexpr int ORDER_MAX_SEQ = 8192;
+constexpr size_t ORDER_OFFSET = 64;                  // bytes from the counter to the order array
+__global__ void __launch_bounds__(1024)
+wkv6_order_kernel(const int32_t* __restrict__ cu, int S, unsigned int* counter, int32_t* order)
+{
+    __shared__ int len[ORDER_MAX_SEQ];
+    if (threadIdx.x == 0) *counter = 0u;
+    if (!order) return;
+    for (int i = threadIdx.x; i < S; i += blockDim.x) len[i] = cu[i + 1] - cu[i];
+    __syncthreads();
+    for (int i = threadIdx.x; i < S; i += blockDim.x) {
+        const int li = len[i];
+        int rank = 0;
+        for (int j = 0; j < S; ++j) rank += (len[j] > li) || (len[j] == li && j < i);
+        order[rank] = i;
+    }
+}
+
+// Scratch a packed call with more units than SMs uses: the counter and the order array.
+inline size_t persistent_scratch_bytes(int n_seq)
+{
+    return ORDER_OFFSET + (n_seq <= ORDER_MAX_SEQ ? (size_t)n_seq * sizeof(int32_t) : 0);
+}
+
 // Launches the chunked kernel.  Dense: cu == nullptr, n_seq = B, T = sequence length.
 // Packed: cu = device cu_seqlens, n_seq = S, T = max_seqlen.  total_rows = rows of the [rows][H*64] tensors.
 // scratch / scratch_bytes: optional device memory for the sequence split (see choose_split); without
@@ -1472,7 +1506,13 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         p.n_units = (int)units;
         if (cu) {
             p.ticket = reinterpret_cast<unsigned int*>(scratch);
-            if (cudaMemsetAsync(p.ticket, 0, sizeof(unsigned int), st) != cudaSuccess) return GF_ERR_CUDA;
+            int32_t* order = nullptr;
+            if (n_seq <= ORDER_MAX_SEQ && scratch_bytes >= persistent_scratch_bytes(n_seq))
+                order = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(scratch) + ORDER_OFFSET);
+            p.order = order;
+            wkv6_order_kernel<<<1, 1024, 0, st>>>(cu, n_seq, p.ticket, order);
+            launches->fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
         }
         if (c2) ck::wkv6_chunked_kernel<false, true, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
         else ck::wkv6_chunked_kernel<false, false, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
