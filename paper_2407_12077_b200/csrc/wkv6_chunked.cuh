@@ -34,10 +34,12 @@
 // accumulator rows 16*(warp mod 4) .. +15 of a 64-row tile.
 // Every wait is bounded: on expiry the kernel raises a status flag and all roles leave.
 //
-// Two template parameters select variants of the same pipeline: SUMMARY (the first pass of a call
-// that splits its sequences into segments: state only, no r / scores / outputs; see Params) and C2
+// Three template parameters select variants of the same pipeline: SUMMARY (the first pass of a call
+// that splits its sequences into segments: state only, no r / scores / outputs; see Params), C2
 // (the Finch-C2 form: keys times one minus their decay, no bonus, optional per-token vector added to
-// the output).
+// the output) and PERSIST (calls with more units than SMs: one CTA per SM walks a stream of units,
+// the producer leaving a descriptor per chunk and two end markers that every role hands on, so that
+// the pipeline is filled and drained once per CTA instead of once per unit).
 #pragma once
 #include <atomic>
 #include <cuda.h>
