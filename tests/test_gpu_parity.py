@@ -520,3 +520,44 @@ def test_persistent_launch_without_states_and_in_place_state():
     check(y0, s0, y_ref0, s_ref0, 5e-3, "zero state")
     check(y1, s1, y_ref1, s_ref1, 5e-3, "in place")
     assert torch.equal(y1, y2)
+
+
+def test_random_many_unit_shapes_against_oracle():
+    """Seeded sweep over calls with more units than SMs: dense and packed, lengths with every kind of tail, decay
+    ranges from tame to chunks that all take the token-by-token path; every unit against the oracle."""
+    import random
+    rng = random.Random(20240713)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    for it in range(14):
+        H = rng.choice([1, 2, 3, 5, 8, 16])
+        units = rng.randint(149, 900)
+        x_lo, x_hi = rng.choice([(-6.0, -1.0), (-6.0, -1.0), (-3.0, 1.5), (-1.0, 2.5), (-8.0, 0.5)])
+        if rng.random() < 0.5:
+            S = max(1, units // H)
+            lens = [rng.choice([0, 1, 63, 64, 65, 128, rng.randint(1, 330)]) for _ in range(S)]
+            lens[0] = max(lens[0], 3)
+            cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+            inp = synth.make_varlen(cu, H, 64, "bf16", seed=9100 + it, state_std=0.1, x_lo=x_lo, x_hi=x_hi)
+            d = inp.to(DEV)
+            y, s = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, max(lens), d.state_in)
+            gf.last_device_status()
+            y_ref, s_ref = orc.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, cu, inp.state_in)
+            yn, sn = y.float().cpu().numpy(), s.cpu().numpy()
+            for i, n in enumerate(lens):
+                a, b = int(cu[i]), int(cu[i + 1])
+                for h in range(H):
+                    if n == 0:
+                        assert np.array_equal(sn[i, h], inp.state_in[i, h].numpy()), (it, i, h)
+                    else:
+                        assert orc.rel_l2(yn[a:b, h], y_ref[a:b, h]) <= 6e-3 and orc.rel_l2(sn[i, h], s_ref[i, h]) <= 6e-3, (it, i, h, n)
+        else:
+            B, T = max(1, units // H), rng.choice([1, 7, 64, 65, 128, 129, 192, rng.randint(2, 330)])
+            inp = synth.make_dense(B, T, H, 64, "bf16", seed=9100 + it, state_std=0.1, x_lo=x_lo, x_hi=x_hi)
+            d = inp.to(DEV)
+            y, s = gf.prefill(d.r, d.k, d.v, d.x, d.u, d.state_in)
+            gf.last_device_status()
+            y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+            yn, sn = y.float().cpu().numpy(), s.cpu().numpy()
+            for b in range(B):
+                for h in range(H):
+                    assert orc.rel_l2(yn[b, :, h], y_ref[b, :, h]) <= 6e-3 and orc.rel_l2(sn[b, h], s_ref[b, h]) <= 6e-3, (it, b, h, T)
