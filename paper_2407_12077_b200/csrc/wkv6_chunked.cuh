@@ -786,26 +786,26 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             for (int c = from; c < issued; ++c)
                 mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
         } else {
-        int issued = 0;
-        int s = 0, ph = 1;                       // ring stage and the parity of its previous release
-        int row = (int)row0;
-        for (int c = 0; c < nchunks; ++c, row += L) {
-            if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) break;
-            const uint32_t dst = sbase + OFF_RING + s * STAGE;
-            if (elect_one()) {
-                mbar_expect_tx(bar(BAR_FULL_RKV + s), SUMMARY ? 3 * TILE : STAGE);
-                tma_load_2d(dst, &tm_x, col0, row, bar(BAR_FULL_RKV + s));
-                if (!SUMMARY) tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
-                tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
-                tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
+            int issued = 0;
+            int s = 0, ph = 1;                       // ring stage and the parity of its previous release
+            int row = (int)row0;
+            for (int c = 0; c < nchunks; ++c, row += L) {
+                if (c >= NS && !mbar_wait_warp(bar(BAR_EMPTY_RKV + s), ph, abort_flag)) break;
+                const uint32_t dst = sbase + OFF_RING + s * STAGE;
+                if (elect_one()) {
+                    mbar_expect_tx(bar(BAR_FULL_RKV + s), SUMMARY ? 3 * TILE : STAGE);
+                    tma_load_2d(dst, &tm_x, col0, row, bar(BAR_FULL_RKV + s));
+                    if (!SUMMARY) tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BAR_FULL_RKV + s));
+                    tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BAR_FULL_RKV + s));
+                    tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BAR_FULL_RKV + s));
+                }
+                __syncwarp();
+                issued = c + 1;
+                if (++s == NS) { s = 0; ph ^= 1; }
             }
-            __syncwarp();
-            issued = c + 1;
-            if (++s == NS) { s = 0; ph ^= 1; }
-        }
-        // do not leave while copies into this CTA's shared memory may still be in flight
-        for (int c = max(0, issued - NS); c < issued; ++c)
-            mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
+            // do not leave while copies into this CTA's shared memory may still be in flight
+            for (int c = max(0, issued - NS); c < issued; ++c)
+                mbar_wait_warp(bar(BAR_FULL_RKV + c % NS), (c / NS) & 1, abort_flag, false);
         }
     } else if (warp == WARP_MMA_F) {
         // ============================== MMA issuer, input-only products ==============================
