@@ -33,7 +33,7 @@ STATE_BYTES_PER_UNIT = 64 * 64 * 4    # fp32 final state written once per (b,h) 
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (null once the kernel has changed since the counters were taken)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 1275837440  # 4 x (268.50 + 50.46 MB) measured at T=4096, scaled by tokens
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 1275564032  # 4 x (268.53 + 50.36 MB) measured at T=4096, scaled by tokens
 
 
 def parse():
