@@ -304,6 +304,36 @@ def main():
                  "achieved": ln_bytes / (ln_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                  "frac": ln_bytes / (ln_ms * 1e-3) / 1e9 / peak, "algorithmic_bytes": ln_bytes}
 
+    # ---- batched serving prefill (packed variable-length call, 64 sequences of 128..4096 tokens: more units than SMs,
+    # one persistent CTA per SM), timed on its own after the step like the LayerNorm above
+    packed = None
+    if world == 1:
+        c4 = synth.CONFIGS["cfg4"]
+        cu = synth.make_lengths(c4["S"], c4["len_min"], c4["len_max"], seed=4000)
+        vin = synth.make_varlen(cu, c4["H"], N, "bf16", seed=4001, device=dev, state_std=c4["state_std"])
+        v_total, v_max = int(cu[-1]), int((cu[1:] - cu[:-1]).max())
+        v_y = torch.empty_like(vin.r)
+        v_s = torch.empty((c4["S"], c4["H"], N, N), device=dev)
+        v_call = lambda: gf.prefill_varlen(vin.r, vin.k, vin.v, vin.x, vin.u, vin.cu_seqlens, v_max, vin.state_in,
+                                           state_out=v_s, y=v_y, stream=stream)
+        for _ in range(3):
+            v_call()
+        v_a, v_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        v_a.record(stream)
+        for _ in range(10):
+            v_call()
+        v_b.record(stream)
+        torch.cuda.synchronize()
+        gf.last_device_status()
+        v_ms = v_a.elapsed_time(v_b) / 10
+        v_bytes = v_total * c4["H"] * BYTES_PER_TOKEN_HEAD + 2 * c4["S"] * c4["H"] * STATE_BYTES_PER_UNIT
+        packed = {"kernel": "gf_wkv6_prefill_varlen (one call: rank kernel + persistent prefill kernel)",
+                  "workload": f"cfg4: {c4['S']} sequences of {c4['len_min']}..{c4['len_max']} tokens, {v_total} tokens, H={c4['H']}",
+                  "call_ms": v_ms, "value": v_total * c4["H"] / (v_ms * 1e-3), "unit": UNIT, "bound": "hbm",
+                  "achieved": v_bytes / (v_ms * 1e-3) / 1e9, "peak": peak, "frac": v_bytes / (v_ms * 1e-3) / 1e9 / peak,
+                  "algorithmic_bytes": v_bytes}
+        del vin, v_y, v_s
+
     # ---- end to end through the host-buffer entry point: pinned host inputs -> y on the host
     e2e = None
     if not args.no_e2e:
@@ -369,7 +399,8 @@ def main():
                        "precision": "bf16 r/k/v/x/y and tensor-core operands, fp32 accumulation, decay sums and state",
                        "l2": "inputs larger than L2 (1.34 GB per call, distinct buffers per call)",
                        "parallelism": f"(b,h) units replicated per GPU x{world}, no collective"},
-            "roofline": roofline, "layernorm_heads": layernorm, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "roofline": roofline, "layernorm_heads": layernorm, "packed_prefill": packed, "cpu_baseline": cpu_baseline,
+            "e2e": e2e,
             "gpu_launches": launches,
             "clocks": clocks,
         }
