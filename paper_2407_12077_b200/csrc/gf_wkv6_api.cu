@@ -142,9 +142,9 @@ gf_status_t step_impl(const IO* r, const IO* k, const IO* v, const IO* x, const 
     if (s != GF_OK) return s;
     const long long units = (long long)B * H;
     if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
-    gf::wkv6_step_kernel<IO><<<(unsigned)units, gf::ST_THREADS, 0, st>>>(r, k, v, x, u, state_in, state_out, y, H);
+    const cudaError_t e = gf::launch_step<IO, false>((unsigned)units, st, r, k, v, x, u, state_in, state_out, y, H, nullptr);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return launch_result();
+    return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
 
 }  // namespace
@@ -258,10 +258,10 @@ gf_status_t gf_wkv6_step_c2(const void* r, const void* k, const void* v, const v
     if (y == r || y == k || y == v || y == x || y == u2) return GF_ERR_INVALID_ARG;
     const long long units = (long long)B * H;
     if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
-    gf::wkv6_step_kernel<bf, true><<<(unsigned)units, gf::ST_THREADS, 0, (cudaStream_t)stream>>>(
-        (const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, nullptr, state_in, state_out, (bf*)y, H, (const bf*)u2);
+    const cudaError_t e = gf::launch_step<bf, true>((unsigned)units, (cudaStream_t)stream, (const bf*)r, (const bf*)k, (const bf*)v,
+                                                   (const bf*)x, nullptr, state_in, state_out, (bf*)y, H, (const bf*)u2);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return launch_result();
+    return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
 
 gf_status_t gf_wkv6_sequence_summary(const void* k, const void* v, const void* x, float* summary, int B, int T, int H,

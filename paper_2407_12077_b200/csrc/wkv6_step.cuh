@@ -25,11 +25,16 @@ wkv6_step_kernel(const IO* __restrict__ r, const IO* __restrict__ k, const IO* _
     __shared__ __align__(16) float rs[64], ks[64], vs[64], ws[64];
     __shared__ float ruk[2];
     __shared__ __align__(16) float part[16][64];
+    // Launched with programmatic stream serialisation: the next step kernel of the stream may be scheduled while
+    // this one drains (it holds at its own wait below), and this one touches no global memory before the kernels
+    // ahead of it have completed and flushed.  Without that launch attribute both instructions do nothing.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int unit = blockIdx.x, h = unit % H;
     const int tid = threadIdx.x;
     const size_t voff = (size_t)unit * 64;
     const size_t sbase = (size_t)unit * 64 * 64;
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // issue the state loads first so they overlap the vector staging
     const int ig = tid >> 4, jq = tid & 15;
     float4 S[4];
@@ -73,6 +78,24 @@ wkv6_step_kernel(const IO* __restrict__ r, const IO* __restrict__ k, const IO* _
         if (C2 && u2) s += to_f32(u2[voff + tid]);
         y[voff + tid] = from_f32<IO>(s);
     }
+}
+
+// Launch with programmatic stream serialisation (see the kernel): back-to-back decode steps lose the launch gap.
+template <typename IO, bool C2>
+inline cudaError_t launch_step(unsigned grid, cudaStream_t st, const IO* r, const IO* k, const IO* v, const IO* x, const float* u,
+                               const float* state_in, float* state_out, IO* y, int H, const IO* u2)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(ST_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, wkv6_step_kernel<IO, C2>, r, k, v, x, u, state_in, state_out, y, H, u2);
 }
 
 }  // namespace gf
