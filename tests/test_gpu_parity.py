@@ -561,3 +561,25 @@ def test_random_many_unit_shapes_against_oracle():
             for b in range(B):
                 for h in range(H):
                     assert orc.rel_l2(yn[b, :, h], y_ref[b, :, h]) <= 6e-3 and orc.rel_l2(sn[b, h], s_ref[b, h]) <= 6e-3, (it, b, h, T)
+
+
+@pytest.mark.parametrize("S", [5000, 8200])
+def test_packed_call_with_thousands_of_short_sequences(S):
+    """Thousands of sequences of 0..3 tokens, one head: the rank kernel at its size limit (S = 5000) and the
+    index-order fallback beyond it (S = 8200); every sequence against the oracle."""
+    import random
+    rng = random.Random(S)
+    lens = [rng.randint(0, 3) for _ in range(S)]
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    inp = synth.make_varlen(cu, 1, 64, "bf16", seed=7300 + S, state_std=0.1)
+    d = inp.to(DEV)
+    gf.set_kernel(gf.KERNEL_CHUNKED)
+    y, s = gf.prefill_varlen(d.r, d.k, d.v, d.x, d.u, d.cu_seqlens, 3, d.state_in)
+    gf.last_device_status()
+    y_ref, s_ref = orc.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, cu, inp.state_in)
+    check(y, s, y_ref, s_ref, 5e-3, f"{S} short sequences")
+    sn = s.cpu().numpy()
+    worst = max(orc.rel_l2(sn[i], s_ref[i]) for i in range(S))
+    assert worst <= 6e-3, worst
+    empty = [i for i, n in enumerate(lens) if n == 0]
+    assert all(np.array_equal(sn[i], inp.state_in[i].numpy()) for i in empty[:200])
