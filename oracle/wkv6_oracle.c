@@ -209,3 +209,24 @@ void c2_oracle_layernorm(const double *y, const double *gamma, const double *bet
             o[c] = (yr[c] - mu) * rstd * (gamma ? gamma[c] : 1.0) + (beta ? beta[c] : 0.0);
     }
 }
+
+/* ---------------------------------------------------------------------------------------------------
+ * GOLD key compression: the step that ends linear pre-fill in GoldFinch.  The output x_t of the Finch-C2
+ * layers is multiplied by the learned matrix W^{KD} in R^{D x D/16} and the result stored as the token's
+ * entry of the compressed key cache:
+ *     c_t = x_t W^{KD}                                   (GOLD key compression equation)
+ * x: [rows][D], w: [D][Dc] row-major (Dc = D/16 in the paper; any Dc here), c: [rows][Dc]; every sum in
+ * double, in index order over the D input channels.
+ * Pins (tests/test_oracle_pins_kc.py): brute-force loops on a tiny case, a selection matrix, the all-ones
+ * matrix (row sums), a single non-zero weight (orientation), linearity, the library matrix product in fp64.
+ */
+void gold_oracle_key_compress(const double *x, const double *w, double *c, long rows, long D, long Dc)
+{
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < rows; ++t)
+        for (long n = 0; n < Dc; ++n) {
+            double acc = 0.0;
+            for (long k = 0; k < D; ++k) acc += x[(size_t)t * D + k] * w[(size_t)k * Dc + n];
+            c[(size_t)t * Dc + n] = acc;
+        }
+}

@@ -39,6 +39,7 @@ def _load():
         _lib.wkv6_oracle_prefill_varlen.restype = None
         _lib.wkv6_oracle_prefill_c2.restype = None
         _lib.c2_oracle_layernorm.restype = None
+        _lib.gold_oracle_key_compress.restype = None
     return _lib
 
 
@@ -169,6 +170,21 @@ def layernorm_heads(y, gamma=None, beta=None, eps=1e-5):
     lib.c2_oracle_layernorm(_p(y, d), _p(gamma, d), _p(beta, d), d(float(eps)), _p(out, d),
                             ctypes.c_long(rows), ctypes.c_long(D))
     return out
+
+
+def key_compress(x, w_kd):
+    """GOLD key compression c_t = x_t W^{KD} (the compressed key cache entry of every token).  x: [..., D]
+    (numpy / torch, any float type, widened exactly to float64); w_kd: [D, Dc].  Returns float64 [..., Dc]."""
+    lib = _load()
+    cv = lambda a: np.ascontiguousarray(a.detach().cpu().double().numpy() if hasattr(a, "detach") else np.asarray(a, dtype=np.float64))
+    x, w = cv(x), cv(w_kd)
+    D, Dc = w.shape
+    assert x.shape[-1] == D
+    rows = x.size // D if D else 0
+    c = np.zeros(x.shape[:-1] + (Dc,), dtype=np.float64)
+    d = ctypes.c_double
+    lib.gold_oracle_key_compress(_p(x, d), _p(w, d), _p(c, d), ctypes.c_long(rows), ctypes.c_long(D), ctypes.c_long(Dc))
+    return c
 
 
 def rel_l2(a, b) -> float:
