@@ -242,6 +242,17 @@ GF_API gf_status_t gf_c2_layernorm(const void *y, const float *gamma, const floa
 GF_API gf_status_t gf_c2_layernorm_f32(const float *y, const float *gamma, const float *beta, float eps,
                                 float *out, long long rows, int H, int N, gf_stream_t stream);
 
+/* GOLD key compression, the product that ends linear pre-fill: c_t = x_t W^{KD} (GOLD key compression equation),
+ * the token's entry of the compressed key cache, with W^{KD} the learned D x D/16 matrix.
+ *   x     DEVICE bf16 [rows][D]   (the output of the Finch-C2 layers, one row per token)
+ *   w_kd  DEVICE bf16 [D][Dc]     row-major (Dc = D/16 in the paper)
+ *   c     DEVICE bf16 [rows][Dc]  written; must not alias x or w_kd
+ * bf16 operands on the tensor cores, fp32 accumulation over D, one rounding to bf16.  D must be a multiple of 64
+ * and Dc one of 64, 128, 192, 256 (GF_ERR_UNSUPPORTED otherwise); pointers 16-byte aligned; rows = 0 is a no-op.
+ * Enqueues one kernel on `stream`, allocates nothing, does not synchronise. */
+GF_API gf_status_t gf_gold_key_compress(const void *x, const void *w_kd, void *c, long long rows, int D, int Dc,
+                                 gf_stream_t stream);
+
 GF_API int gf_wkv6_version(void);
 
 #ifdef __cplusplus

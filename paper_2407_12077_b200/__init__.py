@@ -47,6 +47,7 @@ _SIGNATURES = {
     "gf_wkv6_fold_summaries": (_i, [_vp, _vp] + [_i] * 4 + [_vp, _vp]),
     "gf_c2_layernorm": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_c2_layernorm_f32": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
+    "gf_gold_key_compress": (_i, [_vp, _vp, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
     "gf_wkv6_launch_count": (ctypes.c_uint64, []),
@@ -305,6 +306,22 @@ def layernorm_heads(y, gamma=None, beta=None, eps=1e-5, out=None, stream=None):
             _dev(y, "y"), _dev(None if gamma is None else gamma.reshape(H * N), "gamma", torch.float32),
             _dev(None if beta is None else beta.reshape(H * N), "beta", torch.float32), float(eps),
             _dev(out, "out", y.dtype, y.shape), rows, H, N, _stream(stream)), "gf_c2_layernorm" + sfx)
+    return out
+
+
+def key_compress(x, w_kd, out=None, stream=None):
+    """gf_gold_key_compress: c = x @ w_kd.  x: [..., D] bf16 CUDA tensor (contiguous), w_kd: [D, Dc] bf16.
+    Returns c [..., Dc] bf16 (allocated here unless passed as out)."""
+    lib = load_library()
+    D, Dc = w_kd.shape
+    assert x.shape[-1] == D
+    rows = x.numel() // D if D else 0
+    bf = torch.bfloat16
+    if out is None:
+        out = torch.empty(x.shape[:-1] + (Dc,), device=x.device, dtype=bf)
+    with torch.cuda.device(x.device):
+        _check(lib.gf_gold_key_compress(_dev(x, "x", bf), _dev(w_kd, "w_kd", bf, (D, Dc)), _dev(out, "c", bf, x.shape[:-1] + (Dc,)),
+                                        rows, D, Dc, _stream(stream)), "gf_gold_key_compress")
     return out
 
 

@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "key_compress.cuh"
 #include "ln_heads.cuh"
 #include "wkv6_chunked.cuh"
 #include "wkv6_exact.cuh"
@@ -426,6 +427,17 @@ gf_status_t gf_c2_layernorm_f32(const float* y, const float* gamma, const float*
                                 long long rows, int H, int N, gf_stream_t stream)
 {
     return layernorm_call(y, gamma, beta, eps, out, rows, H, N, stream);
+}
+
+gf_status_t gf_gold_key_compress(const void* x, const void* w_kd, void* c, long long rows, int D, int Dc, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (rows < 0 || D < 0 || Dc < 0) return GF_ERR_INVALID_ARG;
+    if (rows == 0 || Dc == 0) return GF_OK;
+    if (D == 0 || (D & 63) || (Dc & 63) || Dc > 256) return GF_ERR_UNSUPPORTED;
+    if (rows >= (1LL << 31) - 256) return GF_ERR_INVALID_ARG;
+    if (!x || !w_kd || !c || misaligned(x) || misaligned(w_kd) || misaligned(c) || c == x || c == w_kd) return GF_ERR_INVALID_ARG;
+    return gf::key_compress((const bf*)x, (const bf*)w_kd, (bf*)c, rows, D, Dc, (cudaStream_t)stream, &g_launches);
 }
 
 const char* gf_status_string(gf_status_t s)

@@ -144,3 +144,16 @@ def test_layernorm_entry_points_validate_before_any_launch():
         assert _call(name, A, A + 4, A, f(1e-5), A, 4, 32, 64, None) == 1
         assert _call(name, A, A, A, f(1e-5), A, 4, 3, 5, None) == 2            # H*N not a multiple of 8
         assert _call(name, A, A, A, f(1e-5), A, 4, 129, 64, None) == 2         # wider than 8192 channels
+
+
+def test_key_compress_entry_point_validates_before_any_launch():
+    name = "gf_gold_key_compress"
+    assert _call(name, A, A + 0x100, A + 0x200, 0, 2048, 128, None) == 0            # no rows: no-op
+    assert _call(name, A, A + 0x100, A + 0x200, -1, 2048, 128, None) == 1
+    assert _call(name, None, A + 0x100, A + 0x200, 8, 2048, 128, None) == 1
+    assert _call(name, A, A + 0x100, None, 8, 2048, 128, None) == 1
+    assert _call(name, A + 2, A + 0x100, A + 0x200, 8, 2048, 128, None) == 1        # misaligned
+    assert _call(name, A, A + 0x100, A, 8, 2048, 128, None) == 1                    # c aliases x
+    assert _call(name, A, A + 0x100, A + 0x200, 8, 2000, 128, None) == 2            # D not a multiple of 64
+    assert _call(name, A, A + 0x100, A + 0x200, 8, 2048, 48, None) == 2             # Dc not a multiple of 64
+    assert _call(name, A, A + 0x100, A + 0x200, 8, 8192, 512, None) == 2            # Dc beyond 256
