@@ -3,7 +3,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
 
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
-cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide
+cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -113,6 +113,18 @@ def run(case, reps, scale):
         fn = lambda: gf.layernorm_heads(y, gamma, beta, 1e-5, out=out)
         return dict(case=case, shape=f"rows={rows} D={H * 64} bf16", units=rows * H, bytes=rows * H * 64 * 4 + 8 * H * 64,
                     ms=_time(fn, reps))
+    if case in ("kc-cfg2", "kc-wide"):      # GOLD key compression over the tokens of cfg2 (D = 2048 -> 128; wide: 4096 -> 256)
+        k = c["cfg2"]
+        rows, D = k["B"] * sc(k["T"]), (4096 if case == "kc-wide" else k["H"] * 64)
+        g = torch.Generator(device=DEV).manual_seed(11)
+        x = torch.randn((rows, D), device=DEV, generator=g).bfloat16()
+        w = (torch.randn((D, D // 16), device=DEV, generator=g) / D ** 0.5).bfloat16()
+        out = torch.empty((rows, D // 16), device=DEV, dtype=torch.bfloat16)
+        fn = lambda: gf.key_compress(x, w, out=out)
+        r = dict(case=case, shape=f"rows={rows} D={D} Dc={D // 16} bf16", units=rows, bytes=rows * D * 2 + rows * (D // 16) * 2 + D * (D // 16) * 2,
+                 ms=_time(fn, reps))
+        r["tflops"] = 2.0 * rows * D * (D // 16) / (r["ms"] * 1e-3) / 1e12
+        return r
     if case in ("cfg4-prefill", "cfg4-decode", "cfg4-decode-layers"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -163,7 +175,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide"]
 
 
 def main():
