@@ -215,7 +215,9 @@ inline gf_status_t key_compress(const __nv_bfloat16* x, const __nv_bfloat16* w, 
     if (n_sm <= 0 || dev < 0) return GF_ERR_CUDA;
     static PerDeviceFlag attr_set;
     if (!attr_set.is_set(dev)) {
-        if (cudaFuncSetAttribute(kc::key_compress_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
+        if (cudaFuncSetAttribute(kc::key_compress_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(kc::key_compress_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(kc::key_compress_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(kc::key_compress_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(kc::key_compress_kernel<1, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(kc::key_compress_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess)
@@ -224,15 +226,21 @@ inline gf_status_t key_compress(const __nv_bfloat16* x, const __nv_bfloat16* w, 
     }
     CUtensorMap tx, tw, tc;
     if (!ck::make_map(&tx, x, rows, D, 64) || !ck::make_map(&tw, w, D, Dc, 64) || !ck::make_map(&tc, c, rows, Dc, 32)) return GF_ERR_CUDA;
-    const int nb = Dc / 64, mblk = nb <= 2 ? 2 : 1;
+    // 256-row tiles halve the re-reads of W but need enough rows to give every SM a tile
+    const int nb = Dc / 64, mblk = (nb <= 2 && rows >= 256LL * n_sm) ? 2 : 1;
     const long long n_tiles = (rows + 128LL * mblk - 1) / (128LL * mblk);
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);
     kc::KcParams p{rows, D / 64};
-    switch (nb) {
-    case 1: kc::key_compress_kernel<2, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
-    case 2: kc::key_compress_kernel<2, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
-    case 3: kc::key_compress_kernel<1, 3><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
-    default: kc::key_compress_kernel<1, 4><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+    if (mblk == 2) {
+        if (nb == 1) kc::key_compress_kernel<2, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);
+        else kc::key_compress_kernel<2, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);
+    } else {
+        switch (nb) {
+        case 1: kc::key_compress_kernel<1, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        case 2: kc::key_compress_kernel<1, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        case 3: kc::key_compress_kernel<1, 3><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        default: kc::key_compress_kernel<1, 4><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        }
     }
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
