@@ -247,8 +247,9 @@ GF_API gf_status_t gf_c2_layernorm_f32(const float *y, const float *gamma, const
  *   x     DEVICE bf16 [rows][D]   (the output of the Finch-C2 layers, one row per token)
  *   w_kd  DEVICE bf16 [D][Dc]     row-major (Dc = D/16 in the paper)
  *   c     DEVICE bf16 [rows][Dc]  written; must not alias x or w_kd
- * bf16 operands on the tensor cores, fp32 accumulation over D, one rounding to bf16.  D must be a multiple of 64
- * and Dc one of 64, 128, 192, 256 (GF_ERR_UNSUPPORTED otherwise); pointers 16-byte aligned; rows = 0 is a no-op.
+ * bf16 operands on the tensor cores, fp32 accumulation over D, one rounding to bf16.  D and Dc must be multiples
+ * of 8 and Dc at most 256 (GF_ERR_UNSUPPORTED otherwise; D = 768 -> 48 and D = 2048 -> 128 are the paper's two
+ * models); pointers 16-byte aligned; rows = 0 is a no-op.
  * Enqueues one kernel on `stream`, allocates nothing, does not synchronise. */
 GF_API gf_status_t gf_gold_key_compress(const void *x, const void *w_kd, void *c, long long rows, int D, int Dc,
                                  gf_stream_t stream);

@@ -434,7 +434,7 @@ gf_status_t gf_gold_key_compress(const void* x, const void* w_kd, void* c, long 
     using bf = __nv_bfloat16;
     if (rows < 0 || D < 0 || Dc < 0) return GF_ERR_INVALID_ARG;
     if (rows == 0 || Dc == 0) return GF_OK;
-    if (D == 0 || (D & 63) || (Dc & 63) || Dc > 256) return GF_ERR_UNSUPPORTED;
+    if (D == 0 || (D & 7) || (Dc & 7) || Dc > 256) return GF_ERR_UNSUPPORTED;
     if (rows >= (1LL << 31) - 256) return GF_ERR_INVALID_ARG;
     if (!x || !w_kd || !c || misaligned(x) || misaligned(w_kd) || misaligned(c) || c == x || c == w_kd) return GF_ERR_INVALID_ARG;
     return gf::key_compress((const bf*)x, (const bf*)w_kd, (bf*)c, rows, D, Dc, (cudaStream_t)stream, &g_launches);

@@ -38,7 +38,7 @@ constexpr uint32_t KC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | 
 
 struct KcParams {
     long long rows;
-    int ksteps;                                       // D / 64
+    int ksteps;                                       // ceil(D / 64)
 };
 
 // One accumulator row per lane: 32 consecutive fp32 columns of the lane's row in this warp's sub-partition.
@@ -205,11 +205,13 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
 
 }  // namespace kc
 
-// c[rows][Dc] = x[rows][D] w[D][Dc]; D a multiple of 64, Dc in {64, 128, 192, 256}.
+// c[rows][Dc] = x[rows][D] w[D][Dc]; D and Dc multiples of 8 (16-byte rows for TMA), Dc <= 256.  Widths that are not
+// multiples of 64 ride on TMA's bounds handling: the missing input channels and output columns are read as zeros
+// and the store clips the columns past Dc.
 inline gf_status_t key_compress(const __nv_bfloat16* x, const __nv_bfloat16* w, __nv_bfloat16* c, long long rows, int D, int Dc,
                                 cudaStream_t st, std::atomic<uint64_t>* launches)
 {
-    if (rows <= 0 || rows >= (1LL << 31) - 256 || D <= 0 || (D & 63) || Dc <= 0 || (Dc & 63) || Dc > 256) return GF_ERR_INVALID_ARG;
+    if (rows <= 0 || rows >= (1LL << 31) - 256 || D <= 0 || (D & 7) || Dc <= 0 || (Dc & 7) || Dc > 256) return GF_ERR_INVALID_ARG;
     const int n_sm = sm_count();
     const int dev = current_device();
     if (n_sm <= 0 || dev < 0) return GF_ERR_CUDA;
@@ -227,10 +229,10 @@ inline gf_status_t key_compress(const __nv_bfloat16* x, const __nv_bfloat16* w, 
     CUtensorMap tx, tw, tc;
     if (!ck::make_map(&tx, x, rows, D, 64) || !ck::make_map(&tw, w, D, Dc, 64) || !ck::make_map(&tc, c, rows, Dc, 32)) return GF_ERR_CUDA;
     // 256-row tiles halve the re-reads of W but need enough rows to give every SM a tile
-    const int nb = Dc / 64, mblk = (nb <= 2 && rows >= 256LL * n_sm) ? 2 : 1;
+    const int nb = (Dc + 63) / 64, mblk = (nb <= 2 && rows >= 256LL * n_sm) ? 2 : 1;
     const long long n_tiles = (rows + 128LL * mblk - 1) / (128LL * mblk);
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);
-    kc::KcParams p{rows, D / 64};
+    kc::KcParams p{rows, (D + 63) / 64};
     if (mblk == 2) {
         if (nb == 1) kc::key_compress_kernel<2, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);
         else kc::key_compress_kernel<2, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);

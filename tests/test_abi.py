@@ -154,6 +154,6 @@ def test_key_compress_entry_point_validates_before_any_launch():
     assert _call(name, A, A + 0x100, None, 8, 2048, 128, None) == 1
     assert _call(name, A + 2, A + 0x100, A + 0x200, 8, 2048, 128, None) == 1        # misaligned
     assert _call(name, A, A + 0x100, A, 8, 2048, 128, None) == 1                    # c aliases x
-    assert _call(name, A, A + 0x100, A + 0x200, 8, 2000, 128, None) == 2            # D not a multiple of 64
-    assert _call(name, A, A + 0x100, A + 0x200, 8, 2048, 48, None) == 2             # Dc not a multiple of 64
+    assert _call(name, A, A + 0x100, A + 0x200, 8, 2044, 128, None) == 2            # D not a multiple of 8
+    assert _call(name, A, A + 0x100, A + 0x200, 8, 2048, 44, None) == 2             # Dc not a multiple of 8
     assert _call(name, A, A + 0x100, A + 0x200, 8, 8192, 512, None) == 2            # Dc beyond 256

@@ -30,7 +30,7 @@ def compare(c, ref, what):
 
 
 @pytest.mark.parametrize("rows", [1, 63, 64, 65, 255, 256, 257, 1000])
-@pytest.mark.parametrize("D,Dc", [(64, 64), (128, 128), (1024, 64), (2048, 128), (3072, 192), (4096, 256)])
+@pytest.mark.parametrize("D,Dc", [(64, 64), (128, 128), (768, 48), (1024, 64), (2048, 128), (3072, 192), (4096, 256), (200, 8), (1000, 136)])
 def test_key_compress_matches_oracle(rows, D, Dc):
     x, w = draw(rows, D, Dc, seed=rows + D)
     canary = torch.full((rows + 2, Dc), 777.0, dtype=torch.bfloat16, device=DEV)
