@@ -5,9 +5,10 @@
 // With Dc = D/16 the product does 2*Dc = 256 flops per 2-byte element of x it reads (D = 2048): it sits at
 // the crossing of the HBM and tensor rooflines, so x is read exactly once and W (D*Dc*2 bytes, L2-resident)
 // as rarely as tensor memory allows.  One persistent CTA per SM walks row tiles of MBLK*128 tokens; a tile's
-// MBLK x NB accumulators (128 rows x 64 fp32 columns each, NB = Dc/64) take at most 256 of the 512 columns
-// of tensor memory, so there are two sets: the products of the next tile run while the epilogue drains
-// this one.  Every 64-row slice of W that enters shared memory serves MBLK*128 tokens.
+// MBLK x NB accumulators (128 rows x 64 fp32 columns each, NB = ceil(Dc/64)) take, up to Dc = 128, at most 256
+// of the 512 columns of tensor memory, so there are two sets: the products of the next tile run while the
+// epilogue drains this one (wider outputs fill all 512 columns with one set).  Every 64-row slice of W that
+// enters shared memory serves MBLK*128 tokens.
 //   warp 0      TMA producer: per 64 input channels, 2*MBLK tiles of x and NB tiles of W into a ring stage
 //   warp 1      tensor-memory allocation; an elected lane issues the MBLK*NB*4 tcgen05.mma (128x64x16) of a stage
 //   warps 2-5   epilogue: the 32 accumulator rows of the own sub-partition -> bf16 slab -> TMA store (32-row
@@ -25,13 +26,12 @@ namespace kc {
 using namespace ck;                                   // PTX wrappers, descriptors, TILE, bounded waits
 
 constexpr int KC_THREADS = 192;
-constexpr int KC_NS = 4;                              // ring stages
-constexpr int KC_MAX_TILES = 6;                       // x tiles + W tiles per stage (48 KB)
-constexpr int KC_STAGE = KC_MAX_TILES * TILE;
-constexpr int KC_OFF_SLAB = KC_NS * KC_STAGE;         // [4 warps][32 rows x 128 B]
+constexpr int KC_RING = 24 * TILE;                    // ring of x and W tiles: 4 stages of up to 6 tiles or 3 of up to 8
+constexpr int KC_MAX_NS = 4;
+constexpr int KC_OFF_SLAB = KC_RING;                  // [4 warps][32 rows x 128 B]
 constexpr int KC_OFF_MISC = KC_OFF_SLAB + 4 * 4096;   // abort word, tensor-memory address, barriers
 constexpr int KC_SMEM = KC_OFF_MISC + 256 + 1024;     // + slack for manual 1024-byte alignment
-enum { KC_FULL = 0, KC_EMPTY = KC_NS, KC_ACC_FULL = 2 * KC_NS, KC_ACC_EMPTY = KC_ACC_FULL + 2, KC_BAR_COUNT = KC_ACC_EMPTY + 2 };
+enum { KC_FULL = 0, KC_EMPTY = KC_MAX_NS, KC_ACC_FULL = 2 * KC_MAX_NS, KC_ACC_EMPTY = KC_ACC_FULL + 2, KC_BAR_COUNT = KC_ACC_EMPTY + 2 };
 static_assert(16 + 8 * KC_BAR_COUNT <= 256, "barrier block");
 // instruction descriptor: fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = 64
 constexpr uint32_t KC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
@@ -61,8 +61,14 @@ __global__ void __launch_bounds__(KC_THREADS, 1)
 key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                     const __grid_constant__ CUtensorMap tm_c32, const KcParams p)
 {
-    static_assert(2 * MBLK + NB <= KC_MAX_TILES && MBLK * NB * 64 <= 256, "tile shape");
-    constexpr int ACC_COLS = 256;                    // one accumulator set; two sets fill tensor memory
+    constexpr int STAGE_TILES = 2 * MBLK + NB;       // x tiles + W tiles per stage
+    constexpr int KC_NS = STAGE_TILES <= 6 ? 4 : 3;  // ring stages
+    constexpr int KC_STAGE = STAGE_TILES * TILE;
+    static_assert(KC_NS * KC_STAGE <= KC_RING && MBLK * NB * 64 <= 512, "tile shape");
+    // a tile's accumulators in up to 256 columns: two sets, the epilogue of one tile overlaps the products of the
+    // next; in 512 columns: one set
+    constexpr int NSETS = MBLK * NB * 64 <= 256 ? 2 : 1;
+    constexpr int ACC_COLS = 512 / NSETS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -85,7 +91,7 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (warp == 1) tmem_alloc(sbase + KC_OFF_MISC + 8, 2 * ACC_COLS);
+    if (warp == 1) tmem_alloc(sbase + KC_OFF_MISC + 8, 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -120,9 +126,9 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
         int it = 0, ti = 0;
         bool alive = true;
         for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
-            const int ab = ti & 1;                   // accumulator set of this tile
-            // the epilogue has read this set's previous tile (two tiles back) out of tensor memory
-            if (ti >= 2 && !mbar_wait_warp(bar(KC_ACC_EMPTY + ab), ((ti >> 1) + 1) & 1, abort_flag)) break;
+            const int ab = NSETS == 2 ? (ti & 1) : 0, use = NSETS == 2 ? (ti >> 1) : ti;   // accumulator set and its use count
+            // the epilogue has read this set's previous tile out of tensor memory
+            if (use >= 1 && !mbar_wait_warp(bar(KC_ACC_EMPTY + ab), (use + 1) & 1, abort_flag)) break;
             tc_fence_after();
             for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
                 const int s = it % KC_NS;
@@ -154,8 +160,8 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
         const uint32_t slab = sbase + KC_OFF_SLAB + (warp - 2) * 4096;
         int ti = 0;
         for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x, ++ti) {
-            const int ab = ti & 1;
-            if (!mbar_wait(bar(KC_ACC_FULL + ab), (ti >> 1) & 1, abort_flag)) break;
+            const int ab = NSETS == 2 ? (ti & 1) : 0, use = NSETS == 2 ? (ti >> 1) : ti;
+            if (!mbar_wait(bar(KC_ACC_FULL + ab), use & 1, abort_flag)) break;
             tc_fence_after();
             const long long row0 = t * tile_rows;
 #pragma unroll
@@ -199,7 +205,7 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, 2 * ACC_COLS);
+        tmem_dealloc(tmem, 512);
     }
 }
 
@@ -222,20 +228,26 @@ inline gf_status_t key_compress(const __nv_bfloat16* x, const __nv_bfloat16* w, 
             cudaFuncSetAttribute(kc::key_compress_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(kc::key_compress_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
             cudaFuncSetAttribute(kc::key_compress_kernel<1, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
-            cudaFuncSetAttribute(kc::key_compress_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess)
+            cudaFuncSetAttribute(kc::key_compress_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(kc::key_compress_kernel<2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(kc::key_compress_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kc::KC_SMEM) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set.set(dev);
     }
     CUtensorMap tx, tw, tc;
     if (!ck::make_map(&tx, x, rows, D, 64) || !ck::make_map(&tw, w, D, Dc, 64) || !ck::make_map(&tc, c, rows, Dc, 32)) return GF_ERR_CUDA;
     // 256-row tiles halve the re-reads of W but need enough rows to give every SM a tile
-    const int nb = (Dc + 63) / 64, mblk = (nb <= 2 && rows >= 256LL * n_sm) ? 2 : 1;
+    const int nb = (Dc + 63) / 64, mblk = rows >= 256LL * n_sm ? 2 : 1;
     const long long n_tiles = (rows + 128LL * mblk - 1) / (128LL * mblk);
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);
     kc::KcParams p{rows, (D + 63) / 64};
     if (mblk == 2) {
-        if (nb == 1) kc::key_compress_kernel<2, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);
-        else kc::key_compress_kernel<2, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p);
+        switch (nb) {
+        case 1: kc::key_compress_kernel<2, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        case 2: kc::key_compress_kernel<2, 2><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        case 3: kc::key_compress_kernel<2, 3><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        default: kc::key_compress_kernel<2, 4><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;
+        }
     } else {
         switch (nb) {
         case 1: kc::key_compress_kernel<1, 1><<<grid, kc::KC_THREADS, kc::KC_SMEM, st>>>(tx, tw, tc, p); break;

@@ -52,9 +52,10 @@ def test_orientation_with_a_selection_matrix_is_exact():
     assert torch.equal(c.cpu(), x[:, ::16])
 
 
-def test_more_row_tiles_than_sms_and_leading_dimensions():
+@pytest.mark.parametrize("D,Dc", [(2048, 128), (3072, 192), (4096, 256), (768, 48)])
+def test_more_row_tiles_than_sms_and_leading_dimensions(D, Dc):
     """[B, T, D] input with enough rows for several tiles per persistent CTA (40000 rows, 157 tiles of 256)."""
-    B, T, D, Dc = 4, 10000, 2048, 128
+    B, T = 4, 10000
     g = torch.Generator().manual_seed(9)
     x = torch.randn(B, T, D, generator=g).bfloat16()
     w = (torch.randn(D, Dc, generator=g) / D ** 0.5).bfloat16()
