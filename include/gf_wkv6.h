@@ -163,11 +163,13 @@ GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
  * longest sequences first, from a counter in the workspace (a small kernel of the call itself, on `stream`,
  * zeroes the counter and ranks the sequences there) and falls back to one CTA per unit without a workspace; a
  * dense one needs none.  gf_wkv6_workspace_bytes returns what gf_wkv6_prefill(B,T,H,N) (packed: B = S,
- * T = max_seqlen) would use on the current device: the summaries of a split, 64 + 4*S bytes (rounded up to
- * 256) for more units than SMs, else 0.  gf_wkv6_set_workspace registers a caller-owned
+ * T = max_seqlen) would use on the current device: the summaries and start-state copies of a split, 64 + 4*S
+ * bytes (rounded up to 256) for more units than SMs, else 0.  gf_wkv6_set_workspace registers a caller-owned
  * DEVICE buffer (256-byte aligned; NULL unregisters) for all later calls of this process; the library
- * never frees it.  A registered buffer that is too small is ignored (the call runs unsplit).  Calls that
- * use the workspace and overlap on the GPU (different streams) race on it. */
+ * never frees it.  With a registered buffer that is too small the call splits into as many segments as fit
+ * (or runs unsplit).  A split call with a start state keeps a copy of it in the workspace and reads only the
+ * copy once its second launch runs, so state_out may be state_in there too.  Calls that use the workspace
+ * and overlap on the GPU (different streams) race on it. */
 GF_API size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N);
 GF_API gf_status_t gf_wkv6_set_workspace(void *dev_ptr, size_t bytes);
 
@@ -181,16 +183,20 @@ GF_API gf_status_t gf_wkv6_set_workspace(void *dev_ptr, size_t bytes);
  * fixed array of GF_WKV6_STATIC_SCRATCH_BYTES in the library's device image (every GPU that loads the
  * library holds it until the process exits).  It allocates and frees nothing and ignores the registered
  * workspace; inputs, outputs, layouts and results are those of gf_wkv6_prefill.
- *   - Limit: a call whose split needs more than the built-in scratch (gf_wkv6_workspace_bytes(B,T,H,N) >
- *     GF_WKV6_STATIC_SCRATCH_BYTES) returns GF_ERR_WORKSPACE and enqueues nothing.  The size covers
- *     B*H <= 32 units at any T (the long-context shape: one sequence, 32 heads); calls that do not split
- *     need no scratch and always pass.
+ *   - Limit: the split takes the largest segment count (at most the one gf_wkv6_prefill would take) whose
+ *     scratch -- per (sequence, head) unit one 16 640-byte summary for every segment but the last and a
+ *     16 384-byte copy of the start state -- fits the array.  The size is that of 32 units cut four ways (one
+ *     long sequence of 32 heads on a 148-SM GPU); up to 64 units fit with two segments.  A call that would
+ *     split but does not fit even with two segments (65 to 74 units on 148 SMs) returns GF_ERR_WORKSPACE
+ *     and enqueues nothing.  Calls that do not split (more units than half the SMs, or fewer than 16 chunks
+ *     of 64 tokens) need no scratch and always pass.
+ *   - It always runs the chunked tensor-core kernel: gf_wkv6_set_kernel is not consulted.
  *   - The first call on each device looks up the array's device address (with that device current), so
  *     make that first call before any stream capture begins on that device.
  *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to be
  *     cleared: the first launch of a call writes every entry its second launch reads.  Calls that overlap
  *     on the GPU (different streams, or different host threads) race on it: serialise them. */
-#define GF_WKV6_STATIC_SCRATCH_BYTES 1597440u      /* 96 segment summaries of (64 + 64*64) floats */
+#define GF_WKV6_STATIC_SCRATCH_BYTES 2121728u      /* 32 units x (3 summaries of (64 + 64*64) floats + 64*64 floats) */
 GF_API gf_status_t gf_wkv6_prefill_static(const void *r, const void *k, const void *v, const void *x,
                                    const float *u, const float *state_in, float *state_out, void *y,
                                    int B, int T, int H, int N, gf_stream_t stream);

@@ -325,14 +325,14 @@ def key_compress(x, w_kd, out=None, stream=None):
     return out
 
 
-STATIC_SCRATCH_BYTES = 1597440       # GF_WKV6_STATIC_SCRATCH_BYTES
+STATIC_SCRATCH_BYTES = 2121728       # GF_WKV6_STATIC_SCRATCH_BYTES
 
 
 def prefill_static(r, k, v, x, u, state_in, state_out, y, stream=None) -> None:
     """gf_wkv6_prefill_static: the dense bf16 prefill for callers that cannot allocate.  Nothing is
     allocated here either: y [B,T,H,N] bf16 and state_out [B,H,N,N] fp32 (or None) are the caller's,
-    and the sequence split uses the scratch built into the library.  Raises GfError(GF_ERR_WORKSPACE)
-    when the call would need more than STATIC_SCRATCH_BYTES of it."""
+    and the sequence split uses the scratch built into the library (as many segments as fit into its
+    STATIC_SCRATCH_BYTES).  Raises GfError(GF_ERR_WORKSPACE) when not even two segments fit."""
     lib = load_library()
     B, T, H, N = r.shape
     bf = torch.bfloat16

@@ -189,10 +189,14 @@ gf_status_t gf_wkv6_prefill_static(const void* r, const void* k, const void* v, 
     if (T == 0) return pass_state(state_in, state_out, (size_t)B * H, st);
     gf_status_t s = check_ptrs(r, k, v, x, u, state_in, state_out, y);
     if (s != GF_OK) return s;
+    // The split takes as many segments as the built-in array holds; a call that would split but does not fit
+    // even with two segments is refused rather than run at a fraction of the GPU.
     int seg_chunks = 0;
     size_t need = 0;
-    gf::choose_split((long long)B * H, T, gf::sm_count(), &seg_chunks, &need);
-    if (need > GF_WKV6_STATIC_SCRATCH_BYTES) return GF_ERR_WORKSPACE;     // beyond the built-in scratch
+    const int n_sm = gf::sm_count();
+    if (gf::choose_split((long long)B * H, T, n_sm, &seg_chunks, &need) > 1 &&
+        gf::choose_split((long long)B * H, T, n_sm, &seg_chunks, &need, GF_WKV6_STATIC_SCRATCH_BYTES) == 1)
+        return GF_ERR_WORKSPACE;                                          // beyond the built-in scratch
     float* scratch = static_scratch();
     if (!scratch) return GF_ERR_CUDA;
     return gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out, (bf*)y,

@@ -470,6 +470,10 @@ struct Params {
     // With a ticket: sequences in the order in which their units are handed out (longest first, so that the
     // launch does not end on a long unit while the other SMs idle); NULL: in index order.
     const int32_t* order;
+    // Split calls with a start state: the summary launch copies state_in[unit] here ([unit][64][64] fp32, in
+    // the scratch) and every CTA of the main launch takes its start state from the copy, so that nothing
+    // reads state_in once the first state_out has been written (state_out may be state_in).  NULL: no copy.
+    float* state_copy;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -884,18 +888,29 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         const size_t sb = (size_t)unit * 4096;
         // S[c][j] in accumulator layout: st[n][0..1] = (c_lo, j = 8n+2q, +1), st[n][2..3] = (c_lo+8, same j)
         float st[8][4];
-        auto load_state = [&](size_t base) {         // this lane's part of state_in[unit] (zero without one)
+        // the start states of this launch: the caller's, or (main launch of a split call) the summary launch's copy
+        const float* s_src = (!SUMMARY && p.state_copy) ? p.state_copy : p.state_in;
+        auto load_state = [&](size_t base) {         // this lane's part of the start state of a unit (zero without one)
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
-                if (!SUMMARY && p.state_in) {
-                    const float2 lo = *reinterpret_cast<const float2*>(p.state_in + base + (size_t)c_lo * 64 + 8 * n + 2 * q);
-                    const float2 hi = *reinterpret_cast<const float2*>(p.state_in + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
+                if (!SUMMARY && s_src) {
+                    const float2 lo = *reinterpret_cast<const float2*>(s_src + base + (size_t)c_lo * 64 + 8 * n + 2 * q);
+                    const float2 hi = *reinterpret_cast<const float2*>(s_src + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
                     st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
                 } else {
                     st[n][0] = st[n][1] = st[n][2] = st[n][3] = 0.f;
                 }
             }
         };
+        if (SUMMARY && seg == 0 && p.state_in && p.state_copy) {
+            // first pass of a split call: keep the unit's start state for the second pass (see Params::state_copy)
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                const size_t lo = sb + (size_t)c_lo * 64 + 8 * n + 2 * q, hi = sb + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q;
+                *reinterpret_cast<float2*>(p.state_copy + lo) = *reinterpret_cast<const float2*>(p.state_in + lo);
+                *reinterpret_cast<float2*>(p.state_copy + hi) = *reinterpret_cast<const float2*>(p.state_in + hi);
+            }
+        }
         auto store_state = [&](size_t base) {
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
@@ -1404,24 +1419,36 @@ inline bool make_map(CUtensorMap* tm, const void* base, long long rows, long lon
 
 // Chooses the sequence split of a call: with fewer (sequence, head) units than half the SMs, each
 // sequence is cut into up to 8 segments of at least 8 chunks so that the grid fills the GPU (T: the
-// sequence length, for a packed call the longest one).  Returns the
-// number of segments (1: no split) and sets seg_chunks; summary_bytes is the scratch the split needs.
-inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_t* summary_bytes)
+// sequence length, for a packed call the longest one).  Returns the number of segments (1: no split) and
+// sets seg_chunks; summary_bytes is the scratch the split uses: per unit one summary for every segment but
+// the last and a copy of the start state.  cap_bytes bounds that scratch: the split takes the largest
+// segment count that fits (1 if not even two segments do).
+constexpr size_t STATE_FLOATS = 64 * 64;
+inline size_t split_scratch_bytes(long long units, int nseg)
+{
+    return (size_t)units * ((size_t)(nseg - 1) * ck::SUMMARY_FLOATS + STATE_FLOATS) * sizeof(float);
+}
+inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_t* summary_bytes,
+                        size_t cap_bytes = ~(size_t)0)
 {
     *seg_chunks = 0;
     *summary_bytes = 0;
     const int nchunks = (T + ck::L - 1) / ck::L;
     if (units <= 0 || n_sm <= 0 || units * 2 > n_sm) return 1;
-    int g = (int)(n_sm / units);
-    if (g > 8) g = 8;
-    if (g > nchunks / 8) g = nchunks / 8;
-    if (g < 2) return 1;
-    const int sc = (nchunks + g - 1) / g;
-    g = (nchunks + sc - 1) / sc;
-    if (g < 2) return 1;
-    *seg_chunks = sc;
-    *summary_bytes = (size_t)units * (g - 1) * ck::SUMMARY_FLOATS * sizeof(float);
-    return g;
+    int want = (int)(n_sm / units);
+    if (want > 8) want = 8;
+    if (want > nchunks / 8) want = nchunks / 8;
+    for (; want >= 2; --want) {
+        const int sc = (nchunks + want - 1) / want;
+        const int g = (nchunks + sc - 1) / sc;
+        if (g < 2) return 1;
+        const size_t bytes = split_scratch_bytes(units, g);
+        if (bytes > cap_bytes) continue;
+        *seg_chunks = sc;
+        *summary_bytes = bytes;
+        return g;
+    }
+    return 1;
 }
 
 // Opts the six instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
@@ -1480,7 +1507,10 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
                                    size_t scratch_bytes = 0, const __nv_bfloat16* u2 = nullptr, int c2 = 0)
 {
     const long long units = (long long)n_seq * H;
-    if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0 || total_rows >= (1LL << 31) - 64) return GF_ERR_INVALID_ARG;
+    if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
+    // what this kernel cannot take (32-bit TMA row coordinates with a chunk of slack; no tensor-map encoder in the
+    // driver) is reported as unsupported, so that the caller can run the token-by-token kernel instead
+    if (total_rows >= (1LL << 31) - 64 || !ck::encode_fn()) return GF_ERR_UNSUPPORTED;
     if (!chunked_kernel_attributes()) return GF_ERR_CUDA;
     CUtensorMap tr, tk, tv, tx, ty, tu2;
     const long long C = (long long)H * 64;
@@ -1491,10 +1521,11 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     int seg_chunks = 0, nseg = 1;
     if (scratch) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
         size_t need = 0;
-        nseg = choose_split(units, T, sm_count(), &seg_chunks, &need);   // (never splits with more units than half the SMs)
-        if (nseg > 1 && (need > scratch_bytes || units * nseg > 0x7fffffffLL)) nseg = 1;
+        nseg = choose_split(units, T, sm_count(), &seg_chunks, &need, scratch_bytes);   // (never splits with more units than half the SMs)
+        if (nseg > 1 && units * nseg > 0x7fffffffLL) nseg = 1;
     }
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
+    if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
     const int n_sm = sm_count();
     // More units than SMs: one CTA per SM walks a stream of units, so that a unit's pipeline fill overlaps the
     // drain of the one before it.  That saves about 4.5 us per unit and costs about 3 % more instructions per
