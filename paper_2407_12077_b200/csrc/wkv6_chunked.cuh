@@ -19,12 +19,12 @@
 // Warp roles (992 threads), pipelined across chunks through mbarriers:
 //   warp 0        TMA producer: {x,r,k,v} tiles of a chunk into one stage of a 5-stage ring
 //   warp 1        tensor-memory allocation; an elected lane issues P = R^ K^^T and dS = K^^T V
-//   warp 2        an elected lane issues Y0 = R^ S_0 and PV = P' V
+//   warp 2        an elected lane issues Y = R^ S_0 + P' V (one accumulator)
 //   warps 3-6     state: S <- diag(2^{a_L}) (S + dS) in fp32 registers for the whole sequence;
 //                 publishes a bf16 copy of every chunk-start state as an MMA operand; for a chunk on
 //                 the token-by-token path it parks the fp32 state in shared memory instead
 //   warps 7-10    scores: P from tensor memory -> P' = tril(P,-1) + diag(bonus) -> bf16 operand tile
-//   warps 11-14   output: Y0 + PV from tensor memory -> bf16 -> TMA store (each warp its own 16 rows);
+//   warps 11-14   output: Y from tensor memory -> bf16 -> TMA store (each warp its own 16 rows);
 //                 runs the token-by-token path (16 value channels per warp) when a chunk needs it
 //   warps 15-30   elementwise, two sets of eight warps taking alternate chunks: decay and
 //                 cumulative sum (phase A), then in place R^ = r 2^{a_{t-1}}, K^ = k 2^{-a_t}
@@ -79,7 +79,7 @@ constexpr int N_EW = 8;                // elementwise warps per set
 constexpr int N_ESET = 2;              // elementwise sets (alternate chunks)
 constexpr int N_GW = 4;                // warps per tensor-memory reader group (one per sub-partition)
 constexpr int WARP_MMA_F = 1;          // issues P = R^ K^^T and dS = K^^T V; owns the tensor-memory allocation
-constexpr int WARP_MMA_B = 2;          // issues Y0 = R^ S_0 and PV = P' V
+constexpr int WARP_MMA_B = 2;          // issues Y = R^ S_0 + P' V
 constexpr int WARP_S0 = 3;             // state warps
 constexpr int WARP_P0 = WARP_S0 + N_GW;   // score warps
 constexpr int WARP_Y0 = WARP_P0 + N_GW;   // output warps
@@ -92,8 +92,8 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 constexpr uint32_t TRY_WAIT_HINT_NS = 20000;                  // a waiting thread may be suspended this long per try
 
 // tensor memory: 64 fp32 columns per 64x64 accumulator, two buffers each
-constexpr int TM_COLS = 512;
-constexpr int TM_P = 0, TM_DS = 128, TM_Y0 = 256, TM_PV = 384;
+constexpr int TM_COLS = 512;          // (384 are used; the allocation is a power of two)
+constexpr int TM_P = 0, TM_DS = 128, TM_Y = 256;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int STAGE = 4 * TILE;                            // one ring stage: x, r -> R^, k -> K^, v
@@ -117,7 +117,7 @@ enum {
     BAR_PP_READY = BAR_S_READY + 2,      // masked-score operand tile written
     BAR_F_FULL = BAR_PP_READY + 2,       // P and dS accumulators complete
     BAR_F_EMPTY = BAR_F_FULL + 2,        // ... and read back by the state and score warps
-    BAR_B_DONE = BAR_F_EMPTY + 2,        // Y0 and PV accumulators complete; state / score operand tiles free again
+    BAR_B_DONE = BAR_F_EMPTY + 2,        // Y accumulator complete; state / score operand tiles free again
     BAR_Y_EMPTY = BAR_B_DONE + 2,        // ... and read back by the output warps
     BAR_ESYNC = BAR_Y_EMPTY + 2,         // one per elementwise set
     BAR_SSYNC = BAR_ESYNC + 2,           // token-by-token path only: state-warp rendezvous after the fp32 copy is re-read,
@@ -517,16 +517,6 @@ __device__ __forceinline__ void add_slab_bf16(float (&acc)[4][4], uint32_t slab,
     }
 }
 
-__device__ __forceinline__ void add_acc(float (&a)[4][4], const float (&b)[4][4])
-{
-#pragma unroll
-    for (int n = 0; n < 4; ++n) {
-        const float2 lo = add2(make_float2(a[n][0], a[n][1]), make_float2(b[n][0], b[n][1]));
-        const float2 hi = add2(make_float2(a[n][2], a[n][3]), make_float2(b[n][2], b[n][3]));
-        a[n][0] = lo.x; a[n][1] = lo.y; a[n][2] = hi.x; a[n][3] = hi.y;
-    }
-}
-
 // P' = tril(P, -1) + diag(bonus) on columns 32*HALF .. +31 of one warp's 16 rows (rows 16*SP + g
 // and + 8) of the score block.
 template <int SP, int HALF>
@@ -556,6 +546,29 @@ __device__ __forceinline__ void mask_scores_sp(int sp, float (&acc)[4][4], int g
     case 2: mask_scores<2, HALF>(acc, g, q, d_lo, d_hi); break;
     default: mask_scores<3, HALF>(acc, g, q, d_lo, d_hi); break;
     }
+}
+
+// oa, ob += the decay totals of the NQ elementwise warps before this one (slots of 64 floats from `tot`; this lane's
+// four channels).  The loads are issued together and the sums formed pairwise, so that the latency is one
+// shared-memory round trip plus log2(NQ) additions rather than NQ of each in a row.
+template <int NQ>
+__device__ __forceinline__ void add_totals(uint32_t tot, float2& oa, float2& ob)
+{
+    constexpr int NB = NQ < 4 ? NQ : 4;          // at most four slots in flight (registers)
+    float2 a[NB], b[NB];
+#pragma unroll
+    for (int q = 0; q < NB; ++q) {
+        const float4 t4 = ldsf4(tot + 256 * q);
+        a[q] = make_float2(t4.x, t4.y); b[q] = make_float2(t4.z, t4.w);
+    }
+#pragma unroll
+    for (int n = NB; n > 1; n = (n + 1) / 2)
+#pragma unroll
+        for (int q = 0; q < n / 2; ++q) {
+            a[q] = add2(a[q], a[n - 1 - q]); b[q] = add2(b[q], b[n - 1 - q]);
+        }
+    oa = add2(oa, a[0]); ob = add2(ob, b[0]);
+    if constexpr (NQ > 4) add_totals<NQ - 4>(tot + 256 * 4, oa, ob);
 }
 
 // Token-by-token fp32 recurrence over `valid` tokens of one chunk for one state warp: the warp owns value
@@ -869,10 +882,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                     const uint64_t dr = smem_desc(tr), dv = smem_desc(tr + 2 * TILE);
                     const uint64_t ds = smem_desc(sbase + OFF_SB + tb * TILE), dp = smem_desc(sbase + OFF_PP + tb * TILE);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        tc_mma(tmem + TM_Y0 + 64 * tb, dr + (uint64_t)(2 * kk), ds + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
-                        tc_mma(tmem + TM_PV + 64 * tb, dp + (uint64_t)(2 * kk), dv + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
-                    }
+                    // one accumulator: Y = [R^ | P'] [S_0 ; V], the state part first (its operands are ready earlier)
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma(tmem + TM_Y + 64 * tb, dr + (uint64_t)(2 * kk), ds + (uint64_t)(128 * kk), IDESC_K_MN, kk > 0);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma(tmem + TM_Y + 64 * tb, dp + (uint64_t)(2 * kk), dv + (uint64_t)(128 * kk), IDESC_K_MN, 1);
                 }
                 tc_commit(bar(BAR_B_DONE + tb));
                 tc_commit(bar(BAR_EMPTY_RKV + s));
@@ -1163,12 +1178,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             // ---- this warp's 16 rows of y -> bf16 slab -> global
             {
-                const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_Y0 + 64 * tb;
-                const uint32_t tc = tmem + ((uint32_t)(32 * sp) << 16) + TM_PV + 64 * tb;
-                float ya[4][4], yb[4][4];
+                const uint32_t ta = tmem + ((uint32_t)(32 * sp) << 16) + TM_Y + 64 * tb;
+                float ya[4][4];
                 tmem_ld_16x32(ta, ya);
-                tmem_ld_16x32(tc, yb);
-                add_acc(ya, yb);
                 if (has_u2) {
                     if (!mbar_wait(bar(BAR_U2 + sp), u2_parity, abort_flag)) break;
                     u2_pending = false;
@@ -1176,11 +1188,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 }
                 store_half_bf16<0>(slab, 0, ya, lane);
                 tmem_ld_16x32(ta + 32, ya);
-                tmem_ld_16x32(tc + 32, yb);
                 tc_fence_before();
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_Y_EMPTY + tb), lane == 0);
-                add_acc(ya, yb);
                 if (has_u2) {
                     add_slab_bf16<1>(ya, u2slab, lane);
                     __syncwarp();
@@ -1295,9 +1305,16 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             __syncwarp();
             mbar_arrive_if(bar(BAR_ESYNC + eset), lane == 0);
             if (!mbar_wait(bar(BAR_ESYNC + eset), (c >> 1) & 1, abort_flag)) break;
-            for (int qq = 0; qq < tq; ++qq) {            // cumulative sum at the end of the warps before this one
-                const float4 t4 = ldsf4(totc + 256 * qq);
-                oa = add2(oa, make_float2(t4.x, t4.y)); ob = add2(ob, make_float2(t4.z, t4.w));
+            // cumulative sum at the end of the warps before this one: their totals, fetched together and added as a tree
+            switch (tq) {
+            case 1: add_totals<1>(totc, oa, ob); break;
+            case 2: add_totals<2>(totc, oa, ob); break;
+            case 3: add_totals<3>(totc, oa, ob); break;
+            case 4: add_totals<4>(totc, oa, ob); break;
+            case 5: add_totals<5>(totc, oa, ob); break;
+            case 6: add_totals<6>(totc, oa, ob); break;
+            case 7: add_totals<7>(totc, oa, ob); break;
+            default: break;
             }
             // ---- phase B, in place: r -> R^ = r 2^{a_{t-1}}, k -> K^ = k 2^{-a_t}; bonus partials
             uint2 rw[4], kw[4];
