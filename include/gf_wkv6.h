@@ -227,6 +227,18 @@ GF_API gf_status_t gf_wkv6_set_kernel(gf_kernel_t kernel);
  * undefined), GF_ERR_CUDA if the stream reports an error, else GF_OK.  Clears the flag. */
 GF_API gf_status_t gf_wkv6_last_device_status(gf_stream_t stream);
 
+/* Every device-side wait of the prefill kernels (on a copy, a tensor-core product, another warp) is bounded: when
+ * it runs out the kernel raises the status flag that gf_wkv6_last_device_status reports and all its warps leave.
+ * gf_wkv6_set_wait_limit sets the bound, in microseconds, for the launches of later calls of this process
+ * (0 restores the default of 2 s; a healthy launch waits microseconds at a time, so the bound only matters when
+ * something is wrong).
+ * gf_wkv6_selftest_wait_timeout shows the mechanism at work without disturbing anything: it enqueues a one-warp
+ * kernel that waits, with that same bounded wait, on a barrier nobody arrives on; after `microseconds` (1 .. 1 000 000)
+ * the wait gives up, the flag is raised and the kernel ends, so the next gf_wkv6_last_device_status returns
+ * GF_ERR_TIMEOUT once and GF_OK afterwards.  No other state of the library or the device is touched. */
+GF_API gf_status_t gf_wkv6_set_wait_limit(unsigned int microseconds);
+GF_API gf_status_t gf_wkv6_selftest_wait_timeout(unsigned int microseconds, gf_stream_t stream);
+
 /* Number of kernels this library has launched in this process (for benchmarks). */
 GF_API uint64_t gf_wkv6_launch_count(void);
 

@@ -17,7 +17,7 @@ from . import _build
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
     "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
-    "launch_count", "status_string", "version",
+    "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
 
@@ -50,6 +50,8 @@ _SIGNATURES = {
     "gf_gold_key_compress": (_i, [_vp, _vp, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
+    "gf_wkv6_set_wait_limit": (_i, [ctypes.c_uint]),
+    "gf_wkv6_selftest_wait_timeout": (_i, [ctypes.c_uint, _vp]),
     "gf_wkv6_launch_count": (ctypes.c_uint64, []),
     "gf_status_string": (ctypes.c_char_p, [_i]),
     "gf_wkv6_version": (_i, []),
@@ -167,6 +169,16 @@ def _ensure_workspace(B, T, H, N, device) -> None:
 def last_device_status(stream=None) -> None:
     """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
     _check(load_library().gf_wkv6_last_device_status(_stream(stream)), "gf_wkv6_last_device_status")
+
+
+def set_wait_limit(microseconds: int) -> None:
+    """gf_wkv6_set_wait_limit: bound of every device-side wait of later launches (0: the default of 2 s)."""
+    _check(load_library().gf_wkv6_set_wait_limit(int(microseconds)), "gf_wkv6_set_wait_limit")
+
+
+def selftest_wait_timeout(microseconds: int, stream=None) -> None:
+    """gf_wkv6_selftest_wait_timeout: enqueue the one-warp kernel whose bounded wait runs out after `microseconds`."""
+    _check(load_library().gf_wkv6_selftest_wait_timeout(int(microseconds), _stream(stream)), "gf_wkv6_selftest_wait_timeout")
 
 
 def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, want_state=True, split=True):

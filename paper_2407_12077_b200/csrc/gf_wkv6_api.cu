@@ -419,6 +419,20 @@ gf_status_t gf_wkv6_last_device_status(gf_stream_t stream)
     return flag ? GF_ERR_TIMEOUT : GF_OK;
 }
 
+gf_status_t gf_wkv6_set_wait_limit(unsigned int microseconds)
+{
+    gf::wait_limit_us().store(microseconds, std::memory_order_relaxed);
+    return GF_OK;
+}
+
+gf_status_t gf_wkv6_selftest_wait_timeout(unsigned int microseconds, gf_stream_t stream)
+{
+    if (microseconds == 0 || microseconds > 1000000u) return GF_ERR_INVALID_ARG;     // one second at most
+    gf::ck::wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(microseconds);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
 uint64_t gf_wkv6_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 gf_status_t gf_c2_layernorm(const void* y, const float* gamma, const float* beta, float eps, void* out,

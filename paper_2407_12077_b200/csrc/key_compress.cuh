@@ -88,6 +88,7 @@ key_compress_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
             mbar_init(bar(KC_ACC_EMPTY + i), 4);
         }
         sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, ck::WAIT_LIMIT_US);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }

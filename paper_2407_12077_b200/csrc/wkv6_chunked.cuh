@@ -88,7 +88,7 @@ constexpr int THREADS = 32 * (WARP_E0 + N_ESET * N_EW);
 constexpr float A2_MAX = 96.f;         // largest in-chunk |cumulative log2 decay| on the tensor-core path
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LOG2_LOG2E = 0.5287663729448977f;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+constexpr uint32_t WAIT_LIMIT_US = 2000000u;                   // default limit of a device-side wait: 2 s
 constexpr uint32_t TRY_WAIT_HINT_NS = 20000;                  // a waiting thread may be suspended this long per try
 
 // tensor memory: 64 fp32 columns per 64x64 accumulator, two buffers each
@@ -209,22 +209,24 @@ __device__ __forceinline__ unsigned long long globaltimer()
     return t;
 }
 // Bounded wait.  Returns false if the CTA is aborting or the wait ran out of time (the
-// status flag is then raised and the CTA-wide abort flag set so every role leaves).
+// status flag is then raised and the CTA-wide abort flag set so every role leaves).  The limit, in
+// microseconds, is the 32-bit word that follows the abort word in shared memory.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t abort_flag, bool poll_abort)
 {
     const unsigned long long t0 = globaltimer();
+    const unsigned long long limit_ns = 1000ull * lds32(abort_flag + 4);
     for (;;) {
         for (int it = 0; it < 64; ++it)
             if (mbar_try_wait(bar, parity)) return true;
         if (poll_abort && lds32(abort_flag)) return false;
-        if (globaltimer() - t0 > WAIT_LIMIT_NS) break;
+        if (globaltimer() - t0 > limit_ns) break;
         __nanosleep(64);
     }
     sts32(abort_flag, 1u);
     atomicExch(&g_dev_status, 1);
     return false;
 }
-// abort_flag: shared-memory address of the CTA-wide abort word
+// abort_flag: shared-memory address of the CTA-wide abort word (followed by the wait limit)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag, bool poll_abort = true)
 {
     if (mbar_try_wait(bar, parity)) return true;
@@ -474,6 +476,7 @@ struct Params {
     // the scratch) and every CTA of the main launch takes its start state from the copy, so that nothing
     // reads state_in once the first state_out has been written (state_out may be state_in).  NULL: no copy.
     float* state_copy;
+    uint32_t wait_limit_us;                // limit of every device-side wait of the launch (0: the default, 2 s)
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -710,6 +713,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         mbar_init(bar(BAR_FB_DONE), N_GW);
         for (int i = 0; i < N_GW; ++i) mbar_init(bar(BAR_U2 + i), 1);
         sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, p.wait_limit_us ? p.wait_limit_us : WAIT_LIMIT_US);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -1225,7 +1229,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     } else {
         // ============================== elementwise warps ==============================
         const int eset = (warp - WARP_E0) / N_EW;        // this set takes chunks eset, eset + 2, ...
-        const int tq = (warp - WARP_E0) % N_EW;          // tokens 8*tq .. 8*tq+7 of the chunk
+        // tokens 8*tq .. 8*tq+7 of the chunk; the warp with the last tokens, which closes the chunk on top of its share,
+        // is the set's first one and so sits on the scheduler (warp index mod 4) that holds no control warp
+        const int tq = ((warp - WARP_E0) % N_EW + N_EW - 1) % N_EW;
         const int cq = lane & 15, th = lane >> 4;        // channels 4*cq .. 4*cq+3, tokens 8*tq + 4*th + (0..3)
         const int etid = tid - 32 * (WARP_E0 + eset * N_EW);   // 0..255 inside the set
         constexpr bool c2 = C2;                          // Finch-C2 form: keys times (1 - w), no bonus
@@ -1400,6 +1406,23 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     }
 }
 
+// One warp that waits, with the kernel's own bounded wait, on a barrier nobody arrives on: the wait runs out after
+// limit_us microseconds, raises the status flag and the kernel returns.  (Exercises the time-out path of the waits
+// above without disturbing anything: see gf_wkv6_selftest_wait_timeout.)
+__global__ void __launch_bounds__(32) wait_timeout_selftest_kernel(uint32_t limit_us)
+{
+    __shared__ __align__(8) unsigned long long words[2];       // {abort word, limit}, mbarrier
+    const uint32_t abort_flag = smem_u32(&words[0]), bar = smem_u32(&words[1]);
+    if (threadIdx.x == 0) {
+        sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, limit_us);
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    mbar_wait_warp(bar, 0, abort_flag);
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1517,6 +1540,13 @@ inline size_t persistent_scratch_bytes(int n_seq)
 // Packed: cu = device cu_seqlens, n_seq = S, T = max_seqlen.  total_rows = rows of the [rows][H*64] tensors.
 // scratch / scratch_bytes: optional device memory for the sequence split (see choose_split); without
 // enough of it the call runs unsplit.
+// limit of the device-side waits of the launches below, in microseconds (0: default); set by gf_wkv6_set_wait_limit
+inline std::atomic<uint32_t>& wait_limit_us()
+{
+    static std::atomic<uint32_t> v{0};
+    return v;
+}
+
 inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                    const __nv_bfloat16* x, const float* u, const float* state_in, float* state_out,
                                    __nv_bfloat16* y, const int32_t* cu, int n_seq, int T, long long total_rows, int H,
@@ -1543,6 +1573,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     }
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
     if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
+    p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     const int n_sm = sm_count();
     // More units than SMs: one CTA per SM walks a stream of units, so that a unit's pipeline fill overlaps the
     // drain of the one before it.  That saves about 4.5 us per unit and costs about 3 % more instructions per
@@ -1597,6 +1628,7 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
     // two nominal segments of which the first covers the whole sequence: the summary launch handles
     // every segment but the last
     ck::Params p{nullptr, k, v, x, nullptr, nullptr, nullptr, nullptr, nullptr, T, H, summary, (T + ck::L - 1) / ck::L, 2, nullptr, c2};
+    p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     launches->fetch_add(1, std::memory_order_relaxed);

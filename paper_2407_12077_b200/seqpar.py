@@ -46,7 +46,13 @@ def prefill_sequence_parallel(r, k, v, x, u, state_in=None, group=None, ops=None
     if world == 1:
         return ops.prefill(r, k, v, x, u, state_in)
     mine = ops.summary(k, v, x).contiguous()                         # [B, H, 64 + 4096]
-    gathered = torch.empty((world,) + tuple(mine.shape), dtype=mine.dtype, device=mine.device)
-    dist.all_gather(list(gathered.unbind(0)), mine, group=group)      # the one exchange step
+    if mine.is_cuda and dist.get_backend(group) != "nccl":
+        # a backend that gathers host memory only (gloo): stage the summaries through the host
+        host = torch.empty((world,) + tuple(mine.shape), dtype=mine.dtype)
+        dist.all_gather(list(host.unbind(0)), mine.cpu(), group=group)
+        gathered = host.to(mine.device)
+    else:
+        gathered = torch.empty((world,) + tuple(mine.shape), dtype=mine.dtype, device=mine.device)
+        dist.all_gather(list(gathered.unbind(0)), mine, group=group)  # the one exchange step
     start = state_in if rank == 0 else ops.fold(state_in, gathered, rank)
     return ops.prefill(r, k, v, x, u, start)

@@ -110,3 +110,53 @@ def test_device_steps_with_ranks_played_in_turn(c2):
     # the fold of all four summaries over the initial state is the final state as well
     s_all = gf.fold_summaries(d.state_in, gathered, P)
     assert orc.rel_l2(s_all.cpu().numpy(), s_ref) <= 5e-3
+
+
+def _device_worker(rank, world, port, out_dir, c2):
+    """One rank of the real thing: the library's kernels around a collective of a process group.  Both ranks use
+    cuda:0 (they meet on the host, in the gather, never inside a kernel); gloo carries the summaries."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import paper_2407_12077_b200 as gf
+    from paper_2407_12077_b200 import seqpar
+    dev = "cuda:0"
+    inp, u2, cut = _device_case()
+    sl = slice(cut[rank], cut[rank + 1])
+    mv = lambda t: t[:, sl].contiguous().to(dev)
+    u_arg = mv(u2) if c2 else inp.u.to(dev)
+    y, s = seqpar.prefill_sequence_parallel(mv(inp.r), mv(inp.k), mv(inp.v), mv(inp.x), u_arg, inp.state_in.to(dev),
+                                            ops=seqpar.DeviceOps(c2=c2))
+    gf.last_device_status()
+    torch.save({"y": y.cpu(), "s": s.cpu(), "launches": gf.launch_count()}, os.path.join(out_dir, f"d{rank}.pt"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def _device_case():
+    # slow decays (w about 0.998 .. 0.99995): the state a rank inherits still weighs on its last token
+    inp = synth.make_dense(2, 2300, 3, 64, "bf16", seed=90, state_std=0.5, x_lo=-10.0, x_hi=-6.0)
+    u2 = torch.randn(inp.r.shape, generator=torch.Generator().manual_seed(91)).bfloat16()
+    return inp, u2, [0, 1237, 2300]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("c2", [False, True])
+def test_two_ranks_with_the_device_steps_under_a_process_group(tmp_path, c2):
+    """prefill_sequence_parallel with DeviceOps end to end: summary kernel -> all_gather -> fold kernel -> prefill,
+    two processes, against the unsplit oracle."""
+    mp.spawn(_device_worker, args=(2, _free_port(), str(tmp_path), c2), nprocs=2, join=True)
+    inp, u2, cut = _device_case()
+    if c2:
+        y_ref, s_ref = orc.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in)
+    else:
+        y_ref, s_ref = orc.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+    out = [torch.load(tmp_path / f"d{r}.pt") for r in range(2)]
+    assert out[0]["launches"] >= 2 and out[1]["launches"] >= 3      # rank 1: summary, fold, prefill
+    y = torch.cat([o["y"] for o in out], 1).float().numpy()
+    assert orc.rel_l2(y, y_ref) <= 5e-3
+    assert orc.rel_l2(y[:, cut[1]:], y_ref[:, cut[1]:]) <= 5e-3      # the second rank's piece on its own
+    assert orc.rel_l2(out[1]["s"].numpy(), s_ref) <= 5e-3
+    # the hand-over matters here: without the first piece the second rank's answer is far off
+    wrong, _ = (orc.prefill_c2 if c2 else orc.prefill)(inp.r[:, cut[1]:], inp.k[:, cut[1]:], inp.v[:, cut[1]:], inp.x[:, cut[1]:],
+                                                        (u2[:, cut[1]:] if c2 else inp.u), None)
+    assert orc.rel_l2(wrong, y_ref[:, cut[1]:]) > 0.05
