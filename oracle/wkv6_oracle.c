@@ -29,6 +29,12 @@
  * form at the end of this file (k (1 - w) keys, second-value vector, no bonus) is pinned in
  * tests/test_oracle_pins_c2.py: brute-force expansion, reduction to the bonus-free recurrence on
  * premultiplied keys, w == 1 / w == 0 special cases, constant w = 1/2 closed form, split-and-carry.
+ * Further down: the LayerNorm across all heads (tests/test_oracle_pins_ln.py), the GOLD key compression
+ * (tests/test_oracle_pins_kc.py), the decay logit d_t = lora_omega(ddlerp_d(x_t, x_{t-1})) of the Finch-C2 block
+ * (tests/test_oracle_pins_dl.py: operator end points, an invertible outer lora that exposes the inner ddlerp, scalar
+ * loops, library routines, a hand value, token-shift laws) and the gradient of the recurrence
+ * (tests/test_oracle_pins_bwd.py: central differences of the forward pass, the one-token closed form, linearity,
+ * split-and-carry of the adjoint).  No function here is unpinned.
  *
  * Inputs arrive as float (an exact carrier for both fp32 and bf16 data) and are
  * widened to double before any arithmetic; every sum runs in double in plain
@@ -228,5 +234,160 @@ void gold_oracle_key_compress(const double *x, const double *w, double *c, long 
             double acc = 0.0;
             for (long k = 0; k < D; ++k) acc += x[(size_t)t * D + k] * w[(size_t)k * Dc + n];
             c[(size_t)t * Dc + n] = acc;
+        }
+}
+
+/*
+ * The decay logit of the Finch-C2 block, d_t = lora_omega( ddlerp_d( x_t, x_{t-1} ) ), with the three
+ * operators the Finch-C2 section defines (all vectors have the D channels of the model dimension, the two
+ * low-rank matrices of a lora are A [D][R] and B [R][D], row-major):
+ *     lerp(a, b, t)   = a + (b - a) .* t
+ *     lora(x)         = lambda + tanh(x A) B
+ *     ddlerp(a, b)    = a + (b - a) .* lora( a + (b - a) .* mu_x )
+ * Each operator is one function below, written as the formula reads, and the logit is their composition:
+ * lora_d (rank Rd: A_d, B_d, lambda_d) inside ddlerp_d, lora_omega (rank Rw) outside.  x_{t-1} of a sequence's
+ * first token is the row x_prev[b] (the token before the call; NULL: zeros).
+ * x: [B][T][D] double, x_prev: [B][D] or NULL, d: [B][T][D] double.  Pinned in tests/test_oracle_pins_dl.py.
+ */
+static void op_lerp(const double *a, const double *b, const double *t, double *out, long D)
+{
+    for (long c = 0; c < D; ++c) out[c] = a[c] + (b[c] - a[c]) * t[c];
+}
+
+static void op_lora(const double *x, const double *A, const double *Bm, const double *lambda, long D, long R,
+                    double *out)
+{
+    double *h = (double *)malloc((size_t)(R > 0 ? R : 1) * sizeof(double));
+    for (long q = 0; q < R; ++q) {
+        double acc = 0.0;
+        for (long c = 0; c < D; ++c) acc += x[c] * A[c * R + q];          /* (x A)[q] */
+        h[q] = tanh(acc);
+    }
+    for (long c = 0; c < D; ++c) {
+        double acc = 0.0;
+        for (long q = 0; q < R; ++q) acc += h[q] * Bm[q * D + c];         /* (tanh(x A) B)[c] */
+        out[c] = lambda[c] + acc;
+    }
+    free(h);
+}
+
+static void op_ddlerp(const double *a, const double *b, const double *mu_x, const double *A, const double *Bm,
+                      const double *lambda, long D, long R, double *out)
+{
+    double *inner = (double *)malloc((size_t)D * sizeof(double));
+    double *mix = (double *)malloc((size_t)D * sizeof(double));
+    op_lerp(a, b, mu_x, inner, D);                 /* a + (b - a) .* mu_x */
+    op_lora(inner, A, Bm, lambda, D, R, mix);      /* lora( . ) */
+    op_lerp(a, b, mix, out, D);                    /* a + (b - a) .* lora( . ) */
+    free(inner);
+    free(mix);
+}
+
+void c2_oracle_decay_logit(const double *x, const double *x_prev, const double *mu_x, const double *A_d,
+                           const double *B_d, const double *lambda_d, long Rd, const double *A_w,
+                           const double *B_w, const double *lambda_w, long Rw, double *d, long B, long T, long D)
+{
+#pragma omp parallel for collapse(2) schedule(static)
+    for (long b = 0; b < B; ++b)
+        for (long t = 0; t < T; ++t) {
+            double *shifted = (double *)malloc((size_t)D * sizeof(double));
+            double *mixed = (double *)malloc((size_t)D * sizeof(double));
+            const double *xt = x + ((size_t)b * T + t) * D;
+            for (long c = 0; c < D; ++c)                                   /* x_{t-1} */
+                shifted[c] = t > 0 ? xt[c - D] : (x_prev ? x_prev[(size_t)b * D + c] : 0.0);
+            op_ddlerp(xt, shifted, mu_x, A_d, B_d, lambda_d, D, Rd, mixed);
+            op_lora(mixed, A_w, B_w, lambda_w, D, Rw, d + ((size_t)b * T + t) * D);
+            free(shifted);
+            free(mixed);
+        }
+}
+
+/*
+ * Gradient of the recurrence at the top of this file (training runs it backwards; the paper trains its models
+ * with it and fine-tunes with the recurrent part frozen).  For a scalar loss L with dy_t = dL/dy_t and
+ * dS_T = dL/dS_T given, the adjoint G_t = dL/dS_t of the state is carried from t = T down to 1 through the two
+ * places S_{t-1} enters (the output y_t and the update to S_t):
+ *     G_{t-1}[i][j] = w_t[i] G_t[i][j] + r_t[i] dy_t[j]
+ * and every input's gradient is read off the forward formulas
+ *     y_t[j]    = sum_i r_t[i] ( S_{t-1}[i][j] + u[i] k_t[i] v_t[j] ),   S_t[i][j] = w_t[i] S_{t-1}[i][j] + k_t[i] v_t[j]:
+ *     dr_t[i]  = sum_j dy_t[j] ( S_{t-1}[i][j] + u[i] k_t[i] v_t[j] )
+ *     dk_t[i]  = r_t[i] u[i] sum_j dy_t[j] v_t[j]  +  sum_j G_t[i][j] v_t[j]
+ *     dv_t[j]  = ( sum_i r_t[i] u[i] k_t[i] ) dy_t[j]  +  sum_i G_t[i][j] k_t[i]
+ *     du[i]   += r_t[i] k_t[i] sum_j dy_t[j] v_t[j]                       (summed over t and over the batch)
+ *     dw_t[i]  = sum_j G_t[i][j] S_{t-1}[i][j],     dx_t[i] = dw_t[i] * ( - w_t[i] exp(x_t[i]) )     (w = exp(-exp(x)))
+ *     dS_0     = G_0.
+ * The forward states S_0 .. S_{T-1} are recomputed first and kept (T N^2 doubles per unit): slow and plain.
+ * Pinned in tests/test_oracle_pins_bwd.py by central finite differences of the forward oracle.
+ * Layouts as in the forward pass; du is [B][H][N] per batch entry (the caller sums over b), all outputs double.
+ */
+static void unit_backward(const float *r, const float *k, const float *v, const float *x, const float *u,
+                          const float *s_in, const double *dy, const double *ds_T, double *dr, double *dk,
+                          double *dv, double *dx, double *du, double *ds_0, long T, long N, long row_stride)
+{
+    const size_t NN = (size_t)N * N;
+    double *S_all = (double *)malloc((size_t)(T > 0 ? T : 1) * NN * sizeof(double));   /* S_{t-1} for t = 1..T */
+    double *S = (double *)malloc(NN * sizeof(double));
+    double *G = (double *)malloc(NN * sizeof(double));
+    for (size_t i = 0; i < NN; ++i) S[i] = s_in ? (double)s_in[i] : 0.0;
+    for (long t = 0; t < T; ++t) {
+        memcpy(S_all + (size_t)t * NN, S, NN * sizeof(double));
+        for (long i = 0; i < N; ++i) {
+            const double w = exp(-exp((double)x[t * row_stride + i]));
+            for (long j = 0; j < N; ++j)
+                S[i * N + j] = w * S[i * N + j] + (double)k[t * row_stride + i] * (double)v[t * row_stride + j];
+        }
+    }
+    for (size_t i = 0; i < NN; ++i) G[i] = ds_T ? ds_T[i] : 0.0;
+    for (long i = 0; i < N; ++i) du[i] = 0.0;
+    for (long t = T - 1; t >= 0; --t) {
+        const float *rt = r + t * row_stride, *kt = k + t * row_stride, *vt = v + t * row_stride, *xt = x + t * row_stride;
+        const double *dyt = dy + t * row_stride, *Sp = S_all + (size_t)t * NN;
+        double dyv = 0.0, ruk = 0.0;
+        for (long j = 0; j < N; ++j) dyv += dyt[j] * (double)vt[j];
+        for (long i = 0; i < N; ++i) ruk += (double)rt[i] * (double)u[i] * (double)kt[i];
+        for (long i = 0; i < N; ++i) {
+            double a_r = 0.0, a_k = 0.0, a_w = 0.0;
+            for (long j = 0; j < N; ++j) {
+                a_r += dyt[j] * (Sp[i * N + j] + (double)u[i] * (double)kt[i] * (double)vt[j]);
+                a_k += G[i * N + j] * (double)vt[j];
+                a_w += G[i * N + j] * Sp[i * N + j];
+            }
+            const double w = exp(-exp((double)xt[i]));
+            dr[t * row_stride + i] = a_r;
+            dk[t * row_stride + i] = (double)rt[i] * (double)u[i] * dyv + a_k;
+            dx[t * row_stride + i] = a_w * (-w * exp((double)xt[i]));
+            du[i] += (double)rt[i] * (double)kt[i] * dyv;
+        }
+        for (long j = 0; j < N; ++j) {
+            double a_v = 0.0;
+            for (long i = 0; i < N; ++i) a_v += G[i * N + j] * (double)kt[i];
+            dv[t * row_stride + j] = ruk * dyt[j] + a_v;
+        }
+        for (long i = 0; i < N; ++i) {
+            const double w = exp(-exp((double)xt[i]));
+            for (long j = 0; j < N; ++j) G[i * N + j] = w * G[i * N + j] + (double)rt[i] * dyt[j];
+        }
+    }
+    if (ds_0) memcpy(ds_0, G, NN * sizeof(double));
+    free(S_all);
+    free(S);
+    free(G);
+}
+
+/* Dense batch: r,k,v,x [B][T][H][N] float carriers, dy [B][T][H][N] double, ds_T [B][H][N][N] double or NULL
+ * (zero); outputs dr,dk,dv,dx [B][T][H][N], du_b [B][H][N] (per batch entry), ds_0 [B][H][N][N] or NULL. */
+void wkv6_oracle_backward(const float *r, const float *k, const float *v, const float *x, const float *u,
+                          const float *state_in, const double *dy, const double *ds_T, double *dr, double *dk,
+                          double *dv, double *dx, double *du_b, double *ds_0, long B, long T, long H, long N)
+{
+    const long C = H * N;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (long b = 0; b < B; ++b)
+        for (long h = 0; h < H; ++h) {
+            const size_t off = (size_t)b * T * C + (size_t)h * N;
+            const size_t soff = ((size_t)b * H + h) * N * N;
+            unit_backward(r + off, k + off, v + off, x + off, u + h * N, state_in ? state_in + soff : NULL,
+                          dy + off, ds_T ? ds_T + soff : NULL, dr + off, dk + off, dv + off, dx + off,
+                          du_b + ((size_t)b * H + h) * N, ds_0 ? ds_0 + soff : NULL, T, N, C);
         }
 }

@@ -40,6 +40,8 @@ def _load():
         _lib.wkv6_oracle_prefill_c2.restype = None
         _lib.c2_oracle_layernorm.restype = None
         _lib.gold_oracle_key_compress.restype = None
+        _lib.c2_oracle_decay_logit.restype = None
+        _lib.wkv6_oracle_backward.restype = None
     return _lib
 
 
@@ -185,6 +187,59 @@ def key_compress(x, w_kd):
     d = ctypes.c_double
     lib.gold_oracle_key_compress(_p(x, d), _p(w, d), _p(c, d), ctypes.c_long(rows), ctypes.c_long(D), ctypes.c_long(Dc))
     return c
+
+
+def _f64(a, shape=None):
+    """Exact float64 numpy copy of a numpy array / torch tensor of any float type."""
+    if a is None:
+        return None
+    if hasattr(a, "detach"):
+        a = a.detach().cpu().double().numpy()
+    a = np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+    if shape is not None:
+        assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def decay_logit(x, mu_x, A_d, B_d, lambda_d, A_w, B_w, lambda_w, x_prev=None):
+    """The decay logit of the Finch-C2 block, d_t = lora_omega(ddlerp_d(x_t, x_{t-1})) (lerp / lora / ddlerp as the
+    Finch-C2 section defines them).  x: [B,T,D]; mu_x, lambda_d, lambda_w: [D]; A_d: [D,Rd], B_d: [Rd,D] (the lora
+    inside ddlerp_d); A_w: [D,Rw], B_w: [Rw,D] (lora_omega); x_prev: [B,D], the token before each sequence's first
+    (None: zeros).  Any float type, widened exactly to float64.  Returns d float64 [B,T,D]."""
+    lib = _load()
+    x = _f64(x)
+    B, T, D = x.shape
+    A_d, A_w = _f64(A_d), _f64(A_w)
+    Rd, Rw = A_d.shape[1], A_w.shape[1]
+    assert A_d.shape == (D, Rd) and A_w.shape == (D, Rw)
+    B_d, B_w = _f64(B_d, (Rd, D)), _f64(B_w, (Rw, D))
+    mu_x, lambda_d, lambda_w = _f64(mu_x, (D,)), _f64(lambda_d, (D,)), _f64(lambda_w, (D,))
+    x_prev = _f64(x_prev, (B, D)) if x_prev is not None else None
+    d = np.zeros((B, T, D), dtype=np.float64)
+    c = ctypes.c_double
+    lib.c2_oracle_decay_logit(_p(x, c), _p(x_prev, c), _p(mu_x, c), _p(A_d, c), _p(B_d, c), _p(lambda_d, c),
+                              ctypes.c_long(Rd), _p(A_w, c), _p(B_w, c), _p(lambda_w, c), ctypes.c_long(Rw),
+                              _p(d, c), ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(D))
+    return d
+
+
+def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None):
+    """Gradient of prefill(): given dy = dL/dy [B,T,H,N] and dstate_out = dL/dS_T [B,H,N,N] (None: zero), returns
+    (dr, dk, dv, dx [B,T,H,N], du [H,N] summed over the batch, dstate_in [B,H,N,N]) in float64.  r,k,v,x,u,state_in
+    as for prefill() (float32 / bfloat16 carriers)."""
+    lib = _load()
+    r, k, v, x, u, state_in = _f32(r), _f32(k), _f32(v), _f32(x), _f32(u), _f32(state_in)
+    B, T, H, N = r.shape
+    dy = _f64(dy, (B, T, H, N))
+    dsT = _f64(dstate_out, (B, H, N, N)) if dstate_out is not None else None
+    outs = [np.zeros((B, T, H, N), dtype=np.float64) for _ in range(4)]
+    du_b = np.zeros((B, H, N), dtype=np.float64)
+    ds0 = np.zeros((B, H, N, N), dtype=np.float64)
+    f, c = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_backward(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(u, f), _p(state_in, f), _p(dy, c), _p(dsT, c),
+                             _p(outs[0], c), _p(outs[1], c), _p(outs[2], c), _p(outs[3], c), _p(du_b, c), _p(ds0, c),
+                             ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(H), ctypes.c_long(N))
+    return outs[0], outs[1], outs[2], outs[3], du_b.sum(axis=0), ds0
 
 
 def rel_l2(a, b) -> float:
