@@ -31,9 +31,13 @@ WORKLOAD = dict(B=4, T=16384, H=32, N=64, calls=16)
 BYTES_PER_TOKEN_HEAD = 640            # bf16 r,k,v,x in (4*64*2) + bf16 y out (64*2)
 STATE_BYTES_PER_UNIT = 64 * 64 * 4    # fp32 final state written once per (b,h) (state_in is NULL)
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (null once the kernel has changed since the counters were taken)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 1275564032  # 4 x (268.53 + 50.36 MB) measured at T=4096, scaled by tokens
+FALLBACK_BF16_TFLOPS = 1590.0
+# DRAM traffic per launch of the dominant kernel, from the ncu capture summarised under profiles/ (taken on a
+# B=4 T=4096 H=32 launch; None once the kernel has changed since the counters were taken).  The reads grow in
+# proportion to the tokens and are scaled to the timed launch; the writes of the capture miss the part of y
+# that is still in L2 when the kernel ends (a fixed amount), so for the timed launch they are only bounded:
+# at least the scaled figure, at most the algorithmic y + state bytes.
+NCU_CAPTURE = None
 
 
 def parse():
@@ -46,17 +50,31 @@ def parse():
     ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help=argparse.SUPPRESS)
     ap.add_argument("--no-e2e", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--no-cpu-baseline", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--no-extras", action="store_true", help=argparse.SUPPRESS)
     return ap.parse_args()
 
 
 def measured_peaks():
+    """(HBM GB/s, bf16 TFLOP/s burst, which) from MEASURED_PEAKS.json, else the fallback figures."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         try:
-            return float(json.load(open(p))["hbm_gbs"]), "measured"
+            j = json.load(open(p))
+            return float(j["hbm_gbs"]), float(j.get("bf16_tflops", FALLBACK_BF16_TFLOPS)), "measured"
         except Exception:
             pass
-    return FALLBACK_HBM_GBS, "fallback"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def traffic_of_launch(tokens_heads: int, alg_write_bytes: int):
+    """DRAM traffic of one timed launch from the ncu capture (see NCU_CAPTURE), or None."""
+    if not NCU_CAPTURE:
+        return None
+    scale = tokens_heads / NCU_CAPTURE["token_heads"]
+    return {"read": int(NCU_CAPTURE["read_bytes"] * scale),
+            "write_at_least": int(NCU_CAPTURE["write_bytes"] * scale), "write_at_most": int(alg_write_bytes),
+            "note": "reads scaled by tokens from the capture in " + NCU_CAPTURE["profile"] +
+                    "; writes: the capture misses the y rows still in L2 at kernel end"}
 
 
 class ClockSampler:
@@ -275,14 +293,20 @@ def main():
 
     # ---- roofline of the dominant kernel (one prefill launch) from the live per-launch events
     per_launch = [a.elapsed_time(b) for a, b in kernel_events]
-    launch_ms = statistics.mean(per_launch)
+    launch_ms, launch_med = statistics.mean(per_launch), statistics.median(per_launch)
     alg_bytes = B * T * H * BYTES_PER_TOKEN_HEAD + B * H * STATE_BYTES_PER_UNIT
-    peak, peak_kind = measured_peaks()
-    achieved = alg_bytes / (launch_ms * 1e-3) / 1e9
+    peak, peak_tf, peak_kind = measured_peaks()
+    gbs = lambda ms: alg_bytes / (ms * 1e-3) / 1e9
+    achieved = gbs(launch_ms)
+    # frac: from the mean of the per-launch events; frac_median: from their median; frac_step: from the step
+    # time the headline value is made of (launch gaps included): the three differ when the clock drifts
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
-                "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms, "launch_ms_median": statistics.median(per_launch),
-                "launch_ms_min": min(per_launch), "launch_ms_max": max(per_launch), "algorithmic_bytes": alg_bytes}
+                "frac_median": gbs(launch_med) / peak, "frac_step": gbs(ms_per_step / calls) / peak,
+                "frac_best": gbs(min(per_launch)) / peak,
+                "traffic": traffic_of_launch(B * T * H, B * T * H * N * 2 + B * H * STATE_BYTES_PER_UNIT),
+                "peak_kind": f"of {peak_kind}", "kernel": "gf_wkv6_prefill (one launch)", "launch_ms": launch_ms,
+                "launch_ms_median": launch_med, "launch_ms_min": min(per_launch), "launch_ms_max": max(per_launch),
+                "algorithmic_bytes": alg_bytes, "launches_timed": len(per_launch)}
 
     # ---- the step that follows the WKV output in the o_t equation (LayerNorm across all heads), timed on its own
     # over the y of every call, outside the step and its numbers: reported beside them, not in them
@@ -333,6 +357,37 @@ def main():
                   "achieved": v_bytes / (v_ms * 1e-3) / 1e9, "peak": peak, "frac": v_bytes / (v_ms * 1e-3) / 1e9 / peak,
                   "algorithmic_bytes": v_bytes}
         del vin, v_y, v_s
+
+    # ---- the other rows of the path, each timed on its own after the step (a few launches each, seeded inputs
+    # of its configuration resident in HBM): not part of the headline value, reported beside it
+    others = None
+    if world == 1 and not args.no_extras:
+        from paper_2407_12077_b200 import cases
+        others = {}
+        for key, case, what in (
+                ("cfg1", "cfg1", "gf_wkv6_prefill, small-model shape B=8 T=4096 H=12 (96 units: one CTA each)"),
+                ("cfg3_one_call", "cfg3", "gf_wkv6_prefill, B=1 T=131072 H=32 in one call (sequence split: 2 launches)"),
+                ("cfg3_eight_segments", "cfg3-segments", "8 x gf_wkv6_prefill of 16384 tokens, state carried in place"),
+                ("prefill_c2", "cfg2-c2", "gf_wkv6_prefill_c2 with the second-value tensor, cfg2 shape (768 B per token*head)"),
+                ("key_compress", "kc-cfg2", "gf_gold_key_compress 65536 x 2048 -> 128"),
+                ("decode_step", "cfg4-decode", "gf_wkv6_step, 64 sequences x 32 heads, 64 steps per graph replay (states stay in L2)"),
+                ("decode_step_layer_stack", "cfg4-decode-layers", "gf_wkv6_step over 12 layers with their own states (streams from HBM)")):
+            r = cases.run(case, 5, 1.0)
+            ms = r["ms"]
+            o = {"kernel": what, "call_ms": ms, "algorithmic_bytes": r["bytes"], "bound": "hbm",
+                 "achieved": r["bytes"] / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                 "value": r["units"] / (ms * 1e-3), "value_unit": "token*heads/s" if "decode" not in key and key != "key_compress" else ("tokens/s" if key == "key_compress" else "step*heads/s")}
+            o["frac"] = o["achieved"] / peak
+            if key == "key_compress":
+                # at the crossing of the two rooflines: the bound is the slower of bytes at HBM rate and flops at tensor rate
+                flops = 2.0 * 65536 * 2048 * 128
+                t_hbm, t_tc = r["bytes"] / (peak * 1e9), flops / (peak_tf * 1e12)
+                o.update(tflops=r["tflops"], peak_tflops=peak_tf, bound="hbm" if t_hbm >= t_tc else "tensor",
+                         frac=max(t_hbm, t_tc) / (ms * 1e-3))
+            if "ms_pre_marshalled_calls_no_graph" in r:
+                o["call_ms_pre_marshalled_no_graph"] = r["ms_pre_marshalled_calls_no_graph"]
+            others[key] = o
+            torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry point: pinned host inputs -> y on the host
     e2e = None
@@ -399,7 +454,8 @@ def main():
                        "precision": "bf16 r/k/v/x/y and tensor-core operands, fp32 accumulation, decay sums and state",
                        "l2": "inputs larger than L2 (1.34 GB per call, distinct buffers per call)",
                        "parallelism": f"(b,h) units replicated per GPU x{world}, no collective"},
-            "roofline": roofline, "layernorm_heads": layernorm, "packed_prefill": packed, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "layernorm_heads": layernorm, "packed_prefill": packed, "other_rows": others,
+            "cpu_baseline": cpu_baseline,
             "e2e": e2e,
             "gpu_launches": launches,
             "clocks": clocks,

@@ -109,6 +109,30 @@ GF_API gf_status_t gf_wkv6_prefill_f32(const float *r, const float *k, const flo
                                 const float *u, const float *state_in, float *state_out, float *y,
                                 int B, int T, int H, int N, gf_stream_t stream);
 
+/* Gradient of gf_wkv6_prefill_f32 (training; the paper trains its models with this recurrence and fine-tunes
+ * long contexts through it): the adjoint of the wkv_t sum and of the output r_t . wkv_t (Finch-C2 wkv_t / o_t
+ * equations) with the bonus term of the recurrence at the top of this file.  Given dy = dL/dy [B][T][H][N] and
+ * dstate_out = dL/dS_T [B][H][N][N] (NULL: zero), with G_t = dL/dS_t carried from t = T down,
+ *     G_{t-1}[i][j] = w_t[i] G_t[i][j] + r_t[i] dy_t[j],
+ * it writes
+ *     dr_t[i] = sum_j dy_t[j] ( S_{t-1}[i][j] + u[i] k_t[i] v_t[j] )
+ *     dk_t[i] = sum_j G_t[i][j] v_t[j] + r_t[i] u[i] (v_t . dy_t)
+ *     dv_t[j] = sum_i G_t[i][j] k_t[i] + ( sum_i r_t[i] u[i] k_t[i] ) dy_t[j]
+ *     dx_t[i] = ( sum_j G_t[i][j] S_{t-1}[i][j] ) * ( -w_t[i] exp(x_t[i]) )        (gradient w.r.t. the decay logit)
+ *     du[i]   = sum over b and t of r_t[i] k_t[i] (v_t . dy_t)                     ([H][N], summed over the batch)
+ *     dstate_in = G_0                                                              ([B][H][N][N]; NULL: not written)
+ * All tensors fp32, layouts as in the forward call; r,k,v,x,u,state_in are the forward call's inputs (state_in
+ * NULL: zero).  dr,dk,dv,dx must not alias r,k,v,x,dy.  Token by token on the ALUs; the states the gradients need are
+ * recomputed from checkpoints kept every 64 tokens in `workspace`, a caller-owned DEVICE buffer of at least
+ * gf_wkv6_backward_workspace_bytes(B,T,H,N) bytes, 16-byte aligned (GF_ERR_WORKSPACE if absent or too small).
+ * Enqueues two kernels on `stream`, allocates nothing, does not synchronise; deterministic (no atomics). */
+GF_API gf_status_t gf_wkv6_backward_f32(const float *r, const float *k, const float *v, const float *x,
+                                 const float *u, const float *state_in, const float *dy,
+                                 const float *dstate_out, float *dr, float *dk, float *dv, float *dx,
+                                 float *du, float *dstate_in, int B, int T, int H, int N,
+                                 void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
+
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a

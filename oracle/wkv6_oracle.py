@@ -11,6 +11,7 @@ inside the C code, so the oracle sees precisely the values the GPU sees.
 from __future__ import annotations
 
 import ctypes
+import hashlib
 import os
 import subprocess
 
@@ -18,14 +19,33 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "wkv6_oracle.c")
-_LIB = os.path.join(_HERE, "libwkv6_oracle.so")
 _lib = None
 
 
+def _host_tag() -> str:
+    """The library is compiled for the host it runs on (-march=native), so its file name carries a tag of the
+    host's instruction-set flags: a copy built on another kind of machine is not picked up."""
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags") or line.startswith("Features"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.md5(flags.encode()).hexdigest()[:8]
+
+
+_LIB = os.path.join(_HERE, f"libwkv6_oracle_{_host_tag()}.so")
+
+
 def build(force: bool = False) -> str:
-    """Compile the C oracle next to its source (gcc, OpenMP) and return the path."""
+    """Compile the C oracle next to its source (gcc, OpenMP) and return the path.  -ffp-contract=off keeps every
+    product and sum a rounding of its own, as the loops are written."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", _LIB, _SRC, "-lm"]
+        cmd = ["gcc", "-O3", "-march=native", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+               "-o", _LIB, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 

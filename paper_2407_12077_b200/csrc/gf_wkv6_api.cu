@@ -9,6 +9,7 @@
 
 #include "key_compress.cuh"
 #include "ln_heads.cuh"
+#include "wkv6_backward.cuh"
 #include "wkv6_chunked.cuh"
 #include "wkv6_exact.cuh"
 #include "wkv6_step.cuh"
@@ -336,6 +337,55 @@ gf_status_t gf_wkv6_step_f32(const float* r, const float* k, const float* v, con
                              gf_stream_t stream)
 {
     return step_impl<float>(r, k, v, x, u, state_in, state_out, y, B, H, N, (cudaStream_t)stream);
+}
+
+size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N)
+{
+    if (B <= 0 || T <= 0 || H <= 0 || N != 64) return 0;
+    return (size_t)B * H * gf::bw::unit_floats(T) * sizeof(float);
+}
+
+gf_status_t gf_wkv6_backward_f32(const float* r, const float* k, const float* v, const float* x, const float* u,
+                                 const float* state_in, const float* dy, const float* dstate_out, float* dr,
+                                 float* dk, float* dv, float* dx, float* du, float* dstate_in, int B, int T, int H,
+                                 int N, void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if ((long long)B * T >= (1LL << 31)) return GF_ERR_INVALID_ARG;
+    if (B == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t sbytes = (size_t)B * H * 64 * 64 * sizeof(float);
+    if (T == 0) {
+        // no token: the state adjoint passes through and the bonus gets no gradient
+        if (misaligned(dstate_out) || misaligned(dstate_in) || misaligned(du)) return GF_ERR_INVALID_ARG;
+        cudaError_t e = cudaSuccess;
+        if (dstate_in && !dstate_out) e = cudaMemsetAsync(dstate_in, 0, sbytes, st);
+        else if (dstate_in && dstate_in != dstate_out) e = cudaMemcpyAsync(dstate_in, dstate_out, sbytes, cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && du) e = cudaMemsetAsync(du, 0, (size_t)H * 64 * sizeof(float), st);
+        return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+    }
+    if (!r || !k || !v || !x || !u || !dy || !dr || !dk || !dv || !dx || !du) return GF_ERR_INVALID_ARG;
+    const void* ptrs[] = {r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, workspace};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    const void* ins[] = {r, k, v, x, dy};
+    const void* outs[] = {dr, dk, dv, dx};
+    for (const void* o : outs)
+        for (const void* in : ins)
+            if (o == in) return GF_ERR_INVALID_ARG;
+    const long long units = (long long)B * H;
+    if (units > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < gf_wkv6_backward_workspace_bytes(B, T, H, N)) return GF_ERR_WORKSPACE;
+    float* ws = static_cast<float*>(workspace);
+    gf::bw::wkv6_backward_kernel<<<(unsigned)units, gf::bw::THREADS, 0, st>>>(r, k, v, x, u, state_in, dy, dstate_out, dr, dk,
+                                                                            dv, dx, dstate_in, ws, T, H);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    const size_t stride = gf::bw::unit_floats(T);
+    gf::bw::wkv6_backward_du_kernel<<<(unsigned)H, gf::bw::N, 0, st>>>(ws, stride, stride - gf::bw::N, B, H, du);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
 }
 
 size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N)
