@@ -370,17 +370,18 @@ def main():
                 ("cfg3_eight_segments", "cfg3-segments", "8 x gf_wkv6_prefill of 16384 tokens, state carried in place"),
                 ("prefill_c2", "cfg2-c2", "gf_wkv6_prefill_c2 with the second-value tensor, cfg2 shape (768 B per token*head)"),
                 ("key_compress", "kc-cfg2", "gf_gold_key_compress 65536 x 2048 -> 128"),
+                ("decay_logit", "dl-cfg2", "gf_c2_decay_logit, 65536 tokens x 2048 channels, ranks 32 and 64 (x read, d written)"),
                 ("decode_step", "cfg4-decode", "gf_wkv6_step, 64 sequences x 32 heads, 64 steps per graph replay (states stay in L2)"),
                 ("decode_step_layer_stack", "cfg4-decode-layers", "gf_wkv6_step over 12 layers with their own states (streams from HBM)")):
             r = cases.run(case, 5, 1.0)
             ms = r["ms"]
             o = {"kernel": what, "call_ms": ms, "algorithmic_bytes": r["bytes"], "bound": "hbm",
                  "achieved": r["bytes"] / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
-                 "value": r["units"] / (ms * 1e-3), "value_unit": "token*heads/s" if "decode" not in key and key != "key_compress" else ("tokens/s" if key == "key_compress" else "step*heads/s")}
+                 "value": r["units"] / (ms * 1e-3), "value_unit": "tokens/s" if key == "key_compress" else ("step*heads/s" if key.startswith("decode_step") else "token*heads/s")}
             o["frac"] = o["achieved"] / peak
-            if key == "key_compress":
-                # at the crossing of the two rooflines: the bound is the slower of bytes at HBM rate and flops at tensor rate
-                flops = 2.0 * 65536 * 2048 * 128
+            if key in ("key_compress", "decay_logit"):
+                # near the crossing of the two rooflines: the bound is the slower of bytes at HBM rate and flops at tensor rate
+                flops = r["tflops"] * 1e12 * ms * 1e-3
                 t_hbm, t_tc = r["bytes"] / (peak * 1e9), flops / (peak_tf * 1e12)
                 o.update(tflops=r["tflops"], peak_tflops=peak_tf, bound="hbm" if t_hbm >= t_tc else "tensor",
                          frac=max(t_hbm, t_tc) / (ms * 1e-3))

@@ -284,6 +284,28 @@ GF_API gf_status_t gf_c2_layernorm(const void *y, const float *gamma, const floa
 GF_API gf_status_t gf_c2_layernorm_f32(const float *y, const float *gamma, const float *beta, float eps,
                                 float *out, long long rows, int H, int N, gf_stream_t stream);
 
+/* The decay logit of the Finch-C2 block, the producer of the x argument of the prefill calls above:
+ *     d_t = lora_omega( ddlerp_d( x_t, x_{t-1} ) )                                   (Finch-C2 block, d_t equation)
+ * with the operators of the Finch-C2 section, lerp(a, b, t) = a + (b - a) t, lora(v) = lambda + tanh(v A) B and
+ * ddlerp(a, b) = a + (b - a) lora( a + (b - a) mu_x ); the decay itself, w_t = exp(-exp(d_t)), is taken inside the
+ * WKV kernels.  Written out: z = x_t + (x_{t-1} - x_t) mu_x; m = x_t + (x_{t-1} - x_t)(lambda_d + tanh(z A_d) B_d);
+ * d_t = lambda_w + tanh(m A_w) B_w.
+ *   x       DEVICE bf16 [B][T][D]   the block's input (D = heads * 64 channels of the model dimension)
+ *   x_prev  DEVICE bf16 [B][D] or NULL: the token before each sequence's first one (NULL: zeros); x_{t-1} of any
+ *           other token is the row above it
+ *   mu_x, lambda_d, lambda_w   DEVICE fp32 [D]
+ *   A_d [D][Rd], B_d [Rd][D]   DEVICE bf16 row-major: the lora inside ddlerp_d
+ *   A_w [D][Rw], B_w [Rw][D]   DEVICE bf16 row-major: lora_omega
+ *   d       DEVICE bf16 [B][T][D]   written; must not alias x
+ * bf16 operands on the tensor cores with fp32 accumulation; z, m, the two tanh vectors and d are each rounded to
+ * bf16 once; tanh is the hardware approximation (relative error about 2^-11).  D must be a multiple of 64; Rd and Rw
+ * multiples of 16, at most 64 (GF_ERR_UNSUPPORTED otherwise; Finch uses 32 and 64); pointers 16-byte aligned.
+ * Enqueues one kernel on `stream`, allocates nothing, does not synchronise. */
+GF_API gf_status_t gf_c2_decay_logit(const void *x, const void *x_prev, const float *mu_x, const void *A_d,
+                              const void *B_d, const float *lambda_d, const void *A_w, const void *B_w,
+                              const float *lambda_w, void *d, int B, int T, int D, int Rd, int Rw,
+                              gf_stream_t stream);
+
 /* GOLD key compression, the product that ends linear pre-fill: c_t = x_t W^{KD} (GOLD key compression equation),
  * the token's entry of the compressed key cache, with W^{KD} the learned D x D/16 matrix.
  *   x     DEVICE bf16 [rows][D]   (the output of the Finch-C2 layers, one row per token)

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -50,6 +50,7 @@ _SIGNATURES = {
     "gf_c2_layernorm": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_c2_layernorm_f32": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
     "gf_gold_key_compress": (_i, [_vp, _vp, _vp, ctypes.c_longlong, _i, _i, _vp]),
+    "gf_c2_decay_logit": (_i, [_vp] * 10 + [_i] * 5 + [_vp]),
     "gf_wkv6_set_kernel": (_i, [_i]),
     "gf_wkv6_last_device_status": (_i, [_vp]),
     "gf_wkv6_set_wait_limit": (_i, [ctypes.c_uint]),
@@ -358,6 +359,25 @@ def key_compress(x, w_kd, out=None, stream=None):
     with torch.cuda.device(x.device):
         _check(lib.gf_gold_key_compress(_dev(x, "x", bf), _dev(w_kd, "w_kd", bf, (D, Dc)), _dev(out, "c", bf, x.shape[:-1] + (Dc,)),
                                         rows, D, Dc, _stream(stream)), "gf_gold_key_compress")
+    return out
+
+
+def decay_logit(x, mu_x, A_d, B_d, lambda_d, A_w, B_w, lambda_w, x_prev=None, out=None, stream=None):
+    """gf_c2_decay_logit: d = lora_omega(ddlerp_d(x_t, x_{t-1})).  x: [B,T,D] bf16 CUDA tensor (contiguous); mu_x,
+    lambda_d, lambda_w: fp32 [D]; A_d [D,Rd], B_d [Rd,D], A_w [D,Rw], B_w [Rw,D]: bf16; x_prev: [B,D] bf16 or None.
+    Returns d [B,T,D] bf16 (allocated here unless passed as out)."""
+    lib = load_library()
+    B, T, D = x.shape
+    Rd, Rw = A_d.shape[1], A_w.shape[1]
+    bf, f32 = torch.bfloat16, torch.float32
+    if out is None:
+        out = torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        _check(lib.gf_c2_decay_logit(
+            _dev(x, "x", bf), _dev(x_prev, "x_prev", bf, (B, D)), _dev(mu_x, "mu_x", f32, (D,)),
+            _dev(A_d, "A_d", bf, (D, Rd)), _dev(B_d, "B_d", bf, (Rd, D)), _dev(lambda_d, "lambda_d", f32, (D,)),
+            _dev(A_w, "A_w", bf, (D, Rw)), _dev(B_w, "B_w", bf, (Rw, D)), _dev(lambda_w, "lambda_w", f32, (D,)),
+            _dev(out, "d", bf, x.shape), B, T, D, Rd, Rw, _stream(stream)), "gf_c2_decay_logit")
     return out
 
 

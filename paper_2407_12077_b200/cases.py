@@ -4,6 +4,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
 cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
+       dl-cfg1 dl-cfg2
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -125,6 +126,17 @@ def run(case, reps, scale):
                  ms=_time(fn, reps))
         r["tflops"] = 2.0 * rows * D * (D // 16) / (r["ms"] * 1e-3) / 1e12
         return r
+    if case in ("dl-cfg1", "dl-cfg2"):      # decay logit d = lora_omega(ddlerp_d(x_t, x_{t-1})) over the tokens of a prefill call
+        k = c["cfg1" if case == "dl-cfg1" else "cfg2"]
+        B, T, D, Rd, Rw = k["B"], sc(k["T"]), k["H"] * 64, 32, 64
+        x, xp = synth.make_block_input(B, T, D, seed=13, device=DEV)
+        w = synth.make_decay_lora(D, Rd, Rw, seed=14, device=DEV)
+        out = torch.empty_like(x)
+        fn = lambda: gf.decay_logit(x, w["mu_x"], w["A_d"], w["B_d"], w["lambda_d"], w["A_w"], w["B_w"], w["lambda_w"], x_prev=xp, out=out)
+        r = dict(case=case, shape=f"B={B} T={T} D={D} Rd={Rd} Rw={Rw} bf16", units=B * T * k["H"],
+                 bytes=2 * B * T * D * 2 + 4 * D * (Rd + Rw) + 12 * D, ms=_time(fn, reps))
+        r["tflops"] = 2.0 * B * T * D * 2 * (Rd + Rw) / (r["ms"] * 1e-3) / 1e12
+        return r
     if case in ("cfg4-prefill", "cfg4-decode", "cfg4-decode-layers"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -174,7 +186,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2"]
 
 
 def main():

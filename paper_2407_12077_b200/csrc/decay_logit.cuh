@@ -1,0 +1,468 @@
+// The decay logit of the Finch-C2 block for sm_100a: d_t = lora_omega( ddlerp_d( x_t, x_{t-1} ) ), i.e. with
+//   lerp(a, b, t) = a + (b - a) t,   lora(v) = lambda + tanh(v A) B,   ddlerp(a, b) = a + (b - a) lora_d(lerp(a, b, mu_x)):
+//   z_t = x_t + (x_{t-1} - x_t) mu_x                       (token shift, per channel)
+//   h1  = tanh(z_t A_d)                                    [R_d]
+//   m_t = x_t + (x_{t-1} - x_t) (lambda_d + h1 B_d)        (the data-dependent mix)
+//   h2  = tanh(m_t A_w)                                    [R_w]
+//   d_t = lambda_w + h2 B_w                                (the logit the WKV kernels take as x: w_t = exp(-exp(d_t)))
+// x, d: [rows][D] bf16 with rows = B*T (x_{t-1} of a sequence's first token: x_prev[b], or zero); A_*: [D][R], B_*: [R][D]
+// bf16; mu_x, lambda_*: [D] fp32.  Four skinny products (2 D (2 R_d + 2 R_w) flops per token) around elementwise
+// work on a tensor that is read twice and written once: HBM-bound (4 D bytes per token when the second read of x
+// hits L2), so the products run on the tensor cores and everything else is shaped to stream.
+//
+// One persistent CTA per SM walks tiles of 128 tokens in three passes over the D channels, 64 at a time:
+//   pass 1: z slice -> bf16 operand tile -> acc1 += z A_d[slice]           then h1 = tanh(acc1) -> operand tile
+//   pass 2: l = h1 B_d[:, slice] -> tensor memory -> m slice -> bf16 operand tile -> acc3 += m A_w[slice]
+//           then h2 = tanh(acc3) -> operand tile
+//   pass 3: d slice = lambda_w + h2 B_w[:, slice] -> bf16 -> TMA store
+//   warp 0      TMA producer: per slice the x rows of the tile (plus the one row before it), the weight tiles and
+//               the 64 per-channel constants of the pass into a 4-stage ring
+//   warp 1      tensor-memory allocation; an elected lane issues the tcgen05.mma (128 x 64 x 16, bf16 -> fp32)
+//   warps 2-9   two sets of four warps taking alternate slices; a lane owns one token row (the accumulator row of
+//               its tensor-memory sub-partition): reads its row and the row above from the swizzled x tiles, forms
+//               z / m / d for the 64 channels of the slice, writes the bf16 operand row (or the output slab)
+// All operand tiles are the 128-byte-swizzled [64 rows][64 bf16] tiles of the prefill kernel; weight tiles narrower
+// than 64 (R < 64) are zero-filled by TMA beyond their extent.  Every wait is bounded, as in the prefill kernel.
+#pragma once
+#include "wkv6_chunked.cuh"
+
+namespace gf {
+namespace dl {
+
+using namespace ck;
+
+constexpr int DL_THREADS = 32 * 10;
+constexpr int DL_NS = 4;                               // ring stages
+constexpr int DL_STAGE = 4 * TILE + 1024;              // x rows 0-63, x rows 64-127, two weight tiles; row above + constants
+constexpr int DL_OFF_PREV = 4 * TILE;                  // [64] bf16: the x row just above the tile (this slice)
+constexpr int DL_OFF_VEC = 4 * TILE + 256;             // [64] fp32: mu_x / lambda_d / lambda_w of this slice
+constexpr int DL_OFF_OP = DL_NS * DL_STAGE;            // [2 sets][128 rows x 128 B]: z / m operand, output slabs in pass 3
+constexpr int DL_OFF_H = DL_OFF_OP + 4 * TILE;         // [128 rows x 128 B]: h1 / h2 operand
+constexpr int DL_OFF_MISC = DL_OFF_H + 2 * TILE;       // abort word + limit, tensor-memory address, barriers
+constexpr int DL_SMEM = DL_OFF_MISC + 256 + 1024;      // + slack for manual 1024-byte alignment
+enum {
+    DL_FULL = 0,                       // ring stage loaded
+    DL_EMPTY = DL_FULL + DL_NS,        // ... and consumed (four worker warps + the products that read it)
+    DL_OP_READY = DL_EMPTY + DL_NS,    // per set: operand rows written
+    DL_OP_FREE = DL_OP_READY + 2,      // per set: the product that read them is done
+    DL_ACC_FULL = DL_OP_FREE + 2,      // per set: l (pass 2) or d (pass 3) of a slice is in tensor memory
+    DL_ACC_FREE = DL_ACC_FULL + 2,     // per set: ... and read back
+    DL_SUM_FULL = DL_ACC_FREE + 2,     // acc1 / acc3 complete
+    DL_H_READY = DL_SUM_FULL + 1,      // h1 / h2 operand written by all eight worker warps
+    DL_BAR_COUNT = DL_H_READY + 1
+};
+static_assert(16 + 8 * DL_BAR_COUNT <= 256, "barrier block");
+static_assert(DL_SMEM <= 232448, "shared memory budget of one sm_100 CTA");
+constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_L = 128, DL_TM_D = 256;       // + 64 * set for the last two
+// fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = 64
+constexpr uint32_t DL_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct DlParams {
+    long long rows;                    // B * T
+    int T;                             // tokens per sequence (token shift restarts every T rows)
+    int nslices;                       // D / 64
+    int kd, kw;                        // 16-wide contraction steps over the two ranks: R_d / 16, R_w / 16
+    const __nv_bfloat16* x_prev;       // [B][D] or NULL
+    int D;
+    const float *mu_x, *lambda_d, *lambda_w;
+};
+
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ float tanh_fast(float v)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(v));
+    return y;
+}
+// 16 consecutive fp32 columns of this lane's accumulator row
+__device__ __forceinline__ void tmem_ld_row16(uint32_t taddr, float (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]),
+          "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15])
+        : "r"(taddr) : "memory");
+}
+
+__global__ void __launch_bounds__(DL_THREADS, 1)
+decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_x1,
+                   const __grid_constant__ CUtensorMap tm_ad, const __grid_constant__ CUtensorMap tm_bd,
+                   const __grid_constant__ CUtensorMap tm_aw, const __grid_constant__ CUtensorMap tm_bw,
+                   const __grid_constant__ CUtensorMap tm_d32, const DlParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t abort_flag = sbase + DL_OFF_MISC;
+    auto bar = [&](int i) { return sbase + DL_OFF_MISC + 16 + 8 * i; };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long n_tiles = (p.rows + 127) / 128;
+    const int S = p.nslices;
+
+    if (tid == 0) {
+        for (int i = 0; i < DL_NS; ++i) {
+            mbar_init(bar(DL_FULL + i), 1);
+            mbar_init(bar(DL_EMPTY + i), 5);              // four worker warps and one commit
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(DL_OP_READY + i), 4);
+            mbar_init(bar(DL_OP_FREE + i), 1);
+            mbar_init(bar(DL_ACC_FULL + i), 1);
+            mbar_init(bar(DL_ACC_FREE + i), 4);
+        }
+        mbar_init(bar(DL_SUM_FULL), 1);
+        mbar_init(bar(DL_H_READY), 8);
+        sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, WAIT_LIMIT_US);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) tmem_alloc(sbase + DL_OFF_MISC + 8, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32(sbase + DL_OFF_MISC + 8);
+
+    if (warp == 0) {
+        // ============================== TMA producer ==============================
+        int it = 0, issued = 0;
+        bool alive = true;
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
+            const int row0 = (int)(t * 128);
+            for (int pass = 0; pass < 3 && alive; ++pass)
+                for (int s = 0; s < S; ++s, ++it) {
+                    const int st = it % DL_NS;
+                    if (it >= DL_NS && !mbar_wait_warp(bar(DL_EMPTY + st), ((it / DL_NS) + 1) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t dst = sbase + st * DL_STAGE, full = bar(DL_FULL + st);
+                    if (elect_one()) {
+                        if (pass < 2) {
+                            mbar_expect_tx(full, (pass == 0 ? 3 : 4) * TILE + 128 + 256);
+                            tma_load_2d(dst, &tm_x, 64 * s, row0, full);
+                            tma_load_2d(dst + TILE, &tm_x, 64 * s, row0 + 64, full);
+                            tma_load_2d(dst + DL_OFF_PREV, &tm_x1, 64 * s, row0 - 1, full);      // (row -1 reads as zero)
+                            if (pass == 0) {
+                                tma_load_2d(dst + 2 * TILE, &tm_ad, 0, 64 * s, full);
+                                bulk_load_1d(dst + DL_OFF_VEC, p.mu_x + 64 * s, 256, full);
+                            } else {
+                                tma_load_2d(dst + 2 * TILE, &tm_bd, 64 * s, 0, full);
+                                tma_load_2d(dst + 3 * TILE, &tm_aw, 0, 64 * s, full);
+                                bulk_load_1d(dst + DL_OFF_VEC, p.lambda_d + 64 * s, 256, full);
+                            }
+                        } else {
+                            mbar_expect_tx(full, TILE + 256);
+                            tma_load_2d(dst + 2 * TILE, &tm_bw, 64 * s, 0, full);
+                            bulk_load_1d(dst + DL_OFF_VEC, p.lambda_w + 64 * s, 256, full);
+                        }
+                    }
+                    __syncwarp();
+                    issued = it + 1;
+                }
+        }
+        // do not leave while copies into this CTA's shared memory may still be in flight
+        for (int c = max(0, issued - DL_NS); c < issued; ++c)
+            mbar_wait_warp(bar(DL_FULL + c % DL_NS), (c / DL_NS) & 1, abort_flag, false);
+    } else if (warp == 1) {
+        // ============================== MMA issuer ==============================
+        int it = 0, ti = 0;
+        int op_uses[2] = {0, 0}, acc_uses[2] = {0, 0};       // per set: operand tiles consumed, l / d accumulators produced
+        bool alive = true;
+        auto stage_full = [&](int i) { return mbar_wait_warp(bar(DL_FULL + i % DL_NS), (i / DL_NS) & 1, abort_flag); };
+        const uint64_t dh = smem_desc(sbase + DL_OFF_H);
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
+            // ---- pass 1: acc1 += z A_d[slice]
+            for (int s = 0; s < S; ++s, ++it) {
+                const int h = s & 1;
+                if (!stage_full(it) || !mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
+                ++op_uses[h];
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
+                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma(tmem + DL_TM_ACC1, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (s > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(bar(DL_OP_FREE + h));
+                    tc_commit(bar(DL_EMPTY + it % DL_NS));
+                    if (s == S - 1) tc_commit(bar(DL_SUM_FULL));
+                }
+                __syncwarp();
+            }
+            if (!alive) break;
+            // ---- pass 2: l = h1 B_d[:, slice] one slice ahead of acc3 += m A_w[slice]
+            if (!mbar_wait_warp(bar(DL_H_READY), 0, abort_flag)) break;          // (two uses per tile: parities 0, 1)
+            tc_fence_after();
+            const int it2 = it;
+            for (int s = 0; s <= S; ++s) {
+                if (s < S) {
+                    const int h = s & 1, i = it2 + s;
+                    if (!stage_full(i)) { alive = false; break; }
+                    if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
+                    ++acc_uses[h];
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 2 * TILE);
+                        for (int kk = 0; kk < p.kd; ++kk)
+                            tc_mma(tmem + DL_TM_L + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
+                        tc_commit(bar(DL_ACC_FULL + h));
+                    }
+                    __syncwarp();
+                }
+                if (s >= 1) {
+                    const int q = s - 1, h = q & 1, i = it2 + q;
+                    if (!mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
+                    ++op_uses[h];
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
+                        const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 3 * TILE);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            tc_mma(tmem + DL_TM_ACC3, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (q > 0 || kk > 0) ? 1u : 0u);
+                        tc_commit(bar(DL_OP_FREE + h));
+                        tc_commit(bar(DL_EMPTY + i % DL_NS));
+                        if (q == S - 1) tc_commit(bar(DL_SUM_FULL));
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!alive) break;
+            it += S;
+            // ---- pass 3: d slice = h2 B_w[:, slice]
+            if (!mbar_wait_warp(bar(DL_H_READY), 1, abort_flag)) break;
+            tc_fence_after();
+            for (int s = 0; s < S; ++s, ++it) {
+                const int h = s & 1;
+                if (!stage_full(it)) { alive = false; break; }
+                if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
+                ++acc_uses[h];
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+                    for (int kk = 0; kk < p.kw; ++kk)
+                        tc_mma(tmem + DL_TM_D + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
+                    tc_commit(bar(DL_ACC_FULL + h));
+                    tc_commit(bar(DL_EMPTY + it % DL_NS));
+                }
+                __syncwarp();
+            }
+        }
+    } else {
+        // ============================== worker warps ==============================
+        const int set = (warp - 2) >> 2;                 // takes the slices s with s mod 2 == set
+        const int sp = warp & 3;                         // tensor-memory sub-partition: accumulator rows 32*sp .. 32*sp+31
+        const int row = 32 * sp + lane;                  // this lane's token row inside the tile
+        const uint32_t tlane = (uint32_t)(32 * sp) << 16;
+        // this lane's 128-byte row in a pair of stacked tiles: byte offset of its 16-byte unit q
+        const uint32_t own_tile = (uint32_t)(row >> 6) * TILE, own_row = (uint32_t)(row & 63);
+        const uint32_t up_tile = (uint32_t)((row - 1) >> 6) * TILE, up_row = (uint32_t)((row - 1) & 63);   // (row > 0)
+        const uint32_t op_rows = sbase + DL_OFF_OP + set * 2 * TILE + own_tile;     // this set's operand tiles (this lane's tile)
+        const uint32_t slab = sbase + DL_OFF_OP + set * 2 * TILE + sp * 4096;       // pass 3: this warp's 32-row output slab
+        const uint32_t h_rows = sbase + DL_OFF_H + own_tile;
+        int op_uses = 0, acc_uses = 0, ti = 0;
+        bool alive = true;
+
+        // z or m for the 64 channels of one slice: out = x + (x_above - x) * mix, mix = vec (+ l from tensor memory)
+        auto mix_slice = [&](uint32_t stage, long long tok, int s, bool with_l, uint32_t tl) {
+            const bool seq_start = (tok % p.T) == 0;     // the row above belongs to another sequence: x_prev or zero
+            const __nv_bfloat16* gp = (seq_start && p.x_prev && tok < p.rows) ? p.x_prev + (tok / p.T) * (long long)p.D + 64 * s : nullptr;
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) {             // 16 channels at a time
+                float l[16];
+                if (with_l) tmem_ld_row16(tl + 16 * q2, l);
+#pragma unroll
+                for (int qq = 0; qq < 2; ++qq) {
+                    const int q = 2 * q2 + qq;           // 16-byte unit = 8 channels
+                    const uint4 a = lds128(stage + own_tile + swz(own_row, q << 4));
+                    uint4 b;
+                    if (seq_start) {
+                        b = gp ? *reinterpret_cast<const uint4*>(gp + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
+                    } else if (row == 0) {
+                        b = lds128(stage + DL_OFF_PREV + 16 * q);
+                    } else {
+                        b = lds128(stage + up_tile + swz(up_row, q << 4));
+                    }
+                    const float4 v0 = ldsf4(stage + DL_OFF_VEC + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 32 * q + 16);
+                    const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+                    uint32_t ow[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 xa = bf_pair(aw[e]), xb = bf_pair(bw[e]);
+                        float2 mix = make_float2(vv[2 * e], vv[2 * e + 1]);
+                        if (with_l) mix = add2(mix, make_float2(l[8 * qq + 2 * e], l[8 * qq + 2 * e + 1]));
+                        const float2 o = fma2(sub2(xb, xa), mix, xa);
+                        ow[e] = pack_bf16(o.x, o.y);
+                    }
+                    sts128(op_rows + swz(own_row, q << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                }
+            }
+        };
+        // h = tanh(acc) for this warp's 32 rows and this set's 32 columns -> bf16 operand rows
+        auto squash = [&](uint32_t tacc) {
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2) {
+                float a[16];
+                tmem_ld_row16(tacc + 32 * set + 16 * q2, a);
+#pragma unroll
+                for (int qq = 0; qq < 2; ++qq) {
+                    uint32_t ow[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        ow[e] = pack_bf16(tanh_fast(a[8 * qq + 2 * e]), tanh_fast(a[8 * qq + 2 * e + 1]));
+                    sts128(h_rows + swz(own_row, (4 * set + 2 * q2 + qq) << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                }
+            }
+        };
+
+        int it = 0;
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
+            const long long tok = t * 128 + row;
+            // ---- passes 1 and 2
+            for (int pass = 0; pass < 2 && alive; ++pass) {
+                for (int s = 0; s < S; ++s, ++it) {
+                    if ((s & 1) != set) continue;
+                    const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
+                    if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
+                    if (pass == 1) {
+                        if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
+                        ++acc_uses;
+                        tc_fence_after();
+                    }
+                    // the operand rows: free of the product that read them last, and of this warp's own output store
+                    if (op_uses >= 1 && !mbar_wait(bar(DL_OP_FREE + set), (op_uses - 1) & 1, abort_flag)) { alive = false; break; }
+                    ++op_uses;
+                    mix_slice(stage, tok, s, pass == 1, tmem + tlane + DL_TM_L + 64 * set);
+                    fence_proxy_async();
+                    if (pass == 1) tc_fence_before();
+                    __syncwarp();
+                    mbar_arrive_if(bar(DL_OP_READY + set), lane == 0);
+                    if (pass == 1) mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                    mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
+                }
+                if (!alive) break;
+                // the pass's low-rank sum is complete: squash it into the operand of the next product
+                if (!mbar_wait(bar(DL_SUM_FULL), pass, abort_flag)) { alive = false; break; }      // (two uses per tile)
+                tc_fence_after();
+                squash(tmem + tlane + (pass == 0 ? DL_TM_ACC1 : DL_TM_ACC3));
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                mbar_arrive_if(bar(DL_H_READY), lane == 0);
+            }
+            if (!alive) break;
+            // ---- pass 3: d slice -> bf16 slab -> TMA store
+            for (int s = 0; s < S; ++s, ++it) {
+                if ((s & 1) != set) continue;
+                const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
+                if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
+                if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
+                ++acc_uses;
+                tc_fence_after();
+                if (lane == 0) bulk_wait_read<0>();      // this warp's previous store has finished reading the slab
+                __syncwarp();
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2) {
+                    float a[16];
+                    tmem_ld_row16(tmem + tlane + DL_TM_D + 64 * set + 16 * q2, a);
+#pragma unroll
+                    for (int qq = 0; qq < 2; ++qq) {
+                        const int q = 2 * q2 + qq;
+                        const float4 v0 = ldsf4(stage + DL_OFF_VEC + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 32 * q + 16);
+                        const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                        uint32_t ow[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            ow[e] = pack_bf16(a[8 * qq + 2 * e] + vv[2 * e], a[8 * qq + 2 * e + 1] + vv[2 * e + 1]);
+                        sts128(slab + swz(lane, q << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                    }
+                }
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                const long long grow = t * 128 + 32 * sp;
+                if (lane == 0 && grow < p.rows) {
+                    tma_store_2d(&tm_d32, 64 * s, (int)grow, slab);
+                    bulk_commit();
+                }
+                mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
+            }
+            // the slab doubles as this warp's operand rows of the next tile
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
+        }
+        if (lane == 0) bulk_wait<0>();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+// [rows][cols] bf16 tensor map with a box of box_rows x box_cols (box_cols * 2 bytes <= 128)
+inline bool make_map_box(CUtensorMap* tm, const void* base, long long rows, long long cols, int box_rows, int box_cols, bool swizzle)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace dl
+
+// d = lora_omega(ddlerp_d(x, shifted x)) over rows = B*T tokens of D channels; see the top of this file.
+inline gf_status_t decay_logit(const __nv_bfloat16* x, const __nv_bfloat16* x_prev, const float* mu_x,
+                               const __nv_bfloat16* A_d, const __nv_bfloat16* B_d, const float* lambda_d,
+                               const __nv_bfloat16* A_w, const __nv_bfloat16* B_w, const float* lambda_w,
+                               __nv_bfloat16* d, int B, int T, int D, int Rd, int Rw, cudaStream_t st,
+                               std::atomic<uint64_t>* launches)
+{
+    const long long rows = (long long)B * T;
+    static PerDeviceFlag attr_set;
+    const int dev = current_device();
+    if (dev < 0) return GF_ERR_CUDA;
+    if (!attr_set.is_set(dev)) {
+        if (cudaFuncSetAttribute(dl::decay_logit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dl::DL_SMEM) != cudaSuccess)
+            return GF_ERR_CUDA;
+        attr_set.set(dev);
+    }
+    CUtensorMap tx, tx1, tad, tbd, taw, tbw, td;
+    if (!dl::make_map_box(&tx, x, rows, D, 64, 64, true) || !dl::make_map_box(&tx1, x, rows, D, 1, 64, false) ||
+        !dl::make_map_box(&tad, A_d, D, Rd, 64, 64, true) || !dl::make_map_box(&tbd, B_d, Rd, D, 64, 64, true) ||
+        !dl::make_map_box(&taw, A_w, D, Rw, 64, 64, true) || !dl::make_map_box(&tbw, B_w, Rw, D, 64, 64, true) ||
+        !dl::make_map_box(&td, d, rows, D, 32, 64, true))
+        return GF_ERR_CUDA;
+    dl::DlParams p{rows, T, D / 64, Rd / 16, Rw / 16, x_prev, D, mu_x, lambda_d, lambda_w};
+    const long long n_tiles = (rows + 127) / 128;
+    const int n_sm = sm_count();
+    const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);
+    dl::decay_logit_kernel<<<grid, dl::DL_THREADS, dl::DL_SMEM, st>>>(tx, tx1, tad, tbd, taw, tbw, td, p);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+}  // namespace gf

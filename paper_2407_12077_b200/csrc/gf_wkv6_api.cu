@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include "decay_logit.cuh"
 #include "key_compress.cuh"
 #include "ln_heads.cuh"
 #include "wkv6_backward.cuh"
@@ -506,6 +507,23 @@ gf_status_t gf_gold_key_compress(const void* x, const void* w_kd, void* c, long 
     if (rows >= (1LL << 31) - 256) return GF_ERR_INVALID_ARG;
     if (!x || !w_kd || !c || misaligned(x) || misaligned(w_kd) || misaligned(c) || c == x || c == w_kd) return GF_ERR_INVALID_ARG;
     return gf::key_compress((const bf*)x, (const bf*)w_kd, (bf*)c, rows, D, Dc, (cudaStream_t)stream, &g_launches);
+}
+
+gf_status_t gf_c2_decay_logit(const void* x, const void* x_prev, const float* mu_x, const void* A_d, const void* B_d,
+                              const float* lambda_d, const void* A_w, const void* B_w, const float* lambda_w, void* d,
+                              int B, int T, int D, int Rd, int Rw, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || D < 0 || Rd < 0 || Rw < 0) return GF_ERR_INVALID_ARG;
+    if (B == 0 || T == 0 || D == 0) return GF_OK;
+    if ((D & 63) || Rd == 0 || Rw == 0 || (Rd & 15) || (Rw & 15) || Rd > 64 || Rw > 64) return GF_ERR_UNSUPPORTED;
+    if ((long long)B * T >= (1LL << 31) - 128) return GF_ERR_INVALID_ARG;
+    if (!x || !mu_x || !A_d || !B_d || !lambda_d || !A_w || !B_w || !lambda_w || !d || d == x) return GF_ERR_INVALID_ARG;
+    const void* ptrs[] = {x, x_prev, mu_x, A_d, B_d, lambda_d, A_w, B_w, lambda_w, d};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    return gf::decay_logit((const bf*)x, (const bf*)x_prev, mu_x, (const bf*)A_d, (const bf*)B_d, lambda_d, (const bf*)A_w,
+                           (const bf*)B_w, lambda_w, (bf*)d, B, T, D, Rd, Rw, (cudaStream_t)stream, &g_launches);
 }
 
 const char* gf_status_string(gf_status_t s)

@@ -97,3 +97,26 @@ def make_step(B, H, N=64, dtype="bf16", seed=0, device="cpu", state_std=0.1) -> 
     """Inputs of one decode step: r,k,v,x [B,H,N], state_in [B,H,N,N]."""
     r, k, v, x, u, s = _draw((B, H, N), B, H, N, dtype, seed, device, state_std, -6.0, -1.0)
     return Wkv6Inputs(r, k, v, x, u, s)
+
+
+def make_decay_lora(D, Rd=32, Rw=64, seed=0, device="cpu"):
+    """Weights of the decay-logit producer of a Finch-C2 block (stand-ins for trained ones): mu_x, lambda_d ~ U(0,1)
+    (token-shift mixes), A ~ N(0, 1/D) so that the low-rank pre-activations are O(1), B ~ N(0, 1/R) so that each
+    lora adds a vector of about unit scale, lambda_w ~ U(-6,-1) (the decay-logit range of the prefill workloads).
+    Matrices are rounded to bf16, vectors stay fp32.  Returns a dict of tensors."""
+    g = _gen(seed, device)
+    f = dict(device=device, dtype=torch.float32, generator=g)
+    bf = torch.bfloat16
+    return dict(mu_x=torch.rand(D, **f), lambda_d=torch.rand(D, **f), lambda_w=torch.rand(D, **f) * 5 - 6,
+                A_d=(torch.randn((D, Rd), **f) / D ** 0.5).to(bf), B_d=(torch.randn((Rd, D), **f) / Rd ** 0.5).to(bf),
+                A_w=(torch.randn((D, Rw), **f) / D ** 0.5).to(bf), B_w=(torch.randn((Rw, D), **f) / Rw ** 0.5).to(bf))
+
+
+def make_block_input(B, T, D, seed=0, device="cpu", with_prev=True):
+    """Input of a Finch-C2 block (a normalised residual stream stand-in): x ~ N(0,1) [B,T,D] bf16 and the token
+    before each sequence's first one [B,D] (or None)."""
+    g = _gen(seed, device)
+    f = dict(device=device, dtype=torch.float32, generator=g)
+    x = torch.randn((B, T, D), **f).to(torch.bfloat16)
+    xp = torch.randn((B, D), **f).to(torch.bfloat16) if with_prev else None
+    return x, xp
