@@ -16,14 +16,18 @@
 //           then h2 = tanh(acc3) -> operand tile
 //   pass 3: d slice = lambda_w + h2 B_w[:, slice] -> bf16 -> TMA store
 //   warp 0      TMA producer: per slice the x rows of the tile (plus the one row before it), the weight tiles and
-//               the 64 per-channel constants of the pass into a 4-stage ring
-//   warp 1      tensor-memory allocation; an elected lane issues the tcgen05.mma (128 x 64 x 16, bf16 -> fp32)
-//   warps 2-9   two sets of four warps taking alternate slices; a lane owns one token row (the accumulator row of
-//               its tensor-memory sub-partition): reads its row and the row above from the swizzled x tiles, forms
-//               z / m / d for the 64 channels of the slice, writes the bf16 operand row (or the output slab)
+//               the 64 per-channel constants of the pass into a 5-stage ring
+//   warp 1      tensor-memory allocation; an elected lane issues the products whose operands come from the ring and
+//               the h tile (z A_d, h1 B_d, h2 B_w; tcgen05.mma 128 x 64 x 16, bf16 -> fp32)
+//   warp 2      an elected lane issues m A_w, the product that waits for the workers inside pass 2 (an issuer of
+//               its own, so that the l products of later slices are not held up behind it)
+//   warps 3-10  two sets of four warps taking alternate slices; a lane owns one token row (the accumulator row
+//               of its tensor-memory sub-partition): reads its row and the row above from the swizzled x tiles,
+//               forms z / m / d for the 64 channels of the slice, writes the bf16 operand row (or the output slab)
 // All operand tiles are the 128-byte-swizzled [64 rows][64 bf16] tiles of the prefill kernel; weight tiles narrower
 // than 64 (R < 64) are zero-filled by TMA beyond their extent.  Every wait is bounded, as in the prefill kernel.
 #pragma once
+#include "key_compress.cuh"
 #include "wkv6_chunked.cuh"
 
 namespace gf {
@@ -31,29 +35,34 @@ namespace dl {
 
 using namespace ck;
 
-constexpr int DL_THREADS = 32 * 10;
-constexpr int DL_NS = 4;                               // ring stages
+constexpr int DL_NSET = 2;                             // worker sets
+constexpr int DL_W0 = 3;                               // first worker warp
+constexpr int DL_THREADS = 32 * (DL_W0 + 4 * DL_NSET);
+constexpr int DL_NS = 5;                               // ring stages: three more than worker sets, so that a slice's loads are
+                                                       // issued about a load latency before its set turns to it
 constexpr int DL_STAGE = 4 * TILE + 1024;              // x rows 0-63, x rows 64-127, two weight tiles; row above + constants
 constexpr int DL_OFF_PREV = 4 * TILE;                  // [64] bf16: the x row just above the tile (this slice)
 constexpr int DL_OFF_VEC = 4 * TILE + 256;             // [64] fp32: mu_x / lambda_d / lambda_w of this slice
-constexpr int DL_OFF_OP = DL_NS * DL_STAGE;            // [2 sets][128 rows x 128 B]: z / m operand, output slabs in pass 3
-constexpr int DL_OFF_H = DL_OFF_OP + 4 * TILE;         // [128 rows x 128 B]: h1 / h2 operand
+constexpr int DL_OFF_OP = DL_NS * DL_STAGE;            // [sets][128 rows x 128 B]: z / m operand, output slabs in pass 3
+constexpr int DL_OFF_H = DL_OFF_OP + DL_NSET * 2 * TILE;         // [128 rows x 128 B]: h1 / h2 operand
 constexpr int DL_OFF_MISC = DL_OFF_H + 2 * TILE;       // abort word + limit, tensor-memory address, barriers
 constexpr int DL_SMEM = DL_OFF_MISC + 256 + 1024;      // + slack for manual 1024-byte alignment
 enum {
     DL_FULL = 0,                       // ring stage loaded
     DL_EMPTY = DL_FULL + DL_NS,        // ... and consumed (four worker warps + the products that read it)
     DL_OP_READY = DL_EMPTY + DL_NS,    // per set: operand rows written
-    DL_OP_FREE = DL_OP_READY + 2,      // per set: the product that read them is done
-    DL_ACC_FULL = DL_OP_FREE + 2,      // per set: l (pass 2) or d (pass 3) of a slice is in tensor memory
-    DL_ACC_FREE = DL_ACC_FULL + 2,     // per set: ... and read back
-    DL_SUM_FULL = DL_ACC_FREE + 2,     // acc1 / acc3 complete
-    DL_H_READY = DL_SUM_FULL + 1,      // h1 / h2 operand written by all eight worker warps
-    DL_BAR_COUNT = DL_H_READY + 1
+    DL_OP_FREE = DL_OP_READY + DL_NSET,    // per set: the product that read them is done
+    DL_ACC_FULL = DL_OP_FREE + DL_NSET,    // per set: l (pass 2) or d (pass 3) of a slice is in tensor memory
+    DL_ACC_FREE = DL_ACC_FULL + DL_NSET,   // per set: ... and read back
+    DL_SUM_FULL = DL_ACC_FREE + DL_NSET,   // acc1 / acc3 complete
+    DL_H_READY = DL_SUM_FULL + 1,      // h1 / h2 operand written by all worker warps
+    DL_PASS2 = DL_H_READY + 1,         // pass 2 of a tile has begun (first issuer -> second issuer: one phase per tile)
+    DL_BAR_COUNT = DL_PASS2 + 1
 };
 static_assert(16 + 8 * DL_BAR_COUNT <= 256, "barrier block");
 static_assert(DL_SMEM <= 232448, "shared memory budget of one sm_100 CTA");
-constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_L = 128, DL_TM_D = 256;       // + 64 * set for the last two
+constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_L = 128, DL_TM_D = 128;       // + 64 * set for the last two (one region:
+                                                                                  // l in pass 2, d in pass 3)
 // fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = 64
 constexpr uint32_t DL_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 
@@ -120,14 +129,15 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             mbar_init(bar(DL_FULL + i), 1);
             mbar_init(bar(DL_EMPTY + i), 5);              // four worker warps and one commit
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < DL_NSET; ++i) {
             mbar_init(bar(DL_OP_READY + i), 4);
             mbar_init(bar(DL_OP_FREE + i), 1);
             mbar_init(bar(DL_ACC_FULL + i), 1);
             mbar_init(bar(DL_ACC_FREE + i), 4);
         }
         mbar_init(bar(DL_SUM_FULL), 1);
-        mbar_init(bar(DL_H_READY), 8);
+        mbar_init(bar(DL_H_READY), 4 * DL_NSET);
+        mbar_init(bar(DL_PASS2), 1);
         sts32(abort_flag, 0u);
         sts32(abort_flag + 4, WAIT_LIMIT_US);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -178,16 +188,16 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         for (int c = max(0, issued - DL_NS); c < issued; ++c)
             mbar_wait_warp(bar(DL_FULL + c % DL_NS), (c / DL_NS) & 1, abort_flag, false);
     } else if (warp == 1) {
-        // ============================== MMA issuer ==============================
-        int it = 0, ti = 0;
-        int op_uses[2] = {0, 0}, acc_uses[2] = {0, 0};       // per set: operand tiles consumed, l / d accumulators produced
+        // ============================== MMA issuer: z A_d, h1 B_d, h2 B_w ==============================
+        int it = 0;
+        int op_uses[DL_NSET] = {}, acc_uses[DL_NSET] = {};   // per set: operand tiles consumed, l / d accumulators produced
         bool alive = true;
         auto stage_full = [&](int i) { return mbar_wait_warp(bar(DL_FULL + i % DL_NS), (i / DL_NS) & 1, abort_flag); };
         const uint64_t dh = smem_desc(sbase + DL_OFF_H);
-        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
             // ---- pass 1: acc1 += z A_d[slice]
             for (int s = 0; s < S; ++s, ++it) {
-                const int h = s & 1;
+                const int h = s % DL_NSET;
                 if (!stage_full(it) || !mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
                 ++op_uses[h];
                 tc_fence_after();
@@ -204,50 +214,32 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 __syncwarp();
             }
             if (!alive) break;
-            // ---- pass 2: l = h1 B_d[:, slice] one slice ahead of acc3 += m A_w[slice]
+            // ---- pass 2: l = h1 B_d[:, slice] (the other issuer follows with acc3 += m A_w[slice] and frees the stage)
             if (!mbar_wait_warp(bar(DL_H_READY), 0, abort_flag)) break;          // (two uses per tile: parities 0, 1)
             tc_fence_after();
-            const int it2 = it;
-            for (int s = 0; s <= S; ++s) {
-                if (s < S) {
-                    const int h = s & 1, i = it2 + s;
-                    if (!stage_full(i)) { alive = false; break; }
-                    if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
-                    ++acc_uses[h];
-                    tc_fence_after();
-                    if (elect_one()) {
-                        const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 2 * TILE);
-                        for (int kk = 0; kk < p.kd; ++kk)
-                            tc_mma(tmem + DL_TM_L + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
-                        tc_commit(bar(DL_ACC_FULL + h));
-                    }
-                    __syncwarp();
+            if (elect_one()) mbar_arrive(bar(DL_PASS2));                           // every operand-row phase of pass 1 is over
+            __syncwarp();
+            for (int s = 0; s < S; ++s, ++it) {
+                const int h = s % DL_NSET;
+                if (!stage_full(it)) { alive = false; break; }
+                if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
+                ++acc_uses[h];
+                ++op_uses[h];                                 // (the other issuer consumes this slice's operand rows)
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+                    for (int kk = 0; kk < p.kd; ++kk)
+                        tc_mma(tmem + DL_TM_L + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
+                    tc_commit(bar(DL_ACC_FULL + h));
                 }
-                if (s >= 1) {
-                    const int q = s - 1, h = q & 1, i = it2 + q;
-                    if (!mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
-                    ++op_uses[h];
-                    tc_fence_after();
-                    if (elect_one()) {
-                        const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
-                        const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 3 * TILE);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            tc_mma(tmem + DL_TM_ACC3, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (q > 0 || kk > 0) ? 1u : 0u);
-                        tc_commit(bar(DL_OP_FREE + h));
-                        tc_commit(bar(DL_EMPTY + i % DL_NS));
-                        if (q == S - 1) tc_commit(bar(DL_SUM_FULL));
-                    }
-                    __syncwarp();
-                }
+                __syncwarp();
             }
             if (!alive) break;
-            it += S;
             // ---- pass 3: d slice = h2 B_w[:, slice]
             if (!mbar_wait_warp(bar(DL_H_READY), 1, abort_flag)) break;
             tc_fence_after();
             for (int s = 0; s < S; ++s, ++it) {
-                const int h = s & 1;
+                const int h = s % DL_NSET;
                 if (!stage_full(it)) { alive = false; break; }
                 if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
                 ++acc_uses[h];
@@ -262,81 +254,137 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 __syncwarp();
             }
         }
+    } else if (warp == 2) {
+        // ============================== MMA issuer: m A_w (pass 2) ==============================
+        int ti = 0;
+        int op_uses[DL_NSET] = {};
+        bool alive = true;
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
+            // A wait names a phase by its parity alone, so it must not start more than one phase ahead of the barrier:
+            // the operand-row barriers go through pass 1's phases first (the other issuer's), hence the go-ahead.
+            if (!mbar_wait_warp(bar(DL_PASS2), ti & 1, abort_flag)) break;
+            for (int s = 0; s < S; ++s) op_uses[s % DL_NSET] += 1;        // pass 1's uses of the operand rows
+            const int it2 = ti * 3 * S + S;                               // ring position of pass 2, slice 0
+            for (int s = 0; s < S; ++s) {
+                const int h = s % DL_NSET, i = it2 + s;
+                // the operand rows are written after the stage was seen full, so the weight tile is in place as well
+                if (!mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
+                ++op_uses[h];
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
+                    const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 3 * TILE);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma(tmem + DL_TM_ACC3, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (s > 0 || kk > 0) ? 1u : 0u);
+                    tc_commit(bar(DL_OP_FREE + h));
+                    tc_commit(bar(DL_EMPTY + i % DL_NS));
+                    if (s == S - 1) tc_commit(bar(DL_SUM_FULL));
+                }
+                __syncwarp();
+            }
+        }
     } else {
         // ============================== worker warps ==============================
-        const int set = (warp - 2) >> 2;                 // takes the slices s with s mod 2 == set
+        const int set = (warp - DL_W0) >> 2;             // takes the slices s with s mod DL_NSET == set
         const int sp = warp & 3;                         // tensor-memory sub-partition: accumulator rows 32*sp .. 32*sp+31
         const int row = 32 * sp + lane;                  // this lane's token row inside the tile
         const uint32_t tlane = (uint32_t)(32 * sp) << 16;
-        // this lane's 128-byte row in a pair of stacked tiles: byte offset of its 16-byte unit q
         const uint32_t own_tile = (uint32_t)(row >> 6) * TILE, own_row = (uint32_t)(row & 63);
         const uint32_t up_tile = (uint32_t)((row - 1) >> 6) * TILE, up_row = (uint32_t)((row - 1) & 63);   // (row > 0)
-        const uint32_t op_rows = sbase + DL_OFF_OP + set * 2 * TILE + own_tile;     // this set's operand tiles (this lane's tile)
+        const uint32_t own_xor = (own_row & 7) << 4;
+        const uint32_t out_base = sbase + DL_OFF_OP + set * 2 * TILE + own_tile + own_row * 128;   // this lane's operand row
         const uint32_t slab = sbase + DL_OFF_OP + set * 2 * TILE + sp * 4096;       // pass 3: this warp's 32-row output slab
-        const uint32_t h_rows = sbase + DL_OFF_H + own_tile;
-        int op_uses = 0, acc_uses = 0, ti = 0;
+        const uint32_t h_row = sbase + DL_OFF_H + own_tile + own_row * 128;
+        int op_uses = 0, acc_uses = 0;
         bool alive = true;
 
-        // z or m for the 64 channels of one slice: out = x + (x_above - x) * mix, mix = vec (+ l from tensor memory)
+        // z or m for the 64 channels of one slice: out = x + (x_above - x) * mix, mix = vec (+ l from tensor memory).
+        // The interpolation itself runs on packed bf16 pairs (difference, then one fused multiply-add with a single
+        // rounding): its inputs and its output are bf16 anyway, and the mix is smooth in them.  32 channels at a time.
         auto mix_slice = [&](uint32_t stage, long long tok, int s, bool with_l, uint32_t tl) {
             const bool seq_start = (tok % p.T) == 0;     // the row above belongs to another sequence: x_prev or zero
+            // the row above: inside the tiles, or (first row of the tile) the extra row of the stage
+            const uint32_t up_base = row == 0 ? stage + DL_OFF_PREV : stage + up_tile + up_row * 128;
+            const uint32_t up_xor = row == 0 ? 0u : (up_row & 7) << 4;
+            const uint32_t own_base = stage + own_tile + own_row * 128;
+            const bool any_start = __any_sync(0xffffffffu, seq_start);
             const __nv_bfloat16* gp = (seq_start && p.x_prev && tok < p.rows) ? p.x_prev + (tok / p.T) * (long long)p.D + 64 * s : nullptr;
 #pragma unroll
-            for (int q2 = 0; q2 < 4; ++q2) {             // 16 channels at a time
-                float l[16];
-                if (with_l) tmem_ld_row16(tl + 16 * q2, l);
-#pragma unroll
-                for (int qq = 0; qq < 2; ++qq) {
-                    const int q = 2 * q2 + qq;           // 16-byte unit = 8 channels
-                    const uint4 a = lds128(stage + own_tile + swz(own_row, q << 4));
-                    uint4 b;
-                    if (seq_start) {
-                        b = gp ? *reinterpret_cast<const uint4*>(gp + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
-                    } else if (row == 0) {
-                        b = lds128(stage + DL_OFF_PREV + 16 * q);
-                    } else {
-                        b = lds128(stage + up_tile + swz(up_row, q << 4));
+            for (int half = 0; half < 2; ++half) {
+                uint32_t mixw[16];                       // the mix of 32 channels as bf16 pairs
+                if (with_l) {
+                    uint32_t l[32];
+                    kc::tmem_ld_row32(tl + 32 * half, l);
+                    if (half == 1) {                     // the accumulator row has been read: hand it back
+                        tc_fence_before();
+                        __syncwarp();
+                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
                     }
-                    const float4 v0 = ldsf4(stage + DL_OFF_VEC + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 32 * q + 16);
-                    const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
+                        mixw[2 * q] = pack_bf16(v4.x + __uint_as_float(l[4 * q]), v4.y + __uint_as_float(l[4 * q + 1]));
+                        mixw[2 * q + 1] = pack_bf16(v4.z + __uint_as_float(l[4 * q + 2]), v4.w + __uint_as_float(l[4 * q + 3]));
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
+                        mixw[2 * q] = pack_bf16(v4.x, v4.y);
+                        mixw[2 * q + 1] = pack_bf16(v4.z, v4.w);
+                    }
+                }
+                uint4 a[4], b[4];                        // this lane's row and the row above: all loads first
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    a[q] = lds128(own_base + ((uint32_t)((4 * half + q) << 4) ^ own_xor));
+                    b[q] = lds128(up_base + ((uint32_t)((4 * half + q) << 4) ^ up_xor));
+                }
+                if (any_start && seq_start) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        b[q] = gp ? *reinterpret_cast<const uint4*>(gp + 8 * (4 * half + q)) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t aw[4] = {a[q].x, a[q].y, a[q].z, a[q].w}, bw[4] = {b[q].x, b[q].y, b[q].z, b[q].w};
                     uint32_t ow[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float2 xa = bf_pair(aw[e]), xb = bf_pair(bw[e]);
-                        float2 mix = make_float2(vv[2 * e], vv[2 * e + 1]);
-                        if (with_l) mix = add2(mix, make_float2(l[8 * qq + 2 * e], l[8 * qq + 2 * e + 1]));
-                        const float2 o = fma2(sub2(xb, xa), mix, xa);
-                        ow[e] = pack_bf16(o.x, o.y);
+                        uint32_t delta;
+                        asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(delta) : "r"(bw[e]), "r"(aw[e]));
+                        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(ow[e]) : "r"(delta), "r"(mixw[4 * q + e]), "r"(aw[e]));
                     }
-                    sts128(op_rows + swz(own_row, q << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                    sts128(out_base + ((uint32_t)((4 * half + q) << 4) ^ own_xor), make_uint4(ow[0], ow[1], ow[2], ow[3]));
                 }
             }
         };
-        // h = tanh(acc) for this warp's 32 rows and this set's 32 columns -> bf16 operand rows
+        // h = tanh(acc) for this warp's 32 rows and this set's share of the 64 columns -> bf16 operand rows
         auto squash = [&](uint32_t tacc) {
+            constexpr int HC = 64 / DL_NSET;             // columns per set
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
+            for (int g = 0; g < HC / 16; ++g) {
                 float a[16];
-                tmem_ld_row16(tacc + 32 * set + 16 * q2, a);
+                tmem_ld_row16(tacc + HC * set + 16 * g, a);
 #pragma unroll
                 for (int qq = 0; qq < 2; ++qq) {
                     uint32_t ow[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
                         ow[e] = pack_bf16(tanh_fast(a[8 * qq + 2 * e]), tanh_fast(a[8 * qq + 2 * e + 1]));
-                    sts128(h_rows + swz(own_row, (4 * set + 2 * q2 + qq) << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                    sts128(h_row + ((uint32_t)((HC / 8 * set + 2 * g + qq) << 4) ^ own_xor), make_uint4(ow[0], ow[1], ow[2], ow[3]));
                 }
             }
         };
 
         int it = 0;
-        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
             const long long tok = t * 128 + row;
             // ---- passes 1 and 2
             for (int pass = 0; pass < 2 && alive; ++pass) {
                 for (int s = 0; s < S; ++s, ++it) {
-                    if ((s & 1) != set) continue;
+                    if (s % DL_NSET != set) continue;
                     const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
                     if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
                     if (pass == 1) {
@@ -344,15 +392,13 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                         ++acc_uses;
                         tc_fence_after();
                     }
-                    // the operand rows: free of the product that read them last, and of this warp's own output store
+                    // the operand rows: free of the product that read them last (and of this warp's own output store)
                     if (op_uses >= 1 && !mbar_wait(bar(DL_OP_FREE + set), (op_uses - 1) & 1, abort_flag)) { alive = false; break; }
                     ++op_uses;
                     mix_slice(stage, tok, s, pass == 1, tmem + tlane + DL_TM_L + 64 * set);
                     fence_proxy_async();
-                    if (pass == 1) tc_fence_before();
                     __syncwarp();
                     mbar_arrive_if(bar(DL_OP_READY + set), lane == 0);
-                    if (pass == 1) mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
                     mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
                 }
                 if (!alive) break;
@@ -368,7 +414,7 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (!alive) break;
             // ---- pass 3: d slice -> bf16 slab -> TMA store
             for (int s = 0; s < S; ++s, ++it) {
-                if ((s & 1) != set) continue;
+                if (s % DL_NSET != set) continue;
                 const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
                 if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
                 if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
@@ -377,30 +423,30 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 if (lane == 0) bulk_wait_read<0>();      // this warp's previous store has finished reading the slab
                 __syncwarp();
 #pragma unroll
-                for (int q2 = 0; q2 < 4; ++q2) {
-                    float a[16];
-                    tmem_ld_row16(tmem + tlane + DL_TM_D + 64 * set + 16 * q2, a);
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t a[32];
+                    kc::tmem_ld_row32(tmem + tlane + DL_TM_D + 64 * set + 32 * half, a);
+                    if (half == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                    }
 #pragma unroll
-                    for (int qq = 0; qq < 2; ++qq) {
-                        const int q = 2 * q2 + qq;
-                        const float4 v0 = ldsf4(stage + DL_OFF_VEC + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 32 * q + 16);
-                        const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-                        uint32_t ow[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            ow[e] = pack_bf16(a[8 * qq + 2 * e] + vv[2 * e], a[8 * qq + 2 * e + 1] + vv[2 * e + 1]);
-                        sts128(slab + swz(lane, q << 4), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 v0 = ldsf4(stage + DL_OFF_VEC + 128 * half + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 128 * half + 32 * q + 16);
+                        const float* f = reinterpret_cast<const float*>(a) + 8 * q;
+                        sts128(slab + swz(lane, (4 * half + q) << 4),
+                               make_uint4(pack_bf16(f[0] + v0.x, f[1] + v0.y), pack_bf16(f[2] + v0.z, f[3] + v0.w),
+                                          pack_bf16(f[4] + v1.x, f[5] + v1.y), pack_bf16(f[6] + v1.z, f[7] + v1.w)));
                     }
                 }
                 fence_proxy_async();
-                tc_fence_before();
                 __syncwarp();
                 const long long grow = t * 128 + 32 * sp;
                 if (lane == 0 && grow < p.rows) {
                     tma_store_2d(&tm_d32, 64 * s, (int)grow, slab);
                     bulk_commit();
                 }
-                mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
                 mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
             }
             // the slab doubles as this warp's operand rows of the next tile
