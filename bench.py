@@ -37,7 +37,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # proportion to the tokens and are scaled to the timed launch; the writes of the capture miss the part of y
 # that is still in L2 when the kernel ends (a fixed amount), so for the timed launch they are only bounded:
 # at least the scaled figure, at most the algorithmic y + state bytes.
-NCU_CAPTURE = None
+NCU_CAPTURE = {"profile": "profiles/ncu_wkv6_chunked_kernel_B4_T4096_H32.txt", "token_heads": 4 * 4096 * 32,
+               "read_bytes": 268504832, "write_bytes": 50730496}
 
 
 def parse():
