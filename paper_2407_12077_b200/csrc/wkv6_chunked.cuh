@@ -647,6 +647,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     auto bar = [&](int i) { return sbase + OFF_BAR + 8 * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // first pass of a split call: the second launch (enqueued with programmatic stream serialisation) may set up and
+    // fill its rings while this one runs; its state warps wait for this grid's results before they read them
+    if (SUMMARY) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int gsegs = SUMMARY ? p.nseg - 1 : p.nseg;      // segments per unit that this launch covers
     const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs;
     const int seq = unit / p.H, h = unit % p.H;
@@ -937,6 +940,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 *reinterpret_cast<float2*>(p.state_out + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
             }
         };
+        // second launch of a split call: the summaries and the start-state copy are the first launch's
+        if (!SUMMARY && !PERSIST && p.nseg > 1) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!PERSIST) load_state(sb);
         if (!SUMMARY) {
             // start state of a later segment: fold the summaries of the segments before it, in order
@@ -1605,6 +1610,23 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    }
+    if (nseg > 1) {
+        // behind the summary launch: may start before it has finished (see the top of the kernel)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(units * nseg));
+        cfg.blockDim = dim3(ck::THREADS);
+        cfg.dynamicSmemBytes = ck::SMEM_ALLOC;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = c2 ? cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, true, false>, tr, tk, tv, tx, ty, tu2, p)
+                                 : cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, false, false>, tr, tk, tv, tx, ty, tu2, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }
     if (c2) ck::wkv6_chunked_kernel<false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
     else ck::wkv6_chunked_kernel<false, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
