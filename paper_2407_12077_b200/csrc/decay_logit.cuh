@@ -15,13 +15,14 @@
 //   pass 2: l = h1 B_d[:, slice] -> tensor memory -> m slice -> bf16 operand tile -> acc3 += m A_w[slice]
 //           then h2 = tanh(acc3) -> operand tile
 //   pass 3: d slice = lambda_w + h2 B_w[:, slice] -> bf16 -> TMA store
-//   warp 0      TMA producer: per slice the x rows of the tile (plus the one row before it), the weight tiles and
-//               the 64 per-channel constants of the pass into a 5-stage ring
-//   warp 1      tensor-memory allocation; an elected lane issues the products whose operands come from the ring and
-//               the h tile (z A_d, h1 B_d, h2 B_w; tcgen05.mma 128 x 64 x 16, bf16 -> fp32)
+//   warp 0      TMA producer of the x ring (5 stages): per slice the x rows of the tile (plus the one row above it)
+//               and the 64 per-channel constants of the pass; a stage is free as soon as its rows are in registers
+//   warp 3      TMA producer of the weight ring (5 stages): the slice's weight tiles, free when their products are done
+//   warp 1      tensor-memory allocation; an elected lane issues the products whose operands come from the weight
+//               ring and the h tile (z A_d, h1 B_d, h2 B_w; tcgen05.mma 128 x 64 x 16, bf16 -> fp32)
 //   warp 2      an elected lane issues m A_w, the product that waits for the workers inside pass 2 (an issuer of
 //               its own, so that the l products of later slices are not held up behind it)
-//   warps 3-10  two sets of four warps taking alternate slices; a lane owns one token row (the accumulator row
+//   warps 4-11  two sets of four warps taking alternate slices; a lane owns one token row (the accumulator row
 //               of its tensor-memory sub-partition): reads its row and the row above from the swizzled x tiles,
 //               forms z / m / d for the 64 channels of the slice, writes the bf16 operand row (or the output slab)
 // All operand tiles are the 128-byte-swizzled [64 rows][64 bf16] tiles of the prefill kernel; weight tiles narrower
@@ -36,21 +37,28 @@ namespace dl {
 using namespace ck;
 
 constexpr int DL_NSET = 2;                             // worker sets
-constexpr int DL_W0 = 3;                               // first worker warp
+constexpr int DL_W0 = 4;                               // first worker warp
 constexpr int DL_THREADS = 32 * (DL_W0 + 4 * DL_NSET);
-constexpr int DL_NS = 5;                               // ring stages: three more than worker sets, so that a slice's loads are
-                                                       // issued about a load latency before its set turns to it
-constexpr int DL_STAGE = 4 * TILE + 1024;              // x rows 0-63, x rows 64-127, two weight tiles; row above + constants
-constexpr int DL_OFF_PREV = 4 * TILE;                  // [64] bf16: the x row just above the tile (this slice)
-constexpr int DL_OFF_VEC = 4 * TILE + 256;             // [64] fp32: mu_x / lambda_d / lambda_w of this slice
-constexpr int DL_OFF_OP = DL_NS * DL_STAGE;            // [sets][128 rows x 128 B]: z / m operand, output slabs in pass 3
+// Two rings.  The x ring holds, per slice, the tile's x rows (two swizzled 64-row tiles), the row above the tile and the
+// pass's 64 per-channel constants; a worker set frees its stage as soon as the rows are in registers, so that ring
+// runs a load latency ahead of the arithmetic.  The weight ring holds up to two weight tiles per slice and is freed
+// by the products that read them (weights come from L2).
+constexpr int DL_NSX = 5, DL_NSW = 5;
+constexpr int DL_XSTAGE = 2 * TILE + 1024;
+constexpr int DL_OFF_PREV = 2 * TILE;                  // [64] bf16: the x row just above the tile (this slice)
+constexpr int DL_OFF_VEC = 2 * TILE + 256;             // [64] fp32: mu_x / lambda_d / lambda_w of this slice
+constexpr int DL_WSTAGE = 2 * TILE;
+constexpr int DL_OFF_W = DL_NSX * DL_XSTAGE;           // weight ring
+constexpr int DL_OFF_OP = DL_OFF_W + DL_NSW * DL_WSTAGE;         // [sets][128 rows x 128 B]: z / m operand, output slabs in pass 3
 constexpr int DL_OFF_H = DL_OFF_OP + DL_NSET * 2 * TILE;         // [128 rows x 128 B]: h1 / h2 operand
 constexpr int DL_OFF_MISC = DL_OFF_H + 2 * TILE;       // abort word + limit, tensor-memory address, barriers
-constexpr int DL_SMEM = DL_OFF_MISC + 256 + 1024;      // + slack for manual 1024-byte alignment
+constexpr int DL_SMEM = DL_OFF_MISC + 512 + 1024;      // + slack for manual 1024-byte alignment
 enum {
-    DL_FULL = 0,                       // ring stage loaded
-    DL_EMPTY = DL_FULL + DL_NS,        // ... and consumed (four worker warps + the products that read it)
-    DL_OP_READY = DL_EMPTY + DL_NS,    // per set: operand rows written
+    DL_XFULL = 0,                      // x stage loaded
+    DL_XEMPTY = DL_XFULL + DL_NSX,     // ... and read into registers by the four warps of its set
+    DL_WFULL = DL_XEMPTY + DL_NSX,     // weight stage loaded
+    DL_WEMPTY = DL_WFULL + DL_NSW,     // ... and the last product that reads it is done
+    DL_OP_READY = DL_WEMPTY + DL_NSW,  // per set: operand rows written
     DL_OP_FREE = DL_OP_READY + DL_NSET,    // per set: the product that read them is done
     DL_ACC_FULL = DL_OP_FREE + DL_NSET,    // per set: l (pass 2) or d (pass 3) of a slice is in tensor memory
     DL_ACC_FREE = DL_ACC_FULL + DL_NSET,   // per set: ... and read back
@@ -59,7 +67,7 @@ enum {
     DL_PASS2 = DL_H_READY + 1,         // pass 2 of a tile has begun (first issuer -> second issuer: one phase per tile)
     DL_BAR_COUNT = DL_PASS2 + 1
 };
-static_assert(16 + 8 * DL_BAR_COUNT <= 256, "barrier block");
+static_assert(16 + 8 * DL_BAR_COUNT <= 512, "barrier block");
 static_assert(DL_SMEM <= 232448, "shared memory budget of one sm_100 CTA");
 constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_L = 128, DL_TM_D = 128;       // + 64 * set for the last two (one region:
                                                                                   // l in pass 2, d in pass 3)
@@ -125,9 +133,13 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const int S = p.nslices;
 
     if (tid == 0) {
-        for (int i = 0; i < DL_NS; ++i) {
-            mbar_init(bar(DL_FULL + i), 1);
-            mbar_init(bar(DL_EMPTY + i), 5);              // four worker warps and one commit
+        for (int i = 0; i < DL_NSX; ++i) {
+            mbar_init(bar(DL_XFULL + i), 1);
+            mbar_init(bar(DL_XEMPTY + i), 4);
+        }
+        for (int i = 0; i < DL_NSW; ++i) {
+            mbar_init(bar(DL_WFULL + i), 1);
+            mbar_init(bar(DL_WEMPTY + i), 1);
         }
         for (int i = 0; i < DL_NSET; ++i) {
             mbar_init(bar(DL_OP_READY + i), 4);
@@ -148,67 +160,88 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = lds32(sbase + DL_OFF_MISC + 8);
+    auto wstage = [&](int i) { return sbase + DL_OFF_W + (i % DL_NSW) * DL_WSTAGE; };
 
     if (warp == 0) {
-        // ============================== TMA producer ==============================
+        // ============================== TMA producer: x rows and per-channel constants ==============================
         int it = 0, issued = 0;
         bool alive = true;
         for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
             const int row0 = (int)(t * 128);
             for (int pass = 0; pass < 3 && alive; ++pass)
                 for (int s = 0; s < S; ++s, ++it) {
-                    const int st = it % DL_NS;
-                    if (it >= DL_NS && !mbar_wait_warp(bar(DL_EMPTY + st), ((it / DL_NS) + 1) & 1, abort_flag)) { alive = false; break; }
-                    const uint32_t dst = sbase + st * DL_STAGE, full = bar(DL_FULL + st);
+                    const int st = it % DL_NSX;
+                    if (it >= DL_NSX && !mbar_wait_warp(bar(DL_XEMPTY + st), ((it / DL_NSX) + 1) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t dst = sbase + st * DL_XSTAGE, full = bar(DL_XFULL + st);
                     if (elect_one()) {
+                        const float* vec = pass == 0 ? p.mu_x : pass == 1 ? p.lambda_d : p.lambda_w;
                         if (pass < 2) {
-                            mbar_expect_tx(full, (pass == 0 ? 3 : 4) * TILE + 128 + 256);
+                            mbar_expect_tx(full, 2 * TILE + 128 + 256);
                             tma_load_2d(dst, &tm_x, 64 * s, row0, full);
                             tma_load_2d(dst + TILE, &tm_x, 64 * s, row0 + 64, full);
                             tma_load_2d(dst + DL_OFF_PREV, &tm_x1, 64 * s, row0 - 1, full);      // (row -1 reads as zero)
-                            if (pass == 0) {
-                                tma_load_2d(dst + 2 * TILE, &tm_ad, 0, 64 * s, full);
-                                bulk_load_1d(dst + DL_OFF_VEC, p.mu_x + 64 * s, 256, full);
-                            } else {
-                                tma_load_2d(dst + 2 * TILE, &tm_bd, 64 * s, 0, full);
-                                tma_load_2d(dst + 3 * TILE, &tm_aw, 0, 64 * s, full);
-                                bulk_load_1d(dst + DL_OFF_VEC, p.lambda_d + 64 * s, 256, full);
-                            }
                         } else {
-                            mbar_expect_tx(full, TILE + 256);
-                            tma_load_2d(dst + 2 * TILE, &tm_bw, 64 * s, 0, full);
-                            bulk_load_1d(dst + DL_OFF_VEC, p.lambda_w + 64 * s, 256, full);
+                            mbar_expect_tx(full, 256);
                         }
+                        bulk_load_1d(dst + DL_OFF_VEC, vec + 64 * s, 256, full);
                     }
                     __syncwarp();
                     issued = it + 1;
                 }
         }
         // do not leave while copies into this CTA's shared memory may still be in flight
-        for (int c = max(0, issued - DL_NS); c < issued; ++c)
-            mbar_wait_warp(bar(DL_FULL + c % DL_NS), (c / DL_NS) & 1, abort_flag, false);
+        for (int c = max(0, issued - DL_NSX); c < issued; ++c)
+            mbar_wait_warp(bar(DL_XFULL + c % DL_NSX), (c / DL_NSX) & 1, abort_flag, false);
+    } else if (warp == 3) {
+        // ============================== TMA producer: weight tiles ==============================
+        int it = 0, issued = 0;
+        bool alive = true;
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x)
+            for (int pass = 0; pass < 3 && alive; ++pass)
+                for (int s = 0; s < S; ++s, ++it) {
+                    const int st = it % DL_NSW;
+                    if (it >= DL_NSW && !mbar_wait_warp(bar(DL_WEMPTY + st), ((it / DL_NSW) + 1) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t dst = wstage(it), full = bar(DL_WFULL + st);
+                    if (elect_one()) {
+                        if (pass == 0) {
+                            mbar_expect_tx(full, TILE);
+                            tma_load_2d(dst, &tm_ad, 0, 64 * s, full);
+                        } else if (pass == 1) {
+                            mbar_expect_tx(full, 2 * TILE);
+                            tma_load_2d(dst, &tm_bd, 64 * s, 0, full);
+                            tma_load_2d(dst + TILE, &tm_aw, 0, 64 * s, full);
+                        } else {
+                            mbar_expect_tx(full, TILE);
+                            tma_load_2d(dst, &tm_bw, 64 * s, 0, full);
+                        }
+                    }
+                    __syncwarp();
+                    issued = it + 1;
+                }
+        for (int c = max(0, issued - DL_NSW); c < issued; ++c)
+            mbar_wait_warp(bar(DL_WFULL + c % DL_NSW), (c / DL_NSW) & 1, abort_flag, false);
     } else if (warp == 1) {
         // ============================== MMA issuer: z A_d, h1 B_d, h2 B_w ==============================
         int it = 0;
         int op_uses[DL_NSET] = {}, acc_uses[DL_NSET] = {};   // per set: operand tiles consumed, l / d accumulators produced
         bool alive = true;
-        auto stage_full = [&](int i) { return mbar_wait_warp(bar(DL_FULL + i % DL_NS), (i / DL_NS) & 1, abort_flag); };
+        auto weights_in = [&](int i) { return mbar_wait_warp(bar(DL_WFULL + i % DL_NSW), (i / DL_NSW) & 1, abort_flag); };
         const uint64_t dh = smem_desc(sbase + DL_OFF_H);
         for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
             // ---- pass 1: acc1 += z A_d[slice]
             for (int s = 0; s < S; ++s, ++it) {
                 const int h = s % DL_NSET;
-                if (!stage_full(it) || !mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
+                if (!weights_in(it) || !mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
                 ++op_uses[h];
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
-                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+                    const uint64_t db = smem_desc(wstage(it));
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         tc_mma(tmem + DL_TM_ACC1, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (s > 0 || kk > 0) ? 1u : 0u);
                     tc_commit(bar(DL_OP_FREE + h));
-                    tc_commit(bar(DL_EMPTY + it % DL_NS));
+                    tc_commit(bar(DL_WEMPTY + it % DL_NSW));
                     if (s == S - 1) tc_commit(bar(DL_SUM_FULL));
                 }
                 __syncwarp();
@@ -221,13 +254,13 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             __syncwarp();
             for (int s = 0; s < S; ++s, ++it) {
                 const int h = s % DL_NSET;
-                if (!stage_full(it)) { alive = false; break; }
+                if (!weights_in(it)) { alive = false; break; }
                 if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
                 ++acc_uses[h];
                 ++op_uses[h];                                 // (the other issuer consumes this slice's operand rows)
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+                    const uint64_t db = smem_desc(wstage(it));
                     for (int kk = 0; kk < p.kd; ++kk)
                         tc_mma(tmem + DL_TM_L + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
                     tc_commit(bar(DL_ACC_FULL + h));
@@ -240,16 +273,16 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             tc_fence_after();
             for (int s = 0; s < S; ++s, ++it) {
                 const int h = s % DL_NSET;
-                if (!stage_full(it)) { alive = false; break; }
+                if (!weights_in(it)) { alive = false; break; }
                 if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
                 ++acc_uses[h];
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint64_t db = smem_desc(sbase + (it % DL_NS) * DL_STAGE + 2 * TILE);
+                    const uint64_t db = smem_desc(wstage(it));
                     for (int kk = 0; kk < p.kw; ++kk)
                         tc_mma(tmem + DL_TM_D + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
                     tc_commit(bar(DL_ACC_FULL + h));
-                    tc_commit(bar(DL_EMPTY + it % DL_NS));
+                    tc_commit(bar(DL_WEMPTY + it % DL_NSW));
                 }
                 __syncwarp();
             }
@@ -267,18 +300,19 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             const int it2 = ti * 3 * S + S;                               // ring position of pass 2, slice 0
             for (int s = 0; s < S; ++s) {
                 const int h = s % DL_NSET, i = it2 + s;
-                // the operand rows are written after the stage was seen full, so the weight tile is in place as well
                 if (!mbar_wait_warp(bar(DL_OP_READY + h), op_uses[h] & 1, abort_flag)) { alive = false; break; }
                 ++op_uses[h];
+                // (complete by now: the other issuer saw this stage full before it made the l this operand was built from)
+                if (!mbar_wait_warp(bar(DL_WFULL + i % DL_NSW), (i / DL_NSW) & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t da = smem_desc(sbase + DL_OFF_OP + h * 2 * TILE);
-                    const uint64_t db = smem_desc(sbase + (i % DL_NS) * DL_STAGE + 3 * TILE);
+                    const uint64_t db = smem_desc(wstage(i) + TILE);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         tc_mma(tmem + DL_TM_ACC3, da + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, (s > 0 || kk > 0) ? 1u : 0u);
                     tc_commit(bar(DL_OP_FREE + h));
-                    tc_commit(bar(DL_EMPTY + i % DL_NS));
+                    tc_commit(bar(DL_WEMPTY + i % DL_NSW));
                     if (s == S - 1) tc_commit(bar(DL_SUM_FULL));
                 }
                 __syncwarp();
@@ -299,67 +333,6 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         int op_uses = 0, acc_uses = 0;
         bool alive = true;
 
-        // z or m for the 64 channels of one slice: out = x + (x_above - x) * mix, mix = vec (+ l from tensor memory).
-        // The interpolation itself runs on packed bf16 pairs (difference, then one fused multiply-add with a single
-        // rounding): its inputs and its output are bf16 anyway, and the mix is smooth in them.  32 channels at a time.
-        auto mix_slice = [&](uint32_t stage, long long tok, int s, bool with_l, uint32_t tl) {
-            const bool seq_start = (tok % p.T) == 0;     // the row above belongs to another sequence: x_prev or zero
-            // the row above: inside the tiles, or (first row of the tile) the extra row of the stage
-            const uint32_t up_base = row == 0 ? stage + DL_OFF_PREV : stage + up_tile + up_row * 128;
-            const uint32_t up_xor = row == 0 ? 0u : (up_row & 7) << 4;
-            const uint32_t own_base = stage + own_tile + own_row * 128;
-            const bool any_start = __any_sync(0xffffffffu, seq_start);
-            const __nv_bfloat16* gp = (seq_start && p.x_prev && tok < p.rows) ? p.x_prev + (tok / p.T) * (long long)p.D + 64 * s : nullptr;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t mixw[16];                       // the mix of 32 channels as bf16 pairs
-                if (with_l) {
-                    uint32_t l[32];
-                    kc::tmem_ld_row32(tl + 32 * half, l);
-                    if (half == 1) {                     // the accumulator row has been read: hand it back
-                        tc_fence_before();
-                        __syncwarp();
-                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
-                    }
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
-                        mixw[2 * q] = pack_bf16(v4.x + __uint_as_float(l[4 * q]), v4.y + __uint_as_float(l[4 * q + 1]));
-                        mixw[2 * q + 1] = pack_bf16(v4.z + __uint_as_float(l[4 * q + 2]), v4.w + __uint_as_float(l[4 * q + 3]));
-                    }
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
-                        mixw[2 * q] = pack_bf16(v4.x, v4.y);
-                        mixw[2 * q + 1] = pack_bf16(v4.z, v4.w);
-                    }
-                }
-                uint4 a[4], b[4];                        // this lane's row and the row above: all loads first
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    a[q] = lds128(own_base + ((uint32_t)((4 * half + q) << 4) ^ own_xor));
-                    b[q] = lds128(up_base + ((uint32_t)((4 * half + q) << 4) ^ up_xor));
-                }
-                if (any_start && seq_start) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        b[q] = gp ? *reinterpret_cast<const uint4*>(gp + 8 * (4 * half + q)) : make_uint4(0u, 0u, 0u, 0u);
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t aw[4] = {a[q].x, a[q].y, a[q].z, a[q].w}, bw[4] = {b[q].x, b[q].y, b[q].z, b[q].w};
-                    uint32_t ow[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        uint32_t delta;
-                        asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(delta) : "r"(bw[e]), "r"(aw[e]));
-                        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(ow[e]) : "r"(delta), "r"(mixw[4 * q + e]), "r"(aw[e]));
-                    }
-                    sts128(out_base + ((uint32_t)((4 * half + q) << 4) ^ own_xor), make_uint4(ow[0], ow[1], ow[2], ow[3]));
-                }
-            }
-        };
         // h = tanh(acc) for this warp's 32 rows and this set's share of the 64 columns -> bf16 operand rows
         auto squash = [&](uint32_t tacc) {
             constexpr int HC = 64 / DL_NSET;             // columns per set
@@ -381,25 +354,80 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         int it = 0;
         for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
             const long long tok = t * 128 + row;
-            // ---- passes 1 and 2
+            const bool seq_start = (tok % p.T) == 0;     // the row above belongs to another sequence: x_prev or zero
+            const bool any_start = __any_sync(0xffffffffu, seq_start);
+            const __nv_bfloat16* gp0 = (seq_start && p.x_prev && tok < p.rows) ? p.x_prev + (tok / p.T) * (long long)p.D : nullptr;
+            // ---- passes 1 and 2: out = x + (x_above - x) * mix, mix = the pass's constants (+ l from tensor memory in pass 2).
+            // The interpolation runs on packed bf16 pairs (difference, then one fused multiply-add with a single rounding):
+            // its inputs and its output are bf16 anyway, and the mix is smooth in them.
             for (int pass = 0; pass < 2 && alive; ++pass) {
                 for (int s = 0; s < S; ++s, ++it) {
                     if (s % DL_NSET != set) continue;
-                    const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
-                    if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
+                    const uint32_t stage = sbase + (it % DL_NSX) * DL_XSTAGE;
+                    if (!mbar_wait(bar(DL_XFULL + it % DL_NSX), (it / DL_NSX) & 1, abort_flag)) { alive = false; break; }
+                    uint32_t mixw[32];                   // the mix of the 64 channels as bf16 pairs
                     if (pass == 1) {
                         if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
                         ++acc_uses;
                         tc_fence_after();
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t l[32];
+                            kc::tmem_ld_row32(tmem + tlane + DL_TM_L + 64 * set + 32 * half, l);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
+                                mixw[16 * half + 2 * q] = pack_bf16(v4.x + __uint_as_float(l[4 * q]), v4.y + __uint_as_float(l[4 * q + 1]));
+                                mixw[16 * half + 2 * q + 1] = pack_bf16(v4.z + __uint_as_float(l[4 * q + 2]), v4.w + __uint_as_float(l[4 * q + 3]));
+                            }
+                        }
+                        tc_fence_before();               // the accumulator row has been read: hand it back
+                        __syncwarp();
+                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            const float4 v4 = ldsf4(stage + DL_OFF_VEC + 16 * q);
+                            mixw[2 * q] = pack_bf16(v4.x, v4.y);
+                            mixw[2 * q + 1] = pack_bf16(v4.z, v4.w);
+                        }
+                    }
+                    // this lane's row and the row above it (inside the tiles, or the extra row of the stage for the tile's
+                    // first row), all into registers; then the stage is free for a later slice
+                    const uint32_t up_base = row == 0 ? stage + DL_OFF_PREV : stage + up_tile + up_row * 128;
+                    const uint32_t up_xor = row == 0 ? 0u : (up_row & 7) << 4;
+                    const uint32_t own_base = stage + own_tile + own_row * 128;
+                    uint4 a[8], b[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        a[q] = lds128(own_base + ((uint32_t)(q << 4) ^ own_xor));
+                        b[q] = lds128(up_base + ((uint32_t)(q << 4) ^ up_xor));
+                    }
+                    __syncwarp();
+                    mbar_arrive_if(bar(DL_XEMPTY + it % DL_NSX), lane == 0);
+                    if (any_start && seq_start) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            b[q] = gp0 ? *reinterpret_cast<const uint4*>(gp0 + 64 * s + 8 * q) : make_uint4(0u, 0u, 0u, 0u);
                     }
                     // the operand rows: free of the product that read them last (and of this warp's own output store)
                     if (op_uses >= 1 && !mbar_wait(bar(DL_OP_FREE + set), (op_uses - 1) & 1, abort_flag)) { alive = false; break; }
                     ++op_uses;
-                    mix_slice(stage, tok, s, pass == 1, tmem + tlane + DL_TM_L + 64 * set);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const uint32_t aw[4] = {a[q].x, a[q].y, a[q].z, a[q].w}, bw[4] = {b[q].x, b[q].y, b[q].z, b[q].w};
+                        uint32_t ow[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            uint32_t delta;
+                            asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(delta) : "r"(bw[e]), "r"(aw[e]));
+                            asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(ow[e]) : "r"(delta), "r"(mixw[4 * q + e]), "r"(aw[e]));
+                        }
+                        sts128(out_base + ((uint32_t)(q << 4) ^ own_xor), make_uint4(ow[0], ow[1], ow[2], ow[3]));
+                    }
                     fence_proxy_async();
                     __syncwarp();
                     mbar_arrive_if(bar(DL_OP_READY + set), lane == 0);
-                    mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
                 }
                 if (!alive) break;
                 // the pass's low-rank sum is complete: squash it into the operand of the next product
@@ -415,8 +443,16 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             // ---- pass 3: d slice -> bf16 slab -> TMA store
             for (int s = 0; s < S; ++s, ++it) {
                 if (s % DL_NSET != set) continue;
-                const uint32_t stage = sbase + (it % DL_NS) * DL_STAGE;
-                if (!mbar_wait(bar(DL_FULL + it % DL_NS), (it / DL_NS) & 1, abort_flag)) { alive = false; break; }
+                const uint32_t stage = sbase + (it % DL_NSX) * DL_XSTAGE;
+                if (!mbar_wait(bar(DL_XFULL + it % DL_NSX), (it / DL_NSX) & 1, abort_flag)) { alive = false; break; }
+                float lam[64];                           // lambda_w of the slice; then its stage is free
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const float4 v4 = ldsf4(stage + DL_OFF_VEC + 16 * q);
+                    lam[4 * q] = v4.x; lam[4 * q + 1] = v4.y; lam[4 * q + 2] = v4.z; lam[4 * q + 3] = v4.w;
+                }
+                __syncwarp();
+                mbar_arrive_if(bar(DL_XEMPTY + it % DL_NSX), lane == 0);
                 if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
                 ++acc_uses;
                 tc_fence_after();
@@ -433,11 +469,12 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        const float4 v0 = ldsf4(stage + DL_OFF_VEC + 128 * half + 32 * q), v1 = ldsf4(stage + DL_OFF_VEC + 128 * half + 32 * q + 16);
-                        const float* f = reinterpret_cast<const float*>(a) + 8 * q;
+                        const float* lm = lam + 32 * half + 8 * q;
                         sts128(slab + swz(lane, (4 * half + q) << 4),
-                               make_uint4(pack_bf16(f[0] + v0.x, f[1] + v0.y), pack_bf16(f[2] + v0.z, f[3] + v0.w),
-                                          pack_bf16(f[4] + v1.x, f[5] + v1.y), pack_bf16(f[6] + v1.z, f[7] + v1.w)));
+                               make_uint4(pack_bf16(__uint_as_float(a[8 * q]) + lm[0], __uint_as_float(a[8 * q + 1]) + lm[1]),
+                                          pack_bf16(__uint_as_float(a[8 * q + 2]) + lm[2], __uint_as_float(a[8 * q + 3]) + lm[3]),
+                                          pack_bf16(__uint_as_float(a[8 * q + 4]) + lm[4], __uint_as_float(a[8 * q + 5]) + lm[5]),
+                                          pack_bf16(__uint_as_float(a[8 * q + 6]) + lm[6], __uint_as_float(a[8 * q + 7]) + lm[7])));
                     }
                 }
                 fence_proxy_async();
@@ -447,7 +484,6 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     tma_store_2d(&tm_d32, 64 * s, (int)grow, slab);
                     bulk_commit();
                 }
-                mbar_arrive_if(bar(DL_EMPTY + it % DL_NS), lane == 0);
             }
             // the slab doubles as this warp's operand rows of the next tile
             if (lane == 0) bulk_wait_read<0>();
