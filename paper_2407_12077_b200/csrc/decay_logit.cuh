@@ -44,6 +44,8 @@ constexpr int DL_THREADS = 32 * (DL_W0 + 4 * DL_NSET);
 // runs a load latency ahead of the arithmetic.  The weight ring holds up to two weight tiles per slice and is freed
 // by the products that read them (weights come from L2).
 constexpr int DL_NSX = 5, DL_NSW = 5;
+constexpr int DL_NACC = 6;                             // l / d accumulators in tensor memory: the products h1 B_d and h2 B_w depend on
+                                                       // nothing the workers make, so they run this many slices ahead of them
 constexpr int DL_XSTAGE = 2 * TILE + 1024;
 constexpr int DL_OFF_PREV = 2 * TILE;                  // [64] bf16: the x row just above the tile (this slice)
 constexpr int DL_OFF_VEC = 2 * TILE + 256;             // [64] fp32: mu_x / lambda_d / lambda_w of this slice
@@ -60,17 +62,17 @@ enum {
     DL_WEMPTY = DL_WFULL + DL_NSW,     // ... and the last product that reads it is done
     DL_OP_READY = DL_WEMPTY + DL_NSW,  // per set: operand rows written
     DL_OP_FREE = DL_OP_READY + DL_NSET,    // per set: the product that read them is done
-    DL_ACC_FULL = DL_OP_FREE + DL_NSET,    // per set: l (pass 2) or d (pass 3) of a slice is in tensor memory
-    DL_ACC_FREE = DL_ACC_FULL + DL_NSET,   // per set: ... and read back
-    DL_SUM_FULL = DL_ACC_FREE + DL_NSET,   // acc1 / acc3 complete
+    DL_ACC_FULL = DL_OP_FREE + DL_NSET,    // per accumulator: l (pass 2) or d (pass 3) of a slice is in tensor memory
+    DL_ACC_FREE = DL_ACC_FULL + DL_NACC,   // ... and read back by the four warps of the slice's set
+    DL_SUM_FULL = DL_ACC_FREE + DL_NACC,   // acc1 / acc3 complete
     DL_H_READY = DL_SUM_FULL + 1,      // h1 / h2 operand written by all worker warps
     DL_PASS2 = DL_H_READY + 1,         // pass 2 of a tile has begun (first issuer -> second issuer: one phase per tile)
     DL_BAR_COUNT = DL_PASS2 + 1
 };
 static_assert(16 + 8 * DL_BAR_COUNT <= 512, "barrier block");
 static_assert(DL_SMEM <= 232448, "shared memory budget of one sm_100 CTA");
-constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_L = 128, DL_TM_D = 128;       // + 64 * set for the last two (one region:
-                                                                                  // l in pass 2, d in pass 3)
+constexpr int DL_TM_ACC1 = 0, DL_TM_ACC3 = 64, DL_TM_RING = 128;       // + 64 * accumulator (l in pass 2, d in pass 3)
+static_assert(DL_TM_RING + 64 * DL_NACC <= 512, "tensor memory columns");
 // fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = 64
 constexpr uint32_t DL_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 
@@ -144,6 +146,8 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         for (int i = 0; i < DL_NSET; ++i) {
             mbar_init(bar(DL_OP_READY + i), 4);
             mbar_init(bar(DL_OP_FREE + i), 1);
+        }
+        for (int i = 0; i < DL_NACC; ++i) {
             mbar_init(bar(DL_ACC_FULL + i), 1);
             mbar_init(bar(DL_ACC_FREE + i), 4);
         }
@@ -223,7 +227,8 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     } else if (warp == 1) {
         // ============================== MMA issuer: z A_d, h1 B_d, h2 B_w ==============================
         int it = 0;
-        int op_uses[DL_NSET] = {}, acc_uses[DL_NSET] = {};   // per set: operand tiles consumed, l / d accumulators produced
+        int op_uses[DL_NSET] = {};                           // per set: operand tiles consumed
+        int an = 0;                                          // l / d accumulators produced so far (their ring position)
         bool alive = true;
         auto weights_in = [&](int i) { return mbar_wait_warp(bar(DL_WFULL + i % DL_NSW), (i / DL_NSW) & 1, abort_flag); };
         const uint64_t dh = smem_desc(sbase + DL_OFF_H);
@@ -255,15 +260,16 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             for (int s = 0; s < S; ++s, ++it) {
                 const int h = s % DL_NSET;
                 if (!weights_in(it)) { alive = false; break; }
-                if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
-                ++acc_uses[h];
+                const int a = an % DL_NACC;
+                if (an >= DL_NACC && !mbar_wait_warp(bar(DL_ACC_FREE + a), ((an / DL_NACC) + 1) & 1, abort_flag)) { alive = false; break; }
+                ++an;
                 ++op_uses[h];                                 // (the other issuer consumes this slice's operand rows)
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t db = smem_desc(wstage(it));
                     for (int kk = 0; kk < p.kd; ++kk)
-                        tc_mma(tmem + DL_TM_L + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
-                    tc_commit(bar(DL_ACC_FULL + h));
+                        tc_mma(tmem + DL_TM_RING + 64 * a, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
+                    tc_commit(bar(DL_ACC_FULL + a));
                 }
                 __syncwarp();
             }
@@ -272,16 +278,16 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (!mbar_wait_warp(bar(DL_H_READY), 1, abort_flag)) break;
             tc_fence_after();
             for (int s = 0; s < S; ++s, ++it) {
-                const int h = s % DL_NSET;
                 if (!weights_in(it)) { alive = false; break; }
-                if (acc_uses[h] >= 1 && !mbar_wait_warp(bar(DL_ACC_FREE + h), (acc_uses[h] - 1) & 1, abort_flag)) { alive = false; break; }
-                ++acc_uses[h];
+                const int a = an % DL_NACC;
+                if (an >= DL_NACC && !mbar_wait_warp(bar(DL_ACC_FREE + a), ((an / DL_NACC) + 1) & 1, abort_flag)) { alive = false; break; }
+                ++an;
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t db = smem_desc(wstage(it));
                     for (int kk = 0; kk < p.kw; ++kk)
-                        tc_mma(tmem + DL_TM_D + 64 * h, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
-                    tc_commit(bar(DL_ACC_FULL + h));
+                        tc_mma(tmem + DL_TM_RING + 64 * a, dh + (uint64_t)(2 * kk), db + (uint64_t)(128 * kk), DL_IDESC, kk > 0 ? 1u : 0u);
+                    tc_commit(bar(DL_ACC_FULL + a));
                     tc_commit(bar(DL_WEMPTY + it % DL_NSW));
                 }
                 __syncwarp();
@@ -330,7 +336,7 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const uint32_t out_base = sbase + DL_OFF_OP + set * 2 * TILE + own_tile + own_row * 128;   // this lane's operand row
         const uint32_t slab = sbase + DL_OFF_OP + set * 2 * TILE + sp * 4096;       // pass 3: this warp's 32-row output slab
         const uint32_t h_row = sbase + DL_OFF_H + own_tile + own_row * 128;
-        int op_uses = 0, acc_uses = 0;
+        int op_uses = 0;
         bool alive = true;
 
         // h = tanh(acc) for this warp's 32 rows and this set's share of the 64 columns -> bf16 operand rows
@@ -351,8 +357,8 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             }
         };
 
-        int it = 0;
-        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x) {
+        int it = 0, ti = 0;
+        for (long long t = blockIdx.x; t < n_tiles && alive; t += gridDim.x, ++ti) {
             const long long tok = t * 128 + row;
             const bool seq_start = (tok % p.T) == 0;     // the row above belongs to another sequence: x_prev or zero
             const bool any_start = __any_sync(0xffffffffu, seq_start);
@@ -367,13 +373,13 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     if (!mbar_wait(bar(DL_XFULL + it % DL_NSX), (it / DL_NSX) & 1, abort_flag)) { alive = false; break; }
                     uint32_t mixw[32];                   // the mix of the 64 channels as bf16 pairs
                     if (pass == 1) {
-                        if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
-                        ++acc_uses;
+                        const int an = ti * 2 * S + s, a = an % DL_NACC;       // this slice's l: the an-th accumulator made
+                        if (!mbar_wait(bar(DL_ACC_FULL + a), (an / DL_NACC) & 1, abort_flag)) { alive = false; break; }
                         tc_fence_after();
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             uint32_t l[32];
-                            kc::tmem_ld_row32(tmem + tlane + DL_TM_L + 64 * set + 32 * half, l);
+                            kc::tmem_ld_row32(tmem + tlane + DL_TM_RING + 64 * a + 32 * half, l);
 #pragma unroll
                             for (int q = 0; q < 8; ++q) {
                                 const float4 v4 = ldsf4(stage + DL_OFF_VEC + 128 * half + 16 * q);
@@ -383,7 +389,7 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                         }
                         tc_fence_before();               // the accumulator row has been read: hand it back
                         __syncwarp();
-                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                        mbar_arrive_if(bar(DL_ACC_FREE + a), lane == 0);
                     } else {
 #pragma unroll
                         for (int q = 0; q < 16; ++q) {
@@ -453,28 +459,28 @@ decay_logit_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 }
                 __syncwarp();
                 mbar_arrive_if(bar(DL_XEMPTY + it % DL_NSX), lane == 0);
-                if (!mbar_wait(bar(DL_ACC_FULL + set), acc_uses & 1, abort_flag)) { alive = false; break; }
-                ++acc_uses;
+                const int an = ti * 2 * S + S + s, a = an % DL_NACC;          // this slice's d: the an-th accumulator made
+                if (!mbar_wait(bar(DL_ACC_FULL + a), (an / DL_NACC) & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
                 if (lane == 0) bulk_wait_read<0>();      // this warp's previous store has finished reading the slab
                 __syncwarp();
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    uint32_t a[32];
-                    kc::tmem_ld_row32(tmem + tlane + DL_TM_D + 64 * set + 32 * half, a);
+                    uint32_t acc[32];
+                    kc::tmem_ld_row32(tmem + tlane + DL_TM_RING + 64 * a + 32 * half, acc);
                     if (half == 1) {
                         tc_fence_before();
                         __syncwarp();
-                        mbar_arrive_if(bar(DL_ACC_FREE + set), lane == 0);
+                        mbar_arrive_if(bar(DL_ACC_FREE + a), lane == 0);
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const float* lm = lam + 32 * half + 8 * q;
                         sts128(slab + swz(lane, (4 * half + q) << 4),
-                               make_uint4(pack_bf16(__uint_as_float(a[8 * q]) + lm[0], __uint_as_float(a[8 * q + 1]) + lm[1]),
-                                          pack_bf16(__uint_as_float(a[8 * q + 2]) + lm[2], __uint_as_float(a[8 * q + 3]) + lm[3]),
-                                          pack_bf16(__uint_as_float(a[8 * q + 4]) + lm[4], __uint_as_float(a[8 * q + 5]) + lm[5]),
-                                          pack_bf16(__uint_as_float(a[8 * q + 6]) + lm[6], __uint_as_float(a[8 * q + 7]) + lm[7])));
+                               make_uint4(pack_bf16(__uint_as_float(acc[8 * q]) + lm[0], __uint_as_float(acc[8 * q + 1]) + lm[1]),
+                                          pack_bf16(__uint_as_float(acc[8 * q + 2]) + lm[2], __uint_as_float(acc[8 * q + 3]) + lm[3]),
+                                          pack_bf16(__uint_as_float(acc[8 * q + 4]) + lm[4], __uint_as_float(acc[8 * q + 5]) + lm[5]),
+                                          pack_bf16(__uint_as_float(acc[8 * q + 6]) + lm[6], __uint_as_float(acc[8 * q + 7]) + lm[7])));
                     }
                 }
                 fence_proxy_async();
