@@ -196,6 +196,13 @@ GF_API size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N);
  * and overlap on the GPU (different streams) race on it. */
 GF_API size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N);
 GF_API gf_status_t gf_wkv6_set_workspace(void *dev_ptr, size_t bytes);
+/* The split a bf16 prefill call of B*H units and T tokens (packed: S, max_seqlen) takes on a GPU of n_sm SMs with at
+ * most scratch_cap bytes of scratch (0: unlimited): *nseg segments per sequence (1: no split) of *seg_chunks 64-token
+ * chunks (the last takes the rest) and *scratch_bytes of scratch: per unit one 16 640-byte summary for every segment
+ * but the last and a 16 384-byte copy of the start state.  Host arithmetic only (no device is touched): what
+ * gf_wkv6_workspace_bytes and gf_wkv6_prefill_static decide with, exposed for planning and for tests. */
+GF_API gf_status_t gf_wkv6_split_plan(int B, int T, int H, int N, int n_sm, size_t scratch_cap, int *nseg,
+                               int *seg_chunks, size_t *scratch_bytes);
 
 /* Dense bf16 prefill for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of gf_wkv6_prefill.)  Some hosts of this library own no allocator at the

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -45,6 +45,7 @@ _SIGNATURES = {
     "gf_wkv6_host_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_set_workspace": (_i, [_vp, _sz]),
+    "gf_wkv6_split_plan": (_i, [_i] * 5 + [_sz, _vp, _vp, _vp]),
     "gf_wkv6_sequence_summary": (_i, [_vp] * 4 + [_i] * 5 + [_vp]),
     "gf_wkv6_fold_summaries": (_i, [_vp, _vp] + [_i] * 4 + [_vp, _vp]),
     "gf_c2_layernorm": (_i, [_vp, _vp, _vp, ctypes.c_float, _vp, ctypes.c_longlong, _i, _i, _vp]),
@@ -148,6 +149,15 @@ _workspace = None            # the registered scratch tensor is kept alive here
 def workspace_bytes(B, T, H, N=64) -> int:
     """Scratch gf_wkv6_prefill(B,T,H,N) would use on the current device (0: the call does not split)."""
     return int(load_library().gf_wkv6_workspace_bytes(int(B), int(T), int(H), int(N)))
+
+
+def split_plan(B, T, H, n_sm, scratch_cap=0, N=64):
+    """gf_wkv6_split_plan: (segments per sequence, chunks per segment, scratch bytes) of a bf16 prefill call on a GPU
+    of n_sm SMs with at most scratch_cap bytes of scratch (0: unlimited).  Host arithmetic, needs no device."""
+    nseg, sc, nb = ctypes.c_int(), ctypes.c_int(), ctypes.c_size_t()
+    _check(load_library().gf_wkv6_split_plan(int(B), int(T), int(H), int(N), int(n_sm), int(scratch_cap),
+                                             ctypes.byref(nseg), ctypes.byref(sc), ctypes.byref(nb)), "gf_wkv6_split_plan")
+    return nseg.value, sc.value, nb.value
 
 
 def set_workspace(buf: torch.Tensor | None) -> None:

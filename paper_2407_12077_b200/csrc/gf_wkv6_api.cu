@@ -445,6 +445,15 @@ size_t gf_wkv6_workspace_bytes(int B, int T, int H, int N)
     return need;
 }
 
+gf_status_t gf_wkv6_split_plan(int B, int T, int H, int N, int n_sm, size_t scratch_cap, int* nseg, int* seg_chunks,
+                               size_t* scratch_bytes)
+{
+    if (B < 0 || T < 0 || H < 0 || n_sm <= 0 || !nseg || !seg_chunks || !scratch_bytes) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    *nseg = gf::choose_split((long long)B * H, T, n_sm, seg_chunks, scratch_bytes, scratch_cap ? scratch_cap : ~(size_t)0);
+    return GF_OK;
+}
+
 gf_status_t gf_wkv6_set_workspace(void* dev_ptr, size_t bytes)
 {
     if (dev_ptr && (reinterpret_cast<uintptr_t>(dev_ptr) & 255u)) return GF_ERR_INVALID_ARG;

@@ -157,3 +157,45 @@ def test_key_compress_entry_point_validates_before_any_launch():
     assert _call(name, A, A + 0x100, A + 0x200, 8, 2044, 128, None) == 2            # D not a multiple of 8
     assert _call(name, A, A + 0x100, A + 0x200, 8, 2048, 44, None) == 2             # Dc not a multiple of 8
     assert _call(name, A, A + 0x100, A + 0x200, 8, 8192, 512, None) == 2            # Dc beyond 256
+
+
+def test_split_plan_and_the_built_in_scratch_limit():
+    """Host arithmetic of the sequence split (no device needed): the plan fills the GPU, respects the scratch cap by
+    taking fewer segments, and on 148 SMs the array of gf_wkv6_prefill_static holds every splitting call of up to
+    64 units (32 units four ways exactly) while 65..74 units do not fit even two ways."""
+    lib = gf.load_library()
+    SUMMARY, STATE = (64 + 64 * 64) * 4, 64 * 64 * 4
+    cap = gf.STATIC_SCRATCH_BYTES
+    # the header's constant, and the layout of this header's scratch formula
+    hdr = open(os.path.join(ROOT, "include", "gf_wkv6.h")).read()
+    assert f"#define GF_WKV6_STATIC_SCRATCH_BYTES {cap}u" in hdr
+    assert cap == 32 * (3 * SUMMARY + STATE)
+    for units in range(1, 149):
+        for T in (64, 1023, 1024, 4096, 16384, 131072):
+            H = units if units <= 64 else units // 2 if units % 2 == 0 else units
+            B = units // H
+            nseg, sc, nb = gf.split_plan(B, T, H, 148)
+            nchunks = -(-T // 64)
+            if units * 2 > 148 or nchunks < 16:
+                assert (nseg, sc, nb) == (1, 0, 0), (units, T)
+                continue
+            assert 2 <= nseg <= 8 and units * nseg <= 148 and sc >= 8, (units, T, nseg, sc)
+            assert (nseg - 1) * sc < nchunks <= nseg * sc                      # the segments cover the sequence, none empty
+            assert nb == units * ((nseg - 1) * SUMMARY + STATE)
+            # under the built-in array's cap: as many segments as fit, never more than unlimited, refusal only beyond 64 units
+            cseg, csc, cnb = gf.split_plan(B, T, H, 148, cap)
+            if units <= 64:
+                assert 2 <= cseg <= nseg and cnb <= cap and cnb == units * ((cseg - 1) * SUMMARY + STATE), (units, T)
+                if nb <= cap:
+                    assert (cseg, csc, cnb) == (nseg, sc, nb)
+            else:
+                assert (cseg, csc, cnb) == (1, 0, 0), (units, T)                # gf_wkv6_prefill_static refuses these
+    assert gf.split_plan(1, 4096, 32, 148) == (4, 16, cap)                      # the long-context shape fills it exactly
+    assert gf.split_plan(1, 8192, 16, 148)[0] == 8 and gf.split_plan(1, 8192, 16, 148, cap)[0] == 7
+    assert gf.split_plan(2, 4096, 12, 148)[0] == 6 and gf.split_plan(2, 4096, 12, 148, cap)[0] == 5
+    # argument checks
+    import ctypes
+    n, s, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_size_t()
+    assert lib.gf_wkv6_split_plan(1, 4096, 4, 32, 148, 0, ctypes.byref(n), ctypes.byref(s), ctypes.byref(b)) == 2
+    assert lib.gf_wkv6_split_plan(1, 4096, 4, 64, 0, 0, ctypes.byref(n), ctypes.byref(s), ctypes.byref(b)) == 1
+    assert lib.gf_wkv6_split_plan(1, 4096, 4, 64, 148, 0, None, ctypes.byref(s), ctypes.byref(b)) == 1
