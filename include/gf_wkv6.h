@@ -133,6 +133,25 @@ GF_API gf_status_t gf_wkv6_backward_f32(const float *r, const float *k, const fl
                                  void *workspace, size_t workspace_bytes, gf_stream_t stream);
 GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
 
+/* The same gradient for bf16 tensors (the gradient of gf_wkv6_prefill): r,k,v,x,dy and dr,dk,dv,dx are
+ * [B][T][H][N] bf16, u, du, state_in, dstate_out, dstate_in fp32 as above; every formula above holds, with the
+ * results rounded to bf16 once at the end.  Chunked on the tensor cores: the sequence is walked backwards in chunks
+ * of 64 tokens with the state adjoint G carried in fp32, nine 64x64x64 bf16 products (fp32 accumulate) per chunk
+ * give the in-chunk parts of dr, dk, dv and of G, and the decay-logit gradient comes from suffix sums of
+ * r*dr - k*dk over the chunk plus rowsum(G * S) at the chunk's end; the chunk-start states come from a state-only
+ * checkpoint pass of the forward kernel.  A chunk in which some channel decays by more than 2^-96 is processed token
+ * by token in fp32 instead, so any decay logit is accepted (x = +inf leaves dx undefined, as in the formula).
+ * `workspace`: caller-owned DEVICE buffer of at least gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes, 16-byte
+ * aligned (one 64x64 fp32 state per chunk and unit, plus 1 MiB per SM for the token-by-token path);
+ * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  Enqueues three
+ * kernels on `stream`, allocates nothing, does not synchronise; deterministic (no atomics).  A device-side wait that
+ * runs out is reported by gf_wkv6_last_device_status as for the forward call. */
+GF_API gf_status_t gf_wkv6_backward(const void *r, const void *k, const void *v, const void *x, const float *u,
+                             const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                             void *dk, void *dv, void *dx, float *du, float *dstate_in, int B, int T, int H,
+                             int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API size_t gf_wkv6_backward_bf16_workspace_bytes(int B, int T, int H, int N);
+
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a

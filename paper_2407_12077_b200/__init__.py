@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -34,6 +34,8 @@ _SIGNATURES = {
     "gf_wkv6_prefill_static": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_backward_f32": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_backward": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_bf16_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_prefill_c2": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_varlen_c2": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step_c2": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -219,26 +221,38 @@ def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, w
     return y, state_out
 
 
-def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None):
-    """gf_wkv6_backward_f32: gradient of the fp32 prefill.  r,k,v,x,dy: [B,T,H,N] fp32 CUDA tensors, u: [H,N],
-    state_in / dstate_out: [B,H,N,N] or None.  Returns (dr, dk, dv, dx, du, dstate_in); outputs and the workspace
-    are allocated here."""
+def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None):
+    """gf_wkv6_backward (bf16 tensors: chunked on the tensor cores) or gf_wkv6_backward_f32 (fp32 tensors: token by
+    token): gradient of the prefill.  r,k,v,x,dy: [B,T,H,N] CUDA tensors of one dtype, u: [H,N] fp32,
+    state_in / dstate_out: [B,H,N,N] fp32 or None.  Returns (dr, dk, dv, dx, du, dstate_in); outputs (and the
+    workspace, unless a uint8 tensor of enough bytes is passed) are allocated here."""
     lib = load_library()
     B, T, H, N = r.shape
     f32 = torch.float32
+    dt = r.dtype
+    if dt not in (torch.bfloat16, f32):
+        raise TypeError("backward: r must be bfloat16 or float32")
+    sfx, wsfn = ("_f32", "gf_wkv6_backward_workspace_bytes") if dt == f32 else ("", "gf_wkv6_backward_bf16_workspace_bytes")
     dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
     du = torch.empty((H, N), device=r.device, dtype=f32)
     ds0 = torch.empty((B, H, N, N), device=r.device, dtype=f32) if want_dstate else None
     with torch.cuda.device(r.device):
-        nbytes = int(lib.gf_wkv6_backward_workspace_bytes(B, T, H, N))
-        ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=r.device)
-        args = [_dev(r, "r", f32), _dev(k, "k", f32, r.shape), _dev(v, "v", f32, r.shape), _dev(x, "x", f32, r.shape),
-                _dev(u, "u", f32, (H, N)), _dev(state_in, "state_in", f32, (B, H, N, N)), _dev(dy, "dy", f32, r.shape),
+        nbytes = int(getattr(lib, wsfn)(B, T, H, N))
+        ws = workspace if workspace is not None and workspace.numel() >= nbytes else torch.empty(max(nbytes, 16), dtype=torch.uint8, device=r.device)
+        args = [_dev(r, "r", dt), _dev(k, "k", dt, r.shape), _dev(v, "v", dt, r.shape), _dev(x, "x", dt, r.shape),
+                _dev(u, "u", f32, (H, N)), _dev(state_in, "state_in", f32, (B, H, N, N)), _dev(dy, "dy", dt, r.shape),
                 _dev(dstate_out, "dstate_out", f32, (B, H, N, N)), _dev(dr, "dr"), _dev(dk, "dk"), _dev(dv, "dv"),
                 _dev(dx, "dx"), _dev(du, "du"), _dev(ds0, "dstate_in")]
-        _check(lib.gf_wkv6_backward_f32(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)),
-               "gf_wkv6_backward_f32")
+        _check(getattr(lib, "gf_wkv6_backward" + sfx)(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)),
+               "gf_wkv6_backward" + sfx)
     return dr, dk, dv, dx, du, ds0
+
+
+def backward_workspace_bytes(B, T, H, N, dtype=torch.bfloat16):
+    """Bytes of workspace backward() needs for tensors of this dtype on the current device."""
+    lib = load_library()
+    fn = "gf_wkv6_backward_workspace_bytes" if dtype == torch.float32 else "gf_wkv6_backward_bf16_workspace_bytes"
+    return int(getattr(lib, fn)(B, T, H, N))
 
 
 def prefill_c2(r, k, v, x, u2=None, state_in=None, state_out=None, y=None, stream=None, want_state=True, split=True):

@@ -11,6 +11,7 @@
 #include "key_compress.cuh"
 #include "ln_heads.cuh"
 #include "wkv6_backward.cuh"
+#include "wkv6_backward_chunked.cuh"
 #include "wkv6_chunked.cuh"
 #include "wkv6_exact.cuh"
 #include "wkv6_step.cuh"
@@ -386,6 +387,55 @@ gf_status_t gf_wkv6_backward_f32(const float* r, const float* k, const float* v,
     const size_t stride = gf::bw::unit_floats(T);
     gf::bw::wkv6_backward_du_kernel<<<(unsigned)H, gf::bw::N, 0, st>>>(ws, stride, stride - gf::bw::N, B, H, du);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    return launch_result();
+}
+
+size_t gf_wkv6_backward_bf16_workspace_bytes(int B, int T, int H, int N)
+{
+    if (B <= 0 || T <= 0 || H <= 0 || N != 64) return 0;
+    const int n_sm = gf::sm_count();
+    if (n_sm <= 0) return 0;
+    return gf::chunked_backward_workspace_bytes((long long)B * H, T, n_sm);
+}
+
+gf_status_t gf_wkv6_backward(const void* r, const void* k, const void* v, const void* x, const float* u,
+                             const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
+                             void* dv, void* dx, float* du, float* dstate_in, int B, int T, int H, int N,
+                             void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t sbytes = (size_t)B * H * 64 * 64 * sizeof(float);
+    if (T == 0) {
+        // no token: the state adjoint passes through and the bonus gets no gradient
+        if (misaligned(dstate_out) || misaligned(dstate_in) || misaligned(du)) return GF_ERR_INVALID_ARG;
+        cudaError_t e = cudaSuccess;
+        if (dstate_in && !dstate_out) e = cudaMemsetAsync(dstate_in, 0, sbytes, st);
+        else if (dstate_in && dstate_in != dstate_out) e = cudaMemcpyAsync(dstate_in, dstate_out, sbytes, cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && du) e = cudaMemsetAsync(du, 0, (size_t)H * 64 * sizeof(float), st);
+        return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+    }
+    if (!r || !k || !v || !x || !u || !dy || !dr || !dk || !dv || !dx || !du) return GF_ERR_INVALID_ARG;
+    const void* ptrs[] = {r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, workspace};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    const void* ins[] = {r, k, v, x, dy};
+    const void* outs[] = {dr, dk, dv, dx};
+    for (const void* o : outs)
+        for (const void* in : ins)
+            if (o == in) return GF_ERR_INVALID_ARG;
+    if ((long long)B * H > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    if ((long long)B * T >= (1LL << 31) - 64) return GF_ERR_UNSUPPORTED;
+    const size_t need = gf_wkv6_backward_bf16_workspace_bytes(B, T, H, N);
+    if (need == 0) return GF_ERR_CUDA;
+    if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
+    const gf_status_t s = gf::chunked_backward((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, (const bf*)dy,
+                                               dstate_out, (bf*)dr, (bf*)dk, (bf*)dv, (bf*)dx, du, dstate_in, B, T, H,
+                                               static_cast<float*>(workspace), st, &g_launches);
+    if (s != GF_OK) return s;
     return launch_result();
 }
 

@@ -1,0 +1,701 @@
+// Gradient of the WKV-6 recurrence in chunks of 64 tokens on the tensor cores (bf16 in and out, fp32 state adjoint).
+//
+// Forward, per (sequence, head), chunk with start state S_0, in-chunk inclusive cumulative log-decay a_t (a_0 = 0),
+// R^_t = r_t e^{a_{t-1}}, K^_i = k_i e^{-a_i}, D = e^{a_L}, b_t = sum_c r_t[c] u[c] k_t[c]:
+//   y_t = R^_t S_0 + sum_{i<t} (R^_t . K^_i) v_i + b_t v_t,      S_L = diag(D) (S_0 + K^^T V).
+// Backward, chunks from the last to the first, with G_L = dL/dS_L carried (G of the last chunk = dstate_out) and
+// G^ = diag(D) G_L, P' = tril(R^ K^^T, -1) + diag(b), dP' = tril(dY V^T, -1), dpd_t = dy_t . v_t:
+//   dV  = P'^T dY + K^ G^                                  dv_i = dV_i
+//   dR^ = dP' K^ + dY S_0^T                                dr_t = dR^_t e^{a_{t-1}} + u k_t dpd_t
+//   dK^ = dP'^T R^ + V G^^T                                dk_i = dK^_i e^{-a_i}    + u r_i dpd_i
+//   G_0 = G^ + R^^T dY                                     du  += sum_t r_t k_t dpd_t
+// and for the decay, with q_t = dR^_t R^_t, m_t = dK^_t K^_t (per channel) and E = rowsum(G_L * S_L):
+//   dL/d(log w_s) = E + sum_{t>s} q_t - sum_{t>=s} m_t,     dx_s = dL/d(log w_s) * log w_s       (log w = -e^x).
+// (log w_s enters a_t for every t >= s: R^_t through a_{t-1}, K^_t through a_t, D through a_L; the D term is
+// rowsum(G_L * diag(D)(S_0 + K^^T V)) = rowsum(G_L * S_L).)
+// Nine 64x64x64 bf16 tcgen05 products per chunk, accumulators in tensor memory.  The chunk-start states S_0 come from
+// a checkpoint pass of the forward kernel (state only), one 64x64 fp32 block per chunk.
+//
+// One CTA of 512 threads per unit works in phases separated by CTA barriers; an elected thread issues the TMA
+// copies and the products.  Every elementwise step uses the accumulator layout of the 64-row products: warp
+// (sp = warp % 4, cq = warp / 4) owns rows 16 sp .. +15 and columns 16 cq .. +15 of every 64x64 tile, a lane
+// (g = lane / 4, q = lane % 4) rows 16 sp + g and + 8, columns 16 cq + 8 n + 2 q + e (n, e in {0, 1}); bf16 tiles
+// move through ldmatrix / stmatrix in that layout, so scale factors computed for the operands stay in registers
+// until the epilogue needs them.  Sums along the tokens (cumulative decay, the suffix sums of the decay gradient)
+// run over lanes by shuffles and over the four row groups through shared memory.
+// A chunk in which some channel decays by more than 2^-96 is processed token by token in fp32 on the ALUs (its
+// states recomputed into a per-SM scratch in global memory), so any decay logit gives the gradient of the exact
+// recurrence.  Every wait is bounded; on expiry the status flag is raised and the whole CTA leaves together.
+#pragma once
+#include "wkv6_chunked.cuh"
+
+namespace gf {
+namespace bc {
+
+using namespace ck;          // PTX wrappers, descriptors, layout helpers of the forward kernel
+
+constexpr int B_THREADS = 512;
+constexpr float LN2 = 0.6931471805599453f;
+// tensor memory columns of the six accumulators
+constexpr int BT_P = 0, BT_DP = 64, BT_DV = 128, BT_DR = 192, BT_DK = 256, BT_DG = 320, BT_COLS = 512;
+// shared memory map (offsets from a 1024-byte aligned base); input stage: x, r, k, v, dy
+constexpr int B_STAGE = 5 * TILE;
+constexpr int BO_IN = 0;                          // [2][B_STAGE]
+constexpr int BO_RH = BO_IN + 2 * B_STAGE;        // R^ [t][c]
+constexpr int BO_KH = BO_RH + TILE;               // K^ [i][c]
+constexpr int BO_PP = BO_KH + TILE;               // P' [t][i]
+constexpr int BO_DPP = BO_PP + TILE;              // dP' [t][i]
+constexpr int BO_SB = BO_DPP + TILE;              // S_0 [c][j] bf16
+constexpr int BO_GB = BO_SB + TILE;               // G^  [c][j] bf16
+constexpr int BO_OUT = BO_GB + TILE;              // dr, dk, dv, dx staging [t][c]
+constexpr int BO_TOT = BO_OUT + 4 * TILE;         // [4][64] float: row-group totals of a scan
+constexpr int BO_EP = BO_TOT + 1024;              // [4][64] float: partial E by column group
+constexpr int BO_BP = BO_EP + 1024;               // [4][64] float: partial bonus by column group
+constexpr int BO_D = BO_BP + 1024;                // [64] float: D = e^{a_L}
+constexpr int BO_DPD = BO_D + 256;                // [64] float: dy_t . v_t
+constexpr int BO_RED = BO_DPD + 256;              // token-by-token path: [4][3][64] + [4][64] + du[64] + 2 floats
+constexpr int BO_RED_V = BO_RED + 4 * 3 * 64 * 4;
+constexpr int BO_DU_FB = BO_RED_V + 4 * 64 * 4;
+constexpr int BO_SCAL = BO_DU_FB + 256;
+constexpr int BO_FLAG = BO_SCAL + 16;             // int: some channel of this chunk decays too fast
+constexpr int BO_ABORT = BO_FLAG + 8;             // abort word, wait limit
+constexpr int BO_TMEM = BO_ABORT + 8;
+constexpr int BO_BAR = BO_TMEM + 8;               // mbarriers: input full [2], first / second group of products done
+enum { BB_IN = 0, BB_MMA1 = 2, BB_MMA2 = 3, BB_COUNT = 4 };
+constexpr int B_SMEM_BYTES = BO_BAR + 8 * BB_COUNT;
+constexpr int B_SMEM_ALLOC = B_SMEM_BYTES + 1024;
+static_assert(B_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
+constexpr size_t FB_SLOT_FLOATS = (size_t)64 * 4096;      // scratch of the token-by-token path per SM: 64 states
+
+struct BParams {
+    const float* u;              // [H][64]
+    const float* dstate_out;     // [units][64][64] or NULL (zero)
+    float* dstate_in;            // [units][64][64] or NULL (not written)
+    const float* ckpt;           // [units][chunks + 1][64][64]
+    float* du_part;              // [units][64]
+    float* fb_scratch;           // [n_slots][64][4096]
+    __nv_bfloat16 *dr, *dk, *dv, *dx;
+    int T, H, n_slots;
+    uint32_t wait_limit_us;
+};
+
+__device__ __forceinline__ float lds_bf16(uint32_t a)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory");
+    return __uint_as_float((uint32_t)v << 16);
+}
+__device__ __forceinline__ void sts_bf16(uint32_t a, float f)
+{
+    const __nv_bfloat16 b = __float2bfloat16_rn(f);
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"(*reinterpret_cast<const uint16_t*>(&b)) : "memory");
+}
+__device__ __forceinline__ void lds_v4(uint32_t a, uint32_t (&w)[4])
+{
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(a) : "memory");
+}
+__device__ __forceinline__ unsigned smid()
+{
+    unsigned v;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
+    return v;
+}
+
+// v[n][0..1] = (row g, columns 8n+2q, +1), v[n][2..3] = (row g+8, same columns) of this warp's 16 x 16 block
+__device__ __forceinline__ void load_block_bf16(uint32_t addr, float (&v)[2][4])
+{
+    uint32_t w0, w1, w2, w3;
+    ldsm_x4(addr, w0, w1, w2, w3);
+    v[0][0] = bf_lo(w0); v[0][1] = bf_hi(w0); v[0][2] = bf_lo(w1); v[0][3] = bf_hi(w1);
+    v[1][0] = bf_lo(w2); v[1][1] = bf_hi(w2); v[1][2] = bf_lo(w3); v[1][3] = bf_hi(w3);
+}
+__device__ __forceinline__ void store_block_bf16(uint32_t addr, const float (&v)[2][4])
+{
+    stsm_x4(addr, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
+}
+
+// Inclusive sums along the 64 rows of a tile held in the accumulator layout: forwards (REV = false: row t gets the
+// sum over rows <= t) or backwards (REV = true: rows >= t).  tot: [4][64] floats of shared memory.  Contains one
+// CTA barrier: all 512 threads call it together.
+template <bool REV>
+__device__ __forceinline__ void scan_rows(float (&v)[2][4], uint32_t tot, int sp, int cq, int lane)
+{
+    const int g = lane >> 2, q = lane & 3;
+#pragma unroll
+    for (int d = 4; d < 32; d <<= 1) {
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float o = REV ? __shfl_down_sync(0xffffffffu, v[n][e], d) : __shfl_up_sync(0xffffffffu, v[n][e], d);
+                if (REV ? lane + d < 32 : lane >= d) v[n][e] += o;
+            }
+    }
+    // the other half's total: rows g+8 follow rows g
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            if (REV) v[n][e] += __shfl_sync(0xffffffffu, v[n][2 + e], q);
+            else v[n][2 + e] += __shfl_sync(0xffffffffu, v[n][e], 28 + q);
+        }
+    if (g == (REV ? 0 : 7)) {
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+            *reinterpret_cast<float2*>(__cvta_shared_to_generic((size_t)(tot + 4 * (sp * 64 + 16 * cq + 8 * n + 2 * q)))) =
+                REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int o = 0; o < 4; ++o) {
+        if (REV ? o > sp : o < sp) {
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                const float2 t = *reinterpret_cast<const float2*>(__cvta_shared_to_generic((size_t)(tot + 4 * (o * 64 + 16 * cq + 8 * n + 2 * q))));
+                v[n][0] += t.x; v[n][1] += t.y; v[n][2] += t.x; v[n][3] += t.y;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(B_THREADS, 1)
+wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
+                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                             const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
+                             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
+                             const __grid_constant__ CUtensorMap tm_dx, const BParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t abort_flag = sbase + BO_ABORT;
+    auto bar = [&](int i) { return sbase + BO_BAR + 8 * i; };
+    auto fsm = [&](int off) { return reinterpret_cast<float*>(smem + off); };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sp = warp & 3, cq = warp >> 2, g = lane >> 2, q = lane & 3;
+    const int unit = blockIdx.x, seq = unit / p.H, h = unit % p.H;
+    const int T = p.T, nchunks = (T + L - 1) / L;
+    const long long row0 = (long long)seq * T;
+    const int col0 = h * 64;
+    const size_t C = (size_t)p.H * 64;
+    const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
+    const int cb = 16 * cq + 2 * q;                  // its columns: cb + 8 n + e
+    // byte offset of this lane's ldmatrix / stmatrix row inside a tile (the warp's 16 x 16 block)
+    const uint32_t moff = swz(16 * sp + (lane & 7) + 8 * ((lane >> 3) & 1), (2 * cq + (lane >> 4)) << 4);
+
+    if (tid == 0) {
+        for (int i = 0; i < BB_COUNT; ++i) mbar_init(bar(i), 1);
+        sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, p.wait_limit_us ? p.wait_limit_us : WAIT_LIMIT_US);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (tid < 64) fsm(BO_DU_FB)[tid] = 0.f;
+    if (warp == 1) tmem_alloc(sbase + BO_TMEM, BT_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32(sbase + BO_TMEM);
+    const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 16 * cq;      // this warp's block of an accumulator
+
+    // A wait by warp 0 whose outcome every thread of the CTA learns (contains a CTA barrier).
+    auto wait_all = [&](uint32_t b, uint32_t parity) -> bool {
+        bool ok = true;
+        if (warp == 0) ok = mbar_wait_warp(b, parity, abort_flag);
+        ok = __syncthreads_and(ok);
+        if (ok) mbar_try_wait(b, parity);            // (completed: every thread observes the phase itself)
+        return ok;
+    };
+    auto issue_loads = [&](int c, int stage) {       // one thread
+        const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
+        const int row = (int)(row0 + (long long)c * L);
+        mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
+        tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
+    };
+    auto load_f32_block = [&](const float* src, float (&v)[2][4]) {      // [64][64] fp32 block, accumulator layout
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)R0 * 64 + cb + 8 * n);
+            const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)R1 * 64 + cb + 8 * n);
+            v[n][0] = lo.x; v[n][1] = lo.y; v[n][2] = hi.x; v[n][3] = hi.y;
+        }
+    };
+
+    float uu[2][2];                                  // bonus of this lane's columns (as channels)
+#pragma unroll
+    for (int n = 0; n < 2; ++n) { uu[n][0] = p.u[col0 + cb + 8 * n]; uu[n][1] = p.u[col0 + cb + 8 * n + 1]; }
+    float G[2][4], SL[2][4], du_acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    const float* ck_unit = p.ckpt + (size_t)unit * (nchunks + 1) * 4096;
+    if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
+    else {
+#pragma unroll
+        for (int n = 0; n < 2; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
+    }
+    load_f32_block(ck_unit + (size_t)nchunks * 4096, SL);
+    if (tid == 0 && nchunks > 0) issue_loads(nchunks - 1, 0);
+    int pend = nchunks > 0 ? 0 : -1;                 // (thread 0) iteration whose input copies may still be in flight
+    int mph = 0;                                     // phase bit of the two product barriers (one phase per chunk on this path)
+    bool alive = true;
+
+    for (int it = 0; it < nchunks; ++it) {
+        const int c = nchunks - 1 - it, stage = it & 1;
+        const int valid = min(L, T - c * L);
+        const uint32_t tin = sbase + BO_IN + stage * B_STAGE;
+        const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
+        if (tid == 0) sts32(sbase + BO_FLAG, 0u);
+        float S0[2][4];
+        load_f32_block(ck_unit + (size_t)c * 4096, S0);
+        // ---- E = rowsum(G_L * S_L): partial over this lane's columns, then over the four lanes of a row
+        {
+            float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                e0 = fmaf(G[n][0], SL[n][0], fmaf(G[n][1], SL[n][1], e0));
+                e1 = fmaf(G[n][2], SL[n][2], fmaf(G[n][3], SL[n][3], e1));
+            }
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
+            if (q == 0) { fsm(BO_EP)[cq * 64 + R0] = e0; fsm(BO_EP)[cq * 64 + R1] = e1; }
+        }
+        if (!wait_all(bar(BB_IN + stage), (it >> 1) & 1)) { alive = false; break; }
+        if (tid == 0) {
+            pend = -1;
+            if (c > 0) { issue_loads(c - 1, stage ^ 1); pend = it + 1; }
+        }
+        if (valid < L) {
+            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
+            for (int i = tid; i < (L - valid) * 8; i += B_THREADS) {
+                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
+                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
+            }
+        }
+        // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
+        float lw2[2][4], a[2][4];
+        {
+            float xv[2][4];
+            load_block_bf16(tx + moff, xv);
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool live = (e < 2 ? R0 : R1) < valid;
+                    lw2[n][e] = live ? -ex2(fmaf(xv[n][e], LOG2E, LOG2_LOG2E)) : 0.f;
+                    a[n][e] = lw2[n][e];
+                }
+        }
+        scan_rows<false>(a, sbase + BO_TOT, sp, cq, lane);       // (barrier: the zeroed rows are visible after it)
+        float sr[2][4], sk[2][4], rv[2][4], kv[2][4];
+        load_block_bf16(tr + moff, rv);
+        load_block_bf16(tk + moff, kv);
+        {
+            float rh[2][4], kh[2][4];
+            float b0 = 0.f, b1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    sr[n][e] = ex2(a[n][e] - lw2[n][e]);
+                    sk[n][e] = ex2(-a[n][e]);
+                    rh[n][e] = rv[n][e] * sr[n][e];
+                    kh[n][e] = kv[n][e] * sk[n][e];
+                    const float t = rv[n][e] * kv[n][e] * uu[n][e & 1];
+                    if (e < 2) b0 += t; else b1 += t;
+                }
+            store_block_bf16(sbase + BO_RH + moff, rh);
+            store_block_bf16(sbase + BO_KH + moff, kh);
+            b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
+            b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
+            if (q == 0) { fsm(BO_BP)[cq * 64 + R0] = b0; fsm(BO_BP)[cq * 64 + R1] = b1; }
+        }
+        if (sp == 3 && g == 7) {                     // row 63 holds a_L
+            bool ok = true;
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                fsm(BO_D)[cb + 8 * n] = ex2(a[n][2]);
+                fsm(BO_D)[cb + 8 * n + 1] = ex2(a[n][3]);
+                ok = ok && (a[n][2] >= -A2_MAX) && (a[n][3] >= -A2_MAX);      // false for NaN as well
+            }
+            if (!ok) sts32(sbase + BO_FLAG, 1u);
+        }
+        store_block_bf16(sbase + BO_SB + moff, S0);
+        __syncthreads();
+        const bool unsafe = lds32(sbase + BO_FLAG) != 0;
+        const float d_lo = fsm(BO_D)[R0], d_hi = fsm(BO_D)[R1];      // decay of the chunk for this lane's rows of G
+
+        if (!unsafe) {
+            {
+                float gh[2][4];
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    gh[n][0] = d_lo * G[n][0]; gh[n][1] = d_lo * G[n][1];
+                    gh[n][2] = d_hi * G[n][2]; gh[n][3] = d_hi * G[n][3];
+                }
+                store_block_bf16(sbase + BO_GB + moff, gh);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                const uint64_t dR = smem_desc(sbase + BO_RH), dK = smem_desc(sbase + BO_KH), dV = smem_desc(tv), dY = smem_desc(tdy);
+                const uint64_t dS = smem_desc(sbase + BO_SB), dG = smem_desc(sbase + BO_GB);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
+                    tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
+                    tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
+                    tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                    tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
+                    tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
+                    tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                }
+                tc_commit(bar(BB_MMA1));
+            }
+            if (!wait_all(bar(BB_MMA1), mph)) { alive = false; break; }
+            tc_fence_after();
+            // ---- masked scores and their adjoint as operands
+            {
+                float pp[2][4], dp[2][4];
+                tmem_ld_16x16(tacc + BT_P, pp);
+                tmem_ld_16x16(tacc + BT_DP, dp);
+                float bon0 = 0.f, bon1 = 0.f;
+                if (cq == sp) {
+#pragma unroll
+                    for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
+                }
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int row = e < 2 ? R0 : R1, col = cb + 8 * n + (e & 1);
+                        if (col == row) fsm(BO_DPD)[row] = dp[n][e];
+                        pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
+                        dp[n][e] = col < row ? dp[n][e] : 0.f;
+                    }
+                store_block_bf16(sbase + BO_PP + moff, pp);
+                store_block_bf16(sbase + BO_DPP + moff, dp);
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
+                const uint64_t dR = smem_desc(sbase + BO_RH), dK = smem_desc(sbase + BO_KH), dY = smem_desc(tdy);
+                const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                    tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
+                    tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
+                }
+                tc_commit(bar(BB_MMA2));
+            }
+            // ---- meanwhile: G_0 = diag(D) G_L + R^^T dY
+            {
+                float dg[2][4];
+                tmem_ld_16x16(tacc + BT_DG, dg);
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
+                    G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
+                }
+            }
+            if (!wait_all(bar(BB_MMA2), mph)) { alive = false; break; }
+            tc_fence_after();
+            mph ^= 1;
+            // ---- epilogue
+            float z[2][4], qv[2][4];
+            {
+                // q and m take the operands as the tensor core saw them (rounded to bf16): the pair terms that q and
+                // m share, and that cancel in the suffix sums, are then the same products on both sides
+                float acc[2][4], o[2][4], hat[2][4];
+                const float pd0 = fsm(BO_DPD)[R0], pd1 = fsm(BO_DPD)[R1];
+                tmem_ld_16x16(tacc + BT_DR, acc);
+                load_block_bf16(sbase + BO_RH + moff, hat);
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float pd = e < 2 ? pd0 : pd1;
+                        o[n][e] = fmaf(uu[n][e & 1] * kv[n][e], pd, acc[n][e] * sr[n][e]);
+                        qv[n][e] = acc[n][e] * hat[n][e];
+                        du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
+                    }
+                store_block_bf16(sbase + BO_OUT + moff, o);
+                tmem_ld_16x16(tacc + BT_DK, acc);
+                load_block_bf16(sbase + BO_KH + moff, hat);
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float pd = e < 2 ? pd0 : pd1;
+                        o[n][e] = fmaf(uu[n][e & 1] * rv[n][e], pd, acc[n][e] * sk[n][e]);
+                        z[n][e] = qv[n][e] - acc[n][e] * hat[n][e];
+                    }
+                store_block_bf16(sbase + BO_OUT + TILE + moff, o);
+                tmem_ld_16x16(tacc + BT_DV, acc);
+                store_block_bf16(sbase + BO_OUT + 2 * TILE + moff, acc);
+            }
+            tc_fence_before();
+            scan_rows<true>(z, sbase + BO_TOT, sp, cq, lane);
+            {
+                float o[2][4];
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    float E0 = 0.f, E1 = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) { E0 += fsm(BO_EP)[w * 64 + cb + 8 * n]; E1 += fsm(BO_EP)[w * 64 + cb + 8 * n + 1]; }
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        o[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
+                }
+                store_block_bf16(sbase + BO_OUT + 3 * TILE + moff, o);
+            }
+        } else {
+            // ---- token by token: the chunk's states recomputed into this SM's scratch, then the reverse recurrence
+            const unsigned slot = smid();
+            if (slot >= (unsigned)p.n_slots) {       // (no scratch for this SM: report it and leave)
+                if (tid == 0) { sts32(abort_flag, 1u); atomicExch(&g_dev_status, 1); }
+                alive = false;
+                __syncthreads();
+                break;
+            }
+            float* scr = p.fb_scratch + (size_t)slot * FB_SLOT_FLOATS + (size_t)tid * 8;
+            // rows are key channels here: this lane's channels R0, R1 of S and G; its columns are value channels
+            float S[2][4];
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) S[n][e] = S0[n][e];
+            for (int t = 0; t < valid; ++t) {
+                *reinterpret_cast<float4*>(scr + (size_t)t * 4096) = make_float4(S[0][0], S[0][1], S[0][2], S[0][3]);
+                *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4) = make_float4(S[1][0], S[1][1], S[1][2], S[1][3]);
+                const float w0 = expf(-expf(lds_bf16(tx + swz(t, 2 * R0)))), w1 = expf(-expf(lds_bf16(tx + swz(t, 2 * R1))));
+                const float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float vj = lds_bf16(tv + swz(t, 2 * (cb + 8 * n + e)));
+                        S[n][e] = fmaf(w0, S[n][e], k0 * vj);
+                        S[n][2 + e] = fmaf(w1, S[n][2 + e], k1 * vj);
+                    }
+            }
+            float* red = fsm(BO_RED);                // [cq][3][64]
+            float* redv = fsm(BO_RED_V);             // [sp][64]
+            float* scal = fsm(BO_SCAL);              // v . dy, sum r u k
+            for (int t = valid - 1; t >= 0; --t) {
+                const float4 sa = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096);
+                const float4 sb4 = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096 + 4);
+                const float Sp[2][4] = {{sa.x, sa.y, sa.z, sa.w}, {sb4.x, sb4.y, sb4.z, sb4.w}};
+                const float x0 = lds_bf16(tx + swz(t, 2 * R0)), x1 = lds_bf16(tx + swz(t, 2 * R1));
+                const float w0 = expf(-expf(x0)), w1 = expf(-expf(x1));
+                const float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                const float r0 = lds_bf16(tr + swz(t, 2 * R0)), r1 = lds_bf16(tr + swz(t, 2 * R1));
+                float pr0 = 0.f, pr1 = 0.f, pk0 = 0.f, pk1 = 0.f, pg0 = 0.f, pg1 = 0.f, pv[2][2];
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int j = cb + 8 * n + e;
+                        const float vj = lds_bf16(tv + swz(t, 2 * j)), dyj = lds_bf16(tdy + swz(t, 2 * j));
+                        pr0 = fmaf(dyj, Sp[n][e], pr0); pr1 = fmaf(dyj, Sp[n][2 + e], pr1);
+                        pk0 = fmaf(G[n][e], vj, pk0); pk1 = fmaf(G[n][2 + e], vj, pk1);
+                        pg0 = fmaf(G[n][e], Sp[n][e], pg0); pg1 = fmaf(G[n][2 + e], Sp[n][2 + e], pg1);
+                        pv[n][e] = fmaf(G[n][e], k0, G[n][2 + e] * k1);
+                        G[n][e] = fmaf(w0, G[n][e], r0 * dyj);
+                        G[n][2 + e] = fmaf(w1, G[n][2 + e], r1 * dyj);
+                    }
+#pragma unroll
+                for (int d = 1; d < 4; d <<= 1) {
+                    pr0 += __shfl_xor_sync(0xffffffffu, pr0, d); pr1 += __shfl_xor_sync(0xffffffffu, pr1, d);
+                    pk0 += __shfl_xor_sync(0xffffffffu, pk0, d); pk1 += __shfl_xor_sync(0xffffffffu, pk1, d);
+                    pg0 += __shfl_xor_sync(0xffffffffu, pg0, d); pg1 += __shfl_xor_sync(0xffffffffu, pg1, d);
+                }
+#pragma unroll
+                for (int d = 4; d < 32; d <<= 1)
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) pv[n][e] += __shfl_xor_sync(0xffffffffu, pv[n][e], d);
+                if (q == 0) {
+                    red[(cq * 3 + 0) * 64 + R0] = pr0; red[(cq * 3 + 0) * 64 + R1] = pr1;
+                    red[(cq * 3 + 1) * 64 + R0] = pk0; red[(cq * 3 + 1) * 64 + R1] = pk1;
+                    red[(cq * 3 + 2) * 64 + R0] = pg0; red[(cq * 3 + 2) * 64 + R1] = pg1;
+                }
+                if (g == 0) {
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) redv[sp * 64 + cb + 8 * n + e] = pv[n][e];
+                }
+                if (warp == 0) {
+                    float vd = 0.f, ruk = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int cc = 2 * lane + e;
+                        vd = fmaf(lds_bf16(tv + swz(t, 2 * cc)), lds_bf16(tdy + swz(t, 2 * cc)), vd);
+                        ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * p.u[col0 + cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
+                    }
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        vd += __shfl_xor_sync(0xffffffffu, vd, d);
+                        ruk += __shfl_xor_sync(0xffffffffu, ruk, d);
+                    }
+                    if (lane == 0) { scal[0] = vd; scal[1] = ruk; }
+                }
+                __syncthreads();
+                if (tid < 64) {
+                    const int cc = tid;
+                    float s_r = 0.f, s_k = 0.f, s_g = 0.f;
+#pragma unroll
+                    for (int o = 0; o < 4; ++o) { s_r += red[(o * 3 + 0) * 64 + cc]; s_k += red[(o * 3 + 1) * 64 + cc]; s_g += red[(o * 3 + 2) * 64 + cc]; }
+                    const float xc = lds_bf16(tx + swz(t, 2 * cc)), kc = lds_bf16(tk + swz(t, 2 * cc)), rc = lds_bf16(tr + swz(t, 2 * cc));
+                    const float uc = p.u[col0 + cc], vd = scal[0];
+                    sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
+                    sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
+                    sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), s_g * (-expf(-expf(xc)) * expf(xc)));
+                    fsm(BO_DU_FB)[cc] = fmaf(rc * kc, vd, fsm(BO_DU_FB)[cc]);
+                } else if (tid < 128) {
+                    const int j = tid - 64;
+                    const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
+                    sts_bf16(sbase + BO_OUT + 2 * TILE + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
+                }
+                __syncthreads();
+            }
+        }
+        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one
+        fence_proxy_async();
+        __syncthreads();
+        if (valid == L) {
+            if (tid == 0) {
+                const int row = (int)(row0 + (long long)c * L);
+                tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
+                tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
+                tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
+                tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
+                bulk_commit();
+                bulk_wait_read<0>();                 // the staging tiles are rewritten next chunk
+            }
+        } else {
+            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
+            for (int i = tid; i < 4 * valid * 8; i += B_THREADS) {
+                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
+                uint32_t w[4];
+                lds_v4(sbase + BO_OUT + tile * TILE + swz(t, blk << 4), w);
+                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) SL[n][e] = S0[n][e];
+    }
+
+    if (alive) {
+        if (p.dstate_in) {
+            float* dst = p.dstate_in + (size_t)unit * 4096;
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                *reinterpret_cast<float2*>(dst + (size_t)R0 * 64 + cb + 8 * n) = make_float2(G[n][0], G[n][1]);
+                *reinterpret_cast<float2*>(dst + (size_t)R1 * 64 + cb + 8 * n) = make_float2(G[n][2], G[n][3]);
+            }
+        }
+        // the bonus gradient of this unit: over the lanes' rows, then over the four row groups, in a fixed order
+#pragma unroll
+        for (int d = 4; d < 32; d <<= 1)
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) du_acc[n][e] += __shfl_xor_sync(0xffffffffu, du_acc[n][e], d);
+        if (g == 0) {
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) fsm(BO_RED_V)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
+        }
+        __syncthreads();
+        if (tid < 64) {
+            const float* rv4 = fsm(BO_RED_V);
+            p.du_part[(size_t)unit * 64 + tid] = ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fsm(BO_DU_FB)[tid];
+        }
+    }
+    if (tid == 0) {
+        bulk_wait<0>();                              // the gradient tiles have reached memory
+        if (pend >= 0)                               // (aborting) no copy into this CTA's shared memory may stay in flight
+            mbar_wait(bar(BB_IN + (pend & 1)), (pend >> 1) & 1, abort_flag, false);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, BT_COLS);
+    }
+}
+
+// du[h][i] = sum over the batch of the units' partial sums, in batch order
+__global__ void __launch_bounds__(64)
+wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H, float* __restrict__ du)
+{
+    const int h = blockIdx.x, i = threadIdx.x;
+    float acc = 0.f;
+    for (int b = 0; b < B; ++b) acc += du_part[((size_t)b * H + h) * 64 + i];
+    du[h * 64 + i] = acc;
+}
+
+}  // namespace bc
+
+// Workspace of the chunked gradient: checkpoints, per-unit bonus gradients, the token-by-token path's scratch.
+inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
+{
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    return ((size_t)units * nck * 4096 + (size_t)units * 64 + (size_t)n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+}
+
+inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                    const __nv_bfloat16* x, const float* u, const float* state_in,
+                                    const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
+                                    __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
+                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches)
+{
+    const long long units = (long long)B * H, rows = (long long)B * T;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return GF_ERR_CUDA;
+    static PerDeviceFlag attr_set;
+    const int dev = current_device();
+    if (dev < 0) return GF_ERR_CUDA;
+    if (!attr_set.is_set(dev)) {
+        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess)
+            return GF_ERR_CUDA;
+        attr_set.set(dev);
+    }
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    float* ckpt = ws;
+    float* du_part = ckpt + (size_t)units * nck * 4096;
+    float* fb = du_part + (size_t)units * 64;
+    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches);
+    if (s != GF_OK) return s;
+    const long long C = (long long)H * 64;
+    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
+    if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||
+        !ck::make_map(&tv, v, rows, C, 64) || !ck::make_map(&tdy, dy, rows, C, 64) || !ck::make_map(&tdr, dr, rows, C, 64) ||
+        !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
+        return GF_ERR_CUDA;
+    bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, n_sm,
+                  wait_limit_us().load(std::memory_order_relaxed)};
+    bc::wkv6_backward_chunked_kernel<<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+}  // namespace gf

@@ -477,6 +477,10 @@ struct Params {
     // reads state_in once the first state_out has been written (state_out may be state_in).  NULL: no copy.
     float* state_copy;
     uint32_t wait_limit_us;                // limit of every device-side wait of the launch (0: the default, 2 s)
+    // Checkpoint pass (a summary launch with one segment per unit, used by the gradient): starts from state_in and
+    // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32) instead of
+    // a summary.  NULL: no checkpoints.
+    float* ckpt;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -650,7 +654,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     // first pass of a split call: the second launch (enqueued with programmatic stream serialisation) may set up and
     // fill its rings while this one runs; its state warps wait for this grid's results before they read them
     if (SUMMARY) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int gsegs = SUMMARY ? p.nseg - 1 : p.nseg;      // segments per unit that this launch covers
+    const int gsegs = (SUMMARY && !p.ckpt) ? p.nseg - 1 : p.nseg;      // segments per unit that this launch covers
     const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs;
     const int seq = unit / p.H, h = unit % p.H;
     long long row0;
@@ -915,7 +919,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         auto load_state = [&](size_t base) {         // this lane's part of the start state of a unit (zero without one)
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
-                if (!SUMMARY && s_src) {
+                if ((!SUMMARY || p.ckpt) && s_src) {
                     const float2 lo = *reinterpret_cast<const float2*>(s_src + base + (size_t)c_lo * 64 + 8 * n + 2 * q);
                     const float2 hi = *reinterpret_cast<const float2*>(s_src + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q);
                     st[n][0] = lo.x; st[n][1] = lo.y; st[n][2] = hi.x; st[n][3] = hi.y;
@@ -933,13 +937,14 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 *reinterpret_cast<float2*>(p.state_copy + hi) = *reinterpret_cast<const float2*>(p.state_in + hi);
             }
         }
-        auto store_state = [&](size_t base) {
+        auto store_to = [&](float* dst) {            // this lane's part of the state into a [64][64] fp32 block
 #pragma unroll
             for (int n = 0; n < 8; ++n) {
-                *reinterpret_cast<float2*>(p.state_out + base + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
-                *reinterpret_cast<float2*>(p.state_out + base + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
+                *reinterpret_cast<float2*>(dst + (size_t)c_lo * 64 + 8 * n + 2 * q) = make_float2(st[n][0], st[n][1]);
+                *reinterpret_cast<float2*>(dst + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = make_float2(st[n][2], st[n][3]);
             }
         };
+        auto store_state = [&](size_t base) { store_to(p.state_out + base); };
         // second launch of a split call: the summaries and the start-state copy are the first launch's
         if (!SUMMARY && !PERSIST && p.nseg > 1) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!PERSIST) load_state(sb);
@@ -967,6 +972,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
+            if (SUMMARY && p.ckpt) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + c) * 4096);   // the state before chunk c
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1059,7 +1065,9 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (SUMMARY) {
+        if (SUMMARY && p.ckpt) {
+            if (!lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + nchunks) * 4096);
+        } else if (SUMMARY) {
             if (!lds32(abort_flag)) {
                 float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
                 if (q == 0) { sm[c_lo] = dprod_lo; sm[c_lo + 8] = dprod_hi; }
@@ -1653,6 +1661,30 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+// Checkpoint pass of dense sequences: the state before every chunk of 64 tokens and after the last one,
+// ckpt [n_seq*H][chunks + 1][64][64] fp32, from state_in (NULL: zero).  One summary-variant launch (state only: reads
+// k, v and the decay logits).
+inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x,
+                                       const float* state_in, float* ckpt, int n_seq, int T, int H, cudaStream_t st,
+                                       std::atomic<uint64_t>* launches)
+{
+    const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
+    if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
+    if (total_rows >= (1LL << 31) - 64 || !ck::encode_fn()) return GF_ERR_UNSUPPORTED;
+    if (!chunked_kernel_attributes()) return GF_ERR_CUDA;
+    CUtensorMap tk, tv, tx, tdummy;
+    const long long C = (long long)H * 64;
+    if (!ck::make_map(&tk, k, total_rows, C, 64) || !ck::make_map(&tv, v, total_rows, C, 64) ||
+        !ck::make_map(&tx, x, total_rows, C, 64) || !ck::make_map(&tdummy, k, total_rows, C, 16))
+        return GF_ERR_CUDA;
+    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, nullptr, (T + ck::L - 1) / ck::L, 1, nullptr, 0};
+    p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
+    p.ckpt = ckpt;
+    ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
