@@ -34,34 +34,36 @@ namespace bc {
 
 using namespace ck;          // PTX wrappers, descriptors, layout helpers of the forward kernel
 
-constexpr int B_THREADS = 512;
+constexpr int B_CTHREADS = 512;                  // 16 compute warps
+constexpr int B_THREADS = B_CTHREADS + 32;       // and the warp that issues the products and the TMA copies
 constexpr float LN2 = 0.6931471805599453f;
 // tensor memory columns of the six accumulators
 constexpr int BT_P = 0, BT_DP = 64, BT_DV = 128, BT_DR = 192, BT_DK = 256, BT_DG = 320, BT_COLS = 512;
 // shared memory map (offsets from a 1024-byte aligned base); input stage: x, r, k, v, dy
 constexpr int B_STAGE = 5 * TILE;
 constexpr int BO_IN = 0;                          // [2][B_STAGE]
-constexpr int BO_RH = BO_IN + 2 * B_STAGE;        // R^ [t][c]
-constexpr int BO_KH = BO_RH + TILE;               // K^ [i][c]
-constexpr int BO_PP = BO_KH + TILE;               // P' [t][i]
+constexpr int BO_RH = BO_IN + 2 * B_STAGE;        // [2] R^ [t][c]        (by chunk parity, like the input stages)
+constexpr int BO_KH = BO_RH + 2 * TILE;           // [2] K^ [i][c]
+constexpr int BO_SB = BO_KH + 2 * TILE;           // [2] S_0 [c][j] bf16
+constexpr int BO_GB = BO_SB + 2 * TILE;           // [2] G^  [c][j] bf16
+constexpr int BO_PP = BO_GB + 2 * TILE;           // P' [t][i]
 constexpr int BO_DPP = BO_PP + TILE;              // dP' [t][i]
-constexpr int BO_SB = BO_DPP + TILE;              // S_0 [c][j] bf16
-constexpr int BO_GB = BO_SB + TILE;               // G^  [c][j] bf16
-constexpr int BO_OUT = BO_GB + TILE;              // dr, dk, dv, dx staging [t][c]
+constexpr int BO_OUT = BO_DPP + TILE;             // dr, dk, dv, dx staging [t][c]
 constexpr int BO_TOT = BO_OUT + 4 * TILE;         // [4][64] float: row-group totals of a scan
-constexpr int BO_EP = BO_TOT + 1024;              // [4][64] float: partial E by column group
-constexpr int BO_BP = BO_EP + 1024;               // [4][64] float: partial bonus by column group
-constexpr int BO_D = BO_BP + 1024;                // [64] float: D = e^{a_L}
-constexpr int BO_DPD = BO_D + 256;                // [64] float: dy_t . v_t
+constexpr int BO_EP = BO_TOT + 1024;              // [2][4][64] float: partial E by column group (by chunk parity)
+constexpr int BO_BP = BO_EP + 2048;               // [4][64] float: partial bonus by column group
+constexpr int BO_DPD = BO_BP + 1024;              // [64] float: dy_t . v_t
 constexpr int BO_RED = BO_DPD + 256;              // token-by-token path: [4][3][64] + [4][64] + du[64] + 2 floats
 constexpr int BO_RED_V = BO_RED + 4 * 3 * 64 * 4;
 constexpr int BO_DU_FB = BO_RED_V + 4 * 64 * 4;
 constexpr int BO_SCAL = BO_DU_FB + 256;
-constexpr int BO_FLAG = BO_SCAL + 16;             // int: some channel of this chunk decays too fast
-constexpr int BO_ABORT = BO_FLAG + 8;             // abort word, wait limit
+constexpr int BO_ABORT = BO_SCAL + 16;            // abort word, wait limit
 constexpr int BO_TMEM = BO_ABORT + 8;
-constexpr int BO_BAR = BO_TMEM + 8;               // mbarriers: input full [2], first / second group of products done
-enum { BB_IN = 0, BB_MMA1 = 2, BB_MMA2 = 3, BB_COUNT = 4 };
+constexpr int BO_CMD = BO_TMEM + 8;               // [4] {command, argument} for the issuing warp
+constexpr int BO_BAR = BO_CMD + 32;               // mbarriers: input full [2], first / second group of products done,
+// ... staging tiles read by the TMA unit, command slots [4]
+enum { BB_IN = 0, BB_MMA1 = 2, BB_MMA2 = 3, BB_STAGING = 4, BB_CMD = 5, BB_COUNT = 9 };
+enum { CMD_QUIT = 0, CMD_MMA1 = 1, CMD_MMA2 = 2, CMD_STORE = 3 };
 constexpr int B_SMEM_BYTES = BO_BAR + 8 * BB_COUNT;
 constexpr int B_SMEM_ALLOC = B_SMEM_BYTES + 1024;
 static_assert(B_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
@@ -101,6 +103,30 @@ __device__ __forceinline__ unsigned smid()
     return v;
 }
 
+// Barrier over the 16 compute warps (the issuing warp does not take part), and the same with an AND over a predicate.
+__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+__device__ __forceinline__ bool cbar_and(bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 1, 512, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)ok) : "memory");
+    return r != 0;
+}
+
+// tcgen05.ld of a 16 x 16 fp32 block without the wait for its data (tmem_ld_done() before the first use): several
+// loads can then be in flight together.
+__device__ __forceinline__ void tmem_ld_16x16_async(uint32_t taddr, float (&v)[2][4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_done() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // v[n][0..1] = (row g, columns 8n+2q, +1), v[n][2..3] = (row g+8, same columns) of this warp's 16 x 16 block
 __device__ __forceinline__ void load_block_bf16(uint32_t addr, float (&v)[2][4])
 {
@@ -116,9 +142,10 @@ __device__ __forceinline__ void store_block_bf16(uint32_t addr, const float (&v)
 
 // Inclusive sums along the 64 rows of a tile held in the accumulator layout: forwards (REV = false: row t gets the
 // sum over rows <= t) or backwards (REV = true: rows >= t).  tot: [4][64] floats of shared memory.  Contains one
-// CTA barrier: all 512 threads call it together.
+// barrier of the compute warps (all 512 threads call it together), which also forms the AND of `ok` over them: the
+// result is returned (a wait that ran out on some thread makes every thread leave together).
 template <bool REV>
-__device__ __forceinline__ void scan_rows(float (&v)[2][4], uint32_t tot, int sp, int cq, int lane)
+__device__ __forceinline__ bool scan_rows(float (&v)[2][4], uint32_t tot, int sp, int cq, int lane, bool ok)
 {
     const int g = lane >> 2, q = lane & 3;
 #pragma unroll
@@ -145,7 +172,7 @@ __device__ __forceinline__ void scan_rows(float (&v)[2][4], uint32_t tot, int sp
             *reinterpret_cast<float2*>(__cvta_shared_to_generic((size_t)(tot + 4 * (sp * 64 + 16 * cq + 8 * n + 2 * q)))) =
                 REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]);
     }
-    __syncthreads();
+    ok = cbar_and(ok);
 #pragma unroll
     for (int o = 0; o < 4; ++o) {
         if (REV ? o > sp : o < sp) {
@@ -156,6 +183,7 @@ __device__ __forceinline__ void scan_rows(float (&v)[2][4], uint32_t tot, int sp
             }
         }
     }
+    return ok;
 }
 
 __global__ void __launch_bounds__(B_THREADS, 1)
@@ -199,24 +227,102 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const uint32_t tmem = lds32(sbase + BO_TMEM);
     const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 16 * cq;      // this warp's block of an accumulator
 
-    // A wait by warp 0 whose outcome every thread of the CTA learns (contains a CTA barrier).
-    auto wait_all = [&](uint32_t b, uint32_t parity) -> bool {
-        bool ok = true;
-        if (warp == 0) ok = mbar_wait_warp(b, parity, abort_flag);
-        ok = __syncthreads_and(ok);
-        if (ok) mbar_try_wait(b, parity);            // (completed: every thread observes the phase itself)
-        return ok;
+    // Chunks are numbered by iteration: iteration `it` handles chunk nchunks - 1 - it; its input stage and the
+    // double-buffered operand tiles are those of parity it & 1.
+    auto chunk_of = [&](int it) { return nchunks - 1 - it; };
+
+    if (warp == B_CTHREADS / 32) {
+        // ============================== issuing warp ==============================
+        // One lane takes commands from the compute warps (a ring of four slots, one mbarrier each: at most three
+        // are ever outstanding) and issues what they ask for: the two groups of products of a chunk, and the TMA
+        // stores of a chunk's gradient tiles followed by the input copies of the chunk two iterations on.  The compute
+        // warps never wait for an instruction to be issued, only for its completion.
+        if (lane == 0) {
+            auto issue_loads = [&](int it) {
+                const int stage = it & 1;
+                const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
+                const int row = (int)(row0 + (long long)chunk_of(it) * L);
+                mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
+                tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
+                tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
+                tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
+                tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
+                tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
+            };
+            int last_load[2] = {-1, -1};             // per stage: the last iteration whose input copies were issued
+            if (nchunks > 0) { issue_loads(0); last_load[0] = 0; }
+            if (nchunks > 1) { issue_loads(1); last_load[1] = 1; }
+            for (int kc = 0;; ++kc) {
+                if (!mbar_wait(bar(BB_CMD + (kc & 3)), (kc >> 2) & 1, abort_flag)) break;
+                const uint32_t cmd = lds32(sbase + BO_CMD + 8 * (kc & 3)), arg = lds32(sbase + BO_CMD + 8 * (kc & 3) + 4);
+                if (cmd == CMD_QUIT) break;
+                if (cmd == CMD_MMA1 || cmd == CMD_MMA2) {
+                    const int pb = (int)arg;
+                    const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
+                    const uint64_t dR = smem_desc(sbase + BO_RH + pb * TILE), dK = smem_desc(sbase + BO_KH + pb * TILE);
+                    const uint64_t dV = smem_desc(tin + 3 * TILE), dY = smem_desc(tin + 4 * TILE);
+                    tc_fence_after();
+                    if (cmd == CMD_MMA1) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
+                            tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
+                            tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
+                            tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                        }
+                        tc_commit(bar(BB_MMA1));
+                    } else {
+                        const uint64_t dS = smem_desc(sbase + BO_SB + pb * TILE), dG = smem_desc(sbase + BO_GB + pb * TILE);
+                        const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t ks = 2 * kk, ms = 128 * kk;
+                            tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                            tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
+                            tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
+                        }
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint64_t ks = 2 * kk, ms = 128 * kk;
+                            tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                            tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
+                            tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
+                        }
+                        tc_commit(bar(BB_MMA2));
+                    }
+                } else {                             // CMD_STORE: arg = iteration, bit 31: whole chunk (TMA stores)
+                    const int it = (int)(arg & 0x7fffffffu);
+                    const bool whole = (arg >> 31) != 0;
+                    if (whole) {
+                        const int row = (int)(row0 + (long long)chunk_of(it) * L);
+                        tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
+                        tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
+                        tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
+                        tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
+                        bulk_commit();
+                    }
+                    if (it + 2 < nchunks) { issue_loads(it + 2); last_load[it & 1] = it + 2; }
+                    if (whole) bulk_wait_read<0>();  // the staging tiles may be rewritten
+                    mbar_arrive(bar(BB_STAGING));
+                }
+            }
+            bulk_wait<0>();                          // the gradient tiles have reached memory
+            for (int s2 = 0; s2 < 2; ++s2)           // no copy into this CTA's shared memory may stay in flight
+                if (last_load[s2] >= 0) mbar_wait(bar(BB_IN + s2), (last_load[s2] >> 1) & 1, abort_flag, false);
+        }
+    } else {
+    // ============================== compute warps ==============================
+    // Every thread waits for itself on an mbarrier; the outcomes are made uniform at the next barrier of the compute
+    // warps (cbar_and), so that after a wait that ran out all of them leave together.
+    int n_cmd = 0;                                   // (thread 0) commands posted so far
+    auto post = [&](uint32_t cmd, uint32_t arg) {    // thread 0, after a barrier that follows the operands' writes
+        const uint32_t slot = sbase + BO_CMD + 8 * (n_cmd & 3);
+        sts32(slot, cmd);
+        sts32(slot + 4, arg);
+        mbar_arrive(bar(BB_CMD + (n_cmd & 3)));
+        ++n_cmd;
     };
-    auto issue_loads = [&](int c, int stage) {       // one thread
-        const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
-        const int row = (int)(row0 + (long long)c * L);
-        mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
-        tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
-    };
+    int n_store = 0;                                 // store commands posted so far (every thread counts)
     auto load_f32_block = [&](const float* src, float (&v)[2][4]) {      // [64][64] fp32 block, accumulator layout
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
@@ -237,20 +343,22 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         for (int n = 0; n < 2; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
     }
     load_f32_block(ck_unit + (size_t)nchunks * 4096, SL);
-    if (tid == 0 && nchunks > 0) issue_loads(nchunks - 1, 0);
-    int pend = nchunks > 0 ? 0 : -1;                 // (thread 0) iteration whose input copies may still be in flight
-    int mph = 0;                                     // phase bit of the two product barriers (one phase per chunk on this path)
+    int mph1 = 0, mph2 = 0;                          // phase bits of the two product barriers
     bool alive = true;
 
-    for (int it = 0; it < nchunks; ++it) {
-        const int c = nchunks - 1 - it, stage = it & 1;
+    // ---- operands of a chunk from its inputs and from the adjoint G = G_L at its end; first group of products.
+    // Returns 0 (products issued), 1 (the chunk decays too fast for this form: nothing issued) or -1 (a wait ran out).
+    // On return SL holds the chunk's start state; a, lw2 its cumulative and per-token log2 decays in this lane's cells.
+    auto prepare = [&](int it, float (&a)[2][4], float (&lw2)[2][4], float (&dch)[2]) -> int {
+        const int c = chunk_of(it), pb = it & 1;
         const int valid = min(L, T - c * L);
-        const uint32_t tin = sbase + BO_IN + stage * B_STAGE;
+        const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
         const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
-        if (tid == 0) sts32(sbase + BO_FLAG, 0u);
+        const uint32_t t_rh = sbase + BO_RH + pb * TILE, t_kh = sbase + BO_KH + pb * TILE;
+        const uint32_t t_sb = sbase + BO_SB + pb * TILE, t_gb = sbase + BO_GB + pb * TILE;
         float S0[2][4];
         load_f32_block(ck_unit + (size_t)c * 4096, S0);
-        // ---- E = rowsum(G_L * S_L): partial over this lane's columns, then over the four lanes of a row
+        // E = rowsum(G_L * S_L): partial over this lane's columns, then over the four lanes of a row
         {
             float e0 = 0.f, e1 = 0.f;
 #pragma unroll
@@ -260,22 +368,17 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             }
             e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
             e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
-            if (q == 0) { fsm(BO_EP)[cq * 64 + R0] = e0; fsm(BO_EP)[cq * 64 + R1] = e1; }
+            if (q == 0) { fsm(BO_EP)[(pb * 4 + cq) * 64 + R0] = e0; fsm(BO_EP)[(pb * 4 + cq) * 64 + R1] = e1; }
         }
-        if (!wait_all(bar(BB_IN + stage), (it >> 1) & 1)) { alive = false; break; }
-        if (tid == 0) {
-            pend = -1;
-            if (c > 0) { issue_loads(c - 1, stage ^ 1); pend = it + 1; }
-        }
+        bool ok = mbar_wait(bar(BB_IN + pb), (it >> 1) & 1, abort_flag);
         if (valid < L) {
             // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
-            for (int i = tid; i < (L - valid) * 8; i += B_THREADS) {
+            for (int i = tid; i < (L - valid) * 8; i += B_CTHREADS) {
                 const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
                 sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
             }
         }
-        // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
-        float lw2[2][4], a[2][4];
+        // decay: log2-domain magnitudes, cumulative sums over the tokens
         {
             float xv[2][4];
             load_block_bf16(tx + moff, xv);
@@ -288,191 +391,107 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     a[n][e] = lw2[n][e];
                 }
         }
-        scan_rows<false>(a, sbase + BO_TOT, sp, cq, lane);       // (barrier: the zeroed rows are visible after it)
-        float sr[2][4], sk[2][4], rv[2][4], kv[2][4];
-        load_block_bf16(tr + moff, rv);
-        load_block_bf16(tk + moff, kv);
+        ok = scan_rows<false>(a, sbase + BO_TOT, sp, cq, lane, ok);      // (barrier: the zeroed rows are visible after it)
+        if (!ok) return -1;
+        // a_L = the sum of the four row-group totals; this lane needs it for the channels that are its rows of G
+        bool safe;
         {
-            float rh[2][4], kh[2][4];
+            float al0 = 0.f, al1 = 0.f;
+#pragma unroll
+            for (int o = 0; o < 4; ++o) { al0 += fsm(BO_TOT)[o * 64 + R0]; al1 += fsm(BO_TOT)[o * 64 + R1]; }
+            dch[0] = ex2(al0); dch[1] = ex2(al1);
+            safe = (al0 >= -A2_MAX) && (al1 >= -A2_MAX);                   // false for NaN as well
+        }
+        {
+            float rv[2][4], kv[2][4];
+            load_block_bf16(tr + moff, rv);
+            load_block_bf16(tk + moff, kv);
             float b0 = 0.f, b1 = 0.f;
 #pragma unroll
             for (int n = 0; n < 2; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    sr[n][e] = ex2(a[n][e] - lw2[n][e]);
-                    sk[n][e] = ex2(-a[n][e]);
-                    rh[n][e] = rv[n][e] * sr[n][e];
-                    kh[n][e] = kv[n][e] * sk[n][e];
                     const float t = rv[n][e] * kv[n][e] * uu[n][e & 1];
                     if (e < 2) b0 += t; else b1 += t;
+                    rv[n][e] *= ex2(a[n][e] - lw2[n][e]);
+                    kv[n][e] *= ex2(-a[n][e]);
                 }
-            store_block_bf16(sbase + BO_RH + moff, rh);
-            store_block_bf16(sbase + BO_KH + moff, kh);
+            store_block_bf16(t_rh + moff, rv);
+            store_block_bf16(t_kh + moff, kv);
             b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
             b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
             if (q == 0) { fsm(BO_BP)[cq * 64 + R0] = b0; fsm(BO_BP)[cq * 64 + R1] = b1; }
         }
-        if (sp == 3 && g == 7) {                     // row 63 holds a_L
-            bool ok = true;
+        store_block_bf16(t_sb + moff, S0);
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) SL[n][e] = S0[n][e];
+        {
+            float gh[2][4];
 #pragma unroll
             for (int n = 0; n < 2; ++n) {
-                fsm(BO_D)[cb + 8 * n] = ex2(a[n][2]);
-                fsm(BO_D)[cb + 8 * n + 1] = ex2(a[n][3]);
-                ok = ok && (a[n][2] >= -A2_MAX) && (a[n][3] >= -A2_MAX);      // false for NaN as well
+                gh[n][0] = dch[0] * G[n][0]; gh[n][1] = dch[0] * G[n][1];
+                gh[n][2] = dch[1] * G[n][2]; gh[n][3] = dch[1] * G[n][3];
             }
-            if (!ok) sts32(sbase + BO_FLAG, 1u);
+            store_block_bf16(t_gb + moff, gh);
         }
-        store_block_bf16(sbase + BO_SB + moff, S0);
-        __syncthreads();
-        const bool unsafe = lds32(sbase + BO_FLAG) != 0;
-        const float d_lo = fsm(BO_D)[R0], d_hi = fsm(BO_D)[R1];      // decay of the chunk for this lane's rows of G
+        fence_proxy_async();
+        tc_fence_before();
+        const bool unsafe = !cbar_and(safe);         // (every channel is some lane's row)
+        if (tid == 0 && !unsafe) post(CMD_MMA1, (uint32_t)pb);
+        return unsafe ? 1 : 0;
+    };
 
-        if (!unsafe) {
-            {
-                float gh[2][4];
-#pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    gh[n][0] = d_lo * G[n][0]; gh[n][1] = d_lo * G[n][1];
-                    gh[n][2] = d_hi * G[n][2]; gh[n][3] = d_hi * G[n][3];
-                }
-                store_block_bf16(sbase + BO_GB + moff, gh);
+    // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one; then the
+    // input stage of this iteration is free for the chunk two iterations on.
+    auto store_and_refill = [&](int it) {
+        const int c = chunk_of(it), valid = min(L, T - c * L);
+        fence_proxy_async();
+        cbar();
+        if (valid < L) {
+            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
+            for (int i = tid; i < 4 * valid * 8; i += B_CTHREADS) {
+                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
+                uint32_t w[4];
+                lds_v4(sbase + BO_OUT + tile * TILE + swz(t, blk << 4), w);
+                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            fence_proxy_async();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-                const uint64_t dR = smem_desc(sbase + BO_RH), dK = smem_desc(sbase + BO_KH), dV = smem_desc(tv), dY = smem_desc(tdy);
-                const uint64_t dS = smem_desc(sbase + BO_SB), dG = smem_desc(sbase + BO_GB);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
-                    tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
-                    tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
-                    tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
-                    tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
-                    tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
-                    tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
-                }
-                tc_commit(bar(BB_MMA1));
-            }
-            if (!wait_all(bar(BB_MMA1), mph)) { alive = false; break; }
-            tc_fence_after();
-            // ---- masked scores and their adjoint as operands
-            {
-                float pp[2][4], dp[2][4];
-                tmem_ld_16x16(tacc + BT_P, pp);
-                tmem_ld_16x16(tacc + BT_DP, dp);
-                float bon0 = 0.f, bon1 = 0.f;
-                if (cq == sp) {
-#pragma unroll
-                    for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
-                }
-#pragma unroll
-                for (int n = 0; n < 2; ++n)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int row = e < 2 ? R0 : R1, col = cb + 8 * n + (e & 1);
-                        if (col == row) fsm(BO_DPD)[row] = dp[n][e];
-                        pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
-                        dp[n][e] = col < row ? dp[n][e] : 0.f;
-                    }
-                store_block_bf16(sbase + BO_PP + moff, pp);
-                store_block_bf16(sbase + BO_DPP + moff, dp);
-            }
-            fence_proxy_async();
-            tc_fence_before();
-            __syncthreads();
-            if (tid == 0) {
-                tc_fence_after();
-                const uint64_t dR = smem_desc(sbase + BO_RH), dK = smem_desc(sbase + BO_KH), dY = smem_desc(tdy);
-                const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;
-                    tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
-                    tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
-                    tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
-                }
-                tc_commit(bar(BB_MMA2));
-            }
-            // ---- meanwhile: G_0 = diag(D) G_L + R^^T dY
-            {
-                float dg[2][4];
-                tmem_ld_16x16(tacc + BT_DG, dg);
-#pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
-                    G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
-                }
-            }
-            if (!wait_all(bar(BB_MMA2), mph)) { alive = false; break; }
-            tc_fence_after();
-            mph ^= 1;
-            // ---- epilogue
-            float z[2][4], qv[2][4];
-            {
-                // q and m take the operands as the tensor core saw them (rounded to bf16): the pair terms that q and
-                // m share, and that cancel in the suffix sums, are then the same products on both sides
-                float acc[2][4], o[2][4], hat[2][4];
-                const float pd0 = fsm(BO_DPD)[R0], pd1 = fsm(BO_DPD)[R1];
-                tmem_ld_16x16(tacc + BT_DR, acc);
-                load_block_bf16(sbase + BO_RH + moff, hat);
-#pragma unroll
-                for (int n = 0; n < 2; ++n)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float pd = e < 2 ? pd0 : pd1;
-                        o[n][e] = fmaf(uu[n][e & 1] * kv[n][e], pd, acc[n][e] * sr[n][e]);
-                        qv[n][e] = acc[n][e] * hat[n][e];
-                        du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
-                    }
-                store_block_bf16(sbase + BO_OUT + moff, o);
-                tmem_ld_16x16(tacc + BT_DK, acc);
-                load_block_bf16(sbase + BO_KH + moff, hat);
-#pragma unroll
-                for (int n = 0; n < 2; ++n)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float pd = e < 2 ? pd0 : pd1;
-                        o[n][e] = fmaf(uu[n][e & 1] * rv[n][e], pd, acc[n][e] * sk[n][e]);
-                        z[n][e] = qv[n][e] - acc[n][e] * hat[n][e];
-                    }
-                store_block_bf16(sbase + BO_OUT + TILE + moff, o);
-                tmem_ld_16x16(tacc + BT_DV, acc);
-                store_block_bf16(sbase + BO_OUT + 2 * TILE + moff, acc);
-            }
-            tc_fence_before();
-            scan_rows<true>(z, sbase + BO_TOT, sp, cq, lane);
-            {
-                float o[2][4];
-#pragma unroll
-                for (int n = 0; n < 2; ++n) {
-                    float E0 = 0.f, E1 = 0.f;
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) { E0 += fsm(BO_EP)[w * 64 + cb + 8 * n]; E1 += fsm(BO_EP)[w * 64 + cb + 8 * n + 1]; }
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        o[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
-                }
-                store_block_bf16(sbase + BO_OUT + 3 * TILE + moff, o);
-            }
-        } else {
+        }
+        if (tid == 0) post(CMD_STORE, (uint32_t)it | (valid == L ? 0x80000000u : 0u));
+        ++n_store;
+    };
+    // The staging tiles may be rewritten once the TMA unit has read the previous chunk's (a barrier of the compute
+    // warps follows in every caller, which also orders a ragged chunk's plain reads before the rewrite).
+    auto staging_free = [&]() -> bool { return n_store == 0 || mbar_wait(bar(BB_STAGING), (n_store - 1) & 1, abort_flag); };
+
+    float a_cur[2][4], lw_cur[2][4], d_cur[2];       // of the chunk in flight: cumulative / per-token log2 decays, chunk decay
+    int st = nchunks > 0 ? prepare(0, a_cur, lw_cur, d_cur) : 0;
+    if (st < 0) alive = false;
+
+    for (int it = 0; alive && it < nchunks; ++it) {
+        const int c = chunk_of(it), pb = it & 1;
+        const int valid = min(L, T - c * L);
+        const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
+        const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
+        const uint32_t t_rh = sbase + BO_RH + pb * TILE, t_kh = sbase + BO_KH + pb * TILE;
+
+        if (st == 1) {
             // ---- token by token: the chunk's states recomputed into this SM's scratch, then the reverse recurrence
             const unsigned slot = smid();
             if (slot >= (unsigned)p.n_slots) {       // (no scratch for this SM: report it and leave)
                 if (tid == 0) { sts32(abort_flag, 1u); atomicExch(&g_dev_status, 1); }
                 alive = false;
-                __syncthreads();
                 break;
             }
+            if (!cbar_and(staging_free())) { alive = false; break; }
             float* scr = p.fb_scratch + (size_t)slot * FB_SLOT_FLOATS + (size_t)tid * 8;
             // rows are key channels here: this lane's channels R0, R1 of S and G; its columns are value channels
             float S[2][4];
 #pragma unroll
             for (int n = 0; n < 2; ++n)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) S[n][e] = S0[n][e];
+                for (int e = 0; e < 4; ++e) S[n][e] = SL[n][e];
             for (int t = 0; t < valid; ++t) {
                 *reinterpret_cast<float4*>(scr + (size_t)t * 4096) = make_float4(S[0][0], S[0][1], S[0][2], S[0][3]);
                 *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4) = make_float4(S[1][0], S[1][1], S[1][2], S[1][3]);
@@ -550,7 +569,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     }
                     if (lane == 0) { scal[0] = vd; scal[1] = ruk; }
                 }
-                __syncthreads();
+                cbar();
                 if (tid < 64) {
                     const int cc = tid;
                     float s_r = 0.f, s_k = 0.f, s_g = 0.f;
@@ -567,38 +586,134 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
                     sts_bf16(sbase + BO_OUT + 2 * TILE + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
                 }
-                __syncthreads();
+                cbar();
             }
+            store_and_refill(it);
+            if (it + 1 < nchunks) {
+                st = prepare(it + 1, a_cur, lw_cur, d_cur);
+                if (st < 0) alive = false;
+            }
+            continue;
         }
-        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one
+
+        // ---- masked scores and their adjoint as operands
+        bool ok = mbar_wait(bar(BB_MMA1), mph1, abort_flag);
+        mph1 ^= 1;
+        tc_fence_after();
+        {
+            float pp[2][4], dp[2][4];
+            tmem_ld_16x16_async(tacc + BT_P, pp);
+            tmem_ld_16x16_async(tacc + BT_DP, dp);
+            tmem_ld_done();
+            float bon0 = 0.f, bon1 = 0.f;
+            if (cq == sp) {
+#pragma unroll
+                for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
+            }
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int row = e < 2 ? R0 : R1, col = cb + 8 * n + (e & 1);
+                    if (col == row) fsm(BO_DPD)[row] = dp[n][e];
+                    pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
+                    dp[n][e] = col < row ? dp[n][e] : 0.f;
+                }
+            store_block_bf16(sbase + BO_PP + moff, pp);
+            store_block_bf16(sbase + BO_DPP + moff, dp);
+        }
         fence_proxy_async();
-        __syncthreads();
-        if (valid == L) {
-            if (tid == 0) {
-                const int row = (int)(row0 + (long long)c * L);
-                tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
-                tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
-                tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
-                tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
-                bulk_commit();
-                bulk_wait_read<0>();                 // the staging tiles are rewritten next chunk
+        tc_fence_before();
+        if (!cbar_and(ok)) { alive = false; break; }
+        if (tid == 0) post(CMD_MMA2, (uint32_t)pb);
+        // ---- G_0 = diag(D) G_L + R^^T dY
+        {
+            const float d_lo = d_cur[0], d_hi = d_cur[1];
+            float dg[2][4];
+            tmem_ld_16x16(tacc + BT_DG, dg);
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
+                G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
             }
-        } else {
-            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
-            for (int i = tid; i < 4 * valid * 8; i += B_THREADS) {
-                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
-                uint32_t w[4];
-                lds_v4(sbase + BO_OUT + tile * TILE + swz(t, blk << 4), w);
-                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+            tc_fence_before();
         }
-        __syncthreads();
+        // ---- while the second group of products runs: the next chunk's operands and its first group of products
+        float a_nxt[2][4], lw_nxt[2][4], d_nxt[2] = {0.f, 0.f};
+        int st_nxt = 0;
+        if (it + 1 < nchunks) {
+            st_nxt = prepare(it + 1, a_nxt, lw_nxt, d_nxt);
+            if (st_nxt < 0) { alive = false; break; }
+        }
+        ok = staging_free() & mbar_wait(bar(BB_MMA2), mph2, abort_flag);     // (made uniform at the barrier of the suffix sums)
+        mph2 ^= 1;
+        tc_fence_after();
+        // ---- epilogue
+        {
+            float z[2][4], qv[2][4];
+            {
+                // q and m take the operands as the tensor core saw them (rounded to bf16): the pair terms that q and
+                // m share, and that cancel in the suffix sums, are then the same products on both sides
+                float acc[2][4], o[2][4], hat[2][4], rv[2][4], kv[2][4];
+                const float pd0 = fsm(BO_DPD)[R0], pd1 = fsm(BO_DPD)[R1];
+                float acc2[2][4], acc3[2][4];
+                tmem_ld_16x16_async(tacc + BT_DR, acc);
+                tmem_ld_16x16_async(tacc + BT_DK, acc2);
+                tmem_ld_16x16_async(tacc + BT_DV, acc3);
+                load_block_bf16(tr + moff, rv);
+                load_block_bf16(tk + moff, kv);
+                load_block_bf16(t_rh + moff, hat);
+                tmem_ld_done();
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float pd = e < 2 ? pd0 : pd1;
+                        o[n][e] = fmaf(uu[n][e & 1] * kv[n][e], pd, acc[n][e] * ex2(a_cur[n][e] - lw_cur[n][e]));
+                        qv[n][e] = acc[n][e] * hat[n][e];
+                        du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
+                    }
+                store_block_bf16(sbase + BO_OUT + moff, o);
+                load_block_bf16(t_kh + moff, hat);
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float pd = e < 2 ? pd0 : pd1;
+                        o[n][e] = fmaf(uu[n][e & 1] * rv[n][e], pd, acc2[n][e] * ex2(-a_cur[n][e]));
+                        z[n][e] = qv[n][e] - acc2[n][e] * hat[n][e];
+                    }
+                store_block_bf16(sbase + BO_OUT + TILE + moff, o);
+                store_block_bf16(sbase + BO_OUT + 2 * TILE + moff, acc3);
+            }
+            tc_fence_before();
+            ok = scan_rows<true>(z, sbase + BO_TOT, sp, cq, lane, ok);
+            if (!ok) { alive = false; break; }
+            float o[2][4];
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                float E0 = 0.f, E1 = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    E0 += fsm(BO_EP)[(pb * 4 + w) * 64 + cb + 8 * n];
+                    E1 += fsm(BO_EP)[(pb * 4 + w) * 64 + cb + 8 * n + 1];
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    o[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw_cur[n][e] * LN2);
+            }
+            store_block_bf16(sbase + BO_OUT + 3 * TILE + moff, o);
+        }
+        store_and_refill(it);
 #pragma unroll
         for (int n = 0; n < 2; ++n)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) SL[n][e] = S0[n][e];
+            for (int e = 0; e < 4; ++e) { a_cur[n][e] = a_nxt[n][e]; lw_cur[n][e] = lw_nxt[n][e]; }
+        d_cur[0] = d_nxt[0]; d_cur[1] = d_nxt[1];
+        st = st_nxt;
     }
 
+    cbar();
     if (alive) {
         if (p.dstate_in) {
             float* dst = p.dstate_in + (size_t)unit * 4096;
@@ -621,17 +736,14 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
                 for (int e = 0; e < 2; ++e) fsm(BO_RED_V)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
         }
-        __syncthreads();
+        cbar();
         if (tid < 64) {
             const float* rv4 = fsm(BO_RED_V);
             p.du_part[(size_t)unit * 64 + tid] = ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fsm(BO_DU_FB)[tid];
         }
     }
-    if (tid == 0) {
-        bulk_wait<0>();                              // the gradient tiles have reached memory
-        if (pend >= 0)                               // (aborting) no copy into this CTA's shared memory may stay in flight
-            mbar_wait(bar(BB_IN + (pend & 1)), (pend >> 1) & 1, abort_flag, false);
-    }
+    if (tid == 0) post(CMD_QUIT, 0u);
+    }   // compute warps
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
