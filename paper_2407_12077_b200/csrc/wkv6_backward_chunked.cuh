@@ -34,8 +34,9 @@ namespace bc {
 
 using namespace ck;          // PTX wrappers, descriptors, layout helpers of the forward kernel
 
+constexpr bool B_ISSUER = false;                 // a 17th warp issues the products and the TMA copies (else thread 0 does)
 constexpr int B_CTHREADS = 512;                  // 16 compute warps
-constexpr int B_THREADS = B_CTHREADS + 32;       // and the warp that issues the products and the TMA copies
+constexpr int B_THREADS = B_CTHREADS + (B_ISSUER ? 32 : 0);
 constexpr float LN2 = 0.6931471805599453f;
 // tensor memory columns of the six accumulators
 constexpr int BT_P = 0, BT_DP = 64, BT_DV = 128, BT_DR = 192, BT_DK = 256, BT_DG = 320, BT_COLS = 512;
@@ -231,84 +232,96 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     // double-buffered operand tiles are those of parity it & 1.
     auto chunk_of = [&](int it) { return nchunks - 1 - it; };
 
-    if (warp == B_CTHREADS / 32) {
-        // ============================== issuing warp ==============================
-        // One lane takes commands from the compute warps (a ring of four slots, one mbarrier each: at most three
-        // are ever outstanding) and issues what they ask for: the two groups of products of a chunk, and the TMA
-        // stores of a chunk's gradient tiles followed by the input copies of the chunk two iterations on.  The compute
-        // warps never wait for an instruction to be issued, only for its completion.
-        if (lane == 0) {
-            auto issue_loads = [&](int it) {
-                const int stage = it & 1;
-                const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
+    // ---- issuing: the products, the TMA stores of a chunk's gradient tiles and the input copies.  With B_ISSUER a
+    // warp of its own does it: one lane takes commands from the compute warps (a ring of four slots, one mbarrier each:
+    // at most three are ever outstanding), so that no compute warp waits for an instruction to be issued, only for
+    // its completion.  Without it thread 0 issues in place.
+    int last_load[2] = {-1, -1};                     // (issuing thread) per stage: the last iteration whose copies were issued
+    auto issue_loads = [&](int it) {
+        const int stage = it & 1;
+        const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
+        const int row = (int)(row0 + (long long)chunk_of(it) * L);
+        mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
+        tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
+        tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
+        last_load[stage] = it;
+    };
+    auto execute = [&](uint32_t cmd, uint32_t arg) {
+        if (cmd == CMD_MMA1 || cmd == CMD_MMA2) {
+            const int pb = (int)arg;
+            const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
+            const uint64_t dR = smem_desc(sbase + BO_RH + pb * TILE), dK = smem_desc(sbase + BO_KH + pb * TILE);
+            const uint64_t dV = smem_desc(tin + 3 * TILE), dY = smem_desc(tin + 4 * TILE);
+            tc_fence_after();
+            if (cmd == CMD_MMA1) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
+                    tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
+                    tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
+                    tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                }
+                tc_commit(bar(BB_MMA1));
+            } else {
+                const uint64_t dS = smem_desc(sbase + BO_SB + pb * TILE), dG = smem_desc(sbase + BO_GB + pb * TILE);
+                const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                    tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
+                    tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                    tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
+                    tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
+                }
+                tc_commit(bar(BB_MMA2));
+            }
+        } else {                             // CMD_STORE: arg = iteration, bit 31: whole chunk (TMA stores)
+            const int it = (int)(arg & 0x7fffffffu);
+            const bool whole = (arg >> 31) != 0;
+            if (whole) {
                 const int row = (int)(row0 + (long long)chunk_of(it) * L);
-                mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
-                tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
-                tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
-                tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
-                tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
-                tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
-            };
-            int last_load[2] = {-1, -1};             // per stage: the last iteration whose input copies were issued
-            if (nchunks > 0) { issue_loads(0); last_load[0] = 0; }
-            if (nchunks > 1) { issue_loads(1); last_load[1] = 1; }
+                tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
+                tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
+                tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
+                tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
+                bulk_commit();
+            }
+            if (it + 2 < nchunks) issue_loads(it + 2);
+            if (B_ISSUER) {
+                if (whole) bulk_wait_read<0>();      // the staging tiles may be rewritten
+                mbar_arrive(bar(BB_STAGING));
+            }
+        }
+    };
+    auto issuer_done = [&]() {
+        bulk_wait<0>();                              // the gradient tiles have reached memory
+        for (int s2 = 0; s2 < 2; ++s2)               // no copy into this CTA's shared memory may stay in flight
+            if (last_load[s2] >= 0) mbar_wait(bar(BB_IN + s2), (last_load[s2] >> 1) & 1, abort_flag, false);
+    };
+    if (B_ISSUER ? (warp == B_CTHREADS / 32 && lane == 0) : tid == 0) {
+        if (nchunks > 0) issue_loads(0);
+        if (nchunks > 1) issue_loads(1);
+    }
+
+    if (B_ISSUER && warp == B_CTHREADS / 32) {
+        // ============================== issuing warp ==============================
+        if (lane == 0) {
             for (int kc = 0;; ++kc) {
                 if (!mbar_wait(bar(BB_CMD + (kc & 3)), (kc >> 2) & 1, abort_flag)) break;
                 const uint32_t cmd = lds32(sbase + BO_CMD + 8 * (kc & 3)), arg = lds32(sbase + BO_CMD + 8 * (kc & 3) + 4);
                 if (cmd == CMD_QUIT) break;
-                if (cmd == CMD_MMA1 || cmd == CMD_MMA2) {
-                    const int pb = (int)arg;
-                    const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
-                    const uint64_t dR = smem_desc(sbase + BO_RH + pb * TILE), dK = smem_desc(sbase + BO_KH + pb * TILE);
-                    const uint64_t dV = smem_desc(tin + 3 * TILE), dY = smem_desc(tin + 4 * TILE);
-                    tc_fence_after();
-                    if (cmd == CMD_MMA1) {
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
-                            tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
-                            tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
-                            tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
-                        }
-                        tc_commit(bar(BB_MMA1));
-                    } else {
-                        const uint64_t dS = smem_desc(sbase + BO_SB + pb * TILE), dG = smem_desc(sbase + BO_GB + pb * TILE);
-                        const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t ks = 2 * kk, ms = 128 * kk;
-                            tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
-                            tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
-                            tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
-                        }
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t ks = 2 * kk, ms = 128 * kk;
-                            tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
-                            tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
-                            tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
-                        }
-                        tc_commit(bar(BB_MMA2));
-                    }
-                } else {                             // CMD_STORE: arg = iteration, bit 31: whole chunk (TMA stores)
-                    const int it = (int)(arg & 0x7fffffffu);
-                    const bool whole = (arg >> 31) != 0;
-                    if (whole) {
-                        const int row = (int)(row0 + (long long)chunk_of(it) * L);
-                        tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
-                        tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
-                        tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
-                        tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
-                        bulk_commit();
-                    }
-                    if (it + 2 < nchunks) { issue_loads(it + 2); last_load[it & 1] = it + 2; }
-                    if (whole) bulk_wait_read<0>();  // the staging tiles may be rewritten
-                    mbar_arrive(bar(BB_STAGING));
-                }
+                execute(cmd, arg);
             }
-            bulk_wait<0>();                          // the gradient tiles have reached memory
-            for (int s2 = 0; s2 < 2; ++s2)           // no copy into this CTA's shared memory may stay in flight
-                if (last_load[s2] >= 0) mbar_wait(bar(BB_IN + s2), (last_load[s2] >> 1) & 1, abort_flag, false);
+            issuer_done();
         }
     } else {
     // ============================== compute warps ==============================
@@ -316,6 +329,10 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     // warps (cbar_and), so that after a wait that ran out all of them leave together.
     int n_cmd = 0;                                   // (thread 0) commands posted so far
     auto post = [&](uint32_t cmd, uint32_t arg) {    // thread 0, after a barrier that follows the operands' writes
+        if (!B_ISSUER) {
+            if (cmd != CMD_QUIT) execute(cmd, arg); else issuer_done();
+            return;
+        }
         const uint32_t slot = sbase + BO_CMD + 8 * (n_cmd & 3);
         sts32(slot, cmd);
         sts32(slot + 4, arg);
@@ -358,6 +375,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         const uint32_t t_sb = sbase + BO_SB + pb * TILE, t_gb = sbase + BO_GB + pb * TILE;
         float S0[2][4];
         load_f32_block(ck_unit + (size_t)c * 4096, S0);
+        if (c > 0 && tid < 128)                      // the next chunk's start state: in L2 by the time it is loaded
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 1) * 4096 + 32 * tid));
         // E = rowsum(G_L * S_L): partial over this lane's columns, then over the four lanes of a row
         {
             float e0 = 0.f, e1 = 0.f;
@@ -463,7 +482,13 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     };
     // The staging tiles may be rewritten once the TMA unit has read the previous chunk's (a barrier of the compute
     // warps follows in every caller, which also orders a ragged chunk's plain reads before the rewrite).
-    auto staging_free = [&]() -> bool { return n_store == 0 || mbar_wait(bar(BB_STAGING), (n_store - 1) & 1, abort_flag); };
+    auto staging_free = [&]() -> bool {
+        if (!B_ISSUER) {                             // thread 0 issued the stores itself: it waits for their reads
+            if (tid == 0) bulk_wait_read<0>();
+            return true;
+        }
+        return n_store == 0 || mbar_wait(bar(BB_STAGING), (n_store - 1) & 1, abort_flag);
+    };
 
     float a_cur[2][4], lw_cur[2][4], d_cur[2];       // of the chunk in flight: cumulative / per-token log2 decays, chunk decay
     int st = nchunks > 0 ? prepare(0, a_cur, lw_cur, d_cur) : 0;
@@ -600,22 +625,32 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         bool ok = mbar_wait(bar(BB_MMA1), mph1, abort_flag);
         mph1 ^= 1;
         tc_fence_after();
-        {
+        if (cq < sp) {
+            // a block below the diagonal: every score and every adjoint entry is kept
             float pp[2][4], dp[2][4];
             tmem_ld_16x16_async(tacc + BT_P, pp);
             tmem_ld_16x16_async(tacc + BT_DP, dp);
             tmem_ld_done();
+            store_block_bf16(sbase + BO_PP + moff, pp);
+            store_block_bf16(sbase + BO_DPP + moff, dp);
+        } else if (cq > sp) {
+            // above the diagonal: masked out
+            stsm_x4(sbase + BO_PP + moff, 0u, 0u, 0u, 0u);
+            stsm_x4(sbase + BO_DPP + moff, 0u, 0u, 0u, 0u);
+        } else {
+            float pp[2][4], dp[2][4];
+            tmem_ld_16x16_async(tacc + BT_P, pp);
+            tmem_ld_16x16_async(tacc + BT_DP, dp);
             float bon0 = 0.f, bon1 = 0.f;
-            if (cq == sp) {
 #pragma unroll
-                for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
-            }
+            for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
+            tmem_ld_done();
 #pragma unroll
             for (int n = 0; n < 2; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int row = e < 2 ? R0 : R1, col = cb + 8 * n + (e & 1);
-                    if (col == row) fsm(BO_DPD)[row] = dp[n][e];
+                    const int row = e < 2 ? g : g + 8, col = 2 * q + 8 * n + (e & 1);       // inside the 16 x 16 block
+                    if (col == row) fsm(BO_DPD)[16 * sp + row] = dp[n][e];
                     pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
                     dp[n][e] = col < row ? dp[n][e] : 0.f;
                 }
