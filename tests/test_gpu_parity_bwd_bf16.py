@@ -82,6 +82,38 @@ def test_cfg1_shape_every_unit():
     print(_run(c["B"], c["T"], c["H"], seed=1000, state_std=c["state_std"], with_dstate=True))
 
 
+def test_cfg2_shape_every_unit_at_the_benchmarked_size():
+    """The launch the benchmark's gradient row times (B=4, T=16384, H=32: 256 chunks per CTA), every unit and every
+    token against the oracle, one batch entry at a time on the CPU side."""
+    c = synth.CONFIGS["cfg2"]
+    B, T, H = c["B"], c["T"], c["H"]
+    inp, dy, dsT = _inputs(B, T, H, 2100, 0.1, True)
+    d = inp.to(DEV)
+    out = gf.backward(d.r, d.k, d.v, d.x, d.u, dy.to(DEV), d.state_in, dsT.to(DEV))
+    gf.last_device_status()
+    out = [t.cpu() for t in out]
+    du_ref = np.zeros((H, 64))
+    for b in range(B):
+        sl = slice(b, b + 1)
+        ref = orc.backward(inp.r[sl], inp.k[sl], inp.v[sl], inp.x[sl], inp.u, dy[sl].double().numpy(), inp.state_in[sl],
+                           dsT[sl].double().numpy())
+        du_ref += ref[4]
+        part = [out[0][sl], out[1][sl], out[2][sl], out[3][sl], None, out[5][sl]]
+        for name, a, r in zip(NAMES, part, ref):
+            if a is None:
+                continue
+            a = a.float().numpy().astype(np.float64)
+            assert np.isfinite(a).all(), (b, name)
+            lim = TOL_DX if name == "dx" else TOL
+            assert orc.rel_l2(a, r) <= lim, (b, name, orc.rel_l2(a, r))
+            if name != "dstate_in":
+                row = ((a - r) ** 2).sum(axis=3)
+                num, den = row.sum(axis=1), (r * r).sum(axis=(1, 3))
+                assert np.sqrt(num / den).max() <= lim, (b, name, "unit")
+                assert np.sqrt(row.max(axis=1) / (den / T)).max() <= TOK_TOL, (b, name, "token")
+    assert orc.rel_l2(out[4].numpy(), du_ref) <= TOL
+
+
 @pytest.mark.parametrize("x_lo,x_hi", [(-12.0, -8.0), (-4.0, -1.0), (-3.0, 0.5), (-2.0, 0.0)])
 def test_slow_to_fast_decays_on_the_tensor_cores(x_lo, x_hi):
     """From w close to one (state and adjoint reach across the whole sequence) to decays close to the limit of the
