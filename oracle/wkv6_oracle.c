@@ -34,7 +34,9 @@
  * (tests/test_oracle_pins_dl.py: operator end points, an invertible outer lora that exposes the inner ddlerp, scalar
  * loops, library routines, a hand value, token-shift laws) and the gradient of the recurrence
  * (tests/test_oracle_pins_bwd.py: central differences of the forward pass, the one-token closed form, linearity,
- * split-and-carry of the adjoint).  No function here is unpinned.
+ * split-and-carry of the adjoint) and of its Finch-C2 form (tests/test_oracle_pins_bwd_c2.py: central differences, the
+ * reduction to the classic gradient on premultiplied keys with the chain rule written out, the one-token closed form).
+ * No function here is unpinned.
  *
  * Inputs arrive as float (an exact carrier for both fp32 and bf16 data) and are
  * widened to double before any arithmetic; every sum runs in double in plain
@@ -389,5 +391,91 @@ void wkv6_oracle_backward(const float *r, const float *k, const float *v, const 
             unit_backward(r + off, k + off, v + off, x + off, u + h * N, state_in ? state_in + soff : NULL,
                           dy + off, ds_T ? ds_T + soff : NULL, dr + off, dk + off, dv + off, dx + off,
                           du_b + ((size_t)b * H + h) * N, ds_0 ? ds_0 + soff : NULL, T, N, C);
+        }
+}
+
+/* ---------------------------------------------------------------------------------------------------
+ * Gradient of the Finch-C2 form (unit_recurrence_c2 above: keys k' = k (1 - w), no bonus, second-value
+ * vector added to the output), the layer the paper trains.  With G_t = dL/dS_t carried from t = T down
+ * (G_T given), every input's gradient is read off the forward formulas
+ *     y_t[j] = sum_i r_t[i] S_{t-1}[i][j] + u2_t[j],   S_t[i][j] = w_t[i] S_{t-1}[i][j] + k_t[i] (1 - w_t[i]) v_t[j]:
+ *     dr_t[i]  = sum_j dy_t[j] S_{t-1}[i][j]
+ *     dkp_t[i] = sum_j G_t[i][j] v_t[j]                      (gradient of the key that enters the state)
+ *     dk_t[i]  = dkp_t[i] (1 - w_t[i])
+ *     dv_t[j]  = sum_i G_t[i][j] k_t[i] (1 - w_t[i])
+ *     dw_t[i]  = sum_j G_t[i][j] S_{t-1}[i][j] - dkp_t[i] k_t[i]        (w_t scales the old state and shrinks the key)
+ *     dx_t[i]  = dw_t[i] * ( -w_t[i] exp(x_t[i]) )                       (w = exp(-exp(x)))
+ *     du2_t    = dy_t                                                    (not returned: it is the argument)
+ *     G_{t-1}[i][j] = w_t[i] G_t[i][j] + r_t[i] dy_t[j],   dS_0 = G_0.
+ * Pins (tests/test_oracle_pins_bwd_c2.py): central differences of the pinned forward oracle of this form, the
+ * reduction to the pinned gradient of the bonus-free recurrence on premultiplied keys plus the chain rule through
+ * k (1 - w), the one-token closed form, linearity in (dy, dS_T), split-and-carry of the adjoint.
+ */
+static void unit_backward_c2(const float *r, const float *k, const float *v, const float *x, const float *s_in,
+                             const double *dy, const double *ds_T, double *dr, double *dk, double *dv, double *dx,
+                             double *ds_0, long T, long N, long row_stride)
+{
+    const size_t NN = (size_t)N * N;
+    double *S_all = (double *)malloc((size_t)(T > 0 ? T : 1) * NN * sizeof(double));   /* S_{t-1} for t = 1..T */
+    double *S = (double *)malloc(NN * sizeof(double));
+    double *G = (double *)malloc(NN * sizeof(double));
+    for (size_t i = 0; i < NN; ++i) S[i] = s_in ? (double)s_in[i] : 0.0;
+    for (long t = 0; t < T; ++t) {
+        memcpy(S_all + (size_t)t * NN, S, NN * sizeof(double));
+        for (long i = 0; i < N; ++i) {
+            const double w = exp(-exp((double)x[t * row_stride + i]));
+            const double kp = (double)k[t * row_stride + i] * (1.0 - w);
+            for (long j = 0; j < N; ++j) S[i * N + j] = w * S[i * N + j] + kp * (double)v[t * row_stride + j];
+        }
+    }
+    for (size_t i = 0; i < NN; ++i) G[i] = ds_T ? ds_T[i] : 0.0;
+    for (long t = T - 1; t >= 0; --t) {
+        const float *rt = r + t * row_stride, *kt = k + t * row_stride, *vt = v + t * row_stride, *xt = x + t * row_stride;
+        const double *dyt = dy + t * row_stride, *Sp = S_all + (size_t)t * NN;
+        for (long i = 0; i < N; ++i) {
+            double a_r = 0.0, a_kp = 0.0, a_gs = 0.0;
+            for (long j = 0; j < N; ++j) {
+                a_r += dyt[j] * Sp[i * N + j];
+                a_kp += G[i * N + j] * (double)vt[j];
+                a_gs += G[i * N + j] * Sp[i * N + j];
+            }
+            const double ex = exp((double)xt[i]), w = exp(-ex);
+            dr[t * row_stride + i] = a_r;
+            dk[t * row_stride + i] = a_kp * (1.0 - w);
+            dx[t * row_stride + i] = (a_gs - a_kp * (double)kt[i]) * (-w * ex);
+        }
+        for (long j = 0; j < N; ++j) {
+            double a_v = 0.0;
+            for (long i = 0; i < N; ++i) {
+                const double w = exp(-exp((double)xt[i]));
+                a_v += G[i * N + j] * (double)kt[i] * (1.0 - w);
+            }
+            dv[t * row_stride + j] = a_v;
+        }
+        for (long i = 0; i < N; ++i) {
+            const double w = exp(-exp((double)xt[i]));
+            for (long j = 0; j < N; ++j) G[i * N + j] = w * G[i * N + j] + (double)rt[i] * dyt[j];
+        }
+    }
+    if (ds_0) memcpy(ds_0, G, NN * sizeof(double));
+    free(S_all);
+    free(S);
+    free(G);
+}
+
+/* Dense batch, layouts as wkv6_oracle_backward (no bonus, so no du). */
+void wkv6_oracle_backward_c2(const float *r, const float *k, const float *v, const float *x, const float *state_in,
+                             const double *dy, const double *ds_T, double *dr, double *dk, double *dv, double *dx,
+                             double *ds_0, long B, long T, long H, long N)
+{
+    const long C = H * N;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (long b = 0; b < B; ++b)
+        for (long h = 0; h < H; ++h) {
+            const size_t off = (size_t)b * T * C + (size_t)h * N;
+            const size_t soff = ((size_t)b * H + h) * N * N;
+            unit_backward_c2(r + off, k + off, v + off, x + off, state_in ? state_in + soff : NULL, dy + off,
+                             ds_T ? ds_T + soff : NULL, dr + off, dk + off, dv + off, dx + off,
+                             ds_0 ? ds_0 + soff : NULL, T, N, C);
         }
 }

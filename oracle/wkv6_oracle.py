@@ -262,6 +262,24 @@ def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None):
     return outs[0], outs[1], outs[2], outs[3], du_b.sum(axis=0), ds0
 
 
+def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None):
+    """Gradient of prefill_c2() (the Finch-C2 form: keys k (1 - w), no bonus; u2 only adds, so its gradient is dy
+    itself and is not returned).  Returns (dr, dk, dv, dx [B,T,H,N], dstate_in [B,H,N,N]) in float64."""
+    lib = _load()
+    r, k, v, x, state_in = _f32(r), _f32(k), _f32(v), _f32(x), _f32(state_in)
+    B, T, H, N = r.shape
+    dy = _f64(dy, (B, T, H, N))
+    dsT = _f64(dstate_out, (B, H, N, N)) if dstate_out is not None else None
+    outs = [np.zeros((B, T, H, N), dtype=np.float64) for _ in range(4)]
+    ds0 = np.zeros((B, H, N, N), dtype=np.float64)
+    f, c = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_backward_c2.restype = None
+    lib.wkv6_oracle_backward_c2(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(state_in, f), _p(dy, c), _p(dsT, c),
+                                _p(outs[0], c), _p(outs[1], c), _p(outs[2], c), _p(outs[3], c), _p(ds0, c),
+                                ctypes.c_long(B), ctypes.c_long(T), ctypes.c_long(H), ctypes.c_long(N))
+    return outs[0], outs[1], outs[2], outs[3], ds0
+
+
 def rel_l2(a, b) -> float:
     """||a - b||_2 / ||b||_2 in float64 (b is the reference)."""
     a = np.asarray(a, dtype=np.float64).ravel()
