@@ -152,6 +152,20 @@ GF_API gf_status_t gf_wkv6_backward(const void *r, const void *k, const void *v,
                              int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
 GF_API size_t gf_wkv6_backward_bf16_workspace_bytes(int B, int T, int H, int N);
 
+/* Gradient of gf_wkv6_prefill_c2, the Finch-C2 form the paper trains (Finch-C2 block: k_t equation with the factor
+ * (1 - w_t), o_t equation without the bonus): the same adjoint recursion with
+ *     dr_t[i] = sum_j dy_t[j] S_{t-1}[i][j]            dkp_t[i] = sum_j G_t[i][j] v_t[j]       dk_t = dkp_t (1 - w_t)
+ *     dv_t[j] = sum_i G_t[i][j] k_t[i] (1 - w_t[i])
+ *     dx_t[i] = ( sum_j G_t[i][j] S_{t-1}[i][j] - dkp_t[i] k_t[i] ) * ( -w_t[i] exp(x_t[i]) )
+ * (the decay logit also reaches the loss through the key factor).  The second-value vector u2 only adds to the
+ * output: its gradient is dy itself, so neither appears here.  k is the key BEFORE the (1 - w) factor, as in the
+ * forward call.  Everything else (dtypes, layouts, workspace, statuses, launches but for the bonus sum) as
+ * gf_wkv6_backward. */
+GF_API gf_status_t gf_wkv6_backward_c2(const void *r, const void *k, const void *v, const void *x,
+                                const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                                void *dk, void *dv, void *dx, float *dstate_in, int B, int T, int H, int N,
+                                void *workspace, size_t workspace_bytes, gf_stream_t stream);
+
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -36,6 +36,7 @@ _SIGNATURES = {
     "gf_wkv6_backward_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_backward": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_bf16_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_backward_c2": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_prefill_c2": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_varlen_c2": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step_c2": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -246,6 +247,26 @@ def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True
         _check(getattr(lib, "gf_wkv6_backward" + sfx)(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)),
                "gf_wkv6_backward" + sfx)
     return dr, dk, dv, dx, du, ds0
+
+
+def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None):
+    """gf_wkv6_backward_c2: gradient of prefill_c2 (bf16 tensors; k is the key before the (1 - w) factor; the
+    second-value vector's gradient is dy itself).  Returns (dr, dk, dv, dx, dstate_in)."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    bf, f32 = torch.bfloat16, torch.float32
+    dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
+    ds0 = torch.empty((B, H, N, N), device=r.device, dtype=f32) if want_dstate else None
+    with torch.cuda.device(r.device):
+        nbytes = int(lib.gf_wkv6_backward_bf16_workspace_bytes(B, T, H, N))
+        ws = workspace if workspace is not None and workspace.numel() >= nbytes else torch.empty(max(nbytes, 16), dtype=torch.uint8, device=r.device)
+        args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape),
+                _dev(state_in, "state_in", f32, (B, H, N, N)), _dev(dy, "dy", bf, r.shape),
+                _dev(dstate_out, "dstate_out", f32, (B, H, N, N)), _dev(dr, "dr"), _dev(dk, "dk"), _dev(dv, "dv"),
+                _dev(dx, "dx"), _dev(ds0, "dstate_in")]
+        _check(lib.gf_wkv6_backward_c2(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)),
+               "gf_wkv6_backward_c2")
+    return dr, dk, dv, dx, ds0
 
 
 def backward_workspace_bytes(B, T, H, N, dtype=torch.bfloat16):

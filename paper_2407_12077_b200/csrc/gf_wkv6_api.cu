@@ -398,10 +398,12 @@ size_t gf_wkv6_backward_bf16_workspace_bytes(int B, int T, int H, int N)
     return gf::chunked_backward_workspace_bytes((long long)B * H, T, n_sm);
 }
 
-gf_status_t gf_wkv6_backward(const void* r, const void* k, const void* v, const void* x, const float* u,
-                             const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
-                             void* dv, void* dx, float* du, float* dstate_in, int B, int T, int H, int N,
-                             void* workspace, size_t workspace_bytes, gf_stream_t stream)
+namespace {
+// bf16 gradient, classic (u, du given) or Finch-C2 form (c2: no bonus)
+gf_status_t backward_bf16(const void* r, const void* k, const void* v, const void* x, const float* u,
+                          const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk, void* dv,
+                          void* dx, float* du, float* dstate_in, int B, int T, int H, int N, void* workspace,
+                          size_t workspace_bytes, gf_stream_t stream, bool c2)
 {
     using bf = __nv_bfloat16;
     if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
@@ -418,7 +420,7 @@ gf_status_t gf_wkv6_backward(const void* r, const void* k, const void* v, const 
         if (e == cudaSuccess && du) e = cudaMemsetAsync(du, 0, (size_t)H * 64 * sizeof(float), st);
         return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }
-    if (!r || !k || !v || !x || !u || !dy || !dr || !dk || !dv || !dx || !du) return GF_ERR_INVALID_ARG;
+    if (!r || !k || !v || !x || !dy || !dr || !dk || !dv || !dx || (!c2 && (!u || !du))) return GF_ERR_INVALID_ARG;
     const void* ptrs[] = {r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, workspace};
     for (const void* q : ptrs)
         if (misaligned(q)) return GF_ERR_INVALID_ARG;
@@ -434,9 +436,28 @@ gf_status_t gf_wkv6_backward(const void* r, const void* k, const void* v, const 
     if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
     const gf_status_t s = gf::chunked_backward((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, (const bf*)dy,
                                                dstate_out, (bf*)dr, (bf*)dk, (bf*)dv, (bf*)dx, du, dstate_in, B, T, H,
-                                               static_cast<float*>(workspace), st, &g_launches);
+                                               static_cast<float*>(workspace), st, &g_launches, c2);
     if (s != GF_OK) return s;
     return launch_result();
+}
+}  // namespace
+
+gf_status_t gf_wkv6_backward(const void* r, const void* k, const void* v, const void* x, const float* u,
+                             const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
+                             void* dv, void* dx, float* du, float* dstate_in, int B, int T, int H, int N,
+                             void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_bf16(r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, B, T, H, N, workspace,
+                         workspace_bytes, stream, false);
+}
+
+gf_status_t gf_wkv6_backward_c2(const void* r, const void* k, const void* v, const void* x, const float* state_in,
+                                const void* dy, const float* dstate_out, void* dr, void* dk, void* dv, void* dx,
+                                float* dstate_in, int B, int T, int H, int N, void* workspace, size_t workspace_bytes,
+                                gf_stream_t stream)
+{
+    return backward_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in, B, T, H, N,
+                         workspace, workspace_bytes, stream, true);
 }
 
 size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N)

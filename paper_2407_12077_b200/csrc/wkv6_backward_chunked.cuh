@@ -118,6 +118,14 @@ __device__ __forceinline__ bool cbar_and(bool ok)
     return r != 0;
 }
 
+// 1 - 2^l for l <= 0 without the cancellation of the direct form near l = 0 (slow decays): the series of -expm1 there.
+__device__ __forceinline__ float one_minus_ex2(float l)
+{
+    const float t = l * LN2;
+    const float series = -t * (1.f + t * (0.5f + t * (0.16666667f + t * 0.041666668f)));
+    return l > -0.125f ? series : 1.f - ex2(l);
+}
+
 // tcgen05.ld of a 16 x 16 fp32 block without the wait for its data (tmem_ld_done() before the first use): several
 // loads can then be in flight together.
 __device__ __forceinline__ void tmem_ld_16x16_async(uint32_t taddr, float (&v)[2][4])
@@ -187,6 +195,9 @@ __device__ __forceinline__ bool scan_rows(float (&v)[2][4], uint32_t tot, int sp
     return ok;
 }
 
+// C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus; the second-value vector only adds to the
+// output, so its gradient is dy itself and nothing here depends on it).
+template <bool C2>
 __global__ void __launch_bounds__(B_THREADS, 1)
 wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
                              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -351,7 +362,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 
     float uu[2][2];                                  // bonus of this lane's columns (as channels)
 #pragma unroll
-    for (int n = 0; n < 2; ++n) { uu[n][0] = p.u[col0 + cb + 8 * n]; uu[n][1] = p.u[col0 + cb + 8 * n + 1]; }
+    for (int n = 0; n < 2; ++n) { uu[n][0] = C2 ? 0.f : p.u[col0 + cb + 8 * n]; uu[n][1] = C2 ? 0.f : p.u[col0 + cb + 8 * n + 1]; }
     float G[2][4], SL[2][4], du_acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
     const float* ck_unit = p.ckpt + (size_t)unit * (nchunks + 1) * 4096;
     if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
@@ -430,6 +441,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             for (int n = 0; n < 2; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
+                    if (C2) kv[n][e] *= one_minus_ex2(lw2[n][e]);      // the key that enters the state
                     const float t = rv[n][e] * kv[n][e] * uu[n][e & 1];
                     if (e < 2) b0 += t; else b1 += t;
                     rv[n][e] *= ex2(a[n][e] - lw2[n][e]);
@@ -520,8 +532,10 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             for (int t = 0; t < valid; ++t) {
                 *reinterpret_cast<float4*>(scr + (size_t)t * 4096) = make_float4(S[0][0], S[0][1], S[0][2], S[0][3]);
                 *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4) = make_float4(S[1][0], S[1][1], S[1][2], S[1][3]);
-                const float w0 = expf(-expf(lds_bf16(tx + swz(t, 2 * R0)))), w1 = expf(-expf(lds_bf16(tx + swz(t, 2 * R1))));
-                const float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                const float e0 = expf(lds_bf16(tx + swz(t, 2 * R0))), e1 = expf(lds_bf16(tx + swz(t, 2 * R1)));
+                const float w0 = expf(-e0), w1 = expf(-e1);
+                float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                if (C2) { k0 *= -expm1f(-e0); k1 *= -expm1f(-e1); }
 #pragma unroll
                 for (int n = 0; n < 2; ++n)
 #pragma unroll
@@ -540,7 +554,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 const float Sp[2][4] = {{sa.x, sa.y, sa.z, sa.w}, {sb4.x, sb4.y, sb4.z, sb4.w}};
                 const float x0 = lds_bf16(tx + swz(t, 2 * R0)), x1 = lds_bf16(tx + swz(t, 2 * R1));
                 const float w0 = expf(-expf(x0)), w1 = expf(-expf(x1));
-                const float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                if (C2) { k0 *= -expm1f(-expf(x0)); k1 *= -expm1f(-expf(x1)); }
                 const float r0 = lds_bf16(tr + swz(t, 2 * R0)), r1 = lds_bf16(tr + swz(t, 2 * R1));
                 float pr0 = 0.f, pr1 = 0.f, pk0 = 0.f, pk1 = 0.f, pg0 = 0.f, pg1 = 0.f, pv[2][2];
 #pragma unroll
@@ -585,7 +600,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     for (int e = 0; e < 2; ++e) {
                         const int cc = 2 * lane + e;
                         vd = fmaf(lds_bf16(tv + swz(t, 2 * cc)), lds_bf16(tdy + swz(t, 2 * cc)), vd);
-                        ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * p.u[col0 + cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
+                        if (!C2) ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * p.u[col0 + cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
                     }
 #pragma unroll
                     for (int d = 1; d < 32; d <<= 1) {
@@ -601,11 +616,18 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
                     for (int o = 0; o < 4; ++o) { s_r += red[(o * 3 + 0) * 64 + cc]; s_k += red[(o * 3 + 1) * 64 + cc]; s_g += red[(o * 3 + 2) * 64 + cc]; }
                     const float xc = lds_bf16(tx + swz(t, 2 * cc)), kc = lds_bf16(tk + swz(t, 2 * cc)), rc = lds_bf16(tr + swz(t, 2 * cc));
-                    const float uc = p.u[col0 + cc], vd = scal[0];
-                    sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
-                    sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
-                    sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), s_g * (-expf(-expf(xc)) * expf(xc)));
-                    fsm(BO_DU_FB)[cc] = fmaf(rc * kc, vd, fsm(BO_DU_FB)[cc]);
+                    const float ec = expf(xc), wc = expf(-ec);
+                    if (C2) {
+                        sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), s_r);
+                        sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), s_k * -expm1f(-ec));
+                        sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
+                    } else {
+                        const float uc = p.u[col0 + cc], vd = scal[0];
+                        sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
+                        sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
+                        sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), s_g * (-wc * ec));
+                        fsm(BO_DU_FB)[cc] = fmaf(rc * kc, vd, fsm(BO_DU_FB)[cc]);
+                    }
                 } else if (tid < 128) {
                     const int j = tid - 64;
                     const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
@@ -706,7 +728,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                         const float pd = e < 2 ? pd0 : pd1;
                         o[n][e] = fmaf(uu[n][e & 1] * kv[n][e], pd, acc[n][e] * ex2(a_cur[n][e] - lw_cur[n][e]));
                         qv[n][e] = acc[n][e] * hat[n][e];
-                        du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
+                        if (!C2) du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
                     }
                 store_block_bf16(sbase + BO_OUT + moff, o);
                 load_block_bf16(t_kh + moff, hat);
@@ -717,6 +739,13 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                         const float pd = e < 2 ? pd0 : pd1;
                         o[n][e] = fmaf(uu[n][e & 1] * rv[n][e], pd, acc2[n][e] * ex2(-a_cur[n][e]));
                         z[n][e] = qv[n][e] - acc2[n][e] * hat[n][e];
+                        if (C2) {
+                            // o is the gradient of k (1 - w): the key gets (1 - w) of it, and the decay logit its
+                            // share through the key factor, folded into the term that leaves the suffix sums
+                            const float omw = one_minus_ex2(lw_cur[n][e]);
+                            qv[n][e] = fmaf(o[n][e] * kv[n][e], 1.f - omw, qv[n][e]);
+                            o[n][e] *= omw;
+                        }
                     }
                 store_block_bf16(sbase + BO_OUT + TILE + moff, o);
                 store_block_bf16(sbase + BO_OUT + 2 * TILE + moff, acc3);
@@ -772,7 +801,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 for (int e = 0; e < 2; ++e) fsm(BO_RED_V)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
         }
         cbar();
-        if (tid < 64) {
+        if (!C2 && tid < 64) {
             const float* rv4 = fsm(BO_RED_V);
             p.du_part[(size_t)unit * 64 + tid] = ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fsm(BO_DU_FB)[tid];
         }
@@ -810,7 +839,8 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
                                     const __nv_bfloat16* x, const float* u, const float* state_in,
                                     const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
                                     __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
-                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches)
+                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
+                                    bool c2 = false)
 {
     const long long units = (long long)B * H, rows = (long long)B * T;
     const int n_sm = sm_count();
@@ -819,7 +849,8 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     const int dev = current_device();
     if (dev < 0) return GF_ERR_CUDA;
     if (!attr_set.is_set(dev)) {
-        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess)
+        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set.set(dev);
     }
@@ -827,7 +858,7 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     float* ckpt = ws;
     float* du_part = ckpt + (size_t)units * nck * 4096;
     float* fb = du_part + (size_t)units * 64;
-    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches);
+    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
     if (s != GF_OK) return s;
     const long long C = (long long)H * 64;
     CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
@@ -837,9 +868,11 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         return GF_ERR_CUDA;
     bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, n_sm,
                   wait_limit_us().load(std::memory_order_relaxed)};
-    bc::wkv6_backward_chunked_kernel<<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    if (c2) return GF_OK;                            // no bonus, no bonus gradient
     bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;

@@ -1670,7 +1670,7 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
 // k, v and the decay logits).
 inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x,
                                        const float* state_in, float* ckpt, int n_seq, int T, int H, cudaStream_t st,
-                                       std::atomic<uint64_t>* launches)
+                                       std::atomic<uint64_t>* launches, int c2 = 0)
 {
     const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
@@ -1681,10 +1681,11 @@ inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat
     if (!ck::make_map(&tk, k, total_rows, C, 64) || !ck::make_map(&tv, v, total_rows, C, 64) ||
         !ck::make_map(&tx, x, total_rows, C, 64) || !ck::make_map(&tdummy, k, total_rows, C, 16))
         return GF_ERR_CUDA;
-    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, nullptr, (T + ck::L - 1) / ck::L, 1, nullptr, 0};
+    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, nullptr, (T + ck::L - 1) / ck::L, 1, nullptr, c2};
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     p.ckpt = ckpt;
-    ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
