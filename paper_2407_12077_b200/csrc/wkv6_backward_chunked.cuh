@@ -828,54 +828,4 @@ wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H,
 
 }  // namespace bc
 
-// Workspace of the chunked gradient: checkpoints, per-unit bonus gradients, the token-by-token path's scratch.
-inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
-{
-    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
-    return ((size_t)units * nck * 4096 + (size_t)units * 64 + (size_t)n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
-}
-
-inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                                    const __nv_bfloat16* x, const float* u, const float* state_in,
-                                    const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
-                                    __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
-                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
-                                    bool c2 = false)
-{
-    const long long units = (long long)B * H, rows = (long long)B * T;
-    const int n_sm = sm_count();
-    if (n_sm <= 0) return GF_ERR_CUDA;
-    static PerDeviceFlag attr_set;
-    const int dev = current_device();
-    if (dev < 0) return GF_ERR_CUDA;
-    if (!attr_set.is_set(dev)) {
-        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess)
-            return GF_ERR_CUDA;
-        attr_set.set(dev);
-    }
-    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
-    float* ckpt = ws;
-    float* du_part = ckpt + (size_t)units * nck * 4096;
-    float* fb = du_part + (size_t)units * 64;
-    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
-    if (s != GF_OK) return s;
-    const long long C = (long long)H * 64;
-    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
-    if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||
-        !ck::make_map(&tv, v, rows, C, 64) || !ck::make_map(&tdy, dy, rows, C, 64) || !ck::make_map(&tdr, dr, rows, C, 64) ||
-        !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
-        return GF_ERR_CUDA;
-    bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, n_sm,
-                  wait_limit_us().load(std::memory_order_relaxed)};
-    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
-    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
-    launches->fetch_add(1, std::memory_order_relaxed);
-    if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
-    if (c2) return GF_OK;                            // no bonus, no bonus gradient
-    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
-    launches->fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
-}
-
 }  // namespace gf

@@ -1,0 +1,800 @@
+// Gradient of the WKV-6 recurrence in chunks of 64 tokens on the tensor cores, two chunks in flight per CTA.
+//
+// The arithmetic is that of wkv6_backward_chunked.cuh (its header carries the derivation): per chunk, from the last
+// to the first, nine 64x64x64 bf16 products around elementwise phases, with the state adjoint G carried in fp32.
+// A chunk's phases (decay -> cumulative sum -> operands -> products -> masks -> products -> epilogue -> suffix sums)
+// depend on one another and each keeps a different pipe busy, so one set of warps that walks them in lock step leaves
+// most issue slots empty.  Here the CTA's 32 warps form two groups of 16 that take alternate chunks and run half a
+// period apart: while one group waits for its products or sits in a latency-bound phase, the other one issues.
+// The only thing a chunk needs from the chunk after it (in time) is the adjoint at its end, G_L = G_0 of that chunk;
+// it enters late (the operand G^ = diag(D) G_L, the row sums E, and G_0 = G^ + R^^T dY, whose product needs no G), so
+// the groups hand G to each other through a pair of fp32 tiles in shared memory, each guarded by an mbarrier that
+// all threads of the writing group arrive on, and the chain G_L -> G_0 is a few hundred cycles per chunk.
+//
+// Layout inside a group of 16 warps: warp (sp = warp % 4, cx = warp / 4 % 4) owns rows 16 sp .. +15 and columns
+// 16 cx .. +15 of every 64x64 tile; lane (g = lane / 4, q = lane % 4) rows 16 sp + g and + 8, columns 16 cx + 8 n + 2 q + e
+// (n, e < 2): 8 cells, the accumulator layout of the 64-row products, in which bf16 tiles move through ldmatrix /
+// stmatrix.  (G_NB = 4 gives groups of 8 warps with 16 cells per lane instead.)  Each group has its own input stage (x, r, k, v, dy by TMA), operand tiles, tensor-memory columns
+// (three accumulators that the second group of products reuses once the first group's have been read) and
+// barriers; the four staging tiles of the gradients alias the operand tiles that are dead by then.  Thread 0 of a
+// group issues its products and copies.  Waits are per thread and bounded; their outcome is made uniform over the
+// group at its next barrier; the hand-over waits watch the CTA's abort word, so both groups leave together.
+// A chunk in which a channel decays by more than 2^-96 runs token by token in fp32 on its group's warps.
+#pragma once
+#include "wkv6_backward_chunked.cuh"
+
+namespace gf {
+namespace bg {
+
+using namespace ck;
+using bc::BParams;
+using bc::LN2;
+using bc::lds_bf16;
+using bc::lds_v4;
+using bc::one_minus_ex2;
+using bc::smid;
+using bc::sts_bf16;
+using bc::tmem_ld_done;
+
+// NB = 8-column blocks per lane: 4 (groups of 8 warps, 16 cells per lane, 128 registers) or 2 (groups of 16 warps,
+// 8 cells per lane, 64 registers: twice the warps per scheduler to hide the phases' latencies)
+constexpr int G_NB = 4;
+constexpr int G_NSLAB = 8 / G_NB;                 // column slabs of 8 NB columns per tile = warps per row group
+constexpr int G_H2 = G_NB / 2;                    // 16-column blocks per lane
+constexpr int G_GT = 32 * 4 * G_NSLAB;            // threads of one group
+constexpr int G_THREADS = 2 * G_GT;               // the CTA
+// tensor memory: per group 256 columns, three accumulators used twice
+constexpr int GT_P = 0, GT_DP = 64, GT_DG = 128, GT_DV = 0, GT_DR = 64, GT_DK = 128, GT_COLS = 512;
+// shared memory of one group
+constexpr int GO_IN = 0;                          // x, r, k, v, dy
+constexpr int GO_RH = GO_IN + 5 * TILE;           // R^ [t][c]
+constexpr int GO_KH = GO_RH + TILE;               // K^ [i][c]
+constexpr int GO_T4 = GO_KH + TILE;               // S_0, G^, P', dP' operand tiles; later the dr, dk, dv, dx staging tiles
+constexpr int GO_TOT = GO_T4 + 4 * TILE;          // [4][64] float: row-group totals of a scan
+constexpr int GO_EP = GO_TOT + 1024;              // [NSLAB][64] float: partial E by column slab
+constexpr int GO_BP = GO_EP + 1024;               // [NSLAB][64] float: partial bonus by column slab
+constexpr int GO_DPD = GO_BP + 1024;              // [64] float: dy_t . v_t
+constexpr int GO_RED = GO_DPD + 256;              // token-by-token path: [NSLAB][3][64]
+constexpr int GO_REDV = GO_RED + 4 * 3 * 64 * 4;  //   [4][64]
+constexpr int GO_DUFB = GO_REDV + 1024;           //   du [64]
+constexpr int GO_SCAL = GO_DUFB + 256;            //   v . dy, sum r u k
+constexpr int GO_BYTES = (GO_SCAL + 16 + 1023) & ~1023;
+// shared by the groups
+constexpr int GS_GBUF = 2 * GO_BYTES;             // [2][64][64] float: the adjoint handed from chunk to chunk
+constexpr int GS_U = GS_GBUF + 2 * 16384;         // [64] float: the bonus
+constexpr int GS_ABORT = GS_U + 256;              // abort word, wait limit
+constexpr int GS_TMEM = GS_ABORT + 8;
+constexpr int GS_BAR = GS_TMEM + 8;               // per group: inputs, first / second group of products; then the hand-over pair
+enum { GB_IN = 0, GB_MA = 1, GB_MB = 2, GB_PER_GROUP = 3, GB_GREADY = 6, GB_COUNT = 8 };
+constexpr int G_SMEM_BYTES = GS_BAR + 8 * GB_COUNT;
+constexpr int G_SMEM_ALLOC = G_SMEM_BYTES + 1024;
+static_assert(G_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
+
+// barrier over one group's 8 warps (ids 1 and 2), plain and with an AND over a predicate
+__device__ __forceinline__ void gbar(int grp) { asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(G_GT) : "memory"); }
+__device__ __forceinline__ bool gbar_and(int grp, bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "bar.red.and.pred q, %1, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(grp + 1), "r"((uint32_t)ok), "n"(G_GT) : "memory");
+    return r != 0;
+}
+
+// explicit shared-space accesses (a pointer rebuilt from an integer would make them generic loads)
+__device__ __forceinline__ float2 ldsf2(uint32_t a)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void stsf2(uint32_t a, float2 v) { asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(a), "f"(v.x), "f"(v.y) : "memory"); }
+
+// 16 rows x 16 columns of an accumulator, without the wait (tmem_ld_done() before the first use)
+__device__ __forceinline__ void tmem_ld_16x16_async2(uint32_t taddr, float (&v)[2][4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3])
+                 : "r"(taddr) : "memory");
+}
+
+// 16 x 16 bf16 blocks of a swizzled tile <-> two column blocks (n = 2 h2, 2 h2 + 1) of the lane's cells
+__device__ __forceinline__ void ld_half(uint32_t addr, float (&v)[2][4])
+{
+    uint32_t w0, w1, w2, w3;
+    ldsm_x4(addr, w0, w1, w2, w3);
+    v[0][0] = bf_lo(w0); v[0][1] = bf_hi(w0); v[0][2] = bf_lo(w1); v[0][3] = bf_hi(w1);
+    v[1][0] = bf_lo(w2); v[1][1] = bf_hi(w2); v[1][2] = bf_lo(w3); v[1][3] = bf_hi(w3);
+}
+__device__ __forceinline__ void st_half(uint32_t addr, const float (&v)[2][4])
+{
+    stsm_x4(addr, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
+}
+__device__ __forceinline__ void ld_tile(uint32_t tile, const uint32_t (&moff)[G_H2], float (&v)[G_NB][4])
+{
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2) ld_half(tile + moff[h2], reinterpret_cast<float (&)[2][4]>(v[2 * h2]));
+}
+__device__ __forceinline__ void st_tile(uint32_t tile, const uint32_t (&moff)[G_H2], const float (&v)[G_NB][4])
+{
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2) st_half(tile + moff[h2], reinterpret_cast<const float (&)[2][4]>(v[2 * h2]));
+}
+
+// Inclusive sums along the 64 rows of a tile in the group's layout, forwards (rows <= t) or backwards (rows >= t).
+// tot: [4][64] floats of the group's shared memory.  Contains one barrier of the group, which also forms the AND of
+// `ok` over it (returned).
+template <bool REV>
+__device__ __forceinline__ bool scan_rows(float (&v)[G_NB][4], uint32_t tot, int grp, int sp, int cb, int lane, bool ok)
+{
+    const int g = lane >> 2, q = lane & 3;           // (cb: the lane's first column, a multiple of 2)
+#pragma unroll
+    for (int d = 4; d < 32; d <<= 1) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float o = REV ? __shfl_down_sync(0xffffffffu, v[n][e], d) : __shfl_up_sync(0xffffffffu, v[n][e], d);
+                if (REV ? lane + d < 32 : lane >= d) v[n][e] += o;
+            }
+    }
+#pragma unroll
+    for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            if (REV) v[n][e] += __shfl_sync(0xffffffffu, v[n][2 + e], q);
+            else v[n][2 + e] += __shfl_sync(0xffffffffu, v[n][e], 28 + q);
+        }
+    if (g == (REV ? 0 : 7)) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+            stsf2(tot + 4 * (sp * 64 + cb + 8 * n), REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]));
+    }
+    ok = gbar_and(grp, ok);
+#pragma unroll
+    for (int o = 0; o < 4; ++o) {
+        if (REV ? o > sp : o < sp) {
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n) {
+                const float2 t = ldsf2(tot + 4 * (o * 64 + cb + 8 * n));
+                v[n][0] += t.x; v[n][1] += t.y; v[n][2] += t.x; v[n][3] += t.y;
+            }
+        }
+    }
+    return ok;
+}
+
+template <bool C2>
+__global__ void __launch_bounds__(G_THREADS, 1)
+wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
+                            const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                            const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
+                            const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
+                            const __grid_constant__ CUtensorMap tm_dx, const BParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t abort_flag = sbase + GS_ABORT;
+    auto bar = [&](int i) { return sbase + GS_BAR + 8 * i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int grp = tid / G_GT, gt = tid % G_GT;                    // group, thread inside the group
+    const int sp = warp & 3, cx = (warp >> 2) % G_NSLAB, g = lane >> 2, q = lane & 3;       // row group, column slab
+    const int unit = blockIdx.x, seq = unit / p.H, h = unit % p.H;
+    const int T = p.T, nchunks = (T + L - 1) / L;
+    const long long row0 = (long long)seq * T;
+    const int col0 = h * 64;
+    const size_t C = (size_t)p.H * 64;
+    const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
+    const int cb = 8 * G_NB * cx + 2 * q;            // its columns: cb + 8 n + e, n < G_NB
+    // byte offsets of this lane's ldmatrix / stmatrix rows inside a tile: the warp's 16 x 16 blocks
+    uint32_t moff[G_H2];
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2)
+        moff[h2] = swz(16 * sp + (lane & 7) + 8 * ((lane >> 3) & 1), (G_NB * cx + 2 * h2 + (lane >> 4)) << 4);
+    const uint32_t gbase = sbase + grp * GO_BYTES;   // this group's shared memory
+    auto gsm = [&](int off) { return reinterpret_cast<float*>(smem + grp * GO_BYTES + off); };
+    // the adjoint tiles handed between the groups: [buffer][cell of the lane][thread of the group] (conflict-free)
+    auto g_put = [&](int b, const float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) stsf(sbase + GS_GBUF + 4 * ((b * 4 * G_NB + 4 * n + e) * G_GT + gt), v[n][e]);
+    };
+    auto g_get = [&](int b, float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[n][e] = ldsf(sbase + GS_GBUF + 4 * ((b * 4 * G_NB + 4 * n + e) * G_GT + gt));
+    };
+    auto gld = [&](int off) { return ldsf(gbase + off); };           // a float of this group's small arrays
+    const float* ub = reinterpret_cast<const float*>(smem + GS_U);
+    auto gb = [&](int i) { return bar(grp * GB_PER_GROUP + i); };      // this group's barriers
+
+    if (tid == 0) {
+        for (int i = 0; i < GB_GREADY; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(GB_GREADY), G_GT);
+        mbar_init(bar(GB_GREADY + 1), G_GT);
+        sts32(abort_flag, 0u);
+        sts32(abort_flag + 4, p.wait_limit_us ? p.wait_limit_us : WAIT_LIMIT_US);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (tid < 64) reinterpret_cast<float*>(smem + GS_U)[tid] = C2 ? 0.f : p.u[col0 + tid];
+    if (gt < 64) gsm(GO_DUFB)[gt] = 0.f;
+    if (warp == 1) tmem_alloc(sbase + GS_TMEM, GT_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32(sbase + GS_TMEM) + 256 * grp;                 // this group's columns
+    const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 8 * G_NB * cx;      // this warp's block of an accumulator
+
+    auto chunk_of = [&](int it) { return nchunks - 1 - it; };
+    const uint32_t tin = gbase + GO_IN;
+    const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
+    const uint32_t t_rh = gbase + GO_RH, t_kh = gbase + GO_KH;
+    const uint32_t t_sb = gbase + GO_T4, t_gb = t_sb + TILE, t_pp = t_sb + 2 * TILE, t_dpp = t_sb + 3 * TILE;
+    const uint32_t t_out = gbase + GO_T4;
+    int last_load = -1;                              // (thread 0 of the group) the last iteration whose copies were issued
+    auto issue_loads = [&](int it) {                 // thread 0 of the group
+        const int row = (int)(row0 + (long long)chunk_of(it) * L);
+        mbar_expect_tx(gb(GB_IN), 5 * TILE);
+        tma_load_2d(tx, &tm_x, col0, row, gb(GB_IN));
+        tma_load_2d(tr, &tm_r, col0, row, gb(GB_IN));
+        tma_load_2d(tk, &tm_k, col0, row, gb(GB_IN));
+        tma_load_2d(tv, &tm_v, col0, row, gb(GB_IN));
+        tma_load_2d(tdy, &tm_dy, col0, row, gb(GB_IN));
+        last_load = it;
+    };
+    auto load_f32_block = [&](const float* src, float (&v)[G_NB][4]) {      // [64][64] fp32 block, the lane's cells
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) {
+            const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)R0 * 64 + cb + 8 * n);
+            const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)R1 * 64 + cb + 8 * n);
+            v[n][0] = lo.x; v[n][1] = lo.y; v[n][2] = hi.x; v[n][3] = hi.y;
+        }
+    };
+    auto store_f32_block = [&](float* dst, const float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) {
+            *reinterpret_cast<float2*>(dst + (size_t)R0 * 64 + cb + 8 * n) = make_float2(v[n][0], v[n][1]);
+            *reinterpret_cast<float2*>(dst + (size_t)R1 * 64 + cb + 8 * n) = make_float2(v[n][2], v[n][3]);
+        }
+    };
+
+    const float* ck_unit = p.ckpt + (size_t)unit * (nchunks + 1) * 4096;
+    float du_acc[G_NB][2];
+#pragma unroll
+    for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
+    if (gt == 0 && grp < nchunks) issue_loads(grp);
+    int mph = 0;                                     // phase bit of this group's two product barriers
+    bool alive = true;
+
+    for (int it = grp; it < nchunks; it += 2) {
+        const int c = chunk_of(it), valid = min(L, T - c * L);
+        const int use = it >> 1;                     // how often this group's input stage has been filled before
+        float S0[G_NB][4];                              // the chunk-start state (requested early: it is used after the scan)
+        load_f32_block(ck_unit + (size_t)c * 4096, S0);
+        // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
+        bool ok = mbar_wait(gb(GB_IN), use & 1, abort_flag);
+        if (gt == 0 && it > 1) bulk_wait_read<0>();  // the previous chunk's staging tiles have been read by the TMA unit
+        if (valid < L) {
+            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
+            for (int i = gt; i < (L - valid) * 8; i += G_GT) {
+                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
+                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
+            }
+        }
+        float a[G_NB][4], lw2[G_NB][4];
+        {
+            float xv[G_NB][4];
+            ld_tile(tx, moff, xv);
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool live = (e < 2 ? R0 : R1) < valid;
+                    lw2[n][e] = live ? -ex2(fmaf(xv[n][e], LOG2E, LOG2_LOG2E)) : 0.f;
+                    a[n][e] = lw2[n][e];
+                }
+        }
+        ok = scan_rows<false>(a, gbase + GO_TOT, grp, sp, cb, lane, ok);      // (barrier: the zeroed rows are visible after it)
+        if (!ok) { alive = false; break; }
+        float d_lo, d_hi;                            // the chunk's decay for the channels that are this lane's rows of G
+        bool safe;
+        {
+            float al0 = 0.f, al1 = 0.f;
+#pragma unroll
+            for (int o = 0; o < 4; ++o) { al0 += gld(GO_TOT + 4 * (o * 64 + R0)); al1 += gld(GO_TOT + 4 * (o * 64 + R1)); }
+            d_lo = ex2(al0); d_hi = ex2(al1);
+            safe = (al0 >= -A2_MAX) && (al1 >= -A2_MAX);                   // false for NaN as well
+        }
+        // ---- operands from the inputs: R^, K^ (and the bonus), the chunk-start state
+        {
+            float rv[G_NB][4], kv[G_NB][4];
+            ld_tile(tr, moff, rv);
+            ld_tile(tk, moff, kv);
+            float b0 = 0.f, b1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (C2) kv[n][e] *= one_minus_ex2(lw2[n][e]);      // the key that enters the state
+                    if (!C2) {
+                        const float t = rv[n][e] * kv[n][e] * ldsf(sbase + GS_U + 4 * (cb + 8 * n + (e & 1)));
+                        if (e < 2) b0 += t; else b1 += t;
+                    }
+                    rv[n][e] *= ex2(a[n][e] - lw2[n][e]);
+                    kv[n][e] *= ex2(-a[n][e]);
+                }
+            st_tile(t_rh, moff, rv);
+            st_tile(t_kh, moff, kv);
+            if (!C2) {
+                b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
+                b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
+                if (q == 0) { stsf(gbase + GO_BP + 4 * (cx * 64 + R0), b0); stsf(gbase + GO_BP + 4 * (cx * 64 + R1), b1); }
+            }
+        }
+        st_tile(t_sb, moff, S0);
+        float SL[G_NB][4];                           // the state at the chunk's end (for E), in flight over the barrier and the hand-over wait
+        load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
+        fence_proxy_async();
+        tc_fence_before();
+        const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
+        if (!unsafe && gt == 0) {
+            // the products that need nothing but the inputs; the adjoint is not needed for R^^T dY either
+            tc_fence_after();
+            const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
+                tc_mma(tmem + GT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                tc_mma(tmem + GT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
+                tc_mma(tmem + GT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
+            }
+            tc_commit(gb(GB_MA));
+        }
+        // ---- the adjoint at the chunk's end, from the other group (the call's dstate_out for the last chunk)
+        float G[G_NB][4];
+        if (it == 0) {
+            if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
+            else {
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
+            }
+        } else {
+            if (!mbar_wait(bar(GB_GREADY + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag)) ok = false;
+            g_get((it - 1) & 1, G);
+        }
+        {
+            // E = rowsum(G_L * S_L), S_L = the state before the next chunk (after the last token for the last chunk)
+            float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n) {
+                e0 = fmaf(G[n][0], SL[n][0], fmaf(G[n][1], SL[n][1], e0));
+                e1 = fmaf(G[n][2], SL[n][2], fmaf(G[n][3], SL[n][3], e1));
+            }
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
+            if (q == 0) { stsf(gbase + GO_EP + 4 * (cx * 64 + R0), e0); stsf(gbase + GO_EP + 4 * (cx * 64 + R1), e1); }
+        }
+
+        if (unsafe) {
+            // ---- token by token: the chunk's states recomputed into this group's scratch, then the reverse recurrence
+            const unsigned slot = 2 * smid() + grp;
+            if (slot >= (unsigned)p.n_slots) {       // (no scratch for this SM: report it and leave)
+                if (gt == 0) { sts32(abort_flag, 1u); atomicExch(&g_dev_status, 1); }
+                alive = false;
+                break;
+            }
+            if (!gbar_and(grp, ok)) { alive = false; break; }
+            float* scr = p.fb_scratch + (size_t)slot * bc::FB_SLOT_FLOATS + (size_t)gt * (4 * G_NB);
+            float S[G_NB][4];
+            load_f32_block(ck_unit + (size_t)c * 4096, S);
+            for (int t = 0; t < valid; ++t) {
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n)
+                    *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4 * n) = make_float4(S[n][0], S[n][1], S[n][2], S[n][3]);
+                const float e0 = expf(lds_bf16(tx + swz(t, 2 * R0))), e1 = expf(lds_bf16(tx + swz(t, 2 * R1)));
+                const float w0 = expf(-e0), w1 = expf(-e1);
+                float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                if (C2) { k0 *= -expm1f(-e0); k1 *= -expm1f(-e1); }
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float vj = lds_bf16(tv + swz(t, 2 * (cb + 8 * n + e)));
+                        S[n][e] = fmaf(w0, S[n][e], k0 * vj);
+                        S[n][2 + e] = fmaf(w1, S[n][2 + e], k1 * vj);
+                    }
+            }
+            float* red = gsm(GO_RED);                // [slab][3][64]
+            float* redv = gsm(GO_REDV);              // [sp][64]
+            float* scal = gsm(GO_SCAL);              // v . dy, sum r u k
+            for (int t = valid - 1; t >= 0; --t) {
+                float Sp[G_NB][4];
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    const float4 s4 = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096 + 4 * n);
+                    Sp[n][0] = s4.x; Sp[n][1] = s4.y; Sp[n][2] = s4.z; Sp[n][3] = s4.w;
+                }
+                const float x0 = lds_bf16(tx + swz(t, 2 * R0)), x1 = lds_bf16(tx + swz(t, 2 * R1));
+                const float w0 = expf(-expf(x0)), w1 = expf(-expf(x1));
+                float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
+                if (C2) { k0 *= -expm1f(-expf(x0)); k1 *= -expm1f(-expf(x1)); }
+                const float r0 = lds_bf16(tr + swz(t, 2 * R0)), r1 = lds_bf16(tr + swz(t, 2 * R1));
+                float pr0 = 0.f, pr1 = 0.f, pk0 = 0.f, pk1 = 0.f, pg0 = 0.f, pg1 = 0.f, pv[G_NB][2];
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int j = cb + 8 * n + e;
+                        const float vj = lds_bf16(tv + swz(t, 2 * j)), dyj = lds_bf16(tdy + swz(t, 2 * j));
+                        pr0 = fmaf(dyj, Sp[n][e], pr0); pr1 = fmaf(dyj, Sp[n][2 + e], pr1);
+                        pk0 = fmaf(G[n][e], vj, pk0); pk1 = fmaf(G[n][2 + e], vj, pk1);
+                        pg0 = fmaf(G[n][e], Sp[n][e], pg0); pg1 = fmaf(G[n][2 + e], Sp[n][2 + e], pg1);
+                        pv[n][e] = fmaf(G[n][e], k0, G[n][2 + e] * k1);
+                        G[n][e] = fmaf(w0, G[n][e], r0 * dyj);
+                        G[n][2 + e] = fmaf(w1, G[n][2 + e], r1 * dyj);
+                    }
+#pragma unroll
+                for (int d = 1; d < 4; d <<= 1) {
+                    pr0 += __shfl_xor_sync(0xffffffffu, pr0, d); pr1 += __shfl_xor_sync(0xffffffffu, pr1, d);
+                    pk0 += __shfl_xor_sync(0xffffffffu, pk0, d); pk1 += __shfl_xor_sync(0xffffffffu, pk1, d);
+                    pg0 += __shfl_xor_sync(0xffffffffu, pg0, d); pg1 += __shfl_xor_sync(0xffffffffu, pg1, d);
+                }
+#pragma unroll
+                for (int d = 4; d < 32; d <<= 1)
+#pragma unroll
+                    for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) pv[n][e] += __shfl_xor_sync(0xffffffffu, pv[n][e], d);
+                if (q == 0) {
+                    red[(cx * 3 + 0) * 64 + R0] = pr0; red[(cx * 3 + 0) * 64 + R1] = pr1;
+                    red[(cx * 3 + 1) * 64 + R0] = pk0; red[(cx * 3 + 1) * 64 + R1] = pk1;
+                    red[(cx * 3 + 2) * 64 + R0] = pg0; red[(cx * 3 + 2) * 64 + R1] = pg1;
+                }
+                if (g == 0) {
+#pragma unroll
+                    for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) redv[sp * 64 + cb + 8 * n + e] = pv[n][e];
+                }
+                if (gt < 32) {
+                    float vd = 0.f, ruk = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int cc = 2 * lane + e;
+                        vd = fmaf(lds_bf16(tv + swz(t, 2 * cc)), lds_bf16(tdy + swz(t, 2 * cc)), vd);
+                        if (!C2) ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * ub[cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
+                    }
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        vd += __shfl_xor_sync(0xffffffffu, vd, d);
+                        ruk += __shfl_xor_sync(0xffffffffu, ruk, d);
+                    }
+                    if (lane == 0) { scal[0] = vd; scal[1] = ruk; }
+                }
+                gbar(grp);
+                if (gt < 64) {
+                    const int cc = gt;
+                    float s_r = 0.f, s_k = 0.f, s_g = 0.f;
+#pragma unroll
+                    for (int o = 0; o < G_NSLAB; ++o) { s_r += red[(o * 3 + 0) * 64 + cc]; s_k += red[(o * 3 + 1) * 64 + cc]; s_g += red[(o * 3 + 2) * 64 + cc]; }
+                    const float xc = lds_bf16(tx + swz(t, 2 * cc)), kc = lds_bf16(tk + swz(t, 2 * cc)), rc = lds_bf16(tr + swz(t, 2 * cc));
+                    const float ec = expf(xc), wc = expf(-ec);
+                    if (C2) {
+                        sts_bf16(t_out + swz(t, 2 * cc), s_r);
+                        sts_bf16(t_out + TILE + swz(t, 2 * cc), s_k * -expm1f(-ec));
+                        sts_bf16(t_out + 3 * TILE + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
+                    } else {
+                        const float uc = ub[cc], vd = scal[0];
+                        sts_bf16(t_out + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
+                        sts_bf16(t_out + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
+                        sts_bf16(t_out + 3 * TILE + swz(t, 2 * cc), s_g * (-wc * ec));
+                        gsm(GO_DUFB)[cc] = fmaf(rc * kc, vd, gsm(GO_DUFB)[cc]);
+                    }
+                } else if (gt < 128) {
+                    const int j = gt - 64;
+                    const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
+                    sts_bf16(t_out + 2 * TILE + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
+                }
+                gbar(grp);
+            }
+            // hand the adjoint on
+            if (it + 1 < nchunks) {
+                g_put(it & 1, G);
+                mbar_arrive(bar(GB_GREADY + (it & 1)));
+            } else if (p.dstate_in) {
+                store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
+            }
+        } else {
+            // ---- G^ as an operand; G_0 = G^ + R^^T dY handed on
+            {
+                float gh[G_NB][4];
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    gh[n][0] = d_lo * G[n][0]; gh[n][1] = d_lo * G[n][1];
+                    gh[n][2] = d_hi * G[n][2]; gh[n][3] = d_hi * G[n][3];
+                }
+                st_tile(t_gb, moff, gh);
+            }
+            if (!mbar_wait(gb(GB_MA), mph, abort_flag)) ok = false;
+            tc_fence_after();
+            {
+                float dg[G_NB][4];
+#pragma unroll
+                for (int h2 = 0; h2 < G_H2; ++h2) tmem_ld_16x16_async2(tacc + GT_DG + 16 * h2, reinterpret_cast<float (&)[2][4]>(dg[2 * h2]));
+                tmem_ld_done();
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
+                    G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
+                }
+            }
+            if (it + 1 < nchunks) {
+                g_put(it & 1, G);
+                mbar_arrive(bar(GB_GREADY + (it & 1)));
+            } else if (p.dstate_in) {
+                store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
+            }
+            // ---- masked scores and their adjoint as operands
+#pragma unroll
+            for (int h2 = 0; h2 < G_H2; ++h2) {
+                const int blk = G_H2 * cx + h2;          // 16-column block of the tile; the diagonal one is blk == sp
+                if (blk < sp) {
+                    float pp[2][4], dp[2][4];
+                    tmem_ld_16x16_async2(tacc + GT_P + 16 * h2, pp);
+                    tmem_ld_16x16_async2(tacc + GT_DP + 16 * h2, dp);
+                    tmem_ld_done();
+                    st_half(t_pp + moff[h2], pp);
+                    st_half(t_dpp + moff[h2], dp);
+                } else if (blk > sp) {
+                    stsm_x4(t_pp + moff[h2], 0u, 0u, 0u, 0u);
+                    stsm_x4(t_dpp + moff[h2], 0u, 0u, 0u, 0u);
+                } else {
+                    float pp[2][4], dp[2][4];
+                    tmem_ld_16x16_async2(tacc + GT_P + 16 * h2, pp);
+                    tmem_ld_16x16_async2(tacc + GT_DP + 16 * h2, dp);
+                    float bon0 = 0.f, bon1 = 0.f;
+                    if (!C2) {
+#pragma unroll
+                        for (int o = 0; o < G_NSLAB; ++o) { bon0 += gld(GO_BP + 4 * (o * 64 + R0)); bon1 += gld(GO_BP + 4 * (o * 64 + R1)); }
+                    }
+                    tmem_ld_done();
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int row = e < 2 ? g : g + 8, col = 2 * q + 8 * n + (e & 1);       // inside the 16 x 16 block
+                            if (col == row) stsf(gbase + GO_DPD + 4 * (16 * sp + row), dp[n][e]);
+                            pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
+                            dp[n][e] = col < row ? dp[n][e] : 0.f;
+                        }
+                    st_half(t_pp + moff[h2], pp);
+                    st_half(t_dpp + moff[h2], dp);
+                }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            if (!gbar_and(grp, ok)) { alive = false; break; }
+            if (gt == 0) {
+                tc_fence_after();
+                const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
+                const uint64_t dS = smem_desc(t_sb), dG = smem_desc(t_gb), dP = smem_desc(t_pp), dD = smem_desc(t_dpp);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                    tc_mma(tmem + GT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
+                    tc_mma(tmem + GT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                    tc_mma(tmem + GT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
+                    tc_mma(tmem + GT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
+                }
+                tc_commit(gb(GB_MB));
+            }
+            ok = mbar_wait(gb(GB_MB), mph, abort_flag);
+            mph ^= 1;
+            tc_fence_after();
+            // ---- epilogue (the staging tiles take the place of the operand tiles S_0, G^, P', dP': all read by now)
+            float z[G_NB][4], qv[G_NB][4];
+#pragma unroll
+            for (int h2 = 0; h2 < G_H2; ++h2) {
+                // q and m take the operands as the tensor core saw them (rounded to bf16): the pair terms that q and
+                // m share, and that cancel in the suffix sums, are then the same products on both sides
+                float acc[2][4], o[2][4], hat[2][4], rv[2][4], kv[2][4];
+                const float pd0 = C2 ? 0.f : gld(GO_DPD + 4 * R0), pd1 = C2 ? 0.f : gld(GO_DPD + 4 * R1);
+                tmem_ld_16x16_async2(tacc + GT_DR + 16 * h2, acc);
+                ld_half(tr + moff[h2], rv);
+                ld_half(tk + moff[h2], kv);
+                ld_half(t_rh + moff[h2], hat);
+                tmem_ld_done();
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int nn = 2 * h2 + n;
+                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
+                        o[n][e] = fmaf(uc * kv[n][e], pd, acc[n][e] * ex2(a[nn][e] - lw2[nn][e]));
+                        qv[nn][e] = acc[n][e] * hat[n][e];
+                        if (!C2) du_acc[nn][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[nn][e & 1]);
+                    }
+                tmem_ld_16x16_async2(tacc + GT_DK + 16 * h2, acc);
+                ld_half(t_kh + moff[h2], hat);
+                tmem_ld_done();
+                st_half(t_out + moff[h2], o);
+#pragma unroll
+                for (int n = 0; n < 2; ++n)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int nn = 2 * h2 + n;
+                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
+                        o[n][e] = fmaf(uc * rv[n][e], pd, acc[n][e] * ex2(-a[nn][e]));
+                        z[nn][e] = qv[nn][e] - acc[n][e] * hat[n][e];
+                        if (C2) {
+                            // o is the gradient of k (1 - w): the key gets (1 - w) of it, and the decay logit its
+                            // share through the key factor, folded into the term that leaves the suffix sums
+                            const float omw = one_minus_ex2(lw2[nn][e]);
+                            qv[nn][e] = fmaf(o[n][e] * kv[n][e], 1.f - omw, qv[nn][e]);
+                            o[n][e] *= omw;
+                        }
+                    }
+                st_half(t_out + TILE + moff[h2], o);
+                tmem_ld_16x16_async2(tacc + GT_DV + 16 * h2, acc);
+                tmem_ld_done();
+                st_half(t_out + 2 * TILE + moff[h2], acc);
+            }
+            tc_fence_before();
+            ok = scan_rows<true>(z, gbase + GO_TOT, grp, sp, cb, lane, ok);
+            if (!ok) { alive = false; break; }
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n) {
+                float E0 = 0.f, E1 = 0.f;
+#pragma unroll
+                for (int o = 0; o < G_NSLAB; ++o) { const float2 ev = ldsf2(gbase + GO_EP + 4 * (o * 64 + cb + 8 * n)); E0 += ev.x; E1 += ev.y; }
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    z[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
+            }
+            st_tile(t_out + 3 * TILE, moff, z);
+        }
+        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one; then the
+        // group's input stage is free for its next chunk
+        fence_proxy_async();
+        gbar(grp);
+        if (valid < L) {
+            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
+            for (int i = gt; i < 4 * valid * 8; i += G_GT) {
+                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
+                uint32_t w[4];
+                lds_v4(t_out + tile * TILE + swz(t, blk << 4), w);
+                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        if (gt == 0) {
+            if (valid == L) {
+                const int row = (int)(row0 + (long long)c * L);
+                tma_store_2d(&tm_dr, col0, row, t_out);
+                tma_store_2d(&tm_dk, col0, row, t_out + TILE);
+                tma_store_2d(&tm_dv, col0, row, t_out + 2 * TILE);
+                tma_store_2d(&tm_dx, col0, row, t_out + 3 * TILE);
+                bulk_commit();
+            }
+            if (it + 2 < nchunks) issue_loads(it + 2);
+        }
+    }
+
+    // ---- the bonus gradient of this unit: over the lanes' rows, the row groups and the two groups, in a fixed order
+    if (!alive && gt == 0) sts32(abort_flag, 1u);    // (the other group's waits see it)
+    if (!C2) {
+#pragma unroll
+        for (int d = 4; d < 32; d <<= 1)
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) du_acc[n][e] += __shfl_xor_sync(0xffffffffu, du_acc[n][e], d);
+        if (g == 0) {
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) gsm(GO_REDV)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
+        }
+    }
+    if (gt == 0) {
+        bulk_wait<0>();                              // the gradient tiles have reached memory
+        if (last_load >= 0) mbar_wait(gb(GB_IN), (last_load >> 1) & 1, abort_flag, false);   // no copy into shared memory may stay in flight
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (!C2 && tid < 64 && !lds32(abort_flag)) {
+        float s = 0.f;
+#pragma unroll
+        for (int gg = 0; gg < 2; ++gg) {
+            const float* rv4 = reinterpret_cast<const float*>(smem + gg * GO_BYTES + GO_REDV);
+            const float* fb = reinterpret_cast<const float*>(smem + gg * GO_BYTES + GO_DUFB);
+            s += ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fb[tid];
+        }
+        p.du_part[(size_t)unit * 64 + tid] = s;
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(lds32(sbase + GS_TMEM), GT_COLS);
+    }
+}
+
+}  // namespace bg
+
+// Which gradient kernel the launcher uses: two groups of warps taking alternate chunks (default) or the single
+// lock-step set of wkv6_backward_chunked.cuh.
+#ifndef GF_BWD_GROUPS
+#define GF_BWD_GROUPS 1
+#endif
+
+// Workspace of the chunked gradient: checkpoints, per-unit bonus gradients, the token-by-token path's scratch (one
+// slot of 64 states per SM and group of warps).
+inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
+{
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    return ((size_t)units * nck * 4096 + (size_t)units * 64 + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+}
+
+inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                    const __nv_bfloat16* x, const float* u, const float* state_in,
+                                    const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
+                                    __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
+                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
+                                    bool c2 = false)
+{
+    const long long units = (long long)B * H, rows = (long long)B * T;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return GF_ERR_CUDA;
+    static PerDeviceFlag attr_set;
+    const int dev = current_device();
+    if (dev < 0) return GF_ERR_CUDA;
+    if (!attr_set.is_set(dev)) {
+        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::B_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bg::wkv6_backward_groups_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bg::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bg::wkv6_backward_groups_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bg::G_SMEM_ALLOC) != cudaSuccess)
+            return GF_ERR_CUDA;
+        attr_set.set(dev);
+    }
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    float* ckpt = ws;
+    float* du_part = ckpt + (size_t)units * nck * 4096;
+    float* fb = du_part + (size_t)units * 64;
+    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
+    if (s != GF_OK) return s;
+    const long long C = (long long)H * 64;
+    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
+    if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||
+        !ck::make_map(&tv, v, rows, C, 64) || !ck::make_map(&tdy, dy, rows, C, 64) || !ck::make_map(&tdr, dr, rows, C, 64) ||
+        !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
+        return GF_ERR_CUDA;
+    bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, GF_BWD_GROUPS ? 2 * n_sm : n_sm,
+                  wait_limit_us().load(std::memory_order_relaxed)};
+#if GF_BWD_GROUPS
+    if (c2) bg::wkv6_backward_groups_kernel<true><<<(unsigned)units, bg::G_THREADS, bg::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else bg::wkv6_backward_groups_kernel<false><<<(unsigned)units, bg::G_THREADS, bg::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+#else
+    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)units, bc::B_THREADS, bc::B_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+#endif
+    launches->fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    if (c2) return GF_OK;                            // no bonus, no bonus gradient
+    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
+
+}  // namespace gf
