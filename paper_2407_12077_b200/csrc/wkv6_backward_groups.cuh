@@ -279,6 +279,16 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
         const int use = it >> 1;                     // how often this group's input stage has been filled before
         float S0[G_NB][4];                              // the chunk-start state (requested early: it is used after the scan)
         load_f32_block(ck_unit + (size_t)c * 4096, S0);
+        if (it + 2 < nchunks) {
+            // this group's next chunk: its start state and its input tiles into L2 now, so that the copies issued at
+            // the end of this iteration and the load above find them there
+            if (gt < 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 2) * 4096 + 32 * gt));
+            if (gt == 128) {
+                const int row = (int)(row0 + (long long)(c - 2) * L);
+                tma_prefetch_2d(&tm_x, col0, row); tma_prefetch_2d(&tm_r, col0, row); tma_prefetch_2d(&tm_k, col0, row);
+                tma_prefetch_2d(&tm_v, col0, row); tma_prefetch_2d(&tm_dy, col0, row);
+            }
+        }
         // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
         bool ok = mbar_wait(gb(GB_IN), use & 1, abort_flag);
         if (gt == 0 && it > 1) bulk_wait_read<0>();  // the previous chunk's staging tiles have been read by the TMA unit
