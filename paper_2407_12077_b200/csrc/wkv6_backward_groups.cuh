@@ -61,11 +61,13 @@ constexpr int GO_SCAL = GO_DUFB + 256;            //   v . dy, sum r u k
 constexpr int GO_BYTES = (GO_SCAL + 16 + 1023) & ~1023;
 // shared by the groups
 constexpr int GS_GBUF = 2 * GO_BYTES;             // [2][64][64] float: the adjoint handed from chunk to chunk
-constexpr int GS_U = GS_GBUF + 2 * 16384;         // [64] float: the bonus
+constexpr int GS_EH = GS_GBUF + 2 * 16384;        // [2][NSLAB][64] float: partial E = rowsum(G * S) handed on with G
+constexpr int GS_U = GS_EH + 2 * G_NSLAB * 256;   // [64] float: the bonus
 constexpr int GS_ABORT = GS_U + 256;              // abort word, wait limit
 constexpr int GS_TMEM = GS_ABORT + 8;
-constexpr int GS_BAR = GS_TMEM + 8;               // per group: inputs, first / second group of products; then the hand-over pair
-enum { GB_IN = 0, GB_MA = 1, GB_MB = 2, GB_PER_GROUP = 3, GB_GREADY = 6, GB_COUNT = 8 };
+// mbarriers, per group: inputs x, v, dy / inputs r, k / first group of products / dR^ and dK^ / dV; then the hand-over pair
+constexpr int GS_BAR = GS_TMEM + 8;
+enum { GB_INA = 0, GB_INB = 1, GB_MA = 2, GB_MRK = 3, GB_MV = 4, GB_PER_GROUP = 5, GB_GREADY = 10, GB_COUNT = 12 };
 constexpr int G_SMEM_BYTES = GS_BAR + 8 * GB_COUNT;
 constexpr int G_SMEM_ALLOC = G_SMEM_BYTES + 1024;
 static_assert(G_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
@@ -238,17 +240,26 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
     const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
     const uint32_t t_rh = gbase + GO_RH, t_kh = gbase + GO_KH;
     const uint32_t t_sb = gbase + GO_T4, t_gb = t_sb + TILE, t_pp = t_sb + 2 * TILE, t_dpp = t_sb + 3 * TILE;
-    const uint32_t t_out = gbase + GO_T4;
-    int last_load = -1;                              // (thread 0 of the group) the last iteration whose copies were issued
-    auto issue_loads = [&](int it) {                 // thread 0 of the group
+    // staging tiles of the four gradients, each over an operand tile that is dead when it is written: dr over S_0 and
+    // dk over dP' (free once dR^ and dK^ are complete), dv over P' and dx over G^ (free once dV is complete)
+    const uint32_t o_dr = t_sb, o_dk = t_dpp, o_dv = t_pp, o_dx = t_gb;
+    // The input copies of a chunk come in two parts, each issued as soon as its tiles are free: x, v, dy once the
+    // chunk before (of this group) has finished its products, r, k once its epilogue has read them.
+    int last_a = -1, last_b = -1;                    // (thread 0 of the group) the last iterations whose copies were issued
+    auto issue_loads_a = [&](int it) {               // thread 0 of the group
         const int row = (int)(row0 + (long long)chunk_of(it) * L);
-        mbar_expect_tx(gb(GB_IN), 5 * TILE);
-        tma_load_2d(tx, &tm_x, col0, row, gb(GB_IN));
-        tma_load_2d(tr, &tm_r, col0, row, gb(GB_IN));
-        tma_load_2d(tk, &tm_k, col0, row, gb(GB_IN));
-        tma_load_2d(tv, &tm_v, col0, row, gb(GB_IN));
-        tma_load_2d(tdy, &tm_dy, col0, row, gb(GB_IN));
-        last_load = it;
+        mbar_expect_tx(gb(GB_INA), 3 * TILE);
+        tma_load_2d(tx, &tm_x, col0, row, gb(GB_INA));
+        tma_load_2d(tv, &tm_v, col0, row, gb(GB_INA));
+        tma_load_2d(tdy, &tm_dy, col0, row, gb(GB_INA));
+        last_a = it;
+    };
+    auto issue_loads_b = [&](int it) {
+        const int row = (int)(row0 + (long long)chunk_of(it) * L);
+        mbar_expect_tx(gb(GB_INB), 2 * TILE);
+        tma_load_2d(tr, &tm_r, col0, row, gb(GB_INB));
+        tma_load_2d(tk, &tm_k, col0, row, gb(GB_INB));
+        last_b = it;
     };
     auto load_f32_block = [&](const float* src, float (&v)[G_NB][4]) {      // [64][64] fp32 block, the lane's cells
 #pragma unroll
@@ -270,7 +281,7 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
-    if (gt == 0 && grp < nchunks) issue_loads(grp);
+    if (gt == 0 && grp < nchunks) { issue_loads_a(grp); issue_loads_b(grp); }
     int mph = 0;                                     // phase bit of this group's two product barriers
     bool alive = true;
 
@@ -290,15 +301,8 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
             }
         }
         // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
-        bool ok = mbar_wait(gb(GB_IN), use & 1, abort_flag);
+        bool ok = mbar_wait(gb(GB_INA), use & 1, abort_flag);
         if (gt == 0 && it > 1) bulk_wait_read<0>();  // the previous chunk's staging tiles have been read by the TMA unit
-        if (valid < L) {
-            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
-            for (int i = gt; i < (L - valid) * 8; i += G_GT) {
-                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
-                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
-            }
-        }
         float a[G_NB][4], lw2[G_NB][4];
         {
             float xv[G_NB][4];
@@ -324,6 +328,15 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
             safe = (al0 >= -A2_MAX) && (al1 >= -A2_MAX);                   // false for NaN as well
         }
         // ---- operands from the inputs: R^, K^ (and the bonus), the chunk-start state
+        if (!mbar_wait(gb(GB_INB), use & 1, abort_flag)) ok = false;        // (made uniform at a later barrier)
+        if (valid < L) {
+            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
+            for (int i = gt; i < (L - valid) * 8; i += G_GT) {
+                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
+                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
+            }
+            gbar(grp);
+        }
         {
             float rv[G_NB][4], kv[G_NB][4];
             ld_tile(tr, moff, rv);
@@ -350,8 +363,6 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
             }
         }
         st_tile(t_sb, moff, S0);
-        float SL[G_NB][4];                           // the state at the chunk's end (for E), in flight over the barrier and the hand-over wait
-        load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
         fence_proxy_async();
         tc_fence_before();
         const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
@@ -380,17 +391,25 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
             if (!mbar_wait(bar(GB_GREADY + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag)) ok = false;
             g_get((it - 1) & 1, G);
         }
-        {
-            // E = rowsum(G_L * S_L), S_L = the state before the next chunk (after the last token for the last chunk)
+        // E = rowsum(G_L * S_L), S_L the state at the chunk's end, as partial sums per column slab: for the call's last
+        // chunk from the final state; else the group that made G_L formed them from its chunk-start state (e_put below)
+        auto e_put = [&](uint32_t dst, const float (&Gm)[G_NB][4], const float (&Sm)[G_NB][4]) {
             float e0 = 0.f, e1 = 0.f;
 #pragma unroll
             for (int n = 0; n < G_NB; ++n) {
-                e0 = fmaf(G[n][0], SL[n][0], fmaf(G[n][1], SL[n][1], e0));
-                e1 = fmaf(G[n][2], SL[n][2], fmaf(G[n][3], SL[n][3], e1));
+                e0 = fmaf(Gm[n][0], Sm[n][0], fmaf(Gm[n][1], Sm[n][1], e0));
+                e1 = fmaf(Gm[n][2], Sm[n][2], fmaf(Gm[n][3], Sm[n][3], e1));
             }
             e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
             e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
-            if (q == 0) { stsf(gbase + GO_EP + 4 * (cx * 64 + R0), e0); stsf(gbase + GO_EP + 4 * (cx * 64 + R1), e1); }
+            if (q == 0) { stsf(dst + 4 * (cx * 64 + R0), e0); stsf(dst + 4 * (cx * 64 + R1), e1); }
+        };
+        if (it == 0) {
+            float SL[G_NB][4];
+            load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
+            e_put(gbase + GO_EP, G, SL);
+        } else if (gt < G_NSLAB * 64) {
+            stsf(gbase + GO_EP + 4 * gt, ldsf(sbase + GS_EH + 4 * (((it - 1) & 1) * G_NSLAB * 64 + gt)));      // (a private copy: the slot is rewritten two chunks on)
         }
 
         if (unsafe) {
@@ -498,26 +517,28 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
                     const float xc = lds_bf16(tx + swz(t, 2 * cc)), kc = lds_bf16(tk + swz(t, 2 * cc)), rc = lds_bf16(tr + swz(t, 2 * cc));
                     const float ec = expf(xc), wc = expf(-ec);
                     if (C2) {
-                        sts_bf16(t_out + swz(t, 2 * cc), s_r);
-                        sts_bf16(t_out + TILE + swz(t, 2 * cc), s_k * -expm1f(-ec));
-                        sts_bf16(t_out + 3 * TILE + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
+                        sts_bf16(o_dr + swz(t, 2 * cc), s_r);
+                        sts_bf16(o_dk + swz(t, 2 * cc), s_k * -expm1f(-ec));
+                        sts_bf16(o_dx + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
                     } else {
                         const float uc = ub[cc], vd = scal[0];
-                        sts_bf16(t_out + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
-                        sts_bf16(t_out + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
-                        sts_bf16(t_out + 3 * TILE + swz(t, 2 * cc), s_g * (-wc * ec));
+                        sts_bf16(o_dr + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
+                        sts_bf16(o_dk + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
+                        sts_bf16(o_dx + swz(t, 2 * cc), s_g * (-wc * ec));
                         gsm(GO_DUFB)[cc] = fmaf(rc * kc, vd, gsm(GO_DUFB)[cc]);
                     }
                 } else if (gt < 128) {
                     const int j = gt - 64;
                     const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
-                    sts_bf16(t_out + 2 * TILE + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
+                    sts_bf16(o_dv + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
                 }
                 gbar(grp);
             }
-            // hand the adjoint on
+            // hand the adjoint on (and the row sums the next chunk needs, from the fp32 state: the operand tile is gone)
             if (it + 1 < nchunks) {
                 g_put(it & 1, G);
+                load_f32_block(ck_unit + (size_t)c * 4096, S);
+                e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, S);
                 mbar_arrive(bar(GB_GREADY + (it & 1)));
             } else if (p.dstate_in) {
                 store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
@@ -548,6 +569,11 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
             }
             if (it + 1 < nchunks) {
                 g_put(it & 1, G);
+                {
+                    float sb[G_NB][4];               // this chunk's start state is the next chunk's end state (bf16 copy: the operand tile)
+                    ld_tile(t_sb, moff, sb);
+                    e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, sb);
+                }
                 mbar_arrive(bar(GB_GREADY + (it & 1)));
             } else if (p.dstate_in) {
                 store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
@@ -596,24 +622,34 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
                 tc_fence_after();
                 const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
                 const uint64_t dS = smem_desc(t_sb), dG = smem_desc(t_gb), dP = smem_desc(t_pp), dD = smem_desc(t_dpp);
+                // dR^ and dK^ first (interleaved: products on one accumulator wait for each other), with a commit of
+                // their own: the epilogue starts on them while dV is still being formed
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;
-                    tc_mma(tmem + GT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                    const uint64_t ks = 2 * kk;
                     tc_mma(tmem + GT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
                     tc_mma(tmem + GT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
                 }
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
                     const uint64_t ks = 2 * kk, ms = 128 * kk;
-                    tc_mma(tmem + GT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
                     tc_mma(tmem + GT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
                     tc_mma(tmem + GT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
                 }
-                tc_commit(gb(GB_MB));
+                tc_commit(gb(GB_MRK));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                }
+                tc_commit(gb(GB_MV));
             }
-            ok = mbar_wait(gb(GB_MB), mph, abort_flag);
-            mph ^= 1;
+            ok = mbar_wait(gb(GB_MRK), mph, abort_flag);
             tc_fence_after();
             // ---- epilogue (the staging tiles take the place of the operand tiles S_0, G^, P', dP': all read by now)
             float z[G_NB][4], qv[G_NB][4];
@@ -641,7 +677,7 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
                 tmem_ld_16x16_async2(tacc + GT_DK + 16 * h2, acc);
                 ld_half(t_kh + moff[h2], hat);
                 tmem_ld_done();
-                st_half(t_out + moff[h2], o);
+                st_half(o_dr + moff[h2], o);
 #pragma unroll
                 for (int n = 0; n < 2; ++n)
 #pragma unroll
@@ -658,14 +694,24 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
                             o[n][e] *= omw;
                         }
                     }
-                st_half(t_out + TILE + moff[h2], o);
-                tmem_ld_16x16_async2(tacc + GT_DV + 16 * h2, acc);
+                st_half(o_dk + moff[h2], o);
+            }
+            // dV: every product of the chunk has completed, so x, v, dy can take the group's next chunk
+            if (!mbar_wait(gb(GB_MV), mph, abort_flag)) ok = false;
+            mph ^= 1;
+            tc_fence_after();
+            if (gt == 0 && it + 2 < nchunks) issue_loads_a(it + 2);
+            {
+                float acc[G_NB][4];
+#pragma unroll
+                for (int h2 = 0; h2 < G_H2; ++h2) tmem_ld_16x16_async2(tacc + GT_DV + 16 * h2, reinterpret_cast<float (&)[2][4]>(acc[2 * h2]));
                 tmem_ld_done();
-                st_half(t_out + 2 * TILE + moff[h2], acc);
+                st_tile(o_dv, moff, acc);
             }
             tc_fence_before();
             ok = scan_rows<true>(z, gbase + GO_TOT, grp, sp, cb, lane, ok);
             if (!ok) { alive = false; break; }
+            if (gt == 0 && it + 2 < nchunks) issue_loads_b(it + 2);      // (r, k were last read before the barrier of the sums)
 #pragma unroll
             for (int n = 0; n < G_NB; ++n) {
                 float E0 = 0.f, E1 = 0.f;
@@ -675,31 +721,30 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
                 for (int e = 0; e < 4; ++e)
                     z[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
             }
-            st_tile(t_out + 3 * TILE, moff, z);
+            st_tile(o_dx, moff, z);
         }
-        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one; then the
-        // group's input stage is free for its next chunk
+        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one
         fence_proxy_async();
         gbar(grp);
         if (valid < L) {
-            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
+            __nv_bfloat16* outs[4] = {p.dr, p.dx, p.dv, p.dk};       // in the order of the staging tiles in shared memory
             for (int i = gt; i < 4 * valid * 8; i += G_GT) {
                 const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
                 uint32_t w[4];
-                lds_v4(t_out + tile * TILE + swz(t, blk << 4), w);
+                lds_v4(t_sb + tile * TILE + swz(t, blk << 4), w);
                 *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
         if (gt == 0) {
             if (valid == L) {
                 const int row = (int)(row0 + (long long)c * L);
-                tma_store_2d(&tm_dr, col0, row, t_out);
-                tma_store_2d(&tm_dk, col0, row, t_out + TILE);
-                tma_store_2d(&tm_dv, col0, row, t_out + 2 * TILE);
-                tma_store_2d(&tm_dx, col0, row, t_out + 3 * TILE);
+                tma_store_2d(&tm_dr, col0, row, o_dr);
+                tma_store_2d(&tm_dk, col0, row, o_dk);
+                tma_store_2d(&tm_dv, col0, row, o_dv);
+                tma_store_2d(&tm_dx, col0, row, o_dx);
                 bulk_commit();
             }
-            if (it + 2 < nchunks) issue_loads(it + 2);
+            if (unsafe && it + 2 < nchunks) { issue_loads_a(it + 2); issue_loads_b(it + 2); }      // (the other path has issued them)
         }
     }
 
@@ -721,7 +766,9 @@ wkv6_backward_groups_kernel(const __grid_constant__ CUtensorMap tm_x, const __gr
     }
     if (gt == 0) {
         bulk_wait<0>();                              // the gradient tiles have reached memory
-        if (last_load >= 0) mbar_wait(gb(GB_IN), (last_load >> 1) & 1, abort_flag, false);   // no copy into shared memory may stay in flight
+        // no copy into shared memory may stay in flight
+        if (last_a >= 0) mbar_wait(gb(GB_INA), (last_a >> 1) & 1, abort_flag, false);
+        if (last_b >= 0) mbar_wait(gb(GB_INB), (last_b >> 1) & 1, abort_flag, false);
     }
     tc_fence_before();
     __syncthreads();
