@@ -12,7 +12,6 @@
 #include "ln_heads.cuh"
 #include "wkv6_backward.cuh"
 #include "wkv6_backward_chunked.cuh"
-#include "wkv6_backward_groups.cuh"
 #include "wkv6_chunked.cuh"
 #include "wkv6_exact.cuh"
 #include "wkv6_step.cuh"

@@ -16,16 +16,31 @@
 // Nine 64x64x64 bf16 tcgen05 products per chunk, accumulators in tensor memory.  The chunk-start states S_0 come from
 // a checkpoint pass of the forward kernel (state only), one 64x64 fp32 block per chunk.
 //
-// One CTA of 512 threads per unit works in phases separated by CTA barriers; an elected thread issues the TMA
-// copies and the products.  Every elementwise step uses the accumulator layout of the 64-row products: warp
-// (sp = warp % 4, cq = warp / 4) owns rows 16 sp .. +15 and columns 16 cq .. +15 of every 64x64 tile, a lane
-// (g = lane / 4, q = lane % 4) rows 16 sp + g and + 8, columns 16 cq + 8 n + 2 q + e (n, e in {0, 1}); bf16 tiles
-// move through ldmatrix / stmatrix in that layout, so scale factors computed for the operands stay in registers
-// until the epilogue needs them.  Sums along the tokens (cumulative decay, the suffix sums of the decay gradient)
-// run over lanes by shuffles and over the four row groups through shared memory.
-// A chunk in which some channel decays by more than 2^-96 is processed token by token in fp32 on the ALUs (its
-// states recomputed into a per-SM scratch in global memory), so any decay logit gives the gradient of the exact
-// recurrence.  Every wait is bounded; on expiry the status flag is raised and the whole CTA leaves together.
+// Two chunks are in flight per CTA.  A chunk's phases (decay -> cumulative sum -> operands -> products -> masks ->
+// products -> epilogue -> suffix sums) depend on one another and each keeps a different pipe busy, so one set of warps
+// that walks them in lock step leaves most issue slots empty.  The CTA's 16 warps therefore form two groups of 8 that
+// take alternate chunks and run half a period apart: while one group waits for its products or sits in a
+// latency-bound phase, the other one issues.  The only thing a chunk needs from the chunk after it (in time) is the
+// adjoint at its end, G_L = G_0 of that chunk, and it enters late (the operand G^ = diag(D) G_L and G_0 = G^ + R^^T dY,
+// whose product needs no G), so the groups hand G to each other through a pair of fp32 tiles in shared memory, each
+// guarded by an mbarrier that all threads of the writing group arrive on; the row sums E travel with it (the group
+// that made G_L forms them from its own chunk-start state, which is the next chunk's end state).
+//
+// Layout inside a group: warp (sp = warp % 4, cx = warp / 4 % 2) owns rows 16 sp .. +15 and columns 32 cx .. +31 of
+// every 64x64 tile; lane (g = lane / 4, q = lane % 4) rows 16 sp + g and + 8, columns 32 cx + 8 n + 2 q + e (n < 4,
+// e < 2): 16 cells, the accumulator layout of the 64-row products, in which bf16 tiles move through ldmatrix /
+// stmatrix, so nothing is transposed and a lane's cells are the same in every phase.  (G_NB = 2 gives groups of 16
+// warps with 8 cells per lane at 64 registers instead: measured slower, the spills cost more than the warps bring.)
+// Each group has its own input stage (x, v, dy and r, k by TMA, each part re-filled as soon as its tiles fall free),
+// operand tiles, tensor-memory columns (three accumulators that the second group of products reuses once the first
+// group's have been read) and barriers; the four staging tiles of the gradients lie over operand tiles that are dead
+// by the time they are written.  Thread 0 of a group issues its products and copies.  Sums along the tokens (the
+// cumulative decay; the suffix sums of the decay gradient) run over lanes by shuffles and across the four row groups
+// through shared memory.  Waits are per thread and bounded; their outcome is made uniform over the group at its next
+// barrier, and the hand-over waits watch the CTA's abort word, so after a wait that ran out both groups leave.
+// A chunk in which a channel decays by more than 2^-96 runs token by token in fp32 on its group's warps (its 64
+// states recomputed into a scratch slot of the workspace), so any decay logit gives the gradient of the exact
+// recurrence.
 #pragma once
 #include "wkv6_chunked.cuh"
 
@@ -34,41 +49,8 @@ namespace bc {
 
 using namespace ck;          // PTX wrappers, descriptors, layout helpers of the forward kernel
 
-constexpr bool B_ISSUER = false;                 // a 17th warp issues the products and the TMA copies (else thread 0 does)
-constexpr int B_CTHREADS = 512;                  // 16 compute warps
-constexpr int B_THREADS = B_CTHREADS + (B_ISSUER ? 32 : 0);
 constexpr float LN2 = 0.6931471805599453f;
-// tensor memory columns of the six accumulators
-constexpr int BT_P = 0, BT_DP = 64, BT_DV = 128, BT_DR = 192, BT_DK = 256, BT_DG = 320, BT_COLS = 512;
-// shared memory map (offsets from a 1024-byte aligned base); input stage: x, r, k, v, dy
-constexpr int B_STAGE = 5 * TILE;
-constexpr int BO_IN = 0;                          // [2][B_STAGE]
-constexpr int BO_RH = BO_IN + 2 * B_STAGE;        // [2] R^ [t][c]        (by chunk parity, like the input stages)
-constexpr int BO_KH = BO_RH + 2 * TILE;           // [2] K^ [i][c]
-constexpr int BO_SB = BO_KH + 2 * TILE;           // [2] S_0 [c][j] bf16
-constexpr int BO_GB = BO_SB + 2 * TILE;           // [2] G^  [c][j] bf16
-constexpr int BO_PP = BO_GB + 2 * TILE;           // P' [t][i]
-constexpr int BO_DPP = BO_PP + TILE;              // dP' [t][i]
-constexpr int BO_OUT = BO_DPP + TILE;             // dr, dk, dv, dx staging [t][c]
-constexpr int BO_TOT = BO_OUT + 4 * TILE;         // [4][64] float: row-group totals of a scan
-constexpr int BO_EP = BO_TOT + 1024;              // [2][4][64] float: partial E by column group (by chunk parity)
-constexpr int BO_BP = BO_EP + 2048;               // [4][64] float: partial bonus by column group
-constexpr int BO_DPD = BO_BP + 1024;              // [64] float: dy_t . v_t
-constexpr int BO_RED = BO_DPD + 256;              // token-by-token path: [4][3][64] + [4][64] + du[64] + 2 floats
-constexpr int BO_RED_V = BO_RED + 4 * 3 * 64 * 4;
-constexpr int BO_DU_FB = BO_RED_V + 4 * 64 * 4;
-constexpr int BO_SCAL = BO_DU_FB + 256;
-constexpr int BO_ABORT = BO_SCAL + 16;            // abort word, wait limit
-constexpr int BO_TMEM = BO_ABORT + 8;
-constexpr int BO_CMD = BO_TMEM + 8;               // [4] {command, argument} for the issuing warp
-constexpr int BO_BAR = BO_CMD + 32;               // mbarriers: input full [2], first / second group of products done,
-// ... staging tiles read by the TMA unit, command slots [4]
-enum { BB_IN = 0, BB_MMA1 = 2, BB_MMA2 = 3, BB_STAGING = 4, BB_CMD = 5, BB_COUNT = 9 };
-enum { CMD_QUIT = 0, CMD_MMA1 = 1, CMD_MMA2 = 2, CMD_STORE = 3 };
-constexpr int B_SMEM_BYTES = BO_BAR + 8 * BB_COUNT;
-constexpr int B_SMEM_ALLOC = B_SMEM_BYTES + 1024;
-static_assert(B_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
-constexpr size_t FB_SLOT_FLOATS = (size_t)64 * 4096;      // scratch of the token-by-token path per SM: 64 states
+constexpr size_t FB_SLOT_FLOATS = (size_t)64 * 4096;      // scratch of the token-by-token path per SM and group: 64 states
 
 struct BParams {
     const float* u;              // [H][64]
@@ -104,20 +86,6 @@ __device__ __forceinline__ unsigned smid()
     return v;
 }
 
-// Barrier over the 16 compute warps (the issuing warp does not take part), and the same with an AND over a predicate.
-__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
-__device__ __forceinline__ bool cbar_and(bool ok)
-{
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.and.pred q, 1, 512, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)ok) : "memory");
-    return r != 0;
-}
-
 // 1 - 2^l for l <= 0 without the cancellation of the direct form near l = 0 (slow decays): the series of -expm1 there.
 __device__ __forceinline__ float one_minus_ex2(float l)
 {
@@ -126,50 +94,117 @@ __device__ __forceinline__ float one_minus_ex2(float l)
     return l > -0.125f ? series : 1.f - ex2(l);
 }
 
-// tcgen05.ld of a 16 x 16 fp32 block without the wait for its data (tmem_ld_done() before the first use): several
-// loads can then be in flight together.
-__device__ __forceinline__ void tmem_ld_16x16_async(uint32_t taddr, float (&v)[2][4])
+__device__ __forceinline__ void tmem_ld_done() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// NB = 8-column blocks per lane: 4 (groups of 8 warps, 16 cells per lane, 128 registers) or 2 (groups of 16 warps,
+// 8 cells per lane, 64 registers)
+constexpr int G_NB = 4;
+constexpr int G_NSLAB = 8 / G_NB;                 // column slabs of 8 NB columns per tile = warps per row group
+constexpr int G_H2 = G_NB / 2;                    // 16-column blocks per lane
+constexpr int G_GT = 32 * 4 * G_NSLAB;            // threads of one group
+constexpr int G_THREADS = 2 * G_GT;               // the CTA
+// tensor memory: per group 256 columns, three accumulators used twice
+constexpr int GT_P = 0, GT_DP = 64, GT_DG = 128, GT_DV = 0, GT_DR = 64, GT_DK = 128, GT_COLS = 512;
+// shared memory of one group
+constexpr int GO_IN = 0;                          // x, r, k, v, dy
+constexpr int GO_RH = GO_IN + 5 * TILE;           // R^ [t][c]
+constexpr int GO_KH = GO_RH + TILE;               // K^ [i][c]
+constexpr int GO_T4 = GO_KH + TILE;               // S_0, G^, P', dP' operand tiles; later the dr, dk, dv, dx staging tiles
+constexpr int GO_TOT = GO_T4 + 4 * TILE;          // [4][64] float: row-group totals of a scan
+constexpr int GO_EP = GO_TOT + 1024;              // [NSLAB][64] float: partial E by column slab
+constexpr int GO_BP = GO_EP + 1024;               // [NSLAB][64] float: partial bonus by column slab
+constexpr int GO_DPD = GO_BP + 1024;              // [64] float: dy_t . v_t
+constexpr int GO_RED = GO_DPD + 256;              // token-by-token path: [NSLAB][3][64]
+constexpr int GO_REDV = GO_RED + 4 * 3 * 64 * 4;  //   [4][64]
+constexpr int GO_DUFB = GO_REDV + 1024;           //   du [64]
+constexpr int GO_SCAL = GO_DUFB + 256;            //   v . dy, sum r u k
+constexpr int GO_BYTES = (GO_SCAL + 16 + 1023) & ~1023;
+// shared by the groups
+constexpr int GS_GBUF = 2 * GO_BYTES;             // [2][64][64] float: the adjoint handed from chunk to chunk
+constexpr int GS_EH = GS_GBUF + 2 * 16384;        // [2][NSLAB][64] float: partial E = rowsum(G * S) handed on with G
+constexpr int GS_U = GS_EH + 2 * G_NSLAB * 256;   // [64] float: the bonus
+constexpr int GS_ABORT = GS_U + 256;              // abort word, wait limit
+constexpr int GS_TMEM = GS_ABORT + 8;
+// mbarriers, per group: inputs x, v, dy / inputs r, k / first group of products / dR^ and dK^ / dV; then the hand-over pair
+constexpr int GS_BAR = GS_TMEM + 8;
+enum { GB_INA = 0, GB_INB = 1, GB_MA = 2, GB_MRK = 3, GB_MV = 4, GB_PER_GROUP = 5, GB_GREADY = 10, GB_COUNT = 12 };
+constexpr int G_SMEM_BYTES = GS_BAR + 8 * GB_COUNT;
+constexpr int G_SMEM_ALLOC = G_SMEM_BYTES + 1024;
+static_assert(G_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
+
+// barrier over one group's 8 warps (ids 1 and 2), plain and with an AND over a predicate
+__device__ __forceinline__ void gbar(int grp) { asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(G_GT) : "memory"); }
+__device__ __forceinline__ bool gbar_and(int grp, bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "bar.red.and.pred q, %1, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(grp + 1), "r"((uint32_t)ok), "n"(G_GT) : "memory");
+    return r != 0;
+}
+
+// explicit shared-space accesses (a pointer rebuilt from an integer would make them generic loads)
+__device__ __forceinline__ float2 ldsf2(uint32_t a)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void stsf2(uint32_t a, float2 v) { asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(a), "f"(v.x), "f"(v.y) : "memory"); }
+
+// 16 rows x 16 columns of an accumulator, without the wait (tmem_ld_done() before the first use)
+__device__ __forceinline__ void tmem_ld_16x16_async2(uint32_t taddr, float (&v)[2][4])
 {
     asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=f"(v[0][0]), "=f"(v[0][1]), "=f"(v[0][2]), "=f"(v[0][3]), "=f"(v[1][0]), "=f"(v[1][1]), "=f"(v[1][2]), "=f"(v[1][3])
                  : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_done() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// v[n][0..1] = (row g, columns 8n+2q, +1), v[n][2..3] = (row g+8, same columns) of this warp's 16 x 16 block
-__device__ __forceinline__ void load_block_bf16(uint32_t addr, float (&v)[2][4])
+// 16 x 16 bf16 blocks of a swizzled tile <-> two column blocks (n = 2 h2, 2 h2 + 1) of the lane's cells
+__device__ __forceinline__ void ld_half(uint32_t addr, float (&v)[2][4])
 {
     uint32_t w0, w1, w2, w3;
     ldsm_x4(addr, w0, w1, w2, w3);
     v[0][0] = bf_lo(w0); v[0][1] = bf_hi(w0); v[0][2] = bf_lo(w1); v[0][3] = bf_hi(w1);
     v[1][0] = bf_lo(w2); v[1][1] = bf_hi(w2); v[1][2] = bf_lo(w3); v[1][3] = bf_hi(w3);
 }
-__device__ __forceinline__ void store_block_bf16(uint32_t addr, const float (&v)[2][4])
+__device__ __forceinline__ void st_half(uint32_t addr, const float (&v)[2][4])
 {
     stsm_x4(addr, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
 }
-
-// Inclusive sums along the 64 rows of a tile held in the accumulator layout: forwards (REV = false: row t gets the
-// sum over rows <= t) or backwards (REV = true: rows >= t).  tot: [4][64] floats of shared memory.  Contains one
-// barrier of the compute warps (all 512 threads call it together), which also forms the AND of `ok` over them: the
-// result is returned (a wait that ran out on some thread makes every thread leave together).
-template <bool REV>
-__device__ __forceinline__ bool scan_rows(float (&v)[2][4], uint32_t tot, int sp, int cq, int lane, bool ok)
+__device__ __forceinline__ void ld_tile(uint32_t tile, const uint32_t (&moff)[G_H2], float (&v)[G_NB][4])
 {
-    const int g = lane >> 2, q = lane & 3;
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2) ld_half(tile + moff[h2], reinterpret_cast<float (&)[2][4]>(v[2 * h2]));
+}
+__device__ __forceinline__ void st_tile(uint32_t tile, const uint32_t (&moff)[G_H2], const float (&v)[G_NB][4])
+{
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2) st_half(tile + moff[h2], reinterpret_cast<const float (&)[2][4]>(v[2 * h2]));
+}
+
+// Inclusive sums along the 64 rows of a tile in the group's layout, forwards (rows <= t) or backwards (rows >= t).
+// tot: [4][64] floats of the group's shared memory.  Contains one barrier of the group, which also forms the AND of
+// `ok` over it (returned).
+template <bool REV>
+__device__ __forceinline__ bool scan_rows(float (&v)[G_NB][4], uint32_t tot, int grp, int sp, int cb, int lane, bool ok)
+{
+    const int g = lane >> 2, q = lane & 3;           // (cb: the lane's first column, a multiple of 2)
 #pragma unroll
     for (int d = 4; d < 32; d <<= 1) {
 #pragma unroll
-        for (int n = 0; n < 2; ++n)
+        for (int n = 0; n < G_NB; ++n)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float o = REV ? __shfl_down_sync(0xffffffffu, v[n][e], d) : __shfl_up_sync(0xffffffffu, v[n][e], d);
                 if (REV ? lane + d < 32 : lane >= d) v[n][e] += o;
             }
     }
-    // the other half's total: rows g+8 follow rows g
 #pragma unroll
-    for (int n = 0; n < 2; ++n)
+    for (int n = 0; n < G_NB; ++n)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             if (REV) v[n][e] += __shfl_sync(0xffffffffu, v[n][2 + e], q);
@@ -177,17 +212,16 @@ __device__ __forceinline__ bool scan_rows(float (&v)[2][4], uint32_t tot, int sp
         }
     if (g == (REV ? 0 : 7)) {
 #pragma unroll
-        for (int n = 0; n < 2; ++n)
-            *reinterpret_cast<float2*>(__cvta_shared_to_generic((size_t)(tot + 4 * (sp * 64 + 16 * cq + 8 * n + 2 * q)))) =
-                REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]);
+        for (int n = 0; n < G_NB; ++n)
+            stsf2(tot + 4 * (sp * 64 + cb + 8 * n), REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]));
     }
-    ok = cbar_and(ok);
+    ok = gbar_and(grp, ok);
 #pragma unroll
     for (int o = 0; o < 4; ++o) {
         if (REV ? o > sp : o < sp) {
 #pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                const float2 t = *reinterpret_cast<const float2*>(__cvta_shared_to_generic((size_t)(tot + 4 * (o * 64 + 16 * cq + 8 * n + 2 * q))));
+            for (int n = 0; n < G_NB; ++n) {
+                const float2 t = ldsf2(tot + 4 * (o * 64 + cb + 8 * n));
                 v[n][0] += t.x; v[n][1] += t.y; v[n][2] += t.x; v[n][3] += t.y;
             }
         }
@@ -195,225 +229,146 @@ __device__ __forceinline__ bool scan_rows(float (&v)[2][4], uint32_t tot, int sp
     return ok;
 }
 
-// C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus; the second-value vector only adds to the
-// output, so its gradient is dy itself and nothing here depends on it).
 template <bool C2>
-__global__ void __launch_bounds__(B_THREADS, 1)
+__global__ void __launch_bounds__(G_THREADS, 1)
 wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
-                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                             const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
-                             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
-                             const __grid_constant__ CUtensorMap tm_dx, const BParams p)
+                            const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                            const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
+                            const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
+                            const __grid_constant__ CUtensorMap tm_dx, const BParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t abort_flag = sbase + BO_ABORT;
-    auto bar = [&](int i) { return sbase + BO_BAR + 8 * i; };
-    auto fsm = [&](int off) { return reinterpret_cast<float*>(smem + off); };
+    const uint32_t abort_flag = sbase + GS_ABORT;
+    auto bar = [&](int i) { return sbase + GS_BAR + 8 * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int sp = warp & 3, cq = warp >> 2, g = lane >> 2, q = lane & 3;
+    const int grp = tid / G_GT, gt = tid % G_GT;                    // group, thread inside the group
+    const int sp = warp & 3, cx = (warp >> 2) % G_NSLAB, g = lane >> 2, q = lane & 3;       // row group, column slab
     const int unit = blockIdx.x, seq = unit / p.H, h = unit % p.H;
     const int T = p.T, nchunks = (T + L - 1) / L;
     const long long row0 = (long long)seq * T;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
-    const int cb = 16 * cq + 2 * q;                  // its columns: cb + 8 n + e
-    // byte offset of this lane's ldmatrix / stmatrix row inside a tile (the warp's 16 x 16 block)
-    const uint32_t moff = swz(16 * sp + (lane & 7) + 8 * ((lane >> 3) & 1), (2 * cq + (lane >> 4)) << 4);
+    const int cb = 8 * G_NB * cx + 2 * q;            // its columns: cb + 8 n + e, n < G_NB
+    // byte offsets of this lane's ldmatrix / stmatrix rows inside a tile: the warp's 16 x 16 blocks
+    uint32_t moff[G_H2];
+#pragma unroll
+    for (int h2 = 0; h2 < G_H2; ++h2)
+        moff[h2] = swz(16 * sp + (lane & 7) + 8 * ((lane >> 3) & 1), (G_NB * cx + 2 * h2 + (lane >> 4)) << 4);
+    const uint32_t gbase = sbase + grp * GO_BYTES;   // this group's shared memory
+    auto gsm = [&](int off) { return reinterpret_cast<float*>(smem + grp * GO_BYTES + off); };
+    // the adjoint tiles handed between the groups: [buffer][cell of the lane][thread of the group] (conflict-free)
+    auto g_put = [&](int b, const float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) stsf(sbase + GS_GBUF + 4 * ((b * 4 * G_NB + 4 * n + e) * G_GT + gt), v[n][e]);
+    };
+    auto g_get = [&](int b, float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) v[n][e] = ldsf(sbase + GS_GBUF + 4 * ((b * 4 * G_NB + 4 * n + e) * G_GT + gt));
+    };
+    auto gld = [&](int off) { return ldsf(gbase + off); };           // a float of this group's small arrays
+    const float* ub = reinterpret_cast<const float*>(smem + GS_U);
+    auto gb = [&](int i) { return bar(grp * GB_PER_GROUP + i); };      // this group's barriers
 
     if (tid == 0) {
-        for (int i = 0; i < BB_COUNT; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < GB_GREADY; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(GB_GREADY), G_GT);
+        mbar_init(bar(GB_GREADY + 1), G_GT);
         sts32(abort_flag, 0u);
         sts32(abort_flag + 4, p.wait_limit_us ? p.wait_limit_us : WAIT_LIMIT_US);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (tid < 64) fsm(BO_DU_FB)[tid] = 0.f;
-    if (warp == 1) tmem_alloc(sbase + BO_TMEM, BT_COLS);
+    if (tid < 64) reinterpret_cast<float*>(smem + GS_U)[tid] = C2 ? 0.f : p.u[col0 + tid];
+    if (gt < 64) gsm(GO_DUFB)[gt] = 0.f;
+    if (warp == 1) tmem_alloc(sbase + GS_TMEM, GT_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = lds32(sbase + BO_TMEM);
-    const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 16 * cq;      // this warp's block of an accumulator
+    const uint32_t tmem = lds32(sbase + GS_TMEM) + 256 * grp;                 // this group's columns
+    const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 8 * G_NB * cx;      // this warp's block of an accumulator
 
-    // Chunks are numbered by iteration: iteration `it` handles chunk nchunks - 1 - it; its input stage and the
-    // double-buffered operand tiles are those of parity it & 1.
     auto chunk_of = [&](int it) { return nchunks - 1 - it; };
-
-    // ---- issuing: the products, the TMA stores of a chunk's gradient tiles and the input copies.  With B_ISSUER a
-    // warp of its own does it: one lane takes commands from the compute warps (a ring of four slots, one mbarrier each:
-    // at most three are ever outstanding), so that no compute warp waits for an instruction to be issued, only for
-    // its completion.  Without it thread 0 issues in place.
-    int last_load[2] = {-1, -1};                     // (issuing thread) per stage: the last iteration whose copies were issued
-    auto issue_loads = [&](int it) {
-        const int stage = it & 1;
-        const uint32_t dst = sbase + BO_IN + stage * B_STAGE;
+    const uint32_t tin = gbase + GO_IN;
+    const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
+    const uint32_t t_rh = gbase + GO_RH, t_kh = gbase + GO_KH;
+    const uint32_t t_sb = gbase + GO_T4, t_gb = t_sb + TILE, t_pp = t_sb + 2 * TILE, t_dpp = t_sb + 3 * TILE;
+    // staging tiles of the four gradients, each over an operand tile that is dead when it is written: dr over S_0 and
+    // dk over dP' (free once dR^ and dK^ are complete), dv over P' and dx over G^ (free once dV is complete)
+    const uint32_t o_dr = t_sb, o_dk = t_dpp, o_dv = t_pp, o_dx = t_gb;
+    // The input copies of a chunk come in two parts, each issued as soon as its tiles are free: x, v, dy once the
+    // chunk before (of this group) has finished its products, r, k once its epilogue has read them.
+    int last_a = -1, last_b = -1;                    // (thread 0 of the group) the last iterations whose copies were issued
+    auto issue_loads_a = [&](int it) {               // thread 0 of the group
         const int row = (int)(row0 + (long long)chunk_of(it) * L);
-        mbar_expect_tx(bar(BB_IN + stage), B_STAGE);
-        tma_load_2d(dst, &tm_x, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + TILE, &tm_r, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 2 * TILE, &tm_k, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 3 * TILE, &tm_v, col0, row, bar(BB_IN + stage));
-        tma_load_2d(dst + 4 * TILE, &tm_dy, col0, row, bar(BB_IN + stage));
-        last_load[stage] = it;
+        mbar_expect_tx(gb(GB_INA), 3 * TILE);
+        tma_load_2d(tx, &tm_x, col0, row, gb(GB_INA));
+        tma_load_2d(tv, &tm_v, col0, row, gb(GB_INA));
+        tma_load_2d(tdy, &tm_dy, col0, row, gb(GB_INA));
+        last_a = it;
     };
-    auto execute = [&](uint32_t cmd, uint32_t arg) {
-        if (cmd == CMD_MMA1 || cmd == CMD_MMA2) {
-            const int pb = (int)arg;
-            const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
-            const uint64_t dR = smem_desc(sbase + BO_RH + pb * TILE), dK = smem_desc(sbase + BO_KH + pb * TILE);
-            const uint64_t dV = smem_desc(tin + 3 * TILE), dY = smem_desc(tin + 4 * TILE);
-            tc_fence_after();
-            if (cmd == CMD_MMA1) {
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
-                    tc_mma(tmem + BT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
-                    tc_mma(tmem + BT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
-                    tc_mma(tmem + BT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
-                }
-                tc_commit(bar(BB_MMA1));
-            } else {
-                const uint64_t dS = smem_desc(sbase + BO_SB + pb * TILE), dG = smem_desc(sbase + BO_GB + pb * TILE);
-                const uint64_t dP = smem_desc(sbase + BO_PP), dD = smem_desc(sbase + BO_DPP);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;
-                    tc_mma(tmem + BT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
-                    tc_mma(tmem + BT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
-                    tc_mma(tmem + BT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
-                }
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ks = 2 * kk, ms = 128 * kk;
-                    tc_mma(tmem + BT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
-                    tc_mma(tmem + BT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
-                    tc_mma(tmem + BT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
-                }
-                tc_commit(bar(BB_MMA2));
-            }
-        } else {                             // CMD_STORE: arg = iteration, bit 31: whole chunk (TMA stores)
-            const int it = (int)(arg & 0x7fffffffu);
-            const bool whole = (arg >> 31) != 0;
-            if (whole) {
-                const int row = (int)(row0 + (long long)chunk_of(it) * L);
-                tma_store_2d(&tm_dr, col0, row, sbase + BO_OUT);
-                tma_store_2d(&tm_dk, col0, row, sbase + BO_OUT + TILE);
-                tma_store_2d(&tm_dv, col0, row, sbase + BO_OUT + 2 * TILE);
-                tma_store_2d(&tm_dx, col0, row, sbase + BO_OUT + 3 * TILE);
-                bulk_commit();
-            }
-            if (it + 2 < nchunks) issue_loads(it + 2);
-            if (B_ISSUER) {
-                if (whole) bulk_wait_read<0>();      // the staging tiles may be rewritten
-                mbar_arrive(bar(BB_STAGING));
-            }
-        }
+    auto issue_loads_b = [&](int it) {
+        const int row = (int)(row0 + (long long)chunk_of(it) * L);
+        mbar_expect_tx(gb(GB_INB), 2 * TILE);
+        tma_load_2d(tr, &tm_r, col0, row, gb(GB_INB));
+        tma_load_2d(tk, &tm_k, col0, row, gb(GB_INB));
+        last_b = it;
     };
-    auto issuer_done = [&]() {
-        bulk_wait<0>();                              // the gradient tiles have reached memory
-        for (int s2 = 0; s2 < 2; ++s2)               // no copy into this CTA's shared memory may stay in flight
-            if (last_load[s2] >= 0) mbar_wait(bar(BB_IN + s2), (last_load[s2] >> 1) & 1, abort_flag, false);
-    };
-    if (B_ISSUER ? (warp == B_CTHREADS / 32 && lane == 0) : tid == 0) {
-        if (nchunks > 0) issue_loads(0);
-        if (nchunks > 1) issue_loads(1);
-    }
-
-    if (B_ISSUER && warp == B_CTHREADS / 32) {
-        // ============================== issuing warp ==============================
-        if (lane == 0) {
-            for (int kc = 0;; ++kc) {
-                if (!mbar_wait(bar(BB_CMD + (kc & 3)), (kc >> 2) & 1, abort_flag)) break;
-                const uint32_t cmd = lds32(sbase + BO_CMD + 8 * (kc & 3)), arg = lds32(sbase + BO_CMD + 8 * (kc & 3) + 4);
-                if (cmd == CMD_QUIT) break;
-                execute(cmd, arg);
-            }
-            issuer_done();
-        }
-    } else {
-    // ============================== compute warps ==============================
-    // Every thread waits for itself on an mbarrier; the outcomes are made uniform at the next barrier of the compute
-    // warps (cbar_and), so that after a wait that ran out all of them leave together.
-    int n_cmd = 0;                                   // (thread 0) commands posted so far
-    auto post = [&](uint32_t cmd, uint32_t arg) {    // thread 0, after a barrier that follows the operands' writes
-        if (!B_ISSUER) {
-            if (cmd != CMD_QUIT) execute(cmd, arg); else issuer_done();
-            return;
-        }
-        const uint32_t slot = sbase + BO_CMD + 8 * (n_cmd & 3);
-        sts32(slot, cmd);
-        sts32(slot + 4, arg);
-        mbar_arrive(bar(BB_CMD + (n_cmd & 3)));
-        ++n_cmd;
-    };
-    int n_store = 0;                                 // store commands posted so far (every thread counts)
-    auto load_f32_block = [&](const float* src, float (&v)[2][4]) {      // [64][64] fp32 block, accumulator layout
+    auto load_f32_block = [&](const float* src, float (&v)[G_NB][4]) {      // [64][64] fp32 block, the lane's cells
 #pragma unroll
-        for (int n = 0; n < 2; ++n) {
+        for (int n = 0; n < G_NB; ++n) {
             const float2 lo = *reinterpret_cast<const float2*>(src + (size_t)R0 * 64 + cb + 8 * n);
             const float2 hi = *reinterpret_cast<const float2*>(src + (size_t)R1 * 64 + cb + 8 * n);
             v[n][0] = lo.x; v[n][1] = lo.y; v[n][2] = hi.x; v[n][3] = hi.y;
         }
     };
+    auto store_f32_block = [&](float* dst, const float (&v)[G_NB][4]) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) {
+            *reinterpret_cast<float2*>(dst + (size_t)R0 * 64 + cb + 8 * n) = make_float2(v[n][0], v[n][1]);
+            *reinterpret_cast<float2*>(dst + (size_t)R1 * 64 + cb + 8 * n) = make_float2(v[n][2], v[n][3]);
+        }
+    };
 
-    float uu[2][2];                                  // bonus of this lane's columns (as channels)
-#pragma unroll
-    for (int n = 0; n < 2; ++n) { uu[n][0] = C2 ? 0.f : p.u[col0 + cb + 8 * n]; uu[n][1] = C2 ? 0.f : p.u[col0 + cb + 8 * n + 1]; }
-    float G[2][4], SL[2][4], du_acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
     const float* ck_unit = p.ckpt + (size_t)unit * (nchunks + 1) * 4096;
-    if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
-    else {
+    float du_acc[G_NB][2];
 #pragma unroll
-        for (int n = 0; n < 2; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
-    }
-    load_f32_block(ck_unit + (size_t)nchunks * 4096, SL);
-    int mph1 = 0, mph2 = 0;                          // phase bits of the two product barriers
+    for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
+    if (gt == 0 && grp < nchunks) { issue_loads_a(grp); issue_loads_b(grp); }
+    int mph = 0;                                     // phase bit of this group's two product barriers
     bool alive = true;
 
-    // ---- operands of a chunk from its inputs and from the adjoint G = G_L at its end; first group of products.
-    // Returns 0 (products issued), 1 (the chunk decays too fast for this form: nothing issued) or -1 (a wait ran out).
-    // On return SL holds the chunk's start state; a, lw2 its cumulative and per-token log2 decays in this lane's cells.
-    auto prepare = [&](int it, float (&a)[2][4], float (&lw2)[2][4], float (&dch)[2]) -> int {
-        const int c = chunk_of(it), pb = it & 1;
-        const int valid = min(L, T - c * L);
-        const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
-        const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
-        const uint32_t t_rh = sbase + BO_RH + pb * TILE, t_kh = sbase + BO_KH + pb * TILE;
-        const uint32_t t_sb = sbase + BO_SB + pb * TILE, t_gb = sbase + BO_GB + pb * TILE;
-        float S0[2][4];
+    for (int it = grp; it < nchunks; it += 2) {
+        const int c = chunk_of(it), valid = min(L, T - c * L);
+        const int use = it >> 1;                     // how often this group's input stage has been filled before
+        float S0[G_NB][4];                              // the chunk-start state (requested early: it is used after the scan)
         load_f32_block(ck_unit + (size_t)c * 4096, S0);
-        if (c > 0 && tid < 128)                      // the next chunk's start state: in L2 by the time it is loaded
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 1) * 4096 + 32 * tid));
-        // E = rowsum(G_L * S_L): partial over this lane's columns, then over the four lanes of a row
-        {
-            float e0 = 0.f, e1 = 0.f;
-#pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                e0 = fmaf(G[n][0], SL[n][0], fmaf(G[n][1], SL[n][1], e0));
-                e1 = fmaf(G[n][2], SL[n][2], fmaf(G[n][3], SL[n][3], e1));
-            }
-            e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
-            e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
-            if (q == 0) { fsm(BO_EP)[(pb * 4 + cq) * 64 + R0] = e0; fsm(BO_EP)[(pb * 4 + cq) * 64 + R1] = e1; }
-        }
-        bool ok = mbar_wait(bar(BB_IN + pb), (it >> 1) & 1, abort_flag);
-        if (valid < L) {
-            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
-            for (int i = tid; i < (L - valid) * 8; i += B_CTHREADS) {
-                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
-                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
+        if (it + 2 < nchunks) {
+            // this group's next chunk: its start state and its input tiles into L2 now, so that the copies issued at
+            // the end of this iteration and the load above find them there
+            if (gt < 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 2) * 4096 + 32 * gt));
+            if (gt == 128) {
+                const int row = (int)(row0 + (long long)(c - 2) * L);
+                tma_prefetch_2d(&tm_x, col0, row); tma_prefetch_2d(&tm_r, col0, row); tma_prefetch_2d(&tm_k, col0, row);
+                tma_prefetch_2d(&tm_v, col0, row); tma_prefetch_2d(&tm_dy, col0, row);
             }
         }
-        // decay: log2-domain magnitudes, cumulative sums over the tokens
+        // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
+        bool ok = mbar_wait(gb(GB_INA), use & 1, abort_flag);
+        if (gt == 0 && it > 1) bulk_wait_read<0>();  // the previous chunk's staging tiles have been read by the TMA unit
+        float a[G_NB][4], lw2[G_NB][4];
         {
-            float xv[2][4];
-            load_block_bf16(tx + moff, xv);
+            float xv[G_NB][4];
+            ld_tile(tx, moff, xv);
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
+            for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const bool live = (e < 2 ? R0 : R1) < valid;
@@ -421,123 +376,124 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     a[n][e] = lw2[n][e];
                 }
         }
-        ok = scan_rows<false>(a, sbase + BO_TOT, sp, cq, lane, ok);      // (barrier: the zeroed rows are visible after it)
-        if (!ok) return -1;
-        // a_L = the sum of the four row-group totals; this lane needs it for the channels that are its rows of G
+        ok = scan_rows<false>(a, gbase + GO_TOT, grp, sp, cb, lane, ok);      // (barrier: the zeroed rows are visible after it)
+        if (!ok) { alive = false; break; }
+        float d_lo, d_hi;                            // the chunk's decay for the channels that are this lane's rows of G
         bool safe;
         {
             float al0 = 0.f, al1 = 0.f;
 #pragma unroll
-            for (int o = 0; o < 4; ++o) { al0 += fsm(BO_TOT)[o * 64 + R0]; al1 += fsm(BO_TOT)[o * 64 + R1]; }
-            dch[0] = ex2(al0); dch[1] = ex2(al1);
+            for (int o = 0; o < 4; ++o) { al0 += gld(GO_TOT + 4 * (o * 64 + R0)); al1 += gld(GO_TOT + 4 * (o * 64 + R1)); }
+            d_lo = ex2(al0); d_hi = ex2(al1);
             safe = (al0 >= -A2_MAX) && (al1 >= -A2_MAX);                   // false for NaN as well
         }
+        // ---- operands from the inputs: R^, K^ (and the bonus), the chunk-start state
+        if (!mbar_wait(gb(GB_INB), use & 1, abort_flag)) ok = false;        // (made uniform at a later barrier)
+        if (valid < L) {
+            // ragged last chunk: the rows past the sequence's end hold other tokens (or the out-of-range fill)
+            for (int i = gt; i < (L - valid) * 8; i += G_GT) {
+                const uint32_t o = (valid + (i >> 3)) * 128 + ((i & 7) << 4);
+                sts128z(tr + o); sts128z(tk + o); sts128z(tv + o); sts128z(tdy + o);
+            }
+            gbar(grp);
+        }
         {
-            float rv[2][4], kv[2][4];
-            load_block_bf16(tr + moff, rv);
-            load_block_bf16(tk + moff, kv);
+            float rv[G_NB][4], kv[G_NB][4];
+            ld_tile(tr, moff, rv);
+            ld_tile(tk, moff, kv);
             float b0 = 0.f, b1 = 0.f;
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
+            for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if (C2) kv[n][e] *= one_minus_ex2(lw2[n][e]);      // the key that enters the state
-                    const float t = rv[n][e] * kv[n][e] * uu[n][e & 1];
-                    if (e < 2) b0 += t; else b1 += t;
+                    if (!C2) {
+                        const float t = rv[n][e] * kv[n][e] * ldsf(sbase + GS_U + 4 * (cb + 8 * n + (e & 1)));
+                        if (e < 2) b0 += t; else b1 += t;
+                    }
                     rv[n][e] *= ex2(a[n][e] - lw2[n][e]);
                     kv[n][e] *= ex2(-a[n][e]);
                 }
-            store_block_bf16(t_rh + moff, rv);
-            store_block_bf16(t_kh + moff, kv);
-            b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
-            b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
-            if (q == 0) { fsm(BO_BP)[cq * 64 + R0] = b0; fsm(BO_BP)[cq * 64 + R1] = b1; }
-        }
-        store_block_bf16(t_sb + moff, S0);
-#pragma unroll
-        for (int n = 0; n < 2; ++n)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) SL[n][e] = S0[n][e];
-        {
-            float gh[2][4];
-#pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                gh[n][0] = dch[0] * G[n][0]; gh[n][1] = dch[0] * G[n][1];
-                gh[n][2] = dch[1] * G[n][2]; gh[n][3] = dch[1] * G[n][3];
+            st_tile(t_rh, moff, rv);
+            st_tile(t_kh, moff, kv);
+            if (!C2) {
+                b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
+                b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
+                if (q == 0) { stsf(gbase + GO_BP + 4 * (cx * 64 + R0), b0); stsf(gbase + GO_BP + 4 * (cx * 64 + R1), b1); }
             }
-            store_block_bf16(t_gb + moff, gh);
         }
+        st_tile(t_sb, moff, S0);
         fence_proxy_async();
         tc_fence_before();
-        const bool unsafe = !cbar_and(safe);         // (every channel is some lane's row)
-        if (tid == 0 && !unsafe) post(CMD_MMA1, (uint32_t)pb);
-        return unsafe ? 1 : 0;
-    };
-
-    // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one; then the
-    // input stage of this iteration is free for the chunk two iterations on.
-    auto store_and_refill = [&](int it) {
-        const int c = chunk_of(it), valid = min(L, T - c * L);
-        fence_proxy_async();
-        cbar();
-        if (valid < L) {
-            __nv_bfloat16* outs[4] = {p.dr, p.dk, p.dv, p.dx};
-            for (int i = tid; i < 4 * valid * 8; i += B_CTHREADS) {
-                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
-                uint32_t w[4];
-                lds_v4(sbase + BO_OUT + tile * TILE + swz(t, blk << 4), w);
-                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
+        const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
+        if (!unsafe && gt == 0) {
+            // the products that need nothing but the inputs; the adjoint is not needed for R^^T dY either
+            tc_fence_after();
+            const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
+                tc_mma(tmem + GT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                tc_mma(tmem + GT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
+                tc_mma(tmem + GT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
             }
+            tc_commit(gb(GB_MA));
         }
-        if (tid == 0) post(CMD_STORE, (uint32_t)it | (valid == L ? 0x80000000u : 0u));
-        ++n_store;
-    };
-    // The staging tiles may be rewritten once the TMA unit has read the previous chunk's (a barrier of the compute
-    // warps follows in every caller, which also orders a ragged chunk's plain reads before the rewrite).
-    auto staging_free = [&]() -> bool {
-        if (!B_ISSUER) {                             // thread 0 issued the stores itself: it waits for their reads
-            if (tid == 0) bulk_wait_read<0>();
-            return true;
+        // ---- the adjoint at the chunk's end, from the other group (the call's dstate_out for the last chunk)
+        float G[G_NB][4];
+        if (it == 0) {
+            if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
+            else {
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
+            }
+        } else {
+            if (!mbar_wait(bar(GB_GREADY + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag)) ok = false;
+            g_get((it - 1) & 1, G);
         }
-        return n_store == 0 || mbar_wait(bar(BB_STAGING), (n_store - 1) & 1, abort_flag);
-    };
+        // E = rowsum(G_L * S_L), S_L the state at the chunk's end, as partial sums per column slab: for the call's last
+        // chunk from the final state; else the group that made G_L formed them from its chunk-start state (e_put below)
+        auto e_put = [&](uint32_t dst, const float (&Gm)[G_NB][4], const float (&Sm)[G_NB][4]) {
+            float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n) {
+                e0 = fmaf(Gm[n][0], Sm[n][0], fmaf(Gm[n][1], Sm[n][1], e0));
+                e1 = fmaf(Gm[n][2], Sm[n][2], fmaf(Gm[n][3], Sm[n][3], e1));
+            }
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 1); e1 += __shfl_xor_sync(0xffffffffu, e1, 1);
+            e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
+            if (q == 0) { stsf(dst + 4 * (cx * 64 + R0), e0); stsf(dst + 4 * (cx * 64 + R1), e1); }
+        };
+        if (it == 0) {
+            float SL[G_NB][4];
+            load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
+            e_put(gbase + GO_EP, G, SL);
+        } else if (gt < G_NSLAB * 64) {
+            stsf(gbase + GO_EP + 4 * gt, ldsf(sbase + GS_EH + 4 * (((it - 1) & 1) * G_NSLAB * 64 + gt)));      // (a private copy: the slot is rewritten two chunks on)
+        }
 
-    float a_cur[2][4], lw_cur[2][4], d_cur[2];       // of the chunk in flight: cumulative / per-token log2 decays, chunk decay
-    int st = nchunks > 0 ? prepare(0, a_cur, lw_cur, d_cur) : 0;
-    if (st < 0) alive = false;
-
-    for (int it = 0; alive && it < nchunks; ++it) {
-        const int c = chunk_of(it), pb = it & 1;
-        const int valid = min(L, T - c * L);
-        const uint32_t tin = sbase + BO_IN + pb * B_STAGE;
-        const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
-        const uint32_t t_rh = sbase + BO_RH + pb * TILE, t_kh = sbase + BO_KH + pb * TILE;
-
-        if (st == 1) {
-            // ---- token by token: the chunk's states recomputed into this SM's scratch, then the reverse recurrence
-            const unsigned slot = smid();
+        if (unsafe) {
+            // ---- token by token: the chunk's states recomputed into this group's scratch, then the reverse recurrence
+            const unsigned slot = 2 * smid() + grp;
             if (slot >= (unsigned)p.n_slots) {       // (no scratch for this SM: report it and leave)
-                if (tid == 0) { sts32(abort_flag, 1u); atomicExch(&g_dev_status, 1); }
+                if (gt == 0) { sts32(abort_flag, 1u); atomicExch(&g_dev_status, 1); }
                 alive = false;
                 break;
             }
-            if (!cbar_and(staging_free())) { alive = false; break; }
-            float* scr = p.fb_scratch + (size_t)slot * FB_SLOT_FLOATS + (size_t)tid * 8;
-            // rows are key channels here: this lane's channels R0, R1 of S and G; its columns are value channels
-            float S[2][4];
-#pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) S[n][e] = SL[n][e];
+            if (!gbar_and(grp, ok)) { alive = false; break; }
+            float* scr = p.fb_scratch + (size_t)slot * FB_SLOT_FLOATS + (size_t)gt * (4 * G_NB);
+            float S[G_NB][4];
+            load_f32_block(ck_unit + (size_t)c * 4096, S);
             for (int t = 0; t < valid; ++t) {
-                *reinterpret_cast<float4*>(scr + (size_t)t * 4096) = make_float4(S[0][0], S[0][1], S[0][2], S[0][3]);
-                *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4) = make_float4(S[1][0], S[1][1], S[1][2], S[1][3]);
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n)
+                    *reinterpret_cast<float4*>(scr + (size_t)t * 4096 + 4 * n) = make_float4(S[n][0], S[n][1], S[n][2], S[n][3]);
                 const float e0 = expf(lds_bf16(tx + swz(t, 2 * R0))), e1 = expf(lds_bf16(tx + swz(t, 2 * R1)));
                 const float w0 = expf(-e0), w1 = expf(-e1);
                 float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
                 if (C2) { k0 *= -expm1f(-e0); k1 *= -expm1f(-e1); }
 #pragma unroll
-                for (int n = 0; n < 2; ++n)
+                for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const float vj = lds_bf16(tv + swz(t, 2 * (cb + 8 * n + e)));
@@ -545,21 +501,24 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                         S[n][2 + e] = fmaf(w1, S[n][2 + e], k1 * vj);
                     }
             }
-            float* red = fsm(BO_RED);                // [cq][3][64]
-            float* redv = fsm(BO_RED_V);             // [sp][64]
-            float* scal = fsm(BO_SCAL);              // v . dy, sum r u k
+            float* red = gsm(GO_RED);                // [slab][3][64]
+            float* redv = gsm(GO_REDV);              // [sp][64]
+            float* scal = gsm(GO_SCAL);              // v . dy, sum r u k
             for (int t = valid - 1; t >= 0; --t) {
-                const float4 sa = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096);
-                const float4 sb4 = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096 + 4);
-                const float Sp[2][4] = {{sa.x, sa.y, sa.z, sa.w}, {sb4.x, sb4.y, sb4.z, sb4.w}};
+                float Sp[G_NB][4];
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    const float4 s4 = *reinterpret_cast<const float4*>(scr + (size_t)t * 4096 + 4 * n);
+                    Sp[n][0] = s4.x; Sp[n][1] = s4.y; Sp[n][2] = s4.z; Sp[n][3] = s4.w;
+                }
                 const float x0 = lds_bf16(tx + swz(t, 2 * R0)), x1 = lds_bf16(tx + swz(t, 2 * R1));
                 const float w0 = expf(-expf(x0)), w1 = expf(-expf(x1));
                 float k0 = lds_bf16(tk + swz(t, 2 * R0)), k1 = lds_bf16(tk + swz(t, 2 * R1));
                 if (C2) { k0 *= -expm1f(-expf(x0)); k1 *= -expm1f(-expf(x1)); }
                 const float r0 = lds_bf16(tr + swz(t, 2 * R0)), r1 = lds_bf16(tr + swz(t, 2 * R1));
-                float pr0 = 0.f, pr1 = 0.f, pk0 = 0.f, pk1 = 0.f, pg0 = 0.f, pg1 = 0.f, pv[2][2];
+                float pr0 = 0.f, pr1 = 0.f, pk0 = 0.f, pk1 = 0.f, pg0 = 0.f, pg1 = 0.f, pv[G_NB][2];
 #pragma unroll
-                for (int n = 0; n < 2; ++n)
+                for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const int j = cb + 8 * n + e;
@@ -580,27 +539,27 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
                 for (int d = 4; d < 32; d <<= 1)
 #pragma unroll
-                    for (int n = 0; n < 2; ++n)
+                    for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) pv[n][e] += __shfl_xor_sync(0xffffffffu, pv[n][e], d);
                 if (q == 0) {
-                    red[(cq * 3 + 0) * 64 + R0] = pr0; red[(cq * 3 + 0) * 64 + R1] = pr1;
-                    red[(cq * 3 + 1) * 64 + R0] = pk0; red[(cq * 3 + 1) * 64 + R1] = pk1;
-                    red[(cq * 3 + 2) * 64 + R0] = pg0; red[(cq * 3 + 2) * 64 + R1] = pg1;
+                    red[(cx * 3 + 0) * 64 + R0] = pr0; red[(cx * 3 + 0) * 64 + R1] = pr1;
+                    red[(cx * 3 + 1) * 64 + R0] = pk0; red[(cx * 3 + 1) * 64 + R1] = pk1;
+                    red[(cx * 3 + 2) * 64 + R0] = pg0; red[(cx * 3 + 2) * 64 + R1] = pg1;
                 }
                 if (g == 0) {
 #pragma unroll
-                    for (int n = 0; n < 2; ++n)
+                    for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) redv[sp * 64 + cb + 8 * n + e] = pv[n][e];
                 }
-                if (warp == 0) {
+                if (gt < 32) {
                     float vd = 0.f, ruk = 0.f;
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const int cc = 2 * lane + e;
                         vd = fmaf(lds_bf16(tv + swz(t, 2 * cc)), lds_bf16(tdy + swz(t, 2 * cc)), vd);
-                        if (!C2) ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * p.u[col0 + cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
+                        if (!C2) ruk = fmaf(lds_bf16(tr + swz(t, 2 * cc)) * ub[cc], lds_bf16(tk + swz(t, 2 * cc)), ruk);
                     }
 #pragma unroll
                     for (int d = 1; d < 32; d <<= 1) {
@@ -609,210 +568,283 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     }
                     if (lane == 0) { scal[0] = vd; scal[1] = ruk; }
                 }
-                cbar();
-                if (tid < 64) {
-                    const int cc = tid;
+                gbar(grp);
+                if (gt < 64) {
+                    const int cc = gt;
                     float s_r = 0.f, s_k = 0.f, s_g = 0.f;
 #pragma unroll
-                    for (int o = 0; o < 4; ++o) { s_r += red[(o * 3 + 0) * 64 + cc]; s_k += red[(o * 3 + 1) * 64 + cc]; s_g += red[(o * 3 + 2) * 64 + cc]; }
+                    for (int o = 0; o < G_NSLAB; ++o) { s_r += red[(o * 3 + 0) * 64 + cc]; s_k += red[(o * 3 + 1) * 64 + cc]; s_g += red[(o * 3 + 2) * 64 + cc]; }
                     const float xc = lds_bf16(tx + swz(t, 2 * cc)), kc = lds_bf16(tk + swz(t, 2 * cc)), rc = lds_bf16(tr + swz(t, 2 * cc));
                     const float ec = expf(xc), wc = expf(-ec);
                     if (C2) {
-                        sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), s_r);
-                        sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), s_k * -expm1f(-ec));
-                        sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
+                        sts_bf16(o_dr + swz(t, 2 * cc), s_r);
+                        sts_bf16(o_dk + swz(t, 2 * cc), s_k * -expm1f(-ec));
+                        sts_bf16(o_dx + swz(t, 2 * cc), (s_g - s_k * kc) * (-wc * ec));
                     } else {
-                        const float uc = p.u[col0 + cc], vd = scal[0];
-                        sts_bf16(sbase + BO_OUT + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
-                        sts_bf16(sbase + BO_OUT + TILE + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
-                        sts_bf16(sbase + BO_OUT + 3 * TILE + swz(t, 2 * cc), s_g * (-wc * ec));
-                        fsm(BO_DU_FB)[cc] = fmaf(rc * kc, vd, fsm(BO_DU_FB)[cc]);
+                        const float uc = ub[cc], vd = scal[0];
+                        sts_bf16(o_dr + swz(t, 2 * cc), fmaf(uc * kc, vd, s_r));
+                        sts_bf16(o_dk + swz(t, 2 * cc), fmaf(rc * uc, vd, s_k));
+                        sts_bf16(o_dx + swz(t, 2 * cc), s_g * (-wc * ec));
+                        gsm(GO_DUFB)[cc] = fmaf(rc * kc, vd, gsm(GO_DUFB)[cc]);
                     }
-                } else if (tid < 128) {
-                    const int j = tid - 64;
+                } else if (gt < 128) {
+                    const int j = gt - 64;
                     const float s_v = redv[j] + redv[64 + j] + redv[128 + j] + redv[192 + j];
-                    sts_bf16(sbase + BO_OUT + 2 * TILE + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
+                    sts_bf16(o_dv + swz(t, 2 * j), fmaf(scal[1], lds_bf16(tdy + swz(t, 2 * j)), s_v));
                 }
-                cbar();
+                gbar(grp);
             }
-            store_and_refill(it);
+            // hand the adjoint on (and the row sums the next chunk needs, from the fp32 state: the operand tile is gone)
             if (it + 1 < nchunks) {
-                st = prepare(it + 1, a_cur, lw_cur, d_cur);
-                if (st < 0) alive = false;
+                g_put(it & 1, G);
+                load_f32_block(ck_unit + (size_t)c * 4096, S);
+                e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, S);
+                mbar_arrive(bar(GB_GREADY + (it & 1)));
+            } else if (p.dstate_in) {
+                store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
             }
-            continue;
-        }
-
-        // ---- masked scores and their adjoint as operands
-        bool ok = mbar_wait(bar(BB_MMA1), mph1, abort_flag);
-        mph1 ^= 1;
-        tc_fence_after();
-        if (cq < sp) {
-            // a block below the diagonal: every score and every adjoint entry is kept
-            float pp[2][4], dp[2][4];
-            tmem_ld_16x16_async(tacc + BT_P, pp);
-            tmem_ld_16x16_async(tacc + BT_DP, dp);
-            tmem_ld_done();
-            store_block_bf16(sbase + BO_PP + moff, pp);
-            store_block_bf16(sbase + BO_DPP + moff, dp);
-        } else if (cq > sp) {
-            // above the diagonal: masked out
-            stsm_x4(sbase + BO_PP + moff, 0u, 0u, 0u, 0u);
-            stsm_x4(sbase + BO_DPP + moff, 0u, 0u, 0u, 0u);
         } else {
-            float pp[2][4], dp[2][4];
-            tmem_ld_16x16_async(tacc + BT_P, pp);
-            tmem_ld_16x16_async(tacc + BT_DP, dp);
-            float bon0 = 0.f, bon1 = 0.f;
-#pragma unroll
-            for (int o = 0; o < 4; ++o) { bon0 += fsm(BO_BP)[o * 64 + R0]; bon1 += fsm(BO_BP)[o * 64 + R1]; }
-            tmem_ld_done();
-#pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int row = e < 2 ? g : g + 8, col = 2 * q + 8 * n + (e & 1);       // inside the 16 x 16 block
-                    if (col == row) fsm(BO_DPD)[16 * sp + row] = dp[n][e];
-                    pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
-                    dp[n][e] = col < row ? dp[n][e] : 0.f;
-                }
-            store_block_bf16(sbase + BO_PP + moff, pp);
-            store_block_bf16(sbase + BO_DPP + moff, dp);
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        if (!cbar_and(ok)) { alive = false; break; }
-        if (tid == 0) post(CMD_MMA2, (uint32_t)pb);
-        // ---- G_0 = diag(D) G_L + R^^T dY
-        {
-            const float d_lo = d_cur[0], d_hi = d_cur[1];
-            float dg[2][4];
-            tmem_ld_16x16(tacc + BT_DG, dg);
-#pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
-                G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
-            }
-            tc_fence_before();
-        }
-        // ---- while the second group of products runs: the next chunk's operands and its first group of products
-        float a_nxt[2][4], lw_nxt[2][4], d_nxt[2] = {0.f, 0.f};
-        int st_nxt = 0;
-        if (it + 1 < nchunks) {
-            st_nxt = prepare(it + 1, a_nxt, lw_nxt, d_nxt);
-            if (st_nxt < 0) { alive = false; break; }
-        }
-        ok = staging_free() & mbar_wait(bar(BB_MMA2), mph2, abort_flag);     // (made uniform at the barrier of the suffix sums)
-        mph2 ^= 1;
-        tc_fence_after();
-        // ---- epilogue
-        {
-            float z[2][4], qv[2][4];
+            // ---- G^ as an operand; G_0 = G^ + R^^T dY handed on
             {
+                float gh[G_NB][4];
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    gh[n][0] = d_lo * G[n][0]; gh[n][1] = d_lo * G[n][1];
+                    gh[n][2] = d_hi * G[n][2]; gh[n][3] = d_hi * G[n][3];
+                }
+                st_tile(t_gb, moff, gh);
+            }
+            if (!mbar_wait(gb(GB_MA), mph, abort_flag)) ok = false;
+            tc_fence_after();
+            {
+                float dg[G_NB][4];
+#pragma unroll
+                for (int h2 = 0; h2 < G_H2; ++h2) tmem_ld_16x16_async2(tacc + GT_DG + 16 * h2, reinterpret_cast<float (&)[2][4]>(dg[2 * h2]));
+                tmem_ld_done();
+#pragma unroll
+                for (int n = 0; n < G_NB; ++n) {
+                    G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
+                    G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
+                }
+            }
+            if (it + 1 < nchunks) {
+                g_put(it & 1, G);
+                {
+                    float sb[G_NB][4];               // this chunk's start state is the next chunk's end state (bf16 copy: the operand tile)
+                    ld_tile(t_sb, moff, sb);
+                    e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, sb);
+                }
+                mbar_arrive(bar(GB_GREADY + (it & 1)));
+            } else if (p.dstate_in) {
+                store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
+            }
+            // ---- masked scores and their adjoint as operands
+#pragma unroll
+            for (int h2 = 0; h2 < G_H2; ++h2) {
+                const int blk = G_H2 * cx + h2;          // 16-column block of the tile; the diagonal one is blk == sp
+                if (blk < sp) {
+                    float pp[2][4], dp[2][4];
+                    tmem_ld_16x16_async2(tacc + GT_P + 16 * h2, pp);
+                    tmem_ld_16x16_async2(tacc + GT_DP + 16 * h2, dp);
+                    tmem_ld_done();
+                    st_half(t_pp + moff[h2], pp);
+                    st_half(t_dpp + moff[h2], dp);
+                } else if (blk > sp) {
+                    stsm_x4(t_pp + moff[h2], 0u, 0u, 0u, 0u);
+                    stsm_x4(t_dpp + moff[h2], 0u, 0u, 0u, 0u);
+                } else {
+                    float pp[2][4], dp[2][4];
+                    tmem_ld_16x16_async2(tacc + GT_P + 16 * h2, pp);
+                    tmem_ld_16x16_async2(tacc + GT_DP + 16 * h2, dp);
+                    float bon0 = 0.f, bon1 = 0.f;
+                    if (!C2) {
+#pragma unroll
+                        for (int o = 0; o < G_NSLAB; ++o) { bon0 += gld(GO_BP + 4 * (o * 64 + R0)); bon1 += gld(GO_BP + 4 * (o * 64 + R1)); }
+                    }
+                    tmem_ld_done();
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int row = e < 2 ? g : g + 8, col = 2 * q + 8 * n + (e & 1);       // inside the 16 x 16 block
+                            if (col == row) stsf(gbase + GO_DPD + 4 * (16 * sp + row), dp[n][e]);
+                            pp[n][e] = col < row ? pp[n][e] : (col == row ? (e < 2 ? bon0 : bon1) : 0.f);
+                            dp[n][e] = col < row ? dp[n][e] : 0.f;
+                        }
+                    st_half(t_pp + moff[h2], pp);
+                    st_half(t_dpp + moff[h2], dp);
+                }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            if (!gbar_and(grp, ok)) { alive = false; break; }
+            if (gt == 0) {
+                tc_fence_after();
+                const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
+                const uint64_t dS = smem_desc(t_sb), dG = smem_desc(t_gb), dP = smem_desc(t_pp), dD = smem_desc(t_dpp);
+                // dR^ and dK^ first (interleaved: products on one accumulator wait for each other), with a commit of
+                // their own: the epilogue starts on them while dV is still being formed
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk;
+                    tc_mma(tmem + GT_DR, dY + ks, dS + ks, IDESC_K_K, kk > 0);         // dR[t][c] = dY S_0^T
+                    tc_mma(tmem + GT_DK, dV + ks, dG + ks, IDESC_K_K, kk > 0);         // dK[i][c] = V G^^T
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + GT_DR, dD + ks, dK + ms, IDESC_K_MN, 1);             // dR += dP' K^
+                    tc_mma(tmem + GT_DK, dD + ms, dR + ms, IDESC_MN_MN, 1);            // dK += dP'^T R^
+                }
+                tc_commit(gb(GB_MRK));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ks = 2 * kk, ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dK + ks, dG + ms, IDESC_K_MN, kk > 0);        // dV[i][j] = K^ G^
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ms = 128 * kk;
+                    tc_mma(tmem + GT_DV, dP + ms, dY + ms, IDESC_MN_MN, 1);            // dV += P'^T dY
+                }
+                tc_commit(gb(GB_MV));
+            }
+            ok = mbar_wait(gb(GB_MRK), mph, abort_flag);
+            tc_fence_after();
+            // ---- epilogue (the staging tiles take the place of the operand tiles S_0, G^, P', dP': all read by now)
+            float z[G_NB][4], qv[G_NB][4];
+#pragma unroll
+            for (int h2 = 0; h2 < G_H2; ++h2) {
                 // q and m take the operands as the tensor core saw them (rounded to bf16): the pair terms that q and
                 // m share, and that cancel in the suffix sums, are then the same products on both sides
                 float acc[2][4], o[2][4], hat[2][4], rv[2][4], kv[2][4];
-                const float pd0 = fsm(BO_DPD)[R0], pd1 = fsm(BO_DPD)[R1];
-                float acc2[2][4], acc3[2][4];
-                tmem_ld_16x16_async(tacc + BT_DR, acc);
-                tmem_ld_16x16_async(tacc + BT_DK, acc2);
-                tmem_ld_16x16_async(tacc + BT_DV, acc3);
-                load_block_bf16(tr + moff, rv);
-                load_block_bf16(tk + moff, kv);
-                load_block_bf16(t_rh + moff, hat);
+                const float pd0 = C2 ? 0.f : gld(GO_DPD + 4 * R0), pd1 = C2 ? 0.f : gld(GO_DPD + 4 * R1);
+                tmem_ld_16x16_async2(tacc + GT_DR + 16 * h2, acc);
+                ld_half(tr + moff[h2], rv);
+                ld_half(tk + moff[h2], kv);
+                ld_half(t_rh + moff[h2], hat);
                 tmem_ld_done();
 #pragma unroll
                 for (int n = 0; n < 2; ++n)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float pd = e < 2 ? pd0 : pd1;
-                        o[n][e] = fmaf(uu[n][e & 1] * kv[n][e], pd, acc[n][e] * ex2(a_cur[n][e] - lw_cur[n][e]));
-                        qv[n][e] = acc[n][e] * hat[n][e];
-                        if (!C2) du_acc[n][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[n][e & 1]);
+                        const int nn = 2 * h2 + n;
+                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
+                        o[n][e] = fmaf(uc * kv[n][e], pd, acc[n][e] * ex2(a[nn][e] - lw2[nn][e]));
+                        qv[nn][e] = acc[n][e] * hat[n][e];
+                        if (!C2) du_acc[nn][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[nn][e & 1]);
                     }
-                store_block_bf16(sbase + BO_OUT + moff, o);
-                load_block_bf16(t_kh + moff, hat);
+                tmem_ld_16x16_async2(tacc + GT_DK + 16 * h2, acc);
+                ld_half(t_kh + moff[h2], hat);
+                tmem_ld_done();
+                st_half(o_dr + moff[h2], o);
 #pragma unroll
                 for (int n = 0; n < 2; ++n)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float pd = e < 2 ? pd0 : pd1;
-                        o[n][e] = fmaf(uu[n][e & 1] * rv[n][e], pd, acc2[n][e] * ex2(-a_cur[n][e]));
-                        z[n][e] = qv[n][e] - acc2[n][e] * hat[n][e];
+                        const int nn = 2 * h2 + n;
+                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
+                        o[n][e] = fmaf(uc * rv[n][e], pd, acc[n][e] * ex2(-a[nn][e]));
+                        z[nn][e] = qv[nn][e] - acc[n][e] * hat[n][e];
                         if (C2) {
                             // o is the gradient of k (1 - w): the key gets (1 - w) of it, and the decay logit its
                             // share through the key factor, folded into the term that leaves the suffix sums
-                            const float omw = one_minus_ex2(lw_cur[n][e]);
-                            qv[n][e] = fmaf(o[n][e] * kv[n][e], 1.f - omw, qv[n][e]);
+                            const float omw = one_minus_ex2(lw2[nn][e]);
+                            qv[nn][e] = fmaf(o[n][e] * kv[n][e], 1.f - omw, qv[nn][e]);
                             o[n][e] *= omw;
                         }
                     }
-                store_block_bf16(sbase + BO_OUT + TILE + moff, o);
-                store_block_bf16(sbase + BO_OUT + 2 * TILE + moff, acc3);
+                st_half(o_dk + moff[h2], o);
+            }
+            // dV: every product of the chunk has completed, so x, v, dy can take the group's next chunk
+            if (!mbar_wait(gb(GB_MV), mph, abort_flag)) ok = false;
+            mph ^= 1;
+            tc_fence_after();
+            if (gt == 0 && it + 2 < nchunks) issue_loads_a(it + 2);
+            {
+                float acc[G_NB][4];
+#pragma unroll
+                for (int h2 = 0; h2 < G_H2; ++h2) tmem_ld_16x16_async2(tacc + GT_DV + 16 * h2, reinterpret_cast<float (&)[2][4]>(acc[2 * h2]));
+                tmem_ld_done();
+                st_tile(o_dv, moff, acc);
             }
             tc_fence_before();
-            ok = scan_rows<true>(z, sbase + BO_TOT, sp, cq, lane, ok);
+            ok = scan_rows<true>(z, gbase + GO_TOT, grp, sp, cb, lane, ok);
             if (!ok) { alive = false; break; }
-            float o[2][4];
+            if (gt == 0 && it + 2 < nchunks) issue_loads_b(it + 2);      // (r, k were last read before the barrier of the sums)
 #pragma unroll
-            for (int n = 0; n < 2; ++n) {
+            for (int n = 0; n < G_NB; ++n) {
                 float E0 = 0.f, E1 = 0.f;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    E0 += fsm(BO_EP)[(pb * 4 + w) * 64 + cb + 8 * n];
-                    E1 += fsm(BO_EP)[(pb * 4 + w) * 64 + cb + 8 * n + 1];
-                }
+                for (int o = 0; o < G_NSLAB; ++o) { const float2 ev = ldsf2(gbase + GO_EP + 4 * (o * 64 + cb + 8 * n)); E0 += ev.x; E1 += ev.y; }
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    o[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw_cur[n][e] * LN2);
+                    z[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
             }
-            store_block_bf16(sbase + BO_OUT + 3 * TILE + moff, o);
+            st_tile(o_dx, moff, z);
         }
-        store_and_refill(it);
-#pragma unroll
-        for (int n = 0; n < 2; ++n)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { a_cur[n][e] = a_nxt[n][e]; lw_cur[n][e] = lw_nxt[n][e]; }
-        d_cur[0] = d_nxt[0]; d_cur[1] = d_nxt[1];
-        st = st_nxt;
+        // ---- the chunk's four gradient tiles leave: TMA for a whole chunk, plain stores for a ragged one
+        fence_proxy_async();
+        gbar(grp);
+        if (valid < L) {
+            __nv_bfloat16* outs[4] = {p.dr, p.dx, p.dv, p.dk};       // in the order of the staging tiles in shared memory
+            for (int i = gt; i < 4 * valid * 8; i += G_GT) {
+                const int tile = i / (valid * 8), rem = i % (valid * 8), t = rem >> 3, blk = rem & 7;
+                uint32_t w[4];
+                lds_v4(t_sb + tile * TILE + swz(t, blk << 4), w);
+                *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        if (gt == 0) {
+            if (valid == L) {
+                const int row = (int)(row0 + (long long)c * L);
+                tma_store_2d(&tm_dr, col0, row, o_dr);
+                tma_store_2d(&tm_dk, col0, row, o_dk);
+                tma_store_2d(&tm_dv, col0, row, o_dv);
+                tma_store_2d(&tm_dx, col0, row, o_dx);
+                bulk_commit();
+            }
+            if (unsafe && it + 2 < nchunks) { issue_loads_a(it + 2); issue_loads_b(it + 2); }      // (the other path has issued them)
+        }
     }
 
-    cbar();
-    if (alive) {
-        if (p.dstate_in) {
-            float* dst = p.dstate_in + (size_t)unit * 4096;
-#pragma unroll
-            for (int n = 0; n < 2; ++n) {
-                *reinterpret_cast<float2*>(dst + (size_t)R0 * 64 + cb + 8 * n) = make_float2(G[n][0], G[n][1]);
-                *reinterpret_cast<float2*>(dst + (size_t)R1 * 64 + cb + 8 * n) = make_float2(G[n][2], G[n][3]);
-            }
-        }
-        // the bonus gradient of this unit: over the lanes' rows, then over the four row groups, in a fixed order
+    // ---- the bonus gradient of this unit: over the lanes' rows, the row groups and the two groups, in a fixed order
+    if (!alive && gt == 0) sts32(abort_flag, 1u);    // (the other group's waits see it)
+    if (!C2) {
 #pragma unroll
         for (int d = 4; d < 32; d <<= 1)
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
+            for (int n = 0; n < G_NB; ++n)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) du_acc[n][e] += __shfl_xor_sync(0xffffffffu, du_acc[n][e], d);
         if (g == 0) {
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
+            for (int n = 0; n < G_NB; ++n)
 #pragma unroll
-                for (int e = 0; e < 2; ++e) fsm(BO_RED_V)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
-        }
-        cbar();
-        if (!C2 && tid < 64) {
-            const float* rv4 = fsm(BO_RED_V);
-            p.du_part[(size_t)unit * 64 + tid] = ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fsm(BO_DU_FB)[tid];
+                for (int e = 0; e < 2; ++e) gsm(GO_REDV)[sp * 64 + cb + 8 * n + e] = du_acc[n][e];
         }
     }
-    if (tid == 0) post(CMD_QUIT, 0u);
-    }   // compute warps
+    if (gt == 0) {
+        bulk_wait<0>();                              // the gradient tiles have reached memory
+        // no copy into shared memory may stay in flight
+        if (last_a >= 0) mbar_wait(gb(GB_INA), (last_a >> 1) & 1, abort_flag, false);
+        if (last_b >= 0) mbar_wait(gb(GB_INB), (last_b >> 1) & 1, abort_flag, false);
+    }
     tc_fence_before();
     __syncthreads();
+    if (!C2 && tid < 64 && !lds32(abort_flag)) {
+        float s = 0.f;
+#pragma unroll
+        for (int gg = 0; gg < 2; ++gg) {
+            const float* rv4 = reinterpret_cast<const float*>(smem + gg * GO_BYTES + GO_REDV);
+            const float* fb = reinterpret_cast<const float*>(smem + gg * GO_BYTES + GO_DUFB);
+            s += ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fb[tid];
+        }
+        p.du_part[(size_t)unit * 64 + tid] = s;
+    }
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem, BT_COLS);
+        tmem_dealloc(lds32(sbase + GS_TMEM), GT_COLS);
     }
 }
 
@@ -827,5 +859,57 @@ wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H,
 }
 
 }  // namespace bc
+
+
+// Workspace of the chunked gradient: checkpoints, per-unit bonus gradients, the token-by-token path's scratch (one
+// slot of 64 states per SM and group of warps).
+inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
+{
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    return ((size_t)units * nck * 4096 + (size_t)units * 64 + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+}
+
+inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                    const __nv_bfloat16* x, const float* u, const float* state_in,
+                                    const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
+                                    __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
+                                    int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
+                                    bool c2 = false)
+{
+    const long long units = (long long)B * H, rows = (long long)B * T;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return GF_ERR_CUDA;
+    static PerDeviceFlag attr_set;
+    const int dev = current_device();
+    if (dev < 0) return GF_ERR_CUDA;
+    if (!attr_set.is_set(dev)) {
+        if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
+            return GF_ERR_CUDA;
+        attr_set.set(dev);
+    }
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    float* ckpt = ws;
+    float* du_part = ckpt + (size_t)units * nck * 4096;
+    float* fb = du_part + (size_t)units * 64;
+    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
+    if (s != GF_OK) return s;
+    const long long C = (long long)H * 64;
+    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
+    if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||
+        !ck::make_map(&tv, v, rows, C, 64) || !ck::make_map(&tdy, dy, rows, C, 64) || !ck::make_map(&tdr, dr, rows, C, 64) ||
+        !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
+        return GF_ERR_CUDA;
+    bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
+                  wait_limit_us().load(std::memory_order_relaxed)};
+    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    if (c2) return GF_OK;                            // no bonus, no bonus gradient
+    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
+    launches->fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+}
 
 }  // namespace gf
