@@ -372,7 +372,7 @@ def main():
                 ("prefill_c2", "cfg2-c2", "gf_wkv6_prefill_c2 with the second-value tensor, cfg2 shape (768 B per token*head)"),
                 ("key_compress", "kc-cfg2", "gf_gold_key_compress 65536 x 2048 -> 128"),
                 ("decay_logit", "dl-cfg2", "gf_c2_decay_logit, 65536 tokens x 2048 channels, ranks 32 and 64 (x read, d written)"),
-                ("backward", "bwd-cfg2", "gf_wkv6_backward, cfg2 shape: checkpoint pass + chunked gradient kernel (1152 B per token*head counted; the design moves 2048)"),
+                ("backward", "bwd-cfg2", "gf_wkv6_backward, cfg2 shape: checkpoint pass + chunked gradient kernel, two chunks in flight per SM (1152 B per token*head counted; the design moves 2048)"),
                 ("decode_step", "cfg4-decode", "gf_wkv6_step, 64 sequences x 32 heads, 64 steps per graph replay (states stay in L2)"),
                 ("decode_step_layer_stack", "cfg4-decode-layers", "gf_wkv6_step over 12 layers with their own states (streams from HBM)")):
             r = cases.run(case, 5, 1.0)
