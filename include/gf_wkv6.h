@@ -142,7 +142,7 @@ GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
  * checkpoint pass of the forward kernel.  A chunk in which some channel decays by more than 2^-96 is processed token
  * by token in fp32 instead, so any decay logit is accepted (x = +inf leaves dx undefined, as in the formula).
  * `workspace`: caller-owned DEVICE buffer of at least gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes, 16-byte
- * aligned (one 64x64 fp32 state per chunk and unit, plus 1 MiB per SM for the token-by-token path);
+ * aligned (one 64x64 fp32 state per chunk and unit, plus 2 MiB per SM for the token-by-token path);
  * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  Enqueues three
  * kernels on `stream`, allocates nothing, does not synchronise; deterministic (no atomics).  A device-side wait that
  * runs out is reported by gf_wkv6_last_device_status as for the forward call. */
@@ -165,6 +165,29 @@ GF_API gf_status_t gf_wkv6_backward_c2(const void *r, const void *k, const void 
                                 const float *state_in, const void *dy, const float *dstate_out, void *dr,
                                 void *dk, void *dv, void *dx, float *dstate_in, int B, int T, int H, int N,
                                 void *workspace, size_t workspace_bytes, gf_stream_t stream);
+
+/* A training step's pair.  gf_wkv6_prefill_train / gf_wkv6_prefill_c2_train are gf_wkv6_prefill / gf_wkv6_prefill_c2
+ * (same results, dense, one CTA per (sequence, head), never split) that also leave the state before every chunk of 64
+ * tokens and after the last one at the start of `workspace`, the gradient's workspace
+ * (gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes).  gf_wkv6_backward_saved / gf_wkv6_backward_c2_saved are
+ * gf_wkv6_backward / gf_wkv6_backward_c2 without their first launch: they take those states from the workspace, which
+ * must still hold what the forward call of the SAME r,k,v,x,state_in wrote (the caller's responsibility; nothing
+ * checks it).  One launch forward; two (one for the Finch-C2 form) backward. */
+GF_API gf_status_t gf_wkv6_prefill_train(const void *r, const void *k, const void *v, const void *x, const float *u,
+                                  const float *state_in, float *state_out, void *y, int B, int T, int H, int N,
+                                  void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_prefill_c2_train(const void *r, const void *k, const void *v, const void *x,
+                                     const void *u2, const float *state_in, float *state_out, void *y, int B,
+                                     int T, int H, int N, void *workspace, size_t workspace_bytes,
+                                     gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_backward_saved(const void *r, const void *k, const void *v, const void *x, const float *u,
+                                   const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                                   void *dk, void *dv, void *dx, float *du, float *dstate_in, int B, int T,
+                                   int H, int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_backward_c2_saved(const void *r, const void *k, const void *v, const void *x,
+                                      const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                                      void *dk, void *dv, void *dx, float *dstate_in, int B, int T, int H,
+                                      int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
 
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "prefill_train", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -37,6 +37,10 @@ _SIGNATURES = {
     "gf_wkv6_backward": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_bf16_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_backward_c2": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_saved": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_c2_saved": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_prefill_train": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_prefill_c2_train": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_prefill_c2": (_i, [_vp] * 8 + [_i] * 4 + [_vp]),
     "gf_wkv6_prefill_varlen_c2": (_i, [_vp] * 9 + [_i] * 5 + [_vp]),
     "gf_wkv6_step_c2": (_i, [_vp] * 8 + [_i] * 3 + [_vp]),
@@ -222,7 +226,7 @@ def prefill(r, k, v, x, u, state_in=None, state_out=None, y=None, stream=None, w
     return y, state_out
 
 
-def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None):
+def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None, saved=False):
     """gf_wkv6_backward (bf16 tensors: chunked on the tensor cores) or gf_wkv6_backward_f32 (fp32 tensors: token by
     token): gradient of the prefill.  r,k,v,x,dy: [B,T,H,N] CUDA tensors of one dtype, u: [H,N] fp32,
     state_in / dstate_out: [B,H,N,N] fp32 or None.  Returns (dr, dk, dv, dx, du, dstate_in); outputs (and the
@@ -234,6 +238,10 @@ def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True
     if dt not in (torch.bfloat16, f32):
         raise TypeError("backward: r must be bfloat16 or float32")
     sfx, wsfn = ("_f32", "gf_wkv6_backward_workspace_bytes") if dt == f32 else ("", "gf_wkv6_backward_bf16_workspace_bytes")
+    if saved:       # the workspace holds the checkpoints of prefill_train() of the same inputs
+        if dt == f32 or workspace is None:
+            raise ValueError("backward(saved=True) needs bf16 tensors and the workspace prefill_train() filled")
+        sfx = "_saved"
     dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
     du = torch.empty((H, N), device=r.device, dtype=f32)
     ds0 = torch.empty((B, H, N, N), device=r.device, dtype=f32) if want_dstate else None
@@ -249,7 +257,7 @@ def backward(r, k, v, x, u, dy, state_in=None, dstate_out=None, want_dstate=True
     return dr, dk, dv, dx, du, ds0
 
 
-def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None):
+def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True, stream=None, workspace=None, saved=False):
     """gf_wkv6_backward_c2: gradient of prefill_c2 (bf16 tensors; k is the key before the (1 - w) factor; the
     second-value vector's gradient is dy itself).  Returns (dr, dk, dv, dx, dstate_in)."""
     lib = load_library()
@@ -264,9 +272,30 @@ def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True
                 _dev(state_in, "state_in", f32, (B, H, N, N)), _dev(dy, "dy", bf, r.shape),
                 _dev(dstate_out, "dstate_out", f32, (B, H, N, N)), _dev(dr, "dr"), _dev(dk, "dk"), _dev(dv, "dv"),
                 _dev(dx, "dx"), _dev(ds0, "dstate_in")]
-        _check(lib.gf_wkv6_backward_c2(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)),
-               "gf_wkv6_backward_c2")
+        if saved and workspace is None:
+            raise ValueError("backward_c2(saved=True) needs the workspace prefill_c2_train() filled")
+        fn = "gf_wkv6_backward_c2_saved" if saved else "gf_wkv6_backward_c2"
+        _check(getattr(lib, fn)(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)), fn)
     return dr, dk, dv, dx, ds0
+
+
+def prefill_train(r, k, v, x, u, workspace, state_in=None, c2=False, u2=None, stream=None):
+    """gf_wkv6_prefill_train / gf_wkv6_prefill_c2_train: the forward pass of a training step.  As prefill() /
+    prefill_c2() (u is ignored with c2=True, u2 without), and `workspace` (uint8 CUDA tensor of
+    backward_workspace_bytes(B,T,H,N) bytes) receives the chunk-start states for backward(..., saved=True).
+    Returns (y, state_out)."""
+    lib = load_library()
+    B, T, H, N = r.shape
+    bf, f32 = torch.bfloat16, torch.float32
+    y = torch.empty_like(r)
+    s_out = torch.empty((B, H, N, N), device=r.device, dtype=f32)
+    with torch.cuda.device(r.device):
+        base = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape)]
+        mid = _dev(u2, "u2", bf, r.shape) if c2 else _dev(u, "u", f32, (H, N))
+        fn = "gf_wkv6_prefill_c2_train" if c2 else "gf_wkv6_prefill_train"
+        _check(getattr(lib, fn)(*base, mid, _dev(state_in, "state_in", f32, (B, H, N, N)), _dev(s_out, "state_out"),
+                                _dev(y, "y"), B, T, H, N, _dev(workspace, "workspace"), workspace.numel(), _stream(stream)), fn)
+    return y, s_out
 
 
 def backward_workspace_bytes(B, T, H, N, dtype=torch.bfloat16):

@@ -4,7 +4,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
 cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
-       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2
+       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 train-fwd-cfg2 train-bwd-cfg2
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -150,6 +150,21 @@ def run(case, reps, scale):
         return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H,
                     bytes=B * T * H * 64 * 2 * 9 + B * H * 16384 * (2 if k["state_std"] > 0 else 1),
                     design_bytes=B * T * H * 2048 + B * H * 16384 * 2, ms=_time(fn, reps))
+    if case in ("train-fwd-cfg2", "train-bwd-cfg2"):    # a training step's pair: forward that keeps its chunk-start states, gradient from them
+        k = c["cfg2"]
+        B, T, H = k["B"], sc(k["T"]), k["H"]
+        inp = synth.make_dense(B, T, H, 64, "bf16", seed=7, device=DEV, state_std=k["state_std"])
+        dy = torch.randn(inp.r.shape, device=DEV).bfloat16()
+        ws = torch.empty(gf.backward_workspace_bytes(B, T, H, 64), dtype=torch.uint8, device=DEV)
+        gf.prefill_train(inp.r, inp.k, inp.v, inp.x, inp.u, ws, inp.state_in)
+        if case == "train-fwd-cfg2":
+            fn = lambda: gf.prefill_train(inp.r, inp.k, inp.v, inp.x, inp.u, ws, inp.state_in)
+            nbytes = B * T * H * 640 + B * H * 16384
+        else:
+            fn = lambda: gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, None, workspace=ws, saved=True)
+            nbytes = B * T * H * 64 * 2 * 9 + B * H * 16384
+        # (the checkpoints, 256 B per token*head written by the one and read by the other, are the design's own)
+        return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H, bytes=nbytes, ms=_time(fn, reps))
     if case in ("cfg4-prefill", "cfg4-decode", "cfg4-decode-layers"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -199,7 +214,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "train-fwd-cfg2", "train-bwd-cfg2"]
 
 
 def main():

@@ -403,7 +403,7 @@ namespace {
 gf_status_t backward_bf16(const void* r, const void* k, const void* v, const void* x, const float* u,
                           const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk, void* dv,
                           void* dx, float* du, float* dstate_in, int B, int T, int H, int N, void* workspace,
-                          size_t workspace_bytes, gf_stream_t stream, bool c2)
+                          size_t workspace_bytes, gf_stream_t stream, bool c2, bool saved = false)
 {
     using bf = __nv_bfloat16;
     if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
@@ -436,7 +436,7 @@ gf_status_t backward_bf16(const void* r, const void* k, const void* v, const voi
     if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
     const gf_status_t s = gf::chunked_backward((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, (const bf*)dy,
                                                dstate_out, (bf*)dr, (bf*)dk, (bf*)dv, (bf*)dx, du, dstate_in, B, T, H,
-                                               static_cast<float*>(workspace), st, &g_launches, c2);
+                                               static_cast<float*>(workspace), st, &g_launches, c2, saved);
     if (s != GF_OK) return s;
     return launch_result();
 }
@@ -458,6 +458,68 @@ gf_status_t gf_wkv6_backward_c2(const void* r, const void* k, const void* v, con
 {
     return backward_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in, B, T, H, N,
                          workspace, workspace_bytes, stream, true);
+}
+
+gf_status_t gf_wkv6_backward_saved(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                   const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
+                                   void* dv, void* dx, float* du, float* dstate_in, int B, int T, int H, int N,
+                                   void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_bf16(r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, B, T, H, N, workspace,
+                         workspace_bytes, stream, false, true);
+}
+
+gf_status_t gf_wkv6_backward_c2_saved(const void* r, const void* k, const void* v, const void* x, const float* state_in,
+                                      const void* dy, const float* dstate_out, void* dr, void* dk, void* dv, void* dx,
+                                      float* dstate_in, int B, int T, int H, int N, void* workspace,
+                                      size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in, B, T, H, N,
+                         workspace, workspace_bytes, stream, true, true);
+}
+
+namespace {
+// forward pass of a training step: the prefill that also leaves its chunk-start states in the gradient's workspace
+gf_status_t prefill_train(const void* r, const void* k, const void* v, const void* x, const float* u, const void* u2,
+                          const float* state_in, float* state_out, void* y, int B, int T, int H, int N, void* workspace,
+                          size_t workspace_bytes, gf_stream_t stream, bool c2)
+{
+    using bf = __nv_bfloat16;
+    if (B < 0 || T < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (T == 0) return pass_state(state_in, state_out, (size_t)B * H, st);
+    if (!r || !k || !v || !x || !y || (!c2 && !u)) return GF_ERR_INVALID_ARG;
+    const void* ptrs[] = {r, k, v, x, u, u2, state_in, state_out, y, workspace};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x || (u2 && y == u2)) return GF_ERR_INVALID_ARG;
+    if ((long long)B * H > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    if ((long long)B * T >= (1LL << 31) - 64) return GF_ERR_UNSUPPORTED;
+    const size_t need = gf_wkv6_backward_bf16_workspace_bytes(B, T, H, N);
+    if (need == 0) return GF_ERR_CUDA;
+    if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
+    const gf_status_t s = gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
+                                              (bf*)y, nullptr, B, T, (long long)B * T, H, st, &g_launches, nullptr, 0,
+                                              (const bf*)u2, c2 ? 1 : 0, static_cast<float*>(workspace));
+    if (s != GF_OK) return s;
+    return launch_result();
+}
+}  // namespace
+
+gf_status_t gf_wkv6_prefill_train(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                  const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                                  void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return prefill_train(r, k, v, x, u, nullptr, state_in, state_out, y, B, T, H, N, workspace, workspace_bytes, stream, false);
+}
+
+gf_status_t gf_wkv6_prefill_c2_train(const void* r, const void* k, const void* v, const void* x, const void* u2,
+                                     const float* state_in, float* state_out, void* y, int B, int T, int H, int N,
+                                     void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return prefill_train(r, k, v, x, nullptr, u2, state_in, state_out, y, B, T, H, N, workspace, workspace_bytes, stream, true);
 }
 
 size_t gf_wkv6_host_workspace_bytes(int B, int T, int H, int N)

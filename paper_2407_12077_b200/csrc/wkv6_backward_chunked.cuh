@@ -874,7 +874,7 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
                                     const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
                                     __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
                                     int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
-                                    bool c2 = false)
+                                    bool c2 = false, bool ckpt_saved = false)
 {
     const long long units = (long long)B * H, rows = (long long)B * T;
     const int n_sm = sm_count();
@@ -892,8 +892,10 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     float* ckpt = ws;
     float* du_part = ckpt + (size_t)units * nck * 4096;
     float* fb = du_part + (size_t)units * 64;
-    gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
-    if (s != GF_OK) return s;
+    if (!ckpt_saved) {                               // (else the forward pass of the training step left them there)
+        const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
+        if (s != GF_OK) return s;
+    }
     const long long C = (long long)H * 64;
     CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
     if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||

@@ -636,7 +636,9 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
 // C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus, optional second-value vector).
 // PERSIST = true: the CTA walks a stream of units (see Params::n_units); the producer warp leaves a descriptor per
 // chunk and two end markers, which every role passes down its own signalling path before it leaves.
-template <bool SUMMARY, bool C2, bool PERSIST = false>
+// CKPT = true (single-unit, unsplit launches of the prefill proper): the state before every chunk and after the last
+// one is also left in Params::ckpt, for the gradient call that follows a training step's forward pass.
+template <bool SUMMARY, bool C2, bool PERSIST = false, bool CKPT = false>
 __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
@@ -675,6 +677,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     static_assert(!(PERSIST && SUMMARY), "the summary pass is a single-unit launch");
+    static_assert(!(CKPT && (PERSIST || SUMMARY)), "checkpoints of the prefill proper: single-unit launches only");
 
     // One chunk of this CTA's work.  Single-unit launches derive it from the chunk index; persistent launches
     // read the descriptor the producer warp left for the chunk, which is visible to any warp that has waited
@@ -972,7 +975,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
-            if (SUMMARY && p.ckpt) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + c) * 4096);   // the state before chunk c
+            if (CKPT || (SUMMARY && p.ckpt)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + c) * 4096);   // the state before chunk c
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1065,6 +1068,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
+        if (CKPT && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + nchunks) * 4096);
         if (SUMMARY && p.ckpt) {
             if (!lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + nchunks) * 4096);
         } else if (SUMMARY) {
@@ -1504,7 +1508,7 @@ inline int choose_split(long long units, int T, int n_sm, int* seg_chunks, size_
     return 1;
 }
 
-// Opts the six instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
+// Opts the eight instantiations of the chunked kernel in to their dynamic shared-memory size, once per device.
 inline bool chunked_kernel_attributes()
 {
     static PerDeviceFlag attr_set;                   // zero-initialised
@@ -1516,7 +1520,9 @@ inline bool chunked_kernel_attributes()
             cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(ck::wkv6_chunked_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(ck::wkv6_chunked_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ck::SMEM_ALLOC) != cudaSuccess)
             return false;
         attr_set.set(dev);
     }
@@ -1564,7 +1570,8 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
                                    const __nv_bfloat16* x, const float* u, const float* state_in, float* state_out,
                                    __nv_bfloat16* y, const int32_t* cu, int n_seq, int T, long long total_rows, int H,
                                    cudaStream_t st, std::atomic<uint64_t>* launches, float* scratch = nullptr,
-                                   size_t scratch_bytes = 0, const __nv_bfloat16* u2 = nullptr, int c2 = 0)
+                                   size_t scratch_bytes = 0, const __nv_bfloat16* u2 = nullptr, int c2 = 0,
+                                   float* ckpt = nullptr)
 {
     const long long units = (long long)n_seq * H;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
@@ -1579,7 +1586,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         !ck::make_map(&ty, y, total_rows, C, 16) || !ck::make_map(&tu2, u2 ? (const void*)u2 : (const void*)y, total_rows, C, 16))
         return GF_ERR_CUDA;
     int seg_chunks = 0, nseg = 1;
-    if (scratch) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
+    if (scratch && !ckpt) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
         size_t need = 0;
         nseg = choose_split(units, T, sm_count(), &seg_chunks, &need, scratch_bytes);   // (never splits with more units than half the SMs)
         if (nseg > 1 && units * nseg > 0x7fffffffLL) nseg = 1;
@@ -1587,6 +1594,15 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
     if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
+    if (ckpt) {
+        // a training step's forward pass (dense): one CTA per unit, unsplit, the chunk-start states kept for the gradient
+        if (cu) return GF_ERR_UNSUPPORTED;
+        p.ckpt = ckpt;
+        if (c2) ck::wkv6_chunked_kernel<false, true, false, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        else ck::wkv6_chunked_kernel<false, false, false, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+    }
     const int n_sm = sm_count();
     // More units than SMs: one CTA per SM walks a stream of units, so that a unit's pipeline fill overlaps the
     // drain of the one before it.  That saves about 4.5 us per unit and costs about 3 % more instructions per
