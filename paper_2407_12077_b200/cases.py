@@ -4,7 +4,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
 cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
-       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 train-fwd-cfg2 train-bwd-cfg2
+       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 bwd-cfg3 train-fwd-cfg2 train-bwd-cfg2
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -137,8 +137,8 @@ def run(case, reps, scale):
                  bytes=2 * B * T * D * 2 + 4 * D * (Rd + Rw) + 12 * D, ms=_time(fn, reps))
         r["tflops"] = 2.0 * B * T * D * 2 * (Rd + Rw) / (r["ms"] * 1e-3) / 1e12
         return r
-    if case in ("bwd-cfg1", "bwd-cfg2"):    # gradient of one prefill call (bf16, chunked on the tensor cores)
-        k = c["cfg1" if case == "bwd-cfg1" else "cfg2"]
+    if case in ("bwd-cfg1", "bwd-cfg2", "bwd-cfg3"):    # gradient of one prefill call (bf16, chunked on the tensor cores)
+        k = c[{"bwd-cfg1": "cfg1", "bwd-cfg2": "cfg2", "bwd-cfg3": "cfg3"}[case]]     # (cfg3: 32 units, the sequences split)
         B, T, H = k["B"], sc(k["T"]), k["H"]
         inp = synth.make_dense(B, T, H, 64, "bf16", seed=7, device=DEV, state_std=k["state_std"])
         dy = torch.randn(inp.r.shape, device=DEV).bfloat16()
@@ -214,7 +214,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "train-fwd-cfg2", "train-bwd-cfg2"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "bwd-cfg3", "train-fwd-cfg2", "train-bwd-cfg2"]
 
 
 def main():

@@ -62,7 +62,16 @@ struct BParams {
     __nv_bfloat16 *dr, *dk, *dv, *dx;
     int T, H, n_slots;
     uint32_t wait_limit_us;
+    // Sequence split (calls with few units): every sequence is cut into nseg segments of seg_chunks chunks (the last
+    // takes the rest) and the grid is units x nseg.  The state adjoint at a segment's end follows from dstate_out and the
+    // summaries of the segments after it, G <- diag(D_s) G + dG_s for s = nseg-1 down to seg+1, which a first launch
+    // (the kernel's summary variant, grid units x (nseg-1)) leaves in gsum: [unit][s-1][64 + 64*64] fp32.  nseg = 1: no
+    // split.  du_part is [unit][seg][64].
+    const float* gsum;
+    float* gsum_out;             // summary variant: where the summaries go (same layout)
+    int nseg, seg_chunks;
 };
+constexpr int GSUM_FLOATS = 64 + 64 * 64;
 
 __device__ __forceinline__ float lds_bf16(uint32_t a)
 {
@@ -229,7 +238,10 @@ __device__ __forceinline__ bool scan_rows(float (&v)[G_NB][4], uint32_t tot, int
     return ok;
 }
 
-template <bool C2>
+// GSUM = true: the summary variant of a split call (see BParams::gsum): only the adjoint's own recurrence
+// G <- diag(D) G + R^^T dY over a segment, from zero, and the product of the chunk decays; it reads x, r, dy only and
+// needs no token-by-token path (R^ never exceeds r: no exponent can overflow).
+template <bool C2, bool GSUM = false>
 __global__ void __launch_bounds__(G_THREADS, 1)
 wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -246,8 +258,13 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int grp = tid / G_GT, gt = tid % G_GT;                    // group, thread inside the group
     const int sp = warp & 3, cx = (warp >> 2) % G_NSLAB, g = lane >> 2, q = lane & 3;       // row group, column slab
-    const int unit = blockIdx.x, seq = unit / p.H, h = unit % p.H;
+    // summary variant: segments 1 .. nseg-1 of every unit; else every segment
+    const int gsegs = GSUM ? p.nseg - 1 : p.nseg;
+    const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0), seq = unit / p.H, h = unit % p.H;
     const int T = p.T, nchunks = (T + L - 1) / L;
+    const int c_lo = p.nseg > 1 ? min(nchunks, seg * p.seg_chunks) : 0;                      // this CTA's chunks: c_lo .. c_hi-1,
+    const int c_hi = (p.nseg > 1 && seg < p.nseg - 1) ? min(nchunks, c_lo + p.seg_chunks) : nchunks;   // walked from the last
+    const int nit = c_hi - c_lo;
     const long long row0 = (long long)seq * T;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
@@ -286,7 +303,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (tid < 64) reinterpret_cast<float*>(smem + GS_U)[tid] = C2 ? 0.f : p.u[col0 + tid];
+    if (tid < 64) reinterpret_cast<float*>(smem + GS_U)[tid] = (C2 || GSUM) ? 0.f : p.u[col0 + tid];
     if (gt < 64) gsm(GO_DUFB)[gt] = 0.f;
     if (warp == 1) tmem_alloc(sbase + GS_TMEM, GT_COLS);
     tc_fence_before();
@@ -295,7 +312,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const uint32_t tmem = lds32(sbase + GS_TMEM) + 256 * grp;                 // this group's columns
     const uint32_t tacc = tmem + ((uint32_t)(32 * sp) << 16) + 8 * G_NB * cx;      // this warp's block of an accumulator
 
-    auto chunk_of = [&](int it) { return nchunks - 1 - it; };
+    auto chunk_of = [&](int it) { return c_hi - 1 - it; };
     const uint32_t tin = gbase + GO_IN;
     const uint32_t tx = tin, tr = tin + TILE, tk = tin + 2 * TILE, tv = tin + 3 * TILE, tdy = tin + 4 * TILE;
     const uint32_t t_rh = gbase + GO_RH, t_kh = gbase + GO_KH;
@@ -341,19 +358,20 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
-    if (gt == 0 && grp < nchunks) { issue_loads_a(grp); issue_loads_b(grp); }
+    if (gt == 0 && grp < nit) { issue_loads_a(grp); issue_loads_b(grp); }
     int mph = 0;                                     // phase bit of this group's two product barriers
+    float dprod_lo = 1.f, dprod_hi = 1.f;            // summary variant: product of this group's chunk decays (rows R0, R1)
     bool alive = true;
 
-    for (int it = grp; it < nchunks; it += 2) {
+    for (int it = grp; it < nit; it += 2) {
         const int c = chunk_of(it), valid = min(L, T - c * L);
         const int use = it >> 1;                     // how often this group's input stage has been filled before
         float S0[G_NB][4];                              // the chunk-start state (requested early: it is used after the scan)
-        load_f32_block(ck_unit + (size_t)c * 4096, S0);
-        if (it + 2 < nchunks) {
+        if (!GSUM) load_f32_block(ck_unit + (size_t)c * 4096, S0);
+        if (it + 2 < nit) {
             // this group's next chunk: its start state and its input tiles into L2 now, so that the copies issued at
             // the end of this iteration and the load above find them there
-            if (gt < 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 2) * 4096 + 32 * gt));
+            if (!GSUM && gt < 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 2) * 4096 + 32 * gt));
             if (gt == 128) {
                 const int row = (int)(row0 + (long long)(c - 2) * L);
                 tma_prefetch_2d(&tm_x, col0, row); tma_prefetch_2d(&tm_r, col0, row); tma_prefetch_2d(&tm_k, col0, row);
@@ -385,7 +403,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
             for (int o = 0; o < 4; ++o) { al0 += gld(GO_TOT + 4 * (o * 64 + R0)); al1 += gld(GO_TOT + 4 * (o * 64 + R1)); }
             d_lo = ex2(al0); d_hi = ex2(al1);
-            safe = (al0 >= -A2_MAX) && (al1 >= -A2_MAX);                   // false for NaN as well
+            safe = GSUM || ((al0 >= -A2_MAX) && (al1 >= -A2_MAX));         // false for NaN as well
+            if (GSUM) { dprod_lo *= d_lo; dprod_hi *= d_hi; }
         }
         // ---- operands from the inputs: R^, K^ (and the bonus), the chunk-start state
         if (!mbar_wait(gb(GB_INB), use & 1, abort_flag)) ok = false;        // (made uniform at a later barrier)
@@ -407,7 +426,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if (C2) kv[n][e] *= one_minus_ex2(lw2[n][e]);      // the key that enters the state
-                    if (!C2) {
+                    if (!C2 && !GSUM) {
                         const float t = rv[n][e] * kv[n][e] * ldsf(sbase + GS_U + 4 * (cb + 8 * n + (e & 1)));
                         if (e < 2) b0 += t; else b1 += t;
                     }
@@ -415,14 +434,14 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     kv[n][e] *= ex2(-a[n][e]);
                 }
             st_tile(t_rh, moff, rv);
-            st_tile(t_kh, moff, kv);
-            if (!C2) {
+            if (!GSUM) st_tile(t_kh, moff, kv);
+            if (!C2 && !GSUM) {
                 b0 += __shfl_xor_sync(0xffffffffu, b0, 1); b1 += __shfl_xor_sync(0xffffffffu, b1, 1);
                 b0 += __shfl_xor_sync(0xffffffffu, b0, 2); b1 += __shfl_xor_sync(0xffffffffu, b1, 2);
                 if (q == 0) { stsf(gbase + GO_BP + 4 * (cx * 64 + R0), b0); stsf(gbase + GO_BP + 4 * (cx * 64 + R1), b1); }
             }
         }
-        st_tile(t_sb, moff, S0);
+        if (!GSUM) st_tile(t_sb, moff, S0);
         fence_proxy_async();
         tc_fence_before();
         const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
@@ -434,6 +453,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             for (int kk = 0; kk < 4; ++kk) {
                 const uint64_t ks = 2 * kk, ms = 128 * kk;       // K-major / MN-major step of 16 contraction indices
                 tc_mma(tmem + GT_DG, dR + ms, dY + ms, IDESC_MN_MN, kk > 0);       // dG[c][j] = R^^T dY
+                if (GSUM) continue;
                 tc_mma(tmem + GT_P, dR + ks, dK + ks, IDESC_K_K, kk > 0);          // P[t][i]  = R^ K^^T
                 tc_mma(tmem + GT_DP, dY + ks, dV + ks, IDESC_K_K, kk > 0);         // dP[t][i] = dY V^T
             }
@@ -442,10 +462,24 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         // ---- the adjoint at the chunk's end, from the other group (the call's dstate_out for the last chunk)
         float G[G_NB][4];
         if (it == 0) {
-            if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
+            if (!GSUM && p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
             else {
 #pragma unroll
                 for (int n = 0; n < G_NB; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
+            }
+            if (!GSUM) {
+                // a segment but the last: the adjoint at its end through the segments after it, from the last down
+                for (int sg = p.nseg - 1; sg > seg; --sg) {
+                    const float* sm = p.gsum + ((size_t)unit * (p.nseg - 1) + (sg - 1)) * GSUM_FLOATS;
+                    const float dl = sm[R0], dh = sm[R1];
+                    float dG[G_NB][4];
+                    load_f32_block(sm + 64, dG);
+#pragma unroll
+                    for (int n = 0; n < G_NB; ++n) {
+                        G[n][0] = fmaf(dl, G[n][0], dG[n][0]); G[n][1] = fmaf(dl, G[n][1], dG[n][1]);
+                        G[n][2] = fmaf(dh, G[n][2], dG[n][2]); G[n][3] = fmaf(dh, G[n][3], dG[n][3]);
+                    }
+                }
             }
         } else {
             if (!mbar_wait(bar(GB_GREADY + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag)) ok = false;
@@ -464,7 +498,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             e0 += __shfl_xor_sync(0xffffffffu, e0, 2); e1 += __shfl_xor_sync(0xffffffffu, e1, 2);
             if (q == 0) { stsf(dst + 4 * (cx * 64 + R0), e0); stsf(dst + 4 * (cx * 64 + R1), e1); }
         };
-        if (it == 0) {
+        if (GSUM) {
+        } else if (it == 0) {
             float SL[G_NB][4];
             load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
             e_put(gbase + GO_EP, G, SL);
@@ -595,17 +630,17 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 gbar(grp);
             }
             // hand the adjoint on (and the row sums the next chunk needs, from the fp32 state: the operand tile is gone)
-            if (it + 1 < nchunks) {
+            if (it + 1 < nit) {
                 g_put(it & 1, G);
                 load_f32_block(ck_unit + (size_t)c * 4096, S);
                 e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, S);
                 mbar_arrive(bar(GB_GREADY + (it & 1)));
-            } else if (p.dstate_in) {
+            } else if (p.dstate_in && seg == 0) {
                 store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
             }
         } else {
             // ---- G^ as an operand; G_0 = G^ + R^^T dY handed on
-            {
+            if (!GSUM) {
                 float gh[G_NB][4];
 #pragma unroll
                 for (int n = 0; n < G_NB; ++n) {
@@ -627,16 +662,26 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                     G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
                 }
             }
-            if (it + 1 < nchunks) {
+            if (it + 1 < nit) {
                 g_put(it & 1, G);
-                {
+                if (!GSUM) {
                     float sb[G_NB][4];               // this chunk's start state is the next chunk's end state (bf16 copy: the operand tile)
                     ld_tile(t_sb, moff, sb);
                     e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, sb);
                 }
                 mbar_arrive(bar(GB_GREADY + (it & 1)));
-            } else if (p.dstate_in) {
+            } else if (GSUM) {
+                store_f32_block(p.gsum_out + ((size_t)unit * (p.nseg - 1) + (seg - 1)) * GSUM_FLOATS + 64, G);      // the segment's dG
+            } else if (p.dstate_in && seg == 0) {
                 store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
+            }
+            if (GSUM) {
+                // nothing else in the summary variant: once every lane is done with the tiles, the next chunk's copies
+                mph ^= 1;
+                tc_fence_before();
+                if (!gbar_and(grp, ok)) { alive = false; break; }
+                if (gt == 0 && it + 2 < nit) { issue_loads_a(it + 2); issue_loads_b(it + 2); }
+                continue;
             }
             // ---- masked scores and their adjoint as operands
 #pragma unroll
@@ -760,7 +805,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             if (!mbar_wait(gb(GB_MV), mph, abort_flag)) ok = false;
             mph ^= 1;
             tc_fence_after();
-            if (gt == 0 && it + 2 < nchunks) issue_loads_a(it + 2);
+            if (gt == 0 && it + 2 < nit) issue_loads_a(it + 2);
             {
                 float acc[G_NB][4];
 #pragma unroll
@@ -771,7 +816,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             tc_fence_before();
             ok = scan_rows<true>(z, gbase + GO_TOT, grp, sp, cb, lane, ok);
             if (!ok) { alive = false; break; }
-            if (gt == 0 && it + 2 < nchunks) issue_loads_b(it + 2);      // (r, k were last read before the barrier of the sums)
+            if (gt == 0 && it + 2 < nit) issue_loads_b(it + 2);      // (r, k were last read before the barrier of the sums)
 #pragma unroll
             for (int n = 0; n < G_NB; ++n) {
                 float E0 = 0.f, E1 = 0.f;
@@ -804,13 +849,14 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 tma_store_2d(&tm_dx, col0, row, o_dx);
                 bulk_commit();
             }
-            if (unsafe && it + 2 < nchunks) { issue_loads_a(it + 2); issue_loads_b(it + 2); }      // (the other path has issued them)
+            if (unsafe && it + 2 < nit) { issue_loads_a(it + 2); issue_loads_b(it + 2); }      // (the other path has issued them)
         }
     }
 
     // ---- the bonus gradient of this unit: over the lanes' rows, the row groups and the two groups, in a fixed order
     if (!alive && gt == 0) sts32(abort_flag, 1u);    // (the other group's waits see it)
-    if (!C2) {
+    if (GSUM && cx == 0 && q == 0) { stsf(gbase + GO_REDV + 4 * R0, dprod_lo); stsf(gbase + GO_REDV + 4 * R1, dprod_hi); }
+    if (!C2 && !GSUM) {
 #pragma unroll
         for (int d = 4; d < 32; d <<= 1)
 #pragma unroll
@@ -832,7 +878,10 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     }
     tc_fence_before();
     __syncthreads();
-    if (!C2 && tid < 64 && !lds32(abort_flag)) {
+    if (GSUM && tid < 64 && !lds32(abort_flag))       // the segment's decay: the product over both groups' chunks
+        p.gsum_out[((size_t)unit * (p.nseg - 1) + (seg - 1)) * GSUM_FLOATS + tid] =
+            ldsf(sbase + GO_REDV + 4 * tid) * ldsf(sbase + GO_BYTES + GO_REDV + 4 * tid);
+    if (!C2 && !GSUM && tid < 64 && !lds32(abort_flag)) {
         float s = 0.f;
 #pragma unroll
         for (int gg = 0; gg < 2; ++gg) {
@@ -840,7 +889,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             const float* fb = reinterpret_cast<const float*>(smem + gg * GO_BYTES + GO_DUFB);
             s += ((rv4[tid] + rv4[64 + tid]) + (rv4[128 + tid] + rv4[192 + tid])) + fb[tid];
         }
-        p.du_part[(size_t)unit * 64 + tid] = s;
+        p.du_part[((size_t)unit * p.nseg + seg) * 64 + tid] = s;
     }
     if (warp == 1) {
         tc_fence_after();
@@ -850,23 +899,35 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 
 // du[h][i] = sum over the batch of the units' partial sums, in batch order
 __global__ void __launch_bounds__(64)
-wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H, float* __restrict__ du)
+wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H, int nseg, float* __restrict__ du)
 {
     const int h = blockIdx.x, i = threadIdx.x;
     float acc = 0.f;
-    for (int b = 0; b < B; ++b) acc += du_part[((size_t)b * H + h) * 64 + i];
+    for (int b = 0; b < B; ++b)
+        for (int sg = 0; sg < nseg; ++sg) acc += du_part[(((size_t)b * H + h) * nseg + sg) * 64 + i];
     du[h * 64 + i] = acc;
 }
 
 }  // namespace bc
 
 
-// Workspace of the chunked gradient: checkpoints, per-unit bonus gradients, the token-by-token path's scratch (one
-// slot of 64 states per SM and group of warps).
+// The sequence split of a gradient call: as for the forward pass (choose_split), calls with fewer units than half the
+// SMs cut every sequence into up to 8 segments of at least 8 chunks.
+inline int backward_split(long long units, int T, int n_sm, int* seg_chunks)
+{
+    size_t unused = 0;
+    return choose_split(units, T, n_sm, seg_chunks, &unused);
+}
+
+// Workspace of the chunked gradient: checkpoints, bonus gradients per unit and segment, the adjoint's segment
+// summaries, the token-by-token path's scratch (one slot of 64 states per SM and group of warps).
 inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
 {
     const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
-    return ((size_t)units * nck * 4096 + (size_t)units * 64 + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+    int seg_chunks = 0;
+    const int nseg = backward_split(units, T, n_sm, &seg_chunks);
+    return ((size_t)units * nck * 4096 + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS +
+            (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
 inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
@@ -884,16 +945,22 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     if (dev < 0) return GF_ERR_CUDA;
     if (!attr_set.is_set(dev)) {
         if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set.set(dev);
     }
     const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    int seg_chunks = 0;
+    int nseg = backward_split(units, T, n_sm, &seg_chunks);
+    if (units * nseg > 0x7fffffffLL) nseg = 1;
     float* ckpt = ws;
     float* du_part = ckpt + (size_t)units * nck * 4096;
-    float* fb = du_part + (size_t)units * 64;
+    float* gsum = du_part + (size_t)units * nseg * 64;
+    float* fb = gsum + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
     if (!ckpt_saved) {                               // (else the forward pass of the training step left them there)
-        const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0);
+        // (split calls: the forward summaries borrow the buffer of the adjoint's, which are written after them)
+        const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0, gsum, nseg, seg_chunks);
         if (s != GF_OK) return s;
     }
     const long long C = (long long)H * 64;
@@ -903,13 +970,19 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
         return GF_ERR_CUDA;
     bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
-                  wait_limit_us().load(std::memory_order_relaxed)};
-    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
-    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks};
+    if (nseg > 1) {
+        // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
+        bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    }
+    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     if (c2) return GF_OK;                            // no bonus, no bonus gradient
-    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, du);
+    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, nseg, du);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

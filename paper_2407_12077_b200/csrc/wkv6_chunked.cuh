@@ -477,9 +477,10 @@ struct Params {
     // reads state_in once the first state_out has been written (state_out may be state_in).  NULL: no copy.
     float* state_copy;
     uint32_t wait_limit_us;                // limit of every device-side wait of the launch (0: the default, 2 s)
-    // Checkpoint pass (a summary launch with one segment per unit, used by the gradient): starts from state_in and
-    // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32) instead of
-    // a summary.  NULL: no checkpoints.
+    // Checkpoint pass (a summary-variant launch over every segment, used by the gradient): starts from state_in, folds
+    // the summaries of the segments before its own (nseg > 1: a plain summary launch has left them in `summaries`) and
+    // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32, dense
+    // sequences) instead of a summary.  The prefill proper fills it too in its CKPT instantiations.  NULL: none.
     float* ckpt;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
@@ -951,7 +952,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         // second launch of a split call: the summaries and the start-state copy are the first launch's
         if (!SUMMARY && !PERSIST && p.nseg > 1) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!PERSIST) load_state(sb);
-        if (!SUMMARY) {
+        if (!SUMMARY || p.ckpt) {
             // start state of a later segment: fold the summaries of the segments before it, in order
             for (int gg = 0; gg < seg; ++gg) {
                 const float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + gg) * SUMMARY_FLOATS;
@@ -975,7 +976,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
-            if (CKPT || (SUMMARY && p.ckpt)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + c) * 4096);   // the state before chunk c
+            if (CKPT || (SUMMARY && p.ckpt))         // the state before chunk c of the segment (dense sequences: T / 64 + 1 states per unit)
+                store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + seg * p.seg_chunks + c) * 4096);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1068,9 +1070,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (CKPT && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + nchunks) * 4096);
+        if (CKPT && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
         if (SUMMARY && p.ckpt) {
-            if (!lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * (nchunks + 1) + nchunks) * 4096);
+            if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
+                store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
         } else if (SUMMARY) {
             if (!lds32(abort_flag)) {
                 float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
@@ -1683,10 +1686,12 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
 
 // Checkpoint pass of dense sequences: the state before every chunk of 64 tokens and after the last one,
 // ckpt [n_seq*H][chunks + 1][64][64] fp32, from state_in (NULL: zero).  One summary-variant launch (state only: reads
-// k, v and the decay logits).
+// k, v and the decay logits); with `summaries` (scratch of units x (nseg - 1) summaries) and nseg > 1 two: the sequences
+// split into segments as in a split prefill call.
 inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x,
                                        const float* state_in, float* ckpt, int n_seq, int T, int H, cudaStream_t st,
-                                       std::atomic<uint64_t>* launches, int c2 = 0)
+                                       std::atomic<uint64_t>* launches, int c2 = 0, float* summaries = nullptr,
+                                       int nseg = 1, int seg_chunks = 0)
 {
     const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
@@ -1697,11 +1702,20 @@ inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat
     if (!ck::make_map(&tk, k, total_rows, C, 64) || !ck::make_map(&tv, v, total_rows, C, 64) ||
         !ck::make_map(&tx, x, total_rows, C, 64) || !ck::make_map(&tdummy, k, total_rows, C, 16))
         return GF_ERR_CUDA;
-    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, nullptr, (T + ck::L - 1) / ck::L, 1, nullptr, c2};
+    if (!summaries || nseg < 2) { nseg = 1; seg_chunks = (T + ck::L - 1) / ck::L; }
+    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, summaries, seg_chunks, nseg, nullptr, c2};
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
+    if (nseg > 1) {
+        // few units: the segments' summaries first (every segment but the last, from a zero state), then every segment
+        // side by side from its folded start state, this time keeping the states
+        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+        launches->fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+    }
     p.ckpt = ckpt;
-    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
-    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

@@ -114,6 +114,30 @@ def test_cfg2_shape_every_unit_at_the_benchmarked_size():
     assert orc.rel_l2(out[4].numpy(), du_ref) <= TOL
 
 
+@pytest.mark.parametrize("B,T,H,x_lo,x_hi", [(1, 4096, 2, -6.0, -1.0), (1, 2000, 3, -6.0, -1.0), (2, 1100, 1, -12.0, -8.0),
+                                              (1, 8192, 1, -3.0, 0.3), (1, 1030, 4, -6.0, -1.0)])
+def test_few_units_split_their_sequences(B, T, H, x_lo, x_hi):
+    """Fewer units than half the SMs: every sequence is cut into segments that run side by side; the state adjoint at
+    a segment's end comes from the summaries (decay product, adjoint from zero) of the segments after it.  Slow
+    decays make the hand-over matter across the whole sequence."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert gf.split_plan(B, T, H, sms)[0] > 1       # (the forward pass's rule, which the gradient shares)
+    _run(B, T, H, seed=640 + T, state_std=0.3, with_dstate=True, x_lo=x_lo, x_hi=x_hi)
+
+
+def test_split_with_a_fast_channel_in_a_middle_segment():
+    B, T, H = 1, 4096, 2
+    inp, dy, dsT = _inputs(B, T, H, 660, 0.3, True)
+    x = inp.x.clone()
+    x[0, 2100:2104, 1, 9] = 5.0
+    inp.x = x
+    d = inp.to(DEV)
+    out = gf.backward(d.r, d.k, d.v, d.x, d.u, dy.to(DEV), d.state_in, dsT.to(DEV))
+    gf.last_device_status()
+    ref = orc.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy.double().numpy(), inp.state_in, dsT.double().numpy())
+    _check(out, ref, "split, mixed")
+
+
 @pytest.mark.parametrize("x_lo,x_hi", [(-12.0, -8.0), (-4.0, -1.0), (-3.0, 0.5), (-2.0, 0.0)])
 def test_slow_to_fast_decays_on_the_tensor_cores(x_lo, x_hi):
     """From w close to one (state and adjoint reach across the whole sequence) to decays close to the limit of the

@@ -56,6 +56,11 @@ def test_ragged_lengths_with_states(T, with_dstate):
     _run(2, T, 3, seed=800 + T, state_std=0.1, with_dstate=with_dstate)
 
 
+def test_few_units_split_their_sequences():
+    _run(1, 4096, 2, seed=850, state_std=0.3, with_dstate=True)
+    _run(1, 2000, 3, seed=851, state_std=0.3, with_dstate=True, x_lo=-12.0, x_hi=-8.0)
+
+
 def test_cfg1_shape_every_unit():
     c = synth.CONFIGS["cfg1"]
     print(_run(c["B"], c["T"], c["H"], seed=1100, state_std=c["state_std"], with_dstate=True))
