@@ -144,8 +144,9 @@ GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
  * `workspace`: caller-owned DEVICE buffer of at least gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes, 16-byte
  * aligned (one 64x64 fp32 state per chunk and unit, plus 2 MiB per SM for the token-by-token path);
  * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  Enqueues three
- * kernels on `stream`, allocates nothing, does not synchronise; deterministic (no atomics).  A device-side wait that
- * runs out is reported by gf_wkv6_last_device_status as for the forward call. */
+ * kernels on `stream` (five when B*H is less than half the SMs: the sequences are then cut into segments that run
+ * side by side, as in the forward call), allocates nothing, does not synchronise; deterministic (no atomics).  A
+ * device-side wait that runs out is reported by gf_wkv6_last_device_status as for the forward call. */
 GF_API gf_status_t gf_wkv6_backward(const void *r, const void *k, const void *v, const void *x, const float *u,
                              const float *state_in, const void *dy, const float *dstate_out, void *dr,
                              void *dk, void *dv, void *dx, float *du, float *dstate_in, int B, int T, int H,
