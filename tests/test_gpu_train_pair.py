@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.mark.parametrize("B,T,H", [(2, 300, 3), (1, 64, 1), (4, 1000, 8), (1, 37, 2)])
+@pytest.mark.parametrize("B,T,H", [(2, 300, 3), (1, 64, 1), (4, 1000, 8), (1, 37, 2), (1, 4096, 2)])   # (the last: the gradient splits)
 @pytest.mark.parametrize("c2", [False, True])
 def test_pair_is_bit_identical_to_the_separate_calls(B, T, H, c2):
     inp = synth.make_dense(B, T, H, 64, "bf16", seed=40 + T, state_std=0.1).to(DEV)
@@ -33,7 +33,14 @@ def test_pair_is_bit_identical_to_the_separate_calls(B, T, H, c2):
         gb = gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT)
     gf.last_device_status()
     assert torch.equal(y, y0) and torch.equal(s, s0)
-    assert all(torch.equal(p, q) for p, q in zip(ga, gb))
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    if gf.split_plan(B, T, H, sms)[0] == 1:
+        assert all(torch.equal(p, q) for p, q in zip(ga, gb))
+    else:
+        # a split gradient call makes its own checkpoints segment by segment (folded summaries): the states agree with
+        # the forward pass's to fp32 rounding, the gradients to a bf16 ulp here and there
+        for p, q in zip(ga, gb):
+            assert orc.rel_l2(p.float().cpu().numpy(), q.float().cpu().numpy()) <= 2e-3
 
 
 def test_pair_against_the_oracle_with_mixed_chunks():
