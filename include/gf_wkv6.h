@@ -168,12 +168,12 @@ GF_API gf_status_t gf_wkv6_backward_c2(const void *r, const void *k, const void 
                                 void *workspace, size_t workspace_bytes, gf_stream_t stream);
 
 /* A training step's pair.  gf_wkv6_prefill_train / gf_wkv6_prefill_c2_train are gf_wkv6_prefill / gf_wkv6_prefill_c2
- * (same results, dense, one CTA per (sequence, head), never split) that also leave the state before every chunk of 64
+ * (same results, dense; calls with few units split their sequences as usual) that also leave the state before every chunk of 64
  * tokens and after the last one at the start of `workspace`, the gradient's workspace
  * (gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes).  gf_wkv6_backward_saved / gf_wkv6_backward_c2_saved are
  * gf_wkv6_backward / gf_wkv6_backward_c2 without their first launch: they take those states from the workspace, which
  * must still hold what the forward call of the SAME r,k,v,x,state_in wrote (the caller's responsibility; nothing
- * checks it).  One launch forward; two (one for the Finch-C2 form) backward. */
+ * checks it). */
 GF_API gf_status_t gf_wkv6_prefill_train(const void *r, const void *k, const void *v, const void *x, const float *u,
                                   const float *state_in, float *state_out, void *y, int B, int T, int H, int N,
                                   void *workspace, size_t workspace_bytes, gf_stream_t stream);

@@ -500,8 +500,10 @@ gf_status_t prefill_train(const void* r, const void* k, const void* v, const voi
     const size_t need = gf_wkv6_backward_bf16_workspace_bytes(B, T, H, N);
     if (need == 0) return GF_ERR_CUDA;
     if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
+    size_t sbytes = 0;
+    float* scratch = gf::backward_workspace_forward_scratch(static_cast<float*>(workspace), (long long)B * H, T, gf::sm_count(), &sbytes);
     const gf_status_t s = gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
-                                              (bf*)y, nullptr, B, T, (long long)B * T, H, st, &g_launches, nullptr, 0,
+                                              (bf*)y, nullptr, B, T, (long long)B * T, H, st, &g_launches, scratch, sbytes,
                                               (const bf*)u2, c2 ? 1 : 0, static_cast<float*>(workspace));
     if (s != GF_OK) return s;
     return launch_result();

@@ -930,6 +930,17 @@ inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
             (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
+// The part of the gradient's workspace that a training step's forward pass may use as its split scratch (the
+// token-by-token path's slots: idle until the gradient call).
+inline float* backward_workspace_forward_scratch(float* ws, long long units, int T, int n_sm, size_t* bytes)
+{
+    const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
+    int seg_chunks = 0;
+    const int nseg = backward_split(units, T, n_sm, &seg_chunks);
+    *bytes = (size_t)2 * n_sm * bc::FB_SLOT_FLOATS * sizeof(float);
+    return ws + (size_t)units * nck * 4096 + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
+}
+
 inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                     const __nv_bfloat16* x, const float* u, const float* state_in,
                                     const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,

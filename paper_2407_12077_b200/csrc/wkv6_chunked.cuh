@@ -637,7 +637,7 @@ __device__ __forceinline__ void exact_chunk(float* scr, const Params& p, int h, 
 // C2 = true: the Finch-C2 form (keys times one minus their decay, no bonus, optional second-value vector).
 // PERSIST = true: the CTA walks a stream of units (see Params::n_units); the producer warp leaves a descriptor per
 // chunk and two end markers, which every role passes down its own signalling path before it leaves.
-// CKPT = true (single-unit, unsplit launches of the prefill proper): the state before every chunk and after the last
+// CKPT = true (single-unit launches of the prefill proper, split or not): the state before every chunk and after the last
 // one is also left in Params::ckpt, for the gradient call that follows a training step's forward pass.
 template <bool SUMMARY, bool C2, bool PERSIST = false, bool CKPT = false>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -1070,7 +1070,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (CKPT && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
+        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
         if (SUMMARY && p.ckpt) {
             if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
                 store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
@@ -1589,7 +1589,7 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         !ck::make_map(&ty, y, total_rows, C, 16) || !ck::make_map(&tu2, u2 ? (const void*)u2 : (const void*)y, total_rows, C, 16))
         return GF_ERR_CUDA;
     int seg_chunks = 0, nseg = 1;
-    if (scratch && !ckpt) {                                   // packed calls split by max_seqlen: segments past a sequence's end are empty
+    if (scratch && !(ckpt && cu)) {                           // packed calls split by max_seqlen: segments past a sequence's end are empty
         size_t need = 0;
         nseg = choose_split(units, T, sm_count(), &seg_chunks, &need, scratch_bytes);   // (never splits with more units than half the SMs)
         if (nseg > 1 && units * nseg > 0x7fffffffLL) nseg = 1;
@@ -1598,11 +1598,17 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     if (ckpt) {
-        // a training step's forward pass (dense): one CTA per unit, unsplit, the chunk-start states kept for the gradient
+        // a training step's forward pass (dense): one CTA per unit and segment, the chunk-start states kept for the gradient
         if (cu) return GF_ERR_UNSUPPORTED;
+        if (nseg > 1) {
+            if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+            else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+            launches->fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+        }
         p.ckpt = ckpt;
-        if (c2) ck::wkv6_chunked_kernel<false, true, false, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-        else ck::wkv6_chunked_kernel<false, false, false, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        if (c2) ck::wkv6_chunked_kernel<false, true, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        else ck::wkv6_chunked_kernel<false, false, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }

@@ -24,11 +24,11 @@ def test_pair_is_bit_identical_to_the_separate_calls(B, T, H, c2):
     ws = torch.empty(gf.backward_workspace_bytes(B, T, H, 64), dtype=torch.uint8, device=DEV)
     y, s = gf.prefill_train(inp.r, inp.k, inp.v, inp.x, inp.u, ws, inp.state_in, c2=c2, u2=u2)
     if c2:
-        y0, s0 = gf.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in, split=False)
+        y0, s0 = gf.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in)
         ga = gf.backward_c2(inp.r, inp.k, inp.v, inp.x, dy, inp.state_in, dsT, workspace=ws, saved=True)
         gb = gf.backward_c2(inp.r, inp.k, inp.v, inp.x, dy, inp.state_in, dsT)
     else:
-        y0, s0 = gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in, split=False)
+        y0, s0 = gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
         ga = gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT, workspace=ws, saved=True)
         gb = gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT)
     gf.last_device_status()
