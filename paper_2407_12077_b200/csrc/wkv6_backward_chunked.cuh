@@ -34,7 +34,8 @@
 // Each group has its own input stage (x, v, dy and r, k by TMA, each part re-filled as soon as its tiles fall free),
 // operand tiles, tensor-memory columns (three accumulators that the second group of products reuses once the first
 // group's have been read) and barriers; the four staging tiles of the gradients lie over operand tiles that are dead
-// by the time they are written.  Thread 0 of a group issues its products and copies.  Sums along the tokens (the
+// by the time they are written.  One lane of a group issues its copies, two others (in other warps) its two groups of
+// products, so that no warp carries all the issuing.  Sums along the tokens (the
 // cumulative decay; the suffix sums of the decay gradient) run over lanes by shuffles and across the four row groups
 // through shared memory.  Waits are per thread and bounded; their outcome is made uniform over the group at its next
 // barrier, and the hand-over waits watch the CTA's abort word, so after a wait that ran out both groups leave.
@@ -445,7 +446,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         fence_proxy_async();
         tc_fence_before();
         const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
-        if (!unsafe && gt == 0) {
+        if (!unsafe && gt == 64) {
             // the products that need nothing but the inputs; the adjoint is not needed for R^^T dY either
             tc_fence_after();
             const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
@@ -723,7 +724,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             fence_proxy_async();
             tc_fence_before();
             if (!gbar_and(grp, ok)) { alive = false; break; }
-            if (gt == 0) {
+            if (gt == 160) {
                 tc_fence_after();
                 const uint64_t dR = smem_desc(t_rh), dK = smem_desc(t_kh), dV = smem_desc(tv), dY = smem_desc(tdy);
                 const uint64_t dS = smem_desc(t_sb), dG = smem_desc(t_gb), dP = smem_desc(t_pp), dD = smem_desc(t_dpp);
