@@ -143,7 +143,8 @@ GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
  * by token in fp32 instead, so any decay logit is accepted (x = +inf leaves dx undefined, as in the formula).
  * `workspace`: caller-owned DEVICE buffer of at least gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes, 16-byte
  * aligned (one 64x64 fp32 state per chunk and unit, plus 2 MiB per SM for the token-by-token path);
- * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  Enqueues three
+ * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  dstate_in must
+ * not be dstate_out (GF_ERR_INVALID_ARG).  Enqueues three
  * kernels on `stream` (five when B*H is less than half the SMs: the sequences are then cut into segments that run
  * side by side, as in the forward call), allocates nothing, does not synchronise; deterministic (no atomics).  A
  * device-side wait that runs out is reported by gf_wkv6_last_device_status as for the forward call. */

@@ -429,6 +429,8 @@ gf_status_t backward_bf16(const void* r, const void* k, const void* v, const voi
     for (const void* o : outs)
         for (const void* in : ins)
             if (o == in) return GF_ERR_INVALID_ARG;
+    // (a split call reads dstate_out in every segment's CTA and writes dstate_in from the first segment's: not in place)
+    if (dstate_in && dstate_in == dstate_out) return GF_ERR_INVALID_ARG;
     if ((long long)B * H > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
     if ((long long)B * T >= (1LL << 31) - 64) return GF_ERR_UNSUPPORTED;
     const size_t need = gf_wkv6_backward_bf16_workspace_bytes(B, T, H, N);

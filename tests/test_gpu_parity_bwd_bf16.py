@@ -215,6 +215,9 @@ def test_repeatable_and_argument_checks():
     bad = list(args); bad[8] = p(d.r)                                               # dr aliases r
     assert lib.gf_wkv6_backward(*bad, 2, 300, 2, 64, p(ws), ws.numel(), None) == 1
     assert lib.gf_wkv6_backward(*args, 2, 300, 2, 64, p(ws), ws.numel() - 16, None) == 4
+    ds = torch.zeros((2, 2, 64, 64), device=DEV)
+    inplace = list(args); inplace[7] = p(ds); inplace[13] = p(ds)                      # dstate_in is dstate_out
+    assert lib.gf_wkv6_backward(*inplace, 2, 300, 2, 64, p(ws), ws.numel(), None) == 1
     assert gf.launch_count() == before
     # no token: the adjoint passes through, no bonus gradient
     e = torch.empty((2, 0, 2, 64), device=DEV, dtype=torch.bfloat16)
