@@ -129,3 +129,25 @@ def test_heads_and_batch_entries_are_independent_and_du_sums_over_the_batch():
     # bonus-free recurrence: u = 0 removes the bonus terms (the paper's own r_t . wkv_t form) and du's drivers stay
     z = orc.backward(r, k, v, x, np.zeros_like(u), dy, s0, dsT)
     assert np.allclose(z[4], full[4], rtol=1e-13)      # du does not depend on u
+
+
+def test_against_reverse_mode_differentiation_of_the_definition_in_float64():
+    """The recurrence written out token by token in torch (float64) and differentiated by the library's reverse mode:
+    an independent route to every gradient at once (the oracle's adjoint recursion shares nothing with it)."""
+    import torch
+    B, T, H, N = 2, 9, 2, 5
+    r, k, v, x, u, s0, dy, dsT = _case(B, T, H, N, 21)
+    tr, tk, tv, tx, tu, ts0 = (torch.tensor(a.astype(np.float64), requires_grad=True) for a in (r, k, v, x, u, s0))
+    S = ts0
+    ys = []
+    for t in range(T):
+        w = torch.exp(-torch.exp(tx[:, t]))                                   # [B,H,N]
+        kv = tk[:, t].unsqueeze(-1) * tv[:, t].unsqueeze(-2)                   # [B,H,N,N]
+        ys.append(torch.einsum("bhi,bhij->bhj", tr[:, t], S + tu.unsqueeze(0).unsqueeze(-1) * kv))
+        S = w.unsqueeze(-1) * S + kv
+    y = torch.stack(ys, dim=1)
+    loss = (y * torch.tensor(dy)).sum() + (S * torch.tensor(dsT)).sum()
+    loss.backward()
+    got = orc.backward(r, k, v, x, u, dy, s0, dsT)
+    for name, a, b in zip(("dr", "dk", "dv", "dx", "du", "ds0"), got, (tr.grad, tk.grad, tv.grad, tx.grad, tu.grad, ts0.grad)):
+        assert np.allclose(a, b.numpy(), rtol=1e-11, atol=1e-12), name

@@ -132,3 +132,26 @@ def test_a_planted_mistake_fails():
     w = np.exp(-np.exp(X))
     wrong = (G * S0).sum(axis=1) * (-w * np.exp(X))      # the classic dx: forgets that k (1 - w) depends on x
     assert not np.allclose(dx.reshape(N), wrong, rtol=1e-3)
+
+
+def test_against_reverse_mode_differentiation_of_the_definition_in_float64():
+    """The Finch-C2 recurrence written out token by token in torch (float64) and differentiated by the library's
+    reverse mode; the second-value vector's gradient comes out as dy."""
+    import torch
+    B, T, H, N = 2, 9, 2, 5
+    r, k, v, x, s0, dy, dsT = _case(B, T, H, N, 22)
+    u2 = np.random.default_rng(23).normal(size=dy.shape).astype(np.float32)
+    tr, tk, tv, tx, ts0, tu2 = (torch.tensor(a.astype(np.float64), requires_grad=True) for a in (r, k, v, x, s0, u2))
+    S = ts0
+    ys = []
+    for t in range(T):
+        w = torch.exp(-torch.exp(tx[:, t]))
+        ys.append(torch.einsum("bhi,bhij->bhj", tr[:, t], S) + tu2[:, t])
+        S = w.unsqueeze(-1) * S + (tk[:, t] * (1 - w)).unsqueeze(-1) * tv[:, t].unsqueeze(-2)
+    y = torch.stack(ys, dim=1)
+    loss = (y * torch.tensor(dy)).sum() + (S * torch.tensor(dsT)).sum()
+    loss.backward()
+    got = orc.backward_c2(r, k, v, x, dy, s0, dsT)
+    for name, a, b in zip(("dr", "dk", "dv", "dx", "ds0"), got, (tr.grad, tk.grad, tv.grad, tx.grad, ts0.grad)):
+        assert np.allclose(a, b.numpy(), rtol=1e-11, atol=1e-12), name
+    assert np.allclose(tu2.grad.numpy(), dy, rtol=0, atol=0)
