@@ -422,18 +422,24 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             ld_tile(tr, moff, rv);
             ld_tile(tk, moff, kv);
             float b0 = 0.f, b1 = 0.f;
+            // (two-lane fp32 arithmetic on the pairs of neighbouring columns: half the multiply / add instructions)
 #pragma unroll
-            for (int n = 0; n < G_NB; ++n)
+            for (int n = 0; n < G_NB; ++n) {
+                const float2 u2 = (!C2 && !GSUM) ? ldsf2(sbase + GS_U + 4 * (cb + 8 * n)) : make_float2(0.f, 0.f);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (C2) kv[n][e] *= one_minus_ex2(lw2[n][e]);      // the key that enters the state
+                for (int h = 0; h < 2; ++h) {                          // h = 0: row R0, h = 1: row R1
+                    float2 rr = make_float2(rv[n][2 * h], rv[n][2 * h + 1]), kk = make_float2(kv[n][2 * h], kv[n][2 * h + 1]);
+                    const float2 aa = make_float2(a[n][2 * h], a[n][2 * h + 1]), ll = make_float2(lw2[n][2 * h], lw2[n][2 * h + 1]);
+                    if (C2) kk = mul2(kk, make_float2(one_minus_ex2(ll.x), one_minus_ex2(ll.y)));      // the key that enters the state
                     if (!C2 && !GSUM) {
-                        const float t = rv[n][e] * kv[n][e] * ldsf(sbase + GS_U + 4 * (cb + 8 * n + (e & 1)));
-                        if (e < 2) b0 += t; else b1 += t;
+                        const float2 t = mul2(mul2(rr, kk), u2);
+                        if (h == 0) b0 += t.x + t.y; else b1 += t.x + t.y;
                     }
-                    rv[n][e] *= ex2(a[n][e] - lw2[n][e]);
-                    kv[n][e] *= ex2(-a[n][e]);
+                    rr = mul2(rr, ex2_2(sub2(aa, ll)));
+                    kk = mul2(kk, make_float2(ex2(-aa.x), ex2(-aa.y)));
+                    rv[n][2 * h] = rr.x; rv[n][2 * h + 1] = rr.y; kv[n][2 * h] = kk.x; kv[n][2 * h + 1] = kk.y;
                 }
+            }
             st_tile(t_rh, moff, rv);
             if (!GSUM) st_tile(t_kh, moff, kv);
             if (!C2 && !GSUM) {
@@ -770,36 +776,54 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 ld_half(tk + moff[h2], kv);
                 ld_half(t_rh + moff[h2], hat);
                 tmem_ld_done();
+                // (two-lane fp32 arithmetic on the pairs of neighbouring columns)
 #pragma unroll
-                for (int n = 0; n < 2; ++n)
+                for (int n = 0; n < 2; ++n) {
+                    const int nn = 2 * h2 + n;
+                    const float2 u2 = C2 ? make_float2(0.f, 0.f) : ldsf2(sbase + GS_U + 4 * (cb + 8 * nn));
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int nn = 2 * h2 + n;
-                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
-                        o[n][e] = fmaf(uc * kv[n][e], pd, acc[n][e] * ex2(a[nn][e] - lw2[nn][e]));
-                        qv[nn][e] = acc[n][e] * hat[n][e];
-                        if (!C2) du_acc[nn][e & 1] = fmaf(rv[n][e] * kv[n][e], pd, du_acc[nn][e & 1]);
+                    for (int h = 0; h < 2; ++h) {
+                        const float2 pd = h ? make_float2(pd1, pd1) : make_float2(pd0, pd0);
+                        const float2 ac = make_float2(acc[n][2 * h], acc[n][2 * h + 1]), kk = make_float2(kv[n][2 * h], kv[n][2 * h + 1]);
+                        const float2 sr = ex2_2(sub2(make_float2(a[nn][2 * h], a[nn][2 * h + 1]), make_float2(lw2[nn][2 * h], lw2[nn][2 * h + 1])));
+                        const float2 oo = C2 ? mul2(ac, sr) : fma2(mul2(u2, kk), pd, mul2(ac, sr));
+                        const float2 qq = mul2(ac, make_float2(hat[n][2 * h], hat[n][2 * h + 1]));
+                        o[n][2 * h] = oo.x; o[n][2 * h + 1] = oo.y;
+                        qv[nn][2 * h] = qq.x; qv[nn][2 * h + 1] = qq.y;
+                        if (!C2) {
+                            const float2 dd = fma2(mul2(make_float2(rv[n][2 * h], rv[n][2 * h + 1]), kk), pd, make_float2(du_acc[nn][0], du_acc[nn][1]));
+                            du_acc[nn][0] = dd.x; du_acc[nn][1] = dd.y;
+                        }
                     }
+                }
                 tmem_ld_16x16_async2(tacc + GT_DK + 16 * h2, acc);
                 ld_half(t_kh + moff[h2], hat);
                 tmem_ld_done();
                 st_half(o_dr + moff[h2], o);
 #pragma unroll
-                for (int n = 0; n < 2; ++n)
+                for (int n = 0; n < 2; ++n) {
+                    const int nn = 2 * h2 + n;
+                    const float2 u2 = C2 ? make_float2(0.f, 0.f) : ldsf2(sbase + GS_U + 4 * (cb + 8 * nn));
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int nn = 2 * h2 + n;
-                        const float pd = e < 2 ? pd0 : pd1, uc = ldsf(sbase + GS_U + 4 * (cb + 8 * nn + (e & 1)));
-                        o[n][e] = fmaf(uc * rv[n][e], pd, acc[n][e] * ex2(-a[nn][e]));
-                        z[nn][e] = qv[nn][e] - acc[n][e] * hat[n][e];
+                    for (int h = 0; h < 2; ++h) {
+                        const float2 pd = h ? make_float2(pd1, pd1) : make_float2(pd0, pd0);
+                        const float2 ac = make_float2(acc[n][2 * h], acc[n][2 * h + 1]);
+                        const float2 sk = make_float2(ex2(-a[nn][2 * h]), ex2(-a[nn][2 * h + 1]));
+                        float2 oo = C2 ? mul2(ac, sk) : fma2(mul2(u2, make_float2(rv[n][2 * h], rv[n][2 * h + 1])), pd, mul2(ac, sk));
+                        const float2 zz = sub2(make_float2(qv[nn][2 * h], qv[nn][2 * h + 1]), mul2(ac, make_float2(hat[n][2 * h], hat[n][2 * h + 1])));
+                        z[nn][2 * h] = zz.x; z[nn][2 * h + 1] = zz.y;
                         if (C2) {
-                            // o is the gradient of k (1 - w): the key gets (1 - w) of it, and the decay logit its
+                            // oo is the gradient of k (1 - w): the key gets (1 - w) of it, and the decay logit its
                             // share through the key factor, folded into the term that leaves the suffix sums
-                            const float omw = one_minus_ex2(lw2[nn][e]);
-                            qv[nn][e] = fmaf(o[n][e] * kv[n][e], 1.f - omw, qv[nn][e]);
-                            o[n][e] *= omw;
+                            const float2 omw = make_float2(one_minus_ex2(lw2[nn][2 * h]), one_minus_ex2(lw2[nn][2 * h + 1]));
+                            const float2 qq = fma2(mul2(oo, make_float2(kv[n][2 * h], kv[n][2 * h + 1])), sub2(make_float2(1.f, 1.f), omw),
+                                                   make_float2(qv[nn][2 * h], qv[nn][2 * h + 1]));
+                            qv[nn][2 * h] = qq.x; qv[nn][2 * h + 1] = qq.y;
+                            oo = mul2(oo, omw);
                         }
+                        o[n][2 * h] = oo.x; o[n][2 * h + 1] = oo.y;
                     }
+                }
                 st_half(o_dk + moff[h2], o);
             }
             // dV: every product of the chunk has completed, so x, v, dy can take the group's next chunk
@@ -824,8 +848,11 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
 #pragma unroll
                 for (int o = 0; o < G_NSLAB; ++o) { const float2 ev = ldsf2(gbase + GO_EP + 4 * (o * 64 + cb + 8 * n)); E0 += ev.x; E1 += ev.y; }
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    z[n][e] = ((e & 1 ? E1 : E0) + z[n][e] - qv[n][e]) * (lw2[n][e] * LN2);
+                for (int h = 0; h < 2; ++h) {
+                    const float2 dl = sub2(add2(make_float2(E0, E1), make_float2(z[n][2 * h], z[n][2 * h + 1])), make_float2(qv[n][2 * h], qv[n][2 * h + 1]));
+                    const float2 dx2 = mul2(dl, mul2(make_float2(lw2[n][2 * h], lw2[n][2 * h + 1]), make_float2(LN2, LN2)));
+                    z[n][2 * h] = dx2.x; z[n][2 * h + 1] = dx2.y;
+                }
             }
             st_tile(o_dx, moff, z);
         }
