@@ -651,8 +651,9 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 float gh[G_NB][4];
 #pragma unroll
                 for (int n = 0; n < G_NB; ++n) {
-                    gh[n][0] = d_lo * G[n][0]; gh[n][1] = d_lo * G[n][1];
-                    gh[n][2] = d_hi * G[n][2]; gh[n][3] = d_hi * G[n][3];
+                    const float2 lo = mul2(make_float2(d_lo, d_lo), make_float2(G[n][0], G[n][1]));
+                    const float2 hi = mul2(make_float2(d_hi, d_hi), make_float2(G[n][2], G[n][3]));
+                    gh[n][0] = lo.x; gh[n][1] = lo.y; gh[n][2] = hi.x; gh[n][3] = hi.y;
                 }
                 st_tile(t_gb, moff, gh);
             }
@@ -665,8 +666,9 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 tmem_ld_done();
 #pragma unroll
                 for (int n = 0; n < G_NB; ++n) {
-                    G[n][0] = fmaf(d_lo, G[n][0], dg[n][0]); G[n][1] = fmaf(d_lo, G[n][1], dg[n][1]);
-                    G[n][2] = fmaf(d_hi, G[n][2], dg[n][2]); G[n][3] = fmaf(d_hi, G[n][3], dg[n][3]);
+                    const float2 lo = fma2(make_float2(d_lo, d_lo), make_float2(G[n][0], G[n][1]), make_float2(dg[n][0], dg[n][1]));
+                    const float2 hi = fma2(make_float2(d_hi, d_hi), make_float2(G[n][2], G[n][3]), make_float2(dg[n][2], dg[n][3]));
+                    G[n][0] = lo.x; G[n][1] = lo.y; G[n][2] = hi.x; G[n][3] = hi.y;
                 }
             }
             if (it + 1 < nit) {
