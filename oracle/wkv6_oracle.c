@@ -479,3 +479,45 @@ void wkv6_oracle_backward_c2(const float *r, const float *k, const float *v, con
                              ds_0 ? ds_0 + soff : NULL, T, N, C);
         }
 }
+
+/* Packed variable-length batches of the two gradients: rows cu_seqlens[s] .. cu_seqlens[s+1]-1 of the
+ * [total_T][H][N] tensors form sequence s (wkv6_oracle_prefill_varlen's layout), states and their gradients
+ * are [S][H][N][N], du_s is [S][H][N] (per sequence; the caller sums over s).  Every (sequence, head) unit is
+ * the dense unit gradient on its own rows: the recurrence never crosses a sequence boundary, so neither does
+ * its adjoint.  A sequence without tokens hands its incoming state gradient through (dS_0 = dS_T).
+ * Pinned in tests/test_oracle_pins_bwd_varlen.py. */
+void wkv6_oracle_backward_varlen(const float *r, const float *k, const float *v, const float *x, const float *u,
+                                 const float *state_in, const double *dy, const double *ds_T, double *dr, double *dk,
+                                 double *dv, double *dx, double *du_s, double *ds_0, const int32_t *cu_seqlens,
+                                 long S, long H, long N)
+{
+    const long C = H * N;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (long s = 0; s < S; ++s)
+        for (long h = 0; h < H; ++h) {
+            const long t0 = cu_seqlens[s], len = cu_seqlens[s + 1] - cu_seqlens[s];
+            const size_t off = (size_t)t0 * C + (size_t)h * N;
+            const size_t soff = ((size_t)s * H + h) * N * N;
+            unit_backward(r + off, k + off, v + off, x + off, u + h * N, state_in ? state_in + soff : NULL,
+                          dy + off, ds_T ? ds_T + soff : NULL, dr + off, dk + off, dv + off, dx + off,
+                          du_s + ((size_t)s * H + h) * N, ds_0 ? ds_0 + soff : NULL, len, N, C);
+        }
+}
+
+void wkv6_oracle_backward_c2_varlen(const float *r, const float *k, const float *v, const float *x,
+                                    const float *state_in, const double *dy, const double *ds_T, double *dr,
+                                    double *dk, double *dv, double *dx, double *ds_0, const int32_t *cu_seqlens,
+                                    long S, long H, long N)
+{
+    const long C = H * N;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (long s = 0; s < S; ++s)
+        for (long h = 0; h < H; ++h) {
+            const long t0 = cu_seqlens[s], len = cu_seqlens[s + 1] - cu_seqlens[s];
+            const size_t off = (size_t)t0 * C + (size_t)h * N;
+            const size_t soff = ((size_t)s * H + h) * N * N;
+            unit_backward_c2(r + off, k + off, v + off, x + off, state_in ? state_in + soff : NULL, dy + off,
+                             ds_T ? ds_T + soff : NULL, dr + off, dk + off, dv + off, dx + off,
+                             ds_0 ? ds_0 + soff : NULL, len, N, C);
+        }
+}

@@ -280,6 +280,58 @@ def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None):
     return outs[0], outs[1], outs[2], outs[3], ds0
 
 
+def _cu(cu_seqlens, total_T):
+    if hasattr(cu_seqlens, "detach"):
+        cu_seqlens = cu_seqlens.detach().cpu().numpy()
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    assert cu[0] == 0 and cu[-1] == total_T and np.all(np.diff(cu) >= 0)
+    return cu
+
+
+def backward_varlen(r, k, v, x, u, dy, cu_seqlens, state_in=None, dstate_out=None):
+    """Gradient of prefill_varlen(): r,k,v,x,dy [total_T,H,N], cu_seqlens int32 [S+1], state_in / dstate_out [S,H,N,N]
+    or None (zero).  Returns (dr, dk, dv, dx [total_T,H,N], du [H,N] summed over the sequences, dstate_in [S,H,N,N])
+    in float64."""
+    lib = _load()
+    r, k, v, x, u, state_in = _f32(r), _f32(k), _f32(v), _f32(x), _f32(u), _f32(state_in)
+    total_T, H, N = r.shape
+    cu = _cu(cu_seqlens, total_T)
+    S = cu.shape[0] - 1
+    dy = _f64(dy, (total_T, H, N))
+    dsT = _f64(dstate_out, (S, H, N, N)) if dstate_out is not None else None
+    outs = [np.zeros((total_T, H, N), dtype=np.float64) for _ in range(4)]
+    du_s = np.zeros((S, H, N), dtype=np.float64)
+    ds0 = np.zeros((S, H, N, N), dtype=np.float64)
+    f, c = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_backward_varlen.restype = None
+    lib.wkv6_oracle_backward_varlen(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(u, f), _p(state_in, f), _p(dy, c),
+                                    _p(dsT, c), _p(outs[0], c), _p(outs[1], c), _p(outs[2], c), _p(outs[3], c),
+                                    _p(du_s, c), _p(ds0, c), cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                    ctypes.c_long(S), ctypes.c_long(H), ctypes.c_long(N))
+    return outs[0], outs[1], outs[2], outs[3], du_s.sum(axis=0), ds0
+
+
+def backward_c2_varlen(r, k, v, x, dy, cu_seqlens, state_in=None, dstate_out=None):
+    """Gradient of the Finch-C2 form over a packed batch (layouts as backward_varlen; no bonus, so no du).  Returns
+    (dr, dk, dv, dx [total_T,H,N], dstate_in [S,H,N,N]) in float64."""
+    lib = _load()
+    r, k, v, x, state_in = _f32(r), _f32(k), _f32(v), _f32(x), _f32(state_in)
+    total_T, H, N = r.shape
+    cu = _cu(cu_seqlens, total_T)
+    S = cu.shape[0] - 1
+    dy = _f64(dy, (total_T, H, N))
+    dsT = _f64(dstate_out, (S, H, N, N)) if dstate_out is not None else None
+    outs = [np.zeros((total_T, H, N), dtype=np.float64) for _ in range(4)]
+    ds0 = np.zeros((S, H, N, N), dtype=np.float64)
+    f, c = ctypes.c_float, ctypes.c_double
+    lib.wkv6_oracle_backward_c2_varlen.restype = None
+    lib.wkv6_oracle_backward_c2_varlen(_p(r, f), _p(k, f), _p(v, f), _p(x, f), _p(state_in, f), _p(dy, c), _p(dsT, c),
+                                       _p(outs[0], c), _p(outs[1], c), _p(outs[2], c), _p(outs[3], c), _p(ds0, c),
+                                       cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                       ctypes.c_long(S), ctypes.c_long(H), ctypes.c_long(N))
+    return outs[0], outs[1], outs[2], outs[3], ds0
+
+
 def rel_l2(a, b) -> float:
     """||a - b||_2 / ||b||_2 in float64 (b is the reference)."""
     a = np.asarray(a, dtype=np.float64).ravel()
