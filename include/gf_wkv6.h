@@ -191,6 +191,30 @@ GF_API gf_status_t gf_wkv6_backward_c2_saved(const void *r, const void *k, const
                                       void *dk, void *dv, void *dx, float *dstate_in, int B, int T, int H,
                                       int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
 
+/* Gradients of the packed variable-length prefill (gf_wkv6_prefill_varlen / gf_wkv6_prefill_varlen_c2; bf16 tensors,
+ * fp32 states): the adjoint recursion of gf_wkv6_backward / gf_wkv6_backward_c2 run per (sequence, head) over the
+ * sequence's own rows (the wkv_t recurrence never crosses a sequence boundary, so neither does its adjoint).  r, k, v,
+ * x, dy and the four gradients are packed [total_T][H][N] bf16; cu_seqlens is a DEVICE int32 array of S+1
+ * non-decreasing entries with cu_seqlens[0] = 0 and cu_seqlens[S] = total_T (not read on the host); max_seqlen an
+ * upper bound on any sequence length; state_in / dstate_out (NULL: zero) and dstate_in (NULL: not written) are
+ * [S][H][N][N] fp32; du [H][N] fp32 is summed over the sequences in index order.  A sequence without tokens hands its
+ * state gradient through.  `workspace`: caller-owned DEVICE buffer of at least
+ * gf_wkv6_backward_varlen_workspace_bytes(S,total_T,H,N) bytes, 16-byte aligned (H * (total_T / 64 + 2 S) states of
+ * 64x64 fp32, plus 2 MiB per SM); GF_ERR_WORKSPACE if absent or too small.  One CTA per (sequence, head), never
+ * split: three kernels on `stream` (two for the Finch-C2 form), nothing allocated, no synchronisation, deterministic.
+ * Other statuses as gf_wkv6_backward (dstate_in must not be dstate_out; total_T >= 2^31 - 64 or N != 64 unsupported). */
+GF_API gf_status_t gf_wkv6_backward_varlen(const void *r, const void *k, const void *v, const void *x, const float *u,
+                                    const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                                    void *dk, void *dv, void *dx, float *du, float *dstate_in,
+                                    const int32_t *cu_seqlens, int S, int total_T, int max_seqlen, int H, int N,
+                                    void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_backward_varlen_c2(const void *r, const void *k, const void *v, const void *x,
+                                       const float *state_in, const void *dy, const float *dstate_out, void *dr,
+                                       void *dk, void *dv, void *dx, float *dstate_in, const int32_t *cu_seqlens,
+                                       int S, int total_T, int max_seqlen, int H, int N, void *workspace,
+                                       size_t workspace_bytes, gf_stream_t stream);
+GF_API size_t gf_wkv6_backward_varlen_workspace_bytes(int S, int total_T, int H, int N);
+
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a

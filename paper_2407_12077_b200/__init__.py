@@ -37,6 +37,9 @@ _SIGNATURES = {
     "gf_wkv6_backward": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_bf16_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_backward_c2": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_varlen": (_i, [_vp] * 15 + [_i] * 5 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_varlen_c2": (_i, [_vp] * 13 + [_i] * 5 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_varlen_workspace_bytes": (_sz, [_i] * 4),
     "gf_wkv6_backward_saved": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_c2_saved": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_prefill_train": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
@@ -277,6 +280,34 @@ def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True
         fn = "gf_wkv6_backward_c2_saved" if saved else "gf_wkv6_backward_c2"
         _check(getattr(lib, fn)(*args, B, T, H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)), fn)
     return dr, dk, dv, dx, ds0
+
+
+def backward_varlen(r, k, v, x, u, dy, cu_seqlens, max_seqlen, state_in=None, dstate_out=None, want_dstate=True,
+                    stream=None, workspace=None, c2=False):
+    """gf_wkv6_backward_varlen / gf_wkv6_backward_varlen_c2: gradient of the packed prefill (bf16 tensors).  r,k,v,x,dy:
+    [total_T,H,N]; cu_seqlens: int32 CUDA [S+1]; u: [H,N] fp32 (ignored with c2=True); state_in / dstate_out:
+    [S,H,N,N] fp32 or None.  Returns (dr, dk, dv, dx, du, dstate_in), du None with c2=True."""
+    lib = load_library()
+    total_T, H, N = r.shape
+    S = cu_seqlens.numel() - 1
+    bf, f32 = torch.bfloat16, torch.float32
+    dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
+    du = None if c2 else torch.empty((H, N), device=r.device, dtype=f32)
+    ds0 = torch.empty((S, H, N, N), device=r.device, dtype=f32) if want_dstate else None
+    with torch.cuda.device(r.device):
+        nbytes = int(lib.gf_wkv6_backward_varlen_workspace_bytes(S, total_T, H, N))
+        ws = workspace if workspace is not None and workspace.numel() >= nbytes else torch.empty(max(nbytes, 16), dtype=torch.uint8, device=r.device)
+        args = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape)]
+        if not c2:
+            args.append(_dev(u, "u", f32, (H, N)))
+        args += [_dev(state_in, "state_in", f32, (S, H, N, N)), _dev(dy, "dy", bf, r.shape),
+                 _dev(dstate_out, "dstate_out", f32, (S, H, N, N)), _dev(dr, "dr"), _dev(dk, "dk"), _dev(dv, "dv"), _dev(dx, "dx")]
+        if not c2:
+            args.append(_dev(du, "du"))
+        args += [_dev(ds0, "dstate_in"), _dev(cu_seqlens, "cu_seqlens", torch.int32)]
+        fn = "gf_wkv6_backward_varlen_c2" if c2 else "gf_wkv6_backward_varlen"
+        _check(getattr(lib, fn)(*args, S, total_T, int(max_seqlen), H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)), fn)
+    return dr, dk, dv, dx, du, ds0
 
 
 def prefill_train(r, k, v, x, u, workspace, state_in=None, c2=False, u2=None, stream=None):

@@ -480,6 +480,81 @@ gf_status_t gf_wkv6_backward_c2_saved(const void* r, const void* k, const void* 
                          workspace, workspace_bytes, stream, true, true);
 }
 
+size_t gf_wkv6_backward_varlen_workspace_bytes(int S, int total_T, int H, int N)
+{
+    if (S <= 0 || total_T < 0 || H <= 0 || N != 64) return 0;
+    const int n_sm = gf::sm_count();
+    if (n_sm <= 0) return 0;
+    return gf::chunked_backward_varlen_workspace_bytes(S, total_T, H, n_sm);
+}
+
+namespace {
+// bf16 gradient over packed sequences, classic (u, du given) or Finch-C2 form (c2: no bonus)
+gf_status_t backward_varlen_bf16(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                 const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
+                                 void* dv, void* dx, float* du, float* dstate_in, const int32_t* cu_seqlens, int S,
+                                 int total_T, int max_seqlen, int H, int N, void* workspace, size_t workspace_bytes,
+                                 gf_stream_t stream, bool c2)
+{
+    using bf = __nv_bfloat16;
+    if (S < 0 || total_T < 0 || max_seqlen < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (S == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t sbytes = (size_t)S * H * 64 * 64 * sizeof(float);
+    if (dstate_in && dstate_in == dstate_out) return GF_ERR_INVALID_ARG;
+    if (total_T == 0) {
+        // no token in any sequence: the state adjoints pass through and the bonus gets no gradient
+        if (misaligned(dstate_out) || misaligned(dstate_in) || misaligned(du)) return GF_ERR_INVALID_ARG;
+        cudaError_t e = cudaSuccess;
+        if (dstate_in && !dstate_out) e = cudaMemsetAsync(dstate_in, 0, sbytes, st);
+        else if (dstate_in) e = cudaMemcpyAsync(dstate_in, dstate_out, sbytes, cudaMemcpyDeviceToDevice, st);
+        if (e == cudaSuccess && du) e = cudaMemsetAsync(du, 0, (size_t)H * 64 * sizeof(float), st);
+        return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
+    }
+    if (!r || !k || !v || !x || !dy || !dr || !dk || !dv || !dx || !cu_seqlens || (!c2 && (!u || !du))) return GF_ERR_INVALID_ARG;
+    if (max_seqlen == 0) return GF_ERR_INVALID_ARG;                  // (tokens exist, so some sequence is longer)
+    const void* ptrs[] = {r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, workspace};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(cu_seqlens) % alignof(int32_t)) return GF_ERR_INVALID_ARG;
+    const void* ins[] = {r, k, v, x, dy};
+    const void* outs[] = {dr, dk, dv, dx};
+    for (const void* o : outs)
+        for (const void* in : ins)
+            if (o == in) return GF_ERR_INVALID_ARG;
+    if ((long long)S * H > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    if ((long long)total_T >= (1LL << 31) - 64) return GF_ERR_UNSUPPORTED;
+    const size_t need = gf_wkv6_backward_varlen_workspace_bytes(S, total_T, H, N);
+    if (need == 0) return GF_ERR_CUDA;
+    if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
+    const gf_status_t s = gf::chunked_backward((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, (const bf*)dy,
+                                               dstate_out, (bf*)dr, (bf*)dk, (bf*)dv, (bf*)dx, du, dstate_in, S, max_seqlen, H,
+                                               static_cast<float*>(workspace), st, &g_launches, c2, false, cu_seqlens, total_T);
+    if (s != GF_OK) return s;
+    return launch_result();
+}
+}  // namespace
+
+gf_status_t gf_wkv6_backward_varlen(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                    const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
+                                    void* dv, void* dx, float* du, float* dstate_in, const int32_t* cu_seqlens, int S,
+                                    int total_T, int max_seqlen, int H, int N, void* workspace, size_t workspace_bytes,
+                                    gf_stream_t stream)
+{
+    return backward_varlen_bf16(r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, cu_seqlens, S,
+                                total_T, max_seqlen, H, N, workspace, workspace_bytes, stream, false);
+}
+
+gf_status_t gf_wkv6_backward_varlen_c2(const void* r, const void* k, const void* v, const void* x, const float* state_in,
+                                       const void* dy, const float* dstate_out, void* dr, void* dk, void* dv, void* dx,
+                                       float* dstate_in, const int32_t* cu_seqlens, int S, int total_T, int max_seqlen,
+                                       int H, int N, void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_varlen_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in,
+                                cu_seqlens, S, total_T, max_seqlen, H, N, workspace, workspace_bytes, stream, true);
+}
+
 namespace {
 // forward pass of a training step: the prefill that also leaves its chunk-start states in the gradient's workspace
 gf_status_t prefill_train(const void* r, const void* k, const void* v, const void* x, const float* u, const void* u2,

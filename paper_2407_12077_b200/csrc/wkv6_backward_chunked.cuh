@@ -71,6 +71,11 @@ struct BParams {
     const float* gsum;
     float* gsum_out;             // summary variant: where the summaries go (same layout)
     int nseg, seg_chunks;
+    // Packed sequences (never split): rows cu[s] .. cu[s+1]-1 of the [rows][H*64] tensors form sequence s, T is unused,
+    // and the checkpoints are [H][ckpt_slots][64][64] with sequence s of head h from slot cu[s] / 64 + 2 s on.
+    // NULL: dense.
+    const int32_t* cu;
+    long long ckpt_slots;
 };
 constexpr int GSUM_FLOATS = 64 + 64 * 64;
 
@@ -262,11 +267,11 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     // summary variant: segments 1 .. nseg-1 of every unit; else every segment
     const int gsegs = GSUM ? p.nseg - 1 : p.nseg;
     const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0), seq = unit / p.H, h = unit % p.H;
-    const int T = p.T, nchunks = (T + L - 1) / L;
+    const int T = p.cu ? p.cu[seq + 1] - p.cu[seq] : p.T, nchunks = (T + L - 1) / L;
     const int c_lo = p.nseg > 1 ? min(nchunks, seg * p.seg_chunks) : 0;                      // this CTA's chunks: c_lo .. c_hi-1,
     const int c_hi = (p.nseg > 1 && seg < p.nseg - 1) ? min(nchunks, c_lo + p.seg_chunks) : nchunks;   // walked from the last
     const int nit = c_hi - c_lo;
-    const long long row0 = (long long)seq * T;
+    const long long row0 = p.cu ? (long long)p.cu[seq] : (long long)seq * T;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
@@ -355,7 +360,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     };
 
-    const float* ck_unit = p.ckpt + (size_t)unit * (nchunks + 1) * 4096;
+    const float* ck_unit = p.ckpt + (p.cu ? (size_t)h * p.ckpt_slots + (size_t)(p.cu[seq] >> 6) + 2 * (size_t)seq
+                                         : (size_t)unit * (nchunks + 1)) * 4096;
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
@@ -883,6 +889,16 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     }
 
+    if (!GSUM && nit == 0 && seg == 0 && grp == 0 && p.dstate_in) {
+        // a sequence without tokens hands the state's gradient through
+        float G[G_NB][4];
+        if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
+        else {
+#pragma unroll
+            for (int n = 0; n < G_NB; ++n) G[n][0] = G[n][1] = G[n][2] = G[n][3] = 0.f;
+        }
+        store_f32_block(p.dstate_in + (size_t)unit * 4096, G);
+    }
     // ---- the bonus gradient of this unit: over the lanes' rows, the row groups and the two groups, in a fixed order
     if (!alive && gt == 0) sts32(abort_flag, 1u);    // (the other group's waits see it)
     if (GSUM && cx == 0 && q == 0) { stsf(gbase + GO_REDV + 4 * R0, dprod_lo); stsf(gbase + GO_REDV + 4 * R1, dprod_hi); }
@@ -960,6 +976,13 @@ inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
             (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
+// The same for packed sequences (never split): checkpoints in the packed layout, [H][total_rows / 64 + 2 S] states.
+inline size_t chunked_backward_varlen_workspace_bytes(long long n_seq, long long total_rows, int H, int n_sm)
+{
+    const size_t slots = (size_t)(total_rows / ck::L + 2 * n_seq);
+    return ((size_t)H * slots * 4096 + (size_t)n_seq * H * 64 + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+}
+
 // The part of the gradient's workspace that a training step's forward pass may use as its split scratch (the
 // token-by-token path's slots: idle until the gradient call).
 inline float* backward_workspace_forward_scratch(float* ws, long long units, int T, int n_sm, size_t* bytes)
@@ -976,9 +999,11 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
                                     const __nv_bfloat16* dy, const float* dstate_out, __nv_bfloat16* dr,
                                     __nv_bfloat16* dk, __nv_bfloat16* dv, __nv_bfloat16* dx, float* du, float* dstate_in,
                                     int B, int T, int H, float* ws, cudaStream_t st, std::atomic<uint64_t>* launches,
-                                    bool c2 = false, bool ckpt_saved = false)
+                                    bool c2 = false, bool ckpt_saved = false, const int32_t* cu = nullptr,
+                                    long long packed_rows = 0)
 {
-    const long long units = (long long)B * H, rows = (long long)B * T;
+    // packed sequences: cu = device cu_seqlens of B sequences over packed_rows rows, T = max_seqlen; never split
+    const long long units = (long long)B * H, rows = cu ? packed_rows : (long long)B * T;
     const int n_sm = sm_count();
     if (n_sm <= 0) return GF_ERR_CUDA;
     static PerDeviceFlag attr_set;
@@ -993,15 +1018,16 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     }
     const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
     int seg_chunks = 0;
-    int nseg = backward_split(units, T, n_sm, &seg_chunks);
+    int nseg = cu ? 1 : backward_split(units, T, n_sm, &seg_chunks);
     if (units * nseg > 0x7fffffffLL) nseg = 1;
+    const long long ckpt_slots = cu ? rows / ck::L + 2LL * B : 0;
     float* ckpt = ws;
-    float* du_part = ckpt + (size_t)units * nck * 4096;
+    float* du_part = ckpt + (cu ? (size_t)H * ckpt_slots : (size_t)units * nck) * 4096;
     float* gsum = du_part + (size_t)units * nseg * 64;
     float* fb = gsum + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
     if (!ckpt_saved) {                               // (else the forward pass of the training step left them there)
         // (split calls: the forward summaries borrow the buffer of the adjoint's, which are written after them)
-        const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0, gsum, nseg, seg_chunks);
+        const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0, gsum, nseg, seg_chunks, cu, rows);
         if (s != GF_OK) return s;
     }
     const long long C = (long long)H * 64;
@@ -1011,7 +1037,7 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
         return GF_ERR_CUDA;
     bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
-                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks};
+                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks, cu, ckpt_slots};
     if (nseg > 1) {
         // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
         bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);

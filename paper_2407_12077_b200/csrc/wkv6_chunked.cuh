@@ -481,7 +481,11 @@ struct Params {
     // the summaries of the segments before its own (nseg > 1: a plain summary launch has left them in `summaries`) and
     // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32, dense
     // sequences) instead of a summary.  The prefill proper fills it too in its CKPT instantiations.  NULL: none.
+    // Packed sequences (never split here): [H][ckpt_slots][64][64], sequence s of head h from slot
+    // cu_seqlens[s] / 64 + 2 s on (its chunks + 1 states fit before the next sequence's first slot), with
+    // ckpt_slots = total_T / 64 + 2 S.
     float* ckpt;
+    long long ckpt_slots;
 };
 constexpr int SUMMARY_FLOATS = 64 + 64 * 64;
 
@@ -675,6 +679,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         len = (seg == p.nseg - 1) ? len - first : min(len - first, p.seg_chunks * L);
     }
     const int nchunks = PERSIST ? 0 : (len + L - 1) / L;
+    // checkpoint slots of this unit: the first one, and how many chunks the whole sequence has
+    auto ckpt_first = [&]() -> size_t {
+        return p.cu_seqlens ? (size_t)h * p.ckpt_slots + (size_t)(p.cu_seqlens[seq] >> 6) + 2 * (size_t)seq
+                            : (size_t)unit * ((p.T + L - 1) / L + 1);
+    };
+    auto ckpt_chunks = [&]() -> int { return p.cu_seqlens ? nchunks : (p.T + L - 1) / L; };
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     static_assert(!(PERSIST && SUMMARY), "the summary pass is a single-unit launch");
@@ -977,7 +987,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
             if (CKPT || (SUMMARY && p.ckpt))         // the state before chunk c of the segment (dense sequences: T / 64 + 1 states per unit)
-                store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + seg * p.seg_chunks + c) * 4096);
+                store_to(p.ckpt + (ckpt_first() + seg * p.seg_chunks + c) * 4096);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1070,10 +1080,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
+        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + (ckpt_first() + ckpt_chunks()) * 4096);
         if (SUMMARY && p.ckpt) {
             if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
-                store_to(p.ckpt + ((size_t)unit * ((p.T + L - 1) / L + 1) + (p.T + L - 1) / L) * 4096);
+                store_to(p.ckpt + (ckpt_first() + ckpt_chunks()) * 4096);
         } else if (SUMMARY) {
             if (!lds32(abort_flag)) {
                 float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
@@ -1598,8 +1608,8 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
     if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     if (ckpt) {
-        // a training step's forward pass (dense): one CTA per unit and segment, the chunk-start states kept for the gradient
-        if (cu) return GF_ERR_UNSUPPORTED;
+        // a training step's forward pass: one CTA per unit and segment, the chunk-start states kept for the gradient
+        p.ckpt_slots = cu ? total_rows / ck::L + 2LL * n_seq : 0;
         if (nseg > 1) {
             if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
             else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
@@ -1697,9 +1707,13 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
 inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x,
                                        const float* state_in, float* ckpt, int n_seq, int T, int H, cudaStream_t st,
                                        std::atomic<uint64_t>* launches, int c2 = 0, float* summaries = nullptr,
-                                       int nseg = 1, int seg_chunks = 0)
+                                       int nseg = 1, int seg_chunks = 0, const int32_t* cu = nullptr,
+                                       long long packed_rows = 0)
 {
-    const long long units = (long long)n_seq * H, total_rows = (long long)n_seq * T;
+    // packed sequences (cu: device cu_seqlens of n_seq sequences over packed_rows rows, T = max_seqlen): never split,
+    // checkpoints in the packed layout (Params::ckpt)
+    const long long units = (long long)n_seq * H, total_rows = cu ? packed_rows : (long long)n_seq * T;
+    if (cu) summaries = nullptr;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
     if (total_rows >= (1LL << 31) - 64 || !ck::encode_fn()) return GF_ERR_UNSUPPORTED;
     if (!chunked_kernel_attributes()) return GF_ERR_CUDA;
@@ -1709,8 +1723,9 @@ inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat
         !ck::make_map(&tx, x, total_rows, C, 64) || !ck::make_map(&tdummy, k, total_rows, C, 16))
         return GF_ERR_CUDA;
     if (!summaries || nseg < 2) { nseg = 1; seg_chunks = (T + ck::L - 1) / ck::L; }
-    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, nullptr, T, H, summaries, seg_chunks, nseg, nullptr, c2};
+    ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, cu, T, H, summaries, seg_chunks, nseg, nullptr, c2};
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
+    p.ckpt_slots = cu ? total_rows / ck::L + 2LL * n_seq : 0;
     if (nseg > 1) {
         // few units: the segments' summaries first (every segment but the last, from a zero state), then every segment
         // side by side from its folded start state, this time keeping the states
