@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "prefill_train", "backward_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "prefill_train", "backward_workspace_bytes", "backward_varlen", "backward_varlen_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -334,6 +334,11 @@ def backward_workspace_bytes(B, T, H, N, dtype=torch.bfloat16):
     lib = load_library()
     fn = "gf_wkv6_backward_workspace_bytes" if dtype == torch.float32 else "gf_wkv6_backward_bf16_workspace_bytes"
     return int(getattr(lib, fn)(B, T, H, N))
+
+
+def backward_varlen_workspace_bytes(S, total_T, H, N):
+    """Bytes of workspace backward_varlen() needs on the current device."""
+    return int(load_library().gf_wkv6_backward_varlen_workspace_bytes(S, total_T, H, N))
 
 
 def prefill_c2(r, k, v, x, u2=None, state_in=None, state_out=None, y=None, stream=None, want_state=True, split=True):

@@ -4,7 +4,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
 cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
-       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 bwd-cfg3 train-fwd-cfg2 train-bwd-cfg2
+       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 bwd-cfg3 bwd-cfg4 train-fwd-cfg2 train-bwd-cfg2
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -165,6 +165,17 @@ def run(case, reps, scale):
             nbytes = B * T * H * 64 * 2 * 9 + B * H * 16384
         # (the checkpoints, 256 B per token*head written by the one and read by the other, are the design's own)
         return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H, bytes=nbytes, ms=_time(fn, reps))
+    if case == "bwd-cfg4":       # gradient of the packed serving-mix prefill (64 sequences of 128..4096 tokens)
+        k = c["cfg4"]
+        S, H = k["S"], k["H"]
+        cu = synth.make_lengths(S, max(1, int(k["len_min"] * scale)), max(2, int(k["len_max"] * scale)), seed=4000)
+        inp = synth.make_varlen(cu, H, 64, "bf16", seed=4001, device=DEV, state_std=k["state_std"])
+        total, mx = int(cu[-1]), int((cu[1:] - cu[:-1]).max())
+        dy = torch.randn(inp.r.shape, device=DEV).bfloat16()
+        ws = torch.empty(gf.backward_varlen_workspace_bytes(S, total, H, 64), dtype=torch.uint8, device=DEV)
+        fn = lambda: gf.backward_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.cu_seqlens, mx, inp.state_in, None, workspace=ws)
+        return dict(case=case, shape=f"S={S} total_T={total} H={H} bf16", units=total * H,
+                    bytes=total * H * 64 * 2 * 9 + 2 * S * H * 16384, ms=_time(fn, reps))
     if case in ("cfg4-prefill", "cfg4-decode", "cfg4-decode-layers"):
         k = c["cfg4"]
         S, H = k["S"], k["H"]
@@ -214,7 +225,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "bwd-cfg3", "train-fwd-cfg2", "train-bwd-cfg2"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "bwd-cfg3", "bwd-cfg4", "train-fwd-cfg2", "train-bwd-cfg2"]
 
 
 def main():

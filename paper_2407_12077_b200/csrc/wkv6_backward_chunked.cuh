@@ -76,6 +76,9 @@ struct BParams {
     // NULL: dense.
     const int32_t* cu;
     long long ckpt_slots;
+    // Packed sequences: the sequence indices by decreasing length (the grid's first CTAs take the longest sequences,
+    // so that the launch does not end on a long one while the other SMs idle); NULL: in index order.
+    const int32_t* order;
 };
 constexpr int GSUM_FLOATS = 64 + 64 * 64;
 
@@ -247,7 +250,8 @@ __device__ __forceinline__ bool scan_rows(float (&v)[G_NB][4], uint32_t tot, int
 // GSUM = true: the summary variant of a split call (see BParams::gsum): only the adjoint's own recurrence
 // G <- diag(D) G + R^^T dY over a segment, from zero, and the product of the chunk decays; it reads x, r, dy only and
 // needs no token-by-token path (R^ never exceeds r: no exponent can overflow).
-template <bool C2, bool GSUM = false>
+// PACKED: packed variable-length sequences (BParams::cu), one CTA per sequence and head.
+template <bool C2, bool GSUM = false, bool PACKED = false>
 __global__ void __launch_bounds__(G_THREADS, 1)
 wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_r,
                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -266,12 +270,14 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const int sp = warp & 3, cx = (warp >> 2) % G_NSLAB, g = lane >> 2, q = lane & 3;       // row group, column slab
     // summary variant: segments 1 .. nseg-1 of every unit; else every segment
     const int gsegs = GSUM ? p.nseg - 1 : p.nseg;
-    const int unit = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0), seq = unit / p.H, h = unit % p.H;
-    const int T = p.cu ? p.cu[seq + 1] - p.cu[seq] : p.T, nchunks = (T + L - 1) / L;
+    const int slot = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0), h = slot % p.H;
+    const int seq = (PACKED && p.order) ? p.order[slot / p.H] : slot / p.H, unit = PACKED ? seq * p.H + h : slot;
+    static_assert(!(PACKED && GSUM), "packed sequences are never split");
+    const int T = PACKED ? p.cu[seq + 1] - p.cu[seq] : p.T, nchunks = (T + L - 1) / L;
     const int c_lo = p.nseg > 1 ? min(nchunks, seg * p.seg_chunks) : 0;                      // this CTA's chunks: c_lo .. c_hi-1,
     const int c_hi = (p.nseg > 1 && seg < p.nseg - 1) ? min(nchunks, c_lo + p.seg_chunks) : nchunks;   // walked from the last
     const int nit = c_hi - c_lo;
-    const long long row0 = p.cu ? (long long)p.cu[seq] : (long long)seq * T;
+    const long long row0 = PACKED ? (long long)p.cu[seq] : (long long)seq * T;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
@@ -360,8 +366,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     };
 
-    const float* ck_unit = p.ckpt + (p.cu ? (size_t)h * p.ckpt_slots + (size_t)(p.cu[seq] >> 6) + 2 * (size_t)seq
-                                         : (size_t)unit * (nchunks + 1)) * 4096;
+    const float* ck_unit = p.ckpt + (PACKED ? (size_t)h * p.ckpt_slots + (size_t)(p.cu[seq] >> 6) + 2 * (size_t)seq
+                                            : (size_t)unit * (nchunks + 1)) * 4096;
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
@@ -889,7 +895,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     }
 
-    if (!GSUM && nit == 0 && seg == 0 && grp == 0 && p.dstate_in) {
+    if (PACKED && nit == 0 && grp == 0 && p.dstate_in) {
         // a sequence without tokens hands the state's gradient through
         float G[G_NB][4];
         if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
@@ -977,10 +983,15 @@ inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
 }
 
 // The same for packed sequences (never split): checkpoints in the packed layout, [H][total_rows / 64 + 2 S] states.
+inline size_t backward_order_floats(long long n_seq)       // a counter's 64 bytes and the sequence order, in floats, 16-byte granular
+{
+    return (size_t)((ORDER_OFFSET / 4 + n_seq + 3) / 4 * 4);
+}
 inline size_t chunked_backward_varlen_workspace_bytes(long long n_seq, long long total_rows, int H, int n_sm)
 {
     const size_t slots = (size_t)(total_rows / ck::L + 2 * n_seq);
-    return ((size_t)H * slots * 4096 + (size_t)n_seq * H * 64 + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+    return ((size_t)H * slots * 4096 + (size_t)n_seq * H * 64 + backward_order_floats(n_seq) +
+            (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
 // The part of the gradient's workspace that a training step's forward pass may use as its split scratch (the
@@ -1012,7 +1023,9 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     if (!attr_set.is_set(dev)) {
         if (cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set.set(dev);
     }
@@ -1025,6 +1038,19 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     float* du_part = ckpt + (cu ? (size_t)H * ckpt_slots : (size_t)units * nck) * 4096;
     float* gsum = du_part + (size_t)units * nseg * 64;
     float* fb = gsum + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
+    const int32_t* order = nullptr;
+    if (cu) {
+        // packed: the sequences longest first (the order array lies between the bonus partial sums and the scratch slots)
+        unsigned int* counter = reinterpret_cast<unsigned int*>(fb);
+        if (B <= ORDER_MAX_SEQ) {
+            int32_t* ord = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(fb) + ORDER_OFFSET);
+            wkv6_order_kernel<<<1, 1024, 0, st>>>(cu, B, counter, ord);
+            launches->fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
+            order = ord;
+        }
+        fb += backward_order_floats(B);
+    }
     if (!ckpt_saved) {                               // (else the forward pass of the training step left them there)
         // (split calls: the forward summaries borrow the buffer of the adjoint's, which are written after them)
         const gf_status_t s = chunked_checkpoints(k, v, x, state_in, ckpt, B, T, H, st, launches, c2 ? 1 : 0, gsum, nseg, seg_chunks, cu, rows);
@@ -1037,14 +1063,16 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
         return GF_ERR_CUDA;
     bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
-                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks, cu, ckpt_slots};
+                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks, cu, ckpt_slots, order};
     if (nseg > 1) {
         // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
         bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
-    if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    else if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;

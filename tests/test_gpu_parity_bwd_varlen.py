@@ -159,7 +159,7 @@ def test_argument_checks():
     r, k, v, x, u, dy, s0, dsT, cu = (None if t is None else t.cuda() for t in case)
     need = int(lib.gf_wkv6_backward_varlen_workspace_bytes(2, 100, 2, 64))
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    assert need == (2 * (100 // 64 + 4) * 4096 + 2 * 2 * 64 + 2 * sms * 64 * 4096) * 4
+    assert need == (2 * (100 // 64 + 4) * 4096 + 2 * 2 * 64 + (16 + 2 + 3) // 4 * 4 + 2 * sms * 64 * 4096) * 4
     small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
     dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
     du = torch.empty(2, 64, device="cuda")
