@@ -71,15 +71,19 @@ struct BParams {
     const float* gsum;
     float* gsum_out;             // summary variant: where the summaries go (same layout)
     int nseg, seg_chunks;
+};
+// What the packed variants take on top (the dense variants keep the plain parameter block).
+struct BParamsPacked : BParams {
     // Packed sequences (never split): rows cu[s] .. cu[s+1]-1 of the [rows][H*64] tensors form sequence s, T is unused,
     // and the checkpoints are [H][ckpt_slots][64][64] with sequence s of head h from slot cu[s] / 64 + 2 s on.
-    // NULL: dense.
     const int32_t* cu;
     long long ckpt_slots;
-    // Packed sequences: the sequence indices by decreasing length (the grid's first CTAs take the longest sequences,
-    // so that the launch does not end on a long one while the other SMs idle); NULL: in index order.
+    // The sequence indices by decreasing length (the grid's first CTAs take the longest sequences, so that the launch
+    // does not end on a long one while the other SMs idle); NULL: in index order.
     const int32_t* order;
 };
+template <bool PACKED> struct BParamsOf { using type = BParams; };
+template <> struct BParamsOf<true> { using type = BParamsPacked; };
 constexpr int GSUM_FLOATS = 64 + 64 * 64;
 
 __device__ __forceinline__ float lds_bf16(uint32_t a)
@@ -257,7 +261,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                             const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
                             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
-                            const __grid_constant__ CUtensorMap tm_dx, const BParams p)
+                            const __grid_constant__ CUtensorMap tm_dx, const typename BParamsOf<PACKED>::type p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -270,14 +274,23 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const int sp = warp & 3, cx = (warp >> 2) % G_NSLAB, g = lane >> 2, q = lane & 3;       // row group, column slab
     // summary variant: segments 1 .. nseg-1 of every unit; else every segment
     const int gsegs = GSUM ? p.nseg - 1 : p.nseg;
-    const int slot = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0), h = slot % p.H;
-    const int seq = (PACKED && p.order) ? p.order[slot / p.H] : slot / p.H, unit = PACKED ? seq * p.H + h : slot;
+    const int slot = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0);
+    int unit = slot, seq = unit / p.H;
+    const int h = unit % p.H;
     static_assert(!(PACKED && GSUM), "packed sequences are never split");
-    const int T = PACKED ? p.cu[seq + 1] - p.cu[seq] : p.T, nchunks = (T + L - 1) / L;
+    int T = p.T;
+    long long row0 = (long long)seq * T;
+    size_t ck_first = 0;                             // the unit's first checkpoint slot (packed)
+    if constexpr (PACKED) {
+        if (p.order) { seq = p.order[seq]; unit = seq * p.H + h; }
+        row0 = p.cu[seq];
+        T = p.cu[seq + 1] - p.cu[seq];
+        ck_first = (size_t)h * p.ckpt_slots + (size_t)(p.cu[seq] >> 6) + 2 * (size_t)seq;
+    }
+    const int nchunks = (T + L - 1) / L;
     const int c_lo = p.nseg > 1 ? min(nchunks, seg * p.seg_chunks) : 0;                      // this CTA's chunks: c_lo .. c_hi-1,
     const int c_hi = (p.nseg > 1 && seg < p.nseg - 1) ? min(nchunks, c_lo + p.seg_chunks) : nchunks;   // walked from the last
     const int nit = c_hi - c_lo;
-    const long long row0 = PACKED ? (long long)p.cu[seq] : (long long)seq * T;
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     const int R0 = 16 * sp + g, R1 = R0 + 8;         // this lane's two rows
@@ -366,8 +379,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     };
 
-    const float* ck_unit = p.ckpt + (PACKED ? (size_t)h * p.ckpt_slots + (size_t)(p.cu[seq] >> 6) + 2 * (size_t)seq
-                                            : (size_t)unit * (nchunks + 1)) * 4096;
+    const float* ck_unit = p.ckpt + (PACKED ? ck_first : (size_t)unit * (nchunks + 1)) * 4096;
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
@@ -1063,15 +1075,16 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
         return GF_ERR_CUDA;
     bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
-                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks, cu, ckpt_slots, order};
+                  wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks};
+    const bc::BParamsPacked pp{p, cu, ckpt_slots, order};
     if (nseg > 1) {
         // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
         bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
-    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
-    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
+    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
     else if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     launches->fetch_add(1, std::memory_order_relaxed);

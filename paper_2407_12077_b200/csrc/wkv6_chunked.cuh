@@ -680,9 +680,12 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
     }
     const int nchunks = PERSIST ? 0 : (len + L - 1) / L;
     // checkpoint slots of this unit: the first one, and how many chunks the whole sequence has
-    auto ckpt_first = [&]() -> size_t {
-        return p.cu_seqlens ? (size_t)h * p.ckpt_slots + (size_t)(p.cu_seqlens[seq] >> 6) + 2 * (size_t)seq
-                            : (size_t)unit * ((p.T + L - 1) / L + 1);
+    auto ckpt_slot = [&](int c_abs) -> size_t {       // (the packed form recomputes what it needs: nothing stays live for it)
+        if (p.cu_seqlens) {
+            const int sq = unit / p.H, hh = unit - sq * p.H;
+            return (size_t)hh * p.ckpt_slots + (size_t)(p.cu_seqlens[sq] >> 6) + 2 * (size_t)sq + c_abs;
+        }
+        return (size_t)unit * ((p.T + L - 1) / L + 1) + c_abs;
     };
     auto ckpt_chunks = [&]() -> int { return p.cu_seqlens ? nchunks : (p.T + L - 1) / L; };
     const int col0 = h * 64;
@@ -987,7 +990,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
             if (CKPT || (SUMMARY && p.ckpt))         // the state before chunk c of the segment (dense sequences: T / 64 + 1 states per unit)
-                store_to(p.ckpt + (ckpt_first() + seg * p.seg_chunks + c) * 4096);
+                store_to(p.ckpt + ckpt_slot(seg * p.seg_chunks + c) * 4096);
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1080,10 +1083,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + (ckpt_first() + ckpt_chunks()) * 4096);
+        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + ckpt_slot(ckpt_chunks()) * 4096);
         if (SUMMARY && p.ckpt) {
             if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
-                store_to(p.ckpt + (ckpt_first() + ckpt_chunks()) * 4096);
+                store_to(p.ckpt + ckpt_slot(ckpt_chunks()) * 4096);
         } else if (SUMMARY) {
             if (!lds32(abort_flag)) {
                 float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
