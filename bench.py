@@ -374,6 +374,7 @@ def main():
                 ("decay_logit", "dl-cfg2", "gf_c2_decay_logit, 65536 tokens x 2048 channels, ranks 32 and 64 (x read, d written)"),
                 ("backward", "bwd-cfg2", "gf_wkv6_backward, cfg2 shape: checkpoint pass + chunked gradient kernel, two chunks in flight per SM (1152 B per token*head counted; the design moves 2048)"),
                 ("backward_long_context", "bwd-cfg3", "gf_wkv6_backward, B=1 T=131072 H=32: 32 units, sequences split 4-way with the adjoint's segment summaries (5 launches)"),
+                ("backward_packed", "bwd-cfg4", "gf_wkv6_backward_varlen, the serving mix's shape (64 packed sequences of 128..4096 tokens, 32 heads: 2048 units, longest first)"),
                 ("train_forward", "train-fwd-cfg2", "gf_wkv6_prefill_train, cfg2 shape: the prefill that also keeps its chunk-start states (256 B per token*head more, not counted)"),
                 ("train_backward", "train-bwd-cfg2", "gf_wkv6_backward_saved, cfg2 shape: the gradient kernel alone, from the states the forward pass kept"),
                 ("decode_step", "cfg4-decode", "gf_wkv6_step, 64 sequences x 32 heads, 64 steps per graph replay (states stay in L2)"),

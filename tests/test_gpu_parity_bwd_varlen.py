@@ -138,6 +138,21 @@ def test_serving_mix_of_lengths_more_units_than_sms(c2):
     check(got, ref, case[-1].numpy(), c2, what="mix")
 
 
+def test_serving_mix_at_full_size_every_unit():
+    """The packed batch the benchmark's gradient row times (64 sequences of 128 .. 4096 tokens, 32 heads: 2048 units of
+    different lengths on 148 SMs, longest first), every sequence against the oracle."""
+    c = synth.CONFIGS["cfg4"]
+    cu = synth.make_lengths(c["S"], c["len_min"], c["len_max"], seed=4000)
+    lens = tuple(int(n) for n in np.diff(cu.numpy()))
+    inp = synth.make_varlen(cu, c["H"], 64, "bf16", seed=4001, state_std=c["state_std"])
+    g = torch.Generator().manual_seed(4002)
+    dy = torch.randn(inp.r.shape, generator=g).to(torch.bfloat16)
+    dsT = torch.randn(len(lens), c["H"], 64, 64, generator=g) * 0.1
+    case = (inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT, cu)
+    got, ref = run_gpu(case), run_oracle(case)
+    check(got, ref, cu.numpy(), what="cfg4")
+
+
 def test_fast_decays_take_the_token_path_in_some_sequences():
     lens = (150, 90, 64)
     case = make(lens, 2, 7400, x_range=(-2.0, 1.5))
