@@ -215,6 +215,35 @@ GF_API gf_status_t gf_wkv6_backward_varlen_c2(const void *r, const void *k, cons
                                        size_t workspace_bytes, gf_stream_t stream);
 GF_API size_t gf_wkv6_backward_varlen_workspace_bytes(int S, int total_T, int H, int N);
 
+/* The training pair for packed sequences, as gf_wkv6_prefill_train / gf_wkv6_backward_saved for dense ones:
+ * gf_wkv6_prefill_varlen_train / gf_wkv6_prefill_varlen_c2_train are gf_wkv6_prefill_varlen / gf_wkv6_prefill_varlen_c2
+ * (same results; one CTA per sequence and head, never split and never persistent) that also leave the state before every
+ * chunk of 64 tokens of every sequence, and after its last token, in `workspace`, the packed gradient's workspace
+ * (gf_wkv6_backward_varlen_workspace_bytes(S,total_T,H,N) bytes); gf_wkv6_backward_varlen_saved /
+ * gf_wkv6_backward_varlen_c2_saved are the packed gradient calls without their checkpoint launch.  The workspace must
+ * still hold what the forward call of the SAME r,k,v,x,state_in,cu_seqlens wrote (nothing checks it). */
+GF_API gf_status_t gf_wkv6_prefill_varlen_train(const void *r, const void *k, const void *v, const void *x,
+                                         const float *u, const float *state_in, float *state_out, void *y,
+                                         const int32_t *cu_seqlens, int S, int total_T, int max_seqlen, int H,
+                                         int N, void *workspace, size_t workspace_bytes, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_prefill_varlen_c2_train(const void *r, const void *k, const void *v, const void *x,
+                                            const void *u2, const float *state_in, float *state_out, void *y,
+                                            const int32_t *cu_seqlens, int S, int total_T, int max_seqlen,
+                                            int H, int N, void *workspace, size_t workspace_bytes,
+                                            gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_backward_varlen_saved(const void *r, const void *k, const void *v, const void *x,
+                                          const float *u, const float *state_in, const void *dy,
+                                          const float *dstate_out, void *dr, void *dk, void *dv, void *dx,
+                                          float *du, float *dstate_in, const int32_t *cu_seqlens, int S,
+                                          int total_T, int max_seqlen, int H, int N, void *workspace,
+                                          size_t workspace_bytes, gf_stream_t stream);
+GF_API gf_status_t gf_wkv6_backward_varlen_c2_saved(const void *r, const void *k, const void *v, const void *x,
+                                             const float *state_in, const void *dy, const float *dstate_out,
+                                             void *dr, void *dk, void *dv, void *dx, float *dstate_in,
+                                             const int32_t *cu_seqlens, int S, int total_T, int max_seqlen,
+                                             int H, int N, void *workspace, size_t workspace_bytes,
+                                             gf_stream_t stream);
+
 /* Packed variable-length prefill (batched serving).  Sequence s occupies rows
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of the [total_T][H][N] tensors; chunking restarts
  * at every sequence start, so a sequence never sees another's tokens.  cu_seqlens is a

@@ -16,7 +16,7 @@ from . import _build
 
 __all__ = [
     "GfError", "load_library", "library_path", "prefill", "prefill_varlen", "step", "bind_step",
-    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "prefill_train", "backward_workspace_bytes", "backward_varlen", "backward_varlen_workspace_bytes", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
+    "sequence_summary", "fold_summaries", "SUMMARY_FLOATS", "backward", "backward_c2", "prefill_train", "backward_workspace_bytes", "backward_varlen", "backward_varlen_workspace_bytes", "prefill_varlen_train", "decay_logit", "prefill_c2", "prefill_varlen_c2", "step_c2", "prefill_static", "STATIC_SCRATCH_BYTES", "prefill_host", "host_workspace_bytes", "workspace_bytes", "split_plan", "set_workspace", "set_kernel", "last_device_status",
     "launch_count", "status_string", "version", "set_wait_limit", "selftest_wait_timeout",
     "KERNEL_AUTO", "KERNEL_EXACT", "KERNEL_CHUNKED",
 ]
@@ -40,6 +40,10 @@ _SIGNATURES = {
     "gf_wkv6_backward_varlen": (_i, [_vp] * 15 + [_i] * 5 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_varlen_c2": (_i, [_vp] * 13 + [_i] * 5 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_varlen_workspace_bytes": (_sz, [_i] * 4),
+    "gf_wkv6_backward_varlen_saved": (_i, [_vp] * 15 + [_i] * 5 + [_vp, _sz, _vp]),
+    "gf_wkv6_backward_varlen_c2_saved": (_i, [_vp] * 13 + [_i] * 5 + [_vp, _sz, _vp]),
+    "gf_wkv6_prefill_varlen_train": (_i, [_vp] * 9 + [_i] * 5 + [_vp, _sz, _vp]),
+    "gf_wkv6_prefill_varlen_c2_train": (_i, [_vp] * 9 + [_i] * 5 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_saved": (_i, [_vp] * 14 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_backward_c2_saved": (_i, [_vp] * 12 + [_i] * 4 + [_vp, _sz, _vp]),
     "gf_wkv6_prefill_train": (_i, [_vp] * 8 + [_i] * 4 + [_vp, _sz, _vp]),
@@ -283,8 +287,9 @@ def backward_c2(r, k, v, x, dy, state_in=None, dstate_out=None, want_dstate=True
 
 
 def backward_varlen(r, k, v, x, u, dy, cu_seqlens, max_seqlen, state_in=None, dstate_out=None, want_dstate=True,
-                    stream=None, workspace=None, c2=False):
-    """gf_wkv6_backward_varlen / gf_wkv6_backward_varlen_c2: gradient of the packed prefill (bf16 tensors).  r,k,v,x,dy:
+                    stream=None, workspace=None, c2=False, saved=False):
+    """gf_wkv6_backward_varlen / gf_wkv6_backward_varlen_c2 (saved=True: their _saved forms, from the states that
+    prefill_varlen_train() left in `workspace`): gradient of the packed prefill (bf16 tensors).  r,k,v,x,dy:
     [total_T,H,N]; cu_seqlens: int32 CUDA [S+1]; u: [H,N] fp32 (ignored with c2=True); state_in / dstate_out:
     [S,H,N,N] fp32 or None.  Returns (dr, dk, dv, dx, du, dstate_in), du None with c2=True."""
     lib = load_library()
@@ -306,6 +311,10 @@ def backward_varlen(r, k, v, x, u, dy, cu_seqlens, max_seqlen, state_in=None, ds
             args.append(_dev(du, "du"))
         args += [_dev(ds0, "dstate_in"), _dev(cu_seqlens, "cu_seqlens", torch.int32)]
         fn = "gf_wkv6_backward_varlen_c2" if c2 else "gf_wkv6_backward_varlen"
+        if saved:
+            if workspace is None or workspace.numel() < nbytes:
+                raise ValueError("backward_varlen(saved=True) needs the workspace prefill_varlen_train() filled")
+            fn += "_saved"
         _check(getattr(lib, fn)(*args, S, total_T, int(max_seqlen), H, N, _dev(ws, "workspace"), ws.numel(), _stream(stream)), fn)
     return dr, dk, dv, dx, du, ds0
 
@@ -334,6 +343,27 @@ def backward_workspace_bytes(B, T, H, N, dtype=torch.bfloat16):
     lib = load_library()
     fn = "gf_wkv6_backward_workspace_bytes" if dtype == torch.float32 else "gf_wkv6_backward_bf16_workspace_bytes"
     return int(getattr(lib, fn)(B, T, H, N))
+
+
+def prefill_varlen_train(r, k, v, x, u, cu_seqlens, max_seqlen, workspace, state_in=None, c2=False, u2=None, stream=None):
+    """gf_wkv6_prefill_varlen_train / gf_wkv6_prefill_varlen_c2_train: the packed forward pass of a training step.  As
+    prefill_varlen() / prefill_varlen_c2() (u is ignored with c2=True, u2 without); `workspace` (uint8 CUDA tensor of
+    backward_varlen_workspace_bytes(S,total_T,H,N) bytes) receives the chunk-start states for
+    backward_varlen(..., saved=True).  Returns (y, state_out)."""
+    lib = load_library()
+    total_T, H, N = r.shape
+    S = cu_seqlens.numel() - 1
+    bf, f32 = torch.bfloat16, torch.float32
+    y = torch.empty_like(r)
+    s_out = torch.empty((S, H, N, N), device=r.device, dtype=f32)
+    with torch.cuda.device(r.device):
+        base = [_dev(r, "r", bf), _dev(k, "k", bf, r.shape), _dev(v, "v", bf, r.shape), _dev(x, "x", bf, r.shape)]
+        mid = _dev(u2, "u2", bf, r.shape) if c2 else _dev(u, "u", f32, (H, N))
+        fn = "gf_wkv6_prefill_varlen_c2_train" if c2 else "gf_wkv6_prefill_varlen_train"
+        _check(getattr(lib, fn)(*base, mid, _dev(state_in, "state_in", f32, (S, H, N, N)), _dev(s_out, "state_out"),
+                                _dev(y, "y"), _dev(cu_seqlens, "cu_seqlens", torch.int32), S, total_T, int(max_seqlen), H, N,
+                                _dev(workspace, "workspace"), workspace.numel(), _stream(stream)), fn)
+    return y, s_out
 
 
 def backward_varlen_workspace_bytes(S, total_T, H, N):

@@ -494,7 +494,7 @@ gf_status_t backward_varlen_bf16(const void* r, const void* k, const void* v, co
                                  const float* state_in, const void* dy, const float* dstate_out, void* dr, void* dk,
                                  void* dv, void* dx, float* du, float* dstate_in, const int32_t* cu_seqlens, int S,
                                  int total_T, int max_seqlen, int H, int N, void* workspace, size_t workspace_bytes,
-                                 gf_stream_t stream, bool c2)
+                                 gf_stream_t stream, bool c2, bool saved = false)
 {
     using bf = __nv_bfloat16;
     if (S < 0 || total_T < 0 || max_seqlen < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
@@ -530,7 +530,7 @@ gf_status_t backward_varlen_bf16(const void* r, const void* k, const void* v, co
     if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
     const gf_status_t s = gf::chunked_backward((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, (const bf*)dy,
                                                dstate_out, (bf*)dr, (bf*)dk, (bf*)dv, (bf*)dx, du, dstate_in, S, max_seqlen, H,
-                                               static_cast<float*>(workspace), st, &g_launches, c2, false, cu_seqlens, total_T);
+                                               static_cast<float*>(workspace), st, &g_launches, c2, saved, cu_seqlens, total_T);
     if (s != GF_OK) return s;
     return launch_result();
 }
@@ -553,6 +553,77 @@ gf_status_t gf_wkv6_backward_varlen_c2(const void* r, const void* k, const void*
 {
     return backward_varlen_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in,
                                 cu_seqlens, S, total_T, max_seqlen, H, N, workspace, workspace_bytes, stream, true);
+}
+
+gf_status_t gf_wkv6_backward_varlen_saved(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                          const float* state_in, const void* dy, const float* dstate_out, void* dr,
+                                          void* dk, void* dv, void* dx, float* du, float* dstate_in,
+                                          const int32_t* cu_seqlens, int S, int total_T, int max_seqlen, int H, int N,
+                                          void* workspace, size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_varlen_bf16(r, k, v, x, u, state_in, dy, dstate_out, dr, dk, dv, dx, du, dstate_in, cu_seqlens, S,
+                                total_T, max_seqlen, H, N, workspace, workspace_bytes, stream, false, true);
+}
+
+gf_status_t gf_wkv6_backward_varlen_c2_saved(const void* r, const void* k, const void* v, const void* x,
+                                             const float* state_in, const void* dy, const float* dstate_out, void* dr,
+                                             void* dk, void* dv, void* dx, float* dstate_in, const int32_t* cu_seqlens,
+                                             int S, int total_T, int max_seqlen, int H, int N, void* workspace,
+                                             size_t workspace_bytes, gf_stream_t stream)
+{
+    return backward_varlen_bf16(r, k, v, x, nullptr, state_in, dy, dstate_out, dr, dk, dv, dx, nullptr, dstate_in,
+                                cu_seqlens, S, total_T, max_seqlen, H, N, workspace, workspace_bytes, stream, true, true);
+}
+
+namespace {
+// forward pass of a training step over packed sequences: the packed prefill that also leaves its chunk-start states
+// (packed layout) in the packed gradient's workspace; one CTA per sequence and head, never split
+gf_status_t prefill_varlen_train(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                 const void* u2, const float* state_in, float* state_out, void* y,
+                                 const int32_t* cu_seqlens, int S, int total_T, int max_seqlen, int H, int N,
+                                 void* workspace, size_t workspace_bytes, gf_stream_t stream, bool c2)
+{
+    using bf = __nv_bfloat16;
+    if (S < 0 || total_T < 0 || max_seqlen < 0 || H < 0 || N < 0) return GF_ERR_INVALID_ARG;
+    if (N != 64) return GF_ERR_UNSUPPORTED;
+    if (S == 0 || H == 0) return GF_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (total_T == 0) return pass_state(state_in, state_out, (size_t)S * H, st);
+    if (!r || !k || !v || !x || !y || !cu_seqlens || (!c2 && !u) || max_seqlen == 0) return GF_ERR_INVALID_ARG;
+    const void* ptrs[] = {r, k, v, x, u, u2, state_in, state_out, y, workspace};
+    for (const void* q : ptrs)
+        if (misaligned(q)) return GF_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(cu_seqlens) % alignof(int32_t)) return GF_ERR_INVALID_ARG;
+    if (y == r || y == k || y == v || y == x || (u2 && y == u2)) return GF_ERR_INVALID_ARG;
+    if ((long long)S * H > 0x7fffffffLL) return GF_ERR_INVALID_ARG;
+    if ((long long)total_T >= (1LL << 31) - 64) return GF_ERR_UNSUPPORTED;
+    const size_t need = gf_wkv6_backward_varlen_workspace_bytes(S, total_T, H, N);
+    if (need == 0) return GF_ERR_CUDA;
+    if (!workspace || workspace_bytes < need) return GF_ERR_WORKSPACE;
+    const gf_status_t s = gf::chunked_prefill((const bf*)r, (const bf*)k, (const bf*)v, (const bf*)x, u, state_in, state_out,
+                                              (bf*)y, cu_seqlens, S, max_seqlen, total_T, H, st, &g_launches, nullptr, 0,
+                                              (const bf*)u2, c2 ? 1 : 0, static_cast<float*>(workspace));
+    if (s != GF_OK) return s;
+    return launch_result();
+}
+}  // namespace
+
+gf_status_t gf_wkv6_prefill_varlen_train(const void* r, const void* k, const void* v, const void* x, const float* u,
+                                         const float* state_in, float* state_out, void* y, const int32_t* cu_seqlens,
+                                         int S, int total_T, int max_seqlen, int H, int N, void* workspace,
+                                         size_t workspace_bytes, gf_stream_t stream)
+{
+    return prefill_varlen_train(r, k, v, x, u, nullptr, state_in, state_out, y, cu_seqlens, S, total_T, max_seqlen, H, N,
+                                workspace, workspace_bytes, stream, false);
+}
+
+gf_status_t gf_wkv6_prefill_varlen_c2_train(const void* r, const void* k, const void* v, const void* x, const void* u2,
+                                            const float* state_in, float* state_out, void* y, const int32_t* cu_seqlens,
+                                            int S, int total_T, int max_seqlen, int H, int N, void* workspace,
+                                            size_t workspace_bytes, gf_stream_t stream)
+{
+    return prefill_varlen_train(r, k, v, x, nullptr, u2, state_in, state_out, y, cu_seqlens, S, total_T, max_seqlen, H, N,
+                                workspace, workspace_bytes, stream, true);
 }
 
 namespace {

@@ -961,15 +961,20 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     }
 }
 
-// du[h][i] = sum over the batch of the units' partial sums, in batch order
-__global__ void __launch_bounds__(64)
+// du[h][i] = sum over the batch of the units' partial sums: eight strided partial sums in batch order, added in a
+// fixed order (deterministic; many sequences do not serialise on one thread)
+__global__ void __launch_bounds__(512)
 wkv6_backward_chunked_du_kernel(const float* __restrict__ du_part, int B, int H, int nseg, float* __restrict__ du)
 {
-    const int h = blockIdx.x, i = threadIdx.x;
+    __shared__ float part[8][64];
+    const int h = blockIdx.x, i = threadIdx.x & 63, grp = threadIdx.x >> 6;
     float acc = 0.f;
-    for (int b = 0; b < B; ++b)
+    for (int b = grp; b < B; b += 8)
         for (int sg = 0; sg < nseg; ++sg) acc += du_part[(((size_t)b * H + h) * nseg + sg) * 64 + i];
-    du[h * 64 + i] = acc;
+    part[grp][i] = acc;
+    __syncthreads();
+    if (grp == 0)
+        du[h * 64 + i] = ((part[0][i] + part[1][i]) + (part[2][i] + part[3][i])) + ((part[4][i] + part[5][i]) + (part[6][i] + part[7][i]));
 }
 
 }  // namespace bc
@@ -1090,7 +1095,7 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     launches->fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     if (c2) return GF_OK;                            // no bonus, no bonus gradient
-    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 64, 0, st>>>(du_part, B, H, nseg, du);
+    bc::wkv6_backward_chunked_du_kernel<<<(unsigned)H, 512, 0, st>>>(du_part, B, H, nseg, du);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }

@@ -74,3 +74,41 @@ def test_argument_checks():
     assert lib.gf_wkv6_prefill_train(*args, 1, 100, 2, 64, None, 0, None) == 4          # no workspace
     assert lib.gf_wkv6_prefill_train(*args, 1, 100, 2, 32, None, 0, None) == 2          # head size
     assert gf.launch_count() == before
+
+
+@pytest.mark.parametrize("lens", [(300, 64, 0, 37, 129), (1,), (4096, 100), (65, 65, 65, 1000)])
+@pytest.mark.parametrize("c2", [False, True])
+def test_packed_pair_is_bit_identical_to_the_separate_packed_calls(lens, c2):
+    """gf_wkv6_prefill_varlen_train + gf_wkv6_backward_varlen_saved: same kernels on the same inputs as the packed
+    prefill (unsplit) and the packed gradient, the checkpoints in the packed layout written by the forward pass."""
+    H = 3
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32)
+    inp = synth.make_varlen(cu, H, 64, "bf16", seed=90 + sum(lens), state_std=0.1).to(DEV)
+    S, total, mx = len(lens), int(sum(lens)), max(lens)
+    g = torch.Generator(device=DEV).manual_seed(total)
+    dy = torch.randn(inp.r.shape, generator=g, device=DEV).bfloat16()
+    u2 = torch.randn(inp.r.shape, generator=g, device=DEV).bfloat16() if c2 else None
+    dsT = torch.randn((S, H, 64, 64), generator=g, device=DEV) * 0.1
+    ws = torch.empty(gf.backward_varlen_workspace_bytes(S, total, H, 64), dtype=torch.uint8, device=DEV)
+    y, s = gf.prefill_varlen_train(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, mx, ws, inp.state_in, c2=c2, u2=u2)
+    ga = gf.backward_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.cu_seqlens, mx, inp.state_in, dsT, workspace=ws, c2=c2, saved=True)
+    gb = gf.backward_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.cu_seqlens, mx, inp.state_in, dsT, c2=c2)
+    if c2:
+        y0, s0 = gf.prefill_varlen_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.cu_seqlens, mx, inp.state_in, split=False)
+    else:
+        y0, s0 = gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, mx, inp.state_in, split=False)
+    gf.last_device_status()
+    assert torch.equal(y, y0) and torch.equal(s, s0)
+    for p, q in zip(ga, gb):
+        assert (p is None and q is None) or torch.equal(p, q)
+    # and once against the oracle
+    dyn = dy.float().cpu().numpy().astype(np.float64)
+    c = inp.to("cpu")
+    if c2:
+        ref = orc.backward_c2_varlen(c.r, c.k, c.v, c.x, dyn, cu, c.state_in, dsT.cpu().numpy().astype(np.float64))
+        got = [ga[0], ga[1], ga[2], ga[3], ga[5]]
+    else:
+        ref = orc.backward_varlen(c.r, c.k, c.v, c.x, c.u, dyn, cu, c.state_in, dsT.cpu().numpy().astype(np.float64))
+        got = list(ga)
+    for i, (p, q) in enumerate(zip(got, ref)):
+        assert orc.rel_l2(p.float().cpu().numpy(), q) <= (8e-3 if i == 3 else 5e-3), i
