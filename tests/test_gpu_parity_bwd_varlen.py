@@ -194,3 +194,15 @@ def test_argument_checks():
                                      p(ds0), p(cu), 2, 100, 70, 2, 32, p(big), big.numel(), None)
     assert st == GF_ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+def test_more_sequences_than_the_order_kernel_ranks():
+    """Past 8192 sequences the call keeps index order (no ranking): thousands of tiny sequences, many of them empty."""
+    rng = np.random.default_rng(7700)
+    lens = tuple(int(n) for n in rng.integers(0, 4, size=8300))
+    case = make(lens, 1, 7700)
+    got, ref = run_gpu(case), run_oracle(case)
+    check(got, ref, case[-1].numpy(), what="8300 sequences")
+    dsT = case[7].numpy()
+    empty = np.flatnonzero(np.asarray(lens) == 0)
+    assert len(empty) > 1000 and all(np.array_equal(got[5][s], dsT[s]) for s in empty[:50])
