@@ -200,8 +200,10 @@ GF_API gf_status_t gf_wkv6_backward_c2_saved(const void *r, const void *k, const
  * [S][H][N][N] fp32; du [H][N] fp32 is summed over the sequences in index order.  A sequence without tokens hands its
  * state gradient through.  `workspace`: caller-owned DEVICE buffer of at least
  * gf_wkv6_backward_varlen_workspace_bytes(S,total_T,H,N) bytes, 16-byte aligned (H * (total_T / 64 + 2 S) states of
- * 64x64 fp32, plus 2 MiB per SM); GF_ERR_WORKSPACE if absent or too small.  One CTA per (sequence, head), the longest
- * sequences first, never split: four kernels on `stream` (three for the Finch-C2 form), nothing allocated, no synchronisation, deterministic.
+ * 64x64 fp32, plus 2 MiB per SM, plus the segment summaries of the widest split when S*H is less than half the SMs);
+ * GF_ERR_WORKSPACE if absent or too small.  One CTA per (sequence, head), the longest sequences first; with S*H less
+ * than half the SMs every sequence is cut into segments by max_seqlen, as in the dense call (segments past a shorter
+ * sequence's end do no work): four kernels on `stream` (three for the Finch-C2 form), six resp. five when split, nothing allocated, no synchronisation, deterministic.
  * Other statuses as gf_wkv6_backward (dstate_in must not be dstate_out; total_T >= 2^31 - 64 or N != 64 unsupported). */
 GF_API gf_status_t gf_wkv6_backward_varlen(const void *r, const void *k, const void *v, const void *x, const float *u,
                                     const float *state_in, const void *dy, const float *dstate_out, void *dr,

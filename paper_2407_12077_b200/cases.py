@@ -4,7 +4,7 @@ prints one JSON line per case with CUDA-event timings (inputs resident in HBM, s
     python -m paper_2407_12077_b200.cases [--reps N] [--scale F] case [case ...]      (or: all)
 
 cases: cfg0 cfg1 cfg2 cfg2-c2 cfg3 cfg3-segments cfg3-packed cfg4-prefill cfg4-decode cfg4-decode-layers ln-cfg1 ln-cfg2 ln-wide kc-cfg2 kc-wide
-       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 bwd-cfg3 bwd-cfg4 train-fwd-cfg2 train-bwd-cfg2
+       dl-cfg1 dl-cfg2 bwd-cfg1 bwd-cfg2 bwd-cfg3 bwd-cfg3-packed bwd-cfg4 train-fwd-cfg2 train-bwd-cfg2
 --scale shrinks the time axis (T, sequence lengths) for quick runs or profiler captures.
 
 `bytes` is the algorithmic HBM traffic of one run of the case (r,k,v,x in, y out, states in/out), `frac` that
@@ -104,6 +104,16 @@ def run(case, reps, scale):
         fn = lambda: gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, max(lens), None, state_out=s, y=y)
         return dict(case=case, shape=f"S=2 lens={lens} H={H} bf16", units=sum(lens) * H,
                     bytes=sum(lens) * H * 640 + 2 * H * 16384, ms=_time(fn, reps))
+    if case == "bwd-cfg3-packed":           # gradient of that packed call (64 units: the sequences split by the longer one)
+        k = c["cfg3"]
+        H, lens = k["H"], [sc(k["T"]), sc(k["T"] * 3 // 8) + 37]
+        cu = torch.tensor([0, lens[0], lens[0] + lens[1]], dtype=torch.int32)
+        inp = synth.make_varlen(cu, H, 64, "bf16", seed=3001, device=DEV, state_std=0.0)
+        dy = torch.randn(inp.r.shape, device=DEV).bfloat16()
+        ws = torch.empty(gf.backward_varlen_workspace_bytes(2, sum(lens), H, 64), dtype=torch.uint8, device=DEV)
+        fn = lambda: gf.backward_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.cu_seqlens, max(lens), None, None, workspace=ws)
+        return dict(case=case, shape=f"S=2 lens={lens} H={H} bf16", units=sum(lens) * H,
+                    bytes=sum(lens) * H * 64 * 2 * 9 + 2 * H * 16384, ms=_time(fn, reps))
     if case in ("ln-cfg1", "ln-cfg2", "ln-wide"):  # LayerNorm across all heads over the tokens of a prefill's output
         k = c["cfg1" if case == "ln-cfg1" else "cfg2"]
         rows, H = k["B"] * sc(k["T"]), (128 if case == "ln-wide" else k["H"])
@@ -225,7 +235,7 @@ def run(case, reps, scale):
     raise SystemExit(f"unknown case {case}")
 
 
-ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "bwd-cfg3", "bwd-cfg4", "train-fwd-cfg2", "train-bwd-cfg2"]
+ALL = ["cfg0", "cfg1", "cfg2", "cfg2-c2", "cfg3", "cfg3-segments", "cfg3-packed", "cfg4-prefill", "cfg4-decode", "cfg4-decode-layers", "ln-cfg1", "ln-cfg2", "ln-wide", "kc-cfg2", "kc-wide", "dl-cfg1", "dl-cfg2", "bwd-cfg1", "bwd-cfg2", "bwd-cfg3", "bwd-cfg3-packed", "bwd-cfg4", "train-fwd-cfg2", "train-bwd-cfg2"]
 
 
 def main():

@@ -74,7 +74,7 @@ struct BParams {
 };
 // What the packed variants take on top (the dense variants keep the plain parameter block).
 struct BParamsPacked : BParams {
-    // Packed sequences (never split): rows cu[s] .. cu[s+1]-1 of the [rows][H*64] tensors form sequence s, T is unused,
+    // Packed sequences (split by the longest one: segments past a sequence's end are empty): rows cu[s] .. cu[s+1]-1 of the [rows][H*64] tensors form sequence s, T is unused,
     // and the checkpoints are [H][ckpt_slots][64][64] with sequence s of head h from slot cu[s] / 64 + 2 s on.
     const int32_t* cu;
     long long ckpt_slots;
@@ -277,7 +277,6 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const int slot = blockIdx.x / gsegs, seg = blockIdx.x % gsegs + (GSUM ? 1 : 0);
     int unit = slot, seq = unit / p.H;
     const int h = unit % p.H;
-    static_assert(!(PACKED && GSUM), "packed sequences are never split");
     int T = p.T;
     long long row0 = (long long)seq * T;
     size_t ck_first = 0;                             // the unit's first checkpoint slot (packed)
@@ -907,7 +906,14 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     }
 
-    if (PACKED && nit == 0 && grp == 0 && p.dstate_in) {
+    if (PACKED && GSUM && nit == 0 && grp == 0) {
+        // a segment past its sequence's end: the identity summary (the decay product is stored below)
+        float Z[G_NB][4];
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) Z[n][0] = Z[n][1] = Z[n][2] = Z[n][3] = 0.f;
+        store_f32_block(p.gsum_out + ((size_t)unit * (p.nseg - 1) + (seg - 1)) * GSUM_FLOATS + 64, Z);
+    }
+    if (PACKED && !GSUM && nit == 0 && seg == 0 && grp == 0 && p.dstate_in) {
         // a sequence without tokens hands the state's gradient through
         float G[G_NB][4];
         if (p.dstate_out) load_f32_block(p.dstate_out + (size_t)unit * 4096, G);
@@ -1004,11 +1010,20 @@ inline size_t backward_order_floats(long long n_seq)       // a counter's 64 byt
 {
     return (size_t)((ORDER_OFFSET / 4 + n_seq + 3) / 4 * 4);
 }
+// (the most segments a packed call of this many units may be cut into, whatever its longest sequence: the workspace is
+// sized for that, so that its size does not depend on max_seqlen)
+inline int packed_split_max(long long units, int n_sm)
+{
+    if (units <= 0 || n_sm <= 0 || units * 2 > n_sm) return 1;
+    const long long want = n_sm / units;
+    return want > 8 ? 8 : (int)want;
+}
 inline size_t chunked_backward_varlen_workspace_bytes(long long n_seq, long long total_rows, int H, int n_sm)
 {
     const size_t slots = (size_t)(total_rows / ck::L + 2 * n_seq);
-    return ((size_t)H * slots * 4096 + (size_t)n_seq * H * 64 + backward_order_floats(n_seq) +
-            (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
+    const size_t units = (size_t)n_seq * H, nmax = (size_t)packed_split_max((long long)units, n_sm);
+    return ((size_t)H * slots * 4096 + units * nmax * 64 + units * (nmax - 1) * bc::GSUM_FLOATS +
+            backward_order_floats(n_seq) + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
 // The part of the gradient's workspace that a training step's forward pass may use as its split scratch (the
@@ -1030,7 +1045,7 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
                                     bool c2 = false, bool ckpt_saved = false, const int32_t* cu = nullptr,
                                     long long packed_rows = 0)
 {
-    // packed sequences: cu = device cu_seqlens of B sequences over packed_rows rows, T = max_seqlen; never split
+    // packed sequences: cu = device cu_seqlens of B sequences over packed_rows rows, T = max_seqlen (the split is cut by it)
     const long long units = (long long)B * H, rows = cu ? packed_rows : (long long)B * T;
     const int n_sm = sm_count();
     if (n_sm <= 0) return GF_ERR_CUDA;
@@ -1042,19 +1057,21 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
             cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
             cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
-            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess ||
+            cudaFuncSetAttribute(bc::wkv6_backward_chunked_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bc::G_SMEM_ALLOC) != cudaSuccess)
             return GF_ERR_CUDA;
         attr_set.set(dev);
     }
     const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
     int seg_chunks = 0;
-    int nseg = cu ? 1 : backward_split(units, T, n_sm, &seg_chunks);
+    int nseg = backward_split(units, T, n_sm, &seg_chunks);
     if (units * nseg > 0x7fffffffLL) nseg = 1;
+    const int nalloc = cu ? packed_split_max(units, n_sm) : nseg;      // (packed: the workspace is laid out for the widest split)
     const long long ckpt_slots = cu ? rows / ck::L + 2LL * B : 0;
     float* ckpt = ws;
     float* du_part = ckpt + (cu ? (size_t)H * ckpt_slots : (size_t)units * nck) * 4096;
-    float* gsum = du_part + (size_t)units * nseg * 64;
-    float* fb = gsum + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
+    float* gsum = du_part + (size_t)units * nalloc * 64;
+    float* fb = gsum + (size_t)units * (nalloc - 1) * bc::GSUM_FLOATS;
     const int32_t* order = nullptr;
     if (cu) {
         // packed: the sequences longest first (the order array lies between the bonus partial sums and the scratch slots)
@@ -1084,12 +1101,13 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     const bc::BParamsPacked pp{p, cu, ckpt_slots, order};
     if (nseg > 1) {
         // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
-        bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+        if (cu) bc::wkv6_backward_chunked_kernel<false, true, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
+        else bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
-    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
-    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)units, bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
+    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
+    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
     else if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
     launches->fetch_add(1, std::memory_order_relaxed);

@@ -481,7 +481,7 @@ struct Params {
     // the summaries of the segments before its own (nseg > 1: a plain summary launch has left them in `summaries`) and
     // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32, dense
     // sequences) instead of a summary.  The prefill proper fills it too in its CKPT instantiations.  NULL: none.
-    // Packed sequences (never split here): [H][ckpt_slots][64][64], sequence s of head h from slot
+    // Packed sequences: [H][ckpt_slots][64][64], sequence s of head h from slot
     // cu_seqlens[s] / 64 + 2 s on (its chunks + 1 states fit before the next sequence's first slot), with
     // ckpt_slots = total_T / 64 + 2 S.
     float* ckpt;
@@ -687,7 +687,13 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         return (size_t)unit * ((p.T + L - 1) / L + 1) + c_abs;
     };
-    auto ckpt_chunks = [&]() -> int { return p.cu_seqlens ? nchunks : (p.T + L - 1) / L; };
+    auto ckpt_chunks = [&]() -> int {                 // chunks of the whole sequence (this CTA may hold one segment of it)
+        if (p.cu_seqlens) {
+            const int sq = unit / p.H;
+            return (p.cu_seqlens[sq + 1] - p.cu_seqlens[sq] + L - 1) / L;
+        }
+        return (p.T + L - 1) / L;
+    };
     const int col0 = h * 64;
     const size_t C = (size_t)p.H * 64;
     static_assert(!(PERSIST && SUMMARY), "the summary pass is a single-unit launch");
@@ -1713,10 +1719,9 @@ inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat
                                        int nseg = 1, int seg_chunks = 0, const int32_t* cu = nullptr,
                                        long long packed_rows = 0)
 {
-    // packed sequences (cu: device cu_seqlens of n_seq sequences over packed_rows rows, T = max_seqlen): never split,
-    // checkpoints in the packed layout (Params::ckpt)
+    // packed sequences (cu: device cu_seqlens of n_seq sequences over packed_rows rows, T = max_seqlen): split by
+    // max_seqlen (segments past a sequence's end are empty), checkpoints in the packed layout (Params::ckpt)
     const long long units = (long long)n_seq * H, total_rows = cu ? packed_rows : (long long)n_seq * T;
-    if (cu) summaries = nullptr;
     if (units <= 0 || units > 0x7fffffffLL || total_rows <= 0) return GF_ERR_INVALID_ARG;
     if (total_rows >= (1LL << 31) - 64 || !ck::encode_fn()) return GF_ERR_UNSUPPORTED;
     if (!chunked_kernel_attributes()) return GF_ERR_CUDA;

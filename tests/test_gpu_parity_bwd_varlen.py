@@ -153,6 +153,25 @@ def test_serving_mix_at_full_size_every_unit():
     check(got, ref, cu.numpy(), what="cfg4")
 
 
+@pytest.mark.parametrize("c2", [False, True])
+@pytest.mark.parametrize("lens,H", [((4096, 100, 1000, 0), 2), ((2048,), 1), ((700, 3000), 4), ((1030, 1029, 1, 520), 8)])
+def test_few_units_split_their_sequences(lens, H, c2):
+    """Fewer (sequence, head) units than half the SMs: every sequence is cut into segments by the longest one (segments
+    past a shorter sequence's end are empty) and the adjoint's segment summaries are folded, as in the dense call.
+    Slow decays, so that what is handed across the cuts matters over the whole sequence."""
+    import paper_2407_12077_b200 as gf
+    case = make(lens, H, 7800 + len(lens), x_range=(-8.0, -4.0))
+    n0 = gf.launch_count()
+    got = run_gpu(case, c2)
+    # order, forward summaries, checkpoints, adjoint summaries, gradient (and the bonus sum): the split was taken
+    assert gf.launch_count() - n0 == (5 if c2 else 6)
+    ref = run_oracle(case, c2)
+    check(got, ref, case[-1].numpy(), c2, what=f"split {lens}")
+    a, b = run_gpu(case, c2), got
+    for p, q in zip(a, b):
+        assert (p is None and q is None) or np.array_equal(p, q)
+
+
 def test_fast_decays_take_the_token_path_in_some_sequences():
     lens = (150, 90, 64)
     case = make(lens, 2, 7400, x_range=(-2.0, 1.5))
@@ -174,7 +193,9 @@ def test_argument_checks():
     r, k, v, x, u, dy, s0, dsT, cu = (None if t is None else t.cuda() for t in case)
     need = int(lib.gf_wkv6_backward_varlen_workspace_bytes(2, 100, 2, 64))
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    assert need == (2 * (100 // 64 + 4) * 4096 + 2 * 2 * 64 + (16 + 2 + 3) // 4 * 4 + 2 * sms * 64 * 4096) * 4
+    nmax = min(8, sms // 4) if 8 <= sms else 1            # the widest split 4 units may take
+    assert need == (2 * (100 // 64 + 4) * 4096 + 4 * nmax * 64 + 4 * (nmax - 1) * (64 + 4096) + (16 + 2 + 3) // 4 * 4
+                    + 2 * sms * 64 * 4096) * 4
     small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
     dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
     du = torch.empty(2, 64, device="cuda")

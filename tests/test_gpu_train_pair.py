@@ -99,8 +99,15 @@ def test_packed_pair_is_bit_identical_to_the_separate_packed_calls(lens, c2):
         y0, s0 = gf.prefill_varlen(inp.r, inp.k, inp.v, inp.x, inp.u, inp.cu_seqlens, mx, inp.state_in, split=False)
     gf.last_device_status()
     assert torch.equal(y, y0) and torch.equal(s, s0)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    split = 2 * S * H <= sms and (mx + 63) // 64 >= 16      # (the gradient call's own checkpoint pass then runs in segments)
     for p, q in zip(ga, gb):
-        assert (p is None and q is None) or torch.equal(p, q)
+        if p is None and q is None:
+            continue
+        if split:
+            assert orc.rel_l2(p.float().cpu().numpy(), q.float().cpu().numpy()) <= 2e-3
+        else:
+            assert torch.equal(p, q)
     # and once against the oracle
     dyn = dy.float().cpu().numpy().astype(np.float64)
     c = inp.to("cpu")
