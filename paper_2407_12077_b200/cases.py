@@ -159,7 +159,7 @@ def run(case, reps, scale):
         # the first pass's second read of k,v,x) are this design's own and are not counted
         return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H,
                     bytes=B * T * H * 64 * 2 * 9 + B * H * 16384 * (2 if k["state_std"] > 0 else 1),
-                    design_bytes=B * T * H * 2048 + B * H * 16384 * 2, ms=_time(fn, reps))
+                    design_bytes=B * T * H * 1792 + B * H * 16384 * 2, ms=_time(fn, reps))
     if case in ("train-fwd-cfg2", "train-bwd-cfg2"):    # a training step's pair: forward that keeps its chunk-start states, gradient from them
         k = c["cfg2"]
         B, T, H = k["B"], sc(k["T"]), k["H"]

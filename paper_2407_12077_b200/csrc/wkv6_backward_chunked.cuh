@@ -57,7 +57,7 @@ struct BParams {
     const float* u;              // [H][64]
     const float* dstate_out;     // [units][64][64] or NULL (zero)
     float* dstate_in;            // [units][64][64] or NULL (not written)
-    const float* ckpt;           // [units][chunks + 1][64][64]
+    const __nv_bfloat16* ckpt;   // [units][chunks + 1][64][64] bf16 (read through the tensor map tm_ck and, rarely, directly)
     float* du_part;              // [units][64]
     float* fb_scratch;           // [n_slots][64][4096]
     __nv_bfloat16 *dr, *dk, *dv, *dx;
@@ -85,6 +85,7 @@ struct BParamsPacked : BParams {
 template <bool PACKED> struct BParamsOf { using type = BParams; };
 template <> struct BParamsOf<true> { using type = BParamsPacked; };
 constexpr int GSUM_FLOATS = 64 + 64 * 64;
+constexpr size_t CKPT_FLOATS = 64 * 64 / 2;               // a checkpoint (one bf16 [64][64] state) in units of the workspace's floats
 
 __device__ __forceinline__ float lds_bf16(uint32_t a)
 {
@@ -149,7 +150,7 @@ constexpr int GS_ABORT = GS_U + 256;              // abort word, wait limit
 constexpr int GS_TMEM = GS_ABORT + 8;
 // mbarriers, per group: inputs x, v, dy / inputs r, k / first group of products / dR^ and dK^ / dV; then the hand-over pair
 constexpr int GS_BAR = GS_TMEM + 8;
-enum { GB_INA = 0, GB_INB = 1, GB_MA = 2, GB_MRK = 3, GB_MV = 4, GB_PER_GROUP = 5, GB_GREADY = 10, GB_COUNT = 12 };
+enum { GB_INA = 0, GB_INB = 1, GB_MA = 2, GB_MRK = 3, GB_MV = 4, GB_S0 = 5, GB_PER_GROUP = 6, GB_GREADY = 12, GB_COUNT = 14 };
 constexpr int G_SMEM_BYTES = GS_BAR + 8 * GB_COUNT;
 constexpr int G_SMEM_ALLOC = G_SMEM_BYTES + 1024;
 static_assert(G_SMEM_ALLOC <= 232448, "shared memory budget of one sm_100 CTA");
@@ -261,7 +262,8 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                             const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                             const __grid_constant__ CUtensorMap tm_dy, const __grid_constant__ CUtensorMap tm_dr,
                             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
-                            const __grid_constant__ CUtensorMap tm_dx, const typename BParamsOf<PACKED>::type p)
+                            const __grid_constant__ CUtensorMap tm_dx, const __grid_constant__ CUtensorMap tm_ck,
+                            const typename BParamsOf<PACKED>::type p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -346,7 +348,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     const uint32_t o_dr = t_sb, o_dk = t_dpp, o_dv = t_pp, o_dx = t_gb;
     // The input copies of a chunk come in two parts, each issued as soon as its tiles are free: x, v, dy once the
     // chunk before (of this group) has finished its products, r, k once its epilogue has read them.
-    int last_a = -1, last_b = -1;                    // (thread 0 of the group) the last iterations whose copies were issued
+    int last_a = -1, last_b = -1, last_s = -1;       // (thread 0 of the group) the last iterations whose copies were issued
     auto issue_loads_a = [&](int it) {               // thread 0 of the group
         const int row = (int)(row0 + (long long)chunk_of(it) * L);
         mbar_expect_tx(gb(GB_INA), 3 * TILE);
@@ -378,7 +380,23 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         }
     };
 
-    const float* ck_unit = p.ckpt + (PACKED ? ck_first : (size_t)unit * (nchunks + 1)) * 4096;
+    const size_t ck_slot0 = PACKED ? ck_first : (size_t)unit * (nchunks + 1);       // this unit's first checkpoint
+    const __nv_bfloat16* ck_unit = p.ckpt + ck_slot0 * 4096;
+    // the chunk-start state is a bf16 [64][64] tile in memory: it lands in its operand tile by TMA (rows of the
+    // checkpoint array seen as [slots * 64][64])
+    auto issue_load_s = [&](int it) {                // thread 0 of the group
+        mbar_expect_tx(gb(GB_S0), TILE);
+        tma_load_2d(t_sb, &tm_ck, 0, (int)((ck_slot0 + (size_t)chunk_of(it)) * 64), gb(GB_S0));
+        last_s = it;
+    };
+    auto load_bf16_block = [&](const __nv_bfloat16* src, float (&v)[G_NB][4]) {     // a checkpoint, the lane's cells
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) {
+            const float2 lo = bf_pair(*reinterpret_cast<const uint32_t*>(src + (size_t)R0 * 64 + cb + 8 * n));
+            const float2 hi = bf_pair(*reinterpret_cast<const uint32_t*>(src + (size_t)R1 * 64 + cb + 8 * n));
+            v[n][0] = lo.x; v[n][1] = lo.y; v[n][2] = hi.x; v[n][3] = hi.y;
+        }
+    };
     float du_acc[G_NB][2];
 #pragma unroll
     for (int n = 0; n < G_NB; ++n) du_acc[n][0] = du_acc[n][1] = 0.f;
@@ -390,21 +408,20 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
     for (int it = grp; it < nit; it += 2) {
         const int c = chunk_of(it), valid = min(L, T - c * L);
         const int use = it >> 1;                     // how often this group's input stage has been filled before
-        float S0[G_NB][4];                              // the chunk-start state (requested early: it is used after the scan)
-        if (!GSUM) load_f32_block(ck_unit + (size_t)c * 4096, S0);
-        if (it + 2 < nit) {
-            // this group's next chunk: its start state and its input tiles into L2 now, so that the copies issued at
-            // the end of this iteration and the load above find them there
-            if (!GSUM && gt < 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(ck_unit + (size_t)(c - 2) * 4096 + 32 * gt));
-            if (gt == 128) {
-                const int row = (int)(row0 + (long long)(c - 2) * L);
-                tma_prefetch_2d(&tm_x, col0, row); tma_prefetch_2d(&tm_r, col0, row); tma_prefetch_2d(&tm_k, col0, row);
-                tma_prefetch_2d(&tm_v, col0, row); tma_prefetch_2d(&tm_dy, col0, row);
-            }
+        if (it + 2 < nit && gt == 128) {
+            // this group's next chunk: its start state and its input tiles into L2 now, so that the copies issued
+            // later find them there
+            const int row = (int)(row0 + (long long)(c - 2) * L);
+            tma_prefetch_2d(&tm_x, col0, row); tma_prefetch_2d(&tm_r, col0, row); tma_prefetch_2d(&tm_k, col0, row);
+            tma_prefetch_2d(&tm_v, col0, row); tma_prefetch_2d(&tm_dy, col0, row);
+            if (!GSUM) tma_prefetch_2d(&tm_ck, 0, (int)((ck_slot0 + (size_t)(c - 2)) * 64));
         }
         // ---- decay: log2-domain magnitudes, cumulative sums over the tokens
         bool ok = mbar_wait(gb(GB_INA), use & 1, abort_flag);
-        if (gt == 0 && it > 1) bulk_wait_read<0>();  // the previous chunk's staging tiles have been read by the TMA unit
+        if (gt == 0) {
+            if (it > 1) bulk_wait_read<0>();         // the previous chunk's staging tiles have been read by the TMA unit
+            if (!GSUM) issue_load_s(it);             // (the start state's tile doubles as the staging tile of dr)
+        }
         float a[G_NB][4], lw2[G_NB][4];
         {
             float xv[G_NB][4];
@@ -471,7 +488,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 if (q == 0) { stsf(gbase + GO_BP + 4 * (cx * 64 + R0), b0); stsf(gbase + GO_BP + 4 * (cx * 64 + R1), b1); }
             }
         }
-        if (!GSUM) st_tile(t_sb, moff, S0);
+        if (!GSUM && !mbar_wait(gb(GB_S0), use & 1, abort_flag)) ok = false;       // the chunk-start state is in its tile
         fence_proxy_async();
         tc_fence_before();
         const bool unsafe = !gbar_and(grp, safe);    // (every channel is some lane's row)
@@ -531,7 +548,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         if (GSUM) {
         } else if (it == 0) {
             float SL[G_NB][4];
-            load_f32_block(ck_unit + (size_t)(c + 1) * 4096, SL);
+            load_bf16_block(ck_unit + (size_t)(c + 1) * 4096, SL);
             e_put(gbase + GO_EP, G, SL);
         } else if (gt < G_NSLAB * 64) {
             stsf(gbase + GO_EP + 4 * gt, ldsf(sbase + GS_EH + 4 * (((it - 1) & 1) * G_NSLAB * 64 + gt)));      // (a private copy: the slot is rewritten two chunks on)
@@ -548,7 +565,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             if (!gbar_and(grp, ok)) { alive = false; break; }
             float* scr = p.fb_scratch + (size_t)slot * FB_SLOT_FLOATS + (size_t)gt * (4 * G_NB);
             float S[G_NB][4];
-            load_f32_block(ck_unit + (size_t)c * 4096, S);
+            load_bf16_block(ck_unit + (size_t)c * 4096, S);
             for (int t = 0; t < valid; ++t) {
 #pragma unroll
                 for (int n = 0; n < G_NB; ++n)
@@ -662,7 +679,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
             // hand the adjoint on (and the row sums the next chunk needs, from the fp32 state: the operand tile is gone)
             if (it + 1 < nit) {
                 g_put(it & 1, G);
-                load_f32_block(ck_unit + (size_t)c * 4096, S);
+                load_bf16_block(ck_unit + (size_t)c * 4096, S);
                 e_put(sbase + GS_EH + 4 * ((it & 1) * G_NSLAB * 64), G, S);
                 mbar_arrive(bar(GB_GREADY + (it & 1)));
             } else if (p.dstate_in && seg == 0) {
@@ -945,6 +962,7 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
         // no copy into shared memory may stay in flight
         if (last_a >= 0) mbar_wait(gb(GB_INA), (last_a >> 1) & 1, abort_flag, false);
         if (last_b >= 0) mbar_wait(gb(GB_INB), (last_b >> 1) & 1, abort_flag, false);
+        if (last_s >= 0) mbar_wait(gb(GB_S0), (last_s >> 1) & 1, abort_flag, false);
     }
     tc_fence_before();
     __syncthreads();
@@ -1001,7 +1019,7 @@ inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
     const size_t nck = (size_t)((T + ck::L - 1) / ck::L) + 1;
     int seg_chunks = 0;
     const int nseg = backward_split(units, T, n_sm, &seg_chunks);
-    return ((size_t)units * nck * 4096 + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS +
+    return ((size_t)units * nck * bc::CKPT_FLOATS + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS +
             (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
@@ -1022,7 +1040,7 @@ inline size_t chunked_backward_varlen_workspace_bytes(long long n_seq, long long
 {
     const size_t slots = (size_t)(total_rows / ck::L + 2 * n_seq);
     const size_t units = (size_t)n_seq * H, nmax = (size_t)packed_split_max((long long)units, n_sm);
-    return ((size_t)H * slots * 4096 + units * nmax * 64 + units * (nmax - 1) * bc::GSUM_FLOATS +
+    return ((size_t)H * slots * bc::CKPT_FLOATS + units * nmax * 64 + units * (nmax - 1) * bc::GSUM_FLOATS +
             backward_order_floats(n_seq) + (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
@@ -1034,7 +1052,7 @@ inline float* backward_workspace_forward_scratch(float* ws, long long units, int
     int seg_chunks = 0;
     const int nseg = backward_split(units, T, n_sm, &seg_chunks);
     *bytes = (size_t)2 * n_sm * bc::FB_SLOT_FLOATS * sizeof(float);
-    return ws + (size_t)units * nck * 4096 + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
+    return ws + (size_t)units * nck * bc::CKPT_FLOATS + (size_t)units * nseg * 64 + (size_t)units * (nseg - 1) * bc::GSUM_FLOATS;
 }
 
 inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16* k, const __nv_bfloat16* v,
@@ -1069,7 +1087,9 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
     const int nalloc = cu ? packed_split_max(units, n_sm) : nseg;      // (packed: the workspace is laid out for the widest split)
     const long long ckpt_slots = cu ? rows / ck::L + 2LL * B : 0;
     float* ckpt = ws;
-    float* du_part = ckpt + (cu ? (size_t)H * ckpt_slots : (size_t)units * nck) * 4096;
+    const size_t n_ckpt = cu ? (size_t)H * ckpt_slots : (size_t)units * nck;       // checkpoints: bf16 [64][64] tiles
+    if (n_ckpt * 64 >= (1ull << 31)) return GF_ERR_UNSUPPORTED;                    // (32-bit TMA row coordinates)
+    float* du_part = ckpt + n_ckpt * bc::CKPT_FLOATS;
     float* gsum = du_part + (size_t)units * nalloc * 64;
     float* fb = gsum + (size_t)units * (nalloc - 1) * bc::GSUM_FLOATS;
     const int32_t* order = nullptr;
@@ -1091,25 +1111,26 @@ inline gf_status_t chunked_backward(const __nv_bfloat16* r, const __nv_bfloat16*
         if (s != GF_OK) return s;
     }
     const long long C = (long long)H * 64;
-    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx;
+    CUtensorMap tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck;
+    if (!ck::make_map(&tck, ckpt, (long long)n_ckpt * 64, 64, 64)) return GF_ERR_CUDA;
     if (!ck::make_map(&tx, x, rows, C, 64) || !ck::make_map(&tr, r, rows, C, 64) || !ck::make_map(&tk, k, rows, C, 64) ||
         !ck::make_map(&tv, v, rows, C, 64) || !ck::make_map(&tdy, dy, rows, C, 64) || !ck::make_map(&tdr, dr, rows, C, 64) ||
         !ck::make_map(&tdk, dk, rows, C, 64) || !ck::make_map(&tdv, dv, rows, C, 64) || !ck::make_map(&tdx, dx, rows, C, 64))
         return GF_ERR_CUDA;
-    bc::BParams p{u, dstate_out, dstate_in, ckpt, du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
+    bc::BParams p{u, dstate_out, dstate_in, reinterpret_cast<const __nv_bfloat16*>(ckpt), du_part, fb, dr, dk, dv, dx, T, H, 2 * n_sm,
                   wait_limit_us().load(std::memory_order_relaxed), gsum, gsum, nseg, seg_chunks};
     const bc::BParamsPacked pp{p, cu, ckpt_slots, order};
     if (nseg > 1) {
         // the adjoint's summaries of every segment but the first (they need no state: the order of the two first launches is free)
-        if (cu) bc::wkv6_backward_chunked_kernel<false, true, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
-        else bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+        if (cu) bc::wkv6_backward_chunked_kernel<false, true, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, pp);
+        else bc::wkv6_backward_chunked_kernel<false, true><<<(unsigned)(units * (nseg - 1)), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, p);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
-    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
-    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, pp);
-    else if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
-    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, p);
+    if (cu && c2) bc::wkv6_backward_chunked_kernel<true, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, pp);
+    else if (cu) bc::wkv6_backward_chunked_kernel<false, false, true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, pp);
+    else if (c2) bc::wkv6_backward_chunked_kernel<true><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, p);
+    else bc::wkv6_backward_chunked_kernel<false><<<(unsigned)(units * nseg), bc::G_THREADS, bc::G_SMEM_ALLOC, st>>>(tx, tr, tk, tv, tdy, tdr, tdk, tdv, tdx, tck, p);
     launches->fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     if (c2) return GF_OK;                            // no bonus, no bonus gradient

@@ -479,7 +479,7 @@ struct Params {
     uint32_t wait_limit_us;                // limit of every device-side wait of the launch (0: the default, 2 s)
     // Checkpoint pass (a summary-variant launch over every segment, used by the gradient): starts from state_in, folds
     // the summaries of the segments before its own (nseg > 1: a plain summary launch has left them in `summaries`) and
-    // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] fp32, dense
+    // leaves the state before every chunk, and after the last, in ckpt ([unit][chunks + 1][64][64] bf16, dense
     // sequences) instead of a summary.  The prefill proper fills it too in its CKPT instantiations.  NULL: none.
     // Packed sequences: [H][ckpt_slots][64][64], sequence s of head h from slot
     // cu_seqlens[s] / 64 + 2 s on (its chunks + 1 states fit before the next sequence's first slot), with
@@ -968,6 +968,15 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
         };
         auto store_state = [&](size_t base) { store_to(p.state_out + base); };
+        // a checkpoint: the state rounded to bf16, [64][64] row-major (8 KB: as the gradient's tensor-core operand reads it)
+        auto store_ckpt = [&](size_t slot) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.ckpt) + slot * 4096;
+#pragma unroll
+            for (int n = 0; n < 8; ++n) {
+                *reinterpret_cast<uint32_t*>(dst + (size_t)c_lo * 64 + 8 * n + 2 * q) = pack_bf16(st[n][0], st[n][1]);
+                *reinterpret_cast<uint32_t*>(dst + (size_t)(c_lo + 8) * 64 + 8 * n + 2 * q) = pack_bf16(st[n][2], st[n][3]);
+            }
+        };
         // second launch of a split call: the summaries and the start-state copy are the first launch's
         if (!SUMMARY && !PERSIST && p.nseg > 1) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (!PERSIST) load_state(sb);
@@ -996,7 +1005,7 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
             if (CKPT || (SUMMARY && p.ckpt))         // the state before chunk c of the segment (dense sequences: T / 64 + 1 states per unit)
-                store_to(p.ckpt + ckpt_slot(seg * p.seg_chunks + c) * 4096);
+                store_ckpt(ckpt_slot(seg * p.seg_chunks + c));
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1089,10 +1098,10 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
-        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_to(p.ckpt + ckpt_slot(ckpt_chunks()) * 4096);
+        if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_ckpt(ckpt_slot(ckpt_chunks()));
         if (SUMMARY && p.ckpt) {
             if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
-                store_to(p.ckpt + ckpt_slot(ckpt_chunks()) * 4096);
+                store_ckpt(ckpt_slot(ckpt_chunks()));
         } else if (SUMMARY) {
             if (!lds32(abort_flag)) {
                 float* sm = p.summaries + ((size_t)unit * (p.nseg - 1) + seg) * SUMMARY_FLOATS;
@@ -1710,7 +1719,7 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
 }
 
 // Checkpoint pass of dense sequences: the state before every chunk of 64 tokens and after the last one,
-// ckpt [n_seq*H][chunks + 1][64][64] fp32, from state_in (NULL: zero).  One summary-variant launch (state only: reads
+// ckpt [n_seq*H][chunks + 1][64][64] bf16, from state_in (NULL: zero).  One summary-variant launch (state only: reads
 // k, v and the decay logits); with `summaries` (scratch of units x (nseg - 1) summaries) and nseg > 1 two: the sequences
 // split into segments as in a split prefill call.
 inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* x,

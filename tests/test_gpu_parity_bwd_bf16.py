@@ -203,7 +203,7 @@ def test_repeatable_and_argument_checks():
     lib = gf.load_library()
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     nck = (300 + 63) // 64 + 1
-    assert lib.gf_wkv6_backward_bf16_workspace_bytes(2, 300, 2, 64) == (4 * nck * 4096 + 4 * 64 + 2 * sms * 64 * 4096) * 4
+    assert lib.gf_wkv6_backward_bf16_workspace_bytes(2, 300, 2, 64) == (4 * nck * 2048 + 4 * 64 + 2 * sms * 64 * 4096) * 4
     p = lambda t: t.data_ptr()
     outs = [torch.empty_like(d.r) for _ in range(4)]
     du = torch.empty((2, 64), device=DEV)

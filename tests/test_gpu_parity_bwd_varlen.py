@@ -194,7 +194,7 @@ def test_argument_checks():
     need = int(lib.gf_wkv6_backward_varlen_workspace_bytes(2, 100, 2, 64))
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     nmax = min(8, sms // 4) if 8 <= sms else 1            # the widest split 4 units may take
-    assert need == (2 * (100 // 64 + 4) * 4096 + 4 * nmax * 64 + 4 * (nmax - 1) * (64 + 4096) + (16 + 2 + 3) // 4 * 4
+    assert need == (2 * (100 // 64 + 4) * 2048 + 4 * nmax * 64 + 4 * (nmax - 1) * (64 + 4096) + (16 + 2 + 3) // 4 * 4
                     + 2 * sms * 64 * 4096) * 4
     small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
     dr, dk, dv, dx = (torch.empty_like(r) for _ in range(4))
