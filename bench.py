@@ -372,10 +372,10 @@ def main():
                 ("prefill_c2", "cfg2-c2", "gf_wkv6_prefill_c2 with the second-value tensor, cfg2 shape (768 B per token*head)"),
                 ("key_compress", "kc-cfg2", "gf_gold_key_compress 65536 x 2048 -> 128"),
                 ("decay_logit", "dl-cfg2", "gf_c2_decay_logit, 65536 tokens x 2048 channels, ranks 32 and 64 (x read, d written)"),
-                ("backward", "bwd-cfg2", "gf_wkv6_backward, cfg2 shape: checkpoint pass + chunked gradient kernel, two chunks in flight per SM (1152 B per token*head counted; the design moves 2048)"),
+                ("backward", "bwd-cfg2", "gf_wkv6_backward, cfg2 shape: checkpoint pass + chunked gradient kernel, two chunks in flight per SM (1152 B per token*head counted; the design moves 1792)"),
                 ("backward_long_context", "bwd-cfg3", "gf_wkv6_backward, B=1 T=131072 H=32: 32 units, sequences split 4-way with the adjoint's segment summaries (5 launches)"),
                 ("backward_packed", "bwd-cfg4", "gf_wkv6_backward_varlen, the serving mix's shape (64 packed sequences of 128..4096 tokens, 32 heads: 2048 units, longest first)"),
-                ("train_forward", "train-fwd-cfg2", "gf_wkv6_prefill_train, cfg2 shape: the prefill that also keeps its chunk-start states (256 B per token*head more, not counted)"),
+                ("train_forward", "train-fwd-cfg2", "gf_wkv6_prefill_train, cfg2 shape: the prefill that also keeps its chunk-start states (128 B per token*head more, not counted)"),
                 ("train_backward", "train-bwd-cfg2", "gf_wkv6_backward_saved, cfg2 shape: the gradient kernel alone, from the states the forward pass kept"),
                 ("decode_step", "cfg4-decode", "gf_wkv6_step, 64 sequences x 32 heads, 64 steps per graph replay (states stay in L2)"),
                 ("decode_step_layer_stack", "cfg4-decode-layers", "gf_wkv6_step over 12 layers with their own states (streams from HBM)")):

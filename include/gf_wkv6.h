@@ -142,7 +142,7 @@ GF_API size_t gf_wkv6_backward_workspace_bytes(int B, int T, int H, int N);
  * checkpoint pass of the forward kernel.  A chunk in which some channel decays by more than 2^-96 is processed token
  * by token in fp32 instead, so any decay logit is accepted (x = +inf leaves dx undefined, as in the formula).
  * `workspace`: caller-owned DEVICE buffer of at least gf_wkv6_backward_bf16_workspace_bytes(B,T,H,N) bytes, 16-byte
- * aligned (one 64x64 fp32 state per chunk and unit, plus 2 MiB per SM for the token-by-token path);
+ * aligned (one 64x64 bf16 state per chunk and unit, plus 2 MiB per SM for the token-by-token path);
  * GF_ERR_WORKSPACE if absent or too small.  GF_ERR_UNSUPPORTED for B*T >= 2^31 - 64 rows or N != 64.  dstate_in must
  * not be dstate_out (GF_ERR_INVALID_ARG).  Enqueues three
  * kernels on `stream` (five when B*H is less than half the SMs: the sequences are then cut into segments that run
@@ -200,7 +200,7 @@ GF_API gf_status_t gf_wkv6_backward_c2_saved(const void *r, const void *k, const
  * [S][H][N][N] fp32; du [H][N] fp32 is summed over the sequences in index order.  A sequence without tokens hands its
  * state gradient through.  `workspace`: caller-owned DEVICE buffer of at least
  * gf_wkv6_backward_varlen_workspace_bytes(S,total_T,H,N) bytes, 16-byte aligned (H * (total_T / 64 + 2 S) states of
- * 64x64 fp32, plus 2 MiB per SM, plus the segment summaries of the widest split when S*H is less than half the SMs);
+ * 64x64 bf16, plus 2 MiB per SM, plus the segment summaries of the widest split when S*H is less than half the SMs);
  * GF_ERR_WORKSPACE if absent or too small.  One CTA per (sequence, head), the longest sequences first; with S*H less
  * than half the SMs every sequence is cut into segments by max_seqlen, as in the dense call (segments past a shorter
  * sequence's end do no work): four kernels on `stream` (three for the Finch-C2 form), six resp. five when split, nothing allocated, no synchronisation, deterministic.

@@ -155,7 +155,7 @@ def run(case, reps, scale):
         ws = torch.empty(gf.backward_workspace_bytes(B, T, H, 64), dtype=torch.uint8, device=DEV)
         fn = lambda: gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, None, workspace=ws)
         # algorithmic traffic: r,k,v,x,dy read and dr,dk,dv,dx written once (bf16), the start state read, its adjoint
-        # written; the checkpoints (one fp32 state per chunk, written by the first pass and read by the second, and
+        # written; the checkpoints (one bf16 state per chunk, written by the first pass and read by the second, and
         # the first pass's second read of k,v,x) are this design's own and are not counted
         return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H,
                     bytes=B * T * H * 64 * 2 * 9 + B * H * 16384 * (2 if k["state_std"] > 0 else 1),
@@ -173,7 +173,7 @@ def run(case, reps, scale):
         else:
             fn = lambda: gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, None, workspace=ws, saved=True)
             nbytes = B * T * H * 64 * 2 * 9 + B * H * 16384
-        # (the checkpoints, 256 B per token*head written by the one and read by the other, are the design's own)
+        # (the checkpoints, 128 B per token*head written by the one and read by the other, are the design's own)
         return dict(case=case, shape=f"B={B} T={T} H={H} bf16", units=B * T * H, bytes=nbytes, ms=_time(fn, reps))
     if case == "bwd-cfg4":       # gradient of the packed serving-mix prefill (64 sequences of 128..4096 tokens)
         k = c["cfg4"]

@@ -14,7 +14,8 @@
 // (log w_s enters a_t for every t >= s: R^_t through a_{t-1}, K^_t through a_t, D through a_L; the D term is
 // rowsum(G_L * diag(D)(S_0 + K^^T V)) = rowsum(G_L * S_L).)
 // Nine 64x64x64 bf16 tcgen05 products per chunk, accumulators in tensor memory.  The chunk-start states S_0 come from
-// a checkpoint pass of the forward kernel (state only), one 64x64 fp32 block per chunk.
+// a checkpoint pass of the forward kernel (state only), one 64x64 bf16 block per chunk: the operand tile of dY S_0^T,
+// which the kernel fetches by TMA (the state is rounded to bf16 at that use in any case).
 //
 // Two chunks are in flight per CTA.  A chunk's phases (decay -> cumulative sum -> operands -> products -> masks ->
 // products -> epilogue -> suffix sums) depend on one another and each keeps a different pipe busy, so one set of warps
@@ -1023,7 +1024,7 @@ inline size_t chunked_backward_workspace_bytes(long long units, int T, int n_sm)
             (size_t)2 * n_sm * bc::FB_SLOT_FLOATS) * sizeof(float);
 }
 
-// The same for packed sequences (never split): checkpoints in the packed layout, [H][total_rows / 64 + 2 S] states.
+// The same for packed sequences: checkpoints in the packed layout, [H][total_rows / 64 + 2 S] states.
 inline size_t backward_order_floats(long long n_seq)       // a counter's 64 bytes and the sequence order, in floats, 16-byte granular
 {
     return (size_t)((ORDER_OFFSET / 4 + n_seq + 3) / 4 * 4);
