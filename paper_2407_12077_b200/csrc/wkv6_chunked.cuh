@@ -648,7 +648,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_x,
                     const __grid_constant__ CUtensorMap tm_y16, const __grid_constant__ CUtensorMap tm_u2_16,
-                    const Params p)
+                    const Params p, const __grid_constant__ CUtensorMap tm_ck16)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -996,16 +996,32 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
         }
         float dprod_lo = 1.f, dprod_hi = 1.f;    // summary pass: decay product of the segment for this lane's two rows
         int fb_uses = 0;                         // chunks that took the token-by-token path so far
+        // Checkpoints of the chunk-start states: the bf16 copy of the state in its operand tile (the pair of tiles is
+        // idle in a summary pass and written for the checkpoints' sake there) is what the gradient reads, so each state
+        // warp sends its 16 rows of the tile to the checkpoint array by TMA (tm_ck16: the array as [slots * 64][64]).
+        constexpr bool CK_TMA = CKPT || SUMMARY;
+        const bool ck_on = CKPT || (SUMMARY && p.ckpt);
+        auto ckpt_tile = [&](int tile, int c_abs) {      // after the tile's rows are written, fenced and the warp synchronised
+            if (lane == 0) {
+                tma_store_2d(&tm_ck16, 0, (int)(ckpt_slot(c_abs) * 64) + 16 * sp, sbase + OFF_SB + tile * TILE + 16 * sp * 128);
+                bulk_commit();
+            }
+        };
         if (!PERSIST && !SUMMARY && nchunks > 0) {
             store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
             fence_proxy_async();
             __syncwarp();
             mbar_arrive_if(bar(BAR_S_READY), lane == 0);
+            if (CKPT) ckpt_tile(0, seg * p.seg_chunks);
+        }
+        if (SUMMARY && ck_on && nchunks > 0) {
+            store_acc_bf16(sbase + OFF_SB, 16 * sp, st, lane);
+            fence_proxy_async();
+            __syncwarp();
+            ckpt_tile(0, seg * p.seg_chunks);
         }
         for (int c = 0; PERSIST || c < nchunks; ++c) {
             const int tb = c & 1, pt = (c >> 1) & 1, sd = c & (NSIDE - 1);
-            if (CKPT || (SUMMARY && p.ckpt))         // the state before chunk c of the segment (dense sequences: T / 64 + 1 states per unit)
-                store_ckpt(ckpt_slot(seg * p.seg_chunks + c));
             if (!mbar_wait(bar(BAR_F_FULL + tb), pt, abort_flag)) break;
             tc_fence_after();
             const Chunk ck = chunk_at(c);
@@ -1064,6 +1080,8 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
                 if (!SUMMARY && c >= 1 && !mbar_wait(bar(BAR_B_DONE + (tb ^ 1)), ((c - 1) >> 1) & 1, abort_flag)) break;
                 next_tile_free = true;
                 // the fp32 copy overlays the bf16 rows of the other state warps: all of them have stored theirs first
+                // (and the checkpoint copies that read those rows have left shared memory)
+                if (CK_TMA && ck_on && lane == 0) bulk_wait_read<0>();
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_SPRE), lane == 0);
                 if (!mbar_wait(bar(BAR_SPRE), fb_uses & 1, abort_flag)) break;
@@ -1091,13 +1109,28 @@ wkv6_chunked_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_const
             if (!SUMMARY && ck.rem > 0) {
                 const int nb = tb ^ 1;
                 if (!next_tile_free && !mbar_wait(bar(BAR_B_DONE + nb), ((c - 1) >> 1) & 1, abort_flag)) break;
+                if (CKPT) {                          // the checkpoint copy of chunk c - 1 has finished reading this tile
+                    if (lane == 0) bulk_wait_read<1>();
+                    __syncwarp();
+                }
                 store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
                 fence_proxy_async();
                 __syncwarp();
                 mbar_arrive_if(bar(BAR_S_READY + nb), lane == 0);
+                if (CKPT) ckpt_tile(nb, seg * p.seg_chunks + c + 1);
+            }
+            if (SUMMARY && ck_on && ck.rem > 0) {    // (no product reads these tiles in a summary pass)
+                const int nb = tb ^ 1;
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+                store_acc_bf16(sbase + OFF_SB + nb * TILE, 16 * sp, st, lane);
+                fence_proxy_async();
+                __syncwarp();
+                ckpt_tile(nb, seg * p.seg_chunks + c + 1);
             }
             if (PERSIST && ck.rem == 0 && p.state_out && !lds32(abort_flag)) store_state((size_t)ck.unit * 4096);
         }
+        if (CK_TMA && ck_on && lane == 0) bulk_wait<0>();          // this warp's checkpoint copies have reached memory
         if (CKPT && seg == p.nseg - 1 && !lds32(abort_flag)) store_ckpt(ckpt_slot(ckpt_chunks()));
         if (SUMMARY && p.ckpt) {
             if (seg == p.nseg - 1 && !lds32(abort_flag))     // the state after the last token
@@ -1623,20 +1656,24 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         if (nseg > 1 && units * nseg > 0x7fffffffLL) nseg = 1;
     }
     ck::Params p{r, k, v, x, y, u, state_in, state_out, cu, T, H, scratch, seg_chunks, nseg, u2, c2};
+    CUtensorMap tck = ty;                            // (read only by the launches that keep checkpoints)
     if (nseg > 1 && state_in) p.state_copy = scratch + (size_t)units * (nseg - 1) * ck::SUMMARY_FLOATS;
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     if (ckpt) {
         // a training step's forward pass: one CTA per unit and segment, the chunk-start states kept for the gradient
         p.ckpt_slots = cu ? total_rows / ck::L + 2LL * n_seq : 0;
+        const long long n_ckpt = cu ? (long long)H * p.ckpt_slots : units * ((T + ck::L - 1) / ck::L + 1);
+        if (n_ckpt * 64 >= (1LL << 31)) return GF_ERR_UNSUPPORTED;
+        if (!ck::make_map(&tck, ckpt, n_ckpt * 64, 64, 16)) return GF_ERR_CUDA;      // the checkpoints as [slots * 64][64] bf16
         if (nseg > 1) {
-            if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-            else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+            if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
+            else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
             launches->fetch_add(1, std::memory_order_relaxed);
             if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
         }
         p.ckpt = ckpt;
-        if (c2) ck::wkv6_chunked_kernel<false, true, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-        else ck::wkv6_chunked_kernel<false, false, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        if (c2) ck::wkv6_chunked_kernel<false, true, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
+        else ck::wkv6_chunked_kernel<false, false, false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
         launches->fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }
@@ -1661,14 +1698,14 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
             launches->fetch_add(1, std::memory_order_relaxed);
             if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
         }
-        if (c2) ck::wkv6_chunked_kernel<false, true, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-        else ck::wkv6_chunked_kernel<false, false, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        if (c2) ck::wkv6_chunked_kernel<false, true, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
+        else ck::wkv6_chunked_kernel<false, false, true><<<(unsigned)n_sm, ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
         launches->fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }
     if (nseg > 1) {
-        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
+        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
@@ -1684,13 +1721,13 @@ inline gf_status_t chunked_prefill(const __nv_bfloat16* r, const __nv_bfloat16* 
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const cudaError_t e = c2 ? cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, true, false>, tr, tk, tv, tx, ty, tu2, p)
-                                 : cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, false, false>, tr, tk, tv, tx, ty, tu2, p);
+        const cudaError_t e = c2 ? cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, true, false>, tr, tk, tv, tx, ty, tu2, p, tck)
+                                 : cudaLaunchKernelEx(&cfg, ck::wkv6_chunked_kernel<false, false, false>, tr, tk, tv, tx, ty, tu2, p, tck);
         launches->fetch_add(1, std::memory_order_relaxed);
         return e == cudaSuccess ? GF_OK : GF_ERR_CUDA;
     }
-    if (c2) ck::wkv6_chunked_kernel<false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
-    else ck::wkv6_chunked_kernel<false, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p);
+    if (c2) ck::wkv6_chunked_kernel<false, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
+    else ck::wkv6_chunked_kernel<false, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tr, tk, tv, tx, ty, tu2, p, tck);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
@@ -1711,9 +1748,10 @@ inline gf_status_t chunked_summary(const __nv_bfloat16* k, const __nv_bfloat16* 
     // two nominal segments of which the first covers the whole sequence: the summary launch handles
     // every segment but the last
     ck::Params p{nullptr, k, v, x, nullptr, nullptr, nullptr, nullptr, nullptr, T, H, summary, (T + ck::L - 1) / ck::L, 2, nullptr, c2};
+    const CUtensorMap tck = tdummy;
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
-    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
-    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
+    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)units, ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
@@ -1743,17 +1781,21 @@ inline gf_status_t chunked_checkpoints(const __nv_bfloat16* k, const __nv_bfloat
     ck::Params p{nullptr, k, v, x, nullptr, nullptr, state_in, nullptr, cu, T, H, summaries, seg_chunks, nseg, nullptr, c2};
     p.wait_limit_us = wait_limit_us().load(std::memory_order_relaxed);
     p.ckpt_slots = cu ? total_rows / ck::L + 2LL * n_seq : 0;
+    CUtensorMap tck;                                 // the checkpoints as [slots * 64][64] bf16, 16 rows per copy
+    const long long n_ckpt = cu ? (long long)H * p.ckpt_slots : units * ((T + ck::L - 1) / ck::L + 1);
+    if (n_ckpt * 64 >= (1LL << 31)) return GF_ERR_UNSUPPORTED;
+    if (!ck::make_map(&tck, ckpt, n_ckpt * 64, 64, 16)) return GF_ERR_CUDA;
     if (nseg > 1) {
         // few units: the segments' summaries first (every segment but the last, from a zero state), then every segment
         // side by side from its folded start state, this time keeping the states
-        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
-        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+        if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
+        else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * (nseg - 1)), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
         launches->fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return GF_ERR_CUDA;
     }
     p.ckpt = ckpt;
-    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
-    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p);
+    if (c2) ck::wkv6_chunked_kernel<true, true><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
+    else ck::wkv6_chunked_kernel<true, false><<<(unsigned)(units * nseg), ck::THREADS, ck::SMEM_ALLOC, st>>>(tk, tk, tv, tx, tdummy, tdummy, p, tck);
     launches->fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? GF_OK : GF_ERR_CUDA;
 }
