@@ -217,37 +217,60 @@ template <bool REV>
 __device__ __forceinline__ bool scan_rows(float (&v)[G_NB][4], uint32_t tot, int grp, int sp, int cb, int lane, bool ok)
 {
     const int g = lane >> 2, q = lane & 3;           // (cb: the lane's first column, a multiple of 2)
+    // (the additions run on the pairs of neighbouring columns: one two-lane instruction for two cells)
 #pragma unroll
     for (int d = 4; d < 32; d <<= 1) {
+        const bool take = REV ? lane + d < 32 : lane >= d;
 #pragma unroll
         for (int n = 0; n < G_NB; ++n)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float o = REV ? __shfl_down_sync(0xffffffffu, v[n][e], d) : __shfl_up_sync(0xffffffffu, v[n][e], d);
-                if (REV ? lane + d < 32 : lane >= d) v[n][e] += o;
+            for (int h = 0; h < 2; ++h) {
+                float2 o;
+                o.x = REV ? __shfl_down_sync(0xffffffffu, v[n][2 * h], d) : __shfl_up_sync(0xffffffffu, v[n][2 * h], d);
+                o.y = REV ? __shfl_down_sync(0xffffffffu, v[n][2 * h + 1], d) : __shfl_up_sync(0xffffffffu, v[n][2 * h + 1], d);
+                if (take) {
+                    const float2 r = add2(make_float2(v[n][2 * h], v[n][2 * h + 1]), o);
+                    v[n][2 * h] = r.x; v[n][2 * h + 1] = r.y;
+                }
             }
     }
 #pragma unroll
-    for (int n = 0; n < G_NB; ++n)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            if (REV) v[n][e] += __shfl_sync(0xffffffffu, v[n][2 + e], q);
-            else v[n][2 + e] += __shfl_sync(0xffffffffu, v[n][e], 28 + q);
+    for (int n = 0; n < G_NB; ++n) {
+        float2 o;
+        if (REV) {
+            o.x = __shfl_sync(0xffffffffu, v[n][2], q); o.y = __shfl_sync(0xffffffffu, v[n][3], q);
+            const float2 r = add2(make_float2(v[n][0], v[n][1]), o);
+            v[n][0] = r.x; v[n][1] = r.y;
+        } else {
+            o.x = __shfl_sync(0xffffffffu, v[n][0], 28 + q); o.y = __shfl_sync(0xffffffffu, v[n][1], 28 + q);
+            const float2 r = add2(make_float2(v[n][2], v[n][3]), o);
+            v[n][2] = r.x; v[n][3] = r.y;
         }
+    }
     if (g == (REV ? 0 : 7)) {
 #pragma unroll
         for (int n = 0; n < G_NB; ++n)
             stsf2(tot + 4 * (sp * 64 + cb + 8 * n), REV ? make_float2(v[n][0], v[n][1]) : make_float2(v[n][2], v[n][3]));
     }
     ok = gbar_and(grp, ok);
+    // the totals of the row groups before (after) this one: summed first, then added to both rows
+    float2 t[G_NB];
+#pragma unroll
+    for (int n = 0; n < G_NB; ++n) t[n] = make_float2(0.f, 0.f);
+    bool any = false;
 #pragma unroll
     for (int o = 0; o < 4; ++o) {
         if (REV ? o > sp : o < sp) {
 #pragma unroll
-            for (int n = 0; n < G_NB; ++n) {
-                const float2 t = ldsf2(tot + 4 * (o * 64 + cb + 8 * n));
-                v[n][0] += t.x; v[n][1] += t.y; v[n][2] += t.x; v[n][3] += t.y;
-            }
+            for (int n = 0; n < G_NB; ++n) t[n] = add2(t[n], ldsf2(tot + 4 * (o * 64 + cb + 8 * n)));
+            any = true;
+        }
+    }
+    if (any) {
+#pragma unroll
+        for (int n = 0; n < G_NB; ++n) {
+            const float2 lo = add2(make_float2(v[n][0], v[n][1]), t[n]), hi = add2(make_float2(v[n][2], v[n][3]), t[n]);
+            v[n][0] = lo.x; v[n][1] = lo.y; v[n][2] = hi.x; v[n][3] = hi.y;
         }
     }
     return ok;
