@@ -227,3 +227,12 @@ def test_more_sequences_than_the_order_kernel_ranks():
     dsT = case[7].numpy()
     empty = np.flatnonzero(np.asarray(lens) == 0)
     assert len(empty) > 1000 and all(np.array_equal(got[5][s], dsT[s]) for s in empty[:50])
+
+
+@pytest.mark.parametrize("c2", [False, True])
+def test_split_sequences_with_fast_decays(c2):
+    """The split with chunks that take the token-by-token path inside the segments (the adjoint's summaries never do:
+    their operand cannot overflow)."""
+    case = make((2048, 300), 2, 7900, x_range=(-2.0, 1.5))
+    got, ref = run_gpu(case, c2), run_oracle(case, c2)
+    check(got, ref, case[-1].numpy(), c2, tol=4e-2, tol_dx=4e-2, what="split, fast decays")
