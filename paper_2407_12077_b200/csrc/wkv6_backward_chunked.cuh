@@ -933,6 +933,9 @@ wkv6_backward_chunked_kernel(const __grid_constant__ CUtensorMap tm_x, const __g
                 lds_v4(t_sb + tile * TILE + swz(t, blk << 4), w);
                 *reinterpret_cast<uint4*>(outs[tile] + (size_t)(row0 + (long long)c * L + t) * C + col0 + 8 * blk) = make_uint4(w[0], w[1], w[2], w[3]);
             }
+            // every thread has read the staging tiles: the first of them takes the next chunk's start state by TMA at
+            // the top of the group's next iteration, issued by one thread that would otherwise not wait for the others
+            gbar(grp);
         }
         if (gt == 0) {
             if (valid == L) {

@@ -224,3 +224,28 @@ def test_repeatable_and_argument_checks():
     dsT = torch.randn((2, 2, 64, 64), device=DEV)
     o = gf.backward(e, e, e, e, d.u, e, None, dsT)
     assert torch.equal(o[5], dsT) and (o[4] == 0).all()
+
+
+def test_ragged_last_chunk_repeats_bit_for_bit():
+    """The ragged last chunk leaves its staging tiles by plain stores of every thread; the first of those tiles then
+    takes the next chunk's start state from one thread's copy.  Run to run, and against the call that makes its own
+    checkpoints, every bit must agree (a missing rendezvous between the two showed up as a wrong dr row now and then)."""
+    B, T, H = 1, 583, 7
+    inp, dy, dsT = _inputs(B, T, H, 4242, 0.2, True, x_lo=-2.0, x_hi=1.5)
+    d = inp.to(DEV)
+    dyd, dsd = dy.to(DEV), dsT.to(DEV)
+    ws = torch.empty(gf.backward_workspace_bytes(B, T, H, 64), dtype=torch.uint8, device=DEV)
+    ref = None
+    for i in range(40):
+        if i % 2:
+            gf.prefill_train(d.r, d.k, d.v, d.x, d.u, ws, d.state_in)
+            out = gf.backward(d.r, d.k, d.v, d.x, d.u, dyd, d.state_in, dsd, workspace=ws, saved=True)
+        else:
+            out = gf.backward(d.r, d.k, d.v, d.x, d.u, dyd, d.state_in, dsd, workspace=ws)
+        gf.last_device_status()
+        out = [t.clone() for t in out]
+        if ref is None:
+            ref = out
+        else:
+            for name, a, b in zip(NAMES, ref, out):
+                assert torch.equal(a, b), (i, name)
