@@ -91,3 +91,38 @@ def test_argument_checks_before_any_launch():
     assert lib.gf_c2_decay_logit(*base, 0, 64, 64, 32, 64, None) == 0          # empty: no-op
     assert gf.launch_count() == before + 1
     gf.last_device_status()
+
+
+def test_benchmark_size_on_sampled_windows():
+    """The launch the benchmark's decay-logit row times (4 x 16384 tokens x 2048 channels: 512 tiles, three or four per
+    persistent CTA), checked against the oracle on windows of 256 rows spread over the tensor (first and last tiles,
+    sequence starts, tile edges): a window is a sequence of its own whose row above is the tensor's."""
+    B, T, D = 4, 16384, 2048
+    x, xp = synth.make_block_input(B, T, D, seed=77)
+    w = synth.make_decay_lora(D, 32, 64, seed=78)
+    dev = lambda t: t.to(DEV)
+    d = gf.decay_logit(dev(x), dev(w["mu_x"]), dev(w["A_d"]), dev(w["B_d"]), dev(w["lambda_d"]), dev(w["A_w"]),
+                       dev(w["B_w"]), dev(w["lambda_w"]), x_prev=dev(xp))
+    gf.last_device_status()
+    got = d.float().cpu().numpy().reshape(B * T, D)
+    assert np.isfinite(got).all()
+    flat = x.reshape(B * T, D)
+    rng = np.random.default_rng(79)
+    starts = [0, T - 256, T, 2 * T - 100, B * T - 256, 128 * 147, 128 * 148 - 64, 128 * 296 + 5]
+    starts += [int(s) for s in rng.integers(0, B * T - 256, size=8)]
+    worst = 0.0
+    for s0 in starts:
+        rows = flat[s0:s0 + 256]
+        # the row above the window: the tensor's previous row, or x_prev where a sequence starts there; a sequence
+        # start inside the window splits it
+        cuts = [s0] + [t for t in range(s0 + 1, s0 + 256) if t % T == 0] + [s0 + 256]
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            above = xp[a // T] if a % T == 0 else flat[a - 1]
+            ref = orc.decay_logit(flat[a:b][None], w["mu_x"], w["A_d"], w["B_d"], w["lambda_d"], w["A_w"], w["B_w"],
+                                  w["lambda_w"], above[None])[0]
+            err = np.abs(got[a:b] - ref)
+            bound = 2.0 ** -8 * np.abs(ref) + 0.02
+            worst = max(worst, float((err / bound).max()))
+            assert (err <= bound).all(), (s0, a, float((err / bound).max()))
+            assert orc.rel_l2(got[a:b], ref) <= 5e-3, (s0, a)
+    print("worst element / bound", worst)
