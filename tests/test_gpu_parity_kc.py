@@ -66,3 +66,21 @@ def test_more_row_tiles_than_sms_and_leading_dimensions(D, Dc):
     idx = torch.cat([idx, torch.tensor([0, 255, 256, B * T - 1])])
     ref = orc.key_compress(x.reshape(B * T, D)[idx], w)
     compare(c.reshape(B * T, Dc)[idx.to(DEV)], ref, "40000 rows, sampled")
+
+
+def test_benchmark_size_on_sampled_rows():
+    """The launch the benchmark's key-compression row times (65536 tokens x 2048 -> 128: 256 row tiles over the persistent
+    CTAs), rows sampled over the whole tensor plus the tile edges, every element of a row within one bf16 rounding."""
+    rows, D, Dc = 65536, 2048, 128
+    g = torch.Generator().manual_seed(19)
+    x = torch.randn(rows, D, generator=g).bfloat16()
+    w = (torch.randn(D, Dc, generator=g) / D ** 0.5).bfloat16()
+    c = gf.key_compress(x.to(DEV), w.to(DEV))
+    gf.last_device_status()
+    idx = torch.randint(0, rows, (1500,), generator=g)
+    idx = torch.cat([idx, torch.tensor([0, 255, 256, 257, 256 * 147, 256 * 148 - 1, 256 * 148, 256 * 255, rows - 1])])
+    ref = orc.key_compress(x[idx], w)
+    got = c[idx.to(DEV)].float().cpu().numpy()
+    assert np.isfinite(c.float().cpu().numpy()).all()
+    compare(c[idx.to(DEV)], ref, "65536 rows, sampled")
+    assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-3).all()
