@@ -249,3 +249,37 @@ def test_ragged_last_chunk_repeats_bit_for_bit():
         else:
             for name, a, b in zip(NAMES, ref, out):
                 assert torch.equal(a, b), (i, name)
+
+
+def test_long_context_shape_at_the_benchmarked_size_two_heads_in_full():
+    """The launch the benchmark's long-context gradient row times (B=1, T=131072, H=32: 32 units, sequences split
+    4-way), two of the heads against the oracle over all their tokens (the oracle keeps every state of a unit: 4 GB
+    per head), the rest finite and repeatable."""
+    c = synth.CONFIGS["cfg3"]
+    B, T, H = c["B"], c["T"], c["H"]
+    inp, dy, dsT = _inputs(B, T, H, 3100, c["state_std"], True)
+    d = inp.to(DEV)
+    out = gf.backward(d.r, d.k, d.v, d.x, d.u, dy.to(DEV), d.state_in, dsT.to(DEV))
+    gf.last_device_status()
+    out2 = gf.backward(d.r, d.k, d.v, d.x, d.u, dy.to(DEV), d.state_in, dsT.to(DEV))
+    gf.last_device_status()
+    for name, a, b in zip(NAMES, out, out2):
+        assert torch.equal(a, b), name
+        assert torch.isfinite(a.float()).all(), name
+    out = [t.cpu() for t in out]
+    del out2
+    for h in (5, 31):
+        hs = slice(h, h + 1)
+        sin = None if inp.state_in is None else inp.state_in[:, hs]
+        ref = orc.backward(inp.r[:, :, hs], inp.k[:, :, hs], inp.v[:, :, hs], inp.x[:, :, hs], inp.u[hs],
+                           dy[:, :, hs].double().numpy(), sin, dsT[:, hs].double().numpy())
+        part = [out[0][:, :, hs], out[1][:, :, hs], out[2][:, :, hs], out[3][:, :, hs], out[4][hs], out[5][:, hs]]
+        for name, a, r in zip(NAMES, part, ref):
+            a = a.float().numpy().astype(np.float64)
+            lim = TOL_DX if name == "dx" else TOL
+            assert orc.rel_l2(a, r) <= lim, (h, name, orc.rel_l2(a, r))
+            if name in ("dr", "dk", "dv", "dx"):
+                row = ((a - r) ** 2).sum(axis=3)
+                den = (r * r).sum(axis=(1, 3))
+                tok = np.sqrt(row.max(axis=1) / (den / T))
+                assert tok.max() <= TOK_TOL, (h, name, float(tok.max()))

@@ -119,3 +119,29 @@ def test_packed_pair_is_bit_identical_to_the_separate_packed_calls(lens, c2):
         got = list(ga)
     for i, (p, q) in enumerate(zip(got, ref)):
         assert orc.rel_l2(p.float().cpu().numpy(), q) <= (8e-3 if i == 3 else 5e-3), i
+
+
+@pytest.mark.parametrize("c2", [False, True])
+def test_pair_at_the_benchmarked_size(c2):
+    """The two launches the benchmark's training rows time (B=4, T=16384, H=32): the forward pass equals the plain
+    prefill and the gradient from its saved states equals the gradient call that makes its own, bit for bit."""
+    c = synth.CONFIGS["cfg2"]
+    B, T, H = c["B"], c["T"], c["H"]
+    inp = synth.make_dense(B, T, H, 64, "bf16", seed=2200, state_std=0.1).to(DEV)
+    g = torch.Generator(device=DEV).manual_seed(2201)
+    dy = torch.randn(inp.r.shape, generator=g, device=DEV).bfloat16()
+    u2 = torch.randn(inp.r.shape, generator=g, device=DEV).bfloat16() if c2 else None
+    dsT = torch.randn((B, H, 64, 64), generator=g, device=DEV) * 0.1
+    ws = torch.empty(gf.backward_workspace_bytes(B, T, H, 64), dtype=torch.uint8, device=DEV)
+    y, s = gf.prefill_train(inp.r, inp.k, inp.v, inp.x, inp.u, ws, inp.state_in, c2=c2, u2=u2)
+    if c2:
+        y0, s0 = gf.prefill_c2(inp.r, inp.k, inp.v, inp.x, u2, inp.state_in)
+        ga = gf.backward_c2(inp.r, inp.k, inp.v, inp.x, dy, inp.state_in, dsT, workspace=ws, saved=True)
+        gb = gf.backward_c2(inp.r, inp.k, inp.v, inp.x, dy, inp.state_in, dsT)
+    else:
+        y0, s0 = gf.prefill(inp.r, inp.k, inp.v, inp.x, inp.u, inp.state_in)
+        ga = gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT, workspace=ws, saved=True)
+        gb = gf.backward(inp.r, inp.k, inp.v, inp.x, inp.u, dy, inp.state_in, dsT)
+    gf.last_device_status()
+    assert torch.equal(y, y0) and torch.equal(s, s0)
+    assert all(torch.equal(p, q) for p, q in zip(ga, gb))
